@@ -1,0 +1,375 @@
+"""Elementary operations of the paper's models (test infrastructure, CPU oracle).
+
+Each function takes raw words and returns a raw word, following the paper's
+algorithm of the same name step by step with unbounded integers:
+
+    ftz_add / ftz_mul   Algorithm 1        fma        Algorithm 3
+    e_fdpa              Algorithm 6        t_fdpa     Algorithm 7 (+ Table 2)
+    st_fdpa             Algorithm 8        gst_fdpa   Algorithm 9
+    tr_fdpa             Algorithm 10       gtr_fdpa   Algorithm 11
+    special values      Section 4.2
+
+Notation: a product term is kept as an integer ``s`` with ``frac`` fractional
+bits and an exponent ``e`` (value ``s * 2**(e - frac)``), mirroring the paper's
+``s_k`` (product of signed significands) and ``e_k`` (sum of exponents).
+
+Readings chosen where the paper is silent (all "parity unpinned" against real
+hardware; the values the paper prints do not discriminate them):
+ R1  SignedSig/Exp: see oracle/formats.py (subnormals keep Exp = emin, no hidden bit).
+ R2  A zero operand, a zero product and c = 0 take part in the exponent maximum
+     with their minimum exponents.
+ R3  RZ_F truncates the magnitude and keeps the sign; RD_F is floor.
+ R4  Overflow of rho: RZ saturates to the largest finite value, RNE gives inf.
+ R5  Exactly-zero fixed-point sums give +0.0 in every FDPA family; a nonzero
+     sum that rounds to zero keeps its sign.  FMA / FTZ-Add follow IEEE-754
+     signed-zero rules.
+ R6  NaN words: 0x7FFFFFFF / 0x7FFF for T-, ST- and GST-FDPA (Section 4.2);
+     0x7FC00000 / 0x7FF8000000000000 for every other operation (a convention).
+ R7  TR-/GTR-FDPA: a product with magnitude >= 2**128 becomes +-inf before the
+     fused sum (Section 4.2) and then follows the special-value algebra.
+ R8  GTR-FDPA "special truncation": s_c' is replaced by 0 when Exp(c) < E-F-1,
+     tested on the raw exponent of c.
+ R9  A NaN scale factor makes the block result NaN.
+ R10 GST-FDPA: p_g is the dot product of the FP4 *values*; the scale index of
+     group g is floor(g*G / K_block); L/K_block scale factors per operand.
+"""
+from __future__ import annotations
+
+from .formats import Format, FORMATS, decode, decoder, Dec, FINITE, INF, NAN
+from .rounding import round_dyadic, rho, RHO
+
+FP32 = FORMATS["fp32"]
+FP64 = FORMATS["fp64"]
+
+NAN_NV = {"fp32": 0x7FFFFFFF, "fp16": 0x7FFF}
+NAN_IEEE = {"fp32": 0x7FC00000, "fp16": 0x7E00, "fp64": 0x7FF8000000000000}
+
+
+def _inf_word(fmt: Format, sign: int) -> int:
+    top = (1 << fmt.ebits) - 1
+    return (sign << (fmt.ebits + fmt.mbits)) | (top << fmt.mbits)
+
+
+# ----------------------------------------------------------------------------
+# small fixed-point helpers
+# ----------------------------------------------------------------------------
+def _floor_scale(n: int, sh: int) -> int:
+    """floor(n * 2**sh) for any integer n (Python's >> floors)."""
+    return n << sh if sh >= 0 else n >> -sh
+
+
+def rz_scale(n: int, sh: int) -> int:
+    """n * 2**sh truncated toward zero (sign-magnitude truncation, reading R3)."""
+    return _floor_scale(n, sh) if n >= 0 else -_floor_scale(-n, sh)
+
+
+def rd_scale(n: int, sh: int) -> int:
+    """n * 2**sh rounded down (toward minus infinity)."""
+    return _floor_scale(n, sh)
+
+
+def _signed_sig(d: Dec) -> int:
+    return -d.sig if d.sign else d.sig
+
+
+# ----------------------------------------------------------------------------
+# Section 4.2: special values of a dot-product-accumulate block
+# ----------------------------------------------------------------------------
+def _special(da, db, dc, extra_nan=False, extra_inf_signs=()):
+    """None if every term is finite, else 'nan', '+inf' or '-inf'.
+
+    NaN + x = NaN, NaN * x = NaN, inf * 0 = NaN, (+inf) + (-inf) = NaN,
+    inf * z = inf * sign(z), inf + finite = inf.
+    """
+    nan = extra_nan or (dc is not None and dc.cls == NAN)
+    seen = [False, False]                      # [+inf seen, -inf seen]
+    if dc is not None and dc.cls == INF:
+        seen[dc.sign] = True
+    for s in extra_inf_signs:
+        seen[s] = True
+    for x, y in zip(da, db):
+        if x.cls == NAN or y.cls == NAN:
+            nan = True
+        elif x.cls == INF or y.cls == INF:
+            other = y if x.cls == INF else x
+            if other.cls == FINITE and other.sig == 0:
+                nan = True                     # inf * 0
+            else:
+                seen[x.sign ^ y.sign] = True
+    if nan or (seen[0] and seen[1]):
+        return "nan"
+    if seen[0]:
+        return "+inf"
+    if seen[1]:
+        return "-inf"
+    return None
+
+
+def _special_word(kind: str, out_name: str, nan_table) -> int:
+    fmt = FORMATS[out_name]
+    if kind == "nan":
+        return nan_table[out_name]
+    return _inf_word(fmt, 1 if kind == "-inf" else 0)
+
+
+_RHO_OUT = {"RZ-FP32": "fp32", "RZ-E8M13": "fp32", "RNE-FP32": "fp32", "RNE-FP16": "fp16"}
+
+
+# ----------------------------------------------------------------------------
+# Algorithm 7 (T-FDPA), Algorithm 8 (ST-FDPA)
+# ----------------------------------------------------------------------------
+def t_fdpa(a, b, c, fmt_a: Format, fmt_b: Format, fmt_c: Format, F, rho_name: str,
+           scale_exp: int = 0, scale_nan: bool = False) -> int:
+    """One T-FDPA block: words a[0..L), b[0..L), accumulator word c -> output word.
+
+    ``F`` is the number of fractional bits of the fused sum; ``F=None`` means
+    unlimited precision (no truncation), used only by tests.  ``scale_exp`` is
+    the ST-FDPA addend Exp(alpha)+Exp(beta) (0 for plain T-FDPA).
+    """
+    da = list(map(decoder(fmt_a), a))
+    db = list(map(decoder(fmt_b), b))
+    dc = decode(fmt_c, c)
+    sp = _special(da, db, dc, extra_nan=scale_nan)
+    if sp is not None:
+        return _special_word(sp, _RHO_OUT[rho_name], NAN_NV)
+    # Step 1: exact products of signed significands, sums of exponents
+    frac = fmt_a.mbits + fmt_b.mbits
+    s = [_signed_sig(x) * _signed_sig(y) for x, y in zip(da, db)]
+    e = [x.exp + y.exp + scale_exp for x, y in zip(da, db)]
+    # Step 2: truncated fused sum of L+1 terms
+    s_c, e_c = _signed_sig(dc), dc.exp
+    e_max = max(e + [e_c])
+    if F is None:                               # exact sum (test switch)
+        lo = min(min(ek - frac for ek in e), e_c - fmt_c.mbits)
+        S = sum(sk << (ek - frac - lo) for sk, ek in zip(s, e)) + (s_c << (e_c - fmt_c.mbits - lo))
+        return rho(rho_name, S, lo)
+    S = 0
+    for sk, ek in zip(s, e):
+        S += rz_scale(sk, (ek - e_max) + F - frac)          # RZ_F(s_k * 2**(e_k - e_max))
+    S += rz_scale(s_c, (e_c - e_max) + F - fmt_c.mbits)
+    # Step 3: convert
+    return rho(rho_name, S, e_max - F)
+
+
+def st_fdpa(a, b, c, alpha: int, beta: int, fmt_a: Format, fmt_b: Format, F: int,
+            rho_name: str) -> int:
+    """One ST-FDPA block: T-FDPA with Exp(alpha)+Exp(beta) added to every e_k (E8M0 scales)."""
+    e8 = FORMATS["e8m0"]
+    dal, dbe = decode(e8, alpha), decode(e8, beta)
+    nan = dal.cls == NAN or dbe.cls == NAN
+    return t_fdpa(a, b, c, fmt_a, fmt_b, FP32, F, rho_name,
+                  scale_exp=dal.exp + dbe.exp, scale_nan=nan)
+
+
+# ----------------------------------------------------------------------------
+# Algorithm 9 (GST-FDPA)
+# ----------------------------------------------------------------------------
+def gst_fdpa(a, b, c, alphas, betas, scale_fmt: Format, k_block: int, G: int, F: int,
+             rho_name: str) -> int:
+    """One GST-FDPA block over L = len(a) FP4 (E2M1) elements.
+
+    ``alphas`` / ``betas`` hold L/k_block scale words each (reading R10).
+    """
+    f4 = FORMATS["e2m1"]
+    L = len(a)
+    da = list(map(decoder(f4), a))
+    db = list(map(decoder(f4), b))
+    dc = decode(FP32, c)
+    dal = [decode(scale_fmt, w) for w in alphas]
+    dbe = [decode(scale_fmt, w) for w in betas]
+    nan = any(d.cls == NAN for d in dal + dbe)
+    sp = _special([], [], dc, extra_nan=nan)     # FP4 has no inf/NaN
+    if sp is not None:
+        return _special_word(sp, "fp32", NAN_NV)
+    # Step 1: exact dot product per group, times the scale significands
+    vfrac = 2 * f4.mbits                        # fractional bits of sig_a*sig_b
+    sfrac = 2 * scale_fmt.mbits
+    s, e = [], []
+    for g in range(L // G):
+        # p_g as an integer multiple of 2**(2*emin4 - vfrac): align every product at the smallest exponent
+        base = 2 * f4.emin
+        p = 0
+        for k in range(g * G, (g + 1) * G):
+            p += (_signed_sig(da[k]) * _signed_sig(db[k])) << (da[k].exp + db[k].exp - base)
+        j = (g * G) // k_block
+        s.append(p * dal[j].sig * dbe[j].sig)    # frac bits: vfrac + sfrac, plus factor 2**base
+        e.append(dal[j].exp + dbe[j].exp)
+    frac = vfrac + sfrac - 2 * f4.emin           # value of term g = s_g * 2**(e_g - frac)
+    # Step 2: truncated fused sum of L/G + 1 terms
+    s_c, e_c = _signed_sig(dc), dc.exp
+    e_max = max(e + [e_c])
+    S = 0
+    for sg, eg in zip(s, e):
+        S += rz_scale(sg, (eg - e_max) + F - frac)
+    S += rz_scale(s_c, (e_c - e_max) + F - FP32.mbits)
+    return rho(rho_name, S, e_max - F)
+
+
+# ----------------------------------------------------------------------------
+# Algorithm 10 (TR-FDPA), Algorithm 11 (GTR-FDPA)
+# ----------------------------------------------------------------------------
+def _products_with_overflow(da, db, frac):
+    """Exact products; a product with |value| >= 2**128 is reported as an infinity sign (R7)."""
+    s, e, inf_signs = [], [], []
+    for x, y in zip(da, db):
+        if x.cls != FINITE or y.cls != FINITE:
+            s.append(0)
+            e.append(0)
+            continue
+        sk = _signed_sig(x) * _signed_sig(y)
+        ek = x.exp + y.exp
+        # |sk| * 2**(ek - frac) >= 2**128  <=>  |sk| >= 2**(128 - ek + frac)
+        lim = 128 - ek + frac
+        if sk != 0 and (lim <= 0 or abs(sk) >= (1 << lim)):
+            inf_signs.append(1 if sk < 0 else 0)
+        s.append(sk)
+        e.append(ek)
+    return s, e, inf_signs
+
+
+def tr_fdpa(a, b, c, fmt_a: Format, fmt_b: Format, F: int, F2: int, rho_name: str = "RNE-FP32",
+            inner_round: str = "RD") -> int:
+    """One TR-FDPA block.  ``inner_round='RZ'`` gives the paper's hypothetical symmetric variant."""
+    da = list(map(decoder(fmt_a), a))
+    db = list(map(decoder(fmt_b), b))
+    dc = decode(FP32, c)
+    frac = fmt_a.mbits + fmt_b.mbits
+    s, e, inf_signs = _products_with_overflow(da, db, frac)
+    sp = _special(da, db, dc, extra_inf_signs=inf_signs)
+    if sp is not None:
+        return _special_word(sp, "fp32", NAN_IEEE)
+    rnd = rd_scale if inner_round == "RD" else rz_scale
+    # Step 2: truncated fused sum of the L products (c excluded)
+    e_max = max(e)
+    T = sum(rz_scale(sk, (ek - e_max) + F - frac) for sk, ek in zip(s, e))     # units 2**(e_max - F)
+    # Step 3: rounded sum of T and c at E = max(e_max, e_c)
+    s_c, e_c = _signed_sig(dc), dc.exp
+    E = max(e_max, e_c)
+    T2 = rnd(T, (e_max - E) + F2 - F)                      # RD_F2(T * 2**(e_max - E)), units 2**(E - F2)
+    sc2 = rnd(s_c, (e_c - E) + F - FP32.mbits)             # RD_F(s_c * 2**(e_c - E)), units 2**(E - F)
+    S = T2 + (sc2 << (F2 - F))                             # units 2**(E - F2)
+    return rho(rho_name, S, E - F2)
+
+
+def gtr_fdpa(a, b, c, fmt_a: Format, fmt_b: Format, F: int, F2: int,
+             rho_name: str = "RNE-FP32") -> int:
+    """One GTR-FDPA block (even / odd index groups, rounded-down merges, special truncation of c)."""
+    da = list(map(decoder(fmt_a), a))
+    db = list(map(decoder(fmt_b), b))
+    dc = decode(FP32, c)
+    frac = fmt_a.mbits + fmt_b.mbits
+    s, e, inf_signs = _products_with_overflow(da, db, frac)
+    sp = _special(da, db, dc, extra_inf_signs=inf_signs)
+    if sp is not None:
+        return _special_word(sp, "fp32", NAN_IEEE)
+    # Step 2: truncated fused sums of the even- and odd-index products
+    e_even, e_odd = max(e[0::2]), max(e[1::2])
+    T_even = sum(rz_scale(sk, (ek - e_even) + F - frac) for sk, ek in zip(s[0::2], e[0::2]))
+    T_odd = sum(rz_scale(sk, (ek - e_odd) + F - frac) for sk, ek in zip(s[1::2], e[1::2]))
+    # Step 3: rounded sum of the two group sums
+    e_max = max(e_even, e_odd)
+    T = rd_scale(T_even, e_even - e_max) + rd_scale(T_odd, e_odd - e_max)     # units 2**(e_max - F)
+    # Step 4: final rounded sum with c
+    s_c, e_c = _signed_sig(dc), dc.exp
+    E = max(e_max, e_c)
+    T2 = rd_scale(T, (e_max - E) + F2 - F)
+    sc2 = rd_scale(s_c, (e_c - E) + F - FP32.mbits)
+    if e_c < E - F - 1:
+        sc2 = 0                                             # special truncation (R8)
+    S = T2 + (sc2 << (F2 - F))
+    return rho(rho_name, S, E - F2)
+
+
+# ----------------------------------------------------------------------------
+# Algorithm 6 (E-FDPA)
+# ----------------------------------------------------------------------------
+def e_fdpa(a, b, c, fmt_a: Format, fmt_b: Format) -> int:
+    """RNE-FP32(c + sum a_k*b_k) computed exactly."""
+    da = list(map(decoder(fmt_a), a))
+    db = list(map(decoder(fmt_b), b))
+    dc = decode(FP32, c)
+    sp = _special(da, db, dc)
+    if sp is not None:
+        return _special_word(sp, "fp32", NAN_IEEE)
+    frac = fmt_a.mbits + fmt_b.mbits
+    terms = [(_signed_sig(x) * _signed_sig(y), x.exp + y.exp - frac) for x, y in zip(da, db)]
+    terms.append((_signed_sig(dc), dc.exp - FP32.mbits))
+    lo = min(t[1] for t in terms)
+    S = sum(m << (ex - lo) for m, ex in terms)
+    return rho("RNE-FP32", S, lo)
+
+
+# ----------------------------------------------------------------------------
+# Algorithm 3 (FMA), IEEE-754 add / mul, Algorithm 1 (FTZ-Add / FTZ-Mul)
+# ----------------------------------------------------------------------------
+def _ieee_round(fmt: Format, m: int, e: int, zero_sign: int) -> int:
+    return round_dyadic(m, e, fmt.ebits, fmt.mbits, fmt.bias, "RNE", zero_sign)
+
+
+def fma(a: int, b: int, c: int, fmt: Format) -> int:
+    """IEEE-754 fusedMultiplyAdd in round-to-nearest-even; NaN result is the quiet NaN of R6."""
+    x, y, z = decode(fmt, a), decode(fmt, b), decode(fmt, c)
+    sp = _special([x], [y], z)
+    if sp is not None:
+        return _special_word(sp, fmt.name, NAN_IEEE)
+    p = _signed_sig(x) * _signed_sig(y)
+    pe = x.exp + y.exp - 2 * fmt.mbits
+    ce = z.exp - fmt.mbits
+    lo = min(pe, ce)
+    S = (p << (pe - lo)) + (_signed_sig(z) << (ce - lo))
+    psign = x.sign ^ y.sign
+    zero_sign = psign if psign == z.sign else 0     # exact zero: like signs keep it, else +0 (RNE)
+    return _ieee_round(fmt, S, lo, zero_sign)
+
+
+def _ieee_add(x: Dec, y: Dec, fmt_x: Format, fmt_y: Format, out: Format) -> int:
+    if x.cls == NAN or y.cls == NAN or (x.cls == INF and y.cls == INF and x.sign != y.sign):
+        return NAN_IEEE[out.name]
+    if x.cls == INF or y.cls == INF:
+        return _inf_word(out, x.sign if x.cls == INF else y.sign)
+    xe, ye = x.exp - fmt_x.mbits, y.exp - fmt_y.mbits
+    lo = min(xe, ye)
+    S = (_signed_sig(x) << (xe - lo)) + (_signed_sig(y) << (ye - lo))
+    zero_sign = x.sign if x.sign == y.sign else 0   # exact zero: like signs keep it, else +0 (RNE)
+    return _ieee_round(out, S, lo, zero_sign)
+
+
+def ieee_add_f32(x: int, y: int) -> int:
+    """IEEE-754 binary32 addition, RNE, quiet NaN 0x7FC00000."""
+    return _ieee_add(decode(FP32, x), decode(FP32, y), FP32, FP32, FP32)
+
+
+def ieee_mul_f32(x: int, y: int, fmt_x: Format = FP32, fmt_y: Format = FP32) -> int:
+    """RNE-FP32(x*y) for x, y in the given formats; IEEE special values."""
+    dx, dy = decode(fmt_x, x), decode(fmt_y, y)
+    sp = _special([dx], [dy], None)
+    if sp is not None:
+        return _special_word(sp, "fp32", NAN_IEEE)
+    p = _signed_sig(dx) * _signed_sig(dy)
+    return _ieee_round(FP32, p, dx.exp + dy.exp - fmt_x.mbits - fmt_y.mbits, dx.sign ^ dy.sign)
+
+
+def _ftz(z: int) -> int:
+    """z * 0.0 if |z| < 2**-126: sign-preserving flush of an FP32 word (Algorithm 1, last line)."""
+    d = decode(FP32, z)
+    if d.cls == FINITE and d.sig < (1 << FP32.mbits):
+        return d.sign << 31
+    return z
+
+
+def ftz_add(x: int, y: int) -> int:
+    """FTZ-Add on FP32 words: RNE-FP32(x+y), then flush a subnormal result keeping its sign."""
+    return _ftz(ieee_add_f32(x, y))
+
+
+def ftz_mul(x: int, y: int, fmt: Format) -> int:
+    """FTZ-Mul on words of ``fmt`` (BF16 or FP16): RNE-FP32(x*y), then flush."""
+    return _ftz(ieee_mul_f32(x, y, fmt, fmt))
+
+
+def flush_subnormal(w: int, fmt: Format) -> int:
+    """FlushSubnormal of Algorithm 2: a subnormal input becomes +0.0; everything else is kept."""
+    d = decode(fmt, w)
+    if d.cls == FINITE and d.sig != 0 and d.sig < (1 << fmt.mbits):
+        return 0
+    return w
