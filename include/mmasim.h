@@ -1,0 +1,157 @@
+/*
+ * mmasim -- bit-accurate evaluation of GPU matrix-multiply-accumulate arithmetic models on a B200.
+ *
+ * The library evaluates D = Phi(A, B, C) (the paper's Equation 2) where Phi is one of the arithmetic
+ * behaviour models of Section 4 (Table 1: Phi_FTZ-AddMul, Phi_FMA, Phi_E/T/ST/GST/TR/GTR-FDPA), chosen by
+ * (architecture, input type, accumulator type) exactly as Tables 3-7 map instructions to models.
+ * Every output word is a pure function of the input words; there is exactly one correct answer.
+ *
+ * Conventions for every entry point
+ *   - Data pointers are DEVICE pointers owned by the caller unless the name ends in _host.
+ *   - The library never synchronises and enqueues work only on the given stream
+ *     (a cudaStream_t passed as void*; NULL is the default stream).  _host calls are synchronous.
+ *   - No CPU fallback exists: without a CUDA device the compute entry points return MMASIM_ERR_CUDA.
+ *   - Return value: an mmasim_status; mmasim_last_error() gives a thread-local message for the last failure.
+ *   - A is M x K row-major; B is N x K row-major, i.e. the paper's K x N matrix stored column-major
+ *     (both operands are contiguous along K); C and D are M x N row-major in the accumulator type.
+ *   - Element storage: FP64 8 bytes; FP32 and TF32 4 bytes (TF32: the low 13 bits are ignored);
+ *     BF16/FP16 2 bytes; FP8, FP6 and FP4 of the T-/ST-FDPA models one element per byte in the low bits;
+ *     FP4 of the GST-FDPA models (MXF4_GST, NVF4_GST) two per byte, element 2i in the low nibble.
+ *   - K must be a multiple of min(K, L_max) (Algorithm 5 would silently drop a remainder; zero padding of A
+ *     and B is exactly neutral for every FDPA model), of P for Phi_FTZ-AddMul, and of 32 for GST models.
+ */
+#ifndef MMASIM_H
+#define MMASIM_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mmasim_model mmasim_model; /* opaque, host side, immutable, may be shared between threads */
+
+typedef enum {
+    MMASIM_OK = 0,
+    MMASIM_ERR_INVALID_ARG = 1, /* null pointer, bad enum, host pointer where a device pointer is needed */
+    MMASIM_ERR_UNSUPPORTED = 2, /* the (arch, input, accumulator) triple is not in Tables 3-7 */
+    MMASIM_ERR_SHAPE = 3,       /* M, N, K < 1, K not a multiple of the model's block, bad k_chunk or ld */
+    MMASIM_ERR_ALIGN = 4,       /* pointer or leading dimension not aligned as documented */
+    MMASIM_ERR_CUDA = 5,        /* a CUDA runtime call failed (message holds the CUDA error string) */
+    MMASIM_ERR_TIMEOUT = 6      /* reserved: a bounded device-side wait gave up */
+} mmasim_status;
+
+/* The ten architectures of Section 3.2. */
+typedef enum {
+    MMASIM_VOLTA = 0, MMASIM_TURING, MMASIM_AMPERE, MMASIM_ADA, MMASIM_HOPPER, MMASIM_BLACKWELL,
+    MMASIM_RTX_BLACKWELL, MMASIM_CDNA1, MMASIM_CDNA2, MMASIM_CDNA3, MMASIM_ARCH_COUNT
+} mmasim_arch;
+
+/* Input types (first column of Tables 3-7).  MX* are the block-scaled variants of Algorithm 8 (one E8M0
+ * scale per 32 elements); MXF4_GST / NVF4_GST are the group-scaled FP4 variants of Algorithm 9 (E8M0 per 32
+ * elements / UE4M3 per 16 elements).  BF16_1K is the CDNA2 "_1k" BF16 instruction class (P = 4). */
+typedef enum {
+    MMASIM_F64 = 0, MMASIM_F32, MMASIM_TF32, MMASIM_BF16, MMASIM_BF16_1K, MMASIM_F16,
+    MMASIM_E4M3, MMASIM_E5M2, MMASIM_E3M2, MMASIM_E2M3, MMASIM_E2M1,
+    MMASIM_MXE4M3, MMASIM_MXE5M2, MMASIM_MXE3M2, MMASIM_MXE2M3, MMASIM_MXE2M1,
+    MMASIM_MXF4_GST, MMASIM_NVF4_GST, MMASIM_FMT_COUNT
+} mmasim_fmt;
+
+typedef enum { MMASIM_ACC_F32 = 0, MMASIM_ACC_F16, MMASIM_ACC_F64, MMASIM_ACC_COUNT } mmasim_acc;
+
+/* Model families (Table 1) and conversion functions (Table 2). */
+typedef enum {
+    MMASIM_FAM_FMA = 0, MMASIM_FAM_FTZ_ADDMUL, MMASIM_FAM_E_FDPA, MMASIM_FAM_T_FDPA, MMASIM_FAM_ST_FDPA,
+    MMASIM_FAM_GST_FDPA, MMASIM_FAM_TR_FDPA, MMASIM_FAM_GTR_FDPA
+} mmasim_family;
+typedef enum { MMASIM_RHO_NONE = 0, MMASIM_RZ_FP32, MMASIM_RZ_E8M13, MMASIM_RNE_FP32, MMASIM_RNE_FP16 } mmasim_rho;
+
+/* Parameters of a model as the paper's tables give them (0 where a parameter does not apply). */
+typedef struct {
+    int32_t family;       /* mmasim_family */
+    int32_t l_max;        /* L_max of Algorithm 5 (Tables 4, 5, 6, 7) */
+    int32_t F;            /* fractional bits of the fused sum */
+    int32_t F2;           /* TR-/GTR-FDPA second-stage precision (Table 7) */
+    int32_t rho;          /* mmasim_rho */
+    int32_t P;            /* Phi_FTZ-AddMul group size (Table 6) */
+    int32_t G;            /* GST-FDPA group size (Table 5) */
+    int32_t k_block;      /* elements per scale factor: 32 (MX), 16 (NVFP4), 0 = unscaled */
+    int32_t a_bits;       /* storage bits per A element: 64, 32, 16, 8 or 4 */
+    int32_t b_bits;       /* storage bits per B element */
+    int32_t acc_bytes;    /* bytes per C / D element: 8, 4 or 2 */
+    int32_t inner_round;  /* 0 = as in the paper; 1 = TR-FDPA second stage uses RZ (Section 6.2.4 experiment) */
+} mmasim_info;
+
+/* Hypothetical-model overrides for mmasim_create_model_ex (design-space exploration, Section 7).
+ * A negative field keeps the table value. */
+typedef struct {
+    int32_t l_max, F, F2, rho, inner_round;
+} mmasim_overrides;
+
+/* Optional arguments of mmasim_gemm_ex.  Zero-initialise, then set what is needed. */
+typedef struct {
+    int64_t lda, ldb, ldc, ldd; /* leading dimensions in ELEMENTS (GST FP4: in elements, even); 0 = packed */
+    const void* sfa;            /* device, M x ceil(K/k_block) bytes row-major: scale factors of A (ST/GST models) */
+    const void* sfb;            /* device, N x ceil(K/k_block) bytes row-major: scale factors of B */
+    int64_t k_chunk;            /* 0, or a multiple of the model's block: every k_chunk elements of K the model is
+                                   run from a +0 accumulator and its FP32 result is added to an FP32 running sum
+                                   with an IEEE-754 RNE addition (the FP32-promotion workaround the paper motivates
+                                   in Sections 2.2 and 6.3; FP32-accumulator FDPA models only) */
+    const float* row_scale;     /* device, M floats or NULL */
+    const float* col_scale;     /* device, N floats or NULL: D = fl32(fl32(row_scale[i]*col_scale[j]) * d) */
+    int32_t flags;              /* MMASIM_GEMM_FORCE_GENERIC: skip the tuned kernels (used to cross-check them) */
+} mmasim_gemm_opts;
+#define MMASIM_GEMM_FORCE_GENERIC 1
+
+/* Registry lookup (Tables 3-7).  Returns NULL and sets the error message if the triple is not in the paper. */
+mmasim_model* mmasim_create_model(int arch, int in_fmt, int acc_fmt);
+
+/* As above with different A and B element types (Algorithm 7 allows F_A != F_B; both must select the same
+ * table row class, e.g. E4M3 x E5M2) and optional overrides; ov may be NULL. */
+mmasim_model* mmasim_create_model_ex(int arch, int a_fmt, int b_fmt, int acc_fmt, const mmasim_overrides* ov);
+
+void mmasim_destroy_model(mmasim_model* model);
+
+/* Fills *out with the model's parameters. */
+int mmasim_model_info(const mmasim_model* model, mmasim_info* out);
+
+/* D = Phi(A, B, C) (Equation 2; Algorithms 2, 4, 5).  C may be NULL (= +0) and may alias D.
+ * All pointers 16-byte aligned.  Enqueues on stream and returns. */
+int mmasim_gemm(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
+                const void* A, const void* B, const void* C, void* D, void* stream);
+
+/* As mmasim_gemm with leading dimensions, scale factors (Algorithms 8, 9), FP32 promotion of partial sums
+ * and a dequantisation epilogue.  opts may be NULL. */
+int mmasim_gemm_ex(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
+                   const void* A, const void* B, const void* C, void* D,
+                   const mmasim_gemm_opts* opts, void* stream);
+
+/* n independent dot-product-accumulates d_t = Phi(a_t, b_t, c_t) (Equation 4), the shape of the paper's probe
+ * vectors (Section 3.1): A, B are n x K row-major, C (may be NULL) and D hold n accumulator words.
+ * Unscaled models only. */
+int mmasim_dot_batch(const mmasim_model* model, int64_t n, int64_t K,
+                     const void* A, const void* B, const void* C, void* D, void* stream);
+
+/* mmasim_gemm_ex on HOST buffers: allocates device memory, copies A, B, C (and scales) to the device, runs,
+ * copies D back and frees; synchronous.  Fields of opts that are pointers are host pointers here. */
+int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
+                     const void* A, const void* B, const void* C, void* D, const mmasim_gemm_opts* opts);
+
+/* Integer-issue micro-benchmark used as the roofline denominator (no counterpart in the paper): launches
+ * `blocks` CTAs of 256 threads, each thread running `iters` rounds of 8 independent dependent-chain integer
+ * operations of the given kind (0: 3-input add, 1: logic, 2: funnel shift, 3: 32-bit multiply-add, 4: the
+ * add/max/shift/add mix of one emulated MAC).  `sink` (device, >= 4 bytes) receives a value that keeps the
+ * work alive.  The caller times the launch; operations per launch = blocks * 256 * iters * 8 * ops_per_round,
+ * where ops_per_round is returned through *ops_per_round. */
+int mmasim_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t* ops_per_round, void* stream);
+
+/* Name of the kernel variant the last mmasim_gemm* call on this thread dispatched to ("generic", ...). */
+const char* mmasim_last_kernel(void);
+
+/* Thread-local message of the last failing call on this thread ("" if none). */
+const char* mmasim_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MMASIM_H */

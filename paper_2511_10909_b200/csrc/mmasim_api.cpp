@@ -1,0 +1,270 @@
+// C ABI of libmmasim: argument validation, model objects, dispatch to the kernels.
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include "mmasim_internal.h"
+
+namespace mmasim {
+
+static thread_local char g_error[512] = "";
+static thread_local char g_kernel[64] = "";
+
+void set_error(const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_error, sizeof(g_error), fmt, ap);
+    va_end(ap);
+}
+void set_kernel_name(const char* name) { snprintf(g_kernel, sizeof(g_kernel), "%s", name); }
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// MMASIM_OK if p is device-accessible memory; ERR_INVALID_ARG for plain host memory; ERR_CUDA otherwise.
+int check_device_ptr(const void* p, const char* name) {
+    cudaPointerAttributes attr;
+    const cudaError_t err = cudaPointerGetAttributes(&attr, p);
+    if (err != cudaSuccess) {
+        cudaGetLastError();
+        set_error("cudaPointerGetAttributes(%s) failed: %s", name, cudaGetErrorString(err));
+        return MMASIM_ERR_CUDA;
+    }
+    if (attr.type == cudaMemoryTypeDevice || attr.type == cudaMemoryTypeManaged) return MMASIM_OK;
+    set_error("%s is not a device pointer", name);
+    return MMASIM_ERR_INVALID_ARG;
+}
+
+// Shape rules shared by gemm and dot_batch.  Returns MMASIM_OK or an error status.
+int check_k(const DevModel& m, int64_t K) {
+    if (K < 1) { set_error("K must be >= 1"); return MMASIM_ERR_SHAPE; }
+    if (m.family == FAM_FMA) return MMASIM_OK;
+    if (m.family == FAM_FTZ) {
+        if (K % m.P) { set_error("K = %lld is not a multiple of P = %d", (long long)K, m.P); return MMASIM_ERR_SHAPE; }
+        return MMASIM_OK;
+    }
+    const int64_t L = K < m.L ? K : m.L;
+    if (K % L) {
+        set_error("K = %lld is not a multiple of L = min(K, L_max) = %lld", (long long)K, (long long)L);
+        return MMASIM_ERR_SHAPE;
+    }
+    if (m.family == FAM_GST && (L % 32)) { set_error("GST-FDPA models need K to be a multiple of 32"); return MMASIM_ERR_SHAPE; }
+    if (m.family == FAM_GTR && (L % 2)) { set_error("GTR-FDPA models need an even K"); return MMASIM_ERR_SHAPE; }
+    if (m.family == FAM_ST && K > 32 && (K % 32)) { set_error("ST-FDPA models need K to be a multiple of 32"); return MMASIM_ERR_SHAPE; }
+    return MMASIM_OK;
+}
+
+int run_gemm(const mmasim_model* model, const GemmArgs& g, int flags, cudaStream_t stream) {
+    const DevModel& m = model->dev;
+    if (!(flags & MMASIM_GEMM_FORCE_GENERIC) && fast_tfdpa_supported(m, g)) {
+        return launch_fast_tfdpa(m, g, stream);
+    }
+    set_kernel_name("generic");
+    return launch_generic(m, g, stream);
+}
+
+int build_args(const mmasim_model* model, int64_t M, int64_t N, int64_t K, const void* A, const void* B,
+               const void* C, void* D, const mmasim_gemm_opts* opts, GemmArgs* out) {
+    if (!model) { set_error("model is NULL"); return MMASIM_ERR_INVALID_ARG; }
+    if (!A || !B || !D) { set_error("A, B and D must not be NULL"); return MMASIM_ERR_INVALID_ARG; }
+    if (M < 1 || N < 1) { set_error("M and N must be >= 1"); return MMASIM_ERR_SHAPE; }
+    const DevModel& m = model->dev;
+    int st = check_k(m, K);
+    if (st != MMASIM_OK) return st;
+    GemmArgs g;
+    std::memset(&g, 0, sizeof(g));
+    g.M = M; g.N = N; g.K = K;
+    g.A = A; g.B = B; g.C = C; g.D = D;
+    g.lda = g.ldb = K;
+    g.ldc = g.ldd = N;
+    if (m.k_block) g.ld_sfa = g.ld_sfb = (K + m.k_block - 1) / m.k_block;
+    if (opts) {
+        if (opts->lda) g.lda = opts->lda;
+        if (opts->ldb) g.ldb = opts->ldb;
+        if (opts->ldc) g.ldc = opts->ldc;
+        if (opts->ldd) g.ldd = opts->ldd;
+        g.sfa = static_cast<const uint8_t*>(opts->sfa);
+        g.sfb = static_cast<const uint8_t*>(opts->sfb);
+        g.k_chunk = opts->k_chunk;
+        g.row_scale = opts->row_scale;
+        g.col_scale = opts->col_scale;
+    }
+    if (g.lda < K || g.ldb < K || g.ldc < N || g.ldd < N) { set_error("leading dimension smaller than the row length"); return MMASIM_ERR_SHAPE; }
+    if (m.packed4 && ((g.lda | g.ldb | K) & 1)) { set_error("packed FP4 operands need even K and leading dimensions"); return MMASIM_ERR_SHAPE; }
+    if (m.k_block && (!g.sfa || !g.sfb)) { set_error("this model needs scale factors (opts->sfa, opts->sfb)"); return MMASIM_ERR_INVALID_ARG; }
+    if (!m.k_block && (g.sfa || g.sfb)) { set_error("this model takes no scale factors"); return MMASIM_ERR_INVALID_ARG; }
+    const bool fdpa32 = m.family != FAM_FMA && m.family != FAM_FTZ && m.acc == ACC_F32;
+    if (g.k_chunk) {
+        if (!fdpa32) { set_error("k_chunk needs an FDPA model with an FP32 accumulator"); return MMASIM_ERR_UNSUPPORTED; }
+        const int64_t L = K < m.L ? K : m.L;
+        if (g.k_chunk < 0 || g.k_chunk % L || K % g.k_chunk) { set_error("k_chunk must be a multiple of L that divides K"); return MMASIM_ERR_SHAPE; }
+    }
+    if ((g.row_scale != nullptr) != (g.col_scale != nullptr)) { set_error("row_scale and col_scale must be given together"); return MMASIM_ERR_INVALID_ARG; }
+    if (g.row_scale && !fdpa32) { set_error("dequantisation scales need an FDPA model with an FP32 accumulator"); return MMASIM_ERR_UNSUPPORTED; }
+    *out = g;
+    return MMASIM_OK;
+}
+
+}  // namespace
+}  // namespace mmasim
+
+using namespace mmasim;
+
+extern "C" {
+
+mmasim_model* mmasim_create_model_ex(int arch, int a_fmt, int b_fmt, int acc_fmt, const mmasim_overrides* ov) {
+    mmasim_model tmp;
+    const char* why = "";
+    if (!registry_lookup(arch, a_fmt, b_fmt, acc_fmt, &tmp, &why)) {
+        set_error("mmasim_create_model: %s (arch %d, input %d x %d, accumulator %d)", why, arch, a_fmt, b_fmt, acc_fmt);
+        return nullptr;
+    }
+    if (ov) {
+        DevModel& d = tmp.dev;
+        const bool fdpa = d.family == FAM_T || d.family == FAM_ST || d.family == FAM_TR || d.family == FAM_GTR;
+        if ((ov->l_max >= 0 || ov->F >= 0 || ov->F2 >= 0 || ov->rho >= 0 || ov->inner_round >= 0) && !fdpa) {
+            set_error("overrides apply to T-, ST-, TR- and GTR-FDPA models only");
+            return nullptr;
+        }
+        if (ov->l_max >= 0) {
+            if (ov->l_max < 1 || ov->l_max > 64 || (d.family == FAM_GTR && (ov->l_max & 1)) || (d.family == FAM_ST && ov->l_max != 32)) {
+                set_error("l_max override out of range"); return nullptr;
+            }
+            d.L = ov->l_max;
+        }
+        if (ov->F >= 0) { if (ov->F > 30 || ov->F < 1) { set_error("F override must be in 1..30"); return nullptr; } d.F = ov->F; }
+        if (ov->F2 >= 0) { if (d.F2 == 0 || ov->F2 > 36) { set_error("F2 override not applicable"); return nullptr; } d.F2 = ov->F2; }
+        if (d.F2 && d.F2 < d.F) { set_error("F2 must be >= F"); return nullptr; }
+        if (ov->rho >= 0) {
+            const bool fp16 = d.acc == ACC_F16;
+            const bool ok = fp16 ? ov->rho == MMASIM_RNE_FP16 : (ov->rho >= MMASIM_RZ_FP32 && ov->rho <= MMASIM_RNE_FP32);
+            if (!ok) { set_error("rho override does not match the accumulator type"); return nullptr; }
+            d.rho = ov->rho;
+        }
+        if (ov->inner_round >= 0) {
+            if (ov->inner_round > 1 || d.family != FAM_TR) { set_error("inner_round applies to TR-FDPA models only"); return nullptr; }
+            d.inner_round = ov->inner_round;
+        }
+        tmp.info.l_max = d.L; tmp.info.F = d.F; tmp.info.F2 = d.F2; tmp.info.rho = d.rho; tmp.info.inner_round = d.inner_round;
+    }
+    mmasim_model* m = new (std::nothrow) mmasim_model(tmp);
+    if (!m) set_error("out of host memory");
+    return m;
+}
+
+mmasim_model* mmasim_create_model(int arch, int in_fmt, int acc_fmt) {
+    return mmasim_create_model_ex(arch, in_fmt, in_fmt, acc_fmt, nullptr);
+}
+
+void mmasim_destroy_model(mmasim_model* model) { delete model; }
+
+int mmasim_model_info(const mmasim_model* model, mmasim_info* out) {
+    if (!model || !out) { set_error("mmasim_model_info: NULL argument"); return MMASIM_ERR_INVALID_ARG; }
+    *out = model->info;
+    return MMASIM_OK;
+}
+
+int mmasim_gemm_ex(const mmasim_model* model, int64_t M, int64_t N, int64_t K, const void* A, const void* B,
+                   const void* C, void* D, const mmasim_gemm_opts* opts, void* stream) {
+    GemmArgs g;
+    int st = build_args(model, M, N, K, A, B, C, D, opts, &g);
+    if (st != MMASIM_OK) return st;
+    if (!aligned16(A) || !aligned16(B) || !aligned16(D) || (C && !aligned16(C))) {
+        set_error("A, B, C and D must be 16-byte aligned");
+        return MMASIM_ERR_ALIGN;
+    }
+    if ((st = check_device_ptr(A, "A")) != MMASIM_OK) return st;
+    if ((st = check_device_ptr(B, "B")) != MMASIM_OK) return st;
+    if ((st = check_device_ptr(D, "D")) != MMASIM_OK) return st;
+    if (C && (st = check_device_ptr(C, "C")) != MMASIM_OK) return st;
+    return run_gemm(model, g, opts ? opts->flags : 0, static_cast<cudaStream_t>(stream));
+}
+
+int mmasim_gemm(const mmasim_model* model, int64_t M, int64_t N, int64_t K, const void* A, const void* B,
+                const void* C, void* D, void* stream) {
+    return mmasim_gemm_ex(model, M, N, K, A, B, C, D, nullptr, stream);
+}
+
+int mmasim_dot_batch(const mmasim_model* model, int64_t n, int64_t K, const void* A, const void* B,
+                     const void* C, void* D, void* stream) {
+    if (!model) { set_error("model is NULL"); return MMASIM_ERR_INVALID_ARG; }
+    if (!A || !B || !D) { set_error("A, B and D must not be NULL"); return MMASIM_ERR_INVALID_ARG; }
+    if (n < 1) { set_error("n must be >= 1"); return MMASIM_ERR_SHAPE; }
+    const DevModel& m = model->dev;
+    if (m.k_block) { set_error("mmasim_dot_batch supports unscaled models only"); return MMASIM_ERR_UNSUPPORTED; }
+    int st = check_k(m, K);
+    if (st != MMASIM_OK) return st;
+    if (!aligned16(A) || !aligned16(B) || !aligned16(D) || (C && !aligned16(C))) {
+        set_error("A, B, C and D must be 16-byte aligned");
+        return MMASIM_ERR_ALIGN;
+    }
+    if ((st = check_device_ptr(A, "A")) != MMASIM_OK) return st;
+    if ((st = check_device_ptr(B, "B")) != MMASIM_OK) return st;
+    if ((st = check_device_ptr(D, "D")) != MMASIM_OK) return st;
+    if (C && (st = check_device_ptr(C, "C")) != MMASIM_OK) return st;
+    GemmArgs g;
+    std::memset(&g, 0, sizeof(g));
+    g.M = n; g.N = 1; g.K = K;
+    g.A = A; g.B = B; g.C = C; g.D = D;
+    g.lda = g.ldb = K;
+    g.ldc = g.ldd = 1;
+    g.dot_mode = 1;
+    set_kernel_name("generic_dot");
+    return launch_generic(m, g, static_cast<cudaStream_t>(stream));
+}
+
+int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K, const void* A, const void* B,
+                     const void* C, void* D, const mmasim_gemm_opts* opts) {
+    GemmArgs g;
+    int st = build_args(model, M, N, K, A, B, C, D, opts, &g);
+    if (st != MMASIM_OK) return st;
+    const mmasim_info& info = model->info;
+    const size_t a_bytes = size_t((M - 1) * g.lda + K) * info.a_bits / 8;
+    const size_t b_bytes = size_t((N - 1) * g.ldb + K) * info.b_bits / 8;
+    const size_t c_bytes = size_t((M - 1) * g.ldc + N) * info.acc_bytes;
+    const size_t d_bytes = size_t((M - 1) * g.ldd + N) * info.acc_bytes;
+    const size_t sfa_bytes = g.sfa ? size_t(M * g.ld_sfa) : 0, sfb_bytes = g.sfb ? size_t(N * g.ld_sfb) : 0;
+    void *dA = nullptr, *dB = nullptr, *dC = nullptr, *dD = nullptr, *dSA = nullptr, *dSB = nullptr, *dRS = nullptr, *dCS = nullptr;
+    cudaError_t err = cudaSuccess;
+    auto up = [&](void** dst, const void* src, size_t bytes) {
+        if (err != cudaSuccess || !src || !bytes) return;
+        err = cudaMalloc(dst, bytes);
+        if (err == cudaSuccess) err = cudaMemcpy(*dst, src, bytes, cudaMemcpyHostToDevice);
+    };
+    up(&dA, A, a_bytes);
+    up(&dB, B, b_bytes);
+    up(&dC, C, c_bytes);
+    up(&dSA, g.sfa, sfa_bytes);
+    up(&dSB, g.sfb, sfb_bytes);
+    up(&dRS, g.row_scale, size_t(M) * 4);
+    up(&dCS, g.col_scale, size_t(N) * 4);
+    if (err == cudaSuccess) err = cudaMalloc(&dD, d_bytes);
+    if (err == cudaSuccess) {
+        g.A = dA; g.B = dB; g.C = dC; g.D = dD;
+        g.sfa = static_cast<const uint8_t*>(dSA);
+        g.sfb = static_cast<const uint8_t*>(dSB);
+        g.row_scale = static_cast<const float*>(dRS);
+        g.col_scale = static_cast<const float*>(dCS);
+        st = run_gemm(model, g, opts ? opts->flags : 0, nullptr);
+        if (st == MMASIM_OK) err = cudaMemcpy(D, dD, d_bytes, cudaMemcpyDeviceToHost);
+    }
+    cudaFree(dA); cudaFree(dB); cudaFree(dC); cudaFree(dD); cudaFree(dSA); cudaFree(dSB); cudaFree(dRS); cudaFree(dCS);
+    if (err != cudaSuccess) {
+        cudaGetLastError();
+        set_error("mmasim_gemm_host: %s", cudaGetErrorString(err));
+        return MMASIM_ERR_CUDA;
+    }
+    return st;
+}
+
+int mmasim_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t* ops_per_round, void* stream) {
+    if (!sink || !ops_per_round || blocks < 1 || iters < 1 || kind < 0) { set_error("mmasim_int_peak: bad argument"); return MMASIM_ERR_INVALID_ARG; }
+    return launch_int_peak(kind, blocks, iters, sink, ops_per_round, static_cast<cudaStream_t>(stream));
+}
+
+const char* mmasim_last_kernel(void) { return g_kernel; }
+const char* mmasim_last_error(void) { return g_error; }
+
+}  // extern "C"

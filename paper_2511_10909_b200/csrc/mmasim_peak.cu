@@ -1,0 +1,85 @@
+// Issue-rate micro-benchmarks: the denominators of the integer roofline.  Every thread runs eight chains whose
+// operations depend only on earlier operations of the chains, so the instruction mix is exactly what the source
+// says; the host divides the operation count by the measured time.
+#include "mmasim_internal.h"
+
+namespace mmasim {
+namespace {
+
+enum PeakKind : int {
+    PK_IADD3 = 0, PK_LOP3, PK_SHF, PK_IMAD, PK_MACMIX, PK_VIADDMAX, PK_VIADDMAX16X2, PK_F2I, PK_FMUL, PK_POPC,
+    PK_IMAD_PLUS_ALU, PK_FMUL_PLUS_ALU, PK_COUNT
+};
+
+template <int KIND>
+__device__ __forceinline__ void round8(int (&x)[8], float (&f)[8]) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int j = (i + 1) & 7, k = (i + 3) & 7;
+        if (KIND == PK_IADD3) x[i] = x[i] + x[j] + x[k];
+        else if (KIND == PK_LOP3) x[i] = (x[i] & x[j]) ^ x[k];
+        else if (KIND == PK_SHF) x[i] = __funnelshift_rc(x[i], x[j], x[k]);
+        else if (KIND == PK_IMAD) x[i] = x[i] * x[j] + x[k];
+        else if (KIND == PK_MACMIX) {           // exponent add, running max, distance, shift, accumulate
+            const int e = x[j] + x[k];
+            const int m = max(x[i], e);
+            x[i] = x[i] + (int)((unsigned)x[j] >> ((m - e) & 31));
+        } else if (KIND == PK_VIADDMAX) x[i] = __viaddmax_s32(x[j], x[k], x[i]);
+        else if (KIND == PK_VIADDMAX16X2) x[i] = (int)__viaddmax_s16x2((unsigned)x[j], (unsigned)x[k], (unsigned)x[i]);
+        else if (KIND == PK_F2I) x[i] = __float2int_rz(__int_as_float(x[i]));
+        else if (KIND == PK_FMUL) f[i] = f[i] * f[j];
+        else if (KIND == PK_POPC) x[i] = __popc(x[i]) + x[j];
+        else if (KIND == PK_IMAD_PLUS_ALU) { x[i] = x[i] * x[j] + x[k]; x[j] = x[j] + x[k] + x[i]; }
+        else if (KIND == PK_FMUL_PLUS_ALU) { f[i] = f[i] * f[j]; x[i] = x[i] + x[j] + x[k]; }
+    }
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(256) peak_kernel(int64_t iters, int* sink) {
+    int x[8];
+    float f[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        x[i] = threadIdx.x * 2654435 + i * 40503 + blockIdx.x;
+        f[i] = 1.0f + 1e-7f * float(threadIdx.x + i);
+    }
+    for (int64_t it = 0; it < iters; it += 8) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) round8<KIND>(x, f);
+    }
+    int r = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) r ^= x[i] ^ __float_as_int(f[i]);
+    if (r == 0x12345678) *sink = r;             // practically never true: keeps the chains alive
+}
+
+template <int KIND>
+int launch(int64_t blocks, int64_t iters, void* sink, cudaStream_t stream) {
+    peak_kernel<KIND><<<(unsigned)blocks, 256, 0, stream>>>(iters, static_cast<int*>(sink));
+    const cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) { set_error("int_peak launch failed: %s", cudaGetErrorString(err)); return MMASIM_ERR_CUDA; }
+    return MMASIM_OK;
+}
+
+}  // namespace
+
+int launch_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t* ops_per_round, cudaStream_t stream) {
+    iters = (iters + 7) / 8 * 8;
+    switch (kind) {
+        case PK_IADD3: *ops_per_round = 1; return launch<PK_IADD3>(blocks, iters, sink, stream);
+        case PK_LOP3: *ops_per_round = 1; return launch<PK_LOP3>(blocks, iters, sink, stream);
+        case PK_SHF: *ops_per_round = 1; return launch<PK_SHF>(blocks, iters, sink, stream);
+        case PK_IMAD: *ops_per_round = 1; return launch<PK_IMAD>(blocks, iters, sink, stream);
+        case PK_MACMIX: *ops_per_round = 5; return launch<PK_MACMIX>(blocks, iters, sink, stream);
+        case PK_VIADDMAX: *ops_per_round = 1; return launch<PK_VIADDMAX>(blocks, iters, sink, stream);
+        case PK_VIADDMAX16X2: *ops_per_round = 1; return launch<PK_VIADDMAX16X2>(blocks, iters, sink, stream);
+        case PK_F2I: *ops_per_round = 1; return launch<PK_F2I>(blocks, iters, sink, stream);
+        case PK_FMUL: *ops_per_round = 1; return launch<PK_FMUL>(blocks, iters, sink, stream);
+        case PK_POPC: *ops_per_round = 2; return launch<PK_POPC>(blocks, iters, sink, stream);
+        case PK_IMAD_PLUS_ALU: *ops_per_round = 2; return launch<PK_IMAD_PLUS_ALU>(blocks, iters, sink, stream);
+        case PK_FMUL_PLUS_ALU: *ops_per_round = 2; return launch<PK_FMUL_PLUS_ALU>(blocks, iters, sink, stream);
+        default: set_error("mmasim_int_peak: unknown kind %d", kind); return MMASIM_ERR_INVALID_ARG;
+    }
+}
+
+}  // namespace mmasim

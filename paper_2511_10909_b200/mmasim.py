@@ -1,0 +1,242 @@
+"""ctypes binding of libmmasim.so: argument marshalling only, every step of the path runs in the CUDA kernels.
+
+PyTorch is used for device memory and streams.  There is no CPU fallback: if the shared library is missing the
+import fails, and every compute call needs CUDA tensors.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import c_int, c_int32, c_int64, c_void_p, c_char_p, POINTER, Structure, byref
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libmmasim.so")
+
+ARCH = {n: i for i, n in enumerate(
+    ["volta", "turing", "ampere", "ada", "hopper", "blackwell", "rtx_blackwell", "cdna1", "cdna2", "cdna3"])}
+FMT = {n: i for i, n in enumerate(
+    ["fp64", "fp32", "tf32", "bf16", "bf16_1k", "fp16", "e4m3", "e5m2", "e3m2", "e2m3", "e2m1",
+     "mxe4m3", "mxe5m2", "mxe3m2", "mxe2m3", "mxe2m1", "mxf4", "nvf4"])}
+ACC = {"fp32": 0, "fp16": 1, "fp64": 2}
+FAMILY = ["fma", "ftz", "e", "t", "st", "gst", "tr", "gtr"]
+RHO = ["", "RZ-FP32", "RZ-E8M13", "RNE-FP32", "RNE-FP16"]
+FORCE_GENERIC = 1
+
+
+class MmasimError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"mmasim status {status}: {message}")
+        self.status = status
+
+
+class _Info(Structure):
+    _fields_ = [(n, c_int32) for n in ("family", "l_max", "F", "F2", "rho", "P", "G", "k_block", "a_bits", "b_bits",
+                                       "acc_bytes", "inner_round")]
+
+
+class _Overrides(Structure):
+    _fields_ = [(n, c_int32) for n in ("l_max", "F", "F2", "rho", "inner_round")]
+
+
+class _GemmOpts(Structure):
+    _fields_ = [("lda", c_int64), ("ldb", c_int64), ("ldc", c_int64), ("ldd", c_int64),
+                ("sfa", c_void_p), ("sfb", c_void_p), ("k_chunk", c_int64),
+                ("row_scale", c_void_p), ("col_scale", c_void_p), ("flags", c_int32)]
+
+
+def _load():
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2511_10909_b200.build` "
+                          "(there is no CPU fallback)")
+    lib = ctypes.CDLL(_LIB_PATH)
+    lib.mmasim_create_model.restype = c_void_p
+    lib.mmasim_create_model.argtypes = [c_int, c_int, c_int]
+    lib.mmasim_create_model_ex.restype = c_void_p
+    lib.mmasim_create_model_ex.argtypes = [c_int, c_int, c_int, c_int, POINTER(_Overrides)]
+    lib.mmasim_destroy_model.restype = None
+    lib.mmasim_destroy_model.argtypes = [c_void_p]
+    lib.mmasim_model_info.restype = c_int
+    lib.mmasim_model_info.argtypes = [c_void_p, POINTER(_Info)]
+    lib.mmasim_gemm.restype = c_int
+    lib.mmasim_gemm.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.mmasim_gemm_ex.restype = c_int
+    lib.mmasim_gemm_ex.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
+                                   POINTER(_GemmOpts), c_void_p]
+    lib.mmasim_dot_batch.restype = c_int
+    lib.mmasim_dot_batch.argtypes = [c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.mmasim_gemm_host.restype = c_int
+    lib.mmasim_gemm_host.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
+                                     POINTER(_GemmOpts)]
+    lib.mmasim_int_peak.restype = c_int
+    lib.mmasim_int_peak.argtypes = [c_int, c_int64, c_int64, c_void_p, POINTER(c_int32), c_void_p]
+    lib.mmasim_last_kernel.restype = c_char_p
+    lib.mmasim_last_error.restype = c_char_p
+    return lib
+
+
+_lib = _load()
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def _check(status: int):
+    if status != 0:
+        raise MmasimError(status, _lib.mmasim_last_error().decode())
+
+
+def last_kernel() -> str:
+    return _lib.mmasim_last_kernel().decode()
+
+
+class Model:
+    """Handle of one (architecture, input type, accumulator type) model of the paper's Tables 3-7."""
+
+    def __init__(self, arch: str, in_fmt: str, acc: str, b_fmt: str | None = None, **overrides):
+        self.arch, self.in_fmt, self.acc, self.b_fmt = arch, in_fmt, acc, b_fmt or in_fmt
+        ov = None
+        if overrides:
+            vals = {k: -1 for k in ("l_max", "F", "F2", "rho", "inner_round")}
+            for k, v in overrides.items():
+                if k not in vals:
+                    raise TypeError(f"unknown override {k}")
+                vals[k] = RHO.index(v) if k == "rho" and isinstance(v, str) else int(v)
+            ov = byref(_Overrides(**vals))
+        h = _lib.mmasim_create_model_ex(ARCH[arch], FMT[in_fmt], FMT[self.b_fmt], ACC[acc], ov)
+        if not h:
+            raise MmasimError(2, _lib.mmasim_last_error().decode())
+        self._h = c_void_p(h)
+        info = _Info()
+        _check(_lib.mmasim_model_info(self._h, byref(info)))
+        self.family = FAMILY[info.family]
+        self.l_max, self.F, self.F2, self.rho = info.l_max, info.F, info.F2, RHO[info.rho]
+        self.P, self.G, self.k_block = info.P, info.G, info.k_block
+        self.a_bits, self.b_bits, self.acc_bytes = info.a_bits, info.b_bits, info.acc_bytes
+        self.inner_round = info.inner_round
+
+    def __del__(self):
+        h = getattr(self, "_h", None)
+        if h and _lib is not None:
+            _lib.mmasim_destroy_model(h)
+            self._h = None
+
+    def __repr__(self):
+        return f"Model({self.arch}, {self.in_fmt}, {self.acc}: {self.family} L={self.l_max} F={self.F} {self.rho})"
+
+
+def create_model(arch: str, in_fmt: str, acc: str, **kw) -> Model:
+    return Model(arch, in_fmt, acc, **kw)
+
+
+def model_keys():
+    """Every (arch, in_fmt, acc) triple the library accepts with equal A and B types."""
+    keys = []
+    for a in ARCH:
+        for f in FMT:
+            for c in ACC:
+                h = _lib.mmasim_create_model(ARCH[a], FMT[f], ACC[c])
+                if h:
+                    _lib.mmasim_destroy_model(c_void_p(h))
+                    keys.append((a, f, c))
+    return keys
+
+
+def _ptr(t):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return c_void_p(s.cuda_stream)
+
+
+def _acc_dtype(model: Model):
+    import torch
+    return {8: torch.int64, 4: torch.int32, 2: torch.int16}[model.acc_bytes]
+
+
+def _make_opts(sfa=None, sfb=None, k_chunk=0, row_scale=None, col_scale=None, force_generic=False,
+               lda=0, ldb=0, ldc=0, ldd=0):
+    o = _GemmOpts()
+    o.lda, o.ldb, o.ldc, o.ldd = lda, ldb, ldc, ldd
+    o.sfa, o.sfb = sfa, sfb
+    o.k_chunk = k_chunk
+    o.row_scale, o.col_scale = row_scale, col_scale
+    o.flags = FORCE_GENERIC if force_generic else 0
+    return o
+
+
+def gemm(model: Model, A, B, C=None, out=None, *, M=None, N=None, K=None, sfa=None, sfb=None, k_chunk=0,
+         row_scale=None, col_scale=None, force_generic=False, stream=None):
+    """D = Phi(A, B, C) on CUDA tensors of raw words.
+
+    A: M x K, B: N x K (each row is one column of the paper's K x N matrix), C/D: M x N words of the accumulator
+    type (integer tensors of the element width; FP4 of the GST models packed two per byte, so A is M x K/2 uint8
+    and K must be passed).  Returns D (allocated with torch if ``out`` is None).
+    """
+    import torch
+    if not A.is_cuda:
+        raise MmasimError(1, "mmasim.gemm needs CUDA tensors (no CPU fallback); use gemm_host for host buffers")
+    M = A.shape[0] if M is None else M
+    N = B.shape[0] if N is None else N
+    if K is None:
+        K = A.shape[1] * (2 if model.a_bits == 4 else 1)
+    if out is None:
+        out = torch.empty((M, N), dtype=_acc_dtype(model), device=A.device)
+    plain = sfa is None and not k_chunk and row_scale is None and not force_generic
+    if plain:
+        _check(_lib.mmasim_gemm(model._h, M, N, K, _ptr(A), _ptr(B), _ptr(C), _ptr(out), _stream(stream)))
+    else:
+        o = _make_opts(_ptr(sfa), _ptr(sfb), k_chunk, _ptr(row_scale), _ptr(col_scale), force_generic)
+        _check(_lib.mmasim_gemm_ex(model._h, M, N, K, _ptr(A), _ptr(B), _ptr(C), _ptr(out), byref(o), _stream(stream)))
+    return out
+
+
+def dot_batch(model: Model, A, B, C=None, out=None, *, stream=None):
+    """d_t = Phi(a_t, b_t, c_t) for the n rows of A and B (n x K CUDA tensors of raw words)."""
+    import torch
+    if not A.is_cuda:
+        raise MmasimError(1, "mmasim.dot_batch needs CUDA tensors (no CPU fallback)")
+    n, K = A.shape
+    if out is None:
+        out = torch.empty((n,), dtype=_acc_dtype(model), device=A.device)
+    _check(_lib.mmasim_dot_batch(model._h, n, K, _ptr(A), _ptr(B), _ptr(C), _ptr(out), _stream(stream)))
+    return out
+
+
+def gemm_host(model: Model, A, B, C=None, *, K=None, sfa=None, sfb=None, k_chunk=0, row_scale=None, col_scale=None,
+              out=None):
+    """As gemm, on host buffers (numpy arrays or CPU tensors): the library copies to the device and back."""
+    import numpy as np
+
+    def as_np(x):
+        if x is None:
+            return None
+        if hasattr(x, "numpy"):
+            x = x.numpy()
+        return np.ascontiguousarray(x)
+
+    A, B, C, sfa, sfb, row_scale, col_scale = map(as_np, (A, B, C, sfa, sfb, row_scale, col_scale))
+    M, N = A.shape[0], B.shape[0]
+    if K is None:
+        K = A.shape[1] * (2 if model.a_bits == 4 else 1)
+    if out is None:
+        out = np.empty((M, N), dtype={8: np.uint64, 4: np.uint32, 2: np.uint16}[model.acc_bytes])
+    p = lambda x: None if x is None else c_void_p(x.ctypes.data)
+    o = _make_opts(p(sfa), p(sfb), k_chunk, p(row_scale), p(col_scale))
+    _check(_lib.mmasim_gemm_host(model._h, M, N, K, p(A), p(B), p(C), p(out), byref(o)))
+    return out
+
+
+PEAK_KINDS = ["iadd3", "lop3", "shf", "imad", "macmix", "viaddmax", "viaddmax16x2", "f2i", "fmul", "popc",
+              "imad+alu", "fmul+alu"]
+
+
+def int_peak(kind: str, blocks: int, iters: int, sink, stream=None) -> int:
+    """Launch one issue-rate micro-benchmark; returns the number of counted operations of the launch."""
+    opr = c_int32(0)
+    _check(_lib.mmasim_int_peak(PEAK_KINDS.index(kind), blocks, iters, _ptr(sink), byref(opr), _stream(stream)))
+    iters = (iters + 7) // 8 * 8
+    return blocks * 256 * iters * 8 * opr.value
