@@ -1,0 +1,323 @@
+#!/usr/bin/env python
+"""Benchmark of the hot path: bit-exact emulated MACs/s of one MMA model at 4096^3 on a B200.
+
+One "step" is one evaluation D = Phi(A, B, C) of the workload named in ``config.workload`` (default: the FP8 E4M3
+4096 x 4096 x 4096 GEMM under the paper's Hopper FP8 -> FP32 model, L = 32, F = 13, RZ-E8M13) with the inputs
+resident in HBM.  The line also carries the integer-issue roofline of the dominant kernel, the end-to-end number
+through the host-buffer entry point and the CPU oracle timed on a bounded sample.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg3|cfg2|...]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "emulated_macs_per_s"
+UNIT = "MAC/s"
+
+WORKLOADS = {
+    # name: (registry key, (M, N, K), description)
+    "cfg3": (("hopper", "e4m3", "fp32"), (4096, 4096, 4096),
+             "FP8 E4M3 4096x4096x4096, A,B ~ N(0,1) scaled per row to the E4M3 range, C = +0; Hopper FP8->FP32 model (L=32, F=13, RZ-E8M13)"),
+    "cfg3_chunk128": (("hopper", "e4m3", "fp32"), (4096, 4096, 4096),
+                      "as cfg3 with FP32 promotion of partial sums every 128 elements of K and the row/column dequantisation epilogue"),
+    "cfg2": (("ampere", "bf16", "fp32"), (2048, 2048, 2048),
+             "BF16 2048^3, exponents uniform over +-20 binades, C ~ N(0,1); Ampere BF16->FP32 model (L=8, F=24, RZ-FP32)"),
+    "blackwell_e4m3": (("blackwell", "e4m3", "fp32"), (4096, 4096, 4096),
+                       "FP8 E4M3 4096^3 N(0,1) inputs; Blackwell FP8->FP32 model (L=32, F=25, RZ-FP32)"),
+}
+
+
+def algorithmic_ops_per_mac(model) -> float:
+    """Integer operations per emulated MAC of the T-FDPA family: multiply, exponent add, maximum, distance,
+    shift, accumulate (6 per term) plus about 25 per block for the accumulator term, normalisation and rho."""
+    L = max(model.l_max, 1)
+    return 6.0 + 25.0 / L
+
+
+def make_inputs(name):
+    from paper_2511_10909_b200 import workloads as wl
+    key, (M, N, K), _ = WORKLOADS[name]
+    if name.startswith("cfg3"):
+        A, B, C, sa, sb = wl.cfg3(M)
+        inp = {"A": A, "B": B, "C": C}
+        if name == "cfg3_chunk128":
+            inp.update(k_chunk=128, row_scale=sa, col_scale=sb)
+        return inp
+    if name == "cfg2":
+        A, B, C = wl.cfg2(M)
+        return {"A": A, "B": B, "C": C}
+    d = wl.normal_inputs(key[1], key[2], M, N, K, seed=5)
+    return {"A": d["A"], "B": d["B"], "C": d["C"]}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.lines, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        loaded = [x for x in sm if x > 0.5 * max(sm)] if sm else []
+        return {"sm_mhz": float(np.median(loaded)) if loaded else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample_rate(name, inp, seconds_target=15.0, processes=None):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload's outputs; returns (MAC/s, info)."""
+    import oracle
+    from paper_2511_10909_b200 import workloads as wl
+    key, (M, N, K), _ = WORKLOADS[name]
+    m = oracle.lookup(*key)
+    cores = processes or os.cpu_count() or 1
+    kw = {}
+    if "k_chunk" in inp:
+        kw.update(k_chunk=inp["k_chunk"], row_scale=inp["row_scale"].view(np.uint32), col_scale=inp["col_scale"].view(np.uint32))
+    probe = wl.sample_pairs(M, N, 64 * cores, seed=77)
+    t0 = time.perf_counter()
+    oracle.phi_gemm_sampled(m, inp["A"], inp["B"], inp["C"], probe, processes=cores, **kw)
+    dt = time.perf_counter() - t0
+    n = int(max(64 * cores, min(200000, len(probe) * seconds_target / max(dt, 1e-3))))
+    pairs = wl.sample_pairs(M, N, n, seed=78)
+    t0 = time.perf_counter()
+    oracle.phi_gemm_sampled(m, inp["A"], inp["B"], inp["C"], pairs, processes=cores, **kw)
+    dt = time.perf_counter() - t0
+    return n * K / dt, {"cores": cores, "sample": f"{n} seeded output elements x K={K} of {name} ({n * K:.3g} MACs in {dt:.1f} s)"}
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle on this machine's host cores, each step a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2511_10909_b200 import workloads as wl
+    name = args.workload
+    key, (M, N, K), desc = WORKLOADS[name]
+    inp = make_inputs(name)
+    m = oracle.lookup(*key)
+    cores = os.cpu_count() or 1
+    kw = {}
+    if "k_chunk" in inp:
+        kw.update(k_chunk=inp["k_chunk"], row_scale=inp["row_scale"].view(np.uint32), col_scale=inp["col_scale"].view(np.uint32))
+    n = 512 * cores
+    times = []
+    for step in range(args.warmup + args.steps):
+        pairs = wl.sample_pairs(M, N, n, seed=100 + step)
+        t0 = time.perf_counter()
+        oracle.phi_gemm_sampled(m, inp["A"], inp["B"], inp["C"], pairs, processes=cores, **kw)
+        if step >= args.warmup:
+            times.append(time.perf_counter() - t0)
+    total = sum(times)
+    value = n * K * args.steps / total
+    sample = f"{n} seeded output elements x K={K} per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+        "config": {"workload": f"{name}: {desc}", "model": "-".join(key), "M": M, "N": N, "K": K, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def run_ours(args):
+    import torch
+    from paper_2511_10909_b200.build import build
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank == 0:
+        build()
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    from paper_2511_10909_b200 import mmasim
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    name = args.workload
+    key, (M, N, K), desc = WORKLOADS[name]
+    inp = make_inputs(name)          # every rank evaluates its own full batch of the workload (weak scaling, no exchange)
+    model = mmasim.Model(*key)
+
+    def to_dev(x):
+        x = np.ascontiguousarray(x)
+        view = {1: np.uint8, 2: np.int16, 4: np.int32, 8: np.int64}[x.dtype.itemsize]
+        return torch.from_numpy(x.view(view) if x.dtype.kind != "f" else x).to(dev)
+
+    dA, dB, dC = to_dev(inp["A"]), to_dev(inp["B"]), to_dev(inp["C"])
+    kw = {}
+    if "k_chunk" in inp:
+        kw = dict(k_chunk=inp["k_chunk"], row_scale=to_dev(inp["row_scale"]), col_scale=to_dev(inp["col_scale"]))
+    dD = torch.empty((M, N), dtype=torch.int32 if model.acc_bytes == 4 else torch.int16, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # larger than the 126 MB L2
+
+    def step():
+        mmasim.gemm(model, dA, dB, dC, out=dD, **kw)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    kernel_name = mmasim.last_kernel()
+
+    # integer-issue peak, measured live (independent 3-input integer adds on every SM)
+    sink = torch.zeros(4, dtype=torch.int32, device=dev)
+    peaks = {}
+    for kind in ("iadd3", "imad"):
+        mmasim.int_peak(kind, 148 * 8, 2048, sink)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        ops = 0
+        for _ in range(4):
+            ops += mmasim.int_peak(kind, 148 * 8, 4096, sink)
+        e1.record()
+        torch.cuda.synchronize()
+        peaks[kind] = ops / (e0.elapsed_time(e1) * 1e-3)
+
+    # ---- timed region: K steps, device timers, L2 flushed between steps ----
+    sampler = ClockSampler(local_rank)
+    events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    for e0, e1 in events:
+        flush.zero_()
+        e0.record()
+        step()
+        e1.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    clocks = sampler.stop()
+    total_ms = sum(e0.elapsed_time(e1) for e0, e1 in events)
+    if dist is not None:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    macs_per_step = float(M) * N * K * world
+    value = macs_per_step * args.steps / (total_ms * 1e-3)
+
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region) ----
+    e2e = None
+    if rank == 0 or world > 1:
+        def pinned(x):
+            x = np.ascontiguousarray(x)
+            t = torch.from_numpy(x.view({1: np.uint8, 2: np.int16, 4: np.int32, 8: np.int64}[x.dtype.itemsize]) if x.dtype.kind != "f" else x)
+            return t.pin_memory()
+        hA, hB, hC = pinned(inp["A"]), pinned(inp["B"]), pinned(inp["C"])
+        hD = torch.empty((M, N), dtype=dD.dtype).pin_memory()
+        hkw = {}
+        if "k_chunk" in inp:
+            hkw = dict(k_chunk=inp["k_chunk"], row_scale=pinned(inp["row_scale"]), col_scale=pinned(inp["col_scale"]))
+        n_e2e = max(1, min(args.steps, 3))
+        mmasim.gemm_host(model, hA, hB, hC, out=hD.numpy(), **hkw)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            mmasim.gemm_host(model, hA, hB, hC, out=hD.numpy(), **hkw)
+        torch.cuda.synchronize()
+        e2e_s = (time.perf_counter() - t0) / n_e2e
+        if dist is not None:
+            t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
+        h2d = hA.numel() * hA.element_size() + hB.numel() * hB.element_size() + hC.numel() * hC.element_size()
+        e2e = {"value": macs_per_step / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": int(hD.numel() * hD.element_size()), "ms_per_step": 1e3 * e2e_s,
+               "api": "mmasim_gemm_host (cudaMalloc + H2D + kernel + D2H + cudaFree per call)"}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    ops_per_mac = algorithmic_ops_per_mac(model)
+    per_gpu_macs_s = value / world
+    achieved = per_gpu_macs_s * ops_per_mac
+    peak = peaks["iadd3"]
+    roofline = {"bound": "alu", "achieved": achieved / 1e12, "peak": peak / 1e12, "unit": "Tint-op/s",
+                "frac": achieved / peak, "traffic": None,
+                "kernel": kernel_name, "algorithmic_int_ops_per_mac": ops_per_mac,
+                "peak_source": "measured live: independent 3-input integer adds on all SMs (mmasim_int_peak kind 0)",
+                "imad_peak": peaks["imad"] / 1e12}
+    cpu_value, cpu_info = oracle_sample_rate(name, inp)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int32", "data": "synthetic",
+        "config": {"workload": f"{name}: {desc}", "model": "-".join(key), "M": M, "N": N, "K": K,
+                   "l2": "flushed between timed steps (256 MiB write)", "parallelism": f"replicas x{world} (independent batches, no exchange)"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps,
+        "roofline": roofline,
+        "cpu_baseline": {"value": cpu_value, "unit": UNIT, "kind": "oracle", **cpu_info},
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS))
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

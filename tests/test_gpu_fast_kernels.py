@@ -1,0 +1,107 @@
+"""The tuned kernels against the oracle (sampled) and against the generic kernels (every output), bit for bit,
+on ragged shapes, random bit streams (NaN, infinities, subnormals, wide exponent spreads) and extreme accumulators."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2511_10909_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+gu = pytest.importorskip("gpu_util") if torch.cuda.is_available() else None
+
+FAST8 = [("ada", "e4m3", "fp32"), ("ada", "e5m2", "fp16"), ("hopper", "e4m3", "fp32"), ("hopper", "e5m2", "fp32"),
+         ("hopper", "e4m3", "fp16"), ("hopper", "e5m2", "fp16"), ("blackwell", "e4m3", "fp32"), ("blackwell", "e5m2", "fp32"),
+         ("blackwell", "e3m2", "fp32"), ("blackwell", "e2m3", "fp32"), ("blackwell", "e2m1", "fp32"),
+         ("blackwell", "e4m3", "fp16"), ("rtx_blackwell", "e2m3", "fp16")]
+
+
+def _check(key, inp, nsample=600, expect_kernel=None, **kw):
+    from paper_2511_10909_b200 import mmasim
+    D = gu.run_gemm(key, inp, **kw)
+    if expect_kernel:
+        assert mmasim.last_kernel() == expect_kernel
+    G = gu.run_gemm(key, inp, force_generic=True, **kw)
+    assert mmasim.last_kernel() == "generic"
+    bad = np.argwhere(D != G)
+    assert bad.size == 0, (key, len(bad), bad[:4], [hex(int(D[tuple(b)])) for b in bad[:4]], [hex(int(G[tuple(b)])) for b in bad[:4]])
+    M, N = D.shape
+    pairs = wl.sample_pairs(M, N, nsample, seed=M + N)
+    okw = {}
+    if "k_chunk" in kw:
+        okw["k_chunk"] = kw["k_chunk"]
+    if "row_scale" in kw:
+        okw["row_scale"] = gu.host_words(kw["row_scale"])
+        okw["col_scale"] = gu.host_words(kw["col_scale"])
+    gu.assert_samples_equal(D, gu.oracle_samples(key, inp, pairs, **okw), pairs, str(key))
+    return D
+
+
+@pytest.mark.parametrize("key", FAST8, ids=lambda k: "-".join(k))
+def test_fp8_normal_inputs_ragged_shape(key):
+    inp = wl.normal_inputs(key[1], key[2], 200, 100, 256, seed=21)
+    _check(key, inp, expect_kernel="tfdpa8")
+
+
+@pytest.mark.parametrize("key", FAST8, ids=lambda k: "-".join(k))
+def test_fp8_random_bit_stream(key):
+    g = wl.rng(22)
+    M, N, K = 150, 70, 128
+    m = oracle.lookup(*key)
+    bits = 1 + oracle.FORMATS[m.elem].ebits + oracle.FORMATS[m.elem].mbits
+    A = g.integers(0, 1 << bits, (M, K), dtype=np.uint8)
+    B = g.integers(0, 1 << bits, (N, K), dtype=np.uint8)
+    if key[2] == "fp16":
+        C = g.integers(0, 1 << 16, (M, N), dtype=np.uint16)
+    else:
+        C = g.integers(0, 1 << 32, (M, N), dtype=np.uint32)
+    _check(key, {"A": A, "B": B, "C": C}, expect_kernel="tfdpa8")
+
+
+@pytest.mark.parametrize("key", [("hopper", "e4m3", "fp32"), ("blackwell", "e5m2", "fp32"), ("blackwell", "e4m3", "fp16")],
+                         ids=lambda k: "-".join(k))
+def test_fp8_extreme_accumulators(key):
+    # accumulators around the subnormal boundary, around the overflow boundary, and products that cancel exactly
+    g = wl.rng(23)
+    M, N, K = 128, 64, 64
+    inp = wl.normal_inputs(key[1], key[2], M, N, K, seed=24)
+    A = inp["A"].copy()
+    A[:, 1::2] = inp["A"][:, 0::2] ^ 0x80                  # exact cancellation of neighbouring terms in half the rows
+    Bm = inp["B"].copy()
+    Bm[:, 1::2] = inp["B"][:, 0::2]
+    A[M // 2:], Bm[N // 2:] = inp["A"][M // 2:], inp["B"][N // 2:]
+    if key[2] == "fp16":
+        C = ((g.integers(0, 2, (M, N)) << 15) | (g.choice([0, 1, 2, 29, 30], (M, N)) << 10) | g.integers(0, 1024, (M, N))).astype(np.uint16)
+    else:
+        C = ((g.integers(0, 2, (M, N)) << 31) | (g.choice([0, 1, 2, 3, 252, 253, 254], (M, N)) << 23) | g.integers(0, 1 << 23, (M, N))).astype(np.uint32)
+    _check(key, {"A": A, "B": Bm, "C": C}, expect_kernel="tfdpa8")
+
+
+def test_fp8_promotion_and_dequant_ragged():
+    key = ("hopper", "e4m3", "fp32")
+    g = wl.rng(25)
+    inp = wl.normal_inputs("e4m3", "fp32", 130, 66, 512, seed=26)
+    inp["A"][3, 7] = 0x7F                                       # one NaN
+    rs = gu.dev(g.standard_normal(130).astype(np.float32))
+    cs = gu.dev(g.standard_normal(66).astype(np.float32))
+    _check(key, inp, expect_kernel="tfdpa8", k_chunk=128, row_scale=rs, col_scale=cs)
+    _check(key, inp, expect_kernel="tfdpa8", k_chunk=32)
+    _check(key, inp, expect_kernel="tfdpa8", row_scale=rs, col_scale=cs)
+
+
+def test_mixed_fp8_types():
+    from paper_2511_10909_b200 import mmasim
+    g = wl.rng(27)
+    M, N, K = 64, 64, 64
+    A = g.integers(0, 256, (M, K), dtype=np.uint8)
+    B = g.integers(0, 256, (N, K), dtype=np.uint8)
+    C = g.standard_normal((M, N)).astype(np.float32).view(np.uint32)
+    model = mmasim.Model("blackwell", "e4m3", "fp32", b_fmt="e5m2")
+    D = gu.host_words(mmasim.gemm(model, gu.dev(A), gu.dev(B), gu.dev(C)))
+    assert mmasim.last_kernel() == "tfdpa8"
+    F = oracle.FORMATS
+    for i, j in [(0, 0), (5, 9), (63, 63), (17, 40), (33, 2)] + [tuple(p) for p in wl.sample_pairs(M, N, 100, 5)]:
+        d = int(C[i, j])
+        for k in range(0, K, 32):
+            d = oracle.t_fdpa(A[i, k:k + 32].tolist(), B[j, k:k + 32].tolist(), d, F["e4m3"], F["e5m2"], F["fp32"], 25, "RZ-FP32")
+        assert int(D[i, j]) == d, (i, j)
