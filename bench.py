@@ -33,8 +33,16 @@ WORKLOADS = {
              "FP8 E4M3 4096x4096x4096, A,B ~ N(0,1) scaled per row to the E4M3 range, C = +0; Hopper FP8->FP32 model (L=32, F=13, RZ-E8M13)"),
     "cfg3_chunk128": (("hopper", "e4m3", "fp32"), (4096, 4096, 4096),
                       "as cfg3 with FP32 promotion of partial sums every 128 elements of K and the row/column dequantisation epilogue"),
+    "cfg3_2k": (("hopper", "e4m3", "fp32"), (2048, 2048, 2048),
+                "FP8 E4M3 2048^3 (reduced case for profiler captures), inputs as cfg3; Hopper FP8->FP32 model"),
     "cfg2": (("ampere", "bf16", "fp32"), (2048, 2048, 2048),
              "BF16 2048^3, exponents uniform over +-20 binades, C ~ N(0,1); Ampere BF16->FP32 model (L=8, F=24, RZ-FP32)"),
+    "hopper_fp16": (("hopper", "fp16", "fp32"), (4096, 4096, 4096),
+                    "FP16 4096^3 N(0,1) inputs; Hopper FP16->FP32 model (L=16, F=25, RZ-FP32)"),
+    "volta_fp16": (("volta", "fp16", "fp32"), (4096, 4096, 4096),
+                   "FP16 4096^3 N(0,1) inputs; Volta FP16->FP32 model (L=4, F=23, RZ-FP32)"),
+    "ampere_bf16": (("ampere", "bf16", "fp32"), (4096, 4096, 4096),
+                    "BF16 4096^3 N(0,1) inputs; Ampere BF16->FP32 model (L=8, F=24, RZ-FP32)"),
     "blackwell_e4m3": (("blackwell", "e4m3", "fp32"), (4096, 4096, 4096),
                        "FP8 E4M3 4096^3 N(0,1) inputs; Blackwell FP8->FP32 model (L=32, F=25, RZ-FP32)"),
 }
@@ -248,7 +256,7 @@ def run_ours(args):
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region) ----
     e2e = None
-    if rank == 0 or world > 1:
+    if not args.skip_extras and (rank == 0 or world > 1):
         def pinned(x):
             x = np.ascontiguousarray(x)
             t = torch.from_numpy(x.view({1: np.uint8, 2: np.int16, 4: np.int32, 8: np.int64}[x.dtype.itemsize]) if x.dtype.kind != "f" else x)
@@ -289,7 +297,7 @@ def run_ours(args):
                 "kernel": kernel_name, "algorithmic_int_ops_per_mac": ops_per_mac,
                 "peak_source": "measured live: independent 3-input integer adds on all SMs (mmasim_int_peak kind 0)",
                 "imad_peak": peaks["imad"] / 1e12}
-    cpu_value, cpu_info = oracle_sample_rate(name, inp)
+    cpu_value, cpu_info = (None, {"cores": 0, "sample": "skipped (--skip-extras)"}) if args.skip_extras else oracle_sample_rate(name, inp)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -312,6 +320,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS))
+    ap.add_argument("--skip-extras", action="store_true",
+                    help="skip the end-to-end and CPU-oracle legs (profiler captures only; not a valid bench line)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

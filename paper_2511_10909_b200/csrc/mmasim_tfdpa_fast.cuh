@@ -1,0 +1,542 @@
+// Tuned T-FDPA kernel template (Algorithm 5 + Algorithm 7 + Table 2) for GEMM-sized inputs.
+//
+// Work decomposition.  A CTA of 256 threads owns a 128 x 64 tile of D; a thread owns an 8 x 4 micro-tile and keeps
+// its 32 accumulators decoded in registers for the whole K loop: `cs`, the one's-complement signed significand
+// aligned to F fractional bits, and `ce`, the exponent (biased, see below).  K is walked in chunks of 32 elements:
+// the CTA loads the raw A / B words of the chunk, decodes every element once into an operand word and an exponent
+// word (8-bit formats through a 256-entry table, 16/32-bit formats arithmetically) and stores them k-major in
+// shared memory, so that one 16-byte shared load feeds four rows (or columns) of a micro-tile.
+//
+// Per block of L elements and per output (Algorithm 7):
+//   pass 1   e_max = max(Exp(c), max_k(Exp(a_k) + Exp(b_k)))   fused add-max on two 16-bit lanes: half an
+//                                                              instruction per term
+//   pass 2   X_k  = A_op * B_op                                one multiply (FMA pipe)
+//            d_k  = e_max (+ g) - Exp(a_k) - Exp(b_k)          one 3-input add (ALU pipe)
+//            t_k  = X_k >> d_k                                 one shift (ALU pipe), clamped: >= 32 shifts all bits out
+//            S   += t_k                                        issued as multiply-add by one (FMA pipe): the ALU pipe
+//                                                              is the busy one
+//   then the accumulator term, the sign corrections, normalisation and rho (Table 2) - about 25 instructions.
+//
+// Sign-magnitude truncation without per-term sign work.  RZ_F truncates the magnitude of each aligned term, while
+// an arithmetic right shift of a two's-complement number rounds toward minus infinity.  Negative terms are
+// therefore carried in one's complement: -t is represented by ~t = -t - 1, and the number of negative terms of the
+// block (a population count over per-row / per-column sign bit masks) is added back once per block.
+//  * 8-bit inputs (FP8 / FP6 / FP4): the operands are built so that the 32-bit product itself has that form,
+//      X = s * (m << (F - frac + g)) + r,  m = sig_a * sig_b,  s = +-1 the product's sign,  g = mbits_a + 1 guard
+//      bits,  0 <= r < 2^g for s = +1 and -2^g <= r <= -1 for s = -1,
+//    by A_op = +-sig_a and B_op = (+-sig_b << (F - frac + g)) + sign(b), which gives r = +-sig_a.  Then
+//    X >> (d + g) is floor(m * 2^(F - frac) / 2^d) for positive terms and its one's complement for negative ones.
+//    A term counts as negative when the signs differ and sig_a != 0 (with b = +-0 it is -sig_a >> (d+g) = -1).
+//  * 16/32-bit inputs (FP16 / BF16 / TF32): the product would not fit with guard bits, so magnitudes are multiplied
+//    and shifted, and one 3-input logic instruction applies sign_a xor sign_b (full-width masks staged beside the
+//    operands).  Every term whose sign bits differ counts as negative.
+//
+// Exponents are staged with a bias of 512 per element (1024 per product / accumulator) so that they are positive
+// 16-bit lane values.
+//
+// Everything that is rare takes a slow, by-the-book route: NaN / infinity inputs (the threads rescan the raw words
+// of the block and keep sticky NaN / +inf / -inf flags per output, Section 4.2), results outside the normal range of
+// the accumulator format, and block sums that do not fit 32 bits (generic conversion routine on a 64-bit sum).
+#pragma once
+#include "mmasim_device.cuh"
+
+namespace mmasim {
+namespace fast {
+
+constexpr int BM = 128, BN = 64, TM = 8, TN = 4, KC = 32, NT = 256;
+constexpr int EB = 512;            // bias of a staged element exponent
+constexpr int CB = 2 * EB;         // bias of an exponent sum and of the accumulator exponent
+
+enum ElemKind : int { EK_LUT8 = 0, EK_F16 = 1, EK_BF16 = 2, EK_TF32 = 3 };
+
+template <int EK> struct Elem;
+template <> struct Elem<EK_LUT8> { static constexpr int BYTES = 1, TASK = 16, EBITS = 4, MBITS = 3, BIAS = 7, LOW = 0; static constexpr bool SIGNMAG = false; };  // EBITS.. unused: table-decoded
+template <> struct Elem<EK_F16> { static constexpr int BYTES = 2, TASK = 8, EBITS = 5, MBITS = 10, BIAS = 15, LOW = 0; static constexpr bool SIGNMAG = true; };
+template <> struct Elem<EK_BF16> { static constexpr int BYTES = 2, TASK = 8, EBITS = 8, MBITS = 7, BIAS = 127, LOW = 0; static constexpr bool SIGNMAG = true; };
+template <> struct Elem<EK_TF32> { static constexpr int BYTES = 4, TASK = 8, EBITS = 8, MBITS = 10, BIAS = 127, LOW = 13; static constexpr bool SIGNMAG = true; };
+
+struct LutEntry {
+    uint32_t op;        // multiplier operand
+    uint32_t exp;       // Exp(x) + EB (minimum exponent for non-finite inputs, whose operand is zero)
+    uint32_t bits;      // bit 0: sign, bit 16: nonzero significand
+    uint32_t special;   // nonzero for infinity / NaN
+};
+
+template <int EK>
+struct Smem {
+    uint32_t a_op[KC][BM];
+    uint32_t a_exp[KC][BM];
+    uint32_t b_op[KC][BN];
+    uint32_t b_exp[KC][BN];
+    uint32_t a_exp2[KC / 2][BM];    // exponents of elements 2p (low half) and 2p + 1 (high half)
+    uint32_t b_exp2[KC / 2][BN];
+    uint32_t a_msk[Elem<EK>::SIGNMAG ? KC : 1][BM];   // 0 / ~0: sign of the element (sign-magnitude kinds)
+    uint32_t b_msk[Elem<EK>::SIGNMAG ? KC : 1][BN];
+    LutEntry lut_a[Elem<EK>::SIGNMAG ? 1 : 256];
+    LutEntry lut_b[Elem<EK>::SIGNMAG ? 1 : 256];
+    uint32_t a_sgn[BM], a_nz[BM], b_sgn[BN];          // bit k of row r: sign / nonzero of element k of the chunk
+    int special[2];                                   // chunk (by parity) holds an infinity or a NaN
+};
+
+__device__ __forceinline__ int asr_clamp(int x, int d) {
+    int r;
+    asm("shr.s32 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(d));      // amounts above 31 behave as 31 (sign fill)
+    return r;
+}
+__device__ __forceinline__ uint32_t lsr_clamp(uint32_t x, int d) {
+    uint32_t r;
+    asm("shr.u32 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(d));      // amounts above 31 give 0
+    return r;
+}
+__device__ __forceinline__ uint32_t shl_clamp(uint32_t x, int d) {
+    uint32_t r;
+    asm("shl.b32 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(d));      // amounts above 31 give 0
+    return r;
+}
+__device__ __forceinline__ int msb_index(uint32_t x) {
+    int r;
+    asm("bfind.u32 %0, %1;" : "=r"(r) : "r"(x));                // -1 for x == 0
+    return r;
+}
+__device__ __forceinline__ int mad_one(int t, int one, int s) {
+    int r;
+    asm("mad.lo.s32 %0, %1, %2, %3;" : "=r"(r) : "r"(t), "r"(one), "r"(s));
+    return r;
+}
+
+// Accumulator state of one output.
+struct Acc {
+    int cs;     // one's complement signed significand, F fractional bits relative to 2^(ce - CB)
+    int ce;     // Exp(c) + CB
+};
+
+template <int F, bool ACC16>
+__device__ __forceinline__ Acc acc_from_word(uint32_t w, uint32_t& sp) {
+    static_assert(F >= (ACC16 ? 10 : 13), "accumulator significand must not lose bits beyond rho");
+    const AccDec d = decode_acc(w, ACC16);
+    Acc a;
+    if (d.cls != CLS_FINITE) {
+        sp |= (d.cls == CLS_NAN) ? 1u : (d.sign ? 4u : 2u);
+        a.cs = 0;
+        a.ce = (ACC16 ? -14 : -126) + CB;
+        return a;
+    }
+    constexpr int MB = ACC16 ? 10 : 23;
+    // F < 23 (F = 13): the low bits of an FP32 c fall below every block's truncation point anyway
+    const int mag = (F >= MB) ? int(d.sig << (F >= MB ? F - MB : 0)) : int(d.sig >> (F >= MB ? 0 : MB - F));
+    a.cs = d.sign ? ~mag : mag;
+    a.ce = d.exp + CB;
+    return a;
+}
+
+// Accumulator state back to an output word (exact: the state always holds a representable value).
+template <int F, bool ACC16>
+__device__ __forceinline__ uint32_t acc_to_word(const Acc& a, uint32_t sp) {
+    if (sp) {
+        const int kind = ((sp & 1u) || (sp & 6u) == 6u) ? 1 : ((sp & 2u) ? 2 : 3);
+        return special_word(kind, ACC16, true);
+    }
+    constexpr int MB = ACC16 ? 10 : 23;
+    const uint32_t sign = a.cs < 0;
+    const uint32_t magF = uint32_t(sign ? ~a.cs : a.cs);
+    const uint32_t sig = (F >= MB) ? (magF >> (F >= MB ? F - MB : 0)) : (magF << (F >= MB ? 0 : MB - F));
+    const uint32_t field = (sig >> MB) ? uint32_t(a.ce - CB + (ACC16 ? 15 : 127)) : 0u;
+    return (sign << (ACC16 ? 15 : 31)) | (field << MB) | (sig & ((1u << MB) - 1u));
+}
+
+// Slow conversion: any rho, any range.  S is the exact fixed-point sum in units of 2^(e_max - F).
+template <int F, int RHO, bool ACC16>
+__device__ __noinline__ void rho_slow(long long S, int e_max, Acc& a, uint32_t& sp) {
+    const uint32_t w = rho_apply(RHO, S, e_max - F);
+    a = acc_from_word<F, ACC16>(w, sp);
+}
+
+// Fast conversion of a 32-bit block sum whose result is a normal number (or zero); `vmin` / `vmax` collect the result
+// exponents so that the caller can detect, once per block, that some output left the normal range.
+template <int F, int RHO>
+__device__ __forceinline__ void rho_fast(int S, int emaxb, Acc& a, int& vmin, int& vmax) {
+    constexpr bool ACC16 = RHO == RHO_RNE_FP16;
+    constexpr bool RNE = RHO == RHO_RNE_FP16 || RHO == RHO_RNE_FP32;
+    constexpr int MB = RHO == RHO_RZ_E8M13 ? 13 : (ACC16 ? 10 : 23);
+    constexpr int EMINB = (ACC16 ? -14 : -126) + CB;
+    const int sg = S >> 31;
+    const uint32_t mag = uint32_t(abs(S));
+    const int msb = msb_index(mag);
+    const uint32_t norm = shl_clamp(mag, 31 - msb);            // leading one at bit 31 (msb <= 30, so bit 0 is free)
+    uint32_t sig;
+    int ve = emaxb - F + msb;
+    if (RNE) {
+        const uint32_t n2 = norm >> 1;
+        const uint32_t r = (n2 + (((1u << (29 - MB)) - 1u) + ((n2 >> (30 - MB)) & 1u))) >> (30 - MB);
+        const uint32_t carry = r >> (MB + 1);
+        sig = r >> carry;
+        ve += int(carry);
+    } else {
+        sig = norm >> (31 - MB);
+    }
+    ve = mag ? ve : EMINB;                                     // an exactly zero sum is +0 with the minimum exponent
+    vmin = min(vmin, ve);
+    vmax = max(vmax, ve);
+    a.ce = ve;
+    a.cs = int(sig << (F - MB)) ^ sg;
+}
+
+template <int EK>
+__device__ __forceinline__ uint32_t raw_elem(const void* p, int64_t idx) {
+    if (Elem<EK>::BYTES == 1) return static_cast<const uint8_t*>(p)[idx];
+    if (Elem<EK>::BYTES == 2) return static_cast<const uint16_t*>(p)[idx];
+    return static_cast<const uint32_t*>(p)[idx];
+}
+
+// Arithmetic decode of one FP16 / BF16 / TF32 word: significand, biased exponent, sign, special flag.
+template <int EK>
+__device__ __forceinline__ void decode_signmag(uint32_t w, uint32_t& sig, uint32_t& expb, uint32_t& sign, uint32_t& special) {
+    using E = Elem<EK>;
+    const uint32_t x = w >> E::LOW;
+    const uint32_t mant = x & ((1u << E::MBITS) - 1u);
+    const uint32_t field = (x >> E::MBITS) & ((1u << E::EBITS) - 1u);
+    sign = (x >> (E::MBITS + E::EBITS)) & 1u;
+    special = field == ((1u << E::EBITS) - 1u);
+    sig = special ? 0u : (mant | (field ? (1u << E::MBITS) : 0u));
+    expb = uint32_t(int((field && !special) ? field : 1u) - E::BIAS + EB);
+}
+
+template <int EK, int L, int F, int RHO, bool PROMOTE>
+__global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
+    using E = Elem<EK>;
+    constexpr bool SIGNMAG = E::SIGNMAG;
+    constexpr bool ACC16 = RHO == RHO_RNE_FP16;
+    constexpr int EMINB = (ACC16 ? -14 : -126) + CB, EMAXB = (ACC16 ? 15 : 127) + CB;
+    constexpr int NSUM = (F >= 25 && L >= 16) ? 2 : 1;       // 32-bit partial sums per block
+    constexpr int HALF = L / NSUM;
+    constexpr int NBLK = KC / L;
+    static_assert(KC % L == 0 && L % 2 == 0, "blocks tile the chunk; pass 1 handles pairs of elements");
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    Smem<EK>& s = *reinterpret_cast<Smem<EK>*>(smem_raw);
+
+    const int tid = threadIdx.x;
+    const int tx = tid % 16, ty = tid / 16;
+    const int64_t row0 = int64_t(blockIdx.y) * BM, col0 = int64_t(blockIdx.x) * BN;
+    const FmtDesc fa = fmt_desc(m.fmt_a), fb = fmt_desc(m.fmt_b);
+    const int pre = F - (fa.mbits + fb.mbits);      // left shift that gives a product F fractional bits
+    const int guard = SIGNMAG ? 0 : fa.mbits + 1;   // guard bits below the truncation point (8-bit kinds)
+    const int one = int(blockDim.x >> 8);           // 1, but not a compile-time constant (see mad_one)
+
+    if (!SIGNMAG) {                                 // decode tables: entry `tid` of both
+        const uint32_t da = decode_elem(fa, uint32_t(tid)), db = decode_elem(fb, uint32_t(tid));
+        const bool fin_a = dec_cls(da) == CLS_FINITE, fin_b = dec_cls(db) == CLS_FINITE;
+        LutEntry ea, eb;
+        ea.op = fin_a ? uint32_t(dec_ssig(da)) : 0u;
+        ea.exp = uint32_t((fin_a ? dec_exp(da) : 1 - fa.bias) + EB);
+        ea.bits = fin_a ? (dec_sign(da) | (uint32_t(dec_sig(da) != 0u) << 16)) : 0u;
+        ea.special = fin_a ? 0u : 1u;
+        const int sb = fin_b ? dec_ssig(db) : 0;
+        const int ub = fin_b ? (dec_sign(db) ? -1 : 1) : 0;     // also for b = +-0 (see the header comment)
+        eb.op = uint32_t(sb * (1 << (pre + guard)) + ub);
+        eb.exp = uint32_t((fin_b ? dec_exp(db) : 1 - fb.bias) + EB);
+        eb.bits = fin_b ? dec_sign(db) : 0u;
+        eb.special = fin_b ? 0u : 1u;
+        s.lut_a[tid] = ea;
+        s.lut_b[tid] = eb;
+    }
+    if (tid == 0) s.special[0] = s.special[1] = 0;
+
+    Acc acc[TM][TN];
+    uint32_t sp_nan = 0u, sp_pinf = 0u, sp_ninf = 0u;   // per output (bit r * TN + c): NaN / +inf / -inf seen so far
+    float promoted[PROMOTE ? TM : 1][PROMOTE ? TN : 1];
+#define MMASIM_SP_GET(r, c) ((((sp_nan >> ((r) * TN + (c))) & 1u)) | (((sp_pinf >> ((r) * TN + (c))) & 1u) << 1) | (((sp_ninf >> ((r) * TN + (c))) & 1u) << 2))
+#define MMASIM_SP_OR(r, c, v) do { const uint32_t v_ = (v); sp_nan |= (v_ & 1u) << ((r) * TN + (c)); sp_pinf |= ((v_ >> 1) & 1u) << ((r) * TN + (c)); sp_ninf |= ((v_ >> 2) & 1u) << ((r) * TN + (c)); } while (0)
+#pragma unroll
+    for (int r = 0; r < TM; ++r)
+#pragma unroll
+        for (int c = 0; c < TN; ++c) {
+            const int64_t i = row0 + ty * TM + r, j = col0 + tx * TN + c;
+            uint32_t w = 0u;
+            if (g.C && i < g.M && j < g.N)
+                w = ACC16 ? uint32_t(static_cast<const uint16_t*>(g.C)[i * g.ldc + j])
+                          : static_cast<const uint32_t*>(g.C)[i * g.ldc + j];
+            if (PROMOTE) { promoted[PROMOTE ? r : 0][PROMOTE ? c : 0] = __uint_as_float(w); w = 0u; }
+            uint32_t ev = 0u;
+            acc[r][c] = acc_from_word<F, ACC16>(w, ev);
+            MMASIM_SP_OR(r, c, ev);
+        }
+
+    int chunk = 0;
+    for (int64_t k0 = 0; k0 < g.K; k0 += KC, ++chunk) {
+        __syncthreads();
+        // ---- stage the chunk: each task decodes E::TASK consecutive elements of one row ----
+        {
+            constexpr int TPR = KC / E::TASK;                  // tasks per row
+            uint32_t spec = 0u;
+#pragma unroll
+            for (int t0 = 0; t0 < (BM + BN) * TPR; t0 += NT) {
+                const int task = t0 + tid;
+                const bool is_a = task < BM * TPR;
+                if (task >= (BM + BN) * TPR) break;
+                const int u = is_a ? task : task - BM * TPR;
+                const int rows = is_a ? BM : BN;
+                const int r = u % rows, h = u / rows;          // consecutive threads take consecutive rows
+                const int64_t grow = (is_a ? row0 : col0) + r;
+                const bool valid = grow < (is_a ? g.M : g.N);
+                const unsigned char* base = static_cast<const unsigned char*>(is_a ? g.A : g.B) +
+                                            (grow * (is_a ? g.lda : g.ldb) + k0 + h * E::TASK) * E::BYTES;
+                uint32_t wv[E::TASK * E::BYTES / 4];
+#pragma unroll
+                for (int q = 0; q < E::TASK * E::BYTES / 16; ++q) {
+                    uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+                    if (valid) raw = reinterpret_cast<const uint4*>(base)[q];
+                    wv[4 * q] = raw.x; wv[4 * q + 1] = raw.y; wv[4 * q + 2] = raw.z; wv[4 * q + 3] = raw.w;
+                }
+                uint32_t bits = 0u, prev_exp = 0u;
+#pragma unroll
+                for (int q = 0; q < E::TASK; ++q) {
+                    const int kk = h * E::TASK + q;
+                    uint32_t op, expb;
+                    if (!SIGNMAG) {
+                        const uint32_t byte = (wv[q / 4] >> (8 * (q % 4))) & 0xFFu;
+                        const LutEntry e = is_a ? s.lut_a[byte] : s.lut_b[byte];
+                        op = e.op;
+                        expb = e.exp;
+                        bits += e.bits << q;
+                        spec |= e.special;
+                    } else {
+                        const uint32_t w = E::BYTES == 2 ? ((wv[q / 2] >> (16 * (q % 2))) & 0xFFFFu) : wv[q];
+                        uint32_t sig, sign, special;
+                        decode_signmag<EK>(w, sig, expb, sign, special);
+                        op = is_a ? sig : (sig << pre);
+                        bits += sign << q;
+                        spec |= special;
+                        if (is_a) s.a_msk[SIGNMAG ? kk : 0][r] = 0u - sign; else s.b_msk[SIGNMAG ? kk : 0][r] = 0u - sign;
+                    }
+                    if (is_a) { s.a_op[kk][r] = op; s.a_exp[kk][r] = expb; }
+                    else { s.b_op[kk][r] = op; s.b_exp[kk][r] = expb; }
+                    if (q & 1) {
+                        const uint32_t pair = prev_exp | (expb << 16);
+                        if (is_a) s.a_exp2[kk / 2][r] = pair; else s.b_exp2[kk / 2][r] = pair;
+                    }
+                    prev_exp = expb;
+                }
+                // sign (and nonzero) bits of the task's elements go to bits [h * TASK, h * TASK + TASK) of the row's masks
+                if (E::TASK == 16) {
+                    if (is_a) {
+                        reinterpret_cast<uint16_t*>(&s.a_sgn[r])[h] = uint16_t(bits);
+                        reinterpret_cast<uint16_t*>(&s.a_nz[r])[h] = uint16_t(bits >> 16);
+                    } else {
+                        reinterpret_cast<uint16_t*>(&s.b_sgn[r])[h] = uint16_t(bits);
+                    }
+                } else {
+                    if (is_a) reinterpret_cast<uint8_t*>(&s.a_sgn[r])[h] = uint8_t(bits);
+                    else reinterpret_cast<uint8_t*>(&s.b_sgn[r])[h] = uint8_t(bits);
+                }
+            }
+            if (spec) atomicOr(&s.special[chunk & 1], 1);
+        }
+        __syncthreads();
+
+        if (tid == 0) s.special[(chunk + 1) & 1] = 0;
+        const bool chunk_special = s.special[chunk & 1] != 0;
+
+#pragma unroll 1
+        for (int blk = 0; blk < NBLK; ++blk) {
+            const int kb = blk * L;
+            // ---- rare: the chunk holds an infinity or a NaN: special-value events of this block (Section 4.2).
+            // Flags are sticky: once an output is special the finite arithmetic below no longer matters for it.
+            if (chunk_special) {
+#pragma unroll 1
+                for (int r = 0; r < TM; ++r)
+#pragma unroll 1
+                    for (int c = 0; c < TN; ++c) {
+                        const int64_t i = row0 + ty * TM + r, j = col0 + tx * TN + c;
+                        if (i >= g.M || j >= g.N) continue;
+                        Special ev;
+                        for (int kk = kb; kk < kb + L; ++kk) {
+                            const uint32_t x = decode_elem(fa, raw_elem<EK>(g.A, i * g.lda + k0 + kk));
+                            const uint32_t y = decode_elem(fb, raw_elem<EK>(g.B, j * g.ldb + k0 + kk));
+                            ev.product(x, y);
+                        }
+                        const uint32_t bit = 1u << (r * TN + c);
+                        if (ev.nan) sp_nan |= bit;
+                        if (ev.pinf) sp_pinf |= bit;
+                        if (ev.ninf) sp_ninf |= bit;
+                    }
+            }
+
+            int emax[TM][TN];       // e_max + CB, then e_max + CB + guard
+            // ---- pass 1: block maximum of the exponent sums, accumulator included; two elements per instruction ----
+            {
+                uint32_t em2[TM][TN];
+#pragma unroll
+                for (int r = 0; r < TM; ++r)
+#pragma unroll
+                    for (int c = 0; c < TN; ++c) em2[r][c] = uint32_t(acc[r][c].ce) * 0x10001u;
+#pragma unroll 4
+                for (int kp = kb / 2; kp < (kb + L) / 2; ++kp) {
+                    const uint4 ea0 = *reinterpret_cast<const uint4*>(&s.a_exp2[kp][ty * TM]);
+                    const uint4 ea1 = *reinterpret_cast<const uint4*>(&s.a_exp2[kp][ty * TM + 4]);
+                    const uint4 eb = *reinterpret_cast<const uint4*>(&s.b_exp2[kp][tx * TN]);
+                    const uint32_t ea[TM] = {ea0.x, ea0.y, ea0.z, ea0.w, ea1.x, ea1.y, ea1.z, ea1.w};
+                    const uint32_t ebv[TN] = {eb.x, eb.y, eb.z, eb.w};
+#pragma unroll
+                    for (int r = 0; r < TM; ++r)
+#pragma unroll
+                        for (int c = 0; c < TN; ++c) em2[r][c] = __viaddmax_s16x2(ea[r], ebv[c], em2[r][c]);
+                }
+#pragma unroll
+                for (int r = 0; r < TM; ++r)
+#pragma unroll
+                    for (int c = 0; c < TN; ++c) emax[r][c] = max(int(em2[r][c] & 0xFFFFu), int(em2[r][c] >> 16));
+            }
+            // ---- accumulator term: align at e_max and truncate; one's complement keeps sign-magnitude semantics,
+            // the "+1 if c is negative" restores the two's complement value ----
+            int S0[TM][TN], S1[NSUM == 2 ? TM : 1][NSUM == 2 ? TN : 1];
+#pragma unroll
+            for (int r = 0; r < TM; ++r)
+#pragma unroll
+                for (int c = 0; c < TN; ++c) {
+                    S0[r][c] = asr_clamp(acc[r][c].cs, emax[r][c] - acc[r][c].ce) - (acc[r][c].cs >> 31);
+                    if (NSUM == 2) S1[NSUM == 2 ? r : 0][NSUM == 2 ? c : 0] = 0;
+                    emax[r][c] += guard;
+                }
+            // ---- pass 2: multiply, align, truncate, add ----
+#pragma unroll 2
+            for (int kk = kb; kk < kb + L; ++kk) {
+                const bool second = NSUM == 2 && (kk - kb >= HALF);
+                const int4 eb = *reinterpret_cast<const int4*>(&s.b_exp[kk][tx * TN]);
+                const int4 ob = *reinterpret_cast<const int4*>(&s.b_op[kk][tx * TN]);
+                const int ebv[TN] = {eb.x, eb.y, eb.z, eb.w};
+                const int obv[TN] = {ob.x, ob.y, ob.z, ob.w};
+                uint32_t mbv[TN] = {0u, 0u, 0u, 0u};
+                if (SIGNMAG) {
+                    const uint4 mb = *reinterpret_cast<const uint4*>(&s.b_msk[SIGNMAG ? kk : 0][tx * TN]);
+                    mbv[0] = mb.x; mbv[1] = mb.y; mbv[2] = mb.z; mbv[3] = mb.w;
+                }
+#pragma unroll
+                for (int rh = 0; rh < TM; rh += 4) {
+                    const int4 ea = *reinterpret_cast<const int4*>(&s.a_exp[kk][ty * TM + rh]);
+                    const int4 oa = *reinterpret_cast<const int4*>(&s.a_op[kk][ty * TM + rh]);
+                    const int eav[4] = {ea.x, ea.y, ea.z, ea.w};
+                    const int oav[4] = {oa.x, oa.y, oa.z, oa.w};
+                    uint32_t mav[4] = {0u, 0u, 0u, 0u};
+                    if (SIGNMAG) {
+                        const uint4 ma = *reinterpret_cast<const uint4*>(&s.a_msk[SIGNMAG ? kk : 0][ty * TM + rh]);
+                        mav[0] = ma.x; mav[1] = ma.y; mav[2] = ma.z; mav[3] = ma.w;
+                    }
+#pragma unroll
+                    for (int r4 = 0; r4 < 4; ++r4)
+#pragma unroll
+                        for (int c = 0; c < TN; ++c) {
+                            const int r = rh + r4;
+                            const int X = oav[r4] * obv[c];
+                            const int d = emax[r][c] - eav[r4] - ebv[c];
+                            int t;
+                            if (SIGNMAG) t = int(lsr_clamp(uint32_t(X), d) ^ mav[r4] ^ mbv[c]);
+                            else t = asr_clamp(X, d);
+                            if (second) S1[NSUM == 2 ? r : 0][NSUM == 2 ? c : 0] = mad_one(t, one, S1[NSUM == 2 ? r : 0][NSUM == 2 ? c : 0]);
+                            else S0[r][c] = mad_one(t, one, S0[r][c]);
+                        }
+                }
+            }
+            // ---- sign corrections, normalisation, rho ----
+            const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
+            int vmin = EMINB, vmax = EMINB;
+            uint32_t ovf = 0u;                         // sign bit set: a 32-bit block sum overflowed
+#pragma unroll
+            for (int r = 0; r < TM; ++r) {
+                const uint32_t sa = s.a_sgn[ty * TM + r];
+                const uint32_t nza = SIGNMAG ? kmask : (s.a_nz[ty * TM + r] & kmask);
+#pragma unroll
+                for (int c = 0; c < TN; ++c) {
+                    const int nneg = __popc((sa ^ s.b_sgn[tx * TN + c]) & nza);
+                    int S = S0[r][c] + nneg;
+                    if (NSUM == 2) {
+                        const int s1 = S1[NSUM == 2 ? r : 0][NSUM == 2 ? c : 0];
+                        const int sum = S + s1;
+                        ovf |= uint32_t((S ^ sum) & (s1 ^ sum));
+                        S = sum;
+                    }
+                    rho_fast<F, RHO>(S, emax[r][c] - guard, acc[r][c], vmin, vmax);
+                }
+            }
+            if (vmin < EMINB || vmax > EMAXB || int(ovf) < 0) {
+                // some result is subnormal, overflows, or a sum needs 64 bits: redo every output by the book
+#pragma unroll
+                for (int r = 0; r < TM; ++r) {
+                    const uint32_t sa = s.a_sgn[ty * TM + r];
+                    const uint32_t nza = SIGNMAG ? kmask : (s.a_nz[ty * TM + r] & kmask);
+#pragma unroll
+                    for (int c = 0; c < TN; ++c) {
+                        const int nneg = __popc((sa ^ s.b_sgn[tx * TN + c]) & nza);
+                        long long S = (long long)S0[r][c] + nneg;
+                        if (NSUM == 2) S += (long long)S1[NSUM == 2 ? r : 0][NSUM == 2 ? c : 0];
+                        uint32_t ev = 0u;
+                        rho_slow<F, RHO, ACC16>(S, emax[r][c] - guard - CB, acc[r][c], ev);
+                        if (ev && !MMASIM_SP_GET(r, c)) MMASIM_SP_OR(r, c, ev);   // overflow to infinity (RNE only)
+                    }
+                }
+            }
+        }
+        // ---- FP32 promotion of the partial sum every k_chunk elements ----
+        if (PROMOTE && ((k0 + KC) % g.k_chunk) == 0) {
+#pragma unroll
+            for (int r = 0; r < TM; ++r)
+#pragma unroll
+                for (int c = 0; c < TN; ++c) {
+                    const float part = __uint_as_float(acc_to_word<F, ACC16>(acc[r][c], MMASIM_SP_GET(r, c)));
+                    float v = __fadd_rn(promoted[PROMOTE ? r : 0][PROMOTE ? c : 0], part);
+                    if (v != v) v = __uint_as_float(0x7FFFFFFFu);
+                    promoted[PROMOTE ? r : 0][PROMOTE ? c : 0] = v;
+                    uint32_t dummy = 0u;
+                    acc[r][c] = acc_from_word<F, ACC16>(0u, dummy);
+                }
+            sp_nan = sp_pinf = sp_ninf = 0u;
+        }
+    }
+
+    // ---- store ----
+#pragma unroll
+    for (int r = 0; r < TM; ++r)
+#pragma unroll
+        for (int c = 0; c < TN; ++c) {
+            const int64_t i = row0 + ty * TM + r, j = col0 + tx * TN + c;
+            if (i >= g.M || j >= g.N) continue;
+            uint32_t w = PROMOTE ? __float_as_uint(promoted[PROMOTE ? r : 0][PROMOTE ? c : 0])
+                                 : acc_to_word<F, ACC16>(acc[r][c], MMASIM_SP_GET(r, c));
+            if (g.row_scale) {
+                float sc = __fmul_rn(g.row_scale[i], g.col_scale[j]);
+                if (sc != sc) sc = __uint_as_float(0x7FFFFFFFu);
+                float v = __fmul_rn(sc, __uint_as_float(w));
+                if (v != v) v = __uint_as_float(0x7FFFFFFFu);
+                w = __float_as_uint(v);
+            }
+            if (ACC16) static_cast<uint16_t*>(g.D)[i * g.ldd + j] = uint16_t(w);
+            else static_cast<uint32_t*>(g.D)[i * g.ldd + j] = w;
+        }
+#undef MMASIM_SP_GET
+#undef MMASIM_SP_OR
+}
+
+template <int EK, int L, int F, int RHO, bool PROMOTE>
+cudaError_t launch_one(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
+    const size_t sh = sizeof(Smem<EK>);
+    cudaError_t err = cudaFuncSetAttribute(tfdpa_kernel<EK, L, F, RHO, PROMOTE>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
+    if (err != cudaSuccess) return err;
+    dim3 grid((unsigned)((g.N + BN - 1) / BN), (unsigned)((g.M + BM - 1) / BM), 1);
+    tfdpa_kernel<EK, L, F, RHO, PROMOTE><<<grid, NT, sh, stream>>>(m, g);
+    return cudaGetLastError();
+}
+
+// With or without FP32 promotion (FP32 accumulators only).
+template <int EK, int L, int F, int RHO>
+cudaError_t launch_variant(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
+    if (RHO != RHO_RNE_FP16 && g.k_chunk) return launch_one<EK, L, F, RHO, RHO != RHO_RNE_FP16>(m, g, stream);
+    return launch_one<EK, L, F, RHO, false>(m, g, stream);
+}
+
+// Per element kind: returns cudaErrorInvalidValue when (L, F, rho) has no instantiation.
+cudaError_t launch_lut8(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
+cudaError_t launch_f16(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
+cudaError_t launch_bf16(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
+cudaError_t launch_tf32(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
+
+}  // namespace fast
+}  // namespace mmasim

@@ -16,6 +16,12 @@ FAST8 = [("ada", "e4m3", "fp32"), ("ada", "e5m2", "fp16"), ("hopper", "e4m3", "f
          ("blackwell", "e4m3", "fp16"), ("rtx_blackwell", "e2m3", "fp16")]
 
 
+FAST16 = [("volta", "fp16", "fp32"), ("volta", "fp16", "fp16"), ("turing", "fp16", "fp32"), ("ampere", "fp16", "fp16"),
+          ("hopper", "fp16", "fp32"), ("blackwell", "fp16", "fp16"), ("ampere", "bf16", "fp32"), ("hopper", "bf16", "fp32"),
+          ("ampere", "tf32", "fp32"), ("hopper", "tf32", "fp32")]
+KERNEL16 = {"fp16": "tfdpa_f16", "bf16": "tfdpa_bf16", "tf32": "tfdpa_tf32"}
+
+
 def _check(key, inp, nsample=600, expect_kernel=None, **kw):
     from paper_2511_10909_b200 import mmasim
     D = gu.run_gemm(key, inp, **kw)
@@ -40,7 +46,7 @@ def _check(key, inp, nsample=600, expect_kernel=None, **kw):
 @pytest.mark.parametrize("key", FAST8, ids=lambda k: "-".join(k))
 def test_fp8_normal_inputs_ragged_shape(key):
     inp = wl.normal_inputs(key[1], key[2], 200, 100, 256, seed=21)
-    _check(key, inp, expect_kernel="tfdpa8")
+    _check(key, inp, expect_kernel="tfdpa_lut8")
 
 
 @pytest.mark.parametrize("key", FAST8, ids=lambda k: "-".join(k))
@@ -55,7 +61,7 @@ def test_fp8_random_bit_stream(key):
         C = g.integers(0, 1 << 16, (M, N), dtype=np.uint16)
     else:
         C = g.integers(0, 1 << 32, (M, N), dtype=np.uint32)
-    _check(key, {"A": A, "B": B, "C": C}, expect_kernel="tfdpa8")
+    _check(key, {"A": A, "B": B, "C": C}, expect_kernel="tfdpa_lut8")
 
 
 @pytest.mark.parametrize("key", [("hopper", "e4m3", "fp32"), ("blackwell", "e5m2", "fp32"), ("blackwell", "e4m3", "fp16")],
@@ -74,7 +80,7 @@ def test_fp8_extreme_accumulators(key):
         C = ((g.integers(0, 2, (M, N)) << 15) | (g.choice([0, 1, 2, 29, 30], (M, N)) << 10) | g.integers(0, 1024, (M, N))).astype(np.uint16)
     else:
         C = ((g.integers(0, 2, (M, N)) << 31) | (g.choice([0, 1, 2, 3, 252, 253, 254], (M, N)) << 23) | g.integers(0, 1 << 23, (M, N))).astype(np.uint32)
-    _check(key, {"A": A, "B": Bm, "C": C}, expect_kernel="tfdpa8")
+    _check(key, {"A": A, "B": Bm, "C": C}, expect_kernel="tfdpa_lut8")
 
 
 def test_fp8_promotion_and_dequant_ragged():
@@ -84,9 +90,9 @@ def test_fp8_promotion_and_dequant_ragged():
     inp["A"][3, 7] = 0x7F                                       # one NaN
     rs = gu.dev(g.standard_normal(130).astype(np.float32))
     cs = gu.dev(g.standard_normal(66).astype(np.float32))
-    _check(key, inp, expect_kernel="tfdpa8", k_chunk=128, row_scale=rs, col_scale=cs)
-    _check(key, inp, expect_kernel="tfdpa8", k_chunk=32)
-    _check(key, inp, expect_kernel="tfdpa8", row_scale=rs, col_scale=cs)
+    _check(key, inp, expect_kernel="tfdpa_lut8", k_chunk=128, row_scale=rs, col_scale=cs)
+    _check(key, inp, expect_kernel="tfdpa_lut8", k_chunk=32)
+    _check(key, inp, expect_kernel="tfdpa_lut8", row_scale=rs, col_scale=cs)
 
 
 def test_mixed_fp8_types():
@@ -98,10 +104,64 @@ def test_mixed_fp8_types():
     C = g.standard_normal((M, N)).astype(np.float32).view(np.uint32)
     model = mmasim.Model("blackwell", "e4m3", "fp32", b_fmt="e5m2")
     D = gu.host_words(mmasim.gemm(model, gu.dev(A), gu.dev(B), gu.dev(C)))
-    assert mmasim.last_kernel() == "tfdpa8"
+    assert mmasim.last_kernel() == "tfdpa_lut8"
     F = oracle.FORMATS
     for i, j in [(0, 0), (5, 9), (63, 63), (17, 40), (33, 2)] + [tuple(p) for p in wl.sample_pairs(M, N, 100, 5)]:
         d = int(C[i, j])
         for k in range(0, K, 32):
             d = oracle.t_fdpa(A[i, k:k + 32].tolist(), B[j, k:k + 32].tolist(), d, F["e4m3"], F["e5m2"], F["fp32"], 25, "RZ-FP32")
         assert int(D[i, j]) == d, (i, j)
+
+
+@pytest.mark.parametrize("key", FAST16, ids=lambda k: "-".join(k))
+def test_16bit_normal_inputs_ragged_shape(key):
+    inp = wl.normal_inputs(key[1], key[2], 200, 100, 256, seed=31)
+    _check(key, inp, expect_kernel=KERNEL16[key[1]])
+
+
+@pytest.mark.parametrize("key", FAST16, ids=lambda k: "-".join(k))
+def test_16bit_random_bit_stream(key):
+    g = wl.rng(32)
+    M, N, K = 150, 70, 128
+    wbits = 32 if key[1] == "tf32" else 16
+    dt = np.uint32 if wbits == 32 else np.uint16
+    A = g.integers(0, 1 << wbits, (M, K), dtype=np.uint64).astype(dt)
+    B = g.integers(0, 1 << wbits, (N, K), dtype=np.uint64).astype(dt)
+    if key[2] == "fp16":
+        C = g.integers(0, 1 << 16, (M, N), dtype=np.uint16)
+    else:
+        C = g.integers(0, 1 << 32, (M, N), dtype=np.uint32)
+    _check(key, {"A": A, "B": B, "C": C}, expect_kernel=KERNEL16[key[1]])
+
+
+@pytest.mark.parametrize("key", FAST16, ids=lambda k: "-".join(k))
+def test_16bit_config4_classes_as_gemm(key):
+    # the adversarial classes of the probe batch (subnormals, cancellation, outliers, inf / NaN, bit streams) as GEMM operands
+    m = oracle.lookup(*key)
+    A, B, C = wl.cfg4(m.elem, 32, n=1 << 12)
+    A, B = A[:192].reshape(192, 32), B[192:192 + 96].reshape(96, 32)
+    A = np.ascontiguousarray(np.tile(A, (1, 4)))
+    B = np.ascontiguousarray(np.tile(B, (1, 4)))
+    Cm = np.resize(C, (192, 96)).copy()
+    if key[2] == "fp16":
+        Cm = (Cm >> 16).astype(np.uint16)
+    _check(key, {"A": A, "B": B, "C": Cm}, expect_kernel=KERNEL16[key[1]])
+
+
+def test_bf16_wide_exponents_and_extreme_accumulators():
+    key = ("hopper", "bf16", "fp32")
+    g = wl.rng(33)
+    M, N, K = 128, 64, 64
+    def mat(rows):
+        sign = g.integers(0, 2, (rows, K), dtype=np.uint16)
+        exp = g.integers(1, 255, (rows, K)).astype(np.uint16)          # the whole exponent range
+        man = g.integers(0, 128, (rows, K), dtype=np.uint16)
+        return ((sign << 15) | (exp << 7) | man).astype(np.uint16)
+    C = ((g.integers(0, 2, (M, N)) << 31) | (g.choice([0, 1, 2, 100, 127, 150, 253, 254], (M, N)) << 23) | g.integers(0, 1 << 23, (M, N))).astype(np.uint32)
+    _check(key, {"A": mat(M), "B": mat(N), "C": C}, expect_kernel="tfdpa_bf16")
+
+
+def test_16bit_promotion():
+    key = ("hopper", "fp16", "fp32")
+    inp = wl.normal_inputs("fp16", "fp32", 130, 66, 256, seed=34)
+    _check(key, inp, expect_kernel="tfdpa_f16", k_chunk=64)
