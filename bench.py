@@ -313,6 +313,75 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Every registry row at size^3 (config 5 / the per-model headline): MAC/s per model, optional oracle check of
+    seeded sampled outputs, one JSON line per model into gpurun_out/ and a summary line on stdout."""
+    import torch
+    import oracle
+    from paper_2511_10909_b200.build import build
+    build()
+    from paper_2511_10909_b200 import mmasim, workloads as wl
+    torch.cuda.set_device(0)
+    size = args.size
+    M = N = K = size
+    keys = sorted(oracle.REGISTRY)
+    if args.models:
+        keys = [k for k in keys if "-".join(k) in args.models.split(",")]
+    os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
+    out_path = os.path.join(ROOT, "gpurun_out", f"sweep_{size}.jsonl")
+    cache = {}
+    rows = []
+
+    def to_dev(x):
+        x = np.ascontiguousarray(x)
+        return torch.from_numpy(x.view({1: np.uint8, 2: np.int16, 4: np.int32, 8: np.int64}[x.dtype.itemsize])).cuda()
+
+    with open(out_path, "w") as fh:
+        for key in keys:
+            ck = (key[1], key[2])
+            if ck not in cache:
+                cache.clear()
+                cache[ck] = wl.normal_inputs(key[1], key[2], M, N, K, seed=5)
+            inp = cache[ck]
+            model = mmasim.Model(*key)
+            dA, dB, dC = to_dev(inp["A"]), to_dev(inp["B"]), to_dev(inp["C"])
+            kw = {}
+            if "sfa" in inp:
+                kw = dict(sfa=to_dev(inp["sfa"]), sfb=to_dev(inp["sfb"]))
+            D = mmasim.gemm(model, dA, dB, dC, **kw)            # warm-up
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(args.steps):
+                mmasim.gemm(model, dA, dB, dC, out=D, **kw)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / args.steps
+            row = {"model": "-".join(key), "family": model.family, "kernel": mmasim.last_kernel(), "size": size,
+                   "ms": ms, "macs_per_s": float(M) * N * K / (ms * 1e-3)}
+            if args.check:
+                pairs = wl.sample_pairs(M, N, args.check, seed=55)
+                A, B = inp["A"], inp["B"]
+                if key[1] in ("mxf4", "nvf4"):
+                    lo, hi = A & 0xF, A >> 4
+                    A = np.stack([lo, hi], axis=-1).reshape(M, K)
+                    lo, hi = B & 0xF, B >> 4
+                    B = np.stack([lo, hi], axis=-1).reshape(N, K)
+                want = oracle.phi_gemm_sampled(oracle.lookup(*key), A, B, inp["C"], pairs, SFA=inp.get("sfa"), SFB=inp.get("sfb"))
+                got = D.cpu().numpy()
+                got = got.view({2: np.uint16, 4: np.uint32, 8: np.uint64}[got.dtype.itemsize])[pairs[:, 0], pairs[:, 1]].astype(np.uint64)
+                row["checked"] = int(args.check)
+                row["mismatches"] = int((got != want).sum())
+            fh.write(json.dumps(row) + "\n")
+            fh.flush()
+            rows.append(row)
+            del dA, dB, dC, D
+    bad = sum(r.get("mismatches", 0) for r in rows)
+    print(json.dumps({"sweep": size, "models": len(rows), "mismatching_outputs": bad,
+                      "min_macs_per_s": min(r["macs_per_s"] for r in rows), "max_macs_per_s": max(r["macs_per_s"] for r in rows),
+                      "file": os.path.relpath(out_path, ROOT)}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -322,8 +391,14 @@ def main():
     ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS))
     ap.add_argument("--skip-extras", action="store_true",
                     help="skip the end-to-end and CPU-oracle legs (profiler captures only; not a valid bench line)")
+    ap.add_argument("--sweep", action="store_true", help="time every registry row at --size^3 (not the bench line)")
+    ap.add_argument("--size", type=int, default=4096)
+    ap.add_argument("--check", type=int, default=0, help="with --sweep: compare this many seeded sampled outputs per model with the oracle")
+    ap.add_argument("--models", default="", help="with --sweep: comma-separated arch-infmt-acc names (default: all)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

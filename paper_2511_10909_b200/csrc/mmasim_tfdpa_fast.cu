@@ -9,7 +9,12 @@ bool is8(int f) { return f == EF_E4M3 || f == EF_E5M2 || f == EF_E3M2 || f == EF
 
 // 0: no tuned kernel; otherwise 1 + element kind
 int kind_of(const DevModel& m) {
-    if (m.family != FAM_T || m.packed4) return 0;
+    if ((m.family != FAM_T && m.family != FAM_ST) || m.packed4) return 0;
+    if (m.family == FAM_ST) {
+        const bool ok = is8(m.fmt_a) && is8(m.fmt_b) && m.F == 25 && m.L == 32 && m.rho == RHO_RZ_FP32 && m.acc == ACC_F32 &&
+                        m.k_block == 32 && m.scale_fmt == EF_E8M0;
+        return ok ? 1 + fast::EK_LUT8 : 0;
+    }
     const bool acc_ok = (m.rho == RHO_RNE_FP16) == (m.acc == ACC_F16) && m.acc != ACC_F64;
     if (!acc_ok) return 0;
     if (is8(m.fmt_a) && is8(m.fmt_b)) {

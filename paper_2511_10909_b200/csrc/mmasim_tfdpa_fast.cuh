@@ -201,7 +201,7 @@ __device__ __forceinline__ void decode_signmag(uint32_t w, uint32_t& sig, uint32
     expb = uint32_t(int((field && !special) ? field : 1u) - E::BIAS + EB);
 }
 
-template <int EK, int L, int F, int RHO, bool PROMOTE>
+template <int EK, int L, int F, int RHO, bool PROMOTE, bool ST = false>
 __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
     using E = Elem<EK>;
     constexpr bool SIGNMAG = E::SIGNMAG;
@@ -211,6 +211,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
     constexpr int HALF = L / NSUM;
     constexpr int NBLK = KC / L;
     static_assert(KC % L == 0 && L % 2 == 0, "blocks tile the chunk; pass 1 handles pairs of elements");
+    static_assert(!ST || L == KC, "ST-FDPA: one scale factor pair per block of 32 (Algorithm 8)");
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Smem<EK>& s = *reinterpret_cast<Smem<EK>*>(smem_raw);
 
@@ -334,7 +335,29 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
         __syncthreads();
 
         if (tid == 0) s.special[(chunk + 1) & 1] = 0;
-        const bool chunk_special = s.special[chunk & 1] != 0;
+        bool chunk_special = s.special[chunk & 1] != 0;
+
+        // ST-FDPA (Algorithm 8): Exp(alpha) of this thread's rows and Exp(beta) of its columns for this block of 32
+        int sa_exp[ST ? TM : 1], sb_exp[ST ? TN : 1];
+        uint32_t scale_nan = 0u;                    // bit r * TN + c: alpha or beta of that output is NaN
+        if (ST) {
+            const int64_t sblk = k0 / KC;
+#pragma unroll
+            for (int r = 0; r < TM; ++r) {
+                const int64_t i = row0 + ty * TM + r;
+                const uint32_t w = i < g.M ? uint32_t(g.sfa[i * g.ld_sfa + sblk]) : 127u;
+                sa_exp[ST ? r : 0] = int(w) - 127;
+                if (w == 0xFFu) scale_nan |= ((1u << TN) - 1u) << (r * TN);
+            }
+#pragma unroll
+            for (int c = 0; c < TN; ++c) {
+                const int64_t j = col0 + tx * TN + c;
+                const uint32_t w = j < g.N ? uint32_t(g.sfb[j * g.ld_sfb + sblk]) : 127u;
+                sb_exp[ST ? c : 0] = int(w) - 127;
+                if (w == 0xFFu) scale_nan |= 0x11111111u << c;
+            }
+            sp_nan |= scale_nan;                    // a NaN scale factor makes the block result NaN
+        }
 
 #pragma unroll 1
         for (int blk = 0; blk < NBLK; ++blk) {
@@ -368,7 +391,11 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
 #pragma unroll
                 for (int r = 0; r < TM; ++r)
 #pragma unroll
-                    for (int c = 0; c < TN; ++c) em2[r][c] = uint32_t(acc[r][c].ce) * 0x10001u;
+                    for (int c = 0; c < TN; ++c) {
+                        // ST: compare the products against the accumulator exponent minus the block's scale exponents
+                        const int rel = ST ? acc[r][c].ce - sa_exp[ST ? r : 0] - sb_exp[ST ? c : 0] : acc[r][c].ce;
+                        em2[r][c] = uint32_t(rel) * 0x10001u;
+                    }
 #pragma unroll 4
                 for (int kp = kb / 2; kp < (kb + L) / 2; ++kp) {
                     const uint4 ea0 = *reinterpret_cast<const uint4*>(&s.a_exp2[kp][ty * TM]);
@@ -393,7 +420,8 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
             for (int r = 0; r < TM; ++r)
 #pragma unroll
                 for (int c = 0; c < TN; ++c) {
-                    S0[r][c] = asr_clamp(acc[r][c].cs, emax[r][c] - acc[r][c].ce) - (acc[r][c].cs >> 31);
+                    const int rel = ST ? acc[r][c].ce - sa_exp[ST ? r : 0] - sb_exp[ST ? c : 0] : acc[r][c].ce;
+                    S0[r][c] = asr_clamp(acc[r][c].cs, emax[r][c] - rel) - (acc[r][c].cs >> 31);
                     if (NSUM == 2) S1[NSUM == 2 ? r : 0][NSUM == 2 ? c : 0] = 0;
                     emax[r][c] += guard;
                 }
@@ -454,7 +482,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
                         ovf |= uint32_t((S ^ sum) & (s1 ^ sum));
                         S = sum;
                     }
-                    rho_fast<F, RHO>(S, emax[r][c] - guard, acc[r][c], vmin, vmax);
+                    rho_fast<F, RHO>(S, emax[r][c] - guard + (ST ? sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0] : 0), acc[r][c], vmin, vmax);
                 }
             }
             if (vmin < EMINB || vmax > EMAXB || int(ovf) < 0) {
@@ -469,7 +497,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
                         long long S = (long long)S0[r][c] + nneg;
                         if (NSUM == 2) S += (long long)S1[NSUM == 2 ? r : 0][NSUM == 2 ? c : 0];
                         uint32_t ev = 0u;
-                        rho_slow<F, RHO, ACC16>(S, emax[r][c] - guard - CB, acc[r][c], ev);
+                        rho_slow<F, RHO, ACC16>(S, emax[r][c] - guard - CB + (ST ? sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0] : 0), acc[r][c], ev);
                         if (ev && !MMASIM_SP_GET(r, c)) MMASIM_SP_OR(r, c, ev);   // overflow to infinity (RNE only)
                     }
                 }
@@ -515,21 +543,21 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
 #undef MMASIM_SP_OR
 }
 
-template <int EK, int L, int F, int RHO, bool PROMOTE>
+template <int EK, int L, int F, int RHO, bool PROMOTE, bool ST = false>
 cudaError_t launch_one(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
     const size_t sh = sizeof(Smem<EK>);
-    cudaError_t err = cudaFuncSetAttribute(tfdpa_kernel<EK, L, F, RHO, PROMOTE>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
+    cudaError_t err = cudaFuncSetAttribute(tfdpa_kernel<EK, L, F, RHO, PROMOTE, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
     if (err != cudaSuccess) return err;
     dim3 grid((unsigned)((g.N + BN - 1) / BN), (unsigned)((g.M + BM - 1) / BM), 1);
-    tfdpa_kernel<EK, L, F, RHO, PROMOTE><<<grid, NT, sh, stream>>>(m, g);
+    tfdpa_kernel<EK, L, F, RHO, PROMOTE, ST><<<grid, NT, sh, stream>>>(m, g);
     return cudaGetLastError();
 }
 
 // With or without FP32 promotion (FP32 accumulators only).
-template <int EK, int L, int F, int RHO>
+template <int EK, int L, int F, int RHO, bool ST = false>
 cudaError_t launch_variant(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
-    if (RHO != RHO_RNE_FP16 && g.k_chunk) return launch_one<EK, L, F, RHO, RHO != RHO_RNE_FP16>(m, g, stream);
-    return launch_one<EK, L, F, RHO, false>(m, g, stream);
+    if (RHO != RHO_RNE_FP16 && g.k_chunk) return launch_one<EK, L, F, RHO, RHO != RHO_RNE_FP16, ST>(m, g, stream);
+    return launch_one<EK, L, F, RHO, false, ST>(m, g, stream);
 }
 
 // Per element kind: returns cudaErrorInvalidValue when (L, F, rho) has no instantiation.

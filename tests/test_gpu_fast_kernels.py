@@ -165,3 +165,29 @@ def test_16bit_promotion():
     key = ("hopper", "fp16", "fp32")
     inp = wl.normal_inputs("fp16", "fp32", 130, 66, 256, seed=34)
     _check(key, inp, expect_kernel="tfdpa_f16", k_chunk=64)
+
+
+ST_KEYS = [("blackwell", "mxe4m3", "fp32"), ("blackwell", "mxe5m2", "fp32"), ("rtx_blackwell", "mxe3m2", "fp32"),
+           ("blackwell", "mxe2m3", "fp32"), ("rtx_blackwell", "mxe2m1", "fp32")]
+
+
+@pytest.mark.parametrize("key", ST_KEYS, ids=lambda k: "-".join(k))
+def test_st_fdpa_block_scaled(key):
+    inp = wl.normal_inputs(key[1], key[2], 200, 100, 256, seed=41)
+    _check(key, inp, expect_kernel="tfdpa_lut8")
+    # random element bytes, scale factors over the whole E8M0 range including NaN (0xFF), random accumulators
+    g = wl.rng(42)
+    m = oracle.lookup(*key)
+    bits = 1 + oracle.FORMATS[m.elem].ebits + oracle.FORMATS[m.elem].mbits
+    M, N, K = 150, 70, 128
+    inp = {"A": g.integers(0, 1 << bits, (M, K), dtype=np.uint8), "B": g.integers(0, 1 << bits, (N, K), dtype=np.uint8),
+           "C": g.integers(0, 1 << 32, (M, N), dtype=np.uint32),
+           "sfa": g.integers(0, 256, (M, K // 32), dtype=np.uint8), "sfb": g.integers(0, 256, (N, K // 32), dtype=np.uint8)}
+    _check(key, inp, expect_kernel="tfdpa_lut8")
+    # moderate scales (results in the normal range) with a few NaN scale factors
+    inp["sfa"] = g.integers(100, 150, (M, K // 32), dtype=np.uint8)
+    inp["sfb"] = g.integers(100, 150, (N, K // 32), dtype=np.uint8)
+    inp["sfa"][5, 1] = 255
+    inp["sfb"][9, 3] = 255
+    inp["C"] = g.standard_normal((M, N)).astype(np.float32).view(np.uint32)
+    _check(key, inp, expect_kernel="tfdpa_lut8")
