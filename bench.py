@@ -43,6 +43,10 @@ WORKLOADS = {
                    "FP16 4096^3 N(0,1) inputs; Volta FP16->FP32 model (L=4, F=23, RZ-FP32)"),
     "ampere_bf16": (("ampere", "bf16", "fp32"), (4096, 4096, 4096),
                     "BF16 4096^3 N(0,1) inputs; Ampere BF16->FP32 model (L=8, F=24, RZ-FP32)"),
+    "cfg4_dot_hopper_fp16": (("hopper", "fp16", "fp32"), (1 << 20, 1, 32),
+                             "probe-style batch: 2^20 independent dot products of length 32, FP16, eight seeded input classes (subnormals, cancellation, outliers, inf/NaN, bit streams); Hopper FP16->FP32 model via mmasim_dot_batch"),
+    "cfg4_dot_cdna2_fp16": (("cdna2", "fp16", "fp32"), (1 << 20, 1, 32),
+                            "probe-style batch: 2^20 independent dot products of length 32, FP16, eight seeded input classes; CDNA2 FP16 model (FTZ-AddMul, P=4) via mmasim_dot_batch"),
     "blackwell_e4m3": (("blackwell", "e4m3", "fp32"), (4096, 4096, 4096),
                        "FP8 E4M3 4096^3 N(0,1) inputs; Blackwell FP8->FP32 model (L=32, F=25, RZ-FP32)"),
 }
@@ -67,6 +71,9 @@ def make_inputs(name):
     if name == "cfg2":
         A, B, C = wl.cfg2(M)
         return {"A": A, "B": B, "C": C}
+    if name.startswith("cfg4_dot"):
+        A, B, C = wl.cfg4(key[1], K, n=M)
+        return {"A": A, "B": B, "C": C, "dot": True}
     d = wl.normal_inputs(key[1], key[2], M, N, K, seed=5)
     return {"A": d["A"], "B": d["B"], "C": d["C"]}
 
@@ -207,8 +214,15 @@ def run_ours(args):
     dD = torch.empty((M, N), dtype=torch.int32 if model.acc_bytes == 4 else torch.int16, device=dev)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # larger than the 126 MB L2
 
+    is_dot = bool(inp.get("dot"))
+    if is_dot:
+        dD = torch.empty((M,), dtype=torch.int32, device=dev)
+
     def step():
-        mmasim.gemm(model, dA, dB, dC, out=dD, **kw)
+        if is_dot:
+            mmasim.dot_batch(model, dA, dB, dC, out=dD)
+        else:
+            mmasim.gemm(model, dA, dB, dC, out=dD, **kw)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -256,7 +270,7 @@ def run_ours(args):
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region) ----
     e2e = None
-    if not args.skip_extras and (rank == 0 or world > 1):
+    if not args.skip_extras and not is_dot and (rank == 0 or world > 1):
         def pinned(x):
             x = np.ascontiguousarray(x)
             t = torch.from_numpy(x.view({1: np.uint8, 2: np.int16, 4: np.int32, 8: np.int64}[x.dtype.itemsize]) if x.dtype.kind != "f" else x)
@@ -292,12 +306,28 @@ def run_ours(args):
     per_gpu_macs_s = value / world
     achieved = per_gpu_macs_s * ops_per_mac
     peak = peaks["iadd3"]
-    roofline = {"bound": "alu", "achieved": achieved / 1e12, "peak": peak / 1e12, "unit": "Tint-op/s",
-                "frac": achieved / peak, "traffic": None,
-                "kernel": kernel_name, "algorithmic_int_ops_per_mac": ops_per_mac,
-                "peak_source": "measured live: independent 3-input integer adds on all SMs (mmasim_int_peak kind 0)",
-                "imad_peak": peaks["imad"] / 1e12}
-    cpu_value, cpu_info = (None, {"cores": 0, "sample": "skipped (--skip-extras)"}) if args.skip_extras else oracle_sample_rate(name, inp)
+    if is_dot:
+        esz = inp["A"].dtype.itemsize
+        bytes_per_dot = 2 * K * esz + 8
+        hbm_peak, src = 6650.0, "fallback 6.65 TB/s (MEASURED_PEAKS.json absent)"
+        try:
+            hbm_peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["hbm_gbs"])
+            src = "MEASURED_PEAKS.json hbm_gbs (STREAM-style copy)"
+        except (OSError, KeyError, ValueError):
+            pass
+        gbs = per_gpu_macs_s / K * bytes_per_dot / 1e9
+        roofline = {"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gbs / hbm_peak, "traffic": None,
+                    "kernel": kernel_name, "algorithmic_bytes_per_dot": bytes_per_dot, "peak_source": src}
+    else:
+        roofline = {"bound": "alu", "achieved": achieved / 1e12, "peak": peak / 1e12, "unit": "Tint-op/s",
+                    "frac": achieved / peak, "traffic": None,
+                    "kernel": kernel_name, "algorithmic_int_ops_per_mac": ops_per_mac,
+                    "peak_source": "measured live: independent 3-input integer adds on all SMs (mmasim_int_peak kind 0)",
+                    "imad_peak": peaks["imad"] / 1e12}
+    if args.skip_extras or is_dot:
+        cpu_value, cpu_info = None, {"cores": 0, "sample": "skipped"}
+    else:
+        cpu_value, cpu_info = oracle_sample_rate(name, inp)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

@@ -211,6 +211,7 @@ int mmasim_dot_batch(const mmasim_model* model, int64_t n, int64_t K, const void
     g.lda = g.ldb = K;
     g.ldc = g.ldd = 1;
     g.dot_mode = 1;
+    if (dot_stream_supported(m, g)) return launch_dot_stream(m, g, static_cast<cudaStream_t>(stream));
     set_kernel_name("generic_dot");
     return launch_generic(m, g, static_cast<cudaStream_t>(stream));
 }

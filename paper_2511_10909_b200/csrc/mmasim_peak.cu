@@ -8,7 +8,7 @@ namespace {
 
 enum PeakKind : int {
     PK_IADD3 = 0, PK_LOP3, PK_SHF, PK_IMAD, PK_MACMIX, PK_VIADDMAX, PK_VIADDMAX16X2, PK_F2I, PK_FMUL, PK_POPC,
-    PK_IMAD_PLUS_ALU, PK_FMUL_PLUS_ALU, PK_COUNT
+    PK_IMAD_PLUS_ALU, PK_FMUL_PLUS_ALU, PK_IMAD_WIDE, PK_MAC_D1, PK_MAC_D2, PK_COUNT
 };
 
 template <int KIND>
@@ -31,6 +31,20 @@ __device__ __forceinline__ void round8(int (&x)[8], float (&f)[8]) {
         else if (KIND == PK_POPC) x[i] = __popc(x[i]) + x[j];
         else if (KIND == PK_IMAD_PLUS_ALU) { x[i] = x[i] * x[j] + x[k]; x[j] = x[j] + x[k] + x[i]; }
         else if (KIND == PK_FMUL_PLUS_ALU) { f[i] = f[i] * f[j]; x[i] = x[i] + x[j] + x[k]; }
+        else if (KIND == PK_IMAD_WIDE) {            // 32 x 32 -> 64-bit multiply, both halves consumed
+            const long long w = (long long)x[j] * (long long)x[k];
+            x[i] ^= int(w) ^ int(w >> 32);
+        } else if (KIND == PK_MAC_D1) {             // one emulated term: multiply, distance, shift, accumulate-by-multiply
+            const int X = x[j] * x[k];
+            const int d = x[i] - x[j] - x[k];
+            int t;
+            asm("shr.s32 %0, %1, %2;" : "=r"(t) : "r"(X), "r"(d));
+            asm("mad.lo.s32 %0, %1, %2, %0;" : "+r"(x[i]) : "r"(t), "r"(x[(i + 5) & 7]));
+        } else if (KIND == PK_MAC_D2) {             // one emulated term with pre-shifted operands: wide multiply, funnel shift, accumulate
+            const long long w = (long long)x[j] * (long long)x[k];
+            const int t = __funnelshift_rc(int(w), int(w >> 32), x[(i + 2) & 7]);
+            asm("mad.lo.s32 %0, %1, %2, %0;" : "+r"(x[i]) : "r"(t), "r"(x[(i + 5) & 7]));
+        }
     }
 }
 
@@ -78,6 +92,9 @@ int launch_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t
         case PK_POPC: *ops_per_round = 2; return launch<PK_POPC>(blocks, iters, sink, stream);
         case PK_IMAD_PLUS_ALU: *ops_per_round = 2; return launch<PK_IMAD_PLUS_ALU>(blocks, iters, sink, stream);
         case PK_FMUL_PLUS_ALU: *ops_per_round = 2; return launch<PK_FMUL_PLUS_ALU>(blocks, iters, sink, stream);
+        case PK_IMAD_WIDE: *ops_per_round = 1; return launch<PK_IMAD_WIDE>(blocks, iters, sink, stream);
+        case PK_MAC_D1: *ops_per_round = 1; return launch<PK_MAC_D1>(blocks, iters, sink, stream);
+        case PK_MAC_D2: *ops_per_round = 1; return launch<PK_MAC_D2>(blocks, iters, sink, stream);
         default: set_error("mmasim_int_peak: unknown kind %d", kind); return MMASIM_ERR_INVALID_ARG;
     }
 }
