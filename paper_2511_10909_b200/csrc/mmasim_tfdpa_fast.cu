@@ -7,8 +7,17 @@ namespace {
 
 bool is8(int f) { return f == EF_E4M3 || f == EF_E5M2 || f == EF_E3M2 || f == EF_E2M3 || f == EF_E2M1; }
 
-// 0: no tuned kernel; otherwise 1 + element kind
+constexpr int KIND_TR = 100;
+
+// 0: no tuned kernel; KIND_TR: the TR-/GTR-FDPA kernel; otherwise 1 + element kind of the T-FDPA kernel
 int kind_of(const DevModel& m) {
+    if (m.family == FAM_TR || m.family == FAM_GTR) {
+        if (m.F != 24 || m.F2 != 31 || m.rho != RHO_RNE_FP32 || m.inner_round || m.acc != ACC_F32) return 0;
+        if (m.family == FAM_GTR) return (is8(m.fmt_a) && is8(m.fmt_b) && m.L == 16) ? KIND_TR : 0;
+        if (m.fmt_a != m.fmt_b) return 0;
+        const bool ok = (m.fmt_a == EF_F16 && m.L == 8) || (m.fmt_a == EF_BF16 && m.L == 8) || (m.fmt_a == EF_TF32 && m.L == 4);
+        return ok ? KIND_TR : 0;
+    }
     if ((m.family != FAM_T && m.family != FAM_ST) || m.packed4) return 0;
     if (m.family == FAM_ST) {
         const bool ok = is8(m.fmt_a) && is8(m.fmt_b) && m.F == 25 && m.L == 32 && m.rho == RHO_RZ_FP32 && m.acc == ACC_F32 &&
@@ -47,6 +56,7 @@ bool fast_tfdpa_supported(const DevModel& m, const GemmArgs& g) {
     const int bytes = fmt_desc(m.fmt_a).storage_bits / 8;
     if (g.K % fast::KC) return false;
     if (g.k_chunk % fast::KC) return false;
+    if (kind == KIND_TR && g.k_chunk) return false;
     if (((g.lda * bytes) % 16) || ((g.ldb * bytes) % 16)) return false;      // 16-byte row starts for the vector loads
     if (g.M > 65535ll * fast::BM) return false;
     return true;
@@ -54,7 +64,10 @@ bool fast_tfdpa_supported(const DevModel& m, const GemmArgs& g) {
 
 int launch_fast_tfdpa(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
     cudaError_t err = cudaErrorInvalidValue;
-    switch (kind_of(m) - 1) {
+    if (kind_of(m) == KIND_TR) {
+        set_kernel_name(m.family == FAM_GTR ? "gtrfdpa" : "trfdpa");
+        err = fast::launch_tr(m, g, stream);
+    } else switch (kind_of(m) - 1) {
         case fast::EK_LUT8: set_kernel_name("tfdpa_lut8"); err = fast::launch_lut8(m, g, stream); break;
         case fast::EK_F16: set_kernel_name("tfdpa_f16"); err = fast::launch_f16(m, g, stream); break;
         case fast::EK_BF16: set_kernel_name("tfdpa_bf16"); err = fast::launch_bf16(m, g, stream); break;

@@ -201,6 +201,104 @@ __device__ __forceinline__ void decode_signmag(uint32_t w, uint32_t& sig, uint32
     expb = uint32_t(int((field && !special) ? field : 1u) - E::BIAS + EB);
 }
 
+// Decode tables of the 8-bit kinds: entry `tid` of both (256 threads).
+template <int EK>
+__device__ __forceinline__ void init_lut(Smem<EK>& s, const FmtDesc& fa, const FmtDesc& fb, int pre, int guard, int tid) {
+    constexpr bool SIGNMAG = Elem<EK>::SIGNMAG;
+    if (!SIGNMAG) {
+        const uint32_t da = decode_elem(fa, uint32_t(tid)), db = decode_elem(fb, uint32_t(tid));
+        const bool fin_a = dec_cls(da) == CLS_FINITE, fin_b = dec_cls(db) == CLS_FINITE;
+        LutEntry ea, eb;
+        ea.op = fin_a ? uint32_t(dec_ssig(da)) : 0u;
+        ea.exp = uint32_t((fin_a ? dec_exp(da) : 1 - fa.bias) + EB);
+        ea.bits = fin_a ? (dec_sign(da) | (uint32_t(dec_sig(da) != 0u) << 16)) : 0u;
+        ea.special = fin_a ? 0u : 1u;
+        const int sb = fin_b ? dec_ssig(db) : 0;
+        const int ub = fin_b ? (dec_sign(db) ? -1 : 1) : 0;     // also for b = +-0 (see the header comment)
+        eb.op = uint32_t(sb * (1 << (pre + guard)) + ub);
+        eb.exp = uint32_t((fin_b ? dec_exp(db) : 1 - fb.bias) + EB);
+        eb.bits = fin_b ? dec_sign(db) : 0u;
+        eb.special = fin_b ? 0u : 1u;
+        s.lut_a[tid] = ea;
+        s.lut_b[tid] = eb;
+    }
+}
+
+// Stage one chunk of KC elements of K: every task decodes E::TASK consecutive elements of one row of A or B into
+// operand / exponent (/ sign mask) words, k-major in shared memory, plus the row's sign and nonzero bit masks.
+template <int EK>
+__device__ __forceinline__ void stage_chunk(Smem<EK>& s, const GemmArgs& g, int64_t row0, int64_t col0, int64_t k0,
+                                            int chunk, int pre, int tid) {
+    using E = Elem<EK>;
+    constexpr bool SIGNMAG = E::SIGNMAG;
+    {
+        constexpr int TPR = KC / E::TASK;                  // tasks per row
+        uint32_t spec = 0u;
+#pragma unroll
+        for (int t0 = 0; t0 < (BM + BN) * TPR; t0 += NT) {
+            const int task = t0 + tid;
+            const bool is_a = task < BM * TPR;
+            if (task >= (BM + BN) * TPR) break;
+            const int u = is_a ? task : task - BM * TPR;
+            const int rows = is_a ? BM : BN;
+            const int r = u % rows, h = u / rows;          // consecutive threads take consecutive rows
+            const int64_t grow = (is_a ? row0 : col0) + r;
+            const bool valid = grow < (is_a ? g.M : g.N);
+            const unsigned char* base = static_cast<const unsigned char*>(is_a ? g.A : g.B) +
+                                        (grow * (is_a ? g.lda : g.ldb) + k0 + h * E::TASK) * E::BYTES;
+            uint32_t wv[E::TASK * E::BYTES / 4];
+#pragma unroll
+            for (int q = 0; q < E::TASK * E::BYTES / 16; ++q) {
+                uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+                if (valid) raw = reinterpret_cast<const uint4*>(base)[q];
+                wv[4 * q] = raw.x; wv[4 * q + 1] = raw.y; wv[4 * q + 2] = raw.z; wv[4 * q + 3] = raw.w;
+            }
+            uint32_t bits = 0u, prev_exp = 0u;
+#pragma unroll
+            for (int q = 0; q < E::TASK; ++q) {
+                const int kk = h * E::TASK + q;
+                uint32_t op, expb;
+                if (!SIGNMAG) {
+                    const uint32_t byte = (wv[q / 4] >> (8 * (q % 4))) & 0xFFu;
+                    const LutEntry e = is_a ? s.lut_a[byte] : s.lut_b[byte];
+                    op = e.op;
+                    expb = e.exp;
+                    bits += e.bits << q;
+                    spec |= e.special;
+                } else {
+                    const uint32_t w = E::BYTES == 2 ? ((wv[q / 2] >> (16 * (q % 2))) & 0xFFFFu) : wv[q];
+                    uint32_t sig, sign, special;
+                    decode_signmag<EK>(w, sig, expb, sign, special);
+                    op = is_a ? sig : (sig << pre);
+                    bits += sign << q;
+                    spec |= special;
+                    if (is_a) s.a_msk[SIGNMAG ? kk : 0][r] = 0u - sign; else s.b_msk[SIGNMAG ? kk : 0][r] = 0u - sign;
+                }
+                if (is_a) { s.a_op[kk][r] = op; s.a_exp[kk][r] = expb; }
+                else { s.b_op[kk][r] = op; s.b_exp[kk][r] = expb; }
+                if (q & 1) {
+                    const uint32_t pair = prev_exp | (expb << 16);
+                    if (is_a) s.a_exp2[kk / 2][r] = pair; else s.b_exp2[kk / 2][r] = pair;
+                }
+                prev_exp = expb;
+            }
+            // sign (and nonzero) bits of the task's elements go to bits [h * TASK, h * TASK + TASK) of the row's masks
+            if (E::TASK == 16) {
+                if (is_a) {
+                    reinterpret_cast<uint16_t*>(&s.a_sgn[r])[h] = uint16_t(bits);
+                    reinterpret_cast<uint16_t*>(&s.a_nz[r])[h] = uint16_t(bits >> 16);
+                } else {
+                    reinterpret_cast<uint16_t*>(&s.b_sgn[r])[h] = uint16_t(bits);
+                }
+            } else {
+                if (is_a) reinterpret_cast<uint8_t*>(&s.a_sgn[r])[h] = uint8_t(bits);
+                else reinterpret_cast<uint8_t*>(&s.b_sgn[r])[h] = uint8_t(bits);
+            }
+        }
+        if (spec) atomicOr(&s.special[chunk & 1], 1);
+    }
+}
+
 template <int EK, int L, int F, int RHO, bool PROMOTE, bool ST = false>
 __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
     using E = Elem<EK>;
@@ -223,23 +321,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
     const int guard = SIGNMAG ? 0 : fa.mbits + 1;   // guard bits below the truncation point (8-bit kinds)
     const int one = int(blockDim.x >> 8);           // 1, but not a compile-time constant (see mad_one)
 
-    if (!SIGNMAG) {                                 // decode tables: entry `tid` of both
-        const uint32_t da = decode_elem(fa, uint32_t(tid)), db = decode_elem(fb, uint32_t(tid));
-        const bool fin_a = dec_cls(da) == CLS_FINITE, fin_b = dec_cls(db) == CLS_FINITE;
-        LutEntry ea, eb;
-        ea.op = fin_a ? uint32_t(dec_ssig(da)) : 0u;
-        ea.exp = uint32_t((fin_a ? dec_exp(da) : 1 - fa.bias) + EB);
-        ea.bits = fin_a ? (dec_sign(da) | (uint32_t(dec_sig(da) != 0u) << 16)) : 0u;
-        ea.special = fin_a ? 0u : 1u;
-        const int sb = fin_b ? dec_ssig(db) : 0;
-        const int ub = fin_b ? (dec_sign(db) ? -1 : 1) : 0;     // also for b = +-0 (see the header comment)
-        eb.op = uint32_t(sb * (1 << (pre + guard)) + ub);
-        eb.exp = uint32_t((fin_b ? dec_exp(db) : 1 - fb.bias) + EB);
-        eb.bits = fin_b ? dec_sign(db) : 0u;
-        eb.special = fin_b ? 0u : 1u;
-        s.lut_a[tid] = ea;
-        s.lut_b[tid] = eb;
-    }
+    init_lut<EK>(s, fa, fb, pre, guard, tid);
     if (tid == 0) s.special[0] = s.special[1] = 0;
 
     Acc acc[TM][TN];
@@ -265,73 +347,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
     int chunk = 0;
     for (int64_t k0 = 0; k0 < g.K; k0 += KC, ++chunk) {
         __syncthreads();
-        // ---- stage the chunk: each task decodes E::TASK consecutive elements of one row ----
-        {
-            constexpr int TPR = KC / E::TASK;                  // tasks per row
-            uint32_t spec = 0u;
-#pragma unroll
-            for (int t0 = 0; t0 < (BM + BN) * TPR; t0 += NT) {
-                const int task = t0 + tid;
-                const bool is_a = task < BM * TPR;
-                if (task >= (BM + BN) * TPR) break;
-                const int u = is_a ? task : task - BM * TPR;
-                const int rows = is_a ? BM : BN;
-                const int r = u % rows, h = u / rows;          // consecutive threads take consecutive rows
-                const int64_t grow = (is_a ? row0 : col0) + r;
-                const bool valid = grow < (is_a ? g.M : g.N);
-                const unsigned char* base = static_cast<const unsigned char*>(is_a ? g.A : g.B) +
-                                            (grow * (is_a ? g.lda : g.ldb) + k0 + h * E::TASK) * E::BYTES;
-                uint32_t wv[E::TASK * E::BYTES / 4];
-#pragma unroll
-                for (int q = 0; q < E::TASK * E::BYTES / 16; ++q) {
-                    uint4 raw = make_uint4(0u, 0u, 0u, 0u);
-                    if (valid) raw = reinterpret_cast<const uint4*>(base)[q];
-                    wv[4 * q] = raw.x; wv[4 * q + 1] = raw.y; wv[4 * q + 2] = raw.z; wv[4 * q + 3] = raw.w;
-                }
-                uint32_t bits = 0u, prev_exp = 0u;
-#pragma unroll
-                for (int q = 0; q < E::TASK; ++q) {
-                    const int kk = h * E::TASK + q;
-                    uint32_t op, expb;
-                    if (!SIGNMAG) {
-                        const uint32_t byte = (wv[q / 4] >> (8 * (q % 4))) & 0xFFu;
-                        const LutEntry e = is_a ? s.lut_a[byte] : s.lut_b[byte];
-                        op = e.op;
-                        expb = e.exp;
-                        bits += e.bits << q;
-                        spec |= e.special;
-                    } else {
-                        const uint32_t w = E::BYTES == 2 ? ((wv[q / 2] >> (16 * (q % 2))) & 0xFFFFu) : wv[q];
-                        uint32_t sig, sign, special;
-                        decode_signmag<EK>(w, sig, expb, sign, special);
-                        op = is_a ? sig : (sig << pre);
-                        bits += sign << q;
-                        spec |= special;
-                        if (is_a) s.a_msk[SIGNMAG ? kk : 0][r] = 0u - sign; else s.b_msk[SIGNMAG ? kk : 0][r] = 0u - sign;
-                    }
-                    if (is_a) { s.a_op[kk][r] = op; s.a_exp[kk][r] = expb; }
-                    else { s.b_op[kk][r] = op; s.b_exp[kk][r] = expb; }
-                    if (q & 1) {
-                        const uint32_t pair = prev_exp | (expb << 16);
-                        if (is_a) s.a_exp2[kk / 2][r] = pair; else s.b_exp2[kk / 2][r] = pair;
-                    }
-                    prev_exp = expb;
-                }
-                // sign (and nonzero) bits of the task's elements go to bits [h * TASK, h * TASK + TASK) of the row's masks
-                if (E::TASK == 16) {
-                    if (is_a) {
-                        reinterpret_cast<uint16_t*>(&s.a_sgn[r])[h] = uint16_t(bits);
-                        reinterpret_cast<uint16_t*>(&s.a_nz[r])[h] = uint16_t(bits >> 16);
-                    } else {
-                        reinterpret_cast<uint16_t*>(&s.b_sgn[r])[h] = uint16_t(bits);
-                    }
-                } else {
-                    if (is_a) reinterpret_cast<uint8_t*>(&s.a_sgn[r])[h] = uint8_t(bits);
-                    else reinterpret_cast<uint8_t*>(&s.b_sgn[r])[h] = uint8_t(bits);
-                }
-            }
-            if (spec) atomicOr(&s.special[chunk & 1], 1);
-        }
+        stage_chunk<EK>(s, g, row0, col0, k0, chunk, pre, tid);
         __syncthreads();
 
         if (tid == 0) s.special[(chunk + 1) & 1] = 0;
@@ -565,6 +581,7 @@ cudaError_t launch_lut8(const DevModel& m, const GemmArgs& g, cudaStream_t strea
 cudaError_t launch_f16(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
 cudaError_t launch_bf16(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
 cudaError_t launch_tf32(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
+cudaError_t launch_tr(const DevModel& m, const GemmArgs& g, cudaStream_t stream);    // TR-/GTR-FDPA (mmasim_trfdpa_fast.cu)
 
 }  // namespace fast
 }  // namespace mmasim

@@ -191,3 +191,72 @@ def test_st_fdpa_block_scaled(key):
     inp["sfb"][9, 3] = 255
     inp["C"] = g.standard_normal((M, N)).astype(np.float32).view(np.uint32)
     _check(key, inp, expect_kernel="tfdpa_lut8")
+
+
+TR_KEYS = [("cdna3", "fp16", "fp32"), ("cdna3", "bf16", "fp32"), ("cdna3", "tf32", "fp32"), ("cdna3", "e4m3", "fp32"),
+           ("cdna3", "e5m2", "fp32")]
+
+
+def _tr_kernel(key):
+    return "gtrfdpa" if key[1] in ("e4m3", "e5m2") else "trfdpa"
+
+
+@pytest.mark.parametrize("key", TR_KEYS, ids=lambda k: "-".join(k))
+def test_tr_gtr_normal_inputs_and_bias_case(key):
+    inp = wl.normal_inputs(key[1], key[2], 200, 100, 256, seed=51)
+    _check(key, inp, expect_kernel=_tr_kernel(key))
+    # the regime of the paper's bias experiment (Section 6.2.4): large A, B and a small accumulator of either sign
+    g = wl.rng(52)
+    scale = 1000.0 if key[1] not in ("e4m3", "e5m2") else 16.0
+    A = wl.cast(g.standard_normal((130, 128)).astype(np.float32) * scale, key[1])
+    B = wl.cast(g.standard_normal((70, 128)).astype(np.float32) * scale, key[1])
+    C = g.standard_normal((130, 70)).astype(np.float32).view(np.uint32)
+    _check(key, {"A": A, "B": B, "C": C}, expect_kernel=_tr_kernel(key))
+
+
+@pytest.mark.parametrize("key", TR_KEYS, ids=lambda k: "-".join(k))
+def test_tr_gtr_random_bit_stream(key):
+    g = wl.rng(53)
+    M, N, K = 150, 70, 128
+    m = oracle.lookup(*key)
+    if key[1] in ("e4m3", "e5m2"):
+        A = g.integers(0, 256, (M, K), dtype=np.uint8)
+        B = g.integers(0, 256, (N, K), dtype=np.uint8)
+    else:
+        wbits = 32 if key[1] == "tf32" else 16
+        dt = np.uint32 if wbits == 32 else np.uint16
+        A = g.integers(0, 1 << wbits, (M, K), dtype=np.uint64).astype(dt)
+        B = g.integers(0, 1 << wbits, (N, K), dtype=np.uint64).astype(dt)
+    C = g.integers(0, 1 << 32, (M, N), dtype=np.uint32)
+    _check(key, {"A": A, "B": B, "C": C}, expect_kernel=_tr_kernel(key))
+    # products near 2^128 (overflow to infinity) and accumulators at both ends of the exponent range
+    if key[1] in ("bf16", "tf32"):
+        low = 13 if key[1] == "tf32" else 0
+        dt = np.uint32 if key[1] == "tf32" else np.uint16
+        mb = 10 if key[1] == "tf32" else 7
+        def mat(rows):
+            sign = g.integers(0, 2, (rows, K), dtype=np.uint64)
+            exp = g.choice([1, 60, 127, 186, 190, 191, 192, 254], (rows, K)).astype(np.uint64)
+            man = g.integers(0, 1 << mb, (rows, K), dtype=np.uint64)
+            return ((((sign << 8) | exp) << mb | man) << low).astype(dt)
+        C = ((g.integers(0, 2, (M, N)) << 31) | (g.choice([0, 1, 2, 127, 253, 254], (M, N)) << 23) | g.integers(0, 1 << 23, (M, N))).astype(np.uint32)
+        _check(key, {"A": mat(M), "B": mat(N), "C": C}, expect_kernel=_tr_kernel(key))
+
+
+@pytest.mark.parametrize("key", TR_KEYS, ids=lambda k: "-".join(k))
+def test_tr_gtr_config4_classes_as_gemm(key):
+    m = oracle.lookup(*key)
+    if key[1] in ("e4m3", "e5m2"):
+        g = wl.rng(54)
+        A = g.integers(0, 256, (192, 128), dtype=np.uint8)
+        A[:, 1::2] = A[:, 0::2] ^ 0x80                       # neighbouring terms cancel: the even / odd groups matter
+        B = g.integers(0, 256, (96, 128), dtype=np.uint8)
+        B[:, 1::2] = B[:, 0::2]
+        C = g.standard_normal((192, 96)).astype(np.float32).view(np.uint32)
+    else:
+        A, B, C = wl.cfg4(m.elem, 32, n=1 << 12)
+        A, B = A[:192].reshape(192, 32), B[192:192 + 96].reshape(96, 32)
+        A = np.ascontiguousarray(np.tile(A, (1, 4)))
+        B = np.ascontiguousarray(np.tile(B, (1, 4)))
+        C = np.resize(C, (192, 96)).copy()
+    _check(key, {"A": A, "B": B, "C": C}, expect_kernel=_tr_kernel(key))
