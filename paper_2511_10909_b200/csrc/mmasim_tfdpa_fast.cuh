@@ -224,79 +224,109 @@ __device__ __forceinline__ void init_lut(Smem<EK>& s, const FmtDesc& fa, const F
     }
 }
 
-// Stage one chunk of KC elements of K: every task decodes E::TASK consecutive elements of one row of A or B into
-// operand / exponent (/ sign mask) words, k-major in shared memory, plus the row's sign and nonzero bit masks.
+// Staging of one chunk of KC elements of K, in two steps so that the global loads of the next chunk can be in flight
+// while the current one is being computed: (1) every task loads E::TASK consecutive raw elements of one row of A or B
+// into registers, (2) it decodes them into operand / exponent (/ sign mask) words, k-major in shared memory, plus the
+// row's sign and nonzero bit masks.
+template <int EK>
+struct RawChunk {
+    static constexpr int TPR = KC / Elem<EK>::TASK;                              // tasks per row
+    static constexpr int TASKS = (BM + BN) * TPR;
+    static constexpr int PER_THREAD = (TASKS + NT - 1) / NT;
+    static constexpr int WORDS = Elem<EK>::TASK * Elem<EK>::BYTES / 4;           // 32-bit words per task
+    uint32_t w[PER_THREAD][WORDS];
+};
+
+template <int EK>
+__device__ __forceinline__ void load_chunk(RawChunk<EK>& raw, const GemmArgs& g, int64_t row0, int64_t col0, int64_t k0, int tid) {
+    using E = Elem<EK>;
+    using R = RawChunk<EK>;
+#pragma unroll
+    for (int it = 0; it < R::PER_THREAD; ++it) {
+        const int task = it * NT + tid;
+        const bool is_a = task < BM * R::TPR;
+        const int u = is_a ? task : task - BM * R::TPR;
+        const int rows = is_a ? BM : BN;
+        const int r = u % rows, h = u / rows;              // consecutive threads take consecutive rows
+        const int64_t grow = (is_a ? row0 : col0) + r;
+        const bool valid = task < R::TASKS && grow < (is_a ? g.M : g.N);
+        const unsigned char* base = static_cast<const unsigned char*>(is_a ? g.A : g.B) +
+                                    (grow * (is_a ? g.lda : g.ldb) + k0 + h * E::TASK) * E::BYTES;
+#pragma unroll
+        for (int q = 0; q < R::WORDS / 4; ++q) {
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (valid) v = reinterpret_cast<const uint4*>(base)[q];
+            raw.w[it][4 * q] = v.x; raw.w[it][4 * q + 1] = v.y; raw.w[it][4 * q + 2] = v.z; raw.w[it][4 * q + 3] = v.w;
+        }
+    }
+}
+
+template <int EK>
+__device__ __forceinline__ void store_chunk(Smem<EK>& s, const RawChunk<EK>& raw, int chunk, int pre, int tid) {
+    using E = Elem<EK>;
+    using R = RawChunk<EK>;
+    constexpr bool SIGNMAG = E::SIGNMAG;
+    uint32_t spec = 0u;
+#pragma unroll
+    for (int it = 0; it < R::PER_THREAD; ++it) {
+        const int task = it * NT + tid;
+        if (task >= R::TASKS) break;
+        const bool is_a = task < BM * R::TPR;
+        const int u = is_a ? task : task - BM * R::TPR;
+        const int rows = is_a ? BM : BN;
+        const int r = u % rows, h = u / rows;
+        uint32_t bits = 0u, prev_exp = 0u;
+#pragma unroll
+        for (int q = 0; q < E::TASK; ++q) {
+            const int kk = h * E::TASK + q;
+            uint32_t op, expb;
+            if (!SIGNMAG) {
+                const uint32_t byte = (raw.w[it][q / 4] >> (8 * (q % 4))) & 0xFFu;
+                const LutEntry e = is_a ? s.lut_a[byte] : s.lut_b[byte];
+                op = e.op;
+                expb = e.exp;
+                bits += e.bits << q;
+                spec |= e.special;
+            } else {
+                const uint32_t w = E::BYTES == 2 ? ((raw.w[it][q / 2] >> (16 * (q % 2))) & 0xFFFFu) : raw.w[it][q];
+                uint32_t sig, sign, special;
+                decode_signmag<EK>(w, sig, expb, sign, special);
+                op = is_a ? sig : (sig << pre);
+                bits += sign << q;
+                spec |= special;
+                if (is_a) s.a_msk[SIGNMAG ? kk : 0][r] = 0u - sign; else s.b_msk[SIGNMAG ? kk : 0][r] = 0u - sign;
+            }
+            if (is_a) { s.a_op[kk][r] = op; s.a_exp[kk][r] = expb; }
+            else { s.b_op[kk][r] = op; s.b_exp[kk][r] = expb; }
+            if (q & 1) {
+                const uint32_t pair = prev_exp | (expb << 16);
+                if (is_a) s.a_exp2[kk / 2][r] = pair; else s.b_exp2[kk / 2][r] = pair;
+            }
+            prev_exp = expb;
+        }
+        // sign (and nonzero) bits of the task's elements go to bits [h * TASK, h * TASK + TASK) of the row's masks
+        if (E::TASK == 16) {
+            if (is_a) {
+                reinterpret_cast<uint16_t*>(&s.a_sgn[r])[h] = uint16_t(bits);
+                reinterpret_cast<uint16_t*>(&s.a_nz[r])[h] = uint16_t(bits >> 16);
+            } else {
+                reinterpret_cast<uint16_t*>(&s.b_sgn[r])[h] = uint16_t(bits);
+            }
+        } else {
+            if (is_a) reinterpret_cast<uint8_t*>(&s.a_sgn[r])[h] = uint8_t(bits);
+            else reinterpret_cast<uint8_t*>(&s.b_sgn[r])[h] = uint8_t(bits);
+        }
+    }
+    if (spec) atomicOr(&s.special[chunk & 1], 1);
+}
+
+// Load and stage in one go (no prefetch).
 template <int EK>
 __device__ __forceinline__ void stage_chunk(Smem<EK>& s, const GemmArgs& g, int64_t row0, int64_t col0, int64_t k0,
                                             int chunk, int pre, int tid) {
-    using E = Elem<EK>;
-    constexpr bool SIGNMAG = E::SIGNMAG;
-    {
-        constexpr int TPR = KC / E::TASK;                  // tasks per row
-        uint32_t spec = 0u;
-#pragma unroll
-        for (int t0 = 0; t0 < (BM + BN) * TPR; t0 += NT) {
-            const int task = t0 + tid;
-            const bool is_a = task < BM * TPR;
-            if (task >= (BM + BN) * TPR) break;
-            const int u = is_a ? task : task - BM * TPR;
-            const int rows = is_a ? BM : BN;
-            const int r = u % rows, h = u / rows;          // consecutive threads take consecutive rows
-            const int64_t grow = (is_a ? row0 : col0) + r;
-            const bool valid = grow < (is_a ? g.M : g.N);
-            const unsigned char* base = static_cast<const unsigned char*>(is_a ? g.A : g.B) +
-                                        (grow * (is_a ? g.lda : g.ldb) + k0 + h * E::TASK) * E::BYTES;
-            uint32_t wv[E::TASK * E::BYTES / 4];
-#pragma unroll
-            for (int q = 0; q < E::TASK * E::BYTES / 16; ++q) {
-                uint4 raw = make_uint4(0u, 0u, 0u, 0u);
-                if (valid) raw = reinterpret_cast<const uint4*>(base)[q];
-                wv[4 * q] = raw.x; wv[4 * q + 1] = raw.y; wv[4 * q + 2] = raw.z; wv[4 * q + 3] = raw.w;
-            }
-            uint32_t bits = 0u, prev_exp = 0u;
-#pragma unroll
-            for (int q = 0; q < E::TASK; ++q) {
-                const int kk = h * E::TASK + q;
-                uint32_t op, expb;
-                if (!SIGNMAG) {
-                    const uint32_t byte = (wv[q / 4] >> (8 * (q % 4))) & 0xFFu;
-                    const LutEntry e = is_a ? s.lut_a[byte] : s.lut_b[byte];
-                    op = e.op;
-                    expb = e.exp;
-                    bits += e.bits << q;
-                    spec |= e.special;
-                } else {
-                    const uint32_t w = E::BYTES == 2 ? ((wv[q / 2] >> (16 * (q % 2))) & 0xFFFFu) : wv[q];
-                    uint32_t sig, sign, special;
-                    decode_signmag<EK>(w, sig, expb, sign, special);
-                    op = is_a ? sig : (sig << pre);
-                    bits += sign << q;
-                    spec |= special;
-                    if (is_a) s.a_msk[SIGNMAG ? kk : 0][r] = 0u - sign; else s.b_msk[SIGNMAG ? kk : 0][r] = 0u - sign;
-                }
-                if (is_a) { s.a_op[kk][r] = op; s.a_exp[kk][r] = expb; }
-                else { s.b_op[kk][r] = op; s.b_exp[kk][r] = expb; }
-                if (q & 1) {
-                    const uint32_t pair = prev_exp | (expb << 16);
-                    if (is_a) s.a_exp2[kk / 2][r] = pair; else s.b_exp2[kk / 2][r] = pair;
-                }
-                prev_exp = expb;
-            }
-            // sign (and nonzero) bits of the task's elements go to bits [h * TASK, h * TASK + TASK) of the row's masks
-            if (E::TASK == 16) {
-                if (is_a) {
-                    reinterpret_cast<uint16_t*>(&s.a_sgn[r])[h] = uint16_t(bits);
-                    reinterpret_cast<uint16_t*>(&s.a_nz[r])[h] = uint16_t(bits >> 16);
-                } else {
-                    reinterpret_cast<uint16_t*>(&s.b_sgn[r])[h] = uint16_t(bits);
-                }
-            } else {
-                if (is_a) reinterpret_cast<uint8_t*>(&s.a_sgn[r])[h] = uint8_t(bits);
-                else reinterpret_cast<uint8_t*>(&s.b_sgn[r])[h] = uint8_t(bits);
-            }
-        }
-        if (spec) atomicOr(&s.special[chunk & 1], 1);
-    }
+    RawChunk<EK> raw;
+    load_chunk<EK>(raw, g, row0, col0, k0, tid);
+    store_chunk<EK>(s, raw, chunk, pre, tid);
 }
 
 template <int EK, int L, int F, int RHO, bool PROMOTE, bool ST = false>
@@ -344,11 +374,18 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
             MMASIM_SP_OR(r, c, ev);
         }
 
+    // The raw words of the next chunk wait in registers during the compute where the register budget allows it
+    // (the narrow-sum 8-bit variants); elsewhere the extra live registers cost more in spills than the overlap gains.
+    constexpr bool PREFETCH = EK == EK_LUT8 && NSUM == 1;
+    RawChunk<EK> raw;
+    if (PREFETCH) load_chunk<EK>(raw, g, row0, col0, 0, tid);
     int chunk = 0;
     for (int64_t k0 = 0; k0 < g.K; k0 += KC, ++chunk) {
         __syncthreads();
-        stage_chunk<EK>(s, g, row0, col0, k0, chunk, pre, tid);
+        if (!PREFETCH) load_chunk<EK>(raw, g, row0, col0, k0, tid);
+        store_chunk<EK>(s, raw, chunk, pre, tid);
         __syncthreads();
+        if (PREFETCH && k0 + KC < g.K) load_chunk<EK>(raw, g, row0, col0, k0 + KC, tid);
 
         if (tid == 0) s.special[(chunk + 1) & 1] = 0;
         bool chunk_special = s.special[chunk & 1] != 0;
