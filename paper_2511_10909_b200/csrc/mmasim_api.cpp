@@ -58,8 +58,9 @@ int check_k(const DevModel& m, int64_t K) {
 
 int run_gemm(const mmasim_model* model, const GemmArgs& g, int flags, cudaStream_t stream) {
     const DevModel& m = model->dev;
-    if (!(flags & MMASIM_GEMM_FORCE_GENERIC) && fast_tfdpa_supported(m, g)) {
-        return launch_fast_tfdpa(m, g, stream);
+    if (!(flags & MMASIM_GEMM_FORCE_GENERIC)) {
+        if (fast_tfdpa_supported(m, g)) return launch_fast_tfdpa(m, g, stream);
+        if (fast_fp_supported(m, g)) return launch_fast_fp(m, g, stream);
     }
     set_kernel_name("generic");
     return launch_generic(m, g, stream);

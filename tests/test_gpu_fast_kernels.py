@@ -260,3 +260,39 @@ def test_tr_gtr_config4_classes_as_gemm(key):
         B = np.ascontiguousarray(np.tile(B, (1, 4)))
         C = np.resize(C, (192, 96)).copy()
     _check(key, {"A": A, "B": B, "C": C}, expect_kernel=_tr_kernel(key))
+
+
+FP_KEYS = [("cdna3", "fp32", "fp32"), ("cdna1", "fp32", "fp32"), ("hopper", "fp64", "fp64"), ("cdna2", "fp64", "fp64"),
+           ("cdna2", "fp16", "fp32"), ("cdna2", "bf16", "fp32"), ("cdna2", "bf16_1k", "fp32")]
+FP_KERNEL = {"fp32": "fma_f32", "fp64": "fma_f64", "fp16": "ftz_addmul", "bf16": "ftz_addmul", "bf16_1k": "ftz_addmul"}
+
+
+@pytest.mark.parametrize("key", FP_KEYS, ids=lambda k: "-".join(k))
+def test_fp_pipe_models(key):
+    inp = wl.normal_inputs(key[1], key[2], 200, 100, 128, seed=61)
+    _check(key, inp, nsample=300, expect_kernel=FP_KERNEL[key[1]])
+    # random bit streams: NaN, infinities, subnormals, huge exponent spread
+    g = wl.rng(62)
+    m = oracle.lookup(*key)
+    wbits = oracle.FORMATS[m.elem].storage_bits
+    M, N, K = 100, 70, 64
+    A = g.integers(0, 1 << 63, (M, K), dtype=np.uint64).astype(wl.word_dtype(m.elem)) if wbits < 64 else g.integers(0, 1 << 63, (M, K), dtype=np.uint64) * 2 + g.integers(0, 2, (M, K), dtype=np.uint64)
+    B = g.integers(0, 1 << 63, (N, K), dtype=np.uint64).astype(wl.word_dtype(m.elem)) if wbits < 64 else g.integers(0, 1 << 63, (N, K), dtype=np.uint64) * 2 + g.integers(0, 2, (N, K), dtype=np.uint64)
+    cbits = 64 if key[2] == "fp64" else 32
+    C = (g.integers(0, 1 << 63, (M, N), dtype=np.uint64) * 2).astype(np.uint64 if cbits == 64 else np.uint32)
+    _check(key, {"A": A, "B": B, "C": C}, nsample=300, expect_kernel=FP_KERNEL[key[1]])
+
+
+@pytest.mark.parametrize("key", [("cdna2", "fp16", "fp32"), ("cdna2", "bf16", "fp32"), ("cdna2", "bf16_1k", "fp32")], ids=lambda k: "-".join(k))
+def test_ftz_flush_boundary(key):
+    # operands whose products and sums sit around 2^-126: the hardware flush mode must agree with "round, then flush"
+    g = wl.rng(63)
+    M, N, K = 128, 64, 64
+    if key[1] == "fp16":
+        A = ((g.integers(0, 2, (M, K)) << 15) | (g.integers(0, 4, (M, K)) << 10) | g.integers(0, 1024, (M, K))).astype(np.uint16)
+        B = ((g.integers(0, 2, (N, K)) << 15) | (g.integers(0, 4, (N, K)) << 10) | g.integers(0, 1024, (N, K))).astype(np.uint16)
+    else:
+        A = ((g.integers(0, 2, (M, K)) << 15) | (g.integers(0, 70, (M, K)) << 7) | g.integers(0, 128, (M, K))).astype(np.uint16)
+        B = ((g.integers(0, 2, (N, K)) << 15) | (g.integers(58, 130, (N, K)) << 7) | g.integers(0, 128, (N, K))).astype(np.uint16)
+    C = ((g.integers(0, 2, (M, N)) << 31) | (g.integers(0, 4, (M, N)) << 23) | g.integers(0, 1 << 23, (M, N))).astype(np.uint32)
+    _check(key, {"A": A, "B": B, "C": C}, nsample=400, expect_kernel="ftz_addmul")
