@@ -61,6 +61,7 @@ int run_gemm(const mmasim_model* model, const GemmArgs& g, int flags, cudaStream
     if (!(flags & MMASIM_GEMM_FORCE_GENERIC)) {
         if (fast_tfdpa_supported(m, g)) return launch_fast_tfdpa(m, g, stream);
         if (fast_fp_supported(m, g)) return launch_fast_fp(m, g, stream);
+        if (fast_gst_supported(m, g)) return launch_fast_gst(m, g, stream);
     }
     set_kernel_name("generic");
     return launch_generic(m, g, stream);

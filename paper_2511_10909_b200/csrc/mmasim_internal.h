@@ -88,6 +88,9 @@ int launch_fast_tfdpa(const DevModel& m, const GemmArgs& g, cudaStream_t stream)
 // mmasim_fp_fast.cu
 bool fast_fp_supported(const DevModel& m, const GemmArgs& g);
 int launch_fast_fp(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
+// mmasim_gst_fast.cu
+bool fast_gst_supported(const DevModel& m, const GemmArgs& g);
+int launch_fast_gst(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
 // mmasim_dot_stream.cu
 bool dot_stream_supported(const DevModel& m, const GemmArgs& g);
 int launch_dot_stream(const DevModel& m, const GemmArgs& g, cudaStream_t stream);

@@ -231,7 +231,7 @@ def gemm_host(model: Model, A, B, C=None, *, K=None, sfa=None, sfb=None, k_chunk
 
 
 PEAK_KINDS = ["iadd3", "lop3", "shf", "imad", "macmix", "viaddmax", "viaddmax16x2", "f2i", "fmul", "popc",
-              "imad+alu", "fmul+alu", "imad.wide", "mac_d1", "mac_d2"]
+              "imad+alu", "fmul+alu", "imad.wide", "mac_d1", "mac_d2", "dp4a", "dfma"]
 
 
 def int_peak(kind: str, blocks: int, iters: int, sink, stream=None) -> int:

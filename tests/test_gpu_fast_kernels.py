@@ -296,3 +296,28 @@ def test_ftz_flush_boundary(key):
         B = ((g.integers(0, 2, (N, K)) << 15) | (g.integers(58, 130, (N, K)) << 7) | g.integers(0, 128, (N, K))).astype(np.uint16)
     C = ((g.integers(0, 2, (M, N)) << 31) | (g.integers(0, 4, (M, N)) << 23) | g.integers(0, 1 << 23, (M, N))).astype(np.uint32)
     _check(key, {"A": A, "B": B, "C": C}, nsample=400, expect_kernel="ftz_addmul")
+
+
+GST_KEYS = [("blackwell", "mxf4", "fp32"), ("blackwell", "nvf4", "fp32"), ("rtx_blackwell", "nvf4", "fp32")]
+
+
+@pytest.mark.parametrize("key", GST_KEYS, ids=lambda k: "-".join(k))
+def test_gst_fdpa_group_scaled(key):
+    inp = wl.normal_inputs(key[1], key[2], 200, 100, 256, seed=71)
+    _check(key, inp, expect_kernel="gstfdpa")
+    # random nibbles, scale factors over the whole code range (zero, subnormal, NaN scales), random accumulators
+    g = wl.rng(72)
+    M, N, K = 150, 70, 192
+    kb = 16 if key[1] == "nvf4" else 32
+    inp = {"A": g.integers(0, 256, (M, K // 2), dtype=np.uint8), "B": g.integers(0, 256, (N, K // 2), dtype=np.uint8),
+           "C": g.integers(0, 1 << 32, (M, N), dtype=np.uint32),
+           "sfa": g.integers(0, 256, (M, K // kb), dtype=np.uint8), "sfb": g.integers(0, 256, (N, K // kb), dtype=np.uint8)}
+    _check(key, inp, expect_kernel="gstfdpa")
+    # moderate scales and accumulators so that most results are ordinary numbers, with a few NaN scales
+    lo, hi = (0x20, 0x50) if key[1] == "nvf4" else (110, 140)
+    inp["sfa"] = g.integers(lo, hi, (M, K // kb), dtype=np.uint8)
+    inp["sfb"] = g.integers(lo, hi, (N, K // kb), dtype=np.uint8)
+    inp["sfa"][7, 2] = 0xFF
+    inp["sfb"][3, 0] = 0x7F if key[1] == "nvf4" else 0xFF
+    inp["C"] = g.standard_normal((M, N)).astype(np.float32).view(np.uint32)
+    _check(key, inp, expect_kernel="gstfdpa")
