@@ -326,6 +326,34 @@ __device__ __forceinline__ uint32_t efdpa_block(const uint32_t* a, const uint32_
     for (int k = 0; k < L; ++k) sp.product(a[k], b[k]);
     const int kind = sp.result();
     if (kind) return special_word(kind, false, false);
+    // Common case: every term lies inside one 62-bit window, so the exact sum fits a 64-bit integer.
+    {
+        int lo = 1 << 20, hi = -(1 << 20);              // lowest term bit, highest possible term bit
+        for (int k = 0; k < L; ++k) {
+            const uint32_t mag = dec_sig(a[k]) * dec_sig(b[k]);
+            if (mag) {
+                const int e = dec_exp(a[k]) + dec_exp(b[k]) - m.frac;
+                lo = e < lo ? e : lo;
+                hi = e + 22 > hi ? e + 22 : hi;         // products have at most 22 significant bits
+            }
+        }
+        if (dc.sig) {
+            const int e = dc.exp - 23;
+            lo = e < lo ? e : lo;
+            hi = e + 24 > hi ? e + 24 : hi;
+        }
+        if (hi < lo) return 0u;                          // every term is zero
+        if (hi - lo <= 58) {                             // up to five terms: three carry bits on top
+            long long S = 0;
+            for (int k = 0; k < L; ++k) {
+                const long long sk = (long long)dec_ssig(a[k]) * (long long)dec_ssig(b[k]);
+                if (sk) S += sk << (dec_exp(a[k]) + dec_exp(b[k]) - m.frac - lo);
+            }
+            if (dc.sig) S += (dc.sign ? -(long long)dc.sig : (long long)dc.sig) << (dc.exp - 23 - lo);
+            const uint32_t sign = S < 0;
+            return round_pack(sign, sign ? (unsigned long long)(-S) : (unsigned long long)S, lo, 8, 23, 127, true);
+        }
+    }
     uint32_t pos[EF_LIMBS], neg[EF_LIMBS];
     for (int i = 0; i < EF_LIMBS; ++i) pos[i] = neg[i] = 0u;
     for (int k = 0; k < L; ++k) {
