@@ -203,7 +203,8 @@ __device__ __forceinline__ void decode_signmag(uint32_t w, uint32_t& sig, uint32
 
 // Decode tables of the 8-bit kinds: entry `tid` of both (256 threads).
 template <int EK>
-__device__ __forceinline__ void init_lut(Smem<EK>& s, const FmtDesc& fa, const FmtDesc& fb, int pre, int guard, int tid) {
+__device__ __forceinline__ void init_lut(Smem<EK>& s, const FmtDesc& fa, const FmtDesc& fb, int pre, int guard, int tid,
+                                         bool fpsum = false) {
     constexpr bool SIGNMAG = Elem<EK>::SIGNMAG;
     if (!SIGNMAG) {
         const uint32_t da = decode_elem(fa, uint32_t(tid)), db = decode_elem(fb, uint32_t(tid));
@@ -219,6 +220,12 @@ __device__ __forceinline__ void init_lut(Smem<EK>& s, const FmtDesc& fa, const F
         eb.exp = uint32_t((fin_b ? dec_exp(db) : 1 - fb.bias) + EB);
         eb.bits = fin_b ? dec_sign(db) : 0u;
         eb.special = fin_b ? 0u : 1u;
+        if (fpsum) {
+            // floating-point form of the same operands (see the FP32 summation path of the kernel): the operand scaled
+            // by 2^Exp, exact in FP32 (at most 4 + 15 significant bits, exponents far inside the FP32 range)
+            ea.op = __float_as_uint(ldexpf(float(fin_a ? dec_ssig(da) : 0), fin_a ? dec_exp(da) : 0));
+            eb.op = __float_as_uint(ldexpf(float(sb * (1 << (pre + guard)) + ub), fin_b ? dec_exp(db) : 0));
+        }
         s.lut_a[tid] = ea;
         s.lut_b[tid] = eb;
     }
@@ -261,7 +268,7 @@ __device__ __forceinline__ void load_chunk(RawChunk<EK>& raw, const GemmArgs& g,
     }
 }
 
-template <int EK>
+template <int EK, bool STORE_EXP = true>
 __device__ __forceinline__ void store_chunk(Smem<EK>& s, const RawChunk<EK>& raw, int chunk, int pre, int tid) {
     using E = Elem<EK>;
     using R = RawChunk<EK>;
@@ -296,8 +303,8 @@ __device__ __forceinline__ void store_chunk(Smem<EK>& s, const RawChunk<EK>& raw
                 spec |= special;
                 if (is_a) s.a_msk[SIGNMAG ? kk : 0][r] = 0u - sign; else s.b_msk[SIGNMAG ? kk : 0][r] = 0u - sign;
             }
-            if (is_a) { s.a_op[kk][r] = op; s.a_exp[kk][r] = expb; }
-            else { s.b_op[kk][r] = op; s.b_exp[kk][r] = expb; }
+            if (is_a) { s.a_op[kk][r] = op; if (STORE_EXP) s.a_exp[kk][r] = expb; }
+            else { s.b_op[kk][r] = op; if (STORE_EXP) s.b_exp[kk][r] = expb; }
             if (q & 1) {
                 const uint32_t pair = prev_exp | (expb << 16);
                 if (is_a) s.a_exp2[kk / 2][r] = pair; else s.b_exp2[kk / 2][r] = pair;
@@ -351,7 +358,10 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
     const int guard = SIGNMAG ? 0 : fa.mbits + 1;   // guard bits below the truncation point (8-bit kinds)
     const int one = int(blockDim.x >> 8);           // 1, but not a compile-time constant (see mad_one)
 
-    init_lut<EK>(s, fa, fb, pre, guard, tid);
+    // FP32 summation path (8-bit inputs with F <= 13): aligned terms stay below 2^15 and block sums below 2^21, so the
+    // whole of pass 2 runs exactly on the FP32 pipe, two instructions per term (see pass 2 below).
+    constexpr bool FPSUM = !SIGNMAG && F <= 13;
+    init_lut<EK>(s, fa, fb, pre, guard, tid, FPSUM);
     if (tid == 0) s.special[0] = s.special[1] = 0;
 
     Acc acc[TM][TN];
@@ -383,7 +393,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
     for (int64_t k0 = 0; k0 < g.K; k0 += KC, ++chunk) {
         __syncthreads();
         if (!PREFETCH) load_chunk<EK>(raw, g, row0, col0, k0, tid);
-        store_chunk<EK>(s, raw, chunk, pre, tid);
+        store_chunk<EK, !FPSUM>(s, raw, chunk, pre, tid);
         __syncthreads();
         if (PREFETCH && k0 + KC < g.K) load_chunk<EK>(raw, g, row0, col0, k0 + KC, tid);
 
@@ -477,8 +487,46 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
                     S0[r][c] = asr_clamp(acc[r][c].cs, emax[r][c] - rel) - (acc[r][c].cs >> 31);
                     if (NSUM == 2) S1[NSUM == 2 ? r : 0][NSUM == 2 ? c : 0] = 0;
                     emax[r][c] += guard;
+                    if (FPSUM) {
+                        // The sum lives in an FP32 register as 1.5 * 2^23 + S: in [2^23, 2^24) one ulp is one unit of S,
+                        // so integers add exactly and adding a fraction with rounding toward minus infinity is a floor.
+                        S0[r][c] += 0x4B400000;
+                        acc[r][c].ce = emax[r][c];          // Exp(c) is spent; keep e_max + g there for the epilogue
+                        // 2^-(e_max + g); beyond 2^-126 every product vanishes either way (terms are below 2^48)
+                        emax[r][c] = (127 - min(emax[r][c] - CB, 126)) << 23;
+                    }
                 }
             // ---- pass 2: multiply, align, truncate, add ----
+            if (FPSUM) {
+                // X_k * 2^-(d_k + g) = (A_op * 2^Exp(a)) * (B_op * 2^Exp(b)) * 2^-(e_max + g): the first product is exact
+                // in FP32 (19 significant bits), the fused multiply-add computes the second one exactly and rounds the
+                // sum once, toward minus infinity: S <- S + floor(X_k * 2^-(d_k + g)), the same one's-complement term
+                // as the arithmetic shift of the integer path.
+#pragma unroll 4
+                for (int kk = kb; kk < kb + L; ++kk) {
+                    const float4 oa0 = *reinterpret_cast<const float4*>(&s.a_op[kk][ty * TM]);
+                    const float4 oa1 = *reinterpret_cast<const float4*>(&s.a_op[kk][ty * TM + 4]);
+                    const float4 ob = *reinterpret_cast<const float4*>(&s.b_op[kk][tx * TN]);
+                    const float oav[TM] = {oa0.x, oa0.y, oa0.z, oa0.w, oa1.x, oa1.y, oa1.z, oa1.w};
+                    const float obv[TN] = {ob.x, ob.y, ob.z, ob.w};
+#pragma unroll
+                    for (int r = 0; r < TM; ++r)
+#pragma unroll
+                        for (int c = 0; c < TN; ++c) {
+                            const float xs = __fmul_rn(oav[r], obv[c]);
+                            float sum = __int_as_float(S0[r][c]);
+                            asm("fma.rm.f32 %0, %1, %2, %0;" : "+f"(sum) : "f"(xs), "f"(__int_as_float(emax[r][c])));
+                            S0[r][c] = __float_as_int(sum);
+                        }
+                }
+#pragma unroll
+                for (int r = 0; r < TM; ++r)
+#pragma unroll
+                    for (int c = 0; c < TN; ++c) {
+                        S0[r][c] -= 0x4B400000;
+                        emax[r][c] = acc[r][c].ce;
+                    }
+            } else {
 #pragma unroll 2
             for (int kk = kb; kk < kb + L; ++kk) {
                 const bool second = NSUM == 2 && (kk - kb >= HALF);
@@ -516,6 +564,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
                             else S0[r][c] = mad_one(t, one, S0[r][c]);
                         }
                 }
+            }
             }
             // ---- sign corrections, normalisation, rho ----
             const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
