@@ -62,20 +62,26 @@ struct LutEntry {
     uint32_t special;   // nonzero for infinity / NaN
 };
 
-template <int EK>
-struct Smem {
+// Staged operands of one chunk.  SLIM drops the planes that the FP32 summation path does not read.
+template <int EK, bool SLIM = false>
+struct Planes {
     uint32_t a_op[KC][BM];
-    uint32_t a_exp[KC][BM];
     uint32_t b_op[KC][BN];
-    uint32_t b_exp[KC][BN];
+    uint32_t a_exp[SLIM ? 1 : KC][BM];
+    uint32_t b_exp[SLIM ? 1 : KC][BN];
     uint32_t a_exp2[KC / 2][BM];    // exponents of elements 2p (low half) and 2p + 1 (high half)
     uint32_t b_exp2[KC / 2][BN];
     uint32_t a_msk[Elem<EK>::SIGNMAG ? KC : 1][BM];   // 0 / ~0: sign of the element (sign-magnitude kinds)
     uint32_t b_msk[Elem<EK>::SIGNMAG ? KC : 1][BN];
+    uint32_t a_sgn[BM], a_nz[BM], b_sgn[BN];          // bit k of row r: sign / nonzero of element k of the chunk
+};
+
+template <int EK, bool SLIM = false, int NBUF = 1>
+struct Smem {
+    Planes<EK, SLIM> pl[NBUF];
     LutEntry lut_a[Elem<EK>::SIGNMAG ? 1 : 256];
     LutEntry lut_b[Elem<EK>::SIGNMAG ? 1 : 256];
-    uint32_t a_sgn[BM], a_nz[BM], b_sgn[BN];          // bit k of row r: sign / nonzero of element k of the chunk
-    int special[2];                                   // chunk (by parity) holds an infinity or a NaN
+    int special[3];                                   // chunk (by index mod 2 or 3) holds an infinity or a NaN
 };
 
 __device__ __forceinline__ int asr_clamp(int x, int d) {
@@ -202,8 +208,8 @@ __device__ __forceinline__ void decode_signmag(uint32_t w, uint32_t& sig, uint32
 }
 
 // Decode tables of the 8-bit kinds: entry `tid` of both (256 threads).
-template <int EK>
-__device__ __forceinline__ void init_lut(Smem<EK>& s, const FmtDesc& fa, const FmtDesc& fb, int pre, int guard, int tid,
+template <int EK, class SM>
+__device__ __forceinline__ void init_lut(SM& s, const FmtDesc& fa, const FmtDesc& fb, int pre, int guard, int tid,
                                          bool fpsum = false) {
     constexpr bool SIGNMAG = Elem<EK>::SIGNMAG;
     if (!SIGNMAG) {
@@ -268,8 +274,8 @@ __device__ __forceinline__ void load_chunk(RawChunk<EK>& raw, const GemmArgs& g,
     }
 }
 
-template <int EK, bool STORE_EXP = true>
-__device__ __forceinline__ void store_chunk(Smem<EK>& s, const RawChunk<EK>& raw, int chunk, int pre, int tid) {
+template <int EK, bool STORE_EXP = true, class SM, class PL>
+__device__ __forceinline__ void store_chunk(SM& sm, PL& s, const RawChunk<EK>& raw, int flag, int pre, int tid) {
     using E = Elem<EK>;
     using R = RawChunk<EK>;
     constexpr bool SIGNMAG = E::SIGNMAG;
@@ -289,7 +295,7 @@ __device__ __forceinline__ void store_chunk(Smem<EK>& s, const RawChunk<EK>& raw
             uint32_t op, expb;
             if (!SIGNMAG) {
                 const uint32_t byte = (raw.w[it][q / 4] >> (8 * (q % 4))) & 0xFFu;
-                const LutEntry e = is_a ? s.lut_a[byte] : s.lut_b[byte];
+                const LutEntry e = is_a ? sm.lut_a[byte] : sm.lut_b[byte];
                 op = e.op;
                 expb = e.exp;
                 bits += e.bits << q;
@@ -324,17 +330,20 @@ __device__ __forceinline__ void store_chunk(Smem<EK>& s, const RawChunk<EK>& raw
             else reinterpret_cast<uint8_t*>(&s.b_sgn[r])[h] = uint8_t(bits);
         }
     }
-    if (spec) atomicOr(&s.special[chunk & 1], 1);
+    if (spec) atomicOr(&sm.special[flag], 1);
 }
 
 // Load and stage in one go (no prefetch).
-template <int EK>
-__device__ __forceinline__ void stage_chunk(Smem<EK>& s, const GemmArgs& g, int64_t row0, int64_t col0, int64_t k0,
+template <int EK, class SM>
+__device__ __forceinline__ void stage_chunk(SM& s, const GemmArgs& g, int64_t row0, int64_t col0, int64_t k0,
                                             int chunk, int pre, int tid) {
     RawChunk<EK> raw;
     load_chunk<EK>(raw, g, row0, col0, k0, tid);
-    store_chunk<EK>(s, raw, chunk, pre, tid);
+    store_chunk<EK>(s, s.pl[0], raw, chunk & 1, pre, tid);
 }
+
+template <int EK, int F>
+struct TfdpaFpsum { static constexpr bool value = !Elem<EK>::SIGNMAG && F <= 13; };
 
 template <int EK, int L, int F, int RHO, bool PROMOTE, bool ST = false>
 __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
@@ -347,8 +356,14 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
     constexpr int NBLK = KC / L;
     static_assert(KC % L == 0 && L % 2 == 0, "blocks tile the chunk; pass 1 handles pairs of elements");
     static_assert(!ST || L == KC, "ST-FDPA: one scale factor pair per block of 32 (Algorithm 8)");
+    // FP32 summation path (8-bit inputs with F <= 13): aligned terms stay below 2^15 and block sums below 2^21, so the
+    // whole of pass 2 runs exactly on the FP32 pipe, two instructions per term (see pass 2 below).  Its staged planes
+    // are small enough for two buffers: the next chunk is decoded while the current one is computed, one barrier per chunk.
+    constexpr bool FPSUM = TfdpaFpsum<EK, F>::value;
+    constexpr bool DB = FPSUM;
+    using SM = Smem<EK, FPSUM, DB ? 2 : 1>;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    Smem<EK>& s = *reinterpret_cast<Smem<EK>*>(smem_raw);
+    SM& sm = *reinterpret_cast<SM*>(smem_raw);
 
     const int tid = threadIdx.x;
     const int tx = tid % 16, ty = tid / 16;
@@ -358,11 +373,8 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
     const int guard = SIGNMAG ? 0 : fa.mbits + 1;   // guard bits below the truncation point (8-bit kinds)
     const int one = int(blockDim.x >> 8);           // 1, but not a compile-time constant (see mad_one)
 
-    // FP32 summation path (8-bit inputs with F <= 13): aligned terms stay below 2^15 and block sums below 2^21, so the
-    // whole of pass 2 runs exactly on the FP32 pipe, two instructions per term (see pass 2 below).
-    constexpr bool FPSUM = !SIGNMAG && F <= 13;
-    init_lut<EK>(s, fa, fb, pre, guard, tid, FPSUM);
-    if (tid == 0) s.special[0] = s.special[1] = 0;
+    init_lut<EK>(sm, fa, fb, pre, guard, tid, FPSUM);
+    if (tid == 0) sm.special[0] = sm.special[1] = sm.special[2] = 0;
 
     Acc acc[TM][TN];
     uint32_t sp_nan = 0u, sp_pinf = 0u, sp_ninf = 0u;   // per output (bit r * TN + c): NaN / +inf / -inf seen so far
@@ -389,16 +401,34 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
     constexpr bool PREFETCH = EK == EK_LUT8 && NSUM == 1;
     RawChunk<EK> raw;
     if (PREFETCH) load_chunk<EK>(raw, g, row0, col0, 0, tid);
+    if (DB) {
+        __syncthreads();                                   // tables and flags are ready
+        store_chunk<EK, !FPSUM>(sm, sm.pl[0], raw, 0, pre, tid);
+        if (KC < g.K) load_chunk<EK>(raw, g, row0, col0, KC, tid);
+        __syncthreads();
+    }
     int chunk = 0;
     for (int64_t k0 = 0; k0 < g.K; k0 += KC, ++chunk) {
-        __syncthreads();
-        if (!PREFETCH) load_chunk<EK>(raw, g, row0, col0, k0, tid);
-        store_chunk<EK, !FPSUM>(s, raw, chunk, pre, tid);
-        __syncthreads();
-        if (PREFETCH && k0 + KC < g.K) load_chunk<EK>(raw, g, row0, col0, k0 + KC, tid);
-
-        if (tid == 0) s.special[(chunk + 1) & 1] = 0;
-        bool chunk_special = s.special[chunk & 1] != 0;
+        int flag;
+        if (!DB) {
+            __syncthreads();
+            if (!PREFETCH) load_chunk<EK>(raw, g, row0, col0, k0, tid);
+            store_chunk<EK, !FPSUM>(sm, sm.pl[0], raw, chunk & 1, pre, tid);
+            __syncthreads();
+            if (PREFETCH && k0 + KC < g.K) load_chunk<EK>(raw, g, row0, col0, k0 + KC, tid);
+            flag = chunk & 1;
+            if (tid == 0) sm.special[(chunk + 1) & 1] = 0;
+        } else {
+            // decode chunk n + 1 into the other buffer (its raw words arrived during the previous iteration), then fetch n + 2
+            flag = chunk % 3;
+            if (tid == 0) sm.special[(chunk + 2) % 3] = 0;   // last read two barriers ago, next written after the coming one
+            if (k0 + KC < g.K) {
+                store_chunk<EK, !FPSUM>(sm, sm.pl[(chunk + 1) & 1], raw, (chunk + 1) % 3, pre, tid);
+                if (k0 + 2 * KC < g.K) load_chunk<EK>(raw, g, row0, col0, k0 + 2 * KC, tid);
+            }
+        }
+        auto& s = sm.pl[DB ? (chunk & 1) : 0];
+        bool chunk_special = sm.special[flag] != 0;
 
         // ST-FDPA (Algorithm 8): Exp(alpha) of this thread's rows and Exp(beta) of its columns for this block of 32
         int sa_exp[ST ? TM : 1], sb_exp[ST ? TN : 1];
@@ -605,6 +635,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
                 }
             }
         }
+        if (DB) __syncthreads();                           // the other buffer is complete, this one is free
         // ---- FP32 promotion of the partial sum every k_chunk elements ----
         if (PROMOTE && ((k0 + KC) % g.k_chunk) == 0) {
 #pragma unroll
@@ -647,7 +678,8 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
 
 template <int EK, int L, int F, int RHO, bool PROMOTE, bool ST = false>
 cudaError_t launch_one(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
-    const size_t sh = sizeof(Smem<EK>);
+    constexpr bool FPSUM = TfdpaFpsum<EK, F>::value;
+    const size_t sh = sizeof(Smem<EK, FPSUM, FPSUM ? 2 : 1>);
     cudaError_t err = cudaFuncSetAttribute(tfdpa_kernel<EK, L, F, RHO, PROMOTE, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
     if (err != cudaSuccess) return err;
     dim3 grid((unsigned)((g.N + BN - 1) / BN), (unsigned)((g.M + BM - 1) / BM), 1);

@@ -84,7 +84,8 @@ __global__ void __launch_bounds__(NT, 2) trfdpa_kernel(DevModel m, GemmArgs g) {
     constexpr int EMINB = -126 + CB, EMAXB = 127 + CB;
     static_assert(KC % L == 0 && L % 2 == 0, "blocks tile the chunk; pass 1 handles pairs of elements");
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    Smem<EK>& s = *reinterpret_cast<Smem<EK>*>(smem_raw);
+    Smem<EK>& sm = *reinterpret_cast<Smem<EK>*>(smem_raw);
+    auto& s = sm.pl[0];
 
     const int tid = threadIdx.x;
     const int tx = tid % 16, ty = tid / 16;
@@ -96,8 +97,8 @@ __global__ void __launch_bounds__(NT, 2) trfdpa_kernel(DevModel m, GemmArgs g) {
     const int guard = SIGNMAG ? 0 : fa.mbits + 1;
     const int one = int(blockDim.x >> 8);
 
-    init_lut<EK>(s, fa, fb, pre, guard, tid);
-    if (tid == 0) s.special[0] = s.special[1] = 0;
+    init_lut<EK>(sm, fa, fb, pre, guard, tid);
+    if (tid == 0) sm.special[0] = sm.special[1] = 0;
 
     TrAcc acc[TM][TN];
     uint32_t sp_nan = 0u, sp_pinf = 0u, sp_ninf = 0u;
@@ -118,10 +119,10 @@ __global__ void __launch_bounds__(NT, 2) trfdpa_kernel(DevModel m, GemmArgs g) {
     int chunk = 0;
     for (int64_t k0 = 0; k0 < g.K; k0 += KC, ++chunk) {
         __syncthreads();
-        stage_chunk<EK>(s, g, row0, col0, k0, chunk, pre, tid);
+        stage_chunk<EK>(sm, g, row0, col0, k0, chunk, pre, tid);
         __syncthreads();
-        if (tid == 0) s.special[(chunk + 1) & 1] = 0;
-        const bool chunk_special = s.special[chunk & 1] != 0;
+        if (tid == 0) sm.special[(chunk + 1) & 1] = 0;
+        const bool chunk_special = sm.special[chunk & 1] != 0;
 
 #pragma unroll 1
         for (int blk = 0; blk < NBLK; ++blk) {
