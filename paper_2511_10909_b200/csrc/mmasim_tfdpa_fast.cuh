@@ -46,6 +46,7 @@ namespace fast {
 constexpr int BM = 128, BN = 64, TM = 8, TN = 4, KC = 32, NT = 256;
 constexpr int EB = 512;            // bias of a staged element exponent
 constexpr int CB = 2 * EB;         // bias of an exponent sum and of the accumulator exponent
+constexpr int FP_SHIFT = 8;        // FP32 summation path: the B operands are scaled by 2^-FP_SHIFT (see pass 2)
 
 enum ElemKind : int { EK_LUT8 = 0, EK_F16 = 1, EK_BF16 = 2, EK_TF32 = 3 };
 
@@ -230,7 +231,7 @@ __device__ __forceinline__ void init_lut(SM& s, const FmtDesc& fa, const FmtDesc
             // floating-point form of the same operands (see the FP32 summation path of the kernel): the operand scaled
             // by 2^Exp, exact in FP32 (at most 4 + 15 significant bits, exponents far inside the FP32 range)
             ea.op = __float_as_uint(ldexpf(float(fin_a ? dec_ssig(da) : 0), fin_a ? dec_exp(da) : 0));
-            eb.op = __float_as_uint(ldexpf(float(sb * (1 << (pre + guard)) + ub), fin_b ? dec_exp(db) : 0));
+            eb.op = __float_as_uint(ldexpf(float(sb * (1 << (pre + guard)) + ub), (fin_b ? dec_exp(db) : 0) - FP_SHIFT));
         }
         s.lut_a[tid] = ea;
         s.lut_b[tid] = eb;
@@ -521,9 +522,9 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
                         // The sum lives in an FP32 register as 1.5 * 2^23 + S: in [2^23, 2^24) one ulp is one unit of S,
                         // so integers add exactly and adding a fraction with rounding toward minus infinity is a floor.
                         S0[r][c] += 0x4B400000;
-                        acc[r][c].ce = emax[r][c];          // Exp(c) is spent; keep e_max + g there for the epilogue
-                        // 2^-(e_max + g); beyond 2^-126 every product vanishes either way (terms are below 2^48)
-                        emax[r][c] = (127 - min(emax[r][c] - CB, 126)) << 23;
+                        // 2^(FP_SHIFT - (e_max + g)) as an FP32 word (the B operands carry 2^-FP_SHIFT): e_max + g lies in
+                        // [-25, 131], so the exponent field stays inside 1..254 and e_max can be read back from it
+                        emax[r][c] = (127 + FP_SHIFT + CB - emax[r][c]) << 23;
                     }
                 }
             // ---- pass 2: multiply, align, truncate, add ----
@@ -554,7 +555,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
 #pragma unroll
                     for (int c = 0; c < TN; ++c) {
                         S0[r][c] -= 0x4B400000;
-                        emax[r][c] = acc[r][c].ce;
+                        emax[r][c] = 127 + FP_SHIFT + CB - int(uint32_t(emax[r][c]) >> 23);
                     }
             } else {
 #pragma unroll 2
