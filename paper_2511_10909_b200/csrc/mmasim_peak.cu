@@ -12,7 +12,7 @@ enum PeakKind : int {
 };
 
 template <int KIND>
-__device__ __forceinline__ void round8(int (&x)[8], float (&f)[8], double (&dd)[8]) {
+__device__ __forceinline__ void round8(int (&x)[8], float (&f)[8]) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const int j = (i + 1) & 7, k = (i + 3) & 7;
@@ -42,8 +42,6 @@ __device__ __forceinline__ void round8(int (&x)[8], float (&f)[8], double (&dd)[
             asm("mad.lo.s32 %0, %1, %2, %0;" : "+r"(x[i]) : "r"(t), "r"(x[(i + 5) & 7]));
         } else if (KIND == PK_DP4A) {
             x[i] = __dp4a(x[j], x[k], x[i]);
-        } else if (KIND == PK_DFMA) {
-            dd[i] = fma(dd[i], dd[j], dd[k]);
         } else if (KIND == PK_MAC_D2) {             // one emulated term with pre-shifted operands: wide multiply, funnel shift, accumulate
             const long long w = (long long)x[j] * (long long)x[k];
             const int t = __funnelshift_rc(int(w), int(w >> 32), x[(i + 2) & 7]);
@@ -56,21 +54,36 @@ template <int KIND>
 __global__ void __launch_bounds__(256) peak_kernel(int64_t iters, int* sink) {
     int x[8];
     float f[8];
-    double dd[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         x[i] = threadIdx.x * 2654435 + i * 40503 + blockIdx.x;
         f[i] = 1.0f + 1e-7f * float(threadIdx.x + i);
-        dd[i] = 1.0 + 1e-9 * double(threadIdx.x + i);
     }
     for (int64_t it = 0; it < iters; it += 8) {
 #pragma unroll
-        for (int u = 0; u < 8; ++u) round8<KIND>(x, f, dd);
+        for (int u = 0; u < 8; ++u) round8<KIND>(x, f);
     }
     int r = 0;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) r ^= x[i] ^ __float_as_int(f[i]) ^ int(__double_as_longlong(dd[i]));
+    for (int i = 0; i < 8; ++i) r ^= x[i] ^ __float_as_int(f[i]);
     if (r == 0x12345678) *sink = r;             // practically never true: keeps the chains alive
+}
+
+// FP64 fused multiply-add chains (a kernel of its own so that the integer kernels keep their register allocation)
+__global__ void __launch_bounds__(256) peak_kernel_f64(int64_t iters, int* sink) {
+    double d[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) d[i] = 1.0 + 1e-9 * double(threadIdx.x + i);
+    for (int64_t it = 0; it < iters; it += 8) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) d[i] = fma(d[i], d[(i + 1) & 7], d[(i + 3) & 7]);
+    }
+    double r = 0.0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) r += d[i];
+    if (r == 0.12345) *sink = 1;
 }
 
 template <int KIND>
@@ -102,7 +115,13 @@ int launch_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t
         case PK_MAC_D1: *ops_per_round = 1; return launch<PK_MAC_D1>(blocks, iters, sink, stream);
         case PK_MAC_D2: *ops_per_round = 1; return launch<PK_MAC_D2>(blocks, iters, sink, stream);
         case PK_DP4A: *ops_per_round = 1; return launch<PK_DP4A>(blocks, iters, sink, stream);
-        case PK_DFMA: *ops_per_round = 1; return launch<PK_DFMA>(blocks, iters, sink, stream);
+        case PK_DFMA: {
+            *ops_per_round = 1;
+            peak_kernel_f64<<<(unsigned)blocks, 256, 0, stream>>>(iters, static_cast<int*>(sink));
+            const cudaError_t err = cudaGetLastError();
+            if (err != cudaSuccess) { set_error("int_peak launch failed: %s", cudaGetErrorString(err)); return MMASIM_ERR_CUDA; }
+            return MMASIM_OK;
+        }
         default: set_error("mmasim_int_peak: unknown kind %d", kind); return MMASIM_ERR_INVALID_ARG;
     }
 }
