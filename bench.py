@@ -78,6 +78,21 @@ def make_inputs(name):
     return {"A": d["A"], "B": d["B"], "C": d["C"]}
 
 
+def max_over_ranks(value: float, dist=None, device=None) -> float:
+    """The slowest rank's time: every rank contributes its own device-timed milliseconds."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return float(value)
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(macs_per_rank_step: float, steps: int, world: int, slowest_ms: float) -> float:
+    """Aggregate MAC/s of `world` replicas that each evaluate their own batch (weak scaling, no exchange)."""
+    return macs_per_rank_step * world * steps / (slowest_ms * 1e-3)
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -260,13 +275,9 @@ def run_ours(args):
     if dist is not None:
         dist.barrier()
     clocks = sampler.stop()
-    total_ms = sum(e0.elapsed_time(e1) for e0, e1 in events)
-    if dist is not None:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(sum(e0.elapsed_time(e1) for e0, e1 in events), dist, dev)
     macs_per_step = float(M) * N * K * world
-    value = macs_per_step * args.steps / (total_ms * 1e-3)
+    value = whole_job_value(float(M) * N * K, args.steps, world, total_ms)
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region) ----
     e2e = None
@@ -288,10 +299,7 @@ def run_ours(args):
             mmasim.gemm_host(model, hA, hB, hC, out=hD.numpy(), **hkw)
         torch.cuda.synchronize()
         e2e_s = (time.perf_counter() - t0) / n_e2e
-        if dist is not None:
-            t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = float(t.item())
+        e2e_s = max_over_ranks(e2e_s, dist, dev)
         h2d = hA.numel() * hA.element_size() + hB.numel() * hB.element_size() + hC.numel() * hC.element_size()
         e2e = {"value": macs_per_step / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                "d2h_bytes_per_step": int(hD.numel() * hD.element_size()), "ms_per_step": 1e3 * e2e_s,
