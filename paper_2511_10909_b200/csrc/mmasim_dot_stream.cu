@@ -56,24 +56,27 @@ dot_tfdpa_kernel(DevModel m, int64_t n, int64_t K, const void* A, const void* B,
         uint32_t wa[L], wb[L];
         load_block<EK, L>(A, t * K + k0, wa);
         load_block<EK, L>(B, t * K + k0, wb);
-        // Step 1: exact products and exponent sums
-        uint32_t mag[L], neg = 0u, special = 0u;
-        int e[L];
+        // Step 1: exact products and exponent sums.  Decoding is branch-free: the hidden bit is min(field, 1), the
+        // unnormalised exponent max(field, 1); infinities and NaNs are found by the largest exponent field seen.
+        using E = Elem<EK>;
+        constexpr uint32_t TOP = (1u << E::EBITS) - 1u, MM = (1u << E::MBITS) - 1u;
+        constexpr int SIGN_SHIFT = 31 - (E::MBITS + E::EBITS + E::LOW);   // moves the element's sign bit to bit 31
+        int X[L], e[L], sm[L];                            // |product| << pre, exponent sum (field units), sign mask
+        uint32_t fmax_seen = 0u;
 #pragma unroll
         for (int k = 0; k < L; ++k) {
-            uint32_t sa, ea, na, spa, sb, eb, nb, spb;
-            fast::decode_signmag<EK>(wa[k], sa, ea, na, spa);
-            fast::decode_signmag<EK>(wb[k], sb, eb, nb, spb);
-            mag[k] = sa * sb;
-            e[k] = int(ea + eb);                      // biased by CB
-            neg |= (na ^ nb) << k;
-            special |= spa | spb;
+            const uint32_t xa = wa[k] >> E::LOW, xb = wb[k] >> E::LOW;
+            const uint32_t fa = (xa >> E::MBITS) & TOP, fb = (xb >> E::MBITS) & TOP;
+            const uint32_t sa = (xa & MM) | (min(fa, 1u) << E::MBITS);
+            const uint32_t sb = ((xb & MM) | (min(fb, 1u) << E::MBITS)) << pre;
+            X[k] = int(sa * sb);
+            e[k] = int(max(fa, 1u) + max(fb, 1u));        // Exp(a) + Exp(b) + 2 * bias
+            sm[k] = int((wa[k] ^ wb[k]) << SIGN_SHIFT) >> 31;
+            fmax_seen = max(fmax_seen, max(fa, fb));
         }
         const AccDec dc = decode_acc(cw, ACC16);
-        if (special | (dc.cls != CLS_FINITE)) {
+        if (fmax_seen == TOP || dc.cls != CLS_FINITE) {
             // an infinity or a NaN among the 2L + 1 inputs: Section 4.2 decides the result (classes straight from the raw words)
-            using E = Elem<EK>;
-            constexpr uint32_t TOP = (1u << E::EBITS) - 1u, MM = (1u << E::MBITS) - 1u;
             bool nan = dc.cls == CLS_NAN, pinf = dc.cls == CLS_INF && !dc.sign, ninf = dc.cls == CLS_INF && dc.sign;
 #pragma unroll
             for (int k = 0; k < L; ++k) {
@@ -89,20 +92,23 @@ dot_tfdpa_kernel(DevModel m, int64_t n, int64_t K, const void* A, const void* B,
             cw = special_word((nan || (pinf && ninf)) ? 1 : (pinf ? 2 : 3), ACC16, true);
             continue;
         }
-        // Step 2: maximum exponent, alignment, truncation (sign-magnitude), exact sum
+        // Step 2: maximum exponent, alignment, truncation (sign-magnitude), exact sum.  Exponent sums are kept in field
+        // units (biased by 2 * E::BIAS); `ceb` and `emax` below carry the bias CB like everywhere else.
+        constexpr int EBIAS = CB - 2 * E::BIAS;           // e[k] + EBIAS = Exp(a) + Exp(b) + CB
         const int ceb = dc.exp + CB;
-        int emax = ceb;
+        int emax = ceb - EBIAS;
 #pragma unroll
         for (int k = 0; k < L; ++k) emax = max(emax, e[k]);
-        const uint32_t cmag = fast::lsr_clamp(dc.sig << (F >= MB_ACC ? F - MB_ACC : 0), (emax - ceb) + (F >= MB_ACC ? 0 : MB_ACC - F));
+        const uint32_t cmag = fast::lsr_clamp(dc.sig << (F >= MB_ACC ? F - MB_ACC : 0), (emax + EBIAS - ceb) + (F >= MB_ACC ? 0 : MB_ACC - F));
         // terms stay below 2^27 (F <= 25): eight of them and the accumulator fit 32 bits, sixteen need two partial sums
         int S0 = dc.sign ? -int(cmag) : int(cmag), S1 = 0;
 #pragma unroll
         for (int k = 0; k < L; ++k) {
-            const uint32_t tk = fast::lsr_clamp(mag[k] << pre, emax - e[k]);
-            const int sk = ((neg >> k) & 1u) ? -int(tk) : int(tk);
+            const int tk = int(fast::lsr_clamp(uint32_t(X[k]), emax - e[k]));
+            const int sk = (tk ^ sm[k]) - sm[k];
             if (L > 8 && k >= L / 2) S1 += sk; else S0 += sk;
         }
+        emax += EBIAS;
         const long long S = (long long)S0 + (long long)S1;
         // Step 3: rho
         const bool fits = S == (long long)int(S);
