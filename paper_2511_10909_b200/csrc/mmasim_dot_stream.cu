@@ -1,9 +1,14 @@
 // Streaming kernels for mmasim_dot_batch: n independent dot-product-accumulates d_t = Phi(a_t, b_t, c_t) (Equation 4),
-// the shape of the paper's probe vectors (Section 3.1).  One thread owns one dot product and walks its two rows block
-// by block with 16-byte loads; nothing is shared between threads, so the kernel is bound by HBM traffic
-// (2 * K * element bytes + 8 bytes per dot) as long as the per-term integer work stays below it.
-//   T-FDPA (Algorithm 7) for FP16 / BF16 / TF32 inputs, L in {4, 8, 16}, any F, rho in {RZ-FP32, RNE-FP16}
+// the shape of the paper's probe vectors (Section 3.1).  One thread owns one dot product; nothing is shared between
+// dots, so the kernels are bound by HBM traffic (2 * K * element bytes + 8 bytes per dot).
+//   T-FDPA (Algorithm 7) for FP16 / BF16 / TF32 inputs, L in {4, 8, 16}, F in 23..25, rho in {RZ-FP32, RNE-FP16}
 //   Phi_FTZ-AddMul (Algorithm 2) for FP16 / BF16 inputs, P in {2, 4}
+// Two ways to bring the rows in:
+//   staged - rows of 8, 16, 32, 64 or 128 bytes: the CTA's 256 rows of A and of B are one contiguous range each, copied
+//            to shared memory with 16-byte asynchronous copies (consecutive threads, consecutive chunks: every
+//            sector of a request is used), chunks XOR-swizzled so that each thread then reads its own row without bank
+//            conflicts; several CTAs per SM keep the copies of one tile under the arithmetic of another
+//   direct - any other row length: each thread reads its row with 16-byte loads
 // Everything else (8-bit inputs, other families, odd shapes) uses the generic kernels.
 #include <cuda_fp16.h>
 #include "mmasim_tfdpa_fast.cuh"
@@ -18,161 +23,321 @@ using fast::EK_TF32;
 
 constexpr int DOT_THREADS = 256;
 
-// Load L consecutive elements (L * BYTES is 8, 16, 32 or 64 bytes) as raw words.
-template <int EK, int L>
-__device__ __forceinline__ void load_block(const void* base, int64_t elem_index, uint32_t (&w)[L]) {
-    constexpr int BYTES = Elem<EK>::BYTES;
-    const unsigned char* p = static_cast<const unsigned char*>(base) + elem_index * BYTES;
-    uint32_t raw[L * BYTES / 4];
+// ---- where a thread finds its two rows ----
+struct GlobalRows {                      // row pointers into global memory
+    const unsigned char* a;
+    const unsigned char* b;
+    __device__ __forceinline__ uint4 ld16(bool second, int byte_off) const {
+        return *reinterpret_cast<const uint4*>((second ? b : a) + byte_off);
+    }
+    __device__ __forceinline__ uint2 ld8(bool second, int byte_off) const {
+        return *reinterpret_cast<const uint2*>((second ? b : a) + byte_off);
+    }
+};
+struct StagedRows {                      // this thread's rows inside the staged tile (shared memory, swizzled chunks)
+    const unsigned char* a;              // start of the row's chunk group
+    const unsigned char* b;
+    int swz;                             // XOR applied to the chunk index inside the row
+    __device__ __forceinline__ uint4 ld16(bool second, int byte_off) const {
+        return *reinterpret_cast<const uint4*>((second ? b : a) + (((byte_off >> 4) ^ swz) << 4));
+    }
+    __device__ __forceinline__ uint2 ld8(bool second, int byte_off) const {
+        return *reinterpret_cast<const uint2*>((second ? b : a) + (((byte_off >> 4) ^ swz) << 4) + (byte_off & 8));
+    }
+};
+
+// L consecutive elements (L * BYTES is 8, 16, 32 or 64 bytes) as raw 32-bit words (two elements per word for the
+// 16-bit formats).
+template <int BYTES, int L, class Rows>
+__device__ __forceinline__ void load_raw(const Rows& rows, bool second, int elem_index, uint32_t (&raw)[L * BYTES / 4]) {
     if (L * BYTES == 8) {
-        const uint2 v = *reinterpret_cast<const uint2*>(p);
+        const uint2 v = rows.ld8(second, elem_index * BYTES);
         raw[0] = v.x; raw[1] = v.y;
     } else {
 #pragma unroll
         for (int q = 0; q < L * BYTES / 16; ++q) {
-            const uint4 v = reinterpret_cast<const uint4*>(p)[q];
+            const uint4 v = rows.ld16(second, elem_index * BYTES + 16 * q);
             raw[4 * q] = v.x; raw[4 * q + 1] = v.y; raw[4 * q + 2] = v.z; raw[4 * q + 3] = v.w;
         }
     }
-#pragma unroll
-    for (int k = 0; k < L; ++k) w[k] = BYTES == 2 ? ((raw[k / 2] >> (16 * (k % 2))) & 0xFFFFu) : raw[k];
 }
 
-template <int EK, int L, int RHO>
+// Start the copy of one tile's rows of A and B (rows t0 .. t0 + nrows - 1, `row_bytes` each) into one stage of shared
+// memory.  Chunk c of row r lands at chunk position c ^ ((r / rows_per_line) % chunks_per_row) of that row,
+// rows_per_line = 128 bytes / row_bytes: the eight threads of a quarter warp then read eight different 16-byte
+// bank groups.  The caller commits the group and waits for it.
+__device__ __forceinline__ void stage_issue(unsigned char* stage, const void* A, const void* B, int64_t t0, int nrows,
+                                            int row_bytes) {
+    const int tid = threadIdx.x;
+    const int lcpr = row_bytes >= 16 ? 31 - __clz(row_bytes >> 4) : 0;      // log2(chunks per row); rows of 8 bytes: two rows per chunk
+    const int cmask = (1 << lcpr) - 1;
+    const int lrpl = 3 - lcpr;                                              // log2(rows per 128-byte line)
+    const int bytes = nrows * row_bytes;
+    unsigned char* sa = stage;
+    unsigned char* sb = stage + DOT_THREADS * row_bytes;
+    const unsigned char* ga = static_cast<const unsigned char*>(A) + t0 * row_bytes;
+    const unsigned char* gb = static_cast<const unsigned char*>(B) + t0 * row_bytes;
+    for (int g = tid; g < (bytes >> 4); g += DOT_THREADS) {
+        int dst = g;
+        if (row_bytes >= 16) {
+            const int r = g >> lcpr, c = g & cmask;
+            dst = (r << lcpr) + (c ^ ((r >> lrpl) & cmask));
+        }
+        const unsigned da = unsigned(__cvta_generic_to_shared(sa + (dst << 4)));
+        const unsigned db = unsigned(__cvta_generic_to_shared(sb + (dst << 4)));
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(da), "l"(ga + (int64_t(g) << 4)) : "memory");
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(db), "l"(gb + (int64_t(g) << 4)) : "memory");
+    }
+    if ((bytes & 8) && tid == 0) {                                          // 8-byte rows, odd row count: the last row
+        *reinterpret_cast<uint2*>(sa + bytes - 8) = *reinterpret_cast<const uint2*>(ga + bytes - 8);
+        *reinterpret_cast<uint2*>(sb + bytes - 8) = *reinterpret_cast<const uint2*>(gb + bytes - 8);
+    }
+}
+
+// This thread's rows inside a stage.
+__device__ __forceinline__ StagedRows staged_view(const unsigned char* stage, int row_bytes) {
+    const int tid = threadIdx.x;
+    const int lcpr = row_bytes >= 16 ? 31 - __clz(row_bytes >> 4) : 0;
+    StagedRows rows;
+    rows.a = stage + tid * row_bytes;
+    rows.b = stage + (DOT_THREADS + tid) * row_bytes;
+    rows.swz = (tid >> (3 - lcpr)) & ((1 << lcpr) - 1);
+    return rows;
+}
+
+// One tile per CTA: copy, wait, compute.  With 32 KB per tile about six CTAs share an SM, and the copies of some run
+// under the arithmetic of the others.  (A persistent variant with two stages per CTA was slower: the stages cost
+// half of the resident warps.)  `body(rows, t, c)` returns the result word of dot t.
+template <bool ACC16, class Body>
+__device__ __forceinline__ void staged_tile(unsigned char* smem, int64_t n, int row_bytes, const void* A, const void* B,
+                                            const void* C, void* D, Body body) {
+    const int64_t t0 = int64_t(blockIdx.x) * DOT_THREADS, t = t0 + threadIdx.x;
+    stage_issue(smem, A, B, t0, int(min(int64_t(DOT_THREADS), n - t0)), row_bytes);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    uint32_t c = 0u;
+    if (C && t < n) c = ACC16 ? uint32_t(static_cast<const uint16_t*>(C)[t]) : static_cast<const uint32_t*>(C)[t];
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+    if (t >= n) return;
+    const uint32_t w = body(staged_view(smem, row_bytes), t, c);
+    if (ACC16) static_cast<uint16_t*>(D)[t] = uint16_t(w);
+    else static_cast<uint32_t*>(D)[t] = w;
+}
+
+__device__ __forceinline__ double fma_rm(double x, double y, double z) {
+    double r;
+    asm("fma.rm.f64 %0, %1, %2, %3;" : "=d"(r) : "d"(x), "d"(y), "d"(z));
+    return r;
+}
+
+// trunc(p * scale) with the sign of p (RZ_F of Algorithm 7 is sign-magnitude), for |p * scale| < 2^51: the magnitude
+// is floored by one fused multiply-add rounding toward minus infinity onto 2^52 (one ulp = 1), the sign is copied
+// back on the high word.  (Choosing the rounding direction by the sign instead costs more: the compiler turns the two
+// predicated operations into two executed ones plus selects.)
+__device__ __forceinline__ double trunc_scaled(double p, double scale, int sign_word) {
+    const double n = fma_rm(fabs(p), scale, 4503599627370496.0) - 4503599627370496.0;
+    return __hiloint2double(__double2hiint(n) | (sign_word & int(0x80000000u)), __double2loint(n));
+}
+
+// T-FDPA (Algorithm 7) on the FP64 pipe, the chain of Algorithm 5 for one dot product.  A double holds every quantity
+// of a block exactly: products of two 11-bit (8-bit) significands, their scaling by 2^(F - e_max) (a power of two, no
+// underflow in the FP64 range), the truncated terms (< 2^27) and their sum (< 2^32).  Infinities and NaNs need no
+// separate tracking: IEEE arithmetic on the products gives NaN for NaN inputs, inf * 0 and inf - inf, and the
+// surviving infinity otherwise, which is the rule of Section 4.2; the block result is replaced by the canonical
+// word when the sum is not finite.  Only e_max stays on the integer pipe (two terms per instruction, 16-bit lanes).
+template <int EK, int L, int RHO, class Rows>
+__device__ __forceinline__ uint32_t tfdpa_dot(const Rows& rows, int K, int F, uint32_t cw) {
+    using E = Elem<EK>;
+    constexpr bool ACC16 = RHO == RHO_RNE_FP16;
+    constexpr int NRAW = L * E::BYTES / 4;
+    for (int k0 = 0; k0 < K; k0 += L) {
+        uint32_t ra[NRAW], rb[NRAW];
+        load_raw<E::BYTES, L>(rows, false, k0, ra);
+        load_raw<E::BYTES, L>(rows, true, k0, rb);
+        // Step 1: exact products (as FP32 for FP16 inputs, whose products stay inside the FP32 range; as FP64
+        // otherwise) and the largest exponent sum Exp(a) + Exp(b), with Exp = max(field, 1) - bias.
+        float pf[E::BYTES == 2 && EK == EK_F16 ? L : 1];
+        double pd[EK == EK_F16 ? 1 : L];
+        int e_prod;
+        if (E::BYTES == 2) {
+            constexpr uint32_t EXPM = ((1u << E::EBITS) - 1u) << E::MBITS, ONE = 1u << E::MBITS;
+            uint32_t mx = 0u;
+#pragma unroll
+            for (int q = 0; q < NRAW; ++q) {
+                const uint32_t ea = __vmaxu2(ra[q] & (EXPM * 0x10001u), ONE * 0x10001u);
+                const uint32_t eb = __vmaxu2(rb[q] & (EXPM * 0x10001u), ONE * 0x10001u);
+                mx = __vmaxu2(mx, ea + eb);               // field sums stay below 2^16: no carry between the lanes
+                if (EK == EK_F16) {
+                    const float2 fa = __half22float2(*reinterpret_cast<const __half2*>(&ra[q]));
+                    const float2 fb = __half22float2(*reinterpret_cast<const __half2*>(&rb[q]));
+                    pf[2 * q < L ? 2 * q : 0] = __fmul_rn(fa.x, fb.x);
+                    pf[2 * q + 1 < L ? 2 * q + 1 : 0] = __fmul_rn(fa.y, fb.y);
+                } else {
+                    pd[2 * q < L ? 2 * q : 0] = __dmul_rn(double(__uint_as_float(ra[q] << 16)), double(__uint_as_float(rb[q] << 16)));
+                    pd[2 * q + 1 < L ? 2 * q + 1 : 0] = __dmul_rn(double(__uint_as_float(ra[q] & 0xFFFF0000u)), double(__uint_as_float(rb[q] & 0xFFFF0000u)));
+                }
+            }
+            e_prod = int(max(mx & 0xFFFFu, mx >> 16) >> E::MBITS) - 2 * E::BIAS;
+        } else {
+            uint32_t mx = 0u;
+#pragma unroll
+            for (int k = 0; k < L; ++k) {
+                mx = max(mx, max((ra[k] >> 23) & 0xFFu, 1u) + max((rb[k] >> 23) & 0xFFu, 1u));
+                pd[EK == EK_F16 ? 0 : k] = __dmul_rn(double(__uint_as_float(ra[k] & 0xFFFFE000u)), double(__uint_as_float(rb[k] & 0xFFFFE000u)));
+            }
+            e_prod = int(mx) - 2 * E::BIAS;
+        }
+        const uint32_t cfield = ACC16 ? (cw >> 10) & 0x1Fu : (cw >> 23) & 0xFFu;
+        const int e_c = int(max(cfield, 1u)) - (ACC16 ? 15 : 127);
+        const double cd = ACC16 ? double(__half2float(__ushort_as_half((unsigned short)cw))) : double(__uint_as_float(cw));
+
+        // Step 2: e_max over the L + 1 terms, alignment and sign-magnitude truncation to F fractional bits, exact sum
+        const int emax = max(e_prod, e_c);
+        const double scale = __hiloint2double((1023 + F - emax) << 20, 0);
+        double S0 = trunc_scaled(cd, scale, __double2hiint(cd)), S1 = 0.0;
+#pragma unroll
+        for (int k = 0; k < L; ++k) {
+            double tk;
+            if (EK == EK_F16) tk = trunc_scaled(double(pf[EK == EK_F16 ? k : 0]), scale, __float_as_int(pf[EK == EK_F16 ? k : 0]));
+            else tk = trunc_scaled(pd[EK == EK_F16 ? 0 : k], scale, __double2hiint(pd[EK == EK_F16 ? 0 : k]));
+            if (k & 1) S1 += tk; else S0 += tk;
+        }
+        // Step 3: d = rho(S * 2^(e_max - F)).  S (|S| < 2^33) times a power of two is exact in FP64, so rho is one
+        // conversion: RZ-FP32 saturates at the largest finite number, RNE-FP16 overflows to infinity, both keep
+        // subnormal results; an exact zero is +0.  A sum that is not finite gives the NaN / infinity of Section 4.2.
+        const double S = S0 + S1;                         // S1 starts from +0, so an all-zero sum is +0
+        const double v = __dmul_rn(S, __hiloint2double((1023 + emax - F) << 20, 0));
+        if (ACC16) cw = (v != v) ? 0x7FFFu : uint32_t(__half_as_ushort(__double2half(v)));
+        else cw = (v != v) ? 0x7FFFFFFFu : __float_as_uint(__double2float_rz(v));
+    }
+    return cw;
+}
+
+template <int EK, int L, int RHO, bool STAGED>
 __global__ void __launch_bounds__(DOT_THREADS)
 dot_tfdpa_kernel(DevModel m, int64_t n, int64_t K, const void* A, const void* B, const void* C, void* D) {
     constexpr bool ACC16 = RHO == RHO_RNE_FP16;
-    constexpr int CB = fast::CB;
-    constexpr int EMINB = (ACC16 ? -14 : -126) + CB, EMAXB = (ACC16 ? 15 : 127) + CB;
-    const int64_t t = int64_t(blockIdx.x) * DOT_THREADS + threadIdx.x;
-    if (t >= n) return;
+    extern __shared__ __align__(16) unsigned char dot_smem[];
+    const int row_bytes = int(K) * Elem<EK>::BYTES;
     const int F = m.F;
-    const int pre = F - 2 * Elem<EK>::MBITS;
-    const int MB_ACC = ACC16 ? 10 : 23;
-    uint32_t cw = 0u;
-    if (C) cw = ACC16 ? uint32_t(static_cast<const uint16_t*>(C)[t]) : static_cast<const uint32_t*>(C)[t];
-
-    for (int64_t k0 = 0; k0 < K; k0 += L) {
-        uint32_t wa[L], wb[L];
-        load_block<EK, L>(A, t * K + k0, wa);
-        load_block<EK, L>(B, t * K + k0, wb);
-        // Step 1: exact products and exponent sums.  Decoding is branch-free: the hidden bit is min(field, 1), the
-        // unnormalised exponent max(field, 1); infinities and NaNs are found by the largest exponent field seen.
-        using E = Elem<EK>;
-        constexpr uint32_t TOP = (1u << E::EBITS) - 1u, MM = (1u << E::MBITS) - 1u;
-        constexpr int SIGN_SHIFT = 31 - (E::MBITS + E::EBITS + E::LOW);   // moves the element's sign bit to bit 31
-        int X[L], e[L], sm[L];                            // |product| << pre, exponent sum (field units), sign mask
-        uint32_t fmax_seen = 0u;
-#pragma unroll
-        for (int k = 0; k < L; ++k) {
-            const uint32_t xa = wa[k] >> E::LOW, xb = wb[k] >> E::LOW;
-            const uint32_t fa = (xa >> E::MBITS) & TOP, fb = (xb >> E::MBITS) & TOP;
-            const uint32_t sa = (xa & MM) | (min(fa, 1u) << E::MBITS);
-            const uint32_t sb = ((xb & MM) | (min(fb, 1u) << E::MBITS)) << pre;
-            X[k] = int(sa * sb);
-            e[k] = int(max(fa, 1u) + max(fb, 1u));        // Exp(a) + Exp(b) + 2 * bias
-            sm[k] = int((wa[k] ^ wb[k]) << SIGN_SHIFT) >> 31;
-            fmax_seen = max(fmax_seen, max(fa, fb));
-        }
-        const AccDec dc = decode_acc(cw, ACC16);
-        if (fmax_seen == TOP || dc.cls != CLS_FINITE) {
-            // an infinity or a NaN among the 2L + 1 inputs: Section 4.2 decides the result (classes straight from the raw words)
-            bool nan = dc.cls == CLS_NAN, pinf = dc.cls == CLS_INF && !dc.sign, ninf = dc.cls == CLS_INF && dc.sign;
-#pragma unroll
-            for (int k = 0; k < L; ++k) {
-                const uint32_t xa = wa[k] >> E::LOW, xb = wb[k] >> E::LOW;
-                const bool spa = ((xa >> E::MBITS) & TOP) == TOP, spb = ((xb >> E::MBITS) & TOP) == TOP;
-                if (!(spa | spb)) continue;
-                const bool nana = spa && (xa & MM), nanb = spb && (xb & MM);
-                const bool za = (xa & ((1u << (E::MBITS + E::EBITS)) - 1u)) == 0u, zb = (xb & ((1u << (E::MBITS + E::EBITS)) - 1u)) == 0u;
-                if (nana | nanb | (spa && zb) | (spb && za)) nan = true;          // NaN * x, inf * 0
-                else if (((xa ^ xb) >> (E::MBITS + E::EBITS)) & 1u) ninf = true;   // inf * z = inf * sign(z)
-                else pinf = true;
-            }
-            cw = special_word((nan || (pinf && ninf)) ? 1 : (pinf ? 2 : 3), ACC16, true);
-            continue;
-        }
-        // Step 2: maximum exponent, alignment, truncation (sign-magnitude), exact sum.  Exponent sums are kept in field
-        // units (biased by 2 * E::BIAS); `ceb` and `emax` below carry the bias CB like everywhere else.
-        constexpr int EBIAS = CB - 2 * E::BIAS;           // e[k] + EBIAS = Exp(a) + Exp(b) + CB
-        const int ceb = dc.exp + CB;
-        int emax = ceb - EBIAS;
-#pragma unroll
-        for (int k = 0; k < L; ++k) emax = max(emax, e[k]);
-        const uint32_t cmag = fast::lsr_clamp(dc.sig << (F >= MB_ACC ? F - MB_ACC : 0), (emax + EBIAS - ceb) + (F >= MB_ACC ? 0 : MB_ACC - F));
-        // terms stay below 2^27 (F <= 25): eight of them and the accumulator fit 32 bits, sixteen need two partial sums
-        int S0 = dc.sign ? -int(cmag) : int(cmag), S1 = 0;
-#pragma unroll
-        for (int k = 0; k < L; ++k) {
-            const int tk = int(fast::lsr_clamp(uint32_t(X[k]), emax - e[k]));
-            const int sk = (tk ^ sm[k]) - sm[k];
-            if (L > 8 && k >= L / 2) S1 += sk; else S0 += sk;
-        }
-        emax += EBIAS;
-        const long long S = (long long)S0 + (long long)S1;
-        // Step 3: rho
-        const bool fits = S == (long long)int(S);
-        int vmin = EMINB, vmax = EMINB;
-        fast::Acc a;
-        if (fits && F >= MB_ACC && RHO != RHO_RZ_E8M13) {
-            fast::rho_fast<25, RHO>(int(S), emax + (25 - F), a, vmin, vmax);   // value = S * 2^(e_max - F): rescaled to the F = 25 form
-        }
-        if (!fits || F < MB_ACC || vmin < EMINB || vmax > EMAXB) {
-            cw = rho_apply(RHO, S, emax - CB - F);
-        } else {
-            cw = fast::acc_to_word<25, ACC16>(a, 0u);
-        }
+    if (STAGED) {
+        staged_tile<ACC16>(dot_smem, n, row_bytes, A, B, C, D, [&](const StagedRows& rows, int64_t, uint32_t c) {
+            return tfdpa_dot<EK, L, RHO>(rows, int(K), F, c);
+        });
+    } else {
+        const int64_t t = int64_t(blockIdx.x) * DOT_THREADS + threadIdx.x;
+        if (t >= n) return;
+        uint32_t cw = 0u;
+        if (C) cw = ACC16 ? uint32_t(static_cast<const uint16_t*>(C)[t]) : static_cast<const uint32_t*>(C)[t];
+        GlobalRows rows;
+        rows.a = static_cast<const unsigned char*>(A) + t * row_bytes;
+        rows.b = static_cast<const unsigned char*>(B) + t * row_bytes;
+        cw = tfdpa_dot<EK, L, RHO>(rows, int(K), F, cw);
+        if (ACC16) static_cast<uint16_t*>(D)[t] = uint16_t(cw);
+        else static_cast<uint32_t*>(D)[t] = cw;
     }
-    if (ACC16) static_cast<uint16_t*>(D)[t] = uint16_t(cw);
-    else static_cast<uint32_t*>(D)[t] = cw;
 }
 
-// Phi_FTZ-AddMul, one dot per thread.
-template <int EK, int P>
-__global__ void __launch_bounds__(DOT_THREADS)
-dot_ftz_kernel(int64_t n, int64_t K, const void* A, const void* B, const void* C, void* D) {
-    const int64_t t = int64_t(blockIdx.x) * DOT_THREADS + threadIdx.x;
-    if (t >= n) return;
-    float d = 0.0f;
-    if (C) {
-        const uint32_t w = static_cast<const uint32_t*>(C)[t];
-        d = ((w & 0x7F800000u) == 0u && (w & 0x007FFFFFu)) ? 0.0f : __uint_as_float(w);     // FlushSubnormal(C)
-    }
-    constexpr int STEP = 4;                           // elements per load (8 bytes)
-    for (int64_t k0 = 0; k0 < K; k0 += STEP) {
-        uint32_t wa[STEP], wb[STEP];
-        load_block<EK, STEP>(A, t * K + k0, wa);
-        load_block<EK, STEP>(B, t * K + k0, wb);
+// FTZ-Add / FTZ-Mul (Algorithm 1) as the hardware's flush-to-zero operations: operands are never subnormal here
+// (Algorithm 2 flushes the inputs first and every intermediate is flushed), and no result is rounded across 2^-126
+// (products of 16-bit formats have at most 22 significant bits; sums below 2^-125 are multiples of 2^-149).
+__device__ __forceinline__ float hw_ftz_add(float x, float y) {
+    float z;
+    asm("add.rn.ftz.f32 %0, %1, %2;" : "=f"(z) : "f"(x), "f"(y));
+    return z;
+}
+__device__ __forceinline__ float hw_ftz_mul(float x, float y) {
+    float z;
+    asm("mul.rn.ftz.f32 %0, %1, %2;" : "=f"(z) : "f"(x), "f"(y));
+    return z;
+}
+
+// Phi_FTZ-AddMul (Algorithm 2) for one dot product; STEP elements per load and operand.
+template <int EK, int P, int STEP, class Rows>
+__device__ __forceinline__ float ftz_dot(const Rows& rows, int K, float d) {
+    for (int k0 = 0; k0 < K; k0 += STEP) {
+        uint32_t ra[STEP / 2], rb[STEP / 2];
+        load_raw<2, STEP>(rows, false, k0, ra);
+        load_raw<2, STEP>(rows, true, k0, rb);
         float a[STEP], b[STEP];
 #pragma unroll
         for (int k = 0; k < STEP; ++k) {
+            const uint32_t wa = (ra[k / 2] >> (16 * (k % 2))) & 0xFFFFu, wb = (rb[k / 2] >> (16 * (k % 2))) & 0xFFFFu;
             if (EK == EK_BF16) {
-                a[k] = ((wa[k] & 0x7F80u) == 0u && (wa[k] & 0x007Fu)) ? 0.0f : __uint_as_float(wa[k] << 16);
-                b[k] = ((wb[k] & 0x7F80u) == 0u && (wb[k] & 0x007Fu)) ? 0.0f : __uint_as_float(wb[k] << 16);
+                a[k] = ((wa & 0x7F80u) == 0u && (wa & 0x007Fu)) ? 0.0f : __uint_as_float(wa << 16);
+                b[k] = ((wb & 0x7F80u) == 0u && (wb & 0x007Fu)) ? 0.0f : __uint_as_float(wb << 16);
             } else {
-                a[k] = ((wa[k] & 0x7C00u) == 0u && (wa[k] & 0x03FFu)) ? 0.0f : __half2float(__ushort_as_half((unsigned short)wa[k]));
-                b[k] = ((wb[k] & 0x7C00u) == 0u && (wb[k] & 0x03FFu)) ? 0.0f : __half2float(__ushort_as_half((unsigned short)wb[k]));
+                a[k] = ((wa & 0x7C00u) == 0u && (wa & 0x03FFu)) ? 0.0f : __half2float(__ushort_as_half((unsigned short)wa));
+                b[k] = ((wb & 0x7C00u) == 0u && (wb & 0x03FFu)) ? 0.0f : __half2float(__ushort_as_half((unsigned short)wb));
             }
         }
-        if (P == 4) {
-            const float s = ftz_add(ftz_add(ftz_mul(a[0], b[0]), ftz_mul(a[1], b[1])), ftz_add(ftz_mul(a[2], b[2]), ftz_mul(a[3], b[3])));
-            d = ftz_add(d, s);
-        } else {
-            d = ftz_add(d, ftz_add(ftz_mul(a[0], b[0]), ftz_mul(a[1], b[1])));
-            d = ftz_add(d, ftz_add(ftz_mul(a[2], b[2]), ftz_mul(a[3], b[3])));
+#pragma unroll
+        for (int g = 0; g < STEP; g += 4) {
+            if (P == 4) {
+                const float s = hw_ftz_add(hw_ftz_add(hw_ftz_mul(a[g], b[g]), hw_ftz_mul(a[g + 1], b[g + 1])), hw_ftz_add(hw_ftz_mul(a[g + 2], b[g + 2]), hw_ftz_mul(a[g + 3], b[g + 3])));
+                d = hw_ftz_add(d, s);
+            } else {
+                d = hw_ftz_add(d, hw_ftz_add(hw_ftz_mul(a[g], b[g]), hw_ftz_mul(a[g + 1], b[g + 1])));
+                d = hw_ftz_add(d, hw_ftz_add(hw_ftz_mul(a[g + 2], b[g + 2]), hw_ftz_mul(a[g + 3], b[g + 3])));
+            }
         }
     }
-    uint32_t w = __float_as_uint(d);
-    if (d != d) w = 0x7FC00000u;
-    static_cast<uint32_t*>(D)[t] = w;
+    return d;
+}
+
+__device__ __forceinline__ float flush_c(uint32_t w) {       // FlushSubnormal(C) of Algorithm 2
+    return ((w & 0x7F800000u) == 0u && (w & 0x007FFFFFu)) ? 0.0f : __uint_as_float(w);
+}
+__device__ __forceinline__ uint32_t ftz_word(float d) { return d != d ? 0x7FC00000u : __float_as_uint(d); }
+
+template <int EK, int P, int STEP, bool STAGED>
+__global__ void __launch_bounds__(DOT_THREADS)
+dot_ftz_kernel(int64_t n, int64_t K, const void* A, const void* B, const void* C, void* D) {
+    extern __shared__ __align__(16) unsigned char dot_smem[];
+    const int row_bytes = int(K) * 2;
+    if (STAGED) {
+        staged_tile<false>(dot_smem, n, row_bytes, A, B, C, D, [&](const StagedRows& rows, int64_t, uint32_t c) {
+            return ftz_word(ftz_dot<EK, P, STEP>(rows, int(K), flush_c(c)));
+        });
+    } else {
+        const int64_t t = int64_t(blockIdx.x) * DOT_THREADS + threadIdx.x;
+        if (t >= n) return;
+        GlobalRows rows;
+        rows.a = static_cast<const unsigned char*>(A) + t * row_bytes;
+        rows.b = static_cast<const unsigned char*>(B) + t * row_bytes;
+        const float d = ftz_dot<EK, P, STEP>(rows, int(K), flush_c(C ? static_cast<const uint32_t*>(C)[t] : 0u));
+        static_cast<uint32_t*>(D)[t] = ftz_word(d);
+    }
+}
+
+// Rows of 8 to 128 bytes (a power of two) are staged through shared memory: 2 * 256 rows per CTA.
+bool staged_rows(int64_t row_bytes) {
+    return row_bytes == 8 || row_bytes == 16 || row_bytes == 32 || row_bytes == 64 || row_bytes == 128;
+}
+
+template <class Kernel, class... Args>
+cudaError_t launch_dot(Kernel kernel, bool staged, int64_t n, int64_t row_bytes, cudaStream_t st, Args... args) {
+    const unsigned blocks = unsigned((n + DOT_THREADS - 1) / DOT_THREADS);
+    const size_t smem = staged ? size_t(2 * DOT_THREADS * row_bytes) : 0;          // the tile's rows of A and of B
+    if (smem > 48 * 1024) {
+        const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        if (e != cudaSuccess) return e;
+    }
+    kernel<<<blocks, DOT_THREADS, smem, st>>>(args...);
+    return cudaGetLastError();
+}
+
+template <int EK, int L, int RHO>
+cudaError_t launch_t_rho(const DevModel& m, const GemmArgs& g, cudaStream_t st) {
+    const int64_t rb = g.K * Elem<EK>::BYTES;
+    if (staged_rows(rb)) return launch_dot(dot_tfdpa_kernel<EK, L, RHO, true>, true, g.M, rb, st, m, g.M, g.K, g.A, g.B, g.C, g.D);
+    return launch_dot(dot_tfdpa_kernel<EK, L, RHO, false>, false, g.M, rb, st, m, g.M, g.K, g.A, g.B, g.C, g.D);
 }
 
 template <int EK, int L>
 cudaError_t launch_t(const DevModel& m, const GemmArgs& g, cudaStream_t st) {
-    const unsigned blocks = unsigned((g.M + DOT_THREADS - 1) / DOT_THREADS);
-    if (m.rho == RHO_RZ_FP32) dot_tfdpa_kernel<EK, L, RHO_RZ_FP32><<<blocks, DOT_THREADS, 0, st>>>(m, g.M, g.K, g.A, g.B, g.C, g.D);
-    else dot_tfdpa_kernel<EK, L, RHO_RNE_FP16><<<blocks, DOT_THREADS, 0, st>>>(m, g.M, g.K, g.A, g.B, g.C, g.D);
-    return cudaGetLastError();
+    if (m.rho == RHO_RZ_FP32) return launch_t_rho<EK, L, RHO_RZ_FP32>(m, g, st);
+    return launch_t_rho<EK, L, RHO_RNE_FP16>(m, g, st);
 }
 
 template <int EK>
@@ -183,6 +348,18 @@ cudaError_t launch_t_l(const DevModel& m, const GemmArgs& g, int L, cudaStream_t
         case 16: return launch_t<EK, 16>(m, g, st);
         default: return cudaErrorInvalidValue;
     }
+}
+
+template <int EK, int P>
+cudaError_t launch_ftz(const GemmArgs& g, cudaStream_t st) {
+    const int64_t rb = g.K * 2;
+    const bool staged = staged_rows(rb);
+    if (g.K % 8 == 0) {
+        if (staged) return launch_dot(dot_ftz_kernel<EK, P, 8, true>, true, g.M, rb, st, g.M, g.K, g.A, g.B, g.C, g.D);
+        return launch_dot(dot_ftz_kernel<EK, P, 8, false>, false, g.M, rb, st, g.M, g.K, g.A, g.B, g.C, g.D);
+    }
+    if (staged) return launch_dot(dot_ftz_kernel<EK, P, 4, true>, true, g.M, rb, st, g.M, g.K, g.A, g.B, g.C, g.D);
+    return launch_dot(dot_ftz_kernel<EK, P, 4, false>, false, g.M, rb, st, g.M, g.K, g.A, g.B, g.C, g.D);
 }
 
 }  // namespace
@@ -213,11 +390,9 @@ int launch_dot_stream(const DevModel& m, const GemmArgs& g, cudaStream_t stream)
         else err = launch_t_l<EK_TF32>(m, g, L, stream);
     } else {
         set_kernel_name("dot_ftz");
-        const unsigned blocks = unsigned((g.M + DOT_THREADS - 1) / DOT_THREADS);
-        if (m.fmt_a == EF_F16) dot_ftz_kernel<EK_F16, 4><<<blocks, DOT_THREADS, 0, stream>>>(g.M, g.K, g.A, g.B, g.C, g.D);
-        else if (m.P == 4) dot_ftz_kernel<EK_BF16, 4><<<blocks, DOT_THREADS, 0, stream>>>(g.M, g.K, g.A, g.B, g.C, g.D);
-        else dot_ftz_kernel<EK_BF16, 2><<<blocks, DOT_THREADS, 0, stream>>>(g.M, g.K, g.A, g.B, g.C, g.D);
-        err = cudaGetLastError();
+        if (m.fmt_a == EF_F16) err = launch_ftz<EK_F16, 4>(g, stream);
+        else if (m.P == 4) err = launch_ftz<EK_BF16, 4>(g, stream);
+        else err = launch_ftz<EK_BF16, 2>(g, stream);
     }
     if (err != cudaSuccess) {
         set_error("dot_batch kernel launch failed: %s", cudaGetErrorString(err));

@@ -76,6 +76,25 @@ def test_cfg4_classes_every_dot(key, K):
     assert bad.size == 0, (key, K, bad[:5], [hex(int(D[i])) for i in bad[:5]], [hex(int(want[i])) for i in bad[:5]])
 
 
+# ---- ragged dot batches: a last tile that is not full (odd row counts for 8-byte rows), row lengths that are staged
+# through shared memory (8..128 bytes) and row lengths that are read directly (48, 96, 256 bytes, ...) -----------------
+@pytest.mark.parametrize("key,K,n", [
+    (("volta", "fp16", "fp32"), 4, 777), (("volta", "fp16", "fp32"), 4, 1), (("volta", "fp16", "fp16"), 12, 515),
+    (("hopper", "fp16", "fp32"), 32, 1283), (("hopper", "fp16", "fp32"), 64, 300), (("hopper", "fp16", "fp32"), 48, 300),
+    (("hopper", "fp16", "fp16"), 128, 259), (("hopper", "bf16", "fp32"), 16, 257), (("hopper", "bf16", "fp32"), 80, 255),
+    (("hopper", "tf32", "fp32"), 32, 511), (("hopper", "tf32", "fp32"), 24, 513), (("ampere", "tf32", "fp32"), 4, 130),
+    (("cdna2", "fp16", "fp32"), 4, 1001), (("cdna2", "fp16", "fp32"), 64, 258), (("cdna2", "fp16", "fp32"), 20, 258),
+    (("cdna2", "bf16", "fp32"), 8, 3), (("cdna2", "bf16_1k", "fp32"), 24, 600), (("cdna2", "bf16", "fp32"), 256, 70),
+], ids=str)
+def test_dot_batch_ragged(key, K, n):
+    from paper_2511_10909_b200 import mmasim
+    m, A, B, C, D = _dot_case(key, K, n)
+    assert mmasim.last_kernel() in ("dot_tfdpa", "dot_ftz")
+    want = oracle.phi_dot_batch(m, A, B, C)
+    bad = np.flatnonzero(D.astype(np.uint64) != want)
+    assert bad.size == 0, (key, K, n, bad[:5], [hex(int(D[i])) for i in bad[:5]], [hex(int(want[i])) for i in bad[:5]])
+
+
 # ---- config 4 at full size: 2^20 dots, sampled dots checked (all classes), CDNA2 FP16 and an NVIDIA model ----
 @pytest.mark.parametrize("key,K", [(("cdna2", "fp16", "fp32"), 32), (("hopper", "fp16", "fp32"), 32),
                                    (("hopper", "bf16", "fp32"), 16), (("cdna2", "bf16", "fp32"), 4),
