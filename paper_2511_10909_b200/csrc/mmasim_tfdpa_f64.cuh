@@ -1,0 +1,413 @@
+// T-FDPA / ST-FDPA (Algorithms 5, 7, 8 + Table 2) for GEMM-sized inputs with the fused summation on the FP64 pipe.
+// Used for every variant with F >= 23 (FP16 / BF16 / TF32 inputs on all NVIDIA generations, the Blackwell FP8 / FP6 /
+// FP4 and MX rows); F = 13 has its own FP32 form in mmasim_tfdpa_fast.cuh.
+//
+// One fused multiply-add per term.  Within a block every aligned, truncated term is a multiple of q = 2^(e_max - F),
+// and the block sum S * q stays below 2^33 * q.  The accumulator register of an output holds
+//     acc = 1.5 * 2^52 * q  +  S * q                                   (a double in [2^52 q, 2^53 q): one ulp = q)
+// so that `acc = fma.rm.f64(a_k, b_k, acc)` computes a_k * b_k + acc exactly and rounds it once, toward minus infinity,
+// onto the grid of q: S <- S + floor(a_k b_k / q).  The alignment shift by e_max - e_k, the truncation and the
+// addition of Algorithm 7 are that single rounding; the per-output scale lives in the accumulator's exponent field and
+// costs nothing per term.  The operands are the element values themselves as doubles (exact), staged once per CTA.
+//
+// RZ_F is sign-magnitude truncation, floor is not: negative terms are made to floor to the one's complement
+// -floor(|x|) - 1 of the wanted value by an offset far below the term's own granularity but never zero: the staged
+// B operand is b + sign(b) * 2^(Exp(b) - mbits_b - 30) (a zero b becomes that offset alone), and a zero a is staged as
+// sign(a) * 2^(Exp_min(a) - 60).  Every term whose sign bits differ then floors to -floor(|x|) - 1 (zero terms to
+// -1), every other term to floor(|x|), and the number of sign-differing terms of the block, a population count over
+// per-row / per-column sign bit masks, is added back once per block, as an integer added to the bit pattern of acc.
+// The accumulator operand c gets the same treatment: its double has bit 0 of the mantissa set.
+//
+// rho (Table 2) is one conversion instruction per block and output: cvt.rz.f32.f64 (saturates at the largest finite
+// number, keeps subnormals) or cvt.rn.f16.f64 (overflows to infinity, which is recorded as a sticky special value).
+// e_max is computed as in the integer kernels (fused add-max on two 16-bit lanes); NaN / infinity inputs use the same
+// sticky flags and rescan of the raw words (Section 4.2): their staged operands are the zero stand-ins.
+#pragma once
+#include <cuda_fp16.h>
+#include "mmasim_tfdpa_fast.cuh"
+
+namespace mmasim {
+namespace fast64 {
+
+using fast::BM;
+using fast::BN;
+using fast::TM;
+using fast::TN;
+using fast::KC;
+using fast::NT;
+using fast::EB;
+using fast::CB;
+using fast::Elem;
+using fast::RawChunk;
+using fast::load_chunk;
+using fast::raw_elem;
+
+constexpr int G_OFF = 30;          // the B offset sits 30 bits below the element's last significand bit
+constexpr int A_TINY = 60;         // a zero a is 2^(Exp_min - 60)
+
+struct LutEntry64 {
+    double op;          // staged operand
+    uint32_t exp;       // Exp(x) + EB (minimum exponent for non-finite inputs)
+    uint32_t bits;      // bit 0: sign; bit 1: infinity or NaN
+};
+
+template <int EK>
+struct Planes64 {
+    double a_d[KC][BM];
+    double b_d[KC][BN];
+    uint32_t a_exp2[KC / 2][BM];    // exponents of elements 2p (low half) and 2p + 1 (high half)
+    uint32_t b_exp2[KC / 2][BN];
+    uint32_t a_sgn[BM], b_sgn[BN];  // bit k of row r: sign of element k of the chunk
+};
+
+template <int EK>
+struct Smem64 {
+    Planes64<EK> pl;
+    LutEntry64 lut_a[Elem<EK>::SIGNMAG ? 1 : 256];
+    LutEntry64 lut_b[Elem<EK>::SIGNMAG ? 1 : 256];
+    int special[2];                 // chunk (by parity) holds an infinity or a NaN
+};
+
+__device__ __forceinline__ double pow2d(int e) { return __hiloint2double((1023 + e) << 20, 0); }
+
+// Staged operand of one finite element sign * sig * 2^(exp - mbits) (sig = 0 included); see the header comment.
+__device__ __forceinline__ double operand_a(uint32_t sign, uint32_t sig, int exp, int mbits, int exp_min) {
+    const double mag = sig ? __dmul_rn(__uint2double_rn(sig), pow2d(exp - mbits)) : pow2d(exp_min - A_TINY);
+    return sign ? -mag : mag;
+}
+__device__ __forceinline__ double operand_b(uint32_t sign, uint32_t sig, int exp, int mbits) {
+    const double mag = __dadd_rn(__dmul_rn(__uint2double_rn(sig), pow2d(exp - mbits)), pow2d(exp - mbits - G_OFF));
+    return sign ? -mag : mag;
+}
+
+template <int EK, class SM>
+__device__ __forceinline__ void init_lut64(SM& s, const FmtDesc& fa, const FmtDesc& fb, int tid) {
+    if (!Elem<EK>::SIGNMAG) {
+        const uint32_t da = decode_elem(fa, uint32_t(tid)), db = decode_elem(fb, uint32_t(tid));
+        const bool fin_a = dec_cls(da) == CLS_FINITE, fin_b = dec_cls(db) == CLS_FINITE;
+        LutEntry64 ea, eb;
+        ea.op = operand_a(fin_a ? dec_sign(da) : 0u, fin_a ? dec_sig(da) : 0u, fin_a ? dec_exp(da) : 1 - fa.bias, fa.mbits, 1 - fa.bias);
+        ea.exp = uint32_t((fin_a ? dec_exp(da) : 1 - fa.bias) + EB);
+        ea.bits = (fin_a ? dec_sign(da) : 0u) | (fin_a ? 0u : 2u);
+        eb.op = operand_b(fin_b ? dec_sign(db) : 0u, fin_b ? dec_sig(db) : 0u, fin_b ? dec_exp(db) : 1 - fb.bias, fb.mbits);
+        eb.exp = uint32_t((fin_b ? dec_exp(db) : 1 - fb.bias) + EB);
+        eb.bits = (fin_b ? dec_sign(db) : 0u) | (fin_b ? 0u : 2u);
+        s.lut_a[tid] = ea;
+        s.lut_b[tid] = eb;
+    }
+}
+
+// Decode the raw words of a chunk into double operands, packed exponent pairs and sign bit masks.
+template <int EK, class SM>
+__device__ __forceinline__ void store_chunk64(SM& sm, const RawChunk<EK>& raw, int flag, int tid) {
+    using E = Elem<EK>;
+    using R = RawChunk<EK>;
+    auto& s = sm.pl;
+    uint32_t spec = 0u;
+#pragma unroll
+    for (int it = 0; it < R::PER_THREAD; ++it) {
+        const int task = it * NT + tid;
+        if (task >= R::TASKS) break;
+        const bool is_a = task < BM * R::TPR;
+        const int u = is_a ? task : task - BM * R::TPR;
+        const int rows = is_a ? BM : BN;
+        const int r = u % rows, h = u / rows;
+        uint32_t bits = 0u, prev_exp = 0u;
+#pragma unroll
+        for (int q = 0; q < E::TASK; ++q) {
+            const int kk = h * E::TASK + q;
+            double op;
+            uint32_t expb;
+            if (!E::SIGNMAG) {
+                const uint32_t byte = (raw.w[it][q / 4] >> (8 * (q % 4))) & 0xFFu;
+                const LutEntry64 e = is_a ? sm.lut_a[byte] : sm.lut_b[byte];
+                op = e.op;
+                expb = e.exp;
+                bits += (e.bits & 1u) << q;
+                spec |= e.bits & 2u;
+            } else {
+                const uint32_t w = E::BYTES == 2 ? ((raw.w[it][q / 2] >> (16 * (q % 2))) & 0xFFFFu) : raw.w[it][q];
+                uint32_t sig, sign, special;
+                fast::decode_signmag<EK>(w, sig, expb, sign, special);
+                const int exp = int(expb) - EB;
+                op = is_a ? operand_a(sign, sig, exp, E::MBITS, 1 - E::BIAS) : operand_b(sign, sig, exp, E::MBITS);
+                bits += sign << q;
+                spec |= special;
+            }
+            if (is_a) s.a_d[kk][r] = op; else s.b_d[kk][r] = op;
+            if (q & 1) {
+                const uint32_t pair = prev_exp | (expb << 16);
+                if (is_a) s.a_exp2[kk / 2][r] = pair; else s.b_exp2[kk / 2][r] = pair;
+            }
+            prev_exp = expb;
+        }
+        if (E::TASK == 16) {
+            if (is_a) reinterpret_cast<uint16_t*>(&s.a_sgn[r])[h] = uint16_t(bits);
+            else reinterpret_cast<uint16_t*>(&s.b_sgn[r])[h] = uint16_t(bits);
+        } else {
+            if (is_a) reinterpret_cast<uint8_t*>(&s.a_sgn[r])[h] = uint8_t(bits);
+            else reinterpret_cast<uint8_t*>(&s.b_sgn[r])[h] = uint8_t(bits);
+        }
+    }
+    if (spec) atomicOr(&sm.special[flag], 1);
+}
+
+// Columns of a thread's micro-tile: two adjacent pairs, 32 columns apart, so that the sixteen threads of a row of the
+// thread grid read 256 contiguous bytes of B operands per 16-byte load.
+__device__ __forceinline__ int col_of(int tx, int c) { return (c >> 1) * (BN / 2) + tx * 2 + (c & 1); }
+
+template <int EK, int L, int RHO, bool PROMOTE, bool ST>
+__global__ void __launch_bounds__(NT, 2) tfdpa64_kernel(DevModel m, GemmArgs g) {
+    using E = Elem<EK>;
+    constexpr bool ACC16 = RHO == RHO_RNE_FP16;
+    constexpr int NBLK = KC / L;
+    static_assert(RHO == RHO_RZ_FP32 || RHO == RHO_RNE_FP16, "rho is a single conversion from FP64");
+    static_assert(KC % L == 0 && L % 2 == 0, "blocks tile the chunk; pass 1 handles pairs of elements");
+    static_assert(!ST || L == KC, "ST-FDPA: one scale factor pair per block of 32 (Algorithm 8)");
+    using SM = Smem64<EK>;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    SM& sm = *reinterpret_cast<SM*>(smem_raw);
+    auto& s = sm.pl;
+
+    const int tid = threadIdx.x;
+    const int tx = tid % 16, ty = tid / 16;
+    const int64_t row0 = int64_t(blockIdx.y) * BM, col0 = int64_t(blockIdx.x) * BN;
+    const FmtDesc fa = fmt_desc(m.fmt_a), fb = fmt_desc(m.fmt_b);
+    // high word of 1.5 * 2^52 * 2^(e_max - F) is (e_max + CB) * 2^20 + MAGIC_K
+    const int MAGIC_K = ((1023 + 52 - m.F - CB) << 20) | 0x00080000;
+
+    init_lut64<EK>(sm, fa, fb, tid);
+    if (tid == 0) sm.special[0] = sm.special[1] = 0;
+
+    uint32_t cw[TM][TN];                                // the accumulator of each output: a finite FP32 / FP16 word
+    uint32_t sp_nan = 0u, sp_pinf = 0u, sp_ninf = 0u;   // per output (bit r * TN + c): NaN / +inf / -inf seen so far
+    float promoted[PROMOTE ? TM : 1][PROMOTE ? TN : 1];
+#define MMASIM_SP_GET(r, c) ((((sp_nan >> ((r) * TN + (c))) & 1u)) | (((sp_pinf >> ((r) * TN + (c))) & 1u) << 1) | (((sp_ninf >> ((r) * TN + (c))) & 1u) << 2))
+#pragma unroll
+    for (int r = 0; r < TM; ++r)
+#pragma unroll
+        for (int c = 0; c < TN; ++c) {
+            const int64_t i = row0 + ty * TM + r, j = col0 + col_of(tx, c);
+            uint32_t w = 0u;
+            if (g.C && i < g.M && j < g.N)
+                w = ACC16 ? uint32_t(static_cast<const uint16_t*>(g.C)[i * g.ldc + j])
+                          : static_cast<const uint32_t*>(g.C)[i * g.ldc + j];
+            if (PROMOTE) { promoted[PROMOTE ? r : 0][PROMOTE ? c : 0] = __uint_as_float(w); w = 0u; }
+            const AccDec d = decode_acc(w, ACC16);
+            if (d.cls != CLS_FINITE) {
+                const uint32_t bit = 1u << (r * TN + c);
+                if (d.cls == CLS_NAN) sp_nan |= bit; else if (d.sign) sp_ninf |= bit; else sp_pinf |= bit;
+                w = 0u;
+            }
+            cw[r][c] = w;
+        }
+
+    int chunk = 0;
+    for (int64_t k0 = 0; k0 < g.K; k0 += KC, ++chunk) {
+        __syncthreads();
+        {
+            RawChunk<EK> raw;
+            load_chunk<EK>(raw, g, row0, col0, k0, tid);
+            store_chunk64<EK>(sm, raw, chunk & 1, tid);
+        }
+        __syncthreads();
+        const int flag = chunk & 1;
+        if (tid == 0) sm.special[(chunk + 1) & 1] = 0;
+        const bool chunk_special = sm.special[flag] != 0;
+
+        // ST-FDPA (Algorithm 8): Exp(alpha) of this thread's rows and Exp(beta) of its columns for this block of 32
+        int sa_exp[ST ? TM : 1], sb_exp[ST ? TN : 1];
+        if (ST) {
+            const int64_t sblk = k0 / KC;
+            uint32_t scale_nan = 0u;                    // bit r * TN + c: alpha or beta of that output is NaN
+#pragma unroll
+            for (int r = 0; r < TM; ++r) {
+                const int64_t i = row0 + ty * TM + r;
+                const uint32_t w = i < g.M ? uint32_t(g.sfa[i * g.ld_sfa + sblk]) : 127u;
+                sa_exp[ST ? r : 0] = int(w) - 127;
+                if (w == 0xFFu) scale_nan |= ((1u << TN) - 1u) << (r * TN);
+            }
+#pragma unroll
+            for (int c = 0; c < TN; ++c) {
+                const int64_t j = col0 + col_of(tx, c);
+                const uint32_t w = j < g.N ? uint32_t(g.sfb[j * g.ld_sfb + sblk]) : 127u;
+                sb_exp[ST ? c : 0] = int(w) - 127;
+                if (w == 0xFFu) scale_nan |= 0x11111111u << c;
+            }
+            sp_nan |= scale_nan;                        // a NaN scale factor makes the block result NaN
+        }
+
+#pragma unroll 1
+        for (int blk = 0; blk < NBLK; ++blk) {
+            const int kb = blk * L;
+            // ---- rare: the chunk holds an infinity or a NaN: special-value events of this block (Section 4.2).
+            // Flags are sticky: once an output is special the finite arithmetic below no longer matters for it.
+            if (chunk_special) {
+#pragma unroll 1
+                for (int r = 0; r < TM; ++r)
+#pragma unroll 1
+                    for (int c = 0; c < TN; ++c) {
+                        const int64_t i = row0 + ty * TM + r, j = col0 + col_of(tx, c);
+                        if (i >= g.M || j >= g.N) continue;
+                        Special ev;
+                        for (int kk = kb; kk < kb + L; ++kk) {
+                            const uint32_t x = decode_elem(fa, raw_elem<EK>(g.A, i * g.lda + k0 + kk));
+                            const uint32_t y = decode_elem(fb, raw_elem<EK>(g.B, j * g.ldb + k0 + kk));
+                            ev.product(x, y);
+                        }
+                        const uint32_t bit = 1u << (r * TN + c);
+                        if (ev.nan) sp_nan |= bit;
+                        if (ev.pinf) sp_pinf |= bit;
+                        if (ev.ninf) sp_ninf |= bit;
+                    }
+            }
+
+            double acc[TM][TN];
+            {
+                // ---- pass 1: e_max = max(Exp(c), max_k(Exp(a_k) + Exp(b_k))), two elements per instruction.
+                // ST: the products are compared against Exp(c) minus the block's scale exponents.
+                uint32_t em2[TM][TN];
+#pragma unroll
+                for (int r = 0; r < TM; ++r)
+#pragma unroll
+                    for (int c = 0; c < TN; ++c) {
+                        const uint32_t field = ACC16 ? (cw[r][c] >> 10) & 0x1Fu : (cw[r][c] >> 23) & 0xFFu;
+                        int rel = int(max(field, 1u)) + (CB - (ACC16 ? 15 : 127));
+                        if (ST) rel -= sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0];
+                        em2[r][c] = uint32_t(rel) * 0x10001u;
+                    }
+#pragma unroll 4
+                for (int kp = kb / 2; kp < (kb + L) / 2; ++kp) {
+                    const uint4 ea0 = *reinterpret_cast<const uint4*>(&s.a_exp2[kp][ty * TM]);
+                    const uint4 ea1 = *reinterpret_cast<const uint4*>(&s.a_exp2[kp][ty * TM + 4]);
+                    const uint2 eb0 = *reinterpret_cast<const uint2*>(&s.b_exp2[kp][tx * 2]);
+                    const uint2 eb1 = *reinterpret_cast<const uint2*>(&s.b_exp2[kp][BN / 2 + tx * 2]);
+                    const uint32_t ea[TM] = {ea0.x, ea0.y, ea0.z, ea0.w, ea1.x, ea1.y, ea1.z, ea1.w};
+                    const uint32_t ebv[TN] = {eb0.x, eb0.y, eb1.x, eb1.y};
+#pragma unroll
+                    for (int r = 0; r < TM; ++r)
+#pragma unroll
+                        for (int c = 0; c < TN; ++c) em2[r][c] = __viaddmax_s16x2(ea[r], ebv[c], em2[r][c]);
+                }
+                // ---- accumulator term: acc = 1.5 * 2^52 * q + floor(c' / q) * q, c' = c with the lowest mantissa bit of
+                // its double set (never on the grid: a negative c floors to the one's complement), then + 1 if c < 0
+#pragma unroll
+                for (int r = 0; r < TM; ++r)
+#pragma unroll
+                    for (int c = 0; c < TN; ++c) {
+                        const int emax = max(int(em2[r][c] & 0xFFFFu), int(em2[r][c] >> 16));     // e_max + CB
+                        const double magic = __hiloint2double(emax * (1 << 20) + MAGIC_K, 0);
+                        double cd = ACC16 ? double(__half2float(__ushort_as_half((unsigned short)cw[r][c]))) : double(__uint_as_float(cw[r][c]));
+                        if (ST) cd = __dmul_rn(cd, pow2d(-(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0])));
+                        cd = __hiloint2double(__double2hiint(cd), __double2loint(cd) | 1);
+                        const double a0 = __dadd_rd(cd, magic);
+                        const long long bitsum = __double_as_longlong(a0) + (long long)(cw[r][c] >> (ACC16 ? 15 : 31));
+                        acc[r][c] = __longlong_as_double(bitsum);
+                    }
+            }
+            // ---- pass 2: one fused multiply-add per term, rounding toward minus infinity onto the grid of q ----
+#pragma unroll 2
+            for (int kk = kb; kk < kb + L; ++kk) {
+                double av[TM], bv[TN];
+#pragma unroll
+                for (int r = 0; r < TM; r += 2) {
+                    const double2 t = *reinterpret_cast<const double2*>(&s.a_d[kk][ty * TM + r]);
+                    av[r] = t.x; av[r + 1] = t.y;
+                }
+                {
+                    const double2 t0 = *reinterpret_cast<const double2*>(&s.b_d[kk][tx * 2]);
+                    const double2 t1 = *reinterpret_cast<const double2*>(&s.b_d[kk][BN / 2 + tx * 2]);
+                    bv[0] = t0.x; bv[1] = t0.y; bv[2] = t1.x; bv[3] = t1.y;
+                }
+#pragma unroll
+                for (int r = 0; r < TM; ++r)
+#pragma unroll
+                    for (int c = 0; c < TN; ++c)
+                        asm("fma.rm.f64 %0, %1, %2, %0;" : "+d"(acc[r][c]) : "d"(av[r]), "d"(bv[c]));
+            }
+            // ---- sign corrections, rho ----
+            const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
+#pragma unroll
+            for (int r = 0; r < TM; ++r) {
+                const uint32_t sa = s.a_sgn[ty * TM + r];
+#pragma unroll
+                for (int c = 0; c < TN; ++c) {
+                    const int nneg = __popc((sa ^ s.b_sgn[col_of(tx, c)]) & kmask);
+                    const long long bits = __double_as_longlong(acc[r][c]) + (long long)nneg;
+                    const int hi = int(bits >> 32);
+                    const double magic = __hiloint2double((hi & 0x7FF00000) | 0x00080000, 0);
+                    double v = __dsub_rn(__longlong_as_double(bits), magic);          // S * q, exact; +0 when S = 0
+                    if (ST) v = __dmul_rn(v, pow2d(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]));
+                    if (ACC16) {
+                        uint32_t w = uint32_t(__half_as_ushort(__double2half(v)));
+                        if ((w & 0x7FFFu) == 0x7C00u) {                               // RNE-FP16 overflow: +-infinity from now on
+                            const uint32_t bit = 1u << (r * TN + c);
+                            if (!((sp_nan | sp_pinf | sp_ninf) & bit)) { if (w >> 15) sp_ninf |= bit; else sp_pinf |= bit; }
+                            w = 0u;
+                        }
+                        cw[r][c] = w;
+                    } else {
+                        cw[r][c] = __float_as_uint(__double2float_rz(v));
+                    }
+                }
+            }
+        }
+        // ---- FP32 promotion of the partial sum every k_chunk elements ----
+        if (PROMOTE && ((k0 + KC) % g.k_chunk) == 0) {
+#pragma unroll
+            for (int r = 0; r < TM; ++r)
+#pragma unroll
+                for (int c = 0; c < TN; ++c) {
+                    const uint32_t sp = MMASIM_SP_GET(r, c);
+                    const uint32_t pw = sp ? special_word(((sp & 1u) || (sp & 6u) == 6u) ? 1 : ((sp & 2u) ? 2 : 3), ACC16, true) : cw[r][c];
+                    float v = __fadd_rn(promoted[PROMOTE ? r : 0][PROMOTE ? c : 0], __uint_as_float(pw));
+                    if (v != v) v = __uint_as_float(0x7FFFFFFFu);
+                    promoted[PROMOTE ? r : 0][PROMOTE ? c : 0] = v;
+                    cw[r][c] = 0u;
+                }
+            sp_nan = sp_pinf = sp_ninf = 0u;
+        }
+    }
+
+    // ---- store ----
+#pragma unroll
+    for (int r = 0; r < TM; ++r)
+#pragma unroll
+        for (int c = 0; c < TN; ++c) {
+            const int64_t i = row0 + ty * TM + r, j = col0 + col_of(tx, c);
+            if (i >= g.M || j >= g.N) continue;
+            const uint32_t sp = MMASIM_SP_GET(r, c);
+            uint32_t w = PROMOTE ? __float_as_uint(promoted[PROMOTE ? r : 0][PROMOTE ? c : 0])
+                                 : (sp ? special_word(((sp & 1u) || (sp & 6u) == 6u) ? 1 : ((sp & 2u) ? 2 : 3), ACC16, true) : cw[r][c]);
+            if (g.row_scale) {
+                float sc = __fmul_rn(g.row_scale[i], g.col_scale[j]);
+                if (sc != sc) sc = __uint_as_float(0x7FFFFFFFu);
+                float v = __fmul_rn(sc, __uint_as_float(w));
+                if (v != v) v = __uint_as_float(0x7FFFFFFFu);
+                w = __float_as_uint(v);
+            }
+            if (ACC16) static_cast<uint16_t*>(g.D)[i * g.ldd + j] = uint16_t(w);
+            else static_cast<uint32_t*>(g.D)[i * g.ldd + j] = w;
+        }
+#undef MMASIM_SP_GET
+}
+
+template <int EK, int L, int RHO, bool PROMOTE, bool ST = false>
+cudaError_t launch_one64(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
+    const size_t sh = sizeof(Smem64<EK>);
+    cudaError_t err = cudaFuncSetAttribute(tfdpa64_kernel<EK, L, RHO, PROMOTE, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
+    if (err != cudaSuccess) return err;
+    dim3 grid((unsigned)((g.N + BN - 1) / BN), (unsigned)((g.M + BM - 1) / BM), 1);
+    tfdpa64_kernel<EK, L, RHO, PROMOTE, ST><<<grid, NT, sh, stream>>>(m, g);
+    return cudaGetLastError();
+}
+
+// With or without FP32 promotion (FP32 accumulators only).
+template <int EK, int L, int RHO, bool ST = false>
+cudaError_t launch_variant64(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
+    if (RHO != RHO_RNE_FP16 && g.k_chunk) return launch_one64<EK, L, RHO, RHO != RHO_RNE_FP16, ST>(m, g, stream);
+    return launch_one64<EK, L, RHO, false, ST>(m, g, stream);
+}
+
+}  // namespace fast64
+}  // namespace mmasim
