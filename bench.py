@@ -39,6 +39,8 @@ WORKLOADS = {
              "BF16 2048^3, exponents uniform over +-20 binades, C ~ N(0,1); Ampere BF16->FP32 model (L=8, F=24, RZ-FP32)"),
     "hopper_fp16": (("hopper", "fp16", "fp32"), (4096, 4096, 4096),
                     "FP16 4096^3 N(0,1) inputs; Hopper FP16->FP32 model (L=16, F=25, RZ-FP32)"),
+    "hopper_fp16_2k": (("hopper", "fp16", "fp32"), (2048, 2048, 2048),
+                       "FP16 2048^3 N(0,1) inputs (reduced case for profiler captures); Hopper FP16->FP32 model"),
     "volta_fp16": (("volta", "fp16", "fp32"), (4096, 4096, 4096),
                    "FP16 4096^3 N(0,1) inputs; Volta FP16->FP32 model (L=4, F=23, RZ-FP32)"),
     "ampere_bf16": (("ampere", "bf16", "fp32"), (4096, 4096, 4096),

@@ -124,18 +124,12 @@ __device__ __forceinline__ void staged_tile(unsigned char* smem, int64_t n, int 
     else static_cast<uint32_t*>(D)[t] = w;
 }
 
-__device__ __forceinline__ double fma_rm(double x, double y, double z) {
-    double r;
-    asm("fma.rm.f64 %0, %1, %2, %3;" : "=d"(r) : "d"(x), "d"(y), "d"(z));
-    return r;
-}
-
 // trunc(p * scale) with the sign of p (RZ_F of Algorithm 7 is sign-magnitude), for |p * scale| < 2^51: the magnitude
 // is floored by one fused multiply-add rounding toward minus infinity onto 2^52 (one ulp = 1), the sign is copied
 // back on the high word.  (Choosing the rounding direction by the sign instead costs more: the compiler turns the two
 // predicated operations into two executed ones plus selects.)
 __device__ __forceinline__ double trunc_scaled(double p, double scale, int sign_word) {
-    const double n = fma_rm(fabs(p), scale, 4503599627370496.0) - 4503599627370496.0;
+    const double n = __fma_rd(fabs(p), scale, 4503599627370496.0) - 4503599627370496.0;
     return __hiloint2double(__double2hiint(n) | (sign_word & int(0x80000000u)), __double2loint(n));
 }
 

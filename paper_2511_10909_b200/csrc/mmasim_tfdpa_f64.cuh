@@ -31,16 +31,49 @@ namespace fast64 {
 
 using fast::BM;
 using fast::BN;
-using fast::TM;
-using fast::TN;
 using fast::KC;
-using fast::NT;
 using fast::EB;
 using fast::CB;
 using fast::Elem;
-using fast::RawChunk;
-using fast::load_chunk;
 using fast::raw_elem;
+
+// 512 threads own the 128 x 64 tile of D, 4 x 4 outputs each: sixteen warps per SM keep the FP64 pipe fed while the
+// per-thread state (accumulators, product exponents of the next block, operands) stays within 128 registers.
+constexpr int TM = 4, TN = 4, NT = 512;
+
+// The raw words of one chunk, E::TASK consecutive elements of one row of A or B per task (as in the integer kernels).
+template <int EK>
+struct RawChunk {
+    static constexpr int TPR = KC / Elem<EK>::TASK;
+    static constexpr int TASKS = (BM + BN) * TPR;
+    static constexpr int PER_THREAD = (TASKS + NT - 1) / NT;
+    static constexpr int WORDS = Elem<EK>::TASK * Elem<EK>::BYTES / 4;
+    uint32_t w[PER_THREAD][WORDS];
+};
+
+template <int EK>
+__device__ __forceinline__ void load_chunk(RawChunk<EK>& raw, const GemmArgs& g, int64_t row0, int64_t col0, int64_t k0, int tid) {
+    using E = Elem<EK>;
+    using R = RawChunk<EK>;
+#pragma unroll
+    for (int it = 0; it < R::PER_THREAD; ++it) {
+        const int task = it * NT + tid;
+        const bool is_a = task < BM * R::TPR;
+        const int u = is_a ? task : task - BM * R::TPR;
+        const int rows = is_a ? BM : BN;
+        const int r = u % rows, h = u / rows;              // consecutive threads take consecutive rows
+        const int64_t grow = (is_a ? row0 : col0) + r;
+        const bool valid = task < R::TASKS && grow < (is_a ? g.M : g.N);
+        const unsigned char* base = static_cast<const unsigned char*>(is_a ? g.A : g.B) +
+                                    (grow * (is_a ? g.lda : g.ldb) + k0 + h * E::TASK) * E::BYTES;
+#pragma unroll
+        for (int q = 0; q < R::WORDS / 4; ++q) {
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (valid) v = reinterpret_cast<const uint4*>(base)[q];
+            raw.w[it][4 * q] = v.x; raw.w[it][4 * q + 1] = v.y; raw.w[it][4 * q + 2] = v.z; raw.w[it][4 * q + 3] = v.w;
+        }
+    }
+}
 
 constexpr int G_OFF = 30;          // the B offset sits 30 bits below the element's last significand bit
 constexpr int A_TINY = 60;         // a zero a is 2^(Exp_min - 60)
@@ -62,10 +95,10 @@ struct Planes64 {
 
 template <int EK>
 struct Smem64 {
-    Planes64<EK> pl;
+    Planes64<EK> pl[2];             // the chunk being computed and the one being decoded
     LutEntry64 lut_a[Elem<EK>::SIGNMAG ? 1 : 256];
     LutEntry64 lut_b[Elem<EK>::SIGNMAG ? 1 : 256];
-    int special[2];                 // chunk (by parity) holds an infinity or a NaN
+    int special[3];                 // chunk (by index mod 3) holds an infinity or a NaN
 };
 
 __device__ __forceinline__ double pow2d(int e) { return __hiloint2double((1023 + e) << 20, 0); }
@@ -82,7 +115,7 @@ __device__ __forceinline__ double operand_b(uint32_t sign, uint32_t sig, int exp
 
 template <int EK, class SM>
 __device__ __forceinline__ void init_lut64(SM& s, const FmtDesc& fa, const FmtDesc& fb, int tid) {
-    if (!Elem<EK>::SIGNMAG) {
+    if (!Elem<EK>::SIGNMAG && tid < 256) {
         const uint32_t da = decode_elem(fa, uint32_t(tid)), db = decode_elem(fb, uint32_t(tid));
         const bool fin_a = dec_cls(da) == CLS_FINITE, fin_b = dec_cls(db) == CLS_FINITE;
         LutEntry64 ea, eb;
@@ -98,11 +131,10 @@ __device__ __forceinline__ void init_lut64(SM& s, const FmtDesc& fa, const FmtDe
 }
 
 // Decode the raw words of a chunk into double operands, packed exponent pairs and sign bit masks.
-template <int EK, class SM>
-__device__ __forceinline__ void store_chunk64(SM& sm, const RawChunk<EK>& raw, int flag, int tid) {
+template <int EK, class SM, class PL>
+__device__ __forceinline__ void store_chunk64(SM& sm, PL& s, const RawChunk<EK>& raw, int flag, int tid) {
     using E = Elem<EK>;
     using R = RawChunk<EK>;
-    auto& s = sm.pl;
     uint32_t spec = 0u;
 #pragma unroll
     for (int it = 0; it < R::PER_THREAD; ++it) {
@@ -156,8 +188,35 @@ __device__ __forceinline__ void store_chunk64(SM& sm, const RawChunk<EK>& raw, i
 // thread grid read 256 contiguous bytes of B operands per 16-byte load.
 __device__ __forceinline__ int col_of(int tx, int c) { return (c >> 1) * (BN / 2) + tx * 2 + (c & 1); }
 
+// Largest exponent sum of the products of one block (pass 1 of Algorithm 7 without the accumulator), two elements
+// per instruction: lane 0 holds the even elements' maximum, lane 1 the odd ones'.
+template <int L>
+__device__ __forceinline__ void product_exponents(const uint32_t* ea_p, const uint32_t* eb_p, uint32_t (&emp)[TM][TN]) {
+#pragma unroll
+    for (int r = 0; r < TM; ++r)
+#pragma unroll
+        for (int c = 0; c < TN; ++c) emp[r][c] = 0u;
+#pragma unroll
+    for (int kp = 0; kp < L / 2; ++kp) {
+        const uint4 ea0 = *reinterpret_cast<const uint4*>(ea_p + kp * BM);
+        const uint2 eb0 = *reinterpret_cast<const uint2*>(eb_p + kp * BN);
+        const uint2 eb1 = *reinterpret_cast<const uint2*>(eb_p + kp * BN + BN / 2);
+        const uint32_t ea[TM] = {ea0.x, ea0.y, ea0.z, ea0.w};
+        const uint32_t ebv[TN] = {eb0.x, eb0.y, eb1.x, eb1.y};
+#pragma unroll
+        for (int r = 0; r < TM; ++r)
+#pragma unroll
+            for (int c = 0; c < TN; ++c) emp[r][c] = __viaddmax_s16x2(ea[r], ebv[c], emp[r][c]);
+    }
+}
+
+// One CTA per SM, 512 threads, a 4 x 4 micro-tile per thread.  The FP64 pipe is the bound (one fma.rm.f64 per term),
+// so everything else is arranged to run beside it: the staged planes are double-buffered (the next chunk is decoded
+// between two barriers while its raw words were fetched a chunk earlier), and the product-exponent pass of block
+// n + 1 is fused, instruction by instruction, into the multiply-add pass of block n - the integer pipe works in
+// the issue slots that the FP64 pipe leaves free.
 template <int EK, int L, int RHO, bool PROMOTE, bool ST>
-__global__ void __launch_bounds__(NT, 2) tfdpa64_kernel(DevModel m, GemmArgs g) {
+__global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) {
     using E = Elem<EK>;
     constexpr bool ACC16 = RHO == RHO_RNE_FP16;
     constexpr int NBLK = KC / L;
@@ -167,7 +226,6 @@ __global__ void __launch_bounds__(NT, 2) tfdpa64_kernel(DevModel m, GemmArgs g) 
     using SM = Smem64<EK>;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     SM& sm = *reinterpret_cast<SM*>(smem_raw);
-    auto& s = sm.pl;
 
     const int tid = threadIdx.x;
     const int tx = tid % 16, ty = tid / 16;
@@ -177,7 +235,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa64_kernel(DevModel m, GemmArgs g) 
     const int MAGIC_K = ((1023 + 52 - m.F - CB) << 20) | 0x00080000;
 
     init_lut64<EK>(sm, fa, fb, tid);
-    if (tid == 0) sm.special[0] = sm.special[1] = 0;
+    if (tid == 0) sm.special[0] = sm.special[1] = sm.special[2] = 0;
 
     uint32_t cw[TM][TN];                                // the accumulator of each output: a finite FP32 / FP16 word
     uint32_t sp_nan = 0u, sp_pinf = 0u, sp_ninf = 0u;   // per output (bit r * TN + c): NaN / +inf / -inf seen so far
@@ -202,18 +260,28 @@ __global__ void __launch_bounds__(NT, 2) tfdpa64_kernel(DevModel m, GemmArgs g) 
             cw[r][c] = w;
         }
 
+    RawChunk<EK> raw;
+    load_chunk<EK>(raw, g, row0, col0, 0, tid);
+    __syncthreads();                                    // tables and flags are ready
+    store_chunk64<EK>(sm, sm.pl[0], raw, 0, tid);
+    if (KC < g.K) load_chunk<EK>(raw, g, row0, col0, KC, tid);
+    __syncthreads();
+    uint32_t emp[TM][TN];                               // product exponents of the block that comes next
+    product_exponents<L>(&sm.pl[0].a_exp2[0][ty * TM], &sm.pl[0].b_exp2[0][tx * 2], emp);
+
     int chunk = 0;
     for (int64_t k0 = 0; k0 < g.K; k0 += KC, ++chunk) {
-        __syncthreads();
-        {
-            RawChunk<EK> raw;
-            load_chunk<EK>(raw, g, row0, col0, k0, tid);
-            store_chunk64<EK>(sm, raw, chunk & 1, tid);
+        auto& s = sm.pl[chunk & 1];
+        auto& nx = sm.pl[(chunk + 1) & 1];
+        // decode chunk n + 1 into the other buffer (its raw words arrived during the previous iteration), fetch n + 2
+        if (tid == 0) sm.special[(chunk + 2) % 3] = 0;  // last read a chunk ago, next written after the coming barrier
+        __syncthreads();                                // every warp has left the other buffer
+        if (k0 + KC < g.K) {
+            store_chunk64<EK>(sm, nx, raw, (chunk + 1) % 3, tid);
+            if (k0 + 2 * KC < g.K) load_chunk<EK>(raw, g, row0, col0, k0 + 2 * KC, tid);
         }
-        __syncthreads();
-        const int flag = chunk & 1;
-        if (tid == 0) sm.special[(chunk + 1) & 1] = 0;
-        const bool chunk_special = sm.special[flag] != 0;
+        __syncthreads();                                // the other buffer is complete
+        const bool chunk_special = sm.special[chunk % 3] != 0;
 
         // ST-FDPA (Algorithm 8): Exp(alpha) of this thread's rows and Exp(beta) of its columns for this block of 32
         int sa_exp[ST ? TM : 1], sb_exp[ST ? TN : 1];
@@ -262,68 +330,69 @@ __global__ void __launch_bounds__(NT, 2) tfdpa64_kernel(DevModel m, GemmArgs g) 
                     }
             }
 
+            // ---- e_max = max(Exp(c), product exponents) and the accumulator term:
+            // acc = 1.5 * 2^52 * q + floor(c' / q) * q, c' = c with the lowest mantissa bit of its double set (never on
+            // the grid: a negative c floors to the one's complement), then + 1 if c < 0.
+            // ST: the products are compared against Exp(c) minus the block's scale exponents, c is scaled likewise.
             double acc[TM][TN];
+#pragma unroll
+            for (int r = 0; r < TM; ++r)
+#pragma unroll
+                for (int c = 0; c < TN; ++c) {
+                    const uint32_t field = ACC16 ? (cw[r][c] >> 10) & 0x1Fu : (cw[r][c] >> 23) & 0xFFu;
+                    int rel = int(max(field, 1u)) + (CB - (ACC16 ? 15 : 127));
+                    if (ST) rel -= sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0];
+                    const int emax = __vimax3_s32(int(emp[r][c] & 0xFFFFu), int(emp[r][c] >> 16), rel);     // e_max + CB
+                    const double magic = __hiloint2double(emax * (1 << 20) + MAGIC_K, 0);
+                    double cd = ACC16 ? double(__half2float(__ushort_as_half((unsigned short)cw[r][c]))) : double(__uint_as_float(cw[r][c]));
+                    if (ST) cd = __dmul_rn(cd, pow2d(-(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0])));
+                    cd = __hiloint2double(__double2hiint(cd), __double2loint(cd) | 1);
+                    const double a0 = __dadd_rd(cd, magic);
+                    const long long bitsum = __double_as_longlong(a0) + (long long)(cw[r][c] >> (ACC16 ? 15 : 31));
+                    acc[r][c] = __longlong_as_double(bitsum);
+                }
+            // ---- one fused multiply-add per term, rounding toward minus infinity onto the grid of q; beside it the
+            // product exponents of the block that follows (the next chunk's first block after this chunk's last) ----
             {
-                // ---- pass 1: e_max = max(Exp(c), max_k(Exp(a_k) + Exp(b_k))), two elements per instruction.
-                // ST: the products are compared against Exp(c) minus the block's scale exponents.
-                uint32_t em2[TM][TN];
+                const double* a_p = &s.a_d[kb][ty * TM];
+                const double* b_p = &s.b_d[kb][tx * 2];
+                const bool same = blk + 1 < NBLK;
+                const uint32_t* ea_p = same ? &s.a_exp2[(kb + L) / 2 < KC / 2 ? (kb + L) / 2 : 0][ty * TM] : &nx.a_exp2[0][ty * TM];
+                const uint32_t* eb_p = same ? &s.b_exp2[(kb + L) / 2 < KC / 2 ? (kb + L) / 2 : 0][tx * 2] : &nx.b_exp2[0][tx * 2];
 #pragma unroll
                 for (int r = 0; r < TM; ++r)
 #pragma unroll
-                    for (int c = 0; c < TN; ++c) {
-                        const uint32_t field = ACC16 ? (cw[r][c] >> 10) & 0x1Fu : (cw[r][c] >> 23) & 0xFFu;
-                        int rel = int(max(field, 1u)) + (CB - (ACC16 ? 15 : 127));
-                        if (ST) rel -= sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0];
-                        em2[r][c] = uint32_t(rel) * 0x10001u;
+                    for (int c = 0; c < TN; ++c) emp[r][c] = 0u;
+#pragma unroll
+                for (int kq = 0; kq < L; ++kq) {
+                    double av[TM], bv[TN];
+#pragma unroll
+                    for (int r = 0; r < TM; r += 2) {
+                        const double2 t = *reinterpret_cast<const double2*>(a_p + kq * BM + r);
+                        av[r] = t.x; av[r + 1] = t.y;
                     }
-#pragma unroll 4
-                for (int kp = kb / 2; kp < (kb + L) / 2; ++kp) {
-                    const uint4 ea0 = *reinterpret_cast<const uint4*>(&s.a_exp2[kp][ty * TM]);
-                    const uint4 ea1 = *reinterpret_cast<const uint4*>(&s.a_exp2[kp][ty * TM + 4]);
-                    const uint2 eb0 = *reinterpret_cast<const uint2*>(&s.b_exp2[kp][tx * 2]);
-                    const uint2 eb1 = *reinterpret_cast<const uint2*>(&s.b_exp2[kp][BN / 2 + tx * 2]);
-                    const uint32_t ea[TM] = {ea0.x, ea0.y, ea0.z, ea0.w, ea1.x, ea1.y, ea1.z, ea1.w};
-                    const uint32_t ebv[TN] = {eb0.x, eb0.y, eb1.x, eb1.y};
+                    {
+                        const double2 t0 = *reinterpret_cast<const double2*>(b_p + kq * BN);
+                        const double2 t1 = *reinterpret_cast<const double2*>(b_p + kq * BN + BN / 2);
+                        bv[0] = t0.x; bv[1] = t0.y; bv[2] = t1.x; bv[3] = t1.y;
+                    }
+                    uint32_t ea[TM], ebv[TN];
+                    if ((kq & 1) == 0) {
+                        const int kp = kq / 2;
+                        const uint4 ea0 = *reinterpret_cast<const uint4*>(ea_p + kp * BM);
+                        const uint2 eb0 = *reinterpret_cast<const uint2*>(eb_p + kp * BN);
+                        const uint2 eb1 = *reinterpret_cast<const uint2*>(eb_p + kp * BN + BN / 2);
+                        ea[0] = ea0.x; ea[1] = ea0.y; ea[2] = ea0.z; ea[3] = ea0.w;
+                        ebv[0] = eb0.x; ebv[1] = eb0.y; ebv[2] = eb1.x; ebv[3] = eb1.y;
+                    }
 #pragma unroll
                     for (int r = 0; r < TM; ++r)
 #pragma unroll
-                        for (int c = 0; c < TN; ++c) em2[r][c] = __viaddmax_s16x2(ea[r], ebv[c], em2[r][c]);
+                        for (int c = 0; c < TN; ++c) {
+                            acc[r][c] = __fma_rd(av[r], bv[c], acc[r][c]);
+                            if ((kq & 1) == 0) emp[r][c] = __viaddmax_s16x2(ea[r], ebv[c], emp[r][c]);
+                        }
                 }
-                // ---- accumulator term: acc = 1.5 * 2^52 * q + floor(c' / q) * q, c' = c with the lowest mantissa bit of
-                // its double set (never on the grid: a negative c floors to the one's complement), then + 1 if c < 0
-#pragma unroll
-                for (int r = 0; r < TM; ++r)
-#pragma unroll
-                    for (int c = 0; c < TN; ++c) {
-                        const int emax = max(int(em2[r][c] & 0xFFFFu), int(em2[r][c] >> 16));     // e_max + CB
-                        const double magic = __hiloint2double(emax * (1 << 20) + MAGIC_K, 0);
-                        double cd = ACC16 ? double(__half2float(__ushort_as_half((unsigned short)cw[r][c]))) : double(__uint_as_float(cw[r][c]));
-                        if (ST) cd = __dmul_rn(cd, pow2d(-(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0])));
-                        cd = __hiloint2double(__double2hiint(cd), __double2loint(cd) | 1);
-                        const double a0 = __dadd_rd(cd, magic);
-                        const long long bitsum = __double_as_longlong(a0) + (long long)(cw[r][c] >> (ACC16 ? 15 : 31));
-                        acc[r][c] = __longlong_as_double(bitsum);
-                    }
-            }
-            // ---- pass 2: one fused multiply-add per term, rounding toward minus infinity onto the grid of q ----
-#pragma unroll 2
-            for (int kk = kb; kk < kb + L; ++kk) {
-                double av[TM], bv[TN];
-#pragma unroll
-                for (int r = 0; r < TM; r += 2) {
-                    const double2 t = *reinterpret_cast<const double2*>(&s.a_d[kk][ty * TM + r]);
-                    av[r] = t.x; av[r + 1] = t.y;
-                }
-                {
-                    const double2 t0 = *reinterpret_cast<const double2*>(&s.b_d[kk][tx * 2]);
-                    const double2 t1 = *reinterpret_cast<const double2*>(&s.b_d[kk][BN / 2 + tx * 2]);
-                    bv[0] = t0.x; bv[1] = t0.y; bv[2] = t1.x; bv[3] = t1.y;
-                }
-#pragma unroll
-                for (int r = 0; r < TM; ++r)
-#pragma unroll
-                    for (int c = 0; c < TN; ++c)
-                        asm("fma.rm.f64 %0, %1, %2, %0;" : "+d"(acc[r][c]) : "d"(av[r]), "d"(bv[c]));
             }
             // ---- sign corrections, rho ----
             const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
