@@ -47,6 +47,7 @@ constexpr int BM = 128, BN = 64, TM = 8, TN = 4, KC = 32, NT = 256;
 constexpr int EB = 512;            // bias of a staged element exponent
 constexpr int CB = 2 * EB;         // bias of an exponent sum and of the accumulator exponent
 constexpr int FP_SHIFT = 8;        // FP32 summation path: the B operands are scaled by 2^-FP_SHIFT (see pass 2)
+constexpr int FP_EMAX_CLAMP = 100; // FP32 summation path: largest e_max + g that the sum register's exponent carries
 
 enum ElemKind : int { EK_LUT8 = 0, EK_F16 = 1, EK_BF16 = 2, EK_TF32 = 3 };
 
@@ -358,7 +359,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
     static_assert(KC % L == 0 && L % 2 == 0, "blocks tile the chunk; pass 1 handles pairs of elements");
     static_assert(!ST || L == KC, "ST-FDPA: one scale factor pair per block of 32 (Algorithm 8)");
     // FP32 summation path (8-bit inputs with F <= 13): aligned terms stay below 2^15 and block sums below 2^21, so the
-    // whole of pass 2 runs exactly on the FP32 pipe, two instructions per term (see pass 2 below).  Its staged planes
+    // whole of pass 2 runs exactly on the FP32 pipe, one instruction per term (see pass 2 below).  Its staged planes
     // are small enough for two buffers: the next chunk is decoded while the current one is computed, one barrier per chunk.
     constexpr bool FPSUM = TfdpaFpsum<EK, F>::value;
     constexpr bool DB = FPSUM;
@@ -519,20 +520,21 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
                     if (NSUM == 2) S1[NSUM == 2 ? r : 0][NSUM == 2 ? c : 0] = 0;
                     emax[r][c] += guard;
                     if (FPSUM) {
-                        // The sum lives in an FP32 register as 1.5 * 2^23 + S: in [2^23, 2^24) one ulp is one unit of S,
-                        // so integers add exactly and adding a fraction with rounding toward minus infinity is a floor.
-                        S0[r][c] += 0x4B400000;
-                        // 2^(FP_SHIFT - (e_max + g)) as an FP32 word (the B operands carry 2^-FP_SHIFT): e_max + g lies in
-                        // [-25, 131], so the exponent field stays inside 1..254 and e_max can be read back from it
-                        emax[r][c] = (127 + FP_SHIFT + CB - emax[r][c]) << 23;
+                        // The sum lives in an FP32 register as (1.5 * 2^23 + S) * u, u = 2^(e_max + g - FP_SHIFT) the
+                        // value of one unit of S in the scale of the staged operands: in [2^23 u, 2^24 u) one ulp is u,
+                        // so adding a product with rounding toward minus infinity floors it onto the grid of S.
+                        // For e_max above FP_EMAX_CLAMP (only a huge accumulator gets there) the exponent is clamped:
+                        // every product is far below one unit either way and floors to 0 or -1 as it should.
+                        const int ecl = min(emax[r][c], FP_EMAX_CLAMP + CB + guard);
+                        S0[r][c] += ((ecl + (150 - CB - FP_SHIFT)) << 23) | 0x00400000;
                     }
                 }
             // ---- pass 2: multiply, align, truncate, add ----
             if (FPSUM) {
-                // X_k * 2^-(d_k + g) = (A_op * 2^Exp(a)) * (B_op * 2^Exp(b)) * 2^-(e_max + g): the first product is exact
-                // in FP32 (19 significant bits), the fused multiply-add computes the second one exactly and rounds the
-                // sum once, toward minus infinity: S <- S + floor(X_k * 2^-(d_k + g)), the same one's-complement term
-                // as the arithmetic shift of the integer path.
+                // S * u + (A_op * 2^Exp(a)) * (B_op * 2^(Exp(b) - FP_SHIFT)) = (S + X_k * 2^-(d_k + g)) * u: the fused
+                // multiply-add forms it exactly and rounds once, toward minus infinity, onto multiples of u:
+                // S <- S + floor(X_k * 2^-(d_k + g)), the same one's-complement term as the arithmetic shift of the
+                // integer path.  One instruction per term; the alignment scale is the exponent of the sum register.
 #pragma unroll 4
                 for (int kk = kb; kk < kb + L; ++kk) {
                     const float4 oa0 = *reinterpret_cast<const float4*>(&s.a_op[kk][ty * TM]);
@@ -543,19 +545,17 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
 #pragma unroll
                     for (int r = 0; r < TM; ++r)
 #pragma unroll
-                        for (int c = 0; c < TN; ++c) {
-                            const float xs = __fmul_rn(oav[r], obv[c]);
-                            float sum = __int_as_float(S0[r][c]);
-                            asm("fma.rm.f32 %0, %1, %2, %0;" : "+f"(sum) : "f"(xs), "f"(__int_as_float(emax[r][c])));
-                            S0[r][c] = __float_as_int(sum);
-                        }
+                        for (int c = 0; c < TN; ++c)
+                            S0[r][c] = __float_as_int(__fmaf_rd(oav[r], obv[c], __int_as_float(S0[r][c])));
                 }
+                // back to the integer sum; e_max + g from the exponent field, or Exp(c) + g where it was clamped
 #pragma unroll
                 for (int r = 0; r < TM; ++r)
 #pragma unroll
                     for (int c = 0; c < TN; ++c) {
-                        S0[r][c] -= 0x4B400000;
-                        emax[r][c] = 127 + FP_SHIFT + CB - int(uint32_t(emax[r][c]) >> 23);
+                        const int bits = S0[r][c];
+                        S0[r][c] = bits - ((bits & 0x7F800000) | 0x00400000);
+                        emax[r][c] = max((bits >> 23) - (150 - CB - FP_SHIFT), acc[r][c].ce + guard);
                     }
             } else {
 #pragma unroll 2
