@@ -133,9 +133,33 @@ int mmasim_dot_batch(const mmasim_model* model, int64_t n, int64_t K,
                      const void* A, const void* B, const void* C, void* D, void* stream);
 
 /* mmasim_gemm_ex on HOST buffers: allocates device memory, copies A, B, C (and scales) to the device, runs,
- * copies D back and frees; synchronous.  Fields of opts that are pointers are host pointers here. */
+ * copies D back and frees; synchronous.  Fields of opts that are pointers are host pointers here.
+ * The device buffers are stream-ordered allocations (cudaMallocAsync) on a stream of the call's own; the device's
+ * default memory pool is told to keep up to 1 GiB between calls, so repeated calls do not pay for allocation
+ * (cudaMemPoolTrimTo on that pool returns the memory).  Pinned host buffers make the copies asynchronous. */
 int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
                      const void* A, const void* B, const void* C, void* D, const mmasim_gemm_opts* opts);
+
+/* The hardware's own matrix multiply-accumulate, for differential runs of the models against the machine they
+ * describe (Section 3.1, Step 4; Section 3.2: an MMA interface is D = MMA(A, B, C) on one instruction).  Runs the
+ * warp-level `mma.sync` instruction of the given kind on every tile of 16 rows of A (8 for MMASIM_HW_F64):
+ *   D (M x 8) = A (M x K, row-major) * B^T (B is 8 x K, row-major, shared by all tiles) + C (M x 8, may be NULL = +0),
+ * K a multiple of the instruction's K; a longer K chains instructions through the accumulator in ascending k, as
+ * Algorithm 5 does.  Element layouts as for mmasim_gemm (TF32 in 32-bit words, FP8 one element per byte); all
+ * pointers are device pointers; M a multiple of the tile height.  Results are whatever the B200 computes:
+ * comparing them with a model is the caller's business. */
+typedef enum {
+    MMASIM_HW_F16_F32 = 0,      /* m16n8k16, FP16 inputs, FP32 accumulator */
+    MMASIM_HW_F16_F16 = 1,      /* m16n8k16, FP16 inputs, FP16 accumulator */
+    MMASIM_HW_BF16_F32 = 2,     /* m16n8k16 */
+    MMASIM_HW_TF32_F32 = 3,     /* m16n8k8 */
+    MMASIM_HW_E4M3_F32 = 4,     /* m16n8k32 */
+    MMASIM_HW_E5M2_F32 = 5,     /* m16n8k32 */
+    MMASIM_HW_F64 = 6,          /* m8n8k4, FP64 throughout */
+    MMASIM_HW_F16_F32_K8 = 7,   /* m16n8k8 */
+    MMASIM_HW_TF32_F32_K4 = 8   /* m16n8k4 */
+} mmasim_hw_kind;
+int mmasim_hw_mma(int kind, int64_t M, int64_t K, const void* A, const void* B, const void* C, void* D, void* stream);
 
 /* Integer-issue micro-benchmark used as the roofline denominator (no counterpart in the paper): launches
  * `blocks` CTAs of 256 threads, each thread running `iters` rounds of 8 independent dependent-chain integer

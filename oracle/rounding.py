@@ -5,8 +5,9 @@ RNE-FP32, RNE-FP16) and the RNE roundings of Algorithms 1, 3 and 6.
 
 Readings where the paper is silent:
 * gradual underflow everywhere (only the CDNA2 model flushes, Section 4.1);
-* on overflow the round-to-zero conversions saturate to the largest finite
-  value of the target (IEEE-754 roundTowardZero); round-to-nearest gives inf;
+* on overflow every conversion gives +-inf, the round-to-zero ones too (they
+  do not saturate at the largest finite value: the B200's mma.sync, which the
+  Blackwell rows describe, returns +-inf);
 * RZ-E8M13 is an FP32 word whose low 10 mantissa bits are zero: 8 exponent
   bits, 13 mantissa bits, subnormals on a 2**-139 grid.
 """
@@ -56,9 +57,7 @@ def round_dyadic(m: int, e: int, ebits: int, mbits: int, bias: int, mode: str,
         q += 1
     if n >> mbits:                              # normal number
         field = q + mbits + bias
-        if field >= top:                        # overflow
-            if mode == "RZ":
-                return (sign << sign_shift) | ((top - 1) << mbits) | ((1 << mbits) - 1)
+        if field >= top:                        # overflow: +-inf in both modes
             return (sign << sign_shift) | (top << mbits)
         return (sign << sign_shift) | (field << mbits) | (n & ((1 << mbits) - 1))
     return (sign << sign_shift) | n             # subnormal or zero (field 0)

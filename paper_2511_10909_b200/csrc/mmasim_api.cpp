@@ -231,10 +231,22 @@ int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
     const size_t sfa_bytes = g.sfa ? size_t(M * g.ld_sfa) : 0, sfb_bytes = g.sfb ? size_t(N * g.ld_sfb) : 0;
     void *dA = nullptr, *dB = nullptr, *dC = nullptr, *dD = nullptr, *dSA = nullptr, *dSB = nullptr, *dRS = nullptr, *dCS = nullptr;
     cudaError_t err = cudaSuccess;
+    // Stream-ordered allocations on a stream of this call's own: after the first call the buffers come out of the
+    // device's default memory pool (which keeps up to 1 GiB between calls), copies from pinned host memory overlap
+    // nothing but also wait for nothing, and the call synchronises once, at the end.
+    cudaStream_t stream = nullptr;
+    err = cudaStreamCreateWithFlags(&stream, cudaStreamNonBlocking);
+    if (err == cudaSuccess) {
+        int dev = 0;
+        cudaMemPool_t pool = nullptr;
+        unsigned long long keep = 1ull << 30;
+        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess)
+            cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+    }
     auto up = [&](void** dst, const void* src, size_t bytes) {
         if (err != cudaSuccess || !src || !bytes) return;
-        err = cudaMalloc(dst, bytes);
-        if (err == cudaSuccess) err = cudaMemcpy(*dst, src, bytes, cudaMemcpyHostToDevice);
+        err = cudaMallocAsync(dst, bytes, stream);
+        if (err == cudaSuccess) err = cudaMemcpyAsync(*dst, src, bytes, cudaMemcpyHostToDevice, stream);
     };
     up(&dA, A, a_bytes);
     up(&dB, B, b_bytes);
@@ -243,17 +255,23 @@ int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
     up(&dSB, g.sfb, sfb_bytes);
     up(&dRS, g.row_scale, size_t(M) * 4);
     up(&dCS, g.col_scale, size_t(N) * 4);
-    if (err == cudaSuccess) err = cudaMalloc(&dD, d_bytes);
+    if (err == cudaSuccess) err = cudaMallocAsync(&dD, d_bytes, stream);
     if (err == cudaSuccess) {
         g.A = dA; g.B = dB; g.C = dC; g.D = dD;
         g.sfa = static_cast<const uint8_t*>(dSA);
         g.sfb = static_cast<const uint8_t*>(dSB);
         g.row_scale = static_cast<const float*>(dRS);
         g.col_scale = static_cast<const float*>(dCS);
-        st = run_gemm(model, g, opts ? opts->flags : 0, nullptr);
-        if (st == MMASIM_OK) err = cudaMemcpy(D, dD, d_bytes, cudaMemcpyDeviceToHost);
+        st = run_gemm(model, g, opts ? opts->flags : 0, stream);
+        if (st == MMASIM_OK) err = cudaMemcpyAsync(D, dD, d_bytes, cudaMemcpyDeviceToHost, stream);
     }
-    cudaFree(dA); cudaFree(dB); cudaFree(dC); cudaFree(dD); cudaFree(dSA); cudaFree(dSB); cudaFree(dRS); cudaFree(dCS);
+    if (stream) {
+        void* bufs[] = {dA, dB, dC, dD, dSA, dSB, dRS, dCS};
+        for (void* b : bufs) if (b) cudaFreeAsync(b, stream);
+        const cudaError_t e2 = cudaStreamSynchronize(stream);
+        if (err == cudaSuccess) err = e2;
+        cudaStreamDestroy(stream);
+    }
     if (err != cudaSuccess) {
         cudaGetLastError();
         set_error("mmasim_gemm_host: %s", cudaGetErrorString(err));
@@ -265,6 +283,11 @@ int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
 int mmasim_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t* ops_per_round, void* stream) {
     if (!sink || !ops_per_round || blocks < 1 || iters < 1 || kind < 0) { set_error("mmasim_int_peak: bad argument"); return MMASIM_ERR_INVALID_ARG; }
     return launch_int_peak(kind, blocks, iters, sink, ops_per_round, static_cast<cudaStream_t>(stream));
+}
+
+int mmasim_hw_mma(int kind, int64_t M, int64_t K, const void* A, const void* B, const void* C, void* D, void* stream) {
+    if (!A || !B || !D) { set_error("mmasim_hw_mma: A, B and D must not be NULL"); return MMASIM_ERR_INVALID_ARG; }
+    return launch_hw_mma(kind, M, K, A, B, C, D, static_cast<cudaStream_t>(stream));
 }
 
 const char* mmasim_last_kernel(void) { return g_kernel; }

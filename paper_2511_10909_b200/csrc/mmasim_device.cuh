@@ -72,7 +72,7 @@ __device__ __forceinline__ AccDec decode_acc(uint32_t w, bool fp16) {
 
 // ---------------------------------------------------------------------------------------------------------
 // Table 2: convert the exact value (-1)^sign * mag * 2^e to a word.  mode_rne: nearest-even, else truncation.
-// Overflow: truncation saturates to the largest finite value, nearest-even gives infinity.  mag == 0 -> +0.
+// Overflow gives infinity in both modes (truncation does not saturate at the largest finite value).  mag == 0 -> +0.
 // `sticky` marks nonzero bits below mag's last bit (only the exact E-FDPA sum needs it).
 // ---------------------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t round_pack(uint32_t sign, uint64_t mag, int e, int ebits, int mbits, int bias,
@@ -109,10 +109,7 @@ __device__ __forceinline__ uint32_t round_pack(uint32_t sign, uint64_t mag, int 
     const uint32_t sbit = sign << (ebits + mbits);
     if (n >> mbits) {
         const int field = q + mbits + bias;
-        if (field >= int(top)) {
-            if (mode_rne) return sbit | (top << mbits);
-            return sbit | ((top - 1u) << mbits) | ((1u << mbits) - 1u);
-        }
+        if (field >= int(top)) return sbit | (top << mbits);
         return sbit | (uint32_t(field) << mbits) | (uint32_t(n) & ((1u << mbits) - 1u));
     }
     return sbit | uint32_t(n);
@@ -183,14 +180,17 @@ __device__ __forceinline__ uint32_t tfdpa_block(const uint32_t* a, const uint32_
     Special sp;
     sp.nan = scale_nan;
     sp.acc(dc);
-    int e_max = dc.exp;
+    // a term whose value is zero has no exponent: it takes no part in the maximum
+    constexpr int NO_EXP = -100000;
+    int e_max = dc.sig ? dc.exp : NO_EXP;
     for (int k = 0; k < L; ++k) {                                   // Step 1 exponents, Step 2 maximum
         sp.product(a[k], b[k]);
-        const int ek = dec_exp(a[k]) + dec_exp(b[k]) + scale_exp;
+        const int ek = (dec_sig(a[k]) && dec_sig(b[k])) ? dec_exp(a[k]) + dec_exp(b[k]) + scale_exp : NO_EXP;
         e_max = ek > e_max ? ek : e_max;
     }
     const int kind = sp.result();
     if (kind) return special_word(kind, fp16, true);
+    if (e_max == NO_EXP) return 0u;                                 // every term is zero
     int64_t S = 0;
     const int F = m.F, frac = m.frac;
     for (int k = 0; k < L; ++k) {                                   // Step 2: align, truncate, add
@@ -220,7 +220,8 @@ __device__ __forceinline__ uint32_t gst_block(const uint32_t* a, const uint32_t*
     const int ng = L / m.G;
     int64_t s[4];
     int e[4];
-    int e_max = dc.exp;
+    constexpr int NO_EXP = -100000;                                 // zero terms take no part in the maximum
+    int e_max = dc.sig ? dc.exp : NO_EXP;
     for (int g = 0; g < ng; ++g) {                                  // Step 1
         int p = 0;                                                  // units of 2^-2 (E2M1: Exp >= 0, 1 mantissa bit)
         for (int k = g * m.G; k < (g + 1) * m.G; ++k)
@@ -228,8 +229,9 @@ __device__ __forceinline__ uint32_t gst_block(const uint32_t* a, const uint32_t*
         const int j = (g * m.G) / m.k_block;
         s[g] = int64_t(p) * int64_t(dec_sig(sfa[j])) * int64_t(dec_sig(sfb[j]));
         e[g] = dec_exp(sfa[j]) + dec_exp(sfb[j]);
-        e_max = e[g] > e_max ? e[g] : e_max;
+        if (s[g] != 0) e_max = e[g] > e_max ? e[g] : e_max;
     }
+    if (e_max == NO_EXP) return 0u;
     int64_t S = 0;
     for (int g = 0; g < ng; ++g) S += rz_scale(s[g], (e[g] - e_max) + m.F - m.frac);   // Step 2
     const int64_t sc = dc.sign ? -int64_t(dc.sig) : int64_t(dc.sig);
@@ -261,7 +263,7 @@ __device__ __forceinline__ uint32_t tr_block(const uint32_t* a, const uint32_t* 
             const int ek = dec_exp(a[k]) + dec_exp(b[k]);
             if (product_overflows(sk, ek, m.frac)) sp.add_inf(sk < 0);
             const int g = grouped ? (k & 1) : 0;
-            e_grp[g] = ek > e_grp[g] ? ek : e_grp[g];
+            if (sk != 0) e_grp[g] = ek > e_grp[g] ? ek : e_grp[g];  // zero products take no part in the maximum
         }
     }
     const int kind = sp.result();
@@ -276,15 +278,16 @@ __device__ __forceinline__ uint32_t tr_block(const uint32_t* a, const uint32_t* 
     }
     int e_max;
     int64_t T;
-    if (grouped) {                                                  // Algorithm 11, Step 3
+    if (grouped) {                                                  // Algorithm 11, Step 3 (an all-zero group has T = 0)
         e_max = e_grp[0] > e_grp[1] ? e_grp[0] : e_grp[1];
         T = rd_scale(T_grp[0], e_grp[0] - e_max) + rd_scale(T_grp[1], e_grp[1] - e_max);
     } else {
         e_max = e_grp[0];
         T = T_grp[0];
     }
-    const int E = e_max > dc.exp ? e_max : dc.exp;
     const int64_t sc = dc.sign ? -int64_t(dc.sig) : int64_t(dc.sig);
+    if (e_max == -100000) return rho_apply(m.rho, sc, dc.exp - 23);  // every product is zero: the block returns c (or +0)
+    const int E = (dc.sig && dc.exp > e_max) ? dc.exp : e_max;
     int64_t T2, sc2;
     if (m.inner_round == 1) {                                       // hypothetical RZ variant (Section 6.2.4)
         T2 = rz_scale(T, (e_max - E) + F2 - F);

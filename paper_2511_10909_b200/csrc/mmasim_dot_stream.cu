@@ -149,9 +149,11 @@ __device__ __forceinline__ uint32_t tfdpa_dot(const Rows& rows, int K, int F, ui
         load_raw<E::BYTES, L>(rows, false, k0, ra);
         load_raw<E::BYTES, L>(rows, true, k0, rb);
         // Step 1: exact products (as FP32 for FP16 inputs, whose products stay inside the FP32 range; as FP64
-        // otherwise) and the largest exponent sum Exp(a) + Exp(b), with Exp = max(field, 1) - bias.
+        // otherwise) and the largest exponent sum Exp(a) + Exp(b), with Exp = max(field, 1) - bias, over the products
+        // that are not zero (a zero term has no exponent): lanes of a zero product are masked to 0 before the maximum.
         float pf[E::BYTES == 2 && EK == EK_F16 ? L : 1];
         double pd[EK == EK_F16 ? 1 : L];
+        constexpr int NO_EXP = -100000;
         int e_prod;
         if (E::BYTES == 2) {
             constexpr uint32_t EXPM = ((1u << E::EBITS) - 1u) << E::MBITS, ONE = 1u << E::MBITS;
@@ -160,7 +162,9 @@ __device__ __forceinline__ uint32_t tfdpa_dot(const Rows& rows, int K, int F, ui
             for (int q = 0; q < NRAW; ++q) {
                 const uint32_t ea = __vmaxu2(ra[q] & (EXPM * 0x10001u), ONE * 0x10001u);
                 const uint32_t eb = __vmaxu2(rb[q] & (EXPM * 0x10001u), ONE * 0x10001u);
-                mx = __vmaxu2(mx, ea + eb);               // field sums stay below 2^16: no carry between the lanes
+                // 1 per lane where both elements are nonzero, widened to a lane mask
+                const uint32_t live = __vminu2(__vminu2(ra[q] & 0x7FFF7FFFu, rb[q] & 0x7FFF7FFFu), 0x00010001u) * 0xFFFFu;
+                mx = __vmaxu2(mx, (ea + eb) & live);      // field sums stay below 2^16: no carry between the lanes
                 if (EK == EK_F16) {
                     const float2 fa = __half22float2(*reinterpret_cast<const __half2*>(&ra[q]));
                     const float2 fb = __half22float2(*reinterpret_cast<const __half2*>(&rb[q]));
@@ -171,22 +175,25 @@ __device__ __forceinline__ uint32_t tfdpa_dot(const Rows& rows, int K, int F, ui
                     pd[2 * q + 1 < L ? 2 * q + 1 : 0] = __dmul_rn(double(__uint_as_float(ra[q] & 0xFFFF0000u)), double(__uint_as_float(rb[q] & 0xFFFF0000u)));
                 }
             }
-            e_prod = int(max(mx & 0xFFFFu, mx >> 16) >> E::MBITS) - 2 * E::BIAS;
+            const uint32_t m1 = max(mx & 0xFFFFu, mx >> 16);
+            e_prod = m1 ? int(m1 >> E::MBITS) - 2 * E::BIAS : NO_EXP;
         } else {
             uint32_t mx = 0u;
 #pragma unroll
             for (int k = 0; k < L; ++k) {
-                mx = max(mx, max((ra[k] >> 23) & 0xFFu, 1u) + max((rb[k] >> 23) & 0xFFu, 1u));
+                const uint32_t xa = ra[k] & 0x7FFFE000u, xb = rb[k] & 0x7FFFE000u;
+                const uint32_t es = max(xa >> 23, 1u) + max(xb >> 23, 1u);
+                mx = max(mx, (xa && xb) ? es : 0u);
                 pd[EK == EK_F16 ? 0 : k] = __dmul_rn(double(__uint_as_float(ra[k] & 0xFFFFE000u)), double(__uint_as_float(rb[k] & 0xFFFFE000u)));
             }
-            e_prod = int(mx) - 2 * E::BIAS;
+            e_prod = mx ? int(mx) - 2 * E::BIAS : NO_EXP;
         }
         const uint32_t cfield = ACC16 ? (cw >> 10) & 0x1Fu : (cw >> 23) & 0xFFu;
-        const int e_c = int(max(cfield, 1u)) - (ACC16 ? 15 : 127);
+        const int e_c = (cw & (ACC16 ? 0x7FFFu : 0x7FFFFFFFu)) ? int(max(cfield, 1u)) - (ACC16 ? 15 : 127) : NO_EXP;
         const double cd = ACC16 ? double(__half2float(__ushort_as_half((unsigned short)cw))) : double(__uint_as_float(cw));
 
         // Step 2: e_max over the L + 1 terms, alignment and sign-magnitude truncation to F fractional bits, exact sum
-        const int emax = max(e_prod, e_c);
+        const int emax = max(max(e_prod, e_c), -400);     // every term zero: any exponent will do
         const double scale = __hiloint2double((1023 + F - emax) << 20, 0);
         double S0 = trunc_scaled(cd, scale, __double2hiint(cd)), S1 = 0.0;
 #pragma unroll
@@ -197,11 +204,12 @@ __device__ __forceinline__ uint32_t tfdpa_dot(const Rows& rows, int K, int F, ui
             if (k & 1) S1 += tk; else S0 += tk;
         }
         // Step 3: d = rho(S * 2^(e_max - F)).  S (|S| < 2^33) times a power of two is exact in FP64, so rho is one
-        // conversion: RZ-FP32 saturates at the largest finite number, RNE-FP16 overflows to infinity, both keep
+        // conversion: both overflow to infinity (for RZ-FP32 the test is explicit: cvt.rz saturates), both keep
         // subnormal results; an exact zero is +0.  A sum that is not finite gives the NaN / infinity of Section 4.2.
         const double S = S0 + S1;                         // S1 starts from +0, so an all-zero sum is +0
         const double v = __dmul_rn(S, __hiloint2double((1023 + emax - F) << 20, 0));
         if (ACC16) cw = (v != v) ? 0x7FFFu : uint32_t(__half_as_ushort(__double2half(v)));
+        else if (fabs(v) >= 3.402823669209385e38) cw = (__double2hiint(v) < 0 ? 0xFF800000u : 0x7F800000u);   // |v| >= 2^128: overflow
         else cw = (v != v) ? 0x7FFFFFFFu : __float_as_uint(__double2float_rz(v));
     }
     return cw;

@@ -12,14 +12,18 @@
 //
 // RZ_F is sign-magnitude truncation, floor is not: negative terms are made to floor to the one's complement
 // -floor(|x|) - 1 of the wanted value by an offset far below the term's own granularity but never zero: the staged
-// B operand is b + sign(b) * 2^(Exp(b) - mbits_b - 30) (a zero b becomes that offset alone), and a zero a is staged as
-// sign(a) * 2^(Exp_min(a) - 60).  Every term whose sign bits differ then floors to -floor(|x|) - 1 (zero terms to
-// -1), every other term to floor(|x|), and the number of sign-differing terms of the block, a population count over
-// per-row / per-column sign bit masks, is added back once per block, as an integer added to the bit pattern of acc.
-// The accumulator operand c gets the same treatment: its double has bit 0 of the mantissa set.
+// B operand is b + sign(b) * 2^(Exp(b) - mbits_b - 30).  Every nonzero term whose sign bits differ then floors to
+// -floor(|x|) - 1, every other term to floor(|x|), and the number of nonzero sign-differing terms of the block, a
+// population count over per-row / per-column sign and nonzero bit masks, is added back once per block, as an integer
+// added to the bit pattern of acc.  The accumulator operand c gets the same treatment: its double has bit 0 of the
+// mantissa set.  Zero elements (and the stand-ins of infinities and NaNs) are staged as 0: their products vanish.
 //
-// rho (Table 2) is one conversion instruction per block and output: cvt.rz.f32.f64 (saturates at the largest finite
-// number, keeps subnormals) or cvt.rn.f16.f64 (overflows to infinity, which is recorded as a sticky special value).
+// A term whose value is zero has no exponent and takes no part in e_max: zero elements are staged with the exponent
+// word 0, far below every real exponent sum, and a zero c enters the maximum as 0 as well.
+//
+// rho (Table 2) is one conversion instruction per block and output: cvt.rz.f32.f64 (keeps subnormals; a result of
+// magnitude >= 2^128 is an overflow and becomes infinity) or cvt.rn.f16.f64; an infinity is recorded as a sticky
+// special value.
 // e_max is computed as in the integer kernels (fused add-max on two 16-bit lanes); NaN / infinity inputs use the same
 // sticky flags and rescan of the raw words (Section 4.2): their staged operands are the zero stand-ins.
 #pragma once
@@ -76,12 +80,11 @@ __device__ __forceinline__ void load_chunk(RawChunk<EK>& raw, const GemmArgs& g,
 }
 
 constexpr int G_OFF = 30;          // the B offset sits 30 bits below the element's last significand bit
-constexpr int A_TINY = 60;         // a zero a is 2^(Exp_min - 60)
 
 struct LutEntry64 {
     double op;          // staged operand
-    uint32_t exp;       // Exp(x) + EB (minimum exponent for non-finite inputs)
-    uint32_t bits;      // bit 0: sign; bit 1: infinity or NaN
+    uint32_t exp;       // Exp(x) + EB; 0 for zero, infinity and NaN
+    uint32_t bits;      // bit 0: sign; bit 1: infinity or NaN; bit 2: nonzero finite
 };
 
 template <int EK>
@@ -91,6 +94,7 @@ struct Planes64 {
     uint32_t a_exp2[KC / 2][BM];    // exponents of elements 2p (low half) and 2p + 1 (high half)
     uint32_t b_exp2[KC / 2][BN];
     uint32_t a_sgn[BM], b_sgn[BN];  // bit k of row r: sign of element k of the chunk
+    uint32_t a_nz[BM], b_nz[BN];    // bit k of row r: element k is finite and nonzero
 };
 
 template <int EK>
@@ -103,13 +107,13 @@ struct Smem64 {
 
 __device__ __forceinline__ double pow2d(int e) { return __hiloint2double((1023 + e) << 20, 0); }
 
-// Staged operand of one finite element sign * sig * 2^(exp - mbits) (sig = 0 included); see the header comment.
-__device__ __forceinline__ double operand_a(uint32_t sign, uint32_t sig, int exp, int mbits, int exp_min) {
-    const double mag = sig ? __dmul_rn(__uint2double_rn(sig), pow2d(exp - mbits)) : pow2d(exp_min - A_TINY);
+// Staged operand of one finite element sign * sig * 2^(exp - mbits); zero stays zero; see the header comment.
+__device__ __forceinline__ double operand_a(uint32_t sign, uint32_t sig, int exp, int mbits) {
+    const double mag = __dmul_rn(__uint2double_rn(sig), pow2d(exp - mbits));
     return sign ? -mag : mag;
 }
 __device__ __forceinline__ double operand_b(uint32_t sign, uint32_t sig, int exp, int mbits) {
-    const double mag = __dadd_rn(__dmul_rn(__uint2double_rn(sig), pow2d(exp - mbits)), pow2d(exp - mbits - G_OFF));
+    const double mag = sig ? __dadd_rn(__dmul_rn(__uint2double_rn(sig), pow2d(exp - mbits)), pow2d(exp - mbits - G_OFF)) : 0.0;
     return sign ? -mag : mag;
 }
 
@@ -119,12 +123,13 @@ __device__ __forceinline__ void init_lut64(SM& s, const FmtDesc& fa, const FmtDe
         const uint32_t da = decode_elem(fa, uint32_t(tid)), db = decode_elem(fb, uint32_t(tid));
         const bool fin_a = dec_cls(da) == CLS_FINITE, fin_b = dec_cls(db) == CLS_FINITE;
         LutEntry64 ea, eb;
-        ea.op = operand_a(fin_a ? dec_sign(da) : 0u, fin_a ? dec_sig(da) : 0u, fin_a ? dec_exp(da) : 1 - fa.bias, fa.mbits, 1 - fa.bias);
-        ea.exp = uint32_t((fin_a ? dec_exp(da) : 1 - fa.bias) + EB);
-        ea.bits = (fin_a ? dec_sign(da) : 0u) | (fin_a ? 0u : 2u);
-        eb.op = operand_b(fin_b ? dec_sign(db) : 0u, fin_b ? dec_sig(db) : 0u, fin_b ? dec_exp(db) : 1 - fb.bias, fb.mbits);
-        eb.exp = uint32_t((fin_b ? dec_exp(db) : 1 - fb.bias) + EB);
-        eb.bits = (fin_b ? dec_sign(db) : 0u) | (fin_b ? 0u : 2u);
+        const uint32_t sga = fin_a ? dec_sig(da) : 0u, sgb = fin_b ? dec_sig(db) : 0u;
+        ea.op = operand_a(fin_a ? dec_sign(da) : 0u, sga, fin_a ? dec_exp(da) : 0, fa.mbits);
+        ea.exp = sga ? uint32_t(dec_exp(da) + EB) : 0u;
+        ea.bits = (fin_a ? dec_sign(da) : 0u) | (fin_a ? 0u : 2u) | (sga ? 4u : 0u);
+        eb.op = operand_b(fin_b ? dec_sign(db) : 0u, sgb, fin_b ? dec_exp(db) : 0, fb.mbits);
+        eb.exp = sgb ? uint32_t(dec_exp(db) + EB) : 0u;
+        eb.bits = (fin_b ? dec_sign(db) : 0u) | (fin_b ? 0u : 2u) | (sgb ? 4u : 0u);
         s.lut_a[tid] = ea;
         s.lut_b[tid] = eb;
     }
@@ -155,15 +160,16 @@ __device__ __forceinline__ void store_chunk64(SM& sm, PL& s, const RawChunk<EK>&
                 const LutEntry64 e = is_a ? sm.lut_a[byte] : sm.lut_b[byte];
                 op = e.op;
                 expb = e.exp;
-                bits += (e.bits & 1u) << q;
+                bits += ((e.bits & 1u) | ((e.bits & 4u) << 14)) << q;      // sign in the low half, nonzero in the high half
                 spec |= e.bits & 2u;
             } else {
                 const uint32_t w = E::BYTES == 2 ? ((raw.w[it][q / 2] >> (16 * (q % 2))) & 0xFFFFu) : raw.w[it][q];
                 uint32_t sig, sign, special;
                 fast::decode_signmag<EK>(w, sig, expb, sign, special);
                 const int exp = int(expb) - EB;
-                op = is_a ? operand_a(sign, sig, exp, E::MBITS, 1 - E::BIAS) : operand_b(sign, sig, exp, E::MBITS);
-                bits += sign << q;
+                op = is_a ? operand_a(sign, sig, exp, E::MBITS) : operand_b(sign, sig, exp, E::MBITS);
+                if (!sig) expb = 0u;                                        // no exponent: never the maximum
+                bits += (sign | (uint32_t(sig != 0u) << 16)) << q;
                 spec |= special;
             }
             if (is_a) s.a_d[kk][r] = op; else s.b_d[kk][r] = op;
@@ -173,12 +179,13 @@ __device__ __forceinline__ void store_chunk64(SM& sm, PL& s, const RawChunk<EK>&
             }
             prev_exp = expb;
         }
+        // sign and nonzero bits of the task's elements go to bits [h * TASK, h * TASK + TASK) of the row's masks
         if (E::TASK == 16) {
-            if (is_a) reinterpret_cast<uint16_t*>(&s.a_sgn[r])[h] = uint16_t(bits);
-            else reinterpret_cast<uint16_t*>(&s.b_sgn[r])[h] = uint16_t(bits);
+            if (is_a) { reinterpret_cast<uint16_t*>(&s.a_sgn[r])[h] = uint16_t(bits); reinterpret_cast<uint16_t*>(&s.a_nz[r])[h] = uint16_t(bits >> 16); }
+            else { reinterpret_cast<uint16_t*>(&s.b_sgn[r])[h] = uint16_t(bits); reinterpret_cast<uint16_t*>(&s.b_nz[r])[h] = uint16_t(bits >> 16); }
         } else {
-            if (is_a) reinterpret_cast<uint8_t*>(&s.a_sgn[r])[h] = uint8_t(bits);
-            else reinterpret_cast<uint8_t*>(&s.b_sgn[r])[h] = uint8_t(bits);
+            if (is_a) { reinterpret_cast<uint8_t*>(&s.a_sgn[r])[h] = uint8_t(bits); reinterpret_cast<uint8_t*>(&s.a_nz[r])[h] = uint8_t(bits >> 16); }
+            else { reinterpret_cast<uint8_t*>(&s.b_sgn[r])[h] = uint8_t(bits); reinterpret_cast<uint8_t*>(&s.b_nz[r])[h] = uint8_t(bits >> 16); }
         }
     }
     if (spec) atomicOr(&sm.special[flag], 1);
@@ -342,6 +349,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
                     const uint32_t field = ACC16 ? (cw[r][c] >> 10) & 0x1Fu : (cw[r][c] >> 23) & 0xFFu;
                     int rel = int(max(field, 1u)) + (CB - (ACC16 ? 15 : 127));
                     if (ST) rel -= sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0];
+                    if ((cw[r][c] & (ACC16 ? 0x7FFFu : 0x7FFFFFFFu)) == 0u) rel = 0;       // c = 0 has no exponent
                     const int emax = __vimax3_s32(int(emp[r][c] & 0xFFFFu), int(emp[r][c] >> 16), rel);     // e_max + CB
                     const double magic = __hiloint2double(emax * (1 << 20) + MAGIC_K, 0);
                     double cd = ACC16 ? double(__half2float(__ushort_as_half((unsigned short)cw[r][c]))) : double(__uint_as_float(cw[r][c]));
@@ -398,10 +406,10 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
             const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
 #pragma unroll
             for (int r = 0; r < TM; ++r) {
-                const uint32_t sa = s.a_sgn[ty * TM + r];
+                const uint32_t sa = s.a_sgn[ty * TM + r], nza = s.a_nz[ty * TM + r] & kmask;
 #pragma unroll
                 for (int c = 0; c < TN; ++c) {
-                    const int nneg = __popc((sa ^ s.b_sgn[col_of(tx, c)]) & kmask);
+                    const int nneg = __popc((sa ^ s.b_sgn[col_of(tx, c)]) & nza & s.b_nz[col_of(tx, c)]);
                     const long long bits = __double_as_longlong(acc[r][c]) + (long long)nneg;
                     const int hi = int(bits >> 32);
                     const double magic = __hiloint2double((hi & 0x7FF00000) | 0x00080000, 0);
@@ -416,7 +424,13 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
                         }
                         cw[r][c] = w;
                     } else {
-                        cw[r][c] = __float_as_uint(__double2float_rz(v));
+                        uint32_t w = __float_as_uint(__double2float_rz(v));
+                        if ((__double2hiint(v) & 0x7FFFFFFF) >= 0x47F00000) {         // |v| >= 2^128: overflow, +-infinity from now on
+                            const uint32_t bit = 1u << (r * TN + c);
+                            if (!((sp_nan | sp_pinf | sp_ninf) & bit)) { if (w >> 31) sp_ninf |= bit; else sp_pinf |= bit; }
+                            w = 0u;
+                        }
+                        cw[r][c] = w;
                     }
                 }
             }

@@ -1,4 +1,6 @@
-// Tuned T-FDPA kernel template (Algorithm 5 + Algorithm 7 + Table 2) for GEMM-sized inputs.
+// Tuned T-FDPA kernel for 8-bit inputs with F = 13 (the Ada / Hopper FP8 rows; Algorithm 5 + Algorithm 7 + Table 2),
+// and the staging code it shares with the TR- / GTR-FDPA kernels (mmasim_trfdpa_fast.cu).  The F >= 23 variants and
+// ST-FDPA live in mmasim_tfdpa_f64.cuh.
 //
 // Work decomposition.  A CTA of 256 threads owns a 128 x 64 tile of D; a thread owns an 8 x 4 micro-tile and keeps
 // its 32 accumulators decoded in registers for the whole K loop: `cs`, the one's-complement signed significand
@@ -10,33 +12,31 @@
 // Per block of L elements and per output (Algorithm 7):
 //   pass 1   e_max = max(Exp(c), max_k(Exp(a_k) + Exp(b_k)))   fused add-max on two 16-bit lanes: half an
 //                                                              instruction per term
-//   pass 2   X_k  = A_op * B_op                                one multiply (FMA pipe)
-//            d_k  = e_max (+ g) - Exp(a_k) - Exp(b_k)          one 3-input add (ALU pipe)
-//            t_k  = X_k >> d_k                                 one shift (ALU pipe), clamped: >= 32 shifts all bits out
-//            S   += t_k                                        issued as multiply-add by one (FMA pipe): the ALU pipe
-//                                                              is the busy one
+//   pass 2   S <- S + floor(X_k * 2^-(d_k + g))                one FP32 fused multiply-add per term (see the kernel)
 //   then the accumulator term, the sign corrections, normalisation and rho (Table 2) - about 25 instructions.
 //
 // Sign-magnitude truncation without per-term sign work.  RZ_F truncates the magnitude of each aligned term, while
-// an arithmetic right shift of a two's-complement number rounds toward minus infinity.  Negative terms are
-// therefore carried in one's complement: -t is represented by ~t = -t - 1, and the number of negative terms of the
-// block (a population count over per-row / per-column sign bit masks) is added back once per block.
-//  * 8-bit inputs (FP8 / FP6 / FP4): the operands are built so that the 32-bit product itself has that form,
+// a floor (an arithmetic right shift of a two's-complement number, a multiply-add rounding toward minus infinity)
+// rounds down.  Negative terms are therefore carried in one's complement: -t is represented by ~t = -t - 1, and the
+// number of negative terms of the block (a population count over per-row / per-column sign bit masks) is added back
+// once per block.
+//  * 8-bit inputs (FP8 / FP6 / FP4): the operands are built so that the integer product itself has that form,
 //      X = s * (m << (F - frac + g)) + r,  m = sig_a * sig_b,  s = +-1 the product's sign,  g = mbits_a + 1 guard
 //      bits,  0 <= r < 2^g for s = +1 and -2^g <= r <= -1 for s = -1,
 //    by A_op = +-sig_a and B_op = (+-sig_b << (F - frac + g)) + sign(b), which gives r = +-sig_a.  Then
-//    X >> (d + g) is floor(m * 2^(F - frac) / 2^d) for positive terms and its one's complement for negative ones.
-//    A term counts as negative when the signs differ and sig_a != 0 (with b = +-0 it is -sig_a >> (d+g) = -1).
-//  * 16/32-bit inputs (FP16 / BF16 / TF32): the product would not fit with guard bits, so magnitudes are multiplied
-//    and shifted, and one 3-input logic instruction applies sign_a xor sign_b (full-width masks staged beside the
-//    operands).  Every term whose sign bits differ counts as negative.
+//    floor(X * 2^-(d + g)) is floor(m * 2^(F - frac) / 2^d) for positive terms and its one's complement for negative
+//    ones.  A term counts as negative when the signs differ and both significands are nonzero.
+//  * 16/32-bit inputs (FP16 / BF16 / TF32, TR-FDPA kernels): magnitudes are multiplied and shifted, and one 3-input
+//    logic instruction applies sign_a xor sign_b (full-width masks staged beside the operands).  Every term whose sign
+//    bits differ counts as negative.
 //
 // Exponents are staged with a bias of 512 per element (1024 per product / accumulator) so that they are positive
-// 16-bit lane values.
+// 16-bit lane values.  A zero element, like a zero accumulator, has no exponent and must never decide e_max: it is
+// staged as the word 0, which keeps every sum it enters below every sum of two real exponents.
 //
 // Everything that is rare takes a slow, by-the-book route: NaN / infinity inputs (the threads rescan the raw words
-// of the block and keep sticky NaN / +inf / -inf flags per output, Section 4.2), results outside the normal range of
-// the accumulator format, and block sums that do not fit 32 bits (generic conversion routine on a 64-bit sum).
+// of the block and keep sticky NaN / +inf / -inf flags per output, Section 4.2) and results outside the normal range
+// of the accumulator format (generic conversion routine).
 #pragma once
 #include "mmasim_device.cuh"
 
@@ -59,8 +59,8 @@ template <> struct Elem<EK_TF32> { static constexpr int BYTES = 4, TASK = 8, EBI
 
 struct LutEntry {
     uint32_t op;        // multiplier operand
-    uint32_t exp;       // Exp(x) + EB (minimum exponent for non-finite inputs, whose operand is zero)
-    uint32_t bits;      // bit 0: sign, bit 16: nonzero significand
+    uint32_t exp;       // Exp(x) + EB; 0 for zero, infinity and NaN (no exponent)
+    uint32_t bits;      // bit 0: sign, bit 16: finite and nonzero
     uint32_t special;   // nonzero for infinity / NaN
 };
 
@@ -75,7 +75,7 @@ struct Planes {
     uint32_t b_exp2[KC / 2][BN];
     uint32_t a_msk[Elem<EK>::SIGNMAG ? KC : 1][BM];   // 0 / ~0: sign of the element (sign-magnitude kinds)
     uint32_t b_msk[Elem<EK>::SIGNMAG ? KC : 1][BN];
-    uint32_t a_sgn[BM], a_nz[BM], b_sgn[BN];          // bit k of row r: sign / nonzero of element k of the chunk
+    uint32_t a_sgn[BM], a_nz[BM], b_sgn[BN], b_nz[BN];   // bit k of row r: sign / nonzero of element k of the chunk
 };
 
 template <int EK, bool SLIM = false, int NBUF = 1>
@@ -115,7 +115,7 @@ __device__ __forceinline__ int mad_one(int t, int one, int s) {
 // Accumulator state of one output.
 struct Acc {
     int cs;     // one's complement signed significand, F fractional bits relative to 2^(ce - CB)
-    int ce;     // Exp(c) + CB
+    int ce;     // Exp(c) + CB; 0 for c = 0
 };
 
 template <int F, bool ACC16>
@@ -126,14 +126,14 @@ __device__ __forceinline__ Acc acc_from_word(uint32_t w, uint32_t& sp) {
     if (d.cls != CLS_FINITE) {
         sp |= (d.cls == CLS_NAN) ? 1u : (d.sign ? 4u : 2u);
         a.cs = 0;
-        a.ce = (ACC16 ? -14 : -126) + CB;
+        a.ce = 0;
         return a;
     }
     constexpr int MB = ACC16 ? 10 : 23;
     // F < 23 (F = 13): the low bits of an FP32 c fall below every block's truncation point anyway
     const int mag = (F >= MB) ? int(d.sig << (F >= MB ? F - MB : 0)) : int(d.sig >> (F >= MB ? 0 : MB - F));
     a.cs = d.sign ? ~mag : mag;
-    a.ce = d.exp + CB;
+    a.ce = d.sig ? d.exp + CB : 0;      // a zero accumulator has no exponent: 0 never wins the block maximum
     return a;
 }
 
@@ -182,10 +182,10 @@ __device__ __forceinline__ void rho_fast(int S, int emaxb, Acc& a, int& vmin, in
     } else {
         sig = norm >> (31 - MB);
     }
-    ve = mag ? ve : EMINB;                                     // an exactly zero sum is +0 with the minimum exponent
+    ve = mag ? ve : EMINB;                                     // an exactly zero sum is +0
     vmin = min(vmin, ve);
     vmax = max(vmax, ve);
-    a.ce = ve;
+    a.ce = mag ? ve : 0;
     a.cs = int(sig << (F - MB)) ^ sg;
 }
 
@@ -206,7 +206,8 @@ __device__ __forceinline__ void decode_signmag(uint32_t w, uint32_t& sig, uint32
     sign = (x >> (E::MBITS + E::EBITS)) & 1u;
     special = field == ((1u << E::EBITS) - 1u);
     sig = special ? 0u : (mant | (field ? (1u << E::MBITS) : 0u));
-    expb = uint32_t(int((field && !special) ? field : 1u) - E::BIAS + EB);
+    // a zero (and the stand-in of an infinity or NaN) has no exponent: the word 0 lies below every real exponent sum
+    expb = sig ? uint32_t(int(field ? field : 1u) - E::BIAS + EB) : 0u;
 }
 
 // Decode tables of the 8-bit kinds: entry `tid` of both (256 threads).
@@ -218,21 +219,24 @@ __device__ __forceinline__ void init_lut(SM& s, const FmtDesc& fa, const FmtDesc
         const uint32_t da = decode_elem(fa, uint32_t(tid)), db = decode_elem(fb, uint32_t(tid));
         const bool fin_a = dec_cls(da) == CLS_FINITE, fin_b = dec_cls(db) == CLS_FINITE;
         LutEntry ea, eb;
+        const bool nz_a = fin_a && dec_sig(da) != 0u, nz_b = fin_b && dec_sig(db) != 0u;
         ea.op = fin_a ? uint32_t(dec_ssig(da)) : 0u;
-        ea.exp = uint32_t((fin_a ? dec_exp(da) : 1 - fa.bias) + EB);
-        ea.bits = fin_a ? (dec_sign(da) | (uint32_t(dec_sig(da) != 0u) << 16)) : 0u;
+        ea.exp = nz_a ? uint32_t(dec_exp(da) + EB) : 0u;         // zero, infinity, NaN: no exponent
+        ea.bits = fin_a ? (dec_sign(da) | (uint32_t(nz_a) << 16)) : 0u;
         ea.special = fin_a ? 0u : 1u;
         const int sb = fin_b ? dec_ssig(db) : 0;
         const int ub = fin_b ? (dec_sign(db) ? -1 : 1) : 0;     // also for b = +-0 (see the header comment)
         eb.op = uint32_t(sb * (1 << (pre + guard)) + ub);
-        eb.exp = uint32_t((fin_b ? dec_exp(db) : 1 - fb.bias) + EB);
-        eb.bits = fin_b ? dec_sign(db) : 0u;
+        eb.exp = nz_b ? uint32_t(dec_exp(db) + EB) : 0u;
+        eb.bits = fin_b ? (dec_sign(db) | (uint32_t(nz_b) << 16)) : 0u;
         eb.special = fin_b ? 0u : 1u;
         if (fpsum) {
             // floating-point form of the same operands (see the FP32 summation path of the kernel): the operand scaled
-            // by 2^Exp, exact in FP32 (at most 4 + 15 significant bits, exponents far inside the FP32 range)
+            // by 2^Exp, exact in FP32 (at most 4 + 15 significant bits, exponents far inside the FP32 range).  A zero b
+            // is staged as 0 there (its terms vanish and are not counted as negative): with the zero terms outside
+            // e_max nothing bounds sig_a * 2^(Exp(a) + Exp_min(b)) below one unit of the sum any more.
             ea.op = __float_as_uint(ldexpf(float(fin_a ? dec_ssig(da) : 0), fin_a ? dec_exp(da) : 0));
-            eb.op = __float_as_uint(ldexpf(float(sb * (1 << (pre + guard)) + ub), (fin_b ? dec_exp(db) : 0) - FP_SHIFT));
+            eb.op = nz_b ? __float_as_uint(ldexpf(float(sb * (1 << (pre + guard)) + ub), dec_exp(db) - FP_SHIFT)) : 0u;
         }
         s.lut_a[tid] = ea;
         s.lut_b[tid] = eb;
@@ -326,6 +330,7 @@ __device__ __forceinline__ void store_chunk(SM& sm, PL& s, const RawChunk<EK>& r
                 reinterpret_cast<uint16_t*>(&s.a_nz[r])[h] = uint16_t(bits >> 16);
             } else {
                 reinterpret_cast<uint16_t*>(&s.b_sgn[r])[h] = uint16_t(bits);
+                reinterpret_cast<uint16_t*>(&s.b_nz[r])[h] = uint16_t(bits >> 16);
             }
         } else {
             if (is_a) reinterpret_cast<uint8_t*>(&s.a_sgn[r])[h] = uint8_t(bits);
@@ -362,6 +367,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
     // whole of pass 2 runs exactly on the FP32 pipe, one instruction per term (see pass 2 below).  Its staged planes
     // are small enough for two buffers: the next chunk is decoded while the current one is computed, one barrier per chunk.
     constexpr bool FPSUM = TfdpaFpsum<EK, F>::value;
+    static_assert(FPSUM && !ST, "this kernel is the FP32 summation form (8-bit inputs, F <= 13); F >= 23 and ST-FDPA run in mmasim_tfdpa_f64.cuh");
     constexpr bool DB = FPSUM;
     using SM = Smem<EK, FPSUM, DB ? 2 : 1>;
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -557,45 +563,6 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
                         S0[r][c] = bits - ((bits & 0x7F800000) | 0x00400000);
                         emax[r][c] = max((bits >> 23) - (150 - CB - FP_SHIFT), acc[r][c].ce + guard);
                     }
-            } else {
-#pragma unroll 2
-            for (int kk = kb; kk < kb + L; ++kk) {
-                const bool second = NSUM == 2 && (kk - kb >= HALF);
-                const int4 eb = *reinterpret_cast<const int4*>(&s.b_exp[kk][tx * TN]);
-                const int4 ob = *reinterpret_cast<const int4*>(&s.b_op[kk][tx * TN]);
-                const int ebv[TN] = {eb.x, eb.y, eb.z, eb.w};
-                const int obv[TN] = {ob.x, ob.y, ob.z, ob.w};
-                uint32_t mbv[TN] = {0u, 0u, 0u, 0u};
-                if (SIGNMAG) {
-                    const uint4 mb = *reinterpret_cast<const uint4*>(&s.b_msk[SIGNMAG ? kk : 0][tx * TN]);
-                    mbv[0] = mb.x; mbv[1] = mb.y; mbv[2] = mb.z; mbv[3] = mb.w;
-                }
-#pragma unroll
-                for (int rh = 0; rh < TM; rh += 4) {
-                    const int4 ea = *reinterpret_cast<const int4*>(&s.a_exp[kk][ty * TM + rh]);
-                    const int4 oa = *reinterpret_cast<const int4*>(&s.a_op[kk][ty * TM + rh]);
-                    const int eav[4] = {ea.x, ea.y, ea.z, ea.w};
-                    const int oav[4] = {oa.x, oa.y, oa.z, oa.w};
-                    uint32_t mav[4] = {0u, 0u, 0u, 0u};
-                    if (SIGNMAG) {
-                        const uint4 ma = *reinterpret_cast<const uint4*>(&s.a_msk[SIGNMAG ? kk : 0][ty * TM + rh]);
-                        mav[0] = ma.x; mav[1] = ma.y; mav[2] = ma.z; mav[3] = ma.w;
-                    }
-#pragma unroll
-                    for (int r4 = 0; r4 < 4; ++r4)
-#pragma unroll
-                        for (int c = 0; c < TN; ++c) {
-                            const int r = rh + r4;
-                            const int X = oav[r4] * obv[c];
-                            const int d = emax[r][c] - eav[r4] - ebv[c];
-                            int t;
-                            if (SIGNMAG) t = int(lsr_clamp(uint32_t(X), d) ^ mav[r4] ^ mbv[c]);
-                            else t = asr_clamp(X, d);
-                            if (second) S1[NSUM == 2 ? r : 0][NSUM == 2 ? c : 0] = mad_one(t, one, S1[NSUM == 2 ? r : 0][NSUM == 2 ? c : 0]);
-                            else S0[r][c] = mad_one(t, one, S0[r][c]);
-                        }
-                }
-            }
             }
             // ---- sign corrections, normalisation, rho ----
             const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
@@ -607,7 +574,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
                 const uint32_t nza = SIGNMAG ? kmask : (s.a_nz[ty * TM + r] & kmask);
 #pragma unroll
                 for (int c = 0; c < TN; ++c) {
-                    const int nneg = __popc((sa ^ s.b_sgn[tx * TN + c]) & nza);
+                    const int nneg = __popc((sa ^ s.b_sgn[tx * TN + c]) & nza & s.b_nz[tx * TN + c]);
                     int S = S0[r][c] + nneg;
                     if (NSUM == 2) {
                         const int s1 = S1[NSUM == 2 ? r : 0][NSUM == 2 ? c : 0];
@@ -626,7 +593,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
                     const uint32_t nza = SIGNMAG ? kmask : (s.a_nz[ty * TM + r] & kmask);
 #pragma unroll
                     for (int c = 0; c < TN; ++c) {
-                        const int nneg = __popc((sa ^ s.b_sgn[tx * TN + c]) & nza);
+                        const int nneg = __popc((sa ^ s.b_sgn[tx * TN + c]) & nza & s.b_nz[tx * TN + c]);
                         long long S = (long long)S0[r][c] + nneg;
                         if (NSUM == 2) S += (long long)S1[NSUM == 2 ? r : 0][NSUM == 2 ? c : 0];
                         uint32_t ev = 0u;

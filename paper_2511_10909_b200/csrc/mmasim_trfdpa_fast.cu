@@ -9,6 +9,8 @@
 //   * the accumulator enters afterwards at E = max(e_max, Exp(c)): T is rounded down to F2 fractional bits and c to F
 //     (arithmetic right shifts of two's-complement values are round-down), with the "special truncation" of c in
 //     GTR-FDPA; the sum is converted with RNE-FP32 (64-bit, inline);
+//   * zero products have no exponent (their staged exponent words are 0, below every real sum): a group without a
+//     nonzero product has T = 0 and an exponent lane that never wins a maximum;
 //   * a product of magnitude >= 2^128 is an infinity (Section 4.2): whenever a block's e_max could allow that, the
 //     thread rescans the raw words of the block and records the event like any other infinity.
 // The accumulators stay live across the product passes, so a thread handles its 8 rows in two halves of 4.
@@ -21,7 +23,7 @@ namespace {
 
 struct TrAcc {
     int cs;     // signed 24-bit significand (two's complement): value = cs * 2^(ce - CB - 23)
-    int ce;     // Exp(c) + CB
+    int ce;     // Exp(c) + CB; 0 for c = 0
 };
 
 __device__ __forceinline__ TrAcc tr_from_word(uint32_t w, uint32_t& sp) {
@@ -30,11 +32,11 @@ __device__ __forceinline__ TrAcc tr_from_word(uint32_t w, uint32_t& sp) {
     if (d.cls != CLS_FINITE) {
         sp |= (d.cls == CLS_NAN) ? 1u : (d.sign ? 4u : 2u);
         a.cs = 0;
-        a.ce = -126 + CB;
+        a.ce = 0;
         return a;
     }
     a.cs = d.sign ? -int(d.sig) : int(d.sig);
-    a.ce = d.exp + CB;
+    a.ce = d.sig ? d.exp + CB : 0;      // a zero accumulator has no exponent: 0 never decides E
     return a;
 }
 
@@ -66,7 +68,7 @@ __device__ __forceinline__ void rne32_fast(long long S, int eb, TrAcc& a, int& v
     ve = mag ? ve : -126 + CB;
     vmin = min(vmin, ve);
     vmax = max(vmax, ve);
-    a.ce = ve;
+    a.ce = mag ? ve : 0;
     a.cs = sg ? -sig : sig;
 }
 

@@ -69,6 +69,8 @@ def _load():
                                      POINTER(_GemmOpts)]
     lib.mmasim_int_peak.restype = c_int
     lib.mmasim_int_peak.argtypes = [c_int, c_int64, c_int64, c_void_p, POINTER(c_int32), c_void_p]
+    lib.mmasim_hw_mma.restype = c_int
+    lib.mmasim_hw_mma.argtypes = [c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.mmasim_last_kernel.restype = c_char_p
     lib.mmasim_last_error.restype = c_char_p
     return lib
@@ -227,6 +229,24 @@ def gemm_host(model: Model, A, B, C=None, *, K=None, sfa=None, sfb=None, k_chunk
     p = lambda x: None if x is None else c_void_p(x.ctypes.data)
     o = _make_opts(p(sfa), p(sfb), k_chunk, p(row_scale), p(col_scale))
     _check(_lib.mmasim_gemm_host(model._h, M, N, K, p(A), p(B), p(C), p(out), byref(o)))
+    return out
+
+
+HW_KINDS = ["f16_f32", "f16_f16", "bf16_f32", "tf32_f32", "e4m3_f32", "e5m2_f32", "f64", "f16_f32_k8", "tf32_f32_k4"]
+_HW_ACC_BYTES = {"f16_f16": 2, "f64": 8}
+
+
+def hw_mma(kind: str, A, B, C=None, out=None, *, stream=None):
+    """The B200's own `mma.sync` of the given kind on every 16-row tile of A (8 rows for "f64") against the 8 rows
+    of B: D (M x 8) = A (M x K) * B^T + C, CUDA tensors of raw words."""
+    import torch
+    if not A.is_cuda:
+        raise MmasimError(1, "mmasim.hw_mma needs CUDA tensors")
+    M, K = A.shape
+    if out is None:
+        dt = {2: torch.int16, 4: torch.int32, 8: torch.int64}[_HW_ACC_BYTES.get(kind, 4)]
+        out = torch.empty((M, 8), dtype=dt, device=A.device)
+    _check(_lib.mmasim_hw_mma(HW_KINDS.index(kind), M, K, _ptr(A), _ptr(B), _ptr(C), _ptr(out), _stream(stream)))
     return out
 
 
