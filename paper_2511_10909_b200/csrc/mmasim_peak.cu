@@ -8,7 +8,7 @@ namespace {
 
 enum PeakKind : int {
     PK_IADD3 = 0, PK_LOP3, PK_SHF, PK_IMAD, PK_MACMIX, PK_VIADDMAX, PK_VIADDMAX16X2, PK_F2I, PK_FMUL, PK_POPC,
-    PK_IMAD_PLUS_ALU, PK_FMUL_PLUS_ALU, PK_IMAD_WIDE, PK_MAC_D1, PK_MAC_D2, PK_DP4A, PK_DFMA, PK_COUNT
+    PK_IMAD_PLUS_ALU, PK_FMUL_PLUS_ALU, PK_IMAD_WIDE, PK_MAC_D1, PK_MAC_D2, PK_DP4A, PK_DFMA, PK_DFMA_PLUS_ALU, PK_COUNT
 };
 
 template <int KIND>
@@ -69,21 +69,29 @@ __global__ void __launch_bounds__(256) peak_kernel(int64_t iters, int* sink) {
     if (r == 0x12345678) *sink = r;             // practically never true: keeps the chains alive
 }
 
-// FP64 fused multiply-add chains (a kernel of its own so that the integer kernels keep their register allocation)
+// FP64 fused multiply-add chains (a kernel of its own so that the integer kernels keep their register allocation);
+// WITH_ALU adds one independent fused add-max per multiply-add: if the two pipes ran side by side the launch would
+// take as long as the slower of the two streams alone, and it takes about their sum instead.
+template <bool WITH_ALU>
 __global__ void __launch_bounds__(256) peak_kernel_f64(int64_t iters, int* sink) {
     double d[8];
+    int x[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) d[i] = 1.0 + 1e-9 * double(threadIdx.x + i);
+    for (int i = 0; i < 8; ++i) { d[i] = 1.0 + 1e-9 * double(threadIdx.x + i); x[i] = threadIdx.x * 2654435 + i * 40503; }
     for (int64_t it = 0; it < iters; it += 8) {
 #pragma unroll
         for (int u = 0; u < 8; ++u)
 #pragma unroll
-            for (int i = 0; i < 8; ++i) d[i] = fma(d[i], d[(i + 1) & 7], d[(i + 3) & 7]);
+            for (int i = 0; i < 8; ++i) {
+                d[i] = fma(d[i], d[(i + 1) & 7], d[(i + 3) & 7]);
+                if (WITH_ALU) x[i] = (int)__viaddmax_s16x2((unsigned)x[(i + 1) & 7], (unsigned)x[(i + 3) & 7], (unsigned)x[i]);
+            }
     }
     double r = 0.0;
+    int q = 0;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) r += d[i];
-    if (r == 0.12345) *sink = 1;
+    for (int i = 0; i < 8; ++i) { r += d[i]; q ^= x[i]; }
+    if (r == 0.12345 && q == 0x12345678) *sink = 1;
 }
 
 template <int KIND>
@@ -115,9 +123,11 @@ int launch_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t
         case PK_MAC_D1: *ops_per_round = 1; return launch<PK_MAC_D1>(blocks, iters, sink, stream);
         case PK_MAC_D2: *ops_per_round = 1; return launch<PK_MAC_D2>(blocks, iters, sink, stream);
         case PK_DP4A: *ops_per_round = 1; return launch<PK_DP4A>(blocks, iters, sink, stream);
-        case PK_DFMA: {
-            *ops_per_round = 1;
-            peak_kernel_f64<<<(unsigned)blocks, 256, 0, stream>>>(iters, static_cast<int*>(sink));
+        case PK_DFMA:
+        case PK_DFMA_PLUS_ALU: {
+            *ops_per_round = kind == PK_DFMA ? 1 : 2;
+            if (kind == PK_DFMA) peak_kernel_f64<false><<<(unsigned)blocks, 256, 0, stream>>>(iters, static_cast<int*>(sink));
+            else peak_kernel_f64<true><<<(unsigned)blocks, 256, 0, stream>>>(iters, static_cast<int*>(sink));
             const cudaError_t err = cudaGetLastError();
             if (err != cudaSuccess) { set_error("int_peak launch failed: %s", cudaGetErrorString(err)); return MMASIM_ERR_CUDA; }
             return MMASIM_OK;

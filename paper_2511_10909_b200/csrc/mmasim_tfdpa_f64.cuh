@@ -402,35 +402,44 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
                         }
                 }
             }
-            // ---- sign corrections, rho ----
+            // ---- sign corrections, rho.  An overflow (|v| >= 2^128, or an FP16 result that rounds to infinity) is rare
+            // and sticky: the loop only tracks the largest result word, the flags are set in a second pass ----
             const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
+            constexpr uint32_t ABS = ACC16 ? 0x7FFFu : 0x7FFFFFFFu;
+            constexpr uint32_t SUSPECT = ACC16 ? 0x7C00u : 0x7F7FFFFFu;   // FP16: infinity; FP32: cvt.rz saturates at the largest finite word
+            uint32_t wmax = 0u;
+            auto block_value = [&](int r, int c, uint32_t sa, uint32_t nza) -> double {
+                const int nneg = __popc((sa ^ s.b_sgn[col_of(tx, c)]) & nza & s.b_nz[col_of(tx, c)]);
+                const long long bits = __double_as_longlong(acc[r][c]) + (long long)nneg;
+                const int hi = int(bits >> 32);
+                const double magic = __hiloint2double((hi & 0x7FF00000) | 0x00080000, 0);
+                double v = __dsub_rn(__longlong_as_double(bits), magic);              // S * q, exact; +0 when S = 0
+                if (ST) v = __dmul_rn(v, pow2d(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]));
+                return v;
+            };
 #pragma unroll
             for (int r = 0; r < TM; ++r) {
                 const uint32_t sa = s.a_sgn[ty * TM + r], nza = s.a_nz[ty * TM + r] & kmask;
 #pragma unroll
                 for (int c = 0; c < TN; ++c) {
-                    const int nneg = __popc((sa ^ s.b_sgn[col_of(tx, c)]) & nza & s.b_nz[col_of(tx, c)]);
-                    const long long bits = __double_as_longlong(acc[r][c]) + (long long)nneg;
-                    const int hi = int(bits >> 32);
-                    const double magic = __hiloint2double((hi & 0x7FF00000) | 0x00080000, 0);
-                    double v = __dsub_rn(__longlong_as_double(bits), magic);          // S * q, exact; +0 when S = 0
-                    if (ST) v = __dmul_rn(v, pow2d(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]));
-                    if (ACC16) {
-                        uint32_t w = uint32_t(__half_as_ushort(__double2half(v)));
-                        if ((w & 0x7FFFu) == 0x7C00u) {                               // RNE-FP16 overflow: +-infinity from now on
-                            const uint32_t bit = 1u << (r * TN + c);
-                            if (!((sp_nan | sp_pinf | sp_ninf) & bit)) { if (w >> 15) sp_ninf |= bit; else sp_pinf |= bit; }
-                            w = 0u;
-                        }
-                        cw[r][c] = w;
-                    } else {
-                        uint32_t w = __float_as_uint(__double2float_rz(v));
-                        if ((__double2hiint(v) & 0x7FFFFFFF) >= 0x47F00000) {         // |v| >= 2^128: overflow, +-infinity from now on
-                            const uint32_t bit = 1u << (r * TN + c);
-                            if (!((sp_nan | sp_pinf | sp_ninf) & bit)) { if (w >> 31) sp_ninf |= bit; else sp_pinf |= bit; }
-                            w = 0u;
-                        }
-                        cw[r][c] = w;
+                    const double v = block_value(r, c, sa, nza);
+                    const uint32_t w = ACC16 ? uint32_t(__half_as_ushort(__double2half(v))) : __float_as_uint(__double2float_rz(v));
+                    wmax = max(wmax, w & ABS);
+                    cw[r][c] = w;
+                }
+            }
+            if (wmax >= SUSPECT) {
+#pragma unroll
+                for (int r = 0; r < TM; ++r) {
+                    const uint32_t sa = s.a_sgn[ty * TM + r], nza = s.a_nz[ty * TM + r] & kmask;
+#pragma unroll
+                    for (int c = 0; c < TN; ++c) {
+                        if ((cw[r][c] & ABS) != SUSPECT) continue;
+                        const double v = block_value(r, c, sa, nza);
+                        if (!ACC16 && fabs(v) < 3.402823669209385e38) continue;       // below 2^128: the largest finite number, legitimately
+                        const uint32_t bit = 1u << (r * TN + c);
+                        if (!((sp_nan | sp_pinf | sp_ninf) & bit)) { if (v < 0.0) sp_ninf |= bit; else sp_pinf |= bit; }
+                        cw[r][c] = 0u;                                                // +-infinity from now on
                     }
                 }
             }

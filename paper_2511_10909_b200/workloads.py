@@ -269,3 +269,32 @@ def sample_pairs(M: int, N: int, count: int, seed: int):
     """``count`` seeded output positions (i, j) of an M x N result."""
     g = rng(seed, stream=7)
     return np.stack([g.integers(0, M, count), g.integers(0, N, count)], axis=1)
+
+
+def hw_tiles(fmt: str, acc: str, K: int, M: int, seed: int = 9):
+    """Inputs for one hardware MMA shape: A (M x K), B (8 x K), C (M x 8) raw words.
+
+    FP16 / BF16 / TF32: the eight input classes of config 4 (row class = row index mod 8; the eight rows of B take
+    one class each), plus zero-heavy rows (every 16th row of A has about a third of its elements replaced by +-0).
+    FP64: N(0,1) values, every fourth row scaled over +-40 binades.
+    """
+    g = rng(seed, stream=K)
+    if fmt == "fp64":
+        def mat(shape):
+            x = g.standard_normal(shape)
+            wide = (np.arange(shape[0]) % 4 == 3)[:, None]
+            x = np.where(wide, x * np.exp2(g.integers(-40, 40, shape)), x)
+            return np.ascontiguousarray(x.view(np.uint64))
+        return mat((M, K)), mat((8, K)), mat((M, 8))
+    A, _, C1 = cfg4(fmt, K, n=M)
+    _, B, _ = cfg4(fmt, K, n=8)
+    zero_rows = np.flatnonzero(np.arange(M) % 16 == 9)
+    z = g.random((zero_rows.size, K)) < 0.33
+    sign = A.dtype.type(1 << (A.dtype.itemsize * 8 - 1))
+    A[zero_rows] = np.where(z, A[zero_rows] & sign, A[zero_rows])
+    _, _, C2 = cfg4(fmt, K, n=M * 8)
+    C = C2.reshape(M, 8).copy()
+    C[np.arange(M) % 16 == 1] = 0                      # a few all-zero accumulator rows
+    if acc == "fp16":
+        C = (C >> 16).astype(np.uint16)                # the top half of an FP32 word: an arbitrary FP16 word
+    return A, B, np.ascontiguousarray(C)

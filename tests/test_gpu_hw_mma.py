@@ -1,0 +1,101 @@
+"""The Blackwell rows of the registry against the hardware they describe (Section 3.1, Step 4): the B200's own
+mma.sync instruction, run through mmasim_hw_mma, must agree bit for bit with the model evaluated by the CUDA path
+(every output) and by the CPU oracle (sampled outputs), on the input classes of config 4 plus zero-heavy rows.
+These runs also pin two readings of the paper: zero terms take no part in e_max, and rho overflows to infinity."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2511_10909_b200 import workloads as wl
+pytestmark = pytest.mark.gpu
+
+gu = pytest.importorskip("gpu_util") if torch.cuda.is_available() else None
+
+
+def _needs_b200():
+    if torch.cuda.get_device_capability(0)[0] != 10:
+        pytest.skip("the hardware comparison is about the B200 (compute capability 10.x)")
+
+
+# kind -> (element format, accumulator format, K of one instruction)
+KINDS = {"f16_f32": ("fp16", "fp32", 16), "f16_f16": ("fp16", "fp16", 16), "bf16_f32": ("bf16", "fp32", 16),
+         "tf32_f32": ("tf32", "fp32", 8), "f16_f32_k8": ("fp16", "fp32", 8), "tf32_f32_k4": ("tf32", "fp32", 4)}
+
+
+def _run(kind, A, B, C):
+    from paper_2511_10909_b200 import mmasim
+    return gu.host_words(mmasim.hw_mma(kind, gu.dev(A), gu.dev(B), gu.dev(C)))
+
+
+def test_fragment_layouts_with_exact_integers():
+    """Small integers make every product and sum exact: D must be the integer matrix product, whatever the model."""
+    _needs_b200()
+    g = wl.rng(90)
+    M = 64
+    for kind, (fmt, acc, k) in list(KINDS.items()) + [("e4m3_f32", ("e4m3", "fp32", 32)), ("e5m2_f32", ("e5m2", "fp32", 32)),
+                                                       ("f64", ("fp64", "fp64", 4))]:
+        for K in (k, 3 * k):
+            a = g.integers(-2, 3, (M, K)); b = g.integers(-2, 3, (8, K)); c = g.integers(-8, 9, (M, 8))
+            if fmt == "fp64":
+                A, B, C = (x.astype(np.float64).view(np.uint64) for x in (a, b, c))
+            else:
+                A, B = wl.cast(a.astype(np.float32), fmt), wl.cast(b.astype(np.float32), fmt)
+                C = c.astype(np.float32).view(np.uint32) if acc == "fp32" else c.astype(np.float16).view(np.uint16)
+            D = _run(kind, A, B, C)
+            want = a @ b.T + c
+            got = D.view({2: np.float16, 4: np.float32, 8: np.float64}[D.dtype.itemsize]).astype(np.int64)
+            assert np.array_equal(got, want), (kind, K)
+
+
+@pytest.mark.parametrize("kind", list(KINDS))
+@pytest.mark.parametrize("chain", [1, 4])
+def test_blackwell_model_matches_mma_sync(kind, chain):
+    from paper_2511_10909_b200 import mmasim
+    _needs_b200()
+    fmt, acc, k = KINDS[kind]
+    if chain > 1 and kind in ("f16_f32_k8", "tf32_f32_k4"):
+        pytest.skip("a chain of the short instructions is a chain of shorter blocks than the registry row's L")
+    K, M = k * chain, 1 << 13
+    A, B, C = wl.hw_tiles(fmt, acc, K, M)
+    hw = _run(kind, A, B, C)
+    key = ("blackwell", fmt, acc)
+    D = gu.host_words(mmasim.gemm(mmasim.Model(*key), gu.dev(A), gu.dev(B), gu.dev(C)))
+    bad = np.argwhere(hw != D)
+    assert bad.size == 0, (kind, K, len(bad), [(tuple(x), hex(int(hw[tuple(x)])), hex(int(D[tuple(x)]))) for x in bad[:4]])
+    pairs = wl.sample_pairs(M, 8, 768, seed=91)
+    want = gu.oracle_samples(key, {"A": A, "B": B, "C": C}, pairs)
+    gu.assert_samples_equal(hw, want, pairs, f"hardware {kind} K={K} against the oracle")
+
+
+@pytest.mark.parametrize("K", [4, 16])
+def test_fp64_mma_is_a_chain_of_fmas(K):
+    from paper_2511_10909_b200 import mmasim
+    _needs_b200()
+    A, B, C = wl.hw_tiles("fp64", "fp64", K, 1 << 12)
+    hw = _run("f64", A, B, C)
+    key = ("blackwell", "fp64", "fp64")
+    D = gu.host_words(mmasim.gemm(mmasim.Model(*key), gu.dev(A), gu.dev(B), gu.dev(C)))
+    assert np.array_equal(hw, D)
+    pairs = wl.sample_pairs(1 << 12, 8, 512, seed=92)
+    gu.assert_samples_equal(hw, gu.oracle_samples(key, {"A": A, "B": B, "C": C}, pairs), pairs, "FP64 mma against the oracle")
+
+
+def test_the_comparison_discriminates():
+    """The same inputs under the Ampere row (L = 8, F = 24) do differ from the hardware: the harness is not vacuous."""
+    from paper_2511_10909_b200 import mmasim
+    _needs_b200()
+    A, B, C = wl.hw_tiles("fp16", "fp32", 16, 1 << 12)
+    hw = _run("f16_f32", A, B, C)
+    D = gu.host_words(mmasim.gemm(mmasim.Model("ampere", "fp16", "fp32"), gu.dev(A), gu.dev(B), gu.dev(C)))
+    assert (hw != D).sum() > 100
+
+
+def test_hw_mma_rejects_bad_shapes():
+    from paper_2511_10909_b200 import mmasim
+    A = torch.zeros((24, 16), dtype=torch.int16, device="cuda")
+    B = torch.zeros((8, 16), dtype=torch.int16, device="cuda")
+    with pytest.raises(mmasim.MmasimError):
+        mmasim.hw_mma("f16_f32", A, B)                                   # 24 rows: not a multiple of 16
+    with pytest.raises(mmasim.MmasimError):
+        mmasim.hw_mma("f16_f32", A[:16, :8].contiguous(), B[:, :8].contiguous())   # K = 8 with a k16 instruction
