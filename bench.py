@@ -54,6 +54,14 @@ WORKLOADS = {
 }
 
 
+def compute_dtype(kernel: str, model) -> str:
+    """The arithmetic type the timed kernel computes in (the results are exact integers / model words either way)."""
+    if kernel == "tfdpa_lut8" and model.F <= 13:
+        return "f32"
+    return {"tfdpa_lut8": "f64", "tfdpa_f16": "f64", "tfdpa_bf16": "f64", "tfdpa_tf32": "f64", "trfdpa": "f64", "gtrfdpa": "f64",
+            "dot_tfdpa": "f64", "dot_ftz": "f32", "ftz_addmul": "f32", "fma_f32": "f32", "fma_f64": "f64", "gstfdpa": "int32"}.get(kernel, "int64")
+
+
 def algorithmic_ops_per_mac(model) -> float:
     """Integer operations per emulated MAC of the T-FDPA family: multiply, exponent add, maximum, distance,
     shift, accumulate (6 per term) plus about 25 per block for the accumulator term, normalisation and rho."""
@@ -341,7 +349,7 @@ def run_ours(args):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "int32", "data": "synthetic",
+        "dtype": compute_dtype(kernel_name, model), "data": "synthetic",
         "config": {"workload": f"{name}: {desc}", "model": "-".join(key), "M": M, "N": N, "K": K,
                    "l2": "flushed between timed steps (256 MiB write)", "parallelism": f"replicas x{world} (independent batches, no exchange)"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps,

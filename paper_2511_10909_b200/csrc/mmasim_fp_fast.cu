@@ -60,13 +60,17 @@ __global__ void __launch_bounds__(NT, 2) fp_kernel(GemmArgs g) {
     const int tid = threadIdx.x;
     const int tx = tid % 16, ty = tid / 16;
     const int64_t row0 = int64_t(blockIdx.y) * BM, col0 = int64_t(blockIdx.x) * BN;
+    // Columns of a thread's micro-tile: groups of V (one 16-byte shared load), 16 * V columns apart, so that the sixteen
+    // threads of a row of the thread grid read 256 contiguous bytes per load (no bank conflicts).
+    constexpr int V = 16 / int(sizeof(in_t));
+    auto col_of = [&](int c) { return (c / V) * (16 * V) + tx * V + (c % V); };
 
     acc_t d[TM][TN];
 #pragma unroll
     for (int r = 0; r < TM; ++r)
 #pragma unroll
         for (int c = 0; c < TN; ++c) {
-            const int64_t i = row0 + ty * TM + r, j = col0 + tx * TN + c;
+            const int64_t i = row0 + ty * TM + r, j = col0 + col_of(c);
             acc_t v = acc_t(0);
             if (g.C && i < g.M && j < g.N) {
                 if (FTZ) {
@@ -79,23 +83,37 @@ __global__ void __launch_bounds__(NT, 2) fp_kernel(GemmArgs g) {
             d[r][c] = v;
         }
 
-    for (int64_t k0 = 0; k0 < g.K; k0 += KC) {
-        __syncthreads();
-        // ---- stage: 16-byte loads, stored k-major ----
+    // The raw 16-byte words of the next chunk are fetched while the current one is computed.
+    constexpr int TASKS = (BM + BN) * TPR, PER_THREAD = (TASKS + NT - 1) / NT;
+    uint4 raw[PER_THREAD];
+    auto fetch = [&](int64_t k0) {
 #pragma unroll
-        for (int t0 = 0; t0 < (BM + BN) * TPR; t0 += NT) {
-            const int task = t0 + tid;
-            if (task >= (BM + BN) * TPR) break;
+        for (int it = 0; it < PER_THREAD; ++it) {
+            const int task = it * NT + tid;
             const bool is_a = task < BM * TPR;
             const int u = is_a ? task : task - BM * TPR;
             const int rows = is_a ? BM : BN;
             const int r = u % rows, h = u / rows;
             const int64_t grow = (is_a ? row0 : col0) + r;
-            uint4 raw = make_uint4(0u, 0u, 0u, 0u);
-            if (grow < (is_a ? g.M : g.N))
-                raw = *reinterpret_cast<const uint4*>(static_cast<const unsigned char*>(is_a ? g.A : g.B) +
-                                                      (grow * (is_a ? g.lda : g.ldb) + k0 + h * EPT) * T::IN_BYTES);
-            const uint32_t wv[4] = {raw.x, raw.y, raw.z, raw.w};
+            raw[it] = make_uint4(0u, 0u, 0u, 0u);
+            if (task < TASKS && grow < (is_a ? g.M : g.N))
+                raw[it] = *reinterpret_cast<const uint4*>(static_cast<const unsigned char*>(is_a ? g.A : g.B) +
+                                                          (grow * (is_a ? g.lda : g.ldb) + k0 + h * EPT) * T::IN_BYTES);
+        }
+    };
+    fetch(0);
+    for (int64_t k0 = 0; k0 < g.K; k0 += KC) {
+        __syncthreads();
+        // ---- stage: decode the fetched words, stored k-major ----
+#pragma unroll
+        for (int it = 0; it < PER_THREAD; ++it) {
+            const int task = it * NT + tid;
+            if (task >= TASKS) break;
+            const bool is_a = task < BM * TPR;
+            const int u = is_a ? task : task - BM * TPR;
+            const int rows = is_a ? BM : BN;
+            const int r = u % rows, h = u / rows;
+            const uint32_t wv[4] = {raw[it].x, raw[it].y, raw[it].z, raw[it].w};
 #pragma unroll
             for (int q = 0; q < EPT; ++q) {
                 in_t v;
@@ -106,15 +124,18 @@ __global__ void __launch_bounds__(NT, 2) fp_kernel(GemmArgs g) {
             }
         }
         __syncthreads();
+        if (k0 + KC < g.K) fetch(k0 + KC);
 
         if (!FTZ) {
-#pragma unroll 4
+            // fully unrolled: with a partial unroll the compiler rotates the accumulators through register moves
+            // (two moves per multiply-add in the FP64 kernel)
+#pragma unroll
             for (int kk = 0; kk < KC; ++kk) {
                 in_t a[TM], b[TN];
 #pragma unroll
                 for (int r = 0; r < TM; ++r) a[r] = As[kk][ty * TM + r];
 #pragma unroll
-                for (int c = 0; c < TN; ++c) b[c] = Bs[kk][tx * TN + c];
+                for (int c = 0; c < TN; ++c) b[c] = Bs[kk][col_of(c)];
 #pragma unroll
                 for (int r = 0; r < TM; ++r)
 #pragma unroll
@@ -130,7 +151,7 @@ __global__ void __launch_bounds__(NT, 2) fp_kernel(GemmArgs g) {
 #pragma unroll
                     for (int r = 0; r < TM; ++r) a[r] = float(As[kg + l][ty * TM + r]);
 #pragma unroll
-                    for (int c = 0; c < TN; ++c) b[c] = float(Bs[kg + l][tx * TN + c]);
+                    for (int c = 0; c < TN; ++c) b[c] = float(Bs[kg + l][col_of(c)]);
 #pragma unroll
                     for (int r = 0; r < TM; ++r)
 #pragma unroll
@@ -158,7 +179,7 @@ __global__ void __launch_bounds__(NT, 2) fp_kernel(GemmArgs g) {
     for (int r = 0; r < TM; ++r)
 #pragma unroll
         for (int c = 0; c < TN; ++c) {
-            const int64_t i = row0 + ty * TM + r, j = col0 + tx * TN + c;
+            const int64_t i = row0 + ty * TM + r, j = col0 + col_of(c);
             if (i >= g.M || j >= g.N) continue;
             const acc_t v = d[r][c];
             if (sizeof(acc_t) == 4) {

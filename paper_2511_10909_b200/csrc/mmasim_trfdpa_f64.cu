@@ -1,0 +1,319 @@
+// Tuned TR-FDPA (Algorithm 10) and GTR-FDPA (Algorithm 11) kernels: the CDNA3 models.
+//
+// The truncated fused sum of the products is computed like the T-FDPA kernel of mmasim_tfdpa_f64.cuh does it - same
+// tile, staging, one fma.rm.f64 per term into a register that holds 1.5 * 2^52 * q + T * q, q = 2^(e_max - F), with
+// the one's-complement treatment of negative terms and the population-count correction - except that
+//   * the accumulator is not part of that sum: e_max is the maximum over the (nonzero) products only, and the sum
+//     register starts as the bare constant;
+//   * GTR-FDPA keeps two sums, of the even and of the odd elements, each with its own maximum exponent - the two
+//     16-bit lanes of the packed exponent pass are exactly these two maxima - and merges them with round-down.
+// What follows per block and output is integer work on T (read from the low word of the register): T and c are
+// aligned at E = max(e_max, Exp(c)) with round-down (arithmetic right shifts of two's-complement values) to F2 and
+// F fractional bits, with the "special truncation" of c in GTR-FDPA, and the sum is converted with RNE-FP32.
+// A product of magnitude >= 2^128 is an infinity (Section 4.2): whenever a block's e_max could allow that, the thread
+// rescans the raw words of the block and records the event like any other infinity.  Zero products have no
+// exponent: a group without a nonzero product has T = 0 and an exponent lane that never wins a maximum.
+#include "mmasim_tfdpa_f64.cuh"
+
+namespace mmasim {
+namespace fast64 {
+
+namespace {
+
+using fast::EK_LUT8;
+using fast::EK_F16;
+using fast::EK_BF16;
+using fast::EK_TF32;
+
+struct TrAcc {
+    int cs;     // signed 24-bit significand (two's complement): value = cs * 2^(ce - CB - 23)
+    int ce;     // Exp(c) + CB; 0 for c = 0
+};
+
+__device__ __forceinline__ TrAcc tr_from_word(uint32_t w, uint32_t& sp) {
+    const AccDec d = decode_acc(w, false);
+    TrAcc a;
+    if (d.cls != CLS_FINITE) {
+        sp |= (d.cls == CLS_NAN) ? 1u : (d.sign ? 4u : 2u);
+        a.cs = 0;
+        a.ce = 0;
+        return a;
+    }
+    a.cs = d.sign ? -int(d.sig) : int(d.sig);
+    a.ce = d.sig ? d.exp + CB : 0;      // a zero accumulator has no exponent: 0 never decides E
+    return a;
+}
+
+__device__ __forceinline__ uint32_t tr_to_word(const TrAcc& a, uint32_t sp) {
+    if (sp) {
+        const int kind = ((sp & 1u) || (sp & 6u) == 6u) ? 1 : ((sp & 2u) ? 2 : 3);
+        return special_word(kind, false, false);
+    }
+    const uint32_t sign = a.cs < 0;
+    const uint32_t sig = uint32_t(abs(a.cs));
+    const uint32_t field = (sig >> 23) ? uint32_t(a.ce - CB + 127) : 0u;
+    return (sign << 31) | (field << 23) | (sig & 0x7FFFFFu);
+}
+
+__device__ __forceinline__ long long asr64_clamp(long long x, int d) { return x >> (d > 63 ? 63 : d); }
+
+// RNE-FP32 of S * 2^(eb - CB) for a 64-bit S when the result is a normal number or zero; otherwise (vmin / vmax leave
+// the normal range) the caller redoes the conversion with the generic routine.
+__device__ __forceinline__ void rne32_fast(long long S, int eb, TrAcc& a, int& vmin, int& vmax) {
+    const long long sg = S >> 63;
+    const unsigned long long mag = (unsigned long long)((S ^ sg) - sg);
+    const int msb = 63 - __clzll((long long)mag);                   // -1 for zero
+    const unsigned long long norm = msb >= 0 ? (mag << (63 - msb)) : 0ull;
+    const unsigned long long n2 = norm >> 1;                        // leading one at bit 62; 24 bits kept, 39 dropped
+    const unsigned long long r = (n2 + (((1ull << 38) - 1ull) + ((n2 >> 39) & 1ull))) >> 39;
+    const int carry = int(r >> 24);
+    const int sig = int(r >> carry);
+    int ve = eb + msb + carry;
+    ve = mag ? ve : -126 + CB;
+    vmin = min(vmin, ve);
+    vmax = max(vmax, ve);
+    a.ce = mag ? ve : 0;
+    a.cs = sg ? -sig : sig;
+}
+
+__device__ __noinline__ void rne32_slow(long long S, int e, TrAcc& a, uint32_t& sp) {
+    const uint32_t w = rho_apply(RHO_RNE_FP32, S, e);
+    a = tr_from_word(w, sp);
+}
+
+template <int EK, int L, bool GTR>
+__global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g) {
+    constexpr int NBLK = KC / L;
+    constexpr int EMINB = -126 + CB, EMAXB = 127 + CB;
+    static_assert(KC % L == 0 && L % 2 == 0, "blocks tile the chunk; the exponent pass handles pairs of elements");
+    using SM = Smem64<EK>;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    SM& sm = *reinterpret_cast<SM*>(smem_raw);
+
+    const int tid = threadIdx.x;
+    const int tx = tid % 16, ty = tid / 16;
+    const int64_t row0 = int64_t(blockIdx.y) * BM, col0 = int64_t(blockIdx.x) * BN;
+    const FmtDesc fa = fmt_desc(m.fmt_a), fb = fmt_desc(m.fmt_b);
+    const int F = m.F, F2 = m.F2;
+    const int frac = fa.mbits + fb.mbits;
+    // high word of 1.5 * 2^52 * 2^(e_max - F) is (e_max + CB) * 2^20 + MAGIC_K
+    const int MAGIC_E = 1023 + 52 - F - CB;
+    const int MAGIC_K = (MAGIC_E << 20) | 0x00080000;
+
+    init_lut64<EK>(sm, fa, fb, tid);
+    if (tid == 0) sm.special[0] = sm.special[1] = sm.special[2] = 0;
+
+    TrAcc acc[TM][TN];
+    uint32_t sp_nan = 0u, sp_pinf = 0u, sp_ninf = 0u;
+#pragma unroll
+    for (int r = 0; r < TM; ++r)
+#pragma unroll
+        for (int c = 0; c < TN; ++c) {
+            const int64_t i = row0 + ty * TM + r, j = col0 + col_of(tx, c);
+            uint32_t w = 0u;
+            if (g.C && i < g.M && j < g.N) w = static_cast<const uint32_t*>(g.C)[i * g.ldc + j];
+            uint32_t ev = 0u;
+            acc[r][c] = tr_from_word(w, ev);
+            sp_nan |= (ev & 1u) << (r * TN + c);
+            sp_pinf |= ((ev >> 1) & 1u) << (r * TN + c);
+            sp_ninf |= ((ev >> 2) & 1u) << (r * TN + c);
+        }
+
+    RawChunk<EK> raw;
+    load_chunk<EK>(raw, g, row0, col0, 0, tid);
+    __syncthreads();                                    // tables and flags are ready
+    store_chunk64<EK>(sm, sm.pl[0], raw, 0, tid);
+    if (KC < g.K) load_chunk<EK>(raw, g, row0, col0, KC, tid);
+    __syncthreads();
+    uint32_t emp[TM][TN];                               // product exponents of the block that comes next (low lane: even elements)
+    product_exponents<L>(&sm.pl[0].a_exp2[0][ty * TM], &sm.pl[0].b_exp2[0][tx * 2], emp);
+
+    int chunk = 0;
+    for (int64_t k0 = 0; k0 < g.K; k0 += KC, ++chunk) {
+        auto& s = sm.pl[chunk & 1];
+        auto& nx = sm.pl[(chunk + 1) & 1];
+        if (tid == 0) sm.special[(chunk + 2) % 3] = 0;
+        __syncthreads();                                // every warp has left the other buffer
+        if (k0 + KC < g.K) {
+            store_chunk64<EK>(sm, nx, raw, (chunk + 1) % 3, tid);
+            if (k0 + 2 * KC < g.K) load_chunk<EK>(raw, g, row0, col0, k0 + 2 * KC, tid);
+        }
+        __syncthreads();                                // the other buffer is complete
+        const bool chunk_special = sm.special[chunk % 3] != 0;
+
+#pragma unroll 1
+        for (int blk = 0; blk < NBLK; ++blk) {
+            const int kb = blk * L;
+            // ---- sum registers: the bare constants at the maximum exponents of this block's products ----
+            double t0[TM][TN], t1[GTR ? TM : 1][GTR ? TN : 1];
+            int emax_all = 0;
+#pragma unroll
+            for (int r = 0; r < TM; ++r)
+#pragma unroll
+                for (int c = 0; c < TN; ++c) {
+                    const int lo = int(emp[r][c] & 0xFFFFu), hi = int(emp[r][c] >> 16);
+                    if (GTR) {
+                        t0[r][c] = __hiloint2double(lo * (1 << 20) + MAGIC_K, 0);
+                        t1[GTR ? r : 0][GTR ? c : 0] = __hiloint2double(hi * (1 << 20) + MAGIC_K, 0);
+                    } else {
+                        t0[r][c] = __hiloint2double(max(lo, hi) * (1 << 20) + MAGIC_K, 0);
+                    }
+                    emax_all = max(emax_all, max(lo, hi));
+                }
+            // ---- rare: infinities / NaNs in the chunk, or products that may reach 2^128: events of this block ----
+            if (chunk_special || emax_all - CB >= 126) {
+#pragma unroll 1
+                for (int r = 0; r < TM; ++r)
+#pragma unroll 1
+                    for (int c = 0; c < TN; ++c) {
+                        const int64_t i = row0 + ty * TM + r, j = col0 + col_of(tx, c);
+                        if (i >= g.M || j >= g.N) continue;
+                        Special ev;
+                        for (int kk = kb; kk < kb + L; ++kk) {
+                            const uint32_t x = decode_elem(fa, raw_elem<EK>(g.A, i * g.lda + k0 + kk));
+                            const uint32_t y = decode_elem(fb, raw_elem<EK>(g.B, j * g.ldb + k0 + kk));
+                            ev.product(x, y);
+                            if ((dec_cls(x) | dec_cls(y)) == 0u) {
+                                const int sk = dec_ssig(x) * dec_ssig(y);
+                                if (product_overflows(sk, dec_exp(x) + dec_exp(y), frac)) ev.add_inf(sk < 0);
+                            }
+                        }
+                        const uint32_t bit = 1u << (r * TN + c);
+                        if (ev.nan) sp_nan |= bit;
+                        if (ev.pinf) sp_pinf |= bit;
+                        if (ev.ninf) sp_ninf |= bit;
+                    }
+            }
+            // ---- one fused multiply-add per term; beside it the product exponents of the block that follows ----
+            {
+                const double* a_p = &s.a_d[kb][ty * TM];
+                const double* b_p = &s.b_d[kb][tx * 2];
+                const bool same = blk + 1 < NBLK;
+                const uint32_t* ea_p = same ? &s.a_exp2[(kb + L) / 2 < KC / 2 ? (kb + L) / 2 : 0][ty * TM] : &nx.a_exp2[0][ty * TM];
+                const uint32_t* eb_p = same ? &s.b_exp2[(kb + L) / 2 < KC / 2 ? (kb + L) / 2 : 0][tx * 2] : &nx.b_exp2[0][tx * 2];
+#pragma unroll
+                for (int r = 0; r < TM; ++r)
+#pragma unroll
+                    for (int c = 0; c < TN; ++c) emp[r][c] = 0u;
+#pragma unroll
+                for (int kq = 0; kq < L; ++kq) {
+                    double av[TM], bv[TN];
+#pragma unroll
+                    for (int r = 0; r < TM; r += 2) {
+                        const double2 t = *reinterpret_cast<const double2*>(a_p + kq * BM + r);
+                        av[r] = t.x; av[r + 1] = t.y;
+                    }
+                    {
+                        const double2 u0 = *reinterpret_cast<const double2*>(b_p + kq * BN);
+                        const double2 u1 = *reinterpret_cast<const double2*>(b_p + kq * BN + BN / 2);
+                        bv[0] = u0.x; bv[1] = u0.y; bv[2] = u1.x; bv[3] = u1.y;
+                    }
+                    uint32_t ea[TM], ebv[TN];
+                    if ((kq & 1) == 0) {
+                        const int kp = kq / 2;
+                        const uint4 ea0 = *reinterpret_cast<const uint4*>(ea_p + kp * BM);
+                        const uint2 eb0 = *reinterpret_cast<const uint2*>(eb_p + kp * BN);
+                        const uint2 eb1 = *reinterpret_cast<const uint2*>(eb_p + kp * BN + BN / 2);
+                        ea[0] = ea0.x; ea[1] = ea0.y; ea[2] = ea0.z; ea[3] = ea0.w;
+                        ebv[0] = eb0.x; ebv[1] = eb0.y; ebv[2] = eb1.x; ebv[3] = eb1.y;
+                    }
+#pragma unroll
+                    for (int r = 0; r < TM; ++r)
+#pragma unroll
+                        for (int c = 0; c < TN; ++c) {
+                            if (GTR && (kq & 1)) t1[GTR ? r : 0][GTR ? c : 0] = __fma_rd(av[r], bv[c], t1[GTR ? r : 0][GTR ? c : 0]);
+                            else t0[r][c] = __fma_rd(av[r], bv[c], t0[r][c]);
+                            if ((kq & 1) == 0) emp[r][c] = __viaddmax_s16x2(ea[r], ebv[c], emp[r][c]);
+                        }
+                }
+            }
+            // ---- merge, add the accumulator at E = max(e_max, Exp(c)) with round-down, RNE-FP32 ----
+            const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
+#pragma unroll
+            for (int r = 0; r < TM; ++r) {
+                const uint32_t sa = s.a_sgn[ty * TM + r], nza = s.a_nz[ty * TM + r] & kmask;
+#pragma unroll
+                for (int c = 0; c < TN; ++c) {
+                    const uint32_t negm = (sa ^ s.b_sgn[col_of(tx, c)]) & nza & s.b_nz[col_of(tx, c)];
+                    // the low word of a sum register is T (two's complement, |T| < 2^31); its exponent field gives e_max + CB
+                    int T, emaxb;
+                    if (GTR) {
+                        const int te = __double2loint(t0[r][c]) + __popc(negm & 0x55555555u);
+                        const int to = __double2loint(t1[GTR ? r : 0][GTR ? c : 0]) + __popc(negm & 0xAAAAAAAAu);
+                        const int ee = (__double2hiint(t0[r][c]) >> 20) - MAGIC_E;
+                        const int eo = (__double2hiint(t1[GTR ? r : 0][GTR ? c : 0]) >> 20) - MAGIC_E;
+                        emaxb = max(ee, eo);
+                        T = fast::asr_clamp(te, emaxb - ee) + fast::asr_clamp(to, emaxb - eo);      // RD_F of both group sums
+                    } else {
+                        T = __double2loint(t0[r][c]) + __popc(negm);
+                        emaxb = (__double2hiint(t0[r][c]) >> 20) - MAGIC_E;
+                    }
+                    const TrAcc a = acc[r][c];
+                    const int E = max(emaxb, a.ce);
+                    const long long T2 = asr64_clamp((long long)T << (F2 - F), E - emaxb);       // RD_F2
+                    long long sc2 = asr64_clamp((long long)a.cs << (F - 23), E - a.ce);           // RD_F
+                    if (GTR && a.ce < E - F - 1) sc2 = 0;                                         // special truncation
+                    const long long S = T2 + (sc2 << (F2 - F));
+                    int vmin = EMINB, vmax = EMINB;
+                    rne32_fast(S, E - F2, acc[r][c], vmin, vmax);
+                    if (vmin < EMINB || vmax > EMAXB) {
+                        // the result is subnormal or overflows: by the book
+                        uint32_t ev = 0u;
+                        rne32_slow(S, E - CB - F2, acc[r][c], ev);
+                        const uint32_t bit = 1u << (r * TN + c);
+                        if (ev && !((sp_nan | sp_pinf | sp_ninf) & bit)) {         // overflow to infinity
+                            if (ev & 2u) sp_pinf |= bit;
+                            if (ev & 4u) sp_ninf |= bit;
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+#pragma unroll
+    for (int r = 0; r < TM; ++r)
+#pragma unroll
+        for (int c = 0; c < TN; ++c) {
+            const int64_t i = row0 + ty * TM + r, j = col0 + col_of(tx, c);
+            if (i >= g.M || j >= g.N) continue;
+            const uint32_t bit = r * TN + c;
+            const uint32_t spv = ((sp_nan >> bit) & 1u) | (((sp_pinf >> bit) & 1u) << 1) | (((sp_ninf >> bit) & 1u) << 2);
+            uint32_t w = tr_to_word(acc[r][c], spv);
+            if (g.row_scale) {
+                float sc = __fmul_rn(g.row_scale[i], g.col_scale[j]);
+                if (sc != sc) sc = __uint_as_float(0x7FFFFFFFu);
+                float v = __fmul_rn(sc, __uint_as_float(w));
+                if (v != v) v = __uint_as_float(0x7FFFFFFFu);
+                w = __float_as_uint(v);
+            }
+            static_cast<uint32_t*>(g.D)[i * g.ldd + j] = w;
+        }
+}
+
+template <int EK, int L, bool GTR>
+cudaError_t launch_tr_one(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
+    const size_t sh = sizeof(Smem64<EK>);
+    cudaError_t err = cudaFuncSetAttribute(trfdpa64_kernel<EK, L, GTR>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
+    if (err != cudaSuccess) return err;
+    dim3 grid((unsigned)((g.N + BN - 1) / BN), (unsigned)((g.M + BM - 1) / BM), 1);
+    trfdpa64_kernel<EK, L, GTR><<<grid, NT, sh, stream>>>(m, g);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_tr64(const DevModel& m, const GemmArgs& g, cudaStream_t st) {
+    if (m.family == FAM_GTR) return launch_tr_one<EK_LUT8, 16, true>(m, g, st);
+    if (m.fmt_a == EF_F16) return launch_tr_one<EK_F16, 8, false>(m, g, st);
+    if (m.fmt_a == EF_BF16) return launch_tr_one<EK_BF16, 8, false>(m, g, st);
+    if (m.fmt_a == EF_TF32) return launch_tr_one<EK_TF32, 4, false>(m, g, st);
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace fast64
+
+namespace fast {
+cudaError_t launch_tr(const DevModel& m, const GemmArgs& g, cudaStream_t st) { return fast64::launch_tr64(m, g, st); }
+}  // namespace fast
+}  // namespace mmasim
