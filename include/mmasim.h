@@ -161,6 +161,16 @@ typedef enum {
 } mmasim_hw_kind;
 int mmasim_hw_mma(int kind, int64_t M, int64_t K, const void* A, const void* B, const void* C, void* D, void* stream);
 
+/* Error statistics of n model outputs D (accumulator words, acc_fmt MMASIM_ACC_F32 or MMASIM_ACC_F16) against an
+ * FP64 reference `ref` (n doubles): the reduction behind the accuracy analysis of Section 6 - the deviation
+ * delta = D - D_real of Figure 3 (Section 6.2.4), its sign balance and its size.  `stats` (device, 8 doubles) is
+ * ACCUMULATED into (the caller zeroes it; several calls may share it):
+ *   [0] outputs counted (pairs where D or ref is NaN or infinite are skipped)   [1] sum of delta
+ *   [2] sum of |delta|   [3] sum of delta^2   [4] number of delta < 0   [5] number of delta > 0
+ *   [6] max |delta|      [7] sum of |delta| / |ref| over ref != 0
+ * All pointers are device pointers. */
+int mmasim_error_stats(int acc_fmt, int64_t n, const void* D, const double* ref, double* stats, void* stream);
+
 /* Integer-issue micro-benchmark used as the roofline denominator (no counterpart in the paper): launches
  * `blocks` CTAs of 256 threads, each thread running `iters` rounds of 8 independent dependent-chain integer
  * operations of the given kind (0: 3-input add, 1: logic, 2: funnel shift, 3: 32-bit multiply-add, 4: the

@@ -6,7 +6,7 @@ it), ``.build`` compiles the library in-tree, ``.workloads`` holds the seeded in
 import importlib
 
 _BINDING = ("ARCH", "FMT", "ACC", "FAMILY", "RHO", "Model", "MmasimError", "create_model", "gemm", "gemm_host",
-            "dot_batch", "int_peak", "last_kernel", "library_path", "model_keys", "PEAK_KINDS", "hw_mma", "HW_KINDS")
+            "dot_batch", "int_peak", "last_kernel", "library_path", "model_keys", "PEAK_KINDS", "hw_mma", "HW_KINDS", "error_stats", "STAT_NAMES")
 
 
 def __getattr__(name):

@@ -290,6 +290,12 @@ int mmasim_hw_mma(int kind, int64_t M, int64_t K, const void* A, const void* B, 
     return launch_hw_mma(kind, M, K, A, B, C, D, static_cast<cudaStream_t>(stream));
 }
 
+int mmasim_error_stats(int acc_fmt, int64_t n, const void* D, const double* ref, double* stats, void* stream) {
+    if (!D || !ref || !stats || n < 1) { set_error("mmasim_error_stats: bad argument"); return MMASIM_ERR_INVALID_ARG; }
+    return launch_error_stats(acc_fmt == MMASIM_ACC_F16 ? ACC_F16 : (acc_fmt == MMASIM_ACC_F32 ? ACC_F32 : -1), n, D, ref, stats,
+                              static_cast<cudaStream_t>(stream));
+}
+
 const char* mmasim_last_kernel(void) { return g_kernel; }
 const char* mmasim_last_error(void) { return g_error; }
 

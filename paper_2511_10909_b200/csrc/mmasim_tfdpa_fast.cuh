@@ -64,36 +64,27 @@ struct LutEntry {
     uint32_t special;   // nonzero for infinity / NaN
 };
 
-// Staged operands of one chunk.  SLIM drops the planes that the FP32 summation path does not read.
-template <int EK, bool SLIM = false>
+// Staged operands of one chunk (8-bit element kinds; the 16/32-bit kinds are staged by mmasim_tfdpa_f64.cuh).
+template <int EK>
 struct Planes {
-    uint32_t a_op[KC][BM];
-    uint32_t b_op[KC][BN];
-    uint32_t a_exp[SLIM ? 1 : KC][BM];
-    uint32_t b_exp[SLIM ? 1 : KC][BN];
+    uint32_t a_op[KC][BM];          // FP32 words: A_op * 2^Exp(a)
+    uint32_t b_op[KC][BN];          // FP32 words: B_op * 2^(Exp(b) - FP_SHIFT)
     uint32_t a_exp2[KC / 2][BM];    // exponents of elements 2p (low half) and 2p + 1 (high half)
     uint32_t b_exp2[KC / 2][BN];
-    uint32_t a_msk[Elem<EK>::SIGNMAG ? KC : 1][BM];   // 0 / ~0: sign of the element (sign-magnitude kinds)
-    uint32_t b_msk[Elem<EK>::SIGNMAG ? KC : 1][BN];
     uint32_t a_sgn[BM], a_nz[BM], b_sgn[BN], b_nz[BN];   // bit k of row r: sign / nonzero of element k of the chunk
 };
 
-template <int EK, bool SLIM = false, int NBUF = 1>
+template <int EK, int NBUF = 2>
 struct Smem {
-    Planes<EK, SLIM> pl[NBUF];
-    LutEntry lut_a[Elem<EK>::SIGNMAG ? 1 : 256];
-    LutEntry lut_b[Elem<EK>::SIGNMAG ? 1 : 256];
-    int special[3];                                   // chunk (by index mod 2 or 3) holds an infinity or a NaN
+    Planes<EK> pl[NBUF];
+    LutEntry lut_a[256];
+    LutEntry lut_b[256];
+    int special[3];                                   // chunk (by index mod 3) holds an infinity or a NaN
 };
 
 __device__ __forceinline__ int asr_clamp(int x, int d) {
     int r;
     asm("shr.s32 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(d));      // amounts above 31 behave as 31 (sign fill)
-    return r;
-}
-__device__ __forceinline__ uint32_t lsr_clamp(uint32_t x, int d) {
-    uint32_t r;
-    asm("shr.u32 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(d));      // amounts above 31 give 0
     return r;
 }
 __device__ __forceinline__ uint32_t shl_clamp(uint32_t x, int d) {
@@ -106,12 +97,6 @@ __device__ __forceinline__ int msb_index(uint32_t x) {
     asm("bfind.u32 %0, %1;" : "=r"(r) : "r"(x));                // -1 for x == 0
     return r;
 }
-__device__ __forceinline__ int mad_one(int t, int one, int s) {
-    int r;
-    asm("mad.lo.s32 %0, %1, %2, %3;" : "=r"(r) : "r"(t), "r"(one), "r"(s));
-    return r;
-}
-
 // Accumulator state of one output.
 struct Acc {
     int cs;     // one's complement signed significand, F fractional bits relative to 2^(ce - CB)
@@ -210,37 +195,29 @@ __device__ __forceinline__ void decode_signmag(uint32_t w, uint32_t& sig, uint32
     expb = sig ? uint32_t(int(field ? field : 1u) - E::BIAS + EB) : 0u;
 }
 
-// Decode tables of the 8-bit kinds: entry `tid` of both (256 threads).
+// Decode tables of the 8-bit kinds: entry `tid` of both (256 threads).  The staged operands are the floating-point
+// form of the integer operands of the header comment: the operand scaled by 2^Exp, exact in FP32 (at most 4 + 15
+// significant bits, exponents far inside the FP32 range).  A zero b is staged as 0 (its terms vanish and are not
+// counted as negative): with the zero terms outside e_max nothing bounds sig_a * 2^(Exp(a) + Exp_min(b)) below one
+// unit of the sum.
 template <int EK, class SM>
-__device__ __forceinline__ void init_lut(SM& s, const FmtDesc& fa, const FmtDesc& fb, int pre, int guard, int tid,
-                                         bool fpsum = false) {
-    constexpr bool SIGNMAG = Elem<EK>::SIGNMAG;
-    if (!SIGNMAG) {
-        const uint32_t da = decode_elem(fa, uint32_t(tid)), db = decode_elem(fb, uint32_t(tid));
-        const bool fin_a = dec_cls(da) == CLS_FINITE, fin_b = dec_cls(db) == CLS_FINITE;
-        LutEntry ea, eb;
-        const bool nz_a = fin_a && dec_sig(da) != 0u, nz_b = fin_b && dec_sig(db) != 0u;
-        ea.op = fin_a ? uint32_t(dec_ssig(da)) : 0u;
-        ea.exp = nz_a ? uint32_t(dec_exp(da) + EB) : 0u;         // zero, infinity, NaN: no exponent
-        ea.bits = fin_a ? (dec_sign(da) | (uint32_t(nz_a) << 16)) : 0u;
-        ea.special = fin_a ? 0u : 1u;
-        const int sb = fin_b ? dec_ssig(db) : 0;
-        const int ub = fin_b ? (dec_sign(db) ? -1 : 1) : 0;     // also for b = +-0 (see the header comment)
-        eb.op = uint32_t(sb * (1 << (pre + guard)) + ub);
-        eb.exp = nz_b ? uint32_t(dec_exp(db) + EB) : 0u;
-        eb.bits = fin_b ? (dec_sign(db) | (uint32_t(nz_b) << 16)) : 0u;
-        eb.special = fin_b ? 0u : 1u;
-        if (fpsum) {
-            // floating-point form of the same operands (see the FP32 summation path of the kernel): the operand scaled
-            // by 2^Exp, exact in FP32 (at most 4 + 15 significant bits, exponents far inside the FP32 range).  A zero b
-            // is staged as 0 there (its terms vanish and are not counted as negative): with the zero terms outside
-            // e_max nothing bounds sig_a * 2^(Exp(a) + Exp_min(b)) below one unit of the sum any more.
-            ea.op = __float_as_uint(ldexpf(float(fin_a ? dec_ssig(da) : 0), fin_a ? dec_exp(da) : 0));
-            eb.op = nz_b ? __float_as_uint(ldexpf(float(sb * (1 << (pre + guard)) + ub), dec_exp(db) - FP_SHIFT)) : 0u;
-        }
-        s.lut_a[tid] = ea;
-        s.lut_b[tid] = eb;
-    }
+__device__ __forceinline__ void init_lut(SM& s, const FmtDesc& fa, const FmtDesc& fb, int pre, int guard, int tid) {
+    const uint32_t da = decode_elem(fa, uint32_t(tid)), db = decode_elem(fb, uint32_t(tid));
+    const bool fin_a = dec_cls(da) == CLS_FINITE, fin_b = dec_cls(db) == CLS_FINITE;
+    const bool nz_a = fin_a && dec_sig(da) != 0u, nz_b = fin_b && dec_sig(db) != 0u;
+    LutEntry ea, eb;
+    ea.op = __float_as_uint(ldexpf(float(fin_a ? dec_ssig(da) : 0), fin_a ? dec_exp(da) : 0));
+    ea.exp = nz_a ? uint32_t(dec_exp(da) + EB) : 0u;             // zero, infinity, NaN: no exponent
+    ea.bits = fin_a ? (dec_sign(da) | (uint32_t(nz_a) << 16)) : 0u;
+    ea.special = fin_a ? 0u : 1u;
+    const int sb = fin_b ? dec_ssig(db) : 0;
+    const int ub = dec_sign(db) ? -1 : 1;
+    eb.op = nz_b ? __float_as_uint(ldexpf(float(sb * (1 << (pre + guard)) + ub), dec_exp(db) - FP_SHIFT)) : 0u;
+    eb.exp = nz_b ? uint32_t(dec_exp(db) + EB) : 0u;
+    eb.bits = fin_b ? (dec_sign(db) | (uint32_t(nz_b) << 16)) : 0u;
+    eb.special = fin_b ? 0u : 1u;
+    s.lut_a[tid] = ea;
+    s.lut_b[tid] = eb;
 }
 
 // Staging of one chunk of KC elements of K, in two steps so that the global loads of the next chunk can be in flight
@@ -280,11 +257,11 @@ __device__ __forceinline__ void load_chunk(RawChunk<EK>& raw, const GemmArgs& g,
     }
 }
 
-template <int EK, bool STORE_EXP = true, class SM, class PL>
-__device__ __forceinline__ void store_chunk(SM& sm, PL& s, const RawChunk<EK>& raw, int flag, int pre, int tid) {
+template <int EK, class SM, class PL>
+__device__ __forceinline__ void store_chunk(SM& sm, PL& s, const RawChunk<EK>& raw, int flag, int tid) {
     using E = Elem<EK>;
     using R = RawChunk<EK>;
-    constexpr bool SIGNMAG = E::SIGNMAG;
+    static_assert(!E::SIGNMAG && E::TASK == 16, "table-decoded 8-bit elements, sixteen per task");
     uint32_t spec = 0u;
 #pragma unroll
     for (int it = 0; it < R::PER_THREAD; ++it) {
@@ -298,78 +275,40 @@ __device__ __forceinline__ void store_chunk(SM& sm, PL& s, const RawChunk<EK>& r
 #pragma unroll
         for (int q = 0; q < E::TASK; ++q) {
             const int kk = h * E::TASK + q;
-            uint32_t op, expb;
-            if (!SIGNMAG) {
-                const uint32_t byte = (raw.w[it][q / 4] >> (8 * (q % 4))) & 0xFFu;
-                const LutEntry e = is_a ? sm.lut_a[byte] : sm.lut_b[byte];
-                op = e.op;
-                expb = e.exp;
-                bits += e.bits << q;
-                spec |= e.special;
-            } else {
-                const uint32_t w = E::BYTES == 2 ? ((raw.w[it][q / 2] >> (16 * (q % 2))) & 0xFFFFu) : raw.w[it][q];
-                uint32_t sig, sign, special;
-                decode_signmag<EK>(w, sig, expb, sign, special);
-                op = is_a ? sig : (sig << pre);
-                bits += sign << q;
-                spec |= special;
-                if (is_a) s.a_msk[SIGNMAG ? kk : 0][r] = 0u - sign; else s.b_msk[SIGNMAG ? kk : 0][r] = 0u - sign;
-            }
-            if (is_a) { s.a_op[kk][r] = op; if (STORE_EXP) s.a_exp[kk][r] = expb; }
-            else { s.b_op[kk][r] = op; if (STORE_EXP) s.b_exp[kk][r] = expb; }
+            const uint32_t byte = (raw.w[it][q / 4] >> (8 * (q % 4))) & 0xFFu;
+            const LutEntry e = is_a ? sm.lut_a[byte] : sm.lut_b[byte];
+            bits += e.bits << q;
+            spec |= e.special;
+            if (is_a) s.a_op[kk][r] = e.op; else s.b_op[kk][r] = e.op;
             if (q & 1) {
-                const uint32_t pair = prev_exp | (expb << 16);
+                const uint32_t pair = prev_exp | (e.exp << 16);
                 if (is_a) s.a_exp2[kk / 2][r] = pair; else s.b_exp2[kk / 2][r] = pair;
             }
-            prev_exp = expb;
+            prev_exp = e.exp;
         }
-        // sign (and nonzero) bits of the task's elements go to bits [h * TASK, h * TASK + TASK) of the row's masks
-        if (E::TASK == 16) {
-            if (is_a) {
-                reinterpret_cast<uint16_t*>(&s.a_sgn[r])[h] = uint16_t(bits);
-                reinterpret_cast<uint16_t*>(&s.a_nz[r])[h] = uint16_t(bits >> 16);
-            } else {
-                reinterpret_cast<uint16_t*>(&s.b_sgn[r])[h] = uint16_t(bits);
-                reinterpret_cast<uint16_t*>(&s.b_nz[r])[h] = uint16_t(bits >> 16);
-            }
+        // sign and nonzero bits of the task's elements go to bits [h * 16, h * 16 + 16) of the row's masks
+        if (is_a) {
+            reinterpret_cast<uint16_t*>(&s.a_sgn[r])[h] = uint16_t(bits);
+            reinterpret_cast<uint16_t*>(&s.a_nz[r])[h] = uint16_t(bits >> 16);
         } else {
-            if (is_a) reinterpret_cast<uint8_t*>(&s.a_sgn[r])[h] = uint8_t(bits);
-            else reinterpret_cast<uint8_t*>(&s.b_sgn[r])[h] = uint8_t(bits);
+            reinterpret_cast<uint16_t*>(&s.b_sgn[r])[h] = uint16_t(bits);
+            reinterpret_cast<uint16_t*>(&s.b_nz[r])[h] = uint16_t(bits >> 16);
         }
     }
     if (spec) atomicOr(&sm.special[flag], 1);
 }
 
-// Load and stage in one go (no prefetch).
-template <int EK, class SM>
-__device__ __forceinline__ void stage_chunk(SM& s, const GemmArgs& g, int64_t row0, int64_t col0, int64_t k0,
-                                            int chunk, int pre, int tid) {
-    RawChunk<EK> raw;
-    load_chunk<EK>(raw, g, row0, col0, k0, tid);
-    store_chunk<EK>(s, s.pl[0], raw, chunk & 1, pre, tid);
-}
-
-template <int EK, int F>
-struct TfdpaFpsum { static constexpr bool value = !Elem<EK>::SIGNMAG && F <= 13; };
-
-template <int EK, int L, int F, int RHO, bool PROMOTE, bool ST = false>
+template <int EK, int L, int F, int RHO, bool PROMOTE>
 __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
-    using E = Elem<EK>;
-    constexpr bool SIGNMAG = E::SIGNMAG;
     constexpr bool ACC16 = RHO == RHO_RNE_FP16;
     constexpr int EMINB = (ACC16 ? -14 : -126) + CB, EMAXB = (ACC16 ? 15 : 127) + CB;
-    constexpr int NSUM = (F >= 25 && L >= 16) ? 2 : 1;       // 32-bit partial sums per block
-    constexpr int HALF = L / NSUM;
     constexpr int NBLK = KC / L;
     static_assert(KC % L == 0 && L % 2 == 0, "blocks tile the chunk; pass 1 handles pairs of elements");
-    static_assert(!ST || L == KC, "ST-FDPA: one scale factor pair per block of 32 (Algorithm 8)");
-    // FP32 summation path (8-bit inputs with F <= 13): aligned terms stay below 2^15 and block sums below 2^21, so the
-    // whole of pass 2 runs exactly on the FP32 pipe, one instruction per term (see pass 2 below).  Its staged planes
-    // are small enough for two buffers: the next chunk is decoded while the current one is computed, one barrier per chunk.
-    constexpr bool FPSUM = TfdpaFpsum<EK, F>::value;
-    static_assert(FPSUM && !ST, "this kernel is the FP32 summation form (8-bit inputs, F <= 13); F >= 23 and ST-FDPA run in mmasim_tfdpa_f64.cuh");
-    constexpr bool DB = FPSUM;
-    using SM = Smem<EK, FPSUM, DB ? 2 : 1>;
+    // FP32 summation: aligned terms stay below 2^15 and block sums below 2^21, so the whole of pass 2 runs exactly on
+    // the FP32 pipe, one instruction per term (see pass 2 below).  The staged planes are small enough for two buffers:
+    // the next chunk is decoded while the current one is computed, one barrier per chunk.
+    static_assert(!Elem<EK>::SIGNMAG && F <= 13, "8-bit inputs with F <= 13; F >= 23 and ST-FDPA run in mmasim_tfdpa_f64.cuh");
+    using SM = Smem<EK, 2>;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     SM& sm = *reinterpret_cast<SM*>(smem_raw);
 
@@ -378,10 +317,9 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
     const int64_t row0 = int64_t(blockIdx.y) * BM, col0 = int64_t(blockIdx.x) * BN;
     const FmtDesc fa = fmt_desc(m.fmt_a), fb = fmt_desc(m.fmt_b);
     const int pre = F - (fa.mbits + fb.mbits);      // left shift that gives a product F fractional bits
-    const int guard = SIGNMAG ? 0 : fa.mbits + 1;   // guard bits below the truncation point (8-bit kinds)
-    const int one = int(blockDim.x >> 8);           // 1, but not a compile-time constant (see mad_one)
+    const int guard = fa.mbits + 1;                 // guard bits below the truncation point
 
-    init_lut<EK>(sm, fa, fb, pre, guard, tid, FPSUM);
+    init_lut<EK>(sm, fa, fb, pre, guard, tid);
     if (tid == 0) sm.special[0] = sm.special[1] = sm.special[2] = 0;
 
     Acc acc[TM][TN];
@@ -404,61 +342,22 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
             MMASIM_SP_OR(r, c, ev);
         }
 
-    // The raw words of the next chunk wait in registers during the compute where the register budget allows it
-    // (the narrow-sum 8-bit variants); elsewhere the extra live registers cost more in spills than the overlap gains.
-    constexpr bool PREFETCH = EK == EK_LUT8 && NSUM == 1;
     RawChunk<EK> raw;
-    if (PREFETCH) load_chunk<EK>(raw, g, row0, col0, 0, tid);
-    if (DB) {
-        __syncthreads();                                   // tables and flags are ready
-        store_chunk<EK, !FPSUM>(sm, sm.pl[0], raw, 0, pre, tid);
-        if (KC < g.K) load_chunk<EK>(raw, g, row0, col0, KC, tid);
-        __syncthreads();
-    }
+    load_chunk<EK>(raw, g, row0, col0, 0, tid);
+    __syncthreads();                                       // tables and flags are ready
+    store_chunk<EK>(sm, sm.pl[0], raw, 0, tid);
+    if (KC < g.K) load_chunk<EK>(raw, g, row0, col0, KC, tid);
+    __syncthreads();
     int chunk = 0;
     for (int64_t k0 = 0; k0 < g.K; k0 += KC, ++chunk) {
-        int flag;
-        if (!DB) {
-            __syncthreads();
-            if (!PREFETCH) load_chunk<EK>(raw, g, row0, col0, k0, tid);
-            store_chunk<EK, !FPSUM>(sm, sm.pl[0], raw, chunk & 1, pre, tid);
-            __syncthreads();
-            if (PREFETCH && k0 + KC < g.K) load_chunk<EK>(raw, g, row0, col0, k0 + KC, tid);
-            flag = chunk & 1;
-            if (tid == 0) sm.special[(chunk + 1) & 1] = 0;
-        } else {
-            // decode chunk n + 1 into the other buffer (its raw words arrived during the previous iteration), then fetch n + 2
-            flag = chunk % 3;
-            if (tid == 0) sm.special[(chunk + 2) % 3] = 0;   // last read two barriers ago, next written after the coming one
-            if (k0 + KC < g.K) {
-                store_chunk<EK, !FPSUM>(sm, sm.pl[(chunk + 1) & 1], raw, (chunk + 1) % 3, pre, tid);
-                if (k0 + 2 * KC < g.K) load_chunk<EK>(raw, g, row0, col0, k0 + 2 * KC, tid);
-            }
+        // decode chunk n + 1 into the other buffer (its raw words arrived during the previous iteration), then fetch n + 2
+        if (tid == 0) sm.special[(chunk + 2) % 3] = 0;     // last read two barriers ago, next written after the coming one
+        if (k0 + KC < g.K) {
+            store_chunk<EK>(sm, sm.pl[(chunk + 1) & 1], raw, (chunk + 1) % 3, tid);
+            if (k0 + 2 * KC < g.K) load_chunk<EK>(raw, g, row0, col0, k0 + 2 * KC, tid);
         }
-        auto& s = sm.pl[DB ? (chunk & 1) : 0];
-        bool chunk_special = sm.special[flag] != 0;
-
-        // ST-FDPA (Algorithm 8): Exp(alpha) of this thread's rows and Exp(beta) of its columns for this block of 32
-        int sa_exp[ST ? TM : 1], sb_exp[ST ? TN : 1];
-        uint32_t scale_nan = 0u;                    // bit r * TN + c: alpha or beta of that output is NaN
-        if (ST) {
-            const int64_t sblk = k0 / KC;
-#pragma unroll
-            for (int r = 0; r < TM; ++r) {
-                const int64_t i = row0 + ty * TM + r;
-                const uint32_t w = i < g.M ? uint32_t(g.sfa[i * g.ld_sfa + sblk]) : 127u;
-                sa_exp[ST ? r : 0] = int(w) - 127;
-                if (w == 0xFFu) scale_nan |= ((1u << TN) - 1u) << (r * TN);
-            }
-#pragma unroll
-            for (int c = 0; c < TN; ++c) {
-                const int64_t j = col0 + tx * TN + c;
-                const uint32_t w = j < g.N ? uint32_t(g.sfb[j * g.ld_sfb + sblk]) : 127u;
-                sb_exp[ST ? c : 0] = int(w) - 127;
-                if (w == 0xFFu) scale_nan |= 0x11111111u << c;
-            }
-            sp_nan |= scale_nan;                    // a NaN scale factor makes the block result NaN
-        }
+        auto& s = sm.pl[chunk & 1];
+        const bool chunk_special = sm.special[chunk % 3] != 0;
 
 #pragma unroll 1
         for (int blk = 0; blk < NBLK; ++blk) {
@@ -492,11 +391,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
 #pragma unroll
                 for (int r = 0; r < TM; ++r)
 #pragma unroll
-                    for (int c = 0; c < TN; ++c) {
-                        // ST: compare the products against the accumulator exponent minus the block's scale exponents
-                        const int rel = ST ? acc[r][c].ce - sa_exp[ST ? r : 0] - sb_exp[ST ? c : 0] : acc[r][c].ce;
-                        em2[r][c] = uint32_t(rel) * 0x10001u;
-                    }
+                    for (int c = 0; c < TN; ++c) em2[r][c] = uint32_t(acc[r][c].ce) * 0x10001u;
 #pragma unroll 4
                 for (int kp = kb / 2; kp < (kb + L) / 2; ++kp) {
                     const uint4 ea0 = *reinterpret_cast<const uint4*>(&s.a_exp2[kp][ty * TM]);
@@ -516,94 +411,77 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
             }
             // ---- accumulator term: align at e_max and truncate; one's complement keeps sign-magnitude semantics,
             // the "+1 if c is negative" restores the two's complement value ----
-            int S0[TM][TN], S1[NSUM == 2 ? TM : 1][NSUM == 2 ? TN : 1];
+            int S0[TM][TN];
 #pragma unroll
             for (int r = 0; r < TM; ++r)
 #pragma unroll
                 for (int c = 0; c < TN; ++c) {
-                    const int rel = ST ? acc[r][c].ce - sa_exp[ST ? r : 0] - sb_exp[ST ? c : 0] : acc[r][c].ce;
-                    S0[r][c] = asr_clamp(acc[r][c].cs, emax[r][c] - rel) - (acc[r][c].cs >> 31);
-                    if (NSUM == 2) S1[NSUM == 2 ? r : 0][NSUM == 2 ? c : 0] = 0;
+                    S0[r][c] = asr_clamp(acc[r][c].cs, emax[r][c] - acc[r][c].ce) - (acc[r][c].cs >> 31);
                     emax[r][c] += guard;
-                    if (FPSUM) {
-                        // The sum lives in an FP32 register as (1.5 * 2^23 + S) * u, u = 2^(e_max + g - FP_SHIFT) the
-                        // value of one unit of S in the scale of the staged operands: in [2^23 u, 2^24 u) one ulp is u,
-                        // so adding a product with rounding toward minus infinity floors it onto the grid of S.
-                        // For e_max above FP_EMAX_CLAMP (only a huge accumulator gets there) the exponent is clamped:
-                        // every product is far below one unit either way and floors to 0 or -1 as it should.
-                        const int ecl = min(emax[r][c], FP_EMAX_CLAMP + CB + guard);
-                        S0[r][c] += ((ecl + (150 - CB - FP_SHIFT)) << 23) | 0x00400000;
-                    }
+                    // The sum lives in an FP32 register as (1.5 * 2^23 + S) * u, u = 2^(e_max + g - FP_SHIFT) the
+                    // value of one unit of S in the scale of the staged operands: in [2^23 u, 2^24 u) one ulp is u,
+                    // so adding a product with rounding toward minus infinity floors it onto the grid of S.
+                    // For e_max above FP_EMAX_CLAMP (only a huge accumulator gets there) the exponent is clamped:
+                    // every product is far below one unit either way and floors to 0 or -1 as it should.
+                    const int ecl = min(emax[r][c], FP_EMAX_CLAMP + CB + guard);
+                    S0[r][c] += ((ecl + (150 - CB - FP_SHIFT)) << 23) | 0x00400000;
                 }
-            // ---- pass 2: multiply, align, truncate, add ----
-            if (FPSUM) {
-                // S * u + (A_op * 2^Exp(a)) * (B_op * 2^(Exp(b) - FP_SHIFT)) = (S + X_k * 2^-(d_k + g)) * u: the fused
-                // multiply-add forms it exactly and rounds once, toward minus infinity, onto multiples of u:
-                // S <- S + floor(X_k * 2^-(d_k + g)), the same one's-complement term as the arithmetic shift of the
-                // integer path.  One instruction per term; the alignment scale is the exponent of the sum register.
+            // ---- pass 2: S * u + (A_op * 2^Exp(a)) * (B_op * 2^(Exp(b) - FP_SHIFT)) = (S + X_k * 2^-(d_k + g)) * u: the
+            // fused multiply-add forms it exactly and rounds once, toward minus infinity, onto multiples of u:
+            // S <- S + floor(X_k * 2^-(d_k + g)), the one's-complement term of the header comment.  One instruction per
+            // term; the alignment scale is the exponent of the sum register. ----
 #pragma unroll 4
-                for (int kk = kb; kk < kb + L; ++kk) {
-                    const float4 oa0 = *reinterpret_cast<const float4*>(&s.a_op[kk][ty * TM]);
-                    const float4 oa1 = *reinterpret_cast<const float4*>(&s.a_op[kk][ty * TM + 4]);
-                    const float4 ob = *reinterpret_cast<const float4*>(&s.b_op[kk][tx * TN]);
-                    const float oav[TM] = {oa0.x, oa0.y, oa0.z, oa0.w, oa1.x, oa1.y, oa1.z, oa1.w};
-                    const float obv[TN] = {ob.x, ob.y, ob.z, ob.w};
-#pragma unroll
-                    for (int r = 0; r < TM; ++r)
-#pragma unroll
-                        for (int c = 0; c < TN; ++c)
-                            S0[r][c] = __float_as_int(__fmaf_rd(oav[r], obv[c], __int_as_float(S0[r][c])));
-                }
-                // back to the integer sum; e_max + g from the exponent field, or Exp(c) + g where it was clamped
+            for (int kk = kb; kk < kb + L; ++kk) {
+                const float4 oa0 = *reinterpret_cast<const float4*>(&s.a_op[kk][ty * TM]);
+                const float4 oa1 = *reinterpret_cast<const float4*>(&s.a_op[kk][ty * TM + 4]);
+                const float4 ob = *reinterpret_cast<const float4*>(&s.b_op[kk][tx * TN]);
+                const float oav[TM] = {oa0.x, oa0.y, oa0.z, oa0.w, oa1.x, oa1.y, oa1.z, oa1.w};
+                const float obv[TN] = {ob.x, ob.y, ob.z, ob.w};
 #pragma unroll
                 for (int r = 0; r < TM; ++r)
 #pragma unroll
-                    for (int c = 0; c < TN; ++c) {
-                        const int bits = S0[r][c];
-                        S0[r][c] = bits - ((bits & 0x7F800000) | 0x00400000);
-                        emax[r][c] = max((bits >> 23) - (150 - CB - FP_SHIFT), acc[r][c].ce + guard);
-                    }
+                    for (int c = 0; c < TN; ++c)
+                        S0[r][c] = __float_as_int(__fmaf_rd(oav[r], obv[c], __int_as_float(S0[r][c])));
             }
+            // back to the integer sum; e_max + g from the exponent field, or Exp(c) + g where it was clamped
+#pragma unroll
+            for (int r = 0; r < TM; ++r)
+#pragma unroll
+                for (int c = 0; c < TN; ++c) {
+                    const int bits = S0[r][c];
+                    S0[r][c] = bits - ((bits & 0x7F800000) | 0x00400000);
+                    emax[r][c] = max((bits >> 23) - (150 - CB - FP_SHIFT), acc[r][c].ce + guard);
+                }
             // ---- sign corrections, normalisation, rho ----
             const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
             int vmin = EMINB, vmax = EMINB;
-            uint32_t ovf = 0u;                         // sign bit set: a 32-bit block sum overflowed
 #pragma unroll
             for (int r = 0; r < TM; ++r) {
                 const uint32_t sa = s.a_sgn[ty * TM + r];
-                const uint32_t nza = SIGNMAG ? kmask : (s.a_nz[ty * TM + r] & kmask);
+                const uint32_t nza = s.a_nz[ty * TM + r] & kmask;
 #pragma unroll
                 for (int c = 0; c < TN; ++c) {
                     const int nneg = __popc((sa ^ s.b_sgn[tx * TN + c]) & nza & s.b_nz[tx * TN + c]);
-                    int S = S0[r][c] + nneg;
-                    if (NSUM == 2) {
-                        const int s1 = S1[NSUM == 2 ? r : 0][NSUM == 2 ? c : 0];
-                        const int sum = S + s1;
-                        ovf |= uint32_t((S ^ sum) & (s1 ^ sum));
-                        S = sum;
-                    }
-                    rho_fast<F, RHO>(S, emax[r][c] - guard + (ST ? sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0] : 0), acc[r][c], vmin, vmax);
+                    rho_fast<F, RHO>(S0[r][c] + nneg, emax[r][c] - guard, acc[r][c], vmin, vmax);
                 }
             }
-            if (vmin < EMINB || vmax > EMAXB || int(ovf) < 0) {
-                // some result is subnormal, overflows, or a sum needs 64 bits: redo every output by the book
+            if (vmin < EMINB || vmax > EMAXB) {
+                // some result is subnormal or overflows: redo every output by the book
 #pragma unroll
                 for (int r = 0; r < TM; ++r) {
                     const uint32_t sa = s.a_sgn[ty * TM + r];
-                    const uint32_t nza = SIGNMAG ? kmask : (s.a_nz[ty * TM + r] & kmask);
+                    const uint32_t nza = s.a_nz[ty * TM + r] & kmask;
 #pragma unroll
                     for (int c = 0; c < TN; ++c) {
                         const int nneg = __popc((sa ^ s.b_sgn[tx * TN + c]) & nza & s.b_nz[tx * TN + c]);
-                        long long S = (long long)S0[r][c] + nneg;
-                        if (NSUM == 2) S += (long long)S1[NSUM == 2 ? r : 0][NSUM == 2 ? c : 0];
                         uint32_t ev = 0u;
-                        rho_slow<F, RHO, ACC16>(S, emax[r][c] - guard - CB + (ST ? sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0] : 0), acc[r][c], ev);
-                        if (ev && !MMASIM_SP_GET(r, c)) MMASIM_SP_OR(r, c, ev);   // overflow to infinity (RNE only)
+                        rho_slow<F, RHO, ACC16>((long long)S0[r][c] + nneg, emax[r][c] - guard - CB, acc[r][c], ev);
+                        if (ev && !MMASIM_SP_GET(r, c)) MMASIM_SP_OR(r, c, ev);   // overflow to infinity
                     }
                 }
             }
         }
-        if (DB) __syncthreads();                           // the other buffer is complete, this one is free
+        __syncthreads();                                   // the other buffer is complete, this one is free
         // ---- FP32 promotion of the partial sum every k_chunk elements ----
         if (PROMOTE && ((k0 + KC) % g.k_chunk) == 0) {
 #pragma unroll
@@ -644,22 +522,21 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
 #undef MMASIM_SP_OR
 }
 
-template <int EK, int L, int F, int RHO, bool PROMOTE, bool ST = false>
+template <int EK, int L, int F, int RHO, bool PROMOTE>
 cudaError_t launch_one(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
-    constexpr bool FPSUM = TfdpaFpsum<EK, F>::value;
-    const size_t sh = sizeof(Smem<EK, FPSUM, FPSUM ? 2 : 1>);
-    cudaError_t err = cudaFuncSetAttribute(tfdpa_kernel<EK, L, F, RHO, PROMOTE, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
+    const size_t sh = sizeof(Smem<EK, 2>);
+    cudaError_t err = cudaFuncSetAttribute(tfdpa_kernel<EK, L, F, RHO, PROMOTE>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
     if (err != cudaSuccess) return err;
     dim3 grid((unsigned)((g.N + BN - 1) / BN), (unsigned)((g.M + BM - 1) / BM), 1);
-    tfdpa_kernel<EK, L, F, RHO, PROMOTE, ST><<<grid, NT, sh, stream>>>(m, g);
+    tfdpa_kernel<EK, L, F, RHO, PROMOTE><<<grid, NT, sh, stream>>>(m, g);
     return cudaGetLastError();
 }
 
 // With or without FP32 promotion (FP32 accumulators only).
-template <int EK, int L, int F, int RHO, bool ST = false>
+template <int EK, int L, int F, int RHO>
 cudaError_t launch_variant(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
-    if (RHO != RHO_RNE_FP16 && g.k_chunk) return launch_one<EK, L, F, RHO, RHO != RHO_RNE_FP16, ST>(m, g, stream);
-    return launch_one<EK, L, F, RHO, false, ST>(m, g, stream);
+    if (RHO != RHO_RNE_FP16 && g.k_chunk) return launch_one<EK, L, F, RHO, RHO != RHO_RNE_FP16>(m, g, stream);
+    return launch_one<EK, L, F, RHO, false>(m, g, stream);
 }
 
 // Per element kind: returns cudaErrorInvalidValue when (L, F, rho) has no instantiation.
@@ -667,7 +544,7 @@ cudaError_t launch_lut8(const DevModel& m, const GemmArgs& g, cudaStream_t strea
 cudaError_t launch_f16(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
 cudaError_t launch_bf16(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
 cudaError_t launch_tf32(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
-cudaError_t launch_tr(const DevModel& m, const GemmArgs& g, cudaStream_t stream);    // TR-/GTR-FDPA (mmasim_trfdpa_fast.cu)
+cudaError_t launch_tr(const DevModel& m, const GemmArgs& g, cudaStream_t stream);    // TR-/GTR-FDPA (mmasim_trfdpa_f64.cu)
 
 }  // namespace fast
 }  // namespace mmasim

@@ -71,6 +71,8 @@ def _load():
     lib.mmasim_int_peak.argtypes = [c_int, c_int64, c_int64, c_void_p, POINTER(c_int32), c_void_p]
     lib.mmasim_hw_mma.restype = c_int
     lib.mmasim_hw_mma.argtypes = [c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.mmasim_error_stats.restype = c_int
+    lib.mmasim_error_stats.argtypes = [c_int, c_int64, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.mmasim_last_kernel.restype = c_char_p
     lib.mmasim_last_error.restype = c_char_p
     return lib
@@ -230,6 +232,21 @@ def gemm_host(model: Model, A, B, C=None, *, K=None, sfa=None, sfb=None, k_chunk
     o = _make_opts(p(sfa), p(sfb), k_chunk, p(row_scale), p(col_scale))
     _check(_lib.mmasim_gemm_host(model._h, M, N, K, p(A), p(B), p(C), p(out), byref(o)))
     return out
+
+
+STAT_NAMES = ["count", "sum", "sum_abs", "sum_sq", "negative", "positive", "max_abs", "sum_rel"]
+
+
+def error_stats(acc: str, D, ref, stats=None, *, stream=None):
+    """Accumulate the deviation statistics of the output words D against the FP64 reference `ref` (CUDA tensors) into
+    `stats` (8 doubles on the device, created zeroed if not given); returns `stats`."""
+    import torch
+    if not D.is_cuda or not ref.is_cuda or ref.dtype != torch.float64:
+        raise MmasimError(1, "mmasim.error_stats needs CUDA tensors and an FP64 reference")
+    if stats is None:
+        stats = torch.zeros(8, dtype=torch.float64, device=D.device)
+    _check(_lib.mmasim_error_stats(ACC[acc], D.numel(), _ptr(D), _ptr(ref), _ptr(stats), _stream(stream)))
+    return stats
 
 
 HW_KINDS = ["f16_f32", "f16_f16", "bf16_f32", "tf32_f32", "e4m3_f32", "e5m2_f32", "f64", "f16_f32_k8", "tf32_f32_k4"]
