@@ -313,7 +313,7 @@ def run_ours(args):
         h2d = hA.numel() * hA.element_size() + hB.numel() * hB.element_size() + hC.numel() * hC.element_size()
         e2e = {"value": macs_per_step / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                "d2h_bytes_per_step": int(hD.numel() * hD.element_size()), "ms_per_step": 1e3 * e2e_s,
-               "api": "mmasim_gemm_host (cudaMalloc + H2D + kernel + D2H + cudaFree per call)"}
+               "api": "mmasim_gemm_host (stream-ordered allocation + H2D + kernel + D2H + free per call)"}
 
     if rank != 0:
         if dist is not None:
