@@ -38,6 +38,7 @@
 // of the block and keep sticky NaN / +inf / -inf flags per output, Section 4.2) and results outside the normal range
 // of the accumulator format (generic conversion routine).
 #pragma once
+#include <cuda_fp16.h>
 #include "mmasim_device.cuh"
 
 namespace mmasim {
@@ -301,13 +302,13 @@ __device__ __forceinline__ void store_chunk(SM& sm, PL& s, const RawChunk<EK>& r
 template <int EK, int L, int F, int RHO, bool PROMOTE>
 __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
     constexpr bool ACC16 = RHO == RHO_RNE_FP16;
-    constexpr int EMINB = (ACC16 ? -14 : -126) + CB, EMAXB = (ACC16 ? 15 : 127) + CB;
     constexpr int NBLK = KC / L;
     static_assert(KC % L == 0 && L % 2 == 0, "blocks tile the chunk; pass 1 handles pairs of elements");
     // FP32 summation: aligned terms stay below 2^15 and block sums below 2^21, so the whole of pass 2 runs exactly on
     // the FP32 pipe, one instruction per term (see pass 2 below).  The staged planes are small enough for two buffers:
     // the next chunk is decoded while the current one is computed, one barrier per chunk.
     static_assert(!Elem<EK>::SIGNMAG && F <= 13, "8-bit inputs with F <= 13; F >= 23 and ST-FDPA run in mmasim_tfdpa_f64.cuh");
+    static_assert(RHO == RHO_RZ_E8M13 || RHO == RHO_RNE_FP16, "rho of the F = 13 rows of Table 4");
     using SM = Smem<EK, 2>;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     SM& sm = *reinterpret_cast<SM*>(smem_raw);
@@ -318,15 +319,22 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
     const FmtDesc fa = fmt_desc(m.fmt_a), fb = fmt_desc(m.fmt_b);
     const int pre = F - (fa.mbits + fb.mbits);      // left shift that gives a product F fractional bits
     const int guard = fa.mbits + 1;                 // guard bits below the truncation point
+    // The staged operands carry the products in the scale 2^(F + g - FP_SHIFT): a real value x appears as x * c_scale.
+    const float c_scale = __int_as_float((127 + F + guard - FP_SHIFT) << 23);
+    // Exponent sums outside [E_LOW, E_HIGH] (biased by CB) are blocks whose products cannot reach the result: below,
+    // every product is zero (a nonzero FP8 product has an exponent of at least -28); above, only an accumulator of
+    // 2^100 or more gets there and every product is truncated away.  The result is then the accumulator itself,
+    // truncated by rho; the sum register's exponent is clamped so that the arithmetic stays finite.
+    constexpr int E_LOW = CB - 100, E_HIGH = CB + FP_EMAX_CLAMP;
 
     init_lut<EK>(sm, fa, fb, pre, guard, tid);
     if (tid == 0) sm.special[0] = sm.special[1] = sm.special[2] = 0;
 
-    Acc acc[TM][TN];
+    uint32_t cw[TM][TN];                                // the accumulator of each output: a finite FP32 / FP16 word
     uint32_t sp_nan = 0u, sp_pinf = 0u, sp_ninf = 0u;   // per output (bit r * TN + c): NaN / +inf / -inf seen so far
     float promoted[PROMOTE ? TM : 1][PROMOTE ? TN : 1];
 #define MMASIM_SP_GET(r, c) ((((sp_nan >> ((r) * TN + (c))) & 1u)) | (((sp_pinf >> ((r) * TN + (c))) & 1u) << 1) | (((sp_ninf >> ((r) * TN + (c))) & 1u) << 2))
-#define MMASIM_SP_OR(r, c, v) do { const uint32_t v_ = (v); sp_nan |= (v_ & 1u) << ((r) * TN + (c)); sp_pinf |= ((v_ >> 1) & 1u) << ((r) * TN + (c)); sp_ninf |= ((v_ >> 2) & 1u) << ((r) * TN + (c)); } while (0)
+#define MMASIM_SP_WORD(r, c, w) (MMASIM_SP_GET(r, c) ? special_word(((MMASIM_SP_GET(r, c) & 1u) || (MMASIM_SP_GET(r, c) & 6u) == 6u) ? 1 : ((MMASIM_SP_GET(r, c) & 2u) ? 2 : 3), ACC16, true) : (w))
 #pragma unroll
     for (int r = 0; r < TM; ++r)
 #pragma unroll
@@ -337,9 +345,13 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
                 w = ACC16 ? uint32_t(static_cast<const uint16_t*>(g.C)[i * g.ldc + j])
                           : static_cast<const uint32_t*>(g.C)[i * g.ldc + j];
             if (PROMOTE) { promoted[PROMOTE ? r : 0][PROMOTE ? c : 0] = __uint_as_float(w); w = 0u; }
-            uint32_t ev = 0u;
-            acc[r][c] = acc_from_word<F, ACC16>(w, ev);
-            MMASIM_SP_OR(r, c, ev);
+            const AccDec d = decode_acc(w, ACC16);
+            if (d.cls != CLS_FINITE) {
+                const uint32_t bit = 1u << (r * TN + c);
+                if (d.cls == CLS_NAN) sp_nan |= bit; else if (d.sign) sp_ninf |= bit; else sp_pinf |= bit;
+                w = 0u;
+            }
+            cw[r][c] = w;
         }
 
     RawChunk<EK> raw;
@@ -384,14 +396,20 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
                     }
             }
 
-            int emax[TM][TN];       // e_max + CB, then e_max + CB + guard
-            // ---- pass 1: block maximum of the exponent sums, accumulator included; two elements per instruction ----
+            int S0[TM][TN];         // pass 1: e_max + CB; pass 2: the sum register; then the result word
+            int elo = E_HIGH, ehi = E_LOW;
+            // ---- pass 1: block maximum of the exponent sums, accumulator included (a zero accumulator has no
+            // exponent: 0 never wins); two elements per instruction ----
             {
                 uint32_t em2[TM][TN];
 #pragma unroll
                 for (int r = 0; r < TM; ++r)
 #pragma unroll
-                    for (int c = 0; c < TN; ++c) em2[r][c] = uint32_t(acc[r][c].ce) * 0x10001u;
+                    for (int c = 0; c < TN; ++c) {
+                        const uint32_t x = cw[r][c] & (ACC16 ? 0x7FFFu : 0x7FFFFFFFu);
+                        const uint32_t rel = max(x >> (ACC16 ? 10 : 23), 1u) + uint32_t(CB - (ACC16 ? 15 : 127));
+                        em2[r][c] = x ? rel * 0x10001u : 0u;
+                    }
 #pragma unroll 4
                 for (int kp = kb / 2; kp < (kb + L) / 2; ++kp) {
                     const uint4 ea0 = *reinterpret_cast<const uint4*>(&s.a_exp2[kp][ty * TM]);
@@ -407,24 +425,34 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
 #pragma unroll
                 for (int r = 0; r < TM; ++r)
 #pragma unroll
-                    for (int c = 0; c < TN; ++c) emax[r][c] = max(int(em2[r][c] & 0xFFFFu), int(em2[r][c] >> 16));
+                    for (int c = 0; c < TN; ++c) {
+                        const int e = max(int(em2[r][c] & 0xFFFFu), int(em2[r][c] >> 16));
+                        elo = min(elo, e);
+                        ehi = max(ehi, e);
+                        S0[r][c] = e;
+                    }
             }
-            // ---- accumulator term: align at e_max and truncate; one's complement keeps sign-magnitude semantics,
-            // the "+1 if c is negative" restores the two's complement value ----
-            int S0[TM][TN];
+            uint32_t keep = 0u;                            // outputs whose products cannot reach the result (rare)
+            if (elo < E_LOW || ehi > E_HIGH) {
+#pragma unroll
+                for (int r = 0; r < TM; ++r)
+#pragma unroll
+                    for (int c = 0; c < TN; ++c)
+                        if (S0[r][c] < E_LOW || S0[r][c] > E_HIGH) keep |= 1u << (r * TN + c);
+            }
+            // ---- the sum register: (1.5 * 2^23 + S) * u in FP32, u = 2^(e_max + g - FP_SHIFT) the value of one unit
+            // of S in the scale of the staged operands: in [2^23 u, 2^24 u) one ulp is u, so adding a product with
+            // rounding toward minus infinity floors it onto the grid of S.  It starts with the accumulator term:
+            // c' = c with the lowest mantissa bit set is never on the grid, so a negative c floors to the one's
+            // complement of its truncated magnitude (+1 for the sign in the correction below). ----
 #pragma unroll
             for (int r = 0; r < TM; ++r)
 #pragma unroll
                 for (int c = 0; c < TN; ++c) {
-                    S0[r][c] = asr_clamp(acc[r][c].cs, emax[r][c] - acc[r][c].ce) - (acc[r][c].cs >> 31);
-                    emax[r][c] += guard;
-                    // The sum lives in an FP32 register as (1.5 * 2^23 + S) * u, u = 2^(e_max + g - FP_SHIFT) the
-                    // value of one unit of S in the scale of the staged operands: in [2^23 u, 2^24 u) one ulp is u,
-                    // so adding a product with rounding toward minus infinity floors it onto the grid of S.
-                    // For e_max above FP_EMAX_CLAMP (only a huge accumulator gets there) the exponent is clamped:
-                    // every product is far below one unit either way and floors to 0 or -1 as it should.
-                    const int ecl = min(emax[r][c], FP_EMAX_CLAMP + CB + guard);
-                    S0[r][c] += ((ecl + (150 - CB - FP_SHIFT)) << 23) | 0x00400000;
+                    const int ecl = max(min(S0[r][c], E_HIGH), E_LOW) + guard;
+                    const float magic = __int_as_float(((ecl + (150 - CB - FP_SHIFT)) << 23) | 0x00400000);
+                    const float cf = ACC16 ? __half2float(__ushort_as_half((unsigned short)cw[r][c])) : __uint_as_float(cw[r][c]);
+                    S0[r][c] = __float_as_int(__fmaf_rd(__int_as_float(__float_as_int(cf) | 1), c_scale, magic));
                 }
             // ---- pass 2: S * u + (A_op * 2^Exp(a)) * (B_op * 2^(Exp(b) - FP_SHIFT)) = (S + X_k * 2^-(d_k + g)) * u: the
             // fused multiply-add forms it exactly and rounds once, toward minus infinity, onto multiples of u:
@@ -443,18 +471,11 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
                     for (int c = 0; c < TN; ++c)
                         S0[r][c] = __float_as_int(__fmaf_rd(oav[r], obv[c], __int_as_float(S0[r][c])));
             }
-            // back to the integer sum; e_max + g from the exponent field, or Exp(c) + g where it was clamped
-#pragma unroll
-            for (int r = 0; r < TM; ++r)
-#pragma unroll
-                for (int c = 0; c < TN; ++c) {
-                    const int bits = S0[r][c];
-                    S0[r][c] = bits - ((bits & 0x7F800000) | 0x00400000);
-                    emax[r][c] = max((bits >> 23) - (150 - CB - FP_SHIFT), acc[r][c].ce + guard);
-                }
-            // ---- sign corrections, normalisation, rho ----
+            // ---- sign corrections and rho: S = register - constant + (negative terms) + (c < 0), value S * 2^(e_max - F)
+            // (exact in FP32: |S| < 2^22), then RZ-E8M13 = the low 10 mantissa bits cleared, or RNE-FP16 = one
+            // conversion.  The scale is read from the register's exponent field. ----
             const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
-            int vmin = EMINB, vmax = EMINB;
+            uint32_t wmax = 0u;
 #pragma unroll
             for (int r = 0; r < TM; ++r) {
                 const uint32_t sa = s.a_sgn[ty * TM + r];
@@ -462,24 +483,42 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
 #pragma unroll
                 for (int c = 0; c < TN; ++c) {
                     const int nneg = __popc((sa ^ s.b_sgn[tx * TN + c]) & nza & s.b_nz[tx * TN + c]);
-                    rho_fast<F, RHO>(S0[r][c] + nneg, emax[r][c] - guard, acc[r][c], vmin, vmax);
+                    const int bits = S0[r][c];
+                    const int fld = bits & 0x7F800000;
+                    const int S = bits - (fld | 0x00400000) + nneg + int(cw[r][c] >> (ACC16 ? 15 : 31));
+                    const float scale = __int_as_float(fld - ((15 + F + guard) << 23));       // 2^(e_max - F)
+                    const float v = __fmul_rn(__int2float_rn(S), scale);
+                    uint32_t w;
+                    if (ACC16) { w = uint32_t(__half_as_ushort(__float2half_rn(v))); wmax = max(wmax, w & 0x7FFFu); }
+                    else w = __float_as_uint(v) & 0xFFFFFC00u;
+                    S0[r][c] = int(w);
                 }
             }
-            if (vmin < EMINB || vmax > EMAXB) {
-                // some result is subnormal or overflows: redo every output by the book
+            if (keep) {                                    // rare: rho of the accumulator alone; an exactly zero sum is +0
 #pragma unroll
-                for (int r = 0; r < TM; ++r) {
-                    const uint32_t sa = s.a_sgn[ty * TM + r];
-                    const uint32_t nza = s.a_nz[ty * TM + r] & kmask;
+                for (int r = 0; r < TM; ++r)
 #pragma unroll
-                    for (int c = 0; c < TN; ++c) {
-                        const int nneg = __popc((sa ^ s.b_sgn[tx * TN + c]) & nza & s.b_nz[tx * TN + c]);
-                        uint32_t ev = 0u;
-                        rho_slow<F, RHO, ACC16>((long long)S0[r][c] + nneg, emax[r][c] - guard - CB, acc[r][c], ev);
-                        if (ev && !MMASIM_SP_GET(r, c)) MMASIM_SP_OR(r, c, ev);   // overflow to infinity
-                    }
-                }
+                    for (int c = 0; c < TN; ++c)
+                        if ((keep >> (r * TN + c)) & 1u) {
+                            const uint32_t t = ACC16 ? cw[r][c] : (cw[r][c] & 0xFFFFFC00u);
+                            S0[r][c] = int((t & (ACC16 ? 0x7FFFu : 0x7FFFFFFFu)) ? t : 0u);
+                        }
             }
+            if (ACC16 && wmax >= 0x7C00u) {                // rare: RNE-FP16 overflowed: +-infinity from now on
+#pragma unroll
+                for (int r = 0; r < TM; ++r)
+#pragma unroll
+                    for (int c = 0; c < TN; ++c)
+                        if ((uint32_t(S0[r][c]) & 0x7FFFu) == 0x7C00u) {
+                            const uint32_t bit = 1u << (r * TN + c);
+                            if (!((sp_nan | sp_pinf | sp_ninf) & bit)) { if (uint32_t(S0[r][c]) >> 15) sp_ninf |= bit; else sp_pinf |= bit; }
+                            S0[r][c] = 0;
+                        }
+            }
+#pragma unroll
+            for (int r = 0; r < TM; ++r)
+#pragma unroll
+                for (int c = 0; c < TN; ++c) cw[r][c] = uint32_t(S0[r][c]);
         }
         __syncthreads();                                   // the other buffer is complete, this one is free
         // ---- FP32 promotion of the partial sum every k_chunk elements ----
@@ -488,12 +527,11 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
             for (int r = 0; r < TM; ++r)
 #pragma unroll
                 for (int c = 0; c < TN; ++c) {
-                    const float part = __uint_as_float(acc_to_word<F, ACC16>(acc[r][c], MMASIM_SP_GET(r, c)));
+                    const float part = __uint_as_float(MMASIM_SP_WORD(r, c, cw[r][c]));
                     float v = __fadd_rn(promoted[PROMOTE ? r : 0][PROMOTE ? c : 0], part);
                     if (v != v) v = __uint_as_float(0x7FFFFFFFu);
                     promoted[PROMOTE ? r : 0][PROMOTE ? c : 0] = v;
-                    uint32_t dummy = 0u;
-                    acc[r][c] = acc_from_word<F, ACC16>(0u, dummy);
+                    cw[r][c] = 0u;
                 }
             sp_nan = sp_pinf = sp_ninf = 0u;
         }
@@ -506,8 +544,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
         for (int c = 0; c < TN; ++c) {
             const int64_t i = row0 + ty * TM + r, j = col0 + tx * TN + c;
             if (i >= g.M || j >= g.N) continue;
-            uint32_t w = PROMOTE ? __float_as_uint(promoted[PROMOTE ? r : 0][PROMOTE ? c : 0])
-                                 : acc_to_word<F, ACC16>(acc[r][c], MMASIM_SP_GET(r, c));
+            uint32_t w = PROMOTE ? __float_as_uint(promoted[PROMOTE ? r : 0][PROMOTE ? c : 0]) : MMASIM_SP_WORD(r, c, cw[r][c]);
             if (g.row_scale) {
                 float sc = __fmul_rn(g.row_scale[i], g.col_scale[j]);
                 if (sc != sc) sc = __uint_as_float(0x7FFFFFFFu);
@@ -519,7 +556,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_kernel(DevModel m, GemmArgs g) {
             else static_cast<uint32_t*>(g.D)[i * g.ldd + j] = w;
         }
 #undef MMASIM_SP_GET
-#undef MMASIM_SP_OR
+#undef MMASIM_SP_WORD
 }
 
 template <int EK, int L, int F, int RHO, bool PROMOTE>
