@@ -1,0 +1,411 @@
+// T-FDPA for E4M3 inputs with F = 13 (the Ada / Hopper FP8 rows on E4M3 operands; Algorithm 5 + 7 + Table 2): the FP32
+// summation kernel of mmasim_tfdpa_fast.cuh with the exponent maximum taken by the tensor cores.
+//
+// e_max = max_k (Exp(a_k) + Exp(b_k)) is a (max, +) product.  Powers turn it into an ordinary one: with
+// pe(x) = 2^(6 (Exp(x) - 1)) for a nonzero finite x and 0 otherwise,
+//     P = sum_k pe(a_k) * pe(b_k)  lies in  [2^(6 (e_max - 2)), 32 * 2^(6 (e_max - 2))]  (at most 32 terms, 32 < 2^6),
+// so floor(log2 P / 6) + 2 = e_max exactly, whatever the order, rounding or truncation of the summation (terms far
+// below the largest may be dropped, they do not matter).  E4M3 exponents span 15 values: 6 * (Exp - 1) stays within
+// +-42 and P within the FP32 range.  P for the 32 x 32 outputs of a warp and one block of 32 is sixteen
+// mma.sync.m16n8k16 on BF16 planes of pe values (a power of two is exact in BF16), instead of sixteen fused add-max
+// instructions per output; P = 0 (every product zero: no exponent) converts to an exponent below every real one.
+//
+// A warp owns 32 rows x 32 columns of the CTA tile (two by four accumulator fragments), and the micro-tile of a thread is
+// its share of those fragments: rows g, g + 8, g + 16, g + 24 (g = lane / 4) and columns 8 j + 2 t, 8 j + 2 t + 1
+// (t = lane % 4, j = 0..3), so that the maxima arrive in the registers of the thread that needs them.  The operand
+// planes are stored with rows and columns permuted accordingly (the four rows of a thread adjacent, its eight
+// columns contiguous): three 16-byte shared loads feed the 32 fused multiply-adds of one k.
+// Everything else - operands, sum register, sign correction, rho, rare cases - is the FP32 summation kernel.
+#pragma once
+#include "mmasim_tfdpa_fast.cuh"
+
+namespace mmasim {
+namespace trop {
+
+using fast::BM;
+using fast::BN;
+using fast::KC;
+using fast::NT;
+using fast::CB;
+using fast::FP_SHIFT;
+using fast::FP_EMAX_CLAMP;
+using fast::Elem;
+using fast::RawChunk;
+using fast::load_chunk;
+using fast::raw_elem;
+
+constexpr int PE_STRIDE = KC + 8;       // BF16 elements per row of a pe plane: 80 bytes, fragment loads hit 32 different banks
+constexpr int PE_CENTER = 1;            // pe(x) = 2^(6 (Exp(x) - PE_CENTER)); E4M3: Exp in [-6, 8]
+constexpr int TH = 4, TW = 8;           // micro-tile: 4 rows x 8 columns
+
+struct LutEntryT {
+    uint32_t op;        // staged FP32 operand (see mmasim_tfdpa_fast.cuh)
+    uint16_t pe;        // BF16 word of pe(x)
+    uint8_t bits;       // bit 0: sign, bit 1: finite and nonzero
+    uint8_t special;    // infinity / NaN
+};
+
+struct PlanesT {
+    uint32_t a_op[KC][BM];              // [k][permuted row]
+    uint32_t b_op[KC][BN];              // [k][permuted column]
+    uint16_t a_pe[BM][PE_STRIDE];       // [row][k]
+    uint16_t b_pe[BN][PE_STRIDE];       // [column][k]
+    uint32_t a_sgn[BM], a_nz[BM];       // [permuted row]: bit k = sign / nonzero of element k of the chunk
+    uint32_t b_sgn[BN], b_nz[BN];       // [permuted column]
+};
+
+struct SmemT {
+    PlanesT pl[2];
+    LutEntryT lut_a[256];
+    LutEntryT lut_b[256];
+    int special[3];
+};
+
+// Position of a row / column of the CTA tile inside the permuted planes.
+__device__ __forceinline__ int perm_row(int r) { return (r & ~31) | ((r & 7) << 2) | ((r >> 3) & 3); }
+__device__ __forceinline__ int perm_col(int c) { return (c & ~31) | (((c >> 1) & 3) << 3) | (((c >> 3) & 3) << 1) | (c & 1); }
+
+__device__ __forceinline__ void init_lut_t(SmemT& s, const FmtDesc& fa, const FmtDesc& fb, int pre, int guard, int tid) {
+    const uint32_t da = decode_elem(fa, uint32_t(tid)), db = decode_elem(fb, uint32_t(tid));
+    const bool fin_a = dec_cls(da) == CLS_FINITE, fin_b = dec_cls(db) == CLS_FINITE;
+    const bool nz_a = fin_a && dec_sig(da) != 0u, nz_b = fin_b && dec_sig(db) != 0u;
+    LutEntryT ea, eb;
+    ea.op = __float_as_uint(ldexpf(float(fin_a ? dec_ssig(da) : 0), fin_a ? dec_exp(da) : 0));
+    ea.pe = nz_a ? uint16_t((127 + 6 * (dec_exp(da) - PE_CENTER)) << 7) : uint16_t(0);
+    ea.bits = uint8_t(fin_a ? (dec_sign(da) | (uint32_t(nz_a) << 1)) : 0u);
+    ea.special = fin_a ? 0 : 1;
+    const int sb = fin_b ? dec_ssig(db) : 0;
+    const int ub = dec_sign(db) ? -1 : 1;
+    eb.op = nz_b ? __float_as_uint(ldexpf(float(sb * (1 << (pre + guard)) + ub), dec_exp(db) - FP_SHIFT)) : 0u;
+    eb.pe = nz_b ? uint16_t((127 + 6 * (dec_exp(db) - PE_CENTER)) << 7) : uint16_t(0);
+    eb.bits = uint8_t(fin_b ? (dec_sign(db) | (uint32_t(nz_b) << 1)) : 0u);
+    eb.special = fin_b ? 0 : 1;
+    s.lut_a[tid] = ea;
+    s.lut_b[tid] = eb;
+}
+
+template <int EK>
+__device__ __forceinline__ void store_chunk_t(SmemT& sm, PlanesT& s, const RawChunk<EK>& raw, int flag, int tid) {
+    using E = Elem<EK>;
+    using R = RawChunk<EK>;
+    static_assert(!E::SIGNMAG && E::TASK == 16, "table-decoded 8-bit elements, sixteen per task");
+    uint32_t spec = 0u;
+#pragma unroll
+    for (int it = 0; it < R::PER_THREAD; ++it) {
+        const int task = it * NT + tid;
+        if (task >= R::TASKS) break;
+        const bool is_a = task < BM * R::TPR;
+        const int u = is_a ? task : task - BM * R::TPR;
+        const int rows = is_a ? BM : BN;
+        const int r = u % rows, h = u / rows;
+        const int pr = is_a ? perm_row(r) : perm_col(r);
+        uint32_t sgn = 0u, nz = 0u, prev_pe = 0u;
+#pragma unroll
+        for (int q = 0; q < E::TASK; ++q) {
+            const int kk = h * E::TASK + q;
+            const uint32_t byte = (raw.w[it][q / 4] >> (8 * (q % 4))) & 0xFFu;
+            const LutEntryT e = is_a ? sm.lut_a[byte] : sm.lut_b[byte];
+            sgn |= uint32_t(e.bits & 1u) << q;
+            nz |= uint32_t((e.bits >> 1) & 1u) << q;
+            spec |= e.special;
+            if (is_a) s.a_op[kk][pr] = e.op; else s.b_op[kk][pr] = e.op;
+            if (q & 1) {
+                const uint32_t pair = prev_pe | (uint32_t(e.pe) << 16);
+                if (is_a) *reinterpret_cast<uint32_t*>(&s.a_pe[r][kk - 1]) = pair;
+                else *reinterpret_cast<uint32_t*>(&s.b_pe[r][kk - 1]) = pair;
+            }
+            prev_pe = e.pe;
+        }
+        if (is_a) {
+            reinterpret_cast<uint16_t*>(&s.a_sgn[pr])[h] = uint16_t(sgn);
+            reinterpret_cast<uint16_t*>(&s.a_nz[pr])[h] = uint16_t(nz);
+        } else {
+            reinterpret_cast<uint16_t*>(&s.b_sgn[pr])[h] = uint16_t(sgn);
+            reinterpret_cast<uint16_t*>(&s.b_nz[pr])[h] = uint16_t(nz);
+        }
+    }
+    if (spec) atomicOr(&sm.special[flag], 1);
+}
+
+template <int EK, int L, int F, int RHO, bool PROMOTE>
+__global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs g) {
+    constexpr bool ACC16 = RHO == RHO_RNE_FP16;
+    constexpr int NBLK = KC / L;
+    static_assert(KC % L == 0 && L % 16 == 0, "a block is one or two k16 matrix instructions");
+    static_assert(!Elem<EK>::SIGNMAG && F <= 13, "8-bit inputs with F <= 13");
+    static_assert(RHO == RHO_RZ_E8M13 || RHO == RHO_RNE_FP16, "rho of the F = 13 rows of Table 4");
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    SmemT& sm = *reinterpret_cast<SmemT*>(smem_raw);
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int gq = lane >> 2, tq = lane & 3;
+    const int64_t row0 = int64_t(blockIdx.y) * BM, col0 = int64_t(blockIdx.x) * BN;
+    const int wr = warp >> 1, wc = warp & 1;                                   // the warp's 32 x 32 part of the CTA tile
+    auto row_of = [&](int h) { return wr * 32 + gq + 8 * h; };                // inside the CTA tile
+    auto col_of = [&](int x) { return wc * 32 + 8 * (x >> 1) + 2 * tq + (x & 1); };
+    const FmtDesc fa = fmt_desc(m.fmt_a), fb = fmt_desc(m.fmt_b);
+    const int pre = F - (fa.mbits + fb.mbits);
+    const int guard = fa.mbits + 1;
+    const float c_scale = __int_as_float((127 + F + guard - FP_SHIFT) << 23);
+    // Below E_LOW no product is nonzero (a nonzero E4M3 product has an exponent of at least -12; P = 0 converts to
+    // -20), above E_HIGH only a huge accumulator: the result is rho of the accumulator alone (see the FP32 kernel).
+    constexpr int E_LOW = CB - 16, E_HIGH = CB + FP_EMAX_CLAMP;
+    // exponent of P -> e_max + CB: ((field - 43) * 171 >> 10) - 14 + 2 * PE_CENTER + CB, field - 43 = 6 (e_max - 2 PE_CENTER + 14) + 0..5
+    constexpr int CONV_K = -43 * 171 + (CB - 14 + 2 * PE_CENTER) * 1024;
+
+    if (tid < 256) init_lut_t(sm, fa, fb, pre, guard, tid);
+    if (tid == 0) sm.special[0] = sm.special[1] = sm.special[2] = 0;
+
+    uint32_t cw[TH][TW];
+    uint32_t sp_nan = 0u, sp_pinf = 0u, sp_ninf = 0u;   // per output (bit h * TW + x)
+    float promoted[PROMOTE ? TH : 1][PROMOTE ? TW : 1];
+#define MMASIM_SP_GET(h, x) ((((sp_nan >> ((h) * TW + (x))) & 1u)) | (((sp_pinf >> ((h) * TW + (x))) & 1u) << 1) | (((sp_ninf >> ((h) * TW + (x))) & 1u) << 2))
+#define MMASIM_SP_WORD(h, x, w) (MMASIM_SP_GET(h, x) ? special_word(((MMASIM_SP_GET(h, x) & 1u) || (MMASIM_SP_GET(h, x) & 6u) == 6u) ? 1 : ((MMASIM_SP_GET(h, x) & 2u) ? 2 : 3), ACC16, true) : (w))
+#pragma unroll
+    for (int h = 0; h < TH; ++h)
+#pragma unroll
+        for (int x = 0; x < TW; ++x) {
+            const int64_t i = row0 + row_of(h), j = col0 + col_of(x);
+            uint32_t w = 0u;
+            if (g.C && i < g.M && j < g.N)
+                w = ACC16 ? uint32_t(static_cast<const uint16_t*>(g.C)[i * g.ldc + j])
+                          : static_cast<const uint32_t*>(g.C)[i * g.ldc + j];
+            if (PROMOTE) { promoted[PROMOTE ? h : 0][PROMOTE ? x : 0] = __uint_as_float(w); w = 0u; }
+            const AccDec d = decode_acc(w, ACC16);
+            if (d.cls != CLS_FINITE) {
+                const uint32_t bit = 1u << (h * TW + x);
+                if (d.cls == CLS_NAN) sp_nan |= bit; else if (d.sign) sp_ninf |= bit; else sp_pinf |= bit;
+                w = 0u;
+            }
+            cw[h][x] = w;
+        }
+
+    RawChunk<EK> raw;
+    load_chunk<EK>(raw, g, row0, col0, 0, tid);
+    __syncthreads();                                       // tables and flags are ready
+    store_chunk_t<EK>(sm, sm.pl[0], raw, 0, tid);
+    if (KC < g.K) load_chunk<EK>(raw, g, row0, col0, KC, tid);
+    __syncthreads();
+    int chunk = 0;
+    for (int64_t k0 = 0; k0 < g.K; k0 += KC, ++chunk) {
+        if (tid == 0) sm.special[(chunk + 2) % 3] = 0;
+        if (k0 + KC < g.K) {
+            store_chunk_t<EK>(sm, sm.pl[(chunk + 1) & 1], raw, (chunk + 1) % 3, tid);
+            if (k0 + 2 * KC < g.K) load_chunk<EK>(raw, g, row0, col0, k0 + 2 * KC, tid);
+        }
+        PlanesT& s = sm.pl[chunk & 1];
+        const bool chunk_special = sm.special[chunk % 3] != 0;
+
+#pragma unroll 1
+        for (int blk = 0; blk < NBLK; ++blk) {
+            const int kb = blk * L;
+            if (chunk_special) {                           // rare: special-value events of this block (Section 4.2)
+#pragma unroll 1
+                for (int h = 0; h < TH; ++h)
+#pragma unroll 1
+                    for (int x = 0; x < TW; ++x) {
+                        const int64_t i = row0 + row_of(h), j = col0 + col_of(x);
+                        if (i >= g.M || j >= g.N) continue;
+                        Special ev;
+                        for (int kk = kb; kk < kb + L; ++kk) {
+                            const uint32_t xa = decode_elem(fa, raw_elem<EK>(g.A, i * g.lda + k0 + kk));
+                            const uint32_t yb = decode_elem(fb, raw_elem<EK>(g.B, j * g.ldb + k0 + kk));
+                            ev.product(xa, yb);
+                        }
+                        const uint32_t bit = 1u << (h * TW + x);
+                        if (ev.nan) sp_nan |= bit;
+                        if (ev.pinf) sp_pinf |= bit;
+                        if (ev.ninf) sp_ninf |= bit;
+                    }
+            }
+
+            int S0[TH][TW];         // first e_max + CB, then the sum register, then the result word
+            int elo = E_HIGH, ehi = E_LOW;
+            // ---- pass 1 on the tensor cores: P = sum_k pe(a_k) pe(b_k) for the warp's 32 x 32 outputs ----
+            {
+                float P[2][4][4];
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) { P[mt][j][0] = 0.f; P[mt][j][1] = 0.f; P[mt][j][2] = 0.f; P[mt][j][3] = 0.f; }
+#pragma unroll
+                for (int ks = 0; ks < L / 16; ++ks) {
+                    const int kq = kb + 16 * ks + 2 * tq;
+                    uint32_t bf[4][2];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        bf[j][0] = *reinterpret_cast<const uint32_t*>(&s.b_pe[wc * 32 + 8 * j + gq][kq]);
+                        bf[j][1] = *reinterpret_cast<const uint32_t*>(&s.b_pe[wc * 32 + 8 * j + gq][kq + 8]);
+                    }
+#pragma unroll
+                    for (int mt = 0; mt < 2; ++mt) {
+                        const int ar = wr * 32 + 16 * mt + gq;
+                        const uint32_t a0 = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar][kq]);
+                        const uint32_t a1 = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar + 8][kq]);
+                        const uint32_t a2 = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar][kq + 8]);
+                        const uint32_t a3 = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar + 8][kq + 8]);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                         : "+f"(P[mt][j][0]), "+f"(P[mt][j][1]), "+f"(P[mt][j][2]), "+f"(P[mt][j][3])
+                                         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bf[j][0]), "r"(bf[j][1]));
+                    }
+                }
+                // exponent field of P -> e_max + CB; then the accumulator's exponent (none for c = 0)
+#pragma unroll
+                for (int h = 0; h < TH; ++h)
+#pragma unroll
+                    for (int x = 0; x < TW; ++x) {
+                        const int field = __float_as_int(P[h >> 1][x >> 1][2 * (h & 1) + (x & 1)]) >> 23;
+                        const int ep = (field * 171 + CONV_K) >> 10;
+                        const uint32_t ca = cw[h][x] & (ACC16 ? 0x7FFFu : 0x7FFFFFFFu);
+                        const int rel = ca ? int(max(ca >> (ACC16 ? 10 : 23), 1u)) + (CB - (ACC16 ? 15 : 127)) : 0;
+                        const int e = max(ep, rel);
+                        elo = min(elo, e);
+                        ehi = max(ehi, e);
+                        S0[h][x] = e;
+                    }
+            }
+            uint32_t keep = 0u;                            // outputs whose products cannot reach the result (rare)
+            if (elo < E_LOW || ehi > E_HIGH) {
+#pragma unroll
+                for (int h = 0; h < TH; ++h)
+#pragma unroll
+                    for (int x = 0; x < TW; ++x)
+                        if (S0[h][x] < E_LOW || S0[h][x] > E_HIGH) keep |= 1u << (h * TW + x);
+            }
+            // ---- the sum register (1.5 * 2^23 + S) * u with the accumulator term (see the FP32 kernel) ----
+#pragma unroll
+            for (int h = 0; h < TH; ++h)
+#pragma unroll
+                for (int x = 0; x < TW; ++x) {
+                    const int ecl = max(min(S0[h][x], E_HIGH), E_LOW) + guard;
+                    const float magic = __int_as_float(((ecl + (150 - CB - FP_SHIFT)) << 23) | 0x00400000);
+                    const float cf = ACC16 ? __half2float(__ushort_as_half((unsigned short)cw[h][x])) : __uint_as_float(cw[h][x]);
+                    S0[h][x] = __float_as_int(__fmaf_rd(__int_as_float(__float_as_int(cf) | 1), c_scale, magic));
+                }
+            // ---- pass 2: one fused multiply-add per term, rounding toward minus infinity onto the grid of S ----
+#pragma unroll 4
+            for (int kk = kb; kk < kb + L; ++kk) {
+                const float4 oa = *reinterpret_cast<const float4*>(&s.a_op[kk][wr * 32 + 4 * gq]);
+                const float4 ob0 = *reinterpret_cast<const float4*>(&s.b_op[kk][wc * 32 + 8 * tq]);
+                const float4 ob1 = *reinterpret_cast<const float4*>(&s.b_op[kk][wc * 32 + 8 * tq + 4]);
+                const float oav[TH] = {oa.x, oa.y, oa.z, oa.w};
+                const float obv[TW] = {ob0.x, ob0.y, ob0.z, ob0.w, ob1.x, ob1.y, ob1.z, ob1.w};
+#pragma unroll
+                for (int h = 0; h < TH; ++h)
+#pragma unroll
+                    for (int x = 0; x < TW; ++x)
+                        S0[h][x] = __float_as_int(__fmaf_rd(oav[h], obv[x], __int_as_float(S0[h][x])));
+            }
+            // ---- sign corrections and rho ----
+            const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
+            uint32_t wmax = 0u;
+            uint32_t sbv[TW], nzb[TW];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const uint4 u = *reinterpret_cast<const uint4*>(&s.b_sgn[wc * 32 + 8 * tq + 4 * q]);
+                const uint4 v = *reinterpret_cast<const uint4*>(&s.b_nz[wc * 32 + 8 * tq + 4 * q]);
+                sbv[4 * q] = u.x; sbv[4 * q + 1] = u.y; sbv[4 * q + 2] = u.z; sbv[4 * q + 3] = u.w;
+                nzb[4 * q] = v.x; nzb[4 * q + 1] = v.y; nzb[4 * q + 2] = v.z; nzb[4 * q + 3] = v.w;
+            }
+#pragma unroll
+            for (int h = 0; h < TH; ++h) {
+                const uint32_t sa = s.a_sgn[wr * 32 + 4 * gq + h];
+                const uint32_t nza = s.a_nz[wr * 32 + 4 * gq + h] & kmask;
+#pragma unroll
+                for (int x = 0; x < TW; ++x) {
+                    const int nneg = __popc((sa ^ sbv[x]) & nza & nzb[x]);
+                    const int bits = S0[h][x];
+                    const int fld = bits & 0x7F800000;
+                    const int S = bits - (fld | 0x00400000) + nneg + int(cw[h][x] >> (ACC16 ? 15 : 31));
+                    const float scale = __int_as_float(fld - ((15 + F + guard) << 23));       // 2^(e_max - F)
+                    const float v = __fmul_rn(__int2float_rn(S), scale);
+                    uint32_t w;
+                    if (ACC16) { w = uint32_t(__half_as_ushort(__float2half_rn(v))); wmax = max(wmax, w & 0x7FFFu); }
+                    else w = __float_as_uint(v) & 0xFFFFFC00u;
+                    S0[h][x] = int(w);
+                }
+            }
+            if (keep) {                                    // rare: rho of the accumulator alone; an exactly zero sum is +0
+#pragma unroll
+                for (int h = 0; h < TH; ++h)
+#pragma unroll
+                    for (int x = 0; x < TW; ++x)
+                        if ((keep >> (h * TW + x)) & 1u) {
+                            const uint32_t t = ACC16 ? cw[h][x] : (cw[h][x] & 0xFFFFFC00u);
+                            S0[h][x] = int((t & (ACC16 ? 0x7FFFu : 0x7FFFFFFFu)) ? t : 0u);
+                        }
+            }
+            if (ACC16 && wmax >= 0x7C00u) {                // rare: RNE-FP16 overflowed: +-infinity from now on
+#pragma unroll
+                for (int h = 0; h < TH; ++h)
+#pragma unroll
+                    for (int x = 0; x < TW; ++x)
+                        if ((uint32_t(S0[h][x]) & 0x7FFFu) == 0x7C00u) {
+                            const uint32_t bit = 1u << (h * TW + x);
+                            if (!((sp_nan | sp_pinf | sp_ninf) & bit)) { if (uint32_t(S0[h][x]) >> 15) sp_ninf |= bit; else sp_pinf |= bit; }
+                            S0[h][x] = 0;
+                        }
+            }
+#pragma unroll
+            for (int h = 0; h < TH; ++h)
+#pragma unroll
+                for (int x = 0; x < TW; ++x) cw[h][x] = uint32_t(S0[h][x]);
+        }
+        __syncthreads();                                   // the other buffer is complete, this one is free
+        if (PROMOTE && ((k0 + KC) % g.k_chunk) == 0) {     // FP32 promotion of the partial sum every k_chunk elements
+#pragma unroll
+            for (int h = 0; h < TH; ++h)
+#pragma unroll
+                for (int x = 0; x < TW; ++x) {
+                    const float part = __uint_as_float(MMASIM_SP_WORD(h, x, cw[h][x]));
+                    float v = __fadd_rn(promoted[PROMOTE ? h : 0][PROMOTE ? x : 0], part);
+                    if (v != v) v = __uint_as_float(0x7FFFFFFFu);
+                    promoted[PROMOTE ? h : 0][PROMOTE ? x : 0] = v;
+                    cw[h][x] = 0u;
+                }
+            sp_nan = sp_pinf = sp_ninf = 0u;
+        }
+    }
+
+#pragma unroll
+    for (int h = 0; h < TH; ++h)
+#pragma unroll
+        for (int x = 0; x < TW; ++x) {
+            const int64_t i = row0 + row_of(h), j = col0 + col_of(x);
+            if (i >= g.M || j >= g.N) continue;
+            uint32_t w = PROMOTE ? __float_as_uint(promoted[PROMOTE ? h : 0][PROMOTE ? x : 0]) : MMASIM_SP_WORD(h, x, cw[h][x]);
+            if (g.row_scale) {
+                float sc = __fmul_rn(g.row_scale[i], g.col_scale[j]);
+                if (sc != sc) sc = __uint_as_float(0x7FFFFFFFu);
+                float v = __fmul_rn(sc, __uint_as_float(w));
+                if (v != v) v = __uint_as_float(0x7FFFFFFFu);
+                w = __float_as_uint(v);
+            }
+            if (ACC16) static_cast<uint16_t*>(g.D)[i * g.ldd + j] = uint16_t(w);
+            else static_cast<uint32_t*>(g.D)[i * g.ldd + j] = w;
+        }
+#undef MMASIM_SP_GET
+#undef MMASIM_SP_WORD
+}
+
+template <int EK, int L, int F, int RHO, bool PROMOTE>
+cudaError_t launch_one_t(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
+    const size_t sh = sizeof(SmemT);
+    cudaError_t err = cudaFuncSetAttribute(tfdpa_trop_kernel<EK, L, F, RHO, PROMOTE>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
+    if (err != cudaSuccess) return err;
+    dim3 grid((unsigned)((g.N + BN - 1) / BN), (unsigned)((g.M + BM - 1) / BM), 1);
+    tfdpa_trop_kernel<EK, L, F, RHO, PROMOTE><<<grid, NT, sh, stream>>>(m, g);
+    return cudaGetLastError();
+}
+
+template <int EK, int L, int F, int RHO>
+cudaError_t launch_variant_t(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
+    if (RHO != RHO_RNE_FP16 && g.k_chunk) return launch_one_t<EK, L, F, RHO, RHO != RHO_RNE_FP16>(m, g, stream);
+    return launch_one_t<EK, L, F, RHO, false>(m, g, stream);
+}
+
+}  // namespace trop
+}  // namespace mmasim
