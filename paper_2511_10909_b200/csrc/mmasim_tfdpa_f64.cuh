@@ -79,7 +79,7 @@ __device__ __forceinline__ void load_chunk(RawChunk<EK>& raw, const GemmArgs& g,
     }
 }
 
-constexpr int G_OFF = 30;          // the B offset sits 30 bits below the element's last significand bit
+constexpr int G_OFF = 30;          // the B offset sits 30 bits below the element's last significand bit (bit 22 - mbits of a double's low word)
 
 struct LutEntry64 {
     double op;          // staged operand
@@ -164,13 +164,31 @@ __device__ __forceinline__ void store_chunk64(SM& sm, PL& s, const RawChunk<EK>&
                 spec |= e.bits & 2u;
             } else {
                 const uint32_t w = E::BYTES == 2 ? ((raw.w[it][q / 2] >> (16 * (q % 2))) & 0xFFFFu) : raw.w[it][q];
-                uint32_t sig, sign, special;
-                fast::decode_signmag<EK>(w, sig, expb, sign, special);
-                const int exp = int(expb) - EB;
-                op = is_a ? operand_a(sign, sig, exp, E::MBITS) : operand_b(sign, sig, exp, E::MBITS);
-                if (!sig) expb = 0u;                                        // no exponent: never the maximum
-                bits += (sign | (uint32_t(sig != 0u) << 16)) << q;
-                spec |= special;
+                // A normal number becomes a double by moving its exponent and mantissa fields into place and rebiasing
+                // (no arithmetic); the offset of a B operand is then bit 22 - mbits of the low word.  Subnormals take
+                // the arithmetic route; zeros, infinities and NaNs are staged as zero without exponent.
+                constexpr uint32_t TOP = (1u << E::EBITS) - 1u;
+                const uint32_t xx = w >> E::LOW;
+                const uint32_t mag = xx & ((1u << (E::EBITS + E::MBITS)) - 1u);
+                const uint32_t field = mag >> E::MBITS;
+                const uint32_t sign = (xx >> (E::EBITS + E::MBITS)) & 1u;
+                uint32_t hi = 0u, lo = 0u, nzbit = 1u;
+                expb = 0u;
+                if (field - 1u < TOP - 1u) {
+                    hi = (mag << (20 - E::MBITS)) + (uint32_t(1023 - E::BIAS) << 20);
+                    lo = is_a ? 0u : (1u << (22 - E::MBITS));
+                    expb = field + uint32_t(EB - E::BIAS);
+                } else if (field == 0u && mag != 0u) {
+                    const double v = is_a ? operand_a(0u, mag, 1 - E::BIAS, E::MBITS) : operand_b(0u, mag, 1 - E::BIAS, E::MBITS);
+                    hi = uint32_t(__double2hiint(v));
+                    lo = uint32_t(__double2loint(v));
+                    expb = uint32_t(1 - E::BIAS + EB);
+                } else {
+                    nzbit = 0u;
+                    spec |= uint32_t(field == TOP);
+                }
+                op = __hiloint2double(int(hi | (sign << 31)), int(lo));
+                bits += (sign | (nzbit << 16)) << q;
             }
             if (is_a) s.a_d[kk][r] = op; else s.b_d[kk][r] = op;
             if (q & 1) {

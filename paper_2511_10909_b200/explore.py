@@ -1,0 +1,88 @@
+"""Workaround and design-space exploration (Sections 6.3 and 7) on top of the library's entry points.
+
+Three experiments, all at GEMM scale on the GPU, each returning the deviation statistics of `accuracy.deviation_stats`
+against the FP64 real result:
+
+* `design_sweep`    - hypothetical T-FDPA units: the registry row of a model with other (L_max, F, rho), made by
+                      `mmasim_create_model_ex` overrides, to see which parameter buys how much accuracy;
+* `chunk_sweep`     - the FP32-promotion workaround for low-precision accumulation with chunk sizes other than 128;
+* `fp8_via_fp16`    - the workaround that feeds FP8 data to the FP16 instruction (every E4M3 / E5M2 value is an FP16
+                      value): the same architecture's FP16 row evaluated on the widened words.
+
+torch widens FP8 words to FP16 words; every arithmetic step of a model runs in the library's kernels.
+"""
+from __future__ import annotations
+
+from . import accuracy, mmasim
+
+
+def design_sweep(arch: str, in_fmt: str, acc: str, A, B, C=None, l_max=(None,), F=(None,), rho=(None,), ref=None):
+    """Deviation statistics of the (arch, in_fmt, acc) row and of its variants with every combination of the given
+    L_max, F and rho (None = the table's value).  Returns a list of dicts with the parameters actually used."""
+    if ref is None:
+        ref = accuracy.reference_fp64(in_fmt, acc, A, B, C)
+    out = []
+    for L in l_max:
+        for f in F:
+            for r in rho:
+                ov = {}
+                if L is not None:
+                    ov["l_max"] = L
+                if f is not None:
+                    ov["F"] = f
+                if r is not None:
+                    ov["rho"] = r
+                m = mmasim.Model(arch, in_fmt, acc, **ov)
+                s = accuracy.deviation_stats(m, A, B, C, ref)
+                s.update(l_max=m.l_max, F=m.F, rho=m.rho, kernel=mmasim.last_kernel())
+                out.append(s)
+    return out
+
+
+def chunk_sweep(model: mmasim.Model, A, B, chunks=(0, 32, 64, 128, 256, 512), row_scale=None, col_scale=None, ref=None):
+    """Deviation statistics of the model with FP32 promotion every `k_chunk` elements of K (0 = no promotion: the
+    hardware accumulator runs over all of K).  C = +0, as in the workaround; the per-row and per-column scales are
+    given together or not at all and enter the real result too."""
+    if ref is None:
+        ref = accuracy.reference_fp64(model.in_fmt, model.acc, A, B, None)
+        if row_scale is not None:
+            ref = ref * row_scale.double()[:, None]
+        if col_scale is not None:
+            ref = ref * col_scale.double()[None, :]
+    out = []
+    for kc in chunks:
+        kw = dict(k_chunk=kc)
+        if row_scale is not None:
+            kw.update(row_scale=row_scale, col_scale=col_scale)
+        D = mmasim.gemm(model, A, B, None, **kw)
+        s = _stats(model.acc, D, ref)
+        s.update(k_chunk=kc, kernel=mmasim.last_kernel())
+        out.append(s)
+    return out
+
+
+def widen_fp8_to_fp16(fmt: str, words):
+    """E4M3 / E5M2 bytes -> the FP16 words of the same values (exact: both formats are subsets of FP16)."""
+    import torch
+    t = {"e4m3": torch.float8_e4m3fn, "e5m2": torch.float8_e5m2}[fmt]
+    return words.view(t).to(torch.float16).view(torch.int16)
+
+
+def fp8_via_fp16(arch: str, fmt: str, A, B, C=None, acc: str = "fp32", ref=None):
+    """The FP8 row of `arch` against the same architecture's FP16 row fed with the widened FP8 data."""
+    if ref is None:
+        ref = accuracy.reference_fp64(fmt, acc, A, B, C)
+    native = mmasim.Model(arch, fmt, acc)
+    via = mmasim.Model(arch, "fp16", acc)
+    s8 = accuracy.deviation_stats(native, A, B, C, ref)
+    s8.update(model=repr(native))
+    s16 = accuracy.deviation_stats(via, widen_fp8_to_fp16(fmt, A), widen_fp8_to_fp16(fmt, B), C, ref)
+    s16.update(model=repr(via))
+    return {"native": s8, "via_fp16": s16}
+
+
+def _stats(acc: str, D, ref) -> dict:
+    s = mmasim.error_stats(acc, D, ref).cpu().tolist()
+    n = max(s[0], 1.0)
+    return {"count": int(s[0]), "mean": s[1] / n, "mean_abs": s[2] / n, "rms": (s[3] / n) ** 0.5, "negative": s[4] / n,
+            "positive": s[5] / n, "max_abs": s[6], "mean_rel": s[7] / n}
