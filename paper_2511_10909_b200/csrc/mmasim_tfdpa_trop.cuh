@@ -2,21 +2,28 @@
 // summation kernel of mmasim_tfdpa_fast.cuh with the exponent maximum taken by the tensor cores.
 //
 // e_max = max_k (Exp(a_k) + Exp(b_k)) is a (max, +) product.  Powers turn it into an ordinary one: with
-// pe(x) = 2^(6 (Exp(x) - 1)) for a nonzero finite x and 0 otherwise,
-//     P = sum_k pe(a_k) * pe(b_k)  lies in  [2^(6 (e_max - 2)), 32 * 2^(6 (e_max - 2))]  (at most 32 terms, 32 < 2^6),
-// so floor(log2 P / 6) + 2 = e_max exactly, whatever the order, rounding or truncation of the summation (terms far
-// below the largest may be dropped, they do not matter).  E4M3 exponents span 15 values: 6 * (Exp - 1) stays within
-// +-42 and P within the FP32 range.  P for the 32 x 32 outputs of a warp and one block of 32 is sixteen
-// mma.sync.m16n8k16 on BF16 planes of pe values (a power of two is exact in BF16), instead of sixteen fused add-max
-// instructions per output; P = 0 (every product zero: no exponent) converts to an exponent below every real one.
+// pe(x) = 2^(6 (Exp(x) - 1)) for a nonzero finite x and 0 otherwise (the B plane scaled by 2^5 more),
+//     P = sum_k pe(a_k) * pe(b_k)  lies in  2^(6 (e_max + 20) - 127) * [1, 32]  (at most 32 terms, 32 < 2^6),
+// so its FP32 exponent field is 6 (e_max + 20) + 0..5 and floor(field / 6) - 20 = e_max exactly, whatever the order,
+// rounding or truncation of the summation (terms far below the largest may be dropped, they do not matter).  E4M3
+// exponents span 15 values: 6 * (Exp - 1) stays within +-42 and P within the FP32 range.  P for the 32 x 32 outputs
+// of a warp and one block of 32 is sixteen mma.sync.m16n8k16 on BF16 planes of pe values (a power of two is exact in
+// BF16), instead of sixteen fused add-max instructions per output; P = 0 (every product zero: no exponent) converts
+// to an exponent below every real one.  The division by 6 is one high multiply on the bits of P, which leaves the
+// result as an FP32 exponent field in place, comparable with the bits of |c| and a mask away from the sum register's
+// starting value.
 //
 // A warp owns 32 rows x 32 columns of the CTA tile (two by four accumulator fragments), and the micro-tile of a thread is
 // its share of those fragments: rows g, g + 8, g + 16, g + 24 (g = lane / 4) and columns 8 j + 2 t, 8 j + 2 t + 1
 // (t = lane % 4, j = 0..3), so that the maxima arrive in the registers of the thread that needs them.  The operand
 // planes are stored with rows and columns permuted accordingly (the four rows of a thread adjacent, its eight
 // columns contiguous): three 16-byte shared loads feed the 32 fused multiply-adds of one k.
-// Everything else - operands, sum register, sign correction, rho, rare cases - is the FP32 summation kernel.
+// The sum register works as in the FP32 summation kernel, here in the true scale: operands are the element values (B
+// with the small offset that makes negative products inexact), the register is (1.5 * 2^23 + S) * 2^(e_max - F), the
+// accumulator enters by one addition rounded toward minus infinity and the block's value S * 2^(e_max - F) leaves by
+// one exact subtraction; rho is a mask (RZ-E8M13) or a conversion (RNE-FP16).
 #pragma once
+#include <type_traits>
 #include "mmasim_tfdpa_fast.cuh"
 
 namespace mmasim {
@@ -27,8 +34,6 @@ using fast::BN;
 using fast::KC;
 using fast::NT;
 using fast::CB;
-using fast::FP_SHIFT;
-using fast::FP_EMAX_CLAMP;
 using fast::Elem;
 using fast::RawChunk;
 using fast::load_chunk;
@@ -36,6 +41,7 @@ using fast::raw_elem;
 
 constexpr int PE_STRIDE = KC + 8;       // BF16 elements per row of a pe plane: 80 bytes, fragment loads hit 32 different banks
 constexpr int PE_CENTER = 1;            // pe(x) = 2^(6 (Exp(x) - PE_CENTER)); E4M3: Exp in [-6, 8]
+constexpr int PE_B_SHIFT = 5;           // pe(b) carries 2^5 more, so that the exponent field of P is 6 (e_max + 20) + 0..5
 constexpr int TH = 4, TW = 8;           // micro-tile: 4 rows x 8 columns
 
 struct LutEntryT {
@@ -76,8 +82,9 @@ __device__ __forceinline__ void init_lut_t(SmemT& s, const FmtDesc& fa, const Fm
     ea.special = fin_a ? 0 : 1;
     const int sb = fin_b ? dec_ssig(db) : 0;
     const int ub = dec_sign(db) ? -1 : 1;
-    eb.op = nz_b ? __float_as_uint(ldexpf(float(sb * (1 << (pre + guard)) + ub), dec_exp(db) - FP_SHIFT)) : 0u;
-    eb.pe = nz_b ? uint16_t((127 + 6 * (dec_exp(db) - PE_CENTER)) << 7) : uint16_t(0);
+    // a_op * b_op = a * b * (1 + 2^-(pre + guard) / |sig_b|): the true product with the offset that makes a negative one inexact
+    eb.op = nz_b ? __float_as_uint(ldexpf(float(sb * (1 << (pre + guard)) + ub), dec_exp(db) - (fa.mbits + fb.mbits + pre + guard))) : 0u;
+    eb.pe = nz_b ? uint16_t((127 + PE_B_SHIFT + 6 * (dec_exp(db) - PE_CENTER)) << 7) : uint16_t(0);
     eb.bits = uint8_t(fin_b ? (dec_sign(db) | (uint32_t(nz_b) << 1)) : 0u);
     eb.special = fin_b ? 0 : 1;
     s.lut_a[tid] = ea;
@@ -147,13 +154,22 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
     const FmtDesc fa = fmt_desc(m.fmt_a), fb = fmt_desc(m.fmt_b);
     const int pre = F - (fa.mbits + fb.mbits);
     const int guard = fa.mbits + 1;
-    const float c_scale = __int_as_float((127 + F + guard - FP_SHIFT) << 23);
-    // Below E_LOW no product is nonzero (a nonzero E4M3 product has an exponent of at least -12; P = 0 converts to
-    // -20), above E_HIGH only a huge accumulator: the result is rho of the accumulator alone (see the FP32 kernel).
-    constexpr int E_LOW = CB - 16, E_HIGH = CB + FP_EMAX_CLAMP;
-    // exponent of P -> e_max + CB: ((field - 43) * 171 >> 10) - 14 + 2 * PE_CENTER + CB, field - 43 = 6 (e_max - 2 PE_CENTER + 14) + 0..5
-    constexpr int CONV_K = -43 * 171 + (CB - 14 + 2 * PE_CENTER) * 1024;
-
+    // Exponents are handled as FP32 exponent fields in place (bits 23..30) with whatever lies below as a fraction:
+    //   t1 = floor(bits(P) / 6) + (107 << 23): field e_max + 127 for the largest product (P = 0: field 107, e_max = -20,
+    //        below the smallest nonzero E4M3 product, 2^-12); dividing by 6 is a high multiply, inexact by 2^-31 and P is
+    //        never closer than 1/6 to the next multiple;
+    //   ca = |c|: field Exp(c) + 127.
+    // Sum register: (1.5 * 2^23 + S) * 2^(e_max - F), exponent field e + (23 - F).
+    constexpr uint32_t MUL6 = 0x2AAAAAABu, T1_ADD = 107u << 23;
+    constexpr uint32_t FIELD = 0x7F800000u, HALF = 0x00400000u;
+    constexpr uint32_t MAGIC_ADD = (uint32_t(23 - F) << 23) | HALF;
+    // Below E_LOW no product is nonzero, above E_HIGH the register would overflow (and every product is far below one
+    // unit of the accumulator): the result is rho of the accumulator alone.  Such an output rides through pass 2 as a
+    // marker KEEP + payload whose unit exceeds every product, so that a term changes it by -1 or not at all, which the
+    // sign correction undoes.  FP16 accumulators are never out of range.
+    constexpr uint32_t E_LOW = ACC16 ? 0u : (115u << 23), E_HIGH = (241u << 23) - 1u;
+    constexpr uint32_t E_KEEP = 243u << 23, KEEP = E_KEEP + MAGIC_ADD;
+    static_assert(F == 13 || ACC16, "the kept word is carried as its upper 22 bits");
     if (tid < 256) init_lut_t(sm, fa, fb, pre, guard, tid);
     if (tid == 0) sm.special[0] = sm.special[1] = sm.special[2] = 0;
 
@@ -220,73 +236,83 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
                     }
             }
 
-            int S0[TH][TW];         // first e_max + CB, then the sum register, then the result word
-            int elo = E_HIGH, ehi = E_LOW;
             // ---- pass 1 on the tensor cores: P = sum_k pe(a_k) pe(b_k) for the warp's 32 x 32 outputs ----
-            {
-                float P[2][4][4];
+            float P[2][4][4];
 #pragma unroll
-                for (int mt = 0; mt < 2; ++mt)
+            for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) { P[mt][j][0] = 0.f; P[mt][j][1] = 0.f; P[mt][j][2] = 0.f; P[mt][j][3] = 0.f; }
+                for (int j = 0; j < 4; ++j) { P[mt][j][0] = 0.f; P[mt][j][1] = 0.f; P[mt][j][2] = 0.f; P[mt][j][3] = 0.f; }
 #pragma unroll
-                for (int ks = 0; ks < L / 16; ++ks) {
-                    const int kq = kb + 16 * ks + 2 * tq;
-                    uint32_t bf[4][2];
+            for (int ks = 0; ks < L / 16; ++ks) {
+                const int kq = kb + 16 * ks + 2 * tq;
+                uint32_t bf[4][2];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        bf[j][0] = *reinterpret_cast<const uint32_t*>(&s.b_pe[wc * 32 + 8 * j + gq][kq]);
-                        bf[j][1] = *reinterpret_cast<const uint32_t*>(&s.b_pe[wc * 32 + 8 * j + gq][kq + 8]);
-                    }
-#pragma unroll
-                    for (int mt = 0; mt < 2; ++mt) {
-                        const int ar = wr * 32 + 16 * mt + gq;
-                        const uint32_t a0 = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar][kq]);
-                        const uint32_t a1 = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar + 8][kq]);
-                        const uint32_t a2 = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar][kq + 8]);
-                        const uint32_t a3 = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar + 8][kq + 8]);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j)
-                            asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                                         : "+f"(P[mt][j][0]), "+f"(P[mt][j][1]), "+f"(P[mt][j][2]), "+f"(P[mt][j][3])
-                                         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bf[j][0]), "r"(bf[j][1]));
-                    }
+                for (int j = 0; j < 4; ++j) {
+                    bf[j][0] = *reinterpret_cast<const uint32_t*>(&s.b_pe[wc * 32 + 8 * j + gq][kq]);
+                    bf[j][1] = *reinterpret_cast<const uint32_t*>(&s.b_pe[wc * 32 + 8 * j + gq][kq + 8]);
                 }
-                // exponent field of P -> e_max + CB; then the accumulator's exponent (none for c = 0)
 #pragma unroll
-                for (int h = 0; h < TH; ++h)
+                for (int mt = 0; mt < 2; ++mt) {
+                    const int ar = wr * 32 + 16 * mt + gq;
+                    const uint32_t a0 = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar][kq]);
+                    const uint32_t a1 = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar + 8][kq]);
+                    const uint32_t a2 = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar][kq + 8]);
+                    const uint32_t a3 = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar + 8][kq + 8]);
 #pragma unroll
-                    for (int x = 0; x < TW; ++x) {
-                        const int field = __float_as_int(P[h >> 1][x >> 1][2 * (h & 1) + (x & 1)]) >> 23;
-                        const int ep = (field * 171 + CONV_K) >> 10;
-                        const uint32_t ca = cw[h][x] & (ACC16 ? 0x7FFFu : 0x7FFFFFFFu);
-                        const int rel = ca ? int(max(ca >> (ACC16 ? 10 : 23), 1u)) + (CB - (ACC16 ? 15 : 127)) : 0;
-                        const int e = max(ep, rel);
-                        elo = min(elo, e);
-                        ehi = max(ehi, e);
-                        S0[h][x] = e;
-                    }
+                    for (int j = 0; j < 4; ++j)
+                        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                     : "+f"(P[mt][j][0]), "+f"(P[mt][j][1]), "+f"(P[mt][j][2]), "+f"(P[mt][j][3])
+                                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bf[j][0]), "r"(bf[j][1]));
+                }
             }
-            uint32_t keep = 0u;                            // outputs whose products cannot reach the result (rare)
-            if (elo < E_LOW || ehi > E_HIGH) {
-#pragma unroll
-                for (int h = 0; h < TH; ++h)
-#pragma unroll
-                    for (int x = 0; x < TW; ++x)
-                        if (S0[h][x] < E_LOW || S0[h][x] > E_HIGH) keep |= 1u << (h * TW + x);
-            }
-            // ---- the sum register (1.5 * 2^23 + S) * u with the accumulator term (see the FP32 kernel) ----
+            // e = max(exponent of the largest product, exponent of the accumulator), kept in the register of P
+            uint32_t out_of_range = 0u;
 #pragma unroll
             for (int h = 0; h < TH; ++h)
 #pragma unroll
                 for (int x = 0; x < TW; ++x) {
-                    const int ecl = max(min(S0[h][x], E_HIGH), E_LOW) + guard;
-                    const float magic = __int_as_float(((ecl + (150 - CB - FP_SHIFT)) << 23) | 0x00400000);
-                    const float cf = ACC16 ? __half2float(__ushort_as_half((unsigned short)cw[h][x])) : __uint_as_float(cw[h][x]);
-                    S0[h][x] = __float_as_int(__fmaf_rd(__int_as_float(__float_as_int(cf) | 1), c_scale, magic));
+                    float& p = P[h >> 1][x >> 1][2 * (h & 1) + (x & 1)];
+                    const uint32_t t1 = __umulhi(__float_as_uint(p), MUL6) + T1_ADD;
+                    uint32_t e;
+                    if (ACC16) {
+                        // a subnormal FP16 accumulator has the exponent -14, not that of its leading bit; the floor also
+                        // covers c = 0, harmlessly: every nonzero product has an exponent of at least -12
+                        const uint32_t ca = __float_as_uint(__half2float(__ushort_as_half((unsigned short)(cw[h][x] & 0x7FFFu))));
+                        e = uint32_t(__vimax3_s32(int(t1), int(ca), int(113u << 23)));
+                    } else {
+                        e = max(t1, cw[h][x] & 0x7FFFFFFFu);
+                        out_of_range = __viaddmax_u32(e, 0u - E_LOW, out_of_range);
+                    }
+                    p = __uint_as_float(e);
+                }
+            const bool rare = !ACC16 && out_of_range > E_HIGH - E_LOW;
+            if (rare) {                                    // turn the outputs out of range into markers (see above)
+#pragma unroll
+                for (int h = 0; h < TH; ++h)
+#pragma unroll
+                    for (int x = 0; x < TW; ++x) {
+                        float& p = P[h >> 1][x >> 1][2 * (h & 1) + (x & 1)];
+                        if (__float_as_uint(p) - E_LOW > E_HIGH - E_LOW) {
+                            const uint32_t c = cw[h][x];
+                            const uint32_t kept = (c & 0x7FFFFFFFu) ? (c >> 10) : 0u;      // rho(c); an exactly zero sum is +0
+                            p = __uint_as_float(E_KEEP);
+                            cw[h][x] = __float_as_uint(__uint2float_rn(kept) * __uint_as_float(uint32_t(E_KEEP >> 23) + uint32_t(23 - F) - 23u << 23));
+                        }
+                    }
+            }
+            // ---- the sum register with the accumulator term: floor((c + tiny) / unit); a negative c is one short ----
+#pragma unroll
+            for (int h = 0; h < TH; ++h)
+#pragma unroll
+                for (int x = 0; x < TW; ++x) {
+                    const uint32_t e = __float_as_uint(P[h >> 1][x >> 1][2 * (h & 1) + (x & 1)]);
+                    const uint32_t c = cw[h][x];
+                    const uint32_t magic = (e & FIELD) + MAGIC_ADD + (c >> (ACC16 ? 15 : 31));
+                    const float cf = ACC16 ? __half2float(__ushort_as_half((unsigned short)c)) : __uint_as_float(c);
+                    cw[h][x] = __float_as_uint(__fadd_rd(__uint_as_float(__float_as_uint(cf) | 1u), __uint_as_float(magic)));
                 }
             // ---- pass 2: one fused multiply-add per term, rounding toward minus infinity onto the grid of S ----
-#pragma unroll 4
+#pragma unroll
             for (int kk = kb; kk < kb + L; ++kk) {
                 const float4 oa = *reinterpret_cast<const float4*>(&s.a_op[kk][wr * 32 + 4 * gq]);
                 const float4 ob0 = *reinterpret_cast<const float4*>(&s.b_op[kk][wc * 32 + 8 * tq]);
@@ -297,7 +323,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
                 for (int h = 0; h < TH; ++h)
 #pragma unroll
                     for (int x = 0; x < TW; ++x)
-                        S0[h][x] = __float_as_int(__fmaf_rd(oav[h], obv[x], __int_as_float(S0[h][x])));
+                        cw[h][x] = __float_as_uint(__fmaf_rd(oav[h], obv[x], __uint_as_float(cw[h][x])));
             }
             // ---- sign corrections and rho ----
             const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
@@ -310,49 +336,36 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
                 sbv[4 * q] = u.x; sbv[4 * q + 1] = u.y; sbv[4 * q + 2] = u.z; sbv[4 * q + 3] = u.w;
                 nzb[4 * q] = v.x; nzb[4 * q + 1] = v.y; nzb[4 * q + 2] = v.z; nzb[4 * q + 3] = v.w;
             }
+            auto finish = [&](auto with_markers) {
 #pragma unroll
-            for (int h = 0; h < TH; ++h) {
-                const uint32_t sa = s.a_sgn[wr * 32 + 4 * gq + h];
-                const uint32_t nza = s.a_nz[wr * 32 + 4 * gq + h] & kmask;
+                for (int h = 0; h < TH; ++h) {
+                    const uint32_t sa = s.a_sgn[wr * 32 + 4 * gq + h];
+                    const uint32_t nza = s.a_nz[wr * 32 + 4 * gq + h] & kmask;
 #pragma unroll
-                for (int x = 0; x < TW; ++x) {
-                    const int nneg = __popc((sa ^ sbv[x]) & nza & nzb[x]);
-                    const int bits = S0[h][x];
-                    const int fld = bits & 0x7F800000;
-                    const int S = bits - (fld | 0x00400000) + nneg + int(cw[h][x] >> (ACC16 ? 15 : 31));
-                    const float scale = __int_as_float(fld - ((15 + F + guard) << 23));       // 2^(e_max - F)
-                    const float v = __fmul_rn(__int2float_rn(S), scale);
-                    uint32_t w;
-                    if (ACC16) { w = uint32_t(__half_as_ushort(__float2half_rn(v))); wmax = max(wmax, w & 0x7FFFu); }
-                    else w = __float_as_uint(v) & 0xFFFFFC00u;
-                    S0[h][x] = int(w);
+                    for (int x = 0; x < TW; ++x) {
+                        // every negative nonzero term fell one unit short: bits + count is (1.5 * 2^23 + S) * unit
+                        const uint32_t bits = cw[h][x] + uint32_t(__popc((sa ^ sbv[x]) & nza & nzb[x]));
+                        const float v = __fsub_rn(__uint_as_float(bits), __uint_as_float((bits & FIELD) | HALF));   // S * unit, exact
+                        uint32_t w;
+                        if (ACC16) { w = uint32_t(__half_as_ushort(__float2half_rn(v))); wmax = max(wmax, w & 0x7FFFu); }
+                        else w = __float_as_uint(v) & 0xFFFFFC00u;
+                        if (decltype(with_markers)::value && bits >= KEEP) w = (bits - KEEP) << 10;
+                        cw[h][x] = w;
+                    }
                 }
-            }
-            if (keep) {                                    // rare: rho of the accumulator alone; an exactly zero sum is +0
-#pragma unroll
-                for (int h = 0; h < TH; ++h)
-#pragma unroll
-                    for (int x = 0; x < TW; ++x)
-                        if ((keep >> (h * TW + x)) & 1u) {
-                            const uint32_t t = ACC16 ? cw[h][x] : (cw[h][x] & 0xFFFFFC00u);
-                            S0[h][x] = int((t & (ACC16 ? 0x7FFFu : 0x7FFFFFFFu)) ? t : 0u);
-                        }
-            }
+            };
+            if (rare) finish(std::true_type{}); else finish(std::false_type{});
             if (ACC16 && wmax >= 0x7C00u) {                // rare: RNE-FP16 overflowed: +-infinity from now on
 #pragma unroll
                 for (int h = 0; h < TH; ++h)
 #pragma unroll
                     for (int x = 0; x < TW; ++x)
-                        if ((uint32_t(S0[h][x]) & 0x7FFFu) == 0x7C00u) {
+                        if ((cw[h][x] & 0x7FFFu) == 0x7C00u) {
                             const uint32_t bit = 1u << (h * TW + x);
-                            if (!((sp_nan | sp_pinf | sp_ninf) & bit)) { if (uint32_t(S0[h][x]) >> 15) sp_ninf |= bit; else sp_pinf |= bit; }
-                            S0[h][x] = 0;
+                            if (!((sp_nan | sp_pinf | sp_ninf) & bit)) { if (cw[h][x] >> 15) sp_ninf |= bit; else sp_pinf |= bit; }
+                            cw[h][x] = 0u;
                         }
             }
-#pragma unroll
-            for (int h = 0; h < TH; ++h)
-#pragma unroll
-                for (int x = 0; x < TW; ++x) cw[h][x] = uint32_t(S0[h][x]);
         }
         __syncthreads();                                   // the other buffer is complete, this one is free
         if (PROMOTE && ((k0 + KC) % g.k_chunk) == 0) {     // FP32 promotion of the partial sum every k_chunk elements
