@@ -8,7 +8,7 @@ namespace {
 
 enum PeakKind : int {
     PK_IADD3 = 0, PK_LOP3, PK_SHF, PK_IMAD, PK_MACMIX, PK_VIADDMAX, PK_VIADDMAX16X2, PK_F2I, PK_FMUL, PK_POPC,
-    PK_IMAD_PLUS_ALU, PK_FMUL_PLUS_ALU, PK_IMAD_WIDE, PK_MAC_D1, PK_MAC_D2, PK_DP4A, PK_DFMA, PK_DFMA_PLUS_ALU, PK_COUNT
+    PK_IMAD_PLUS_ALU, PK_FMUL_PLUS_ALU, PK_IMAD_WIDE, PK_MAC_D1, PK_MAC_D2, PK_DP4A, PK_DFMA, PK_DFMA_PLUS_ALU, PK_FFMA_RM, PK_FFMA2_RM, PK_COUNT
 };
 
 template <int KIND>
@@ -94,6 +94,41 @@ __global__ void __launch_bounds__(256) peak_kernel_f64(int64_t iters, int* sink)
     if (r == 0.12345 && q == 0x12345678) *sink = 1;
 }
 
+// FP32 fused multiply-add rounded toward minus infinity, the instruction of the FP32 summation kernels: scalar form,
+// and the packed two-lane form of sm_100 (fma.rm.f32x2), eight independent accumulator chains (pairs) per thread.
+template <bool PACKED>
+__global__ void __launch_bounds__(256) peak_kernel_f32(int64_t iters, int* sink) {
+    float a[8], b[8], c[16];
+    unsigned long long a2[8], b2[8], c2[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { a[i] = 1.0f + 1e-7f * float(threadIdx.x + i); b[i] = 1.0f - 1e-7f * float(threadIdx.x + 2 * i); }
+#pragma unroll
+    for (int i = 0; i < 16; ++i) c[i] = float(i);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        asm("mov.b64 %0, {%1, %2};" : "=l"(a2[i]) : "f"(a[i]), "f"(a[(i + 1) & 7]));
+        asm("mov.b64 %0, {%1, %2};" : "=l"(b2[i]) : "f"(b[i]), "f"(b[(i + 1) & 7]));
+        asm("mov.b64 %0, {%1, %2};" : "=l"(c2[i]) : "f"(c[2 * i]), "f"(c[2 * i + 1]));
+    }
+    for (int64_t it = 0; it < iters; it += 8) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (PACKED) asm volatile("fma.rm.f32x2 %0, %1, %2, %0;" : "+l"(c2[i]) : "l"(a2[i]), "l"(b2[u]));
+                else c[i] = __fmaf_rd(a[i], b[u], c[i]);
+            }
+    }
+    float r = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        float lo, hi;
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(c2[i]));
+        r += PACKED ? lo + hi : c[i];
+    }
+    if (r == 0.12345f) *sink = 1;
+}
+
 template <int KIND>
 int launch(int64_t blocks, int64_t iters, void* sink, cudaStream_t stream) {
     peak_kernel<KIND><<<(unsigned)blocks, 256, 0, stream>>>(iters, static_cast<int*>(sink));
@@ -128,6 +163,15 @@ int launch_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t
             *ops_per_round = kind == PK_DFMA ? 1 : 2;
             if (kind == PK_DFMA) peak_kernel_f64<false><<<(unsigned)blocks, 256, 0, stream>>>(iters, static_cast<int*>(sink));
             else peak_kernel_f64<true><<<(unsigned)blocks, 256, 0, stream>>>(iters, static_cast<int*>(sink));
+            const cudaError_t err = cudaGetLastError();
+            if (err != cudaSuccess) { set_error("int_peak launch failed: %s", cudaGetErrorString(err)); return MMASIM_ERR_CUDA; }
+            return MMASIM_OK;
+        }
+        case PK_FFMA_RM:
+        case PK_FFMA2_RM: {
+            *ops_per_round = kind == PK_FFMA_RM ? 1 : 2;
+            if (kind == PK_FFMA_RM) peak_kernel_f32<false><<<(unsigned)blocks, 256, 0, stream>>>(iters, static_cast<int*>(sink));
+            else peak_kernel_f32<true><<<(unsigned)blocks, 256, 0, stream>>>(iters, static_cast<int*>(sink));
             const cudaError_t err = cudaGetLastError();
             if (err != cudaSuccess) { set_error("int_peak launch failed: %s", cudaGetErrorString(err)); return MMASIM_ERR_CUDA; }
             return MMASIM_OK;

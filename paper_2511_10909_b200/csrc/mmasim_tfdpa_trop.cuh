@@ -311,19 +311,36 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
                     const float cf = ACC16 ? __half2float(__ushort_as_half((unsigned short)c)) : __uint_as_float(c);
                     cw[h][x] = __float_as_uint(__fadd_rd(__uint_as_float(__float_as_uint(cf) | 1u), __uint_as_float(magic)));
                 }
-            // ---- pass 2: one fused multiply-add per term, rounding toward minus infinity onto the grid of S ----
-#pragma unroll
-            for (int kk = kb; kk < kb + L; ++kk) {
-                const float4 oa = *reinterpret_cast<const float4*>(&s.a_op[kk][wr * 32 + 4 * gq]);
-                const float4 ob0 = *reinterpret_cast<const float4*>(&s.b_op[kk][wc * 32 + 8 * tq]);
-                const float4 ob1 = *reinterpret_cast<const float4*>(&s.b_op[kk][wc * 32 + 8 * tq + 4]);
-                const float oav[TH] = {oa.x, oa.y, oa.z, oa.w};
-                const float obv[TW] = {ob0.x, ob0.y, ob0.z, ob0.w, ob1.x, ob1.y, ob1.z, ob1.w};
+            // ---- pass 2: one fused multiply-add per term, rounding toward minus infinity onto the grid of S; two
+            // columns of the micro-tile per instruction (fma.rm.f32x2: lanes (a_h, a_h) x (b_x, b_x+1) + (S_h,x, S_h,x+1)) ----
+            {
+                unsigned long long acc[TH][TW / 2];
 #pragma unroll
                 for (int h = 0; h < TH; ++h)
 #pragma unroll
-                    for (int x = 0; x < TW; ++x)
-                        cw[h][x] = __float_as_uint(__fmaf_rd(oav[h], obv[x], __uint_as_float(cw[h][x])));
+                    for (int xp = 0; xp < TW / 2; ++xp)
+                        asm("mov.b64 %0, {%1, %2};" : "=l"(acc[h][xp]) : "r"(cw[h][2 * xp]), "r"(cw[h][2 * xp + 1]));
+#pragma unroll
+                for (int kk = kb; kk < kb + L; ++kk) {
+                    const float4 oa = *reinterpret_cast<const float4*>(&s.a_op[kk][wr * 32 + 4 * gq]);
+                    const ulonglong2 ob0 = *reinterpret_cast<const ulonglong2*>(&s.b_op[kk][wc * 32 + 8 * tq]);
+                    const ulonglong2 ob1 = *reinterpret_cast<const ulonglong2*>(&s.b_op[kk][wc * 32 + 8 * tq + 4]);
+                    const float oas[TH] = {oa.x, oa.y, oa.z, oa.w};
+                    const unsigned long long obv[TW / 2] = {ob0.x, ob0.y, ob1.x, ob1.y};
+#pragma unroll
+                    for (int h = 0; h < TH; ++h) {
+                        unsigned long long oav;
+                        asm("mov.b64 %0, {%1, %1};" : "=l"(oav) : "f"(oas[h]));
+#pragma unroll
+                        for (int xp = 0; xp < TW / 2; ++xp)
+                            asm("fma.rm.f32x2 %0, %1, %2, %0;" : "+l"(acc[h][xp]) : "l"(oav), "l"(obv[xp]));
+                    }
+                }
+#pragma unroll
+                for (int h = 0; h < TH; ++h)
+#pragma unroll
+                    for (int xp = 0; xp < TW / 2; ++xp)
+                        asm("mov.b64 {%0, %1}, %2;" : "=r"(cw[h][2 * xp]), "=r"(cw[h][2 * xp + 1]) : "l"(acc[h][xp]));
             }
             // ---- sign corrections and rho ----
             const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);

@@ -268,7 +268,7 @@ def hw_mma(kind: str, A, B, C=None, out=None, *, stream=None):
 
 
 PEAK_KINDS = ["iadd3", "lop3", "shf", "imad", "macmix", "viaddmax", "viaddmax16x2", "f2i", "fmul", "popc",
-              "imad+alu", "fmul+alu", "imad.wide", "mac_d1", "mac_d2", "dp4a", "dfma", "dfma+alu"]
+              "imad+alu", "fmul+alu", "imad.wide", "mac_d1", "mac_d2", "dp4a", "dfma", "dfma+alu", "ffma.rm", "ffma2.rm"]
 
 
 def int_peak(kind: str, blocks: int, iters: int, sink, stream=None) -> int:
