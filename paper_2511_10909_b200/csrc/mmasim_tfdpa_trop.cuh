@@ -35,8 +35,6 @@ using fast::KC;
 using fast::NT;
 using fast::CB;
 using fast::Elem;
-using fast::RawChunk;
-using fast::load_chunk;
 using fast::raw_elem;
 
 constexpr int PE_STRIDE = KC + 8;       // BF16 elements per row of a pe plane: 80 bytes, fragment loads hit 32 different banks
@@ -44,11 +42,10 @@ constexpr int PE_CENTER = 1;            // pe(x) = 2^(6 (Exp(x) - PE_CENTER)); E
 constexpr int PE_B_SHIFT = 5;           // pe(b) carries 2^5 more, so that the exponent field of P is 6 (e_max + 20) + 0..5
 constexpr int TH = 4, TW = 8;           // micro-tile: 4 rows x 8 columns
 
-struct LutEntryT {
-    uint32_t op;        // staged FP32 operand (see mmasim_tfdpa_fast.cuh)
-    uint16_t pe;        // BF16 word of pe(x)
-    uint8_t bits;       // bit 0: sign, bit 1: finite and nonzero
-    uint8_t special;    // infinity / NaN
+struct LutEntryT {      // 8 bytes: one shared load per staged element
+    uint32_t op;        // staged FP32 operand
+    uint32_t y;         // bits 0..14: BF16 word of pe(x); bit 15: infinity / NaN (a pe of -0: harmless in P);
+                        // bit 16: sign; bit 24: finite and nonzero
 };
 
 struct PlanesT {
@@ -77,61 +74,75 @@ __device__ __forceinline__ void init_lut_t(SmemT& s, const FmtDesc& fa, const Fm
     const bool nz_a = fin_a && dec_sig(da) != 0u, nz_b = fin_b && dec_sig(db) != 0u;
     LutEntryT ea, eb;
     ea.op = __float_as_uint(ldexpf(float(fin_a ? dec_ssig(da) : 0), fin_a ? dec_exp(da) : 0));
-    ea.pe = nz_a ? uint16_t((127 + 6 * (dec_exp(da) - PE_CENTER)) << 7) : uint16_t(0);
-    ea.bits = uint8_t(fin_a ? (dec_sign(da) | (uint32_t(nz_a) << 1)) : 0u);
-    ea.special = fin_a ? 0 : 1;
+    ea.y = (nz_a ? uint32_t((127 + 6 * (dec_exp(da) - PE_CENTER)) << 7) : 0u) | (fin_a ? 0u : 0x8000u) |
+           (fin_a ? (dec_sign(da) << 16) | (uint32_t(nz_a) << 24) : 0u);
     const int sb = fin_b ? dec_ssig(db) : 0;
     const int ub = dec_sign(db) ? -1 : 1;
     // a_op * b_op = a * b * (1 + 2^-(pre + guard) / |sig_b|): the true product with the offset that makes a negative one inexact
     eb.op = nz_b ? __float_as_uint(ldexpf(float(sb * (1 << (pre + guard)) + ub), dec_exp(db) - (fa.mbits + fb.mbits + pre + guard))) : 0u;
-    eb.pe = nz_b ? uint16_t((127 + PE_B_SHIFT + 6 * (dec_exp(db) - PE_CENTER)) << 7) : uint16_t(0);
-    eb.bits = uint8_t(fin_b ? (dec_sign(db) | (uint32_t(nz_b) << 1)) : 0u);
-    eb.special = fin_b ? 0 : 1;
+    eb.y = (nz_b ? uint32_t((127 + PE_B_SHIFT + 6 * (dec_exp(db) - PE_CENTER)) << 7) : 0u) | (fin_b ? 0u : 0x8000u) |
+           (fin_b ? (dec_sign(db) << 16) | (uint32_t(nz_b) << 24) : 0u);
     s.lut_a[tid] = ea;
     s.lut_b[tid] = eb;
 }
 
+// Staging of one chunk of KC = 32 elements of K.  Every thread takes sixteen consecutive elements of one row of A (row
+// tid % 128, half tid / 128) and eight of one column of B (column tid % 64, quarter tid / 64): the same work for all, so
+// that nobody waits at the barrier.  The raw bytes are fetched one chunk ahead into registers.
+struct RawT {
+    uint4 a;
+    uint2 b;
+};
+static_assert(BM == 128 && BN == 64 && KC == 32 && NT == 256, "the task split of the staging");
+
 template <int EK>
-__device__ __forceinline__ void store_chunk_t(SmemT& sm, PlanesT& s, const RawChunk<EK>& raw, int flag, int tid) {
-    using E = Elem<EK>;
-    using R = RawChunk<EK>;
-    static_assert(!E::SIGNMAG && E::TASK == 16, "table-decoded 8-bit elements, sixteen per task");
-    uint32_t spec = 0u;
+__device__ __forceinline__ void load_chunk_t(RawT& raw, const GemmArgs& g, int64_t row0, int64_t col0, int64_t k0, int tid) {
+    static_assert(Elem<EK>::BYTES == 1, "8-bit elements");
+    const int64_t i = row0 + (tid & 127), j = col0 + (tid & 63);
+    raw.a = make_uint4(0u, 0u, 0u, 0u);
+    raw.b = make_uint2(0u, 0u);
+    if (i < g.M) raw.a = *reinterpret_cast<const uint4*>(static_cast<const unsigned char*>(g.A) + i * g.lda + k0 + 16 * (tid >> 7));
+    if (j < g.N) raw.b = *reinterpret_cast<const uint2*>(static_cast<const unsigned char*>(g.B) + j * g.ldb + k0 + 8 * (tid >> 6));
+}
+
+// Sixteen (A) or eight (B) elements of one row: operands k-major, pe words row-major, sign / nonzero bits into the masks.
+template <int N, bool IS_A>
+__device__ __forceinline__ uint32_t stage_row(SmemT& sm, PlanesT& s, const uint32_t (&w)[N / 4], int r, int part) {
+    const LutEntryT* lut = IS_A ? sm.lut_a : sm.lut_b;
+    const int pr = IS_A ? perm_row(r) : perm_col(r);
+    uint32_t* op = IS_A ? &s.a_op[part * N][pr] : &s.b_op[part * N][pr];
+    constexpr int STRIDE = IS_A ? BM : BN;
+    uint32_t acc = 0u, spec = 0u, pw[N / 2];
 #pragma unroll
-    for (int it = 0; it < R::PER_THREAD; ++it) {
-        const int task = it * NT + tid;
-        if (task >= R::TASKS) break;
-        const bool is_a = task < BM * R::TPR;
-        const int u = is_a ? task : task - BM * R::TPR;
-        const int rows = is_a ? BM : BN;
-        const int r = u % rows, h = u / rows;
-        const int pr = is_a ? perm_row(r) : perm_col(r);
-        uint32_t sgn = 0u, nz = 0u, prev_pe = 0u;
-#pragma unroll
-        for (int q = 0; q < E::TASK; ++q) {
-            const int kk = h * E::TASK + q;
-            const uint32_t byte = (raw.w[it][q / 4] >> (8 * (q % 4))) & 0xFFu;
-            const LutEntryT e = is_a ? sm.lut_a[byte] : sm.lut_b[byte];
-            sgn |= uint32_t(e.bits & 1u) << q;
-            nz |= uint32_t((e.bits >> 1) & 1u) << q;
-            spec |= e.special;
-            if (is_a) s.a_op[kk][pr] = e.op; else s.b_op[kk][pr] = e.op;
-            if (q & 1) {
-                const uint32_t pair = prev_pe | (uint32_t(e.pe) << 16);
-                if (is_a) *reinterpret_cast<uint32_t*>(&s.a_pe[r][kk - 1]) = pair;
-                else *reinterpret_cast<uint32_t*>(&s.b_pe[r][kk - 1]) = pair;
-            }
-            prev_pe = e.pe;
-        }
-        if (is_a) {
-            reinterpret_cast<uint16_t*>(&s.a_sgn[pr])[h] = uint16_t(sgn);
-            reinterpret_cast<uint16_t*>(&s.a_nz[pr])[h] = uint16_t(nz);
-        } else {
-            reinterpret_cast<uint16_t*>(&s.b_sgn[pr])[h] = uint16_t(sgn);
-            reinterpret_cast<uint16_t*>(&s.b_nz[pr])[h] = uint16_t(nz);
-        }
+    for (int q = 0; q < N; q += 2) {
+        const uint2 e0 = *reinterpret_cast<const uint2*>(&lut[(w[q / 4] >> (8 * (q % 4))) & 0xFFu]);
+        const uint2 e1 = *reinterpret_cast<const uint2*>(&lut[(w[q / 4] >> (8 * (q % 4) + 8)) & 0xFFu]);
+        op[q * STRIDE] = e0.x;
+        op[(q + 1) * STRIDE] = e1.x;
+        // sign byte -> bits 0.., nonzero byte -> bits 16..
+        acc += (__byte_perm(e0.y, 0u, 0x4342) << q) + (__byte_perm(e1.y, 0u, 0x4342) << (q + 1));
+        spec |= e0.y | e1.y;
+        pw[q / 2] = __byte_perm(e0.y, e1.y, 0x5410);
     }
-    if (spec) atomicOr(&sm.special[flag], 1);
+    uint16_t* pe = IS_A ? &s.a_pe[r][part * N] : &s.b_pe[r][part * N];
+#pragma unroll
+    for (int q = 0; q < N / 8; ++q)
+        reinterpret_cast<uint4*>(pe)[q] = make_uint4(pw[4 * q], pw[4 * q + 1], pw[4 * q + 2], pw[4 * q + 3]);
+    if (IS_A) {
+        reinterpret_cast<uint16_t*>(&s.a_sgn[pr])[part] = uint16_t(acc);
+        reinterpret_cast<uint16_t*>(&s.a_nz[pr])[part] = uint16_t(acc >> 16);
+    } else {
+        reinterpret_cast<uint8_t*>(&s.b_sgn[pr])[part] = uint8_t(acc);
+        reinterpret_cast<uint8_t*>(&s.b_nz[pr])[part] = uint8_t(acc >> 16);
+    }
+    return spec;
+}
+
+__device__ __forceinline__ void store_chunk_t(SmemT& sm, PlanesT& s, const RawT& raw, int flag, int tid) {
+    const uint32_t wa[4] = {raw.a.x, raw.a.y, raw.a.z, raw.a.w};
+    const uint32_t wb[2] = {raw.b.x, raw.b.y};
+    const uint32_t spec = stage_row<16, true>(sm, s, wa, tid & 127, tid >> 7) | stage_row<8, false>(sm, s, wb, tid & 63, tid >> 6);
+    if (spec & 0x8000u) atomicOr(&sm.special[flag], 1);
 }
 
 template <int EK, int L, int F, int RHO, bool PROMOTE>
@@ -197,18 +208,18 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
             cw[h][x] = w;
         }
 
-    RawChunk<EK> raw;
-    load_chunk<EK>(raw, g, row0, col0, 0, tid);
+    RawT raw;
+    load_chunk_t<EK>(raw, g, row0, col0, 0, tid);
     __syncthreads();                                       // tables and flags are ready
-    store_chunk_t<EK>(sm, sm.pl[0], raw, 0, tid);
-    if (KC < g.K) load_chunk<EK>(raw, g, row0, col0, KC, tid);
+    store_chunk_t(sm, sm.pl[0], raw, 0, tid);
+    if (KC < g.K) load_chunk_t<EK>(raw, g, row0, col0, KC, tid);
     __syncthreads();
     int chunk = 0;
     for (int64_t k0 = 0; k0 < g.K; k0 += KC, ++chunk) {
         if (tid == 0) sm.special[(chunk + 2) % 3] = 0;
         if (k0 + KC < g.K) {
-            store_chunk_t<EK>(sm, sm.pl[(chunk + 1) & 1], raw, (chunk + 1) % 3, tid);
-            if (k0 + 2 * KC < g.K) load_chunk<EK>(raw, g, row0, col0, k0 + 2 * KC, tid);
+            store_chunk_t(sm, sm.pl[(chunk + 1) & 1], raw, (chunk + 1) % 3, tid);
+            if (k0 + 2 * KC < g.K) load_chunk_t<EK>(raw, g, row0, col0, k0 + 2 * KC, tid);
         }
         PlanesT& s = sm.pl[chunk & 1];
         const bool chunk_special = sm.special[chunk % 3] != 0;
