@@ -8,16 +8,13 @@ cudaError_t launch_lut8(const DevModel& m, const GemmArgs& g, cudaStream_t st) {
         if (m.F == 25 && m.L == 32 && m.rho == RHO_RZ_FP32) return fast64::launch_variant64<EK_LUT8, 32, RHO_RZ_FP32, true>(m, g, st);
         return cudaErrorInvalidValue;
     }
-    if (m.F == 13 && m.fmt_a == EF_E4M3 && m.fmt_b == EF_E4M3) {       // E4M3 x E4M3: the exponent maximum on the tensor cores
-        if (m.L == 16 && m.rho == RHO_RZ_E8M13) return trop::launch_variant_t<EK_LUT8, 16, 13, RHO_RZ_E8M13>(m, g, st);
-        if (m.L == 16 && m.rho == RHO_RNE_FP16) return trop::launch_variant_t<EK_LUT8, 16, 13, RHO_RNE_FP16>(m, g, st);
-        if (m.L == 32 && m.rho == RHO_RZ_E8M13) return trop::launch_variant_t<EK_LUT8, 32, 13, RHO_RZ_E8M13>(m, g, st);
-        if (m.L == 32 && m.rho == RHO_RNE_FP16) return trop::launch_variant_t<EK_LUT8, 32, 13, RHO_RNE_FP16>(m, g, st);
+    if (m.F == 13) {                                    // FP8 x FP8 with F = 13: the exponent maximum on the tensor cores
+        if (m.L == 16 && m.rho == RHO_RZ_E8M13) return trop::launch_by_types_t<EK_LUT8, 16, 13, RHO_RZ_E8M13>(m, g, st);
+        if (m.L == 16 && m.rho == RHO_RNE_FP16) return trop::launch_by_types_t<EK_LUT8, 16, 13, RHO_RNE_FP16>(m, g, st);
+        if (m.L == 32 && m.rho == RHO_RZ_E8M13) return trop::launch_by_types_t<EK_LUT8, 32, 13, RHO_RZ_E8M13>(m, g, st);
+        if (m.L == 32 && m.rho == RHO_RNE_FP16) return trop::launch_by_types_t<EK_LUT8, 32, 13, RHO_RNE_FP16>(m, g, st);
+        return cudaErrorInvalidValue;
     }
-    if (m.F == 13 && m.L == 16 && m.rho == RHO_RZ_E8M13) return launch_variant<EK_LUT8, 16, 13, RHO_RZ_E8M13>(m, g, st);
-    if (m.F == 13 && m.L == 16 && m.rho == RHO_RNE_FP16) return launch_variant<EK_LUT8, 16, 13, RHO_RNE_FP16>(m, g, st);
-    if (m.F == 13 && m.L == 32 && m.rho == RHO_RZ_E8M13) return launch_variant<EK_LUT8, 32, 13, RHO_RZ_E8M13>(m, g, st);
-    if (m.F == 13 && m.L == 32 && m.rho == RHO_RNE_FP16) return launch_variant<EK_LUT8, 32, 13, RHO_RNE_FP16>(m, g, st);
     if (m.F == 25 && m.L == 32 && m.rho == RHO_RZ_FP32) return fast64::launch_variant64<EK_LUT8, 32, RHO_RZ_FP32>(m, g, st);
     if (m.F == 25 && m.L == 32 && m.rho == RHO_RNE_FP16) return fast64::launch_variant64<EK_LUT8, 32, RHO_RNE_FP16>(m, g, st);
     return cudaErrorInvalidValue;

@@ -1,27 +1,38 @@
-// T-FDPA for E4M3 inputs with F = 13 (the Ada / Hopper FP8 rows on E4M3 operands; Algorithm 5 + 7 + Table 2): the FP32
-// summation kernel of mmasim_tfdpa_fast.cuh with the exponent maximum taken by the tensor cores.
+// T-FDPA for FP8 inputs with F = 13 (the Ada / Hopper FP8 rows, E4M3 and E5M2 in any combination; Algorithm 5 + 7 +
+// Table 2): the sum of a block in an FP32 register, one fused multiply-add per term, and the block's exponent maximum
+// taken by the tensor cores.
+//
+// The sum register.  Aligned terms are below 2^15 and block sums below 2^21, so the fixed-point sum S of Algorithm 7
+// fits an FP32 register as (1.5 * 2^23 + S) * u with u = 2^(e_max - F): in [2^23 u, 2^24 u) one ulp is u, so
+// fma.rm.f32(a, b, register) forms a * b + register exactly and rounds once, toward minus infinity, onto multiples of
+// u - the shift by e_max - e_k, the truncation and the addition of Algorithm 7 in one instruction, the alignment
+// distance carried by the register's exponent.  Operands are the element values (A) and the element values with an
+// offset 2^-(pre + guard) below the last significand bit (B), so that a negative product is never on the grid and
+// floors to the one's complement of its truncated magnitude; a population count over sign / nonzero masks adds the
+// number of negative nonzero terms back.  The accumulator enters by one addition rounded toward minus infinity (its
+// lowest mantissa bit set, so that a negative c floors likewise; the +1 is added to the register's starting value),
+// and the block's value S * u leaves by one exact subtraction of 1.5 * 2^23 * u; rho is a mask (RZ-E8M13) or a
+// conversion (RNE-FP16).  The accumulator between blocks is the output word itself.
 //
 // e_max = max_k (Exp(a_k) + Exp(b_k)) is a (max, +) product.  Powers turn it into an ordinary one: with
 // pe(x) = 2^(6 (Exp(x) - 1)) for a nonzero finite x and 0 otherwise (the B plane scaled by 2^5 more),
 //     P = sum_k pe(a_k) * pe(b_k)  lies in  2^(6 (e_max + 20) - 127) * [1, 32]  (at most 32 terms, 32 < 2^6),
 // so its FP32 exponent field is 6 (e_max + 20) + 0..5 and floor(field / 6) - 20 = e_max exactly, whatever the order,
 // rounding or truncation of the summation (terms far below the largest may be dropped, they do not matter).  E4M3
-// exponents span 15 values: 6 * (Exp - 1) stays within +-42 and P within the FP32 range.  P for the 32 x 32 outputs
+// exponents span 15 values: 6 * (Exp - 1) stays within +-42 and P within the FP32 range; with E5M2 operands the base
+// is 2^5 or 2^4 and P is taken over sub-blocks of 16 or 8 terms (see pe_shift below).  P for the 32 x 32 outputs
 // of a warp and one block of 32 is sixteen mma.sync.m16n8k16 on BF16 planes of pe values (a power of two is exact in
 // BF16), instead of sixteen fused add-max instructions per output; P = 0 (every product zero: no exponent) converts
-// to an exponent below every real one.  The division by 6 is one high multiply on the bits of P, which leaves the
-// result as an FP32 exponent field in place, comparable with the bits of |c| and a mask away from the sum register's
-// starting value.
+// to an exponent below every real one.  The division by the base is one high multiply on the bits of P, which leaves
+// the result as an FP32 exponent field in place, comparable with the bits of |c| and a mask away from the sum
+// register's starting value.
 //
 // A warp owns 32 rows x 32 columns of the CTA tile (two by four accumulator fragments), and the micro-tile of a thread is
 // its share of those fragments: rows g, g + 8, g + 16, g + 24 (g = lane / 4) and columns 8 j + 2 t, 8 j + 2 t + 1
 // (t = lane % 4, j = 0..3), so that the maxima arrive in the registers of the thread that needs them.  The operand
 // planes are stored with rows and columns permuted accordingly (the four rows of a thread adjacent, its eight
-// columns contiguous): three 16-byte shared loads feed the 32 fused multiply-adds of one k.
-// The sum register works as in the FP32 summation kernel, here in the true scale: operands are the element values (B
-// with the small offset that makes negative products inexact), the register is (1.5 * 2^23 + S) * 2^(e_max - F), the
-// accumulator enters by one addition rounded toward minus infinity and the block's value S * 2^(e_max - F) leaves by
-// one exact subtraction; rho is a mask (RZ-E8M13) or a conversion (RNE-FP16).
+// columns contiguous): three 16-byte shared loads feed the 32 fused multiply-adds of one k, which are issued as
+// sixteen packed ones (fma.rm.f32x2: two adjacent columns per instruction).
 #pragma once
 #include <type_traits>
 #include "mmasim_tfdpa_fast.cuh"
@@ -39,7 +50,16 @@ using fast::raw_elem;
 
 constexpr int PE_STRIDE = KC + 8;       // BF16 elements per row of a pe plane: 80 bytes, fragment loads hit 32 different banks
 constexpr int PE_CENTER = 1;            // pe(x) = 2^(6 (Exp(x) - PE_CENTER)); E4M3: Exp in [-6, 8]
-constexpr int PE_B_SHIFT = 5;           // pe(b) carries 2^5 more, so that the exponent field of P is 6 (e_max + 20) + 0..5
+// pe(x) = 2^(BASE (Exp(x) - PE_CENTER)), the B plane times 2^pe_shift so that 127 + pe_shift is a multiple of BASE and
+// the exponent field of P is BASE * (e_max + constant) + 0..BASE-1.  A sum of at most 2^(BASE-1) terms stays within a
+// factor 2^(BASE-1) of its largest term; the spread of the exponents decides which BASE fits the FP32 range:
+//   BASE 6: blocks of up to 32 terms in one accumulation; E4M3 x E4M3 (product exponents -12..16: 6 * 28 = 168 binades)
+//   BASE 5: sub-blocks of 16 terms; E4M3 x E5M2 (-20..23: 5 * 43 = 215 binades)
+//   BASE 4: sub-blocks of 8 terms;  E5M2 x E5M2 (-28..30: 4 * 58 = 232 binades)
+// The block maximum is then the integer maximum of the sub-blocks' P words.
+__host__ __device__ constexpr int pe_shift(int base) { return base == 6 ? 5 : (base == 5 ? 3 : 1); }
+__host__ __device__ constexpr int pe_sub(int base) { return base == 6 ? 32 : (base == 5 ? 16 : 8); }
+__host__ __device__ constexpr uint32_t pe_mul(int base) { return base == 6 ? 0x2AAAAAABu : (base == 5 ? 0x33333334u : 0x40000000u); }  // ceil(2^32 / BASE)
 constexpr int TH = 4, TW = 8;           // micro-tile: 4 rows x 8 columns
 
 struct LutEntryT {      // 8 bytes: one shared load per staged element
@@ -68,19 +88,20 @@ struct SmemT {
 __device__ __forceinline__ int perm_row(int r) { return (r & ~31) | ((r & 7) << 2) | ((r >> 3) & 3); }
 __device__ __forceinline__ int perm_col(int c) { return (c & ~31) | (((c >> 1) & 3) << 3) | (((c >> 3) & 3) << 1) | (c & 1); }
 
+template <int BASE>
 __device__ __forceinline__ void init_lut_t(SmemT& s, const FmtDesc& fa, const FmtDesc& fb, int pre, int guard, int tid) {
     const uint32_t da = decode_elem(fa, uint32_t(tid)), db = decode_elem(fb, uint32_t(tid));
     const bool fin_a = dec_cls(da) == CLS_FINITE, fin_b = dec_cls(db) == CLS_FINITE;
     const bool nz_a = fin_a && dec_sig(da) != 0u, nz_b = fin_b && dec_sig(db) != 0u;
     LutEntryT ea, eb;
     ea.op = __float_as_uint(ldexpf(float(fin_a ? dec_ssig(da) : 0), fin_a ? dec_exp(da) : 0));
-    ea.y = (nz_a ? uint32_t((127 + 6 * (dec_exp(da) - PE_CENTER)) << 7) : 0u) | (fin_a ? 0u : 0x8000u) |
+    ea.y = (nz_a ? uint32_t((127 + BASE * (dec_exp(da) - PE_CENTER)) << 7) : 0u) | (fin_a ? 0u : 0x8000u) |
            (fin_a ? (dec_sign(da) << 16) | (uint32_t(nz_a) << 24) : 0u);
     const int sb = fin_b ? dec_ssig(db) : 0;
     const int ub = dec_sign(db) ? -1 : 1;
     // a_op * b_op = a * b * (1 + 2^-(pre + guard) / |sig_b|): the true product with the offset that makes a negative one inexact
     eb.op = nz_b ? __float_as_uint(ldexpf(float(sb * (1 << (pre + guard)) + ub), dec_exp(db) - (fa.mbits + fb.mbits + pre + guard))) : 0u;
-    eb.y = (nz_b ? uint32_t((127 + PE_B_SHIFT + 6 * (dec_exp(db) - PE_CENTER)) << 7) : 0u) | (fin_b ? 0u : 0x8000u) |
+    eb.y = (nz_b ? uint32_t((127 + pe_shift(BASE) + BASE * (dec_exp(db) - PE_CENTER)) << 7) : 0u) | (fin_b ? 0u : 0x8000u) |
            (fin_b ? (dec_sign(db) << 16) | (uint32_t(nz_b) << 24) : 0u);
     s.lut_a[tid] = ea;
     s.lut_b[tid] = eb;
@@ -145,11 +166,13 @@ __device__ __forceinline__ void store_chunk_t(SmemT& sm, PlanesT& s, const RawT&
     if (spec & 0x8000u) atomicOr(&sm.special[flag], 1);
 }
 
-template <int EK, int L, int F, int RHO, bool PROMOTE>
+template <int EK, int L, int F, int RHO, bool PROMOTE, int BASE>
 __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs g) {
     constexpr bool ACC16 = RHO == RHO_RNE_FP16;
     constexpr int NBLK = KC / L;
     static_assert(KC % L == 0 && L % 16 == 0, "a block is one or two k16 matrix instructions");
+    static_assert(BASE == 4 || BASE == 5 || BASE == 6, "see pe_shift");
+    constexpr int KSUB = pe_sub(BASE) < L ? pe_sub(BASE) : L, NSUB = L / KSUB;        // terms per accumulation of P
     static_assert(!Elem<EK>::SIGNMAG && F <= 13, "8-bit inputs with F <= 13");
     static_assert(RHO == RHO_RZ_E8M13 || RHO == RHO_RNE_FP16, "rho of the F = 13 rows of Table 4");
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -166,22 +189,23 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
     const int pre = F - (fa.mbits + fb.mbits);
     const int guard = fa.mbits + 1;
     // Exponents are handled as FP32 exponent fields in place (bits 23..30) with whatever lies below as a fraction:
-    //   t1 = floor(bits(P) / 6) + (107 << 23): field e_max + 127 for the largest product (P = 0: field 107, e_max = -20,
-    //        below the smallest nonzero E4M3 product, 2^-12); dividing by 6 is a high multiply, inexact by 2^-31 and P is
-    //        never closer than 1/6 to the next multiple;
+    //   t1 = floor(bits(P) / BASE) + T1_ADD: field e_max + 127 for the largest product (P = 0: a field below that of
+    //        the smallest nonzero product); the division is a high multiply, inexact by 2^-30 at most, and P is never
+    //        closer than 1 / BASE to the next multiple;
     //   ca = |c|: field Exp(c) + 127.
     // Sum register: (1.5 * 2^23 + S) * 2^(e_max - F), exponent field e + (23 - F).
-    constexpr uint32_t MUL6 = 0x2AAAAAABu, T1_ADD = 107u << 23;
+    constexpr uint32_t MUL = pe_mul(BASE), T1_ADD = uint32_t(127 - (127 + pe_shift(BASE)) / BASE + 2 * PE_CENTER) << 23;
     constexpr uint32_t FIELD = 0x7F800000u, HALF = 0x00400000u;
     constexpr uint32_t MAGIC_ADD = (uint32_t(23 - F) << 23) | HALF;
     // Below E_LOW no product is nonzero, above E_HIGH the register would overflow (and every product is far below one
     // unit of the accumulator): the result is rho of the accumulator alone.  Such an output rides through pass 2 as a
     // marker KEEP + payload whose unit exceeds every product, so that a term changes it by -1 or not at all, which the
     // sign correction undoes.  FP16 accumulators are never out of range.
-    constexpr uint32_t E_LOW = ACC16 ? 0u : (115u << 23), E_HIGH = (241u << 23) - 1u;
+    const uint32_t E_LOW = ACC16 ? 0u : uint32_t(127 + 2 - fa.bias - fb.bias) << 23;
+    constexpr uint32_t E_HIGH = (241u << 23) - 1u;
     constexpr uint32_t E_KEEP = 243u << 23, KEEP = E_KEEP + MAGIC_ADD;
     static_assert(F == 13 || ACC16, "the kept word is carried as its upper 22 bits");
-    if (tid < 256) init_lut_t(sm, fa, fb, pre, guard, tid);
+    if (tid < 256) init_lut_t<BASE>(sm, fa, fb, pre, guard, tid);
     if (tid == 0) sm.special[0] = sm.special[1] = sm.special[2] = 0;
 
     uint32_t cw[TH][TW];
@@ -247,34 +271,54 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
                     }
             }
 
-            // ---- pass 1 on the tensor cores: P = sum_k pe(a_k) pe(b_k) for the warp's 32 x 32 outputs ----
-            float P[2][4][4];
+            // ---- pass 1 on the tensor cores: P = sum_k pe(a_k) pe(b_k) for the warp's 32 x 32 outputs, one
+            // accumulation per sub-block of KSUB terms, the block's P the integer maximum of their words ----
+            uint32_t P[2][4][4];
 #pragma unroll
-            for (int mt = 0; mt < 2; ++mt)
+            for (int sub = 0; sub < NSUB; ++sub) {
+                constexpr int NK = KSUB >= 16 ? KSUB / 16 : 1;             // matrix instructions per accumulation
+                constexpr int AR = KSUB >= 16 ? 4 : 2, BR = KSUB >= 16 ? 2 : 1;
+                uint32_t af[2][NK][AR], bf[4][NK][BR];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) { P[mt][j][0] = 0.f; P[mt][j][1] = 0.f; P[mt][j][2] = 0.f; P[mt][j][3] = 0.f; }
+                for (int ks = 0; ks < NK; ++ks) {
+                    const int kq = kb + sub * KSUB + 16 * ks + 2 * tq;
 #pragma unroll
-            for (int ks = 0; ks < L / 16; ++ks) {
-                const int kq = kb + 16 * ks + 2 * tq;
-                uint32_t bf[4][2];
+                    for (int j = 0; j < 4; ++j) {
+                        bf[j][ks][0] = *reinterpret_cast<const uint32_t*>(&s.b_pe[wc * 32 + 8 * j + gq][kq]);
+                        if (BR == 2) bf[j][ks][BR - 1] = *reinterpret_cast<const uint32_t*>(&s.b_pe[wc * 32 + 8 * j + gq][kq + 8]);
+                    }
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    bf[j][0] = *reinterpret_cast<const uint32_t*>(&s.b_pe[wc * 32 + 8 * j + gq][kq]);
-                    bf[j][1] = *reinterpret_cast<const uint32_t*>(&s.b_pe[wc * 32 + 8 * j + gq][kq + 8]);
+                    for (int mt = 0; mt < 2; ++mt) {
+                        const int ar = wr * 32 + 16 * mt + gq;
+                        af[mt][ks][0] = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar][kq]);
+                        af[mt][ks][1] = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar + 8][kq]);
+                        if (AR == 4) {
+                            af[mt][ks][AR - 2] = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar][kq + 8]);
+                            af[mt][ks][AR - 1] = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar + 8][kq + 8]);
+                        }
+                    }
                 }
 #pragma unroll
-                for (int mt = 0; mt < 2; ++mt) {
-                    const int ar = wr * 32 + 16 * mt + gq;
-                    const uint32_t a0 = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar][kq]);
-                    const uint32_t a1 = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar + 8][kq]);
-                    const uint32_t a2 = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar][kq + 8]);
-                    const uint32_t a3 = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar + 8][kq + 8]);
+                for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                                     : "+f"(P[mt][j][0]), "+f"(P[mt][j][1]), "+f"(P[mt][j][2]), "+f"(P[mt][j][3])
-                                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bf[j][0]), "r"(bf[j][1]));
-                }
+                    for (int j = 0; j < 4; ++j) {
+                        float d[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                        for (int ks = 0; ks < NK; ++ks) {
+                            if (KSUB >= 16)
+                                asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                             : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                                             : "r"(af[mt][ks][0]), "r"(af[mt][ks][1]), "r"(af[mt][ks][AR - 2]), "r"(af[mt][ks][AR - 1]),
+                                               "r"(bf[j][ks][0]), "r"(bf[j][ks][BR - 1]));
+                            else
+                                asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+                                             : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                                             : "r"(af[mt][ks][0]), "r"(af[mt][ks][1]), "r"(bf[j][ks][0]));
+                        }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            P[mt][j][i] = sub == 0 ? __float_as_uint(d[i]) : max(P[mt][j][i], __float_as_uint(d[i]));
+                    }
             }
             // e = max(exponent of the largest product, exponent of the accumulator), kept in the register of P
             uint32_t out_of_range = 0u;
@@ -282,19 +326,21 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
             for (int h = 0; h < TH; ++h)
 #pragma unroll
                 for (int x = 0; x < TW; ++x) {
-                    float& p = P[h >> 1][x >> 1][2 * (h & 1) + (x & 1)];
-                    const uint32_t t1 = __umulhi(__float_as_uint(p), MUL6) + T1_ADD;
+                    uint32_t& p = P[h >> 1][x >> 1][2 * (h & 1) + (x & 1)];
+                    const uint32_t t1 = __umulhi(p, MUL) + T1_ADD;
                     uint32_t e;
                     if (ACC16) {
-                        // a subnormal FP16 accumulator has the exponent -14, not that of its leading bit; the floor also
-                        // covers c = 0, harmlessly: every nonzero product has an exponent of at least -12
-                        const uint32_t ca = __float_as_uint(__half2float(__ushort_as_half((unsigned short)(cw[h][x] & 0x7FFFu))));
-                        e = uint32_t(__vimax3_s32(int(t1), int(ca), int(113u << 23)));
+                        // a subnormal FP16 accumulator has the exponent -14, not that of its leading bit.  BASE 6: the
+                        // floor also covers c = 0, harmlessly (every nonzero E4M3 product has an exponent of at least
+                        // -12); with E5M2 operands products reach down to 2^-28 and a zero accumulator must not count
+                        uint32_t ca = __float_as_uint(__half2float(__ushort_as_half((unsigned short)(cw[h][x] & 0x7FFFu))));
+                        if (BASE == 6) e = uint32_t(__vimax3_s32(int(t1), int(ca), int(113u << 23)));
+                        else { if (ca) ca = max(ca, 113u << 23); e = max(t1, ca); }
                     } else {
                         e = max(t1, cw[h][x] & 0x7FFFFFFFu);
                         out_of_range = __viaddmax_u32(e, 0u - E_LOW, out_of_range);
                     }
-                    p = __uint_as_float(e);
+                    p = e;
                 }
             const bool rare = !ACC16 && out_of_range > E_HIGH - E_LOW;
             if (rare) {                                    // turn the outputs out of range into markers (see above)
@@ -302,11 +348,11 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
                 for (int h = 0; h < TH; ++h)
 #pragma unroll
                     for (int x = 0; x < TW; ++x) {
-                        float& p = P[h >> 1][x >> 1][2 * (h & 1) + (x & 1)];
-                        if (__float_as_uint(p) - E_LOW > E_HIGH - E_LOW) {
+                        uint32_t& p = P[h >> 1][x >> 1][2 * (h & 1) + (x & 1)];
+                        if (p - E_LOW > E_HIGH - E_LOW) {
                             const uint32_t c = cw[h][x];
                             const uint32_t kept = (c & 0x7FFFFFFFu) ? (c >> 10) : 0u;      // rho(c); an exactly zero sum is +0
-                            p = __uint_as_float(E_KEEP);
+                            p = E_KEEP;
                             cw[h][x] = __float_as_uint(__uint2float_rn(kept) * __uint_as_float(uint32_t(E_KEEP >> 23) + uint32_t(23 - F) - 23u << 23));
                         }
                     }
@@ -316,7 +362,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
             for (int h = 0; h < TH; ++h)
 #pragma unroll
                 for (int x = 0; x < TW; ++x) {
-                    const uint32_t e = __float_as_uint(P[h >> 1][x >> 1][2 * (h & 1) + (x & 1)]);
+                    const uint32_t e = P[h >> 1][x >> 1][2 * (h & 1) + (x & 1)];
                     const uint32_t c = cw[h][x];
                     const uint32_t magic = (e & FIELD) + MAGIC_ADD + (c >> (ACC16 ? 15 : 31));
                     const float cf = ACC16 ? __half2float(__ushort_as_half((unsigned short)c)) : __uint_as_float(c);
@@ -432,20 +478,30 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
 #undef MMASIM_SP_WORD
 }
 
-template <int EK, int L, int F, int RHO, bool PROMOTE>
+template <int EK, int L, int F, int RHO, bool PROMOTE, int BASE>
 cudaError_t launch_one_t(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
     const size_t sh = sizeof(SmemT);
-    cudaError_t err = cudaFuncSetAttribute(tfdpa_trop_kernel<EK, L, F, RHO, PROMOTE>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
+    cudaError_t err = cudaFuncSetAttribute(tfdpa_trop_kernel<EK, L, F, RHO, PROMOTE, BASE>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
     if (err != cudaSuccess) return err;
     dim3 grid((unsigned)((g.N + BN - 1) / BN), (unsigned)((g.M + BM - 1) / BM), 1);
-    tfdpa_trop_kernel<EK, L, F, RHO, PROMOTE><<<grid, NT, sh, stream>>>(m, g);
+    tfdpa_trop_kernel<EK, L, F, RHO, PROMOTE, BASE><<<grid, NT, sh, stream>>>(m, g);
     return cudaGetLastError();
 }
 
-template <int EK, int L, int F, int RHO>
+// BASE by the exponent spread of the two element types (see pe_shift): both E4M3, one E5M2, both E5M2.
+template <int EK, int L, int F, int RHO, int BASE>
 cudaError_t launch_variant_t(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
-    if (RHO != RHO_RNE_FP16 && g.k_chunk) return launch_one_t<EK, L, F, RHO, RHO != RHO_RNE_FP16>(m, g, stream);
-    return launch_one_t<EK, L, F, RHO, false>(m, g, stream);
+    if (RHO != RHO_RNE_FP16 && g.k_chunk) return launch_one_t<EK, L, F, RHO, RHO != RHO_RNE_FP16, BASE>(m, g, stream);
+    return launch_one_t<EK, L, F, RHO, false, BASE>(m, g, stream);
+}
+
+template <int EK, int L, int F, int RHO>
+cudaError_t launch_by_types_t(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
+    const int wide = (m.fmt_a == EF_E5M2) + (m.fmt_b == EF_E5M2);
+    if ((m.fmt_a != EF_E4M3 && m.fmt_a != EF_E5M2) || (m.fmt_b != EF_E4M3 && m.fmt_b != EF_E5M2)) return cudaErrorInvalidValue;
+    if (wide == 0) return launch_variant_t<EK, L, F, RHO, 6>(m, g, stream);
+    if (wide == 1) return launch_variant_t<EK, L, F, RHO, 5>(m, g, stream);
+    return launch_variant_t<EK, L, F, RHO, 4>(m, g, stream);
 }
 
 }  // namespace trop
