@@ -260,7 +260,8 @@ def run_ours(args):
     # the multiply-add the timed kernel sums with (FP32 or FP64, rounded toward minus infinity)
     sink = torch.zeros(4, dtype=torch.int32, device=dev)
     peaks = {}
-    for kind in ("iadd3", "imad", "ffma.rm", "dfma"):
+    fma_kind = {"f32": "ffma.rm", "f64": "dfma"}.get(compute_dtype(kernel_name, model))
+    for kind in ("iadd3", "imad") + ((fma_kind,) if fma_kind else ()):
         best = 0.0
         mmasim.int_peak(kind, 148 * 8, 4096, sink)
         for _ in range(5):
@@ -316,7 +317,7 @@ def run_ours(args):
         h2d = hA.numel() * hA.element_size() + hB.numel() * hB.element_size() + hC.numel() * hC.element_size()
         e2e = {"value": macs_per_step / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                "d2h_bytes_per_step": int(hD.numel() * hD.element_size()), "ms_per_step": 1e3 * e2e_s,
-               "api": "mmasim_gemm_host (stream-ordered allocation + H2D + kernel + D2H + free per call)"}
+               "api": "mmasim_gemm_host (stream-ordered allocation, then row panels: H2D, kernel and D2H of different panels overlap; free; per call)"}
 
     if rank != 0:
         if dist is not None:
@@ -347,7 +348,7 @@ def run_ours(args):
                     "imad_peak": peaks["imad"] / 1e12}
         if dtype in ("f32", "f64") and model.family in ("t", "st", "tr", "gtr"):
             # the fused-summation kernels spend exactly one fused multiply-add per emulated MAC: that pipe is the bound
-            kind = "ffma.rm" if dtype == "f32" else "dfma"
+            kind = fma_kind
             roofline = {"bound": "alu", "achieved": per_gpu_macs_s / 1e12, "peak": peaks[kind] / 1e12, "unit": "Tfma/s",
                         "frac": per_gpu_macs_s / peaks[kind], "traffic": None, "kernel": kernel_name,
                         "algorithmic_fma_per_mac": 1.0,

@@ -232,10 +232,32 @@ int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
     void *dA = nullptr, *dB = nullptr, *dC = nullptr, *dD = nullptr, *dSA = nullptr, *dSB = nullptr, *dRS = nullptr, *dCS = nullptr;
     cudaError_t err = cudaSuccess;
     // Stream-ordered allocations on a stream of this call's own: after the first call the buffers come out of the
-    // device's default memory pool (which keeps up to 1 GiB between calls), copies from pinned host memory overlap
-    // nothing but also wait for nothing, and the call synchronises once, at the end.
-    cudaStream_t stream = nullptr;
-    err = cudaStreamCreateWithFlags(&stream, cudaStreamNonBlocking);
+    // device's default memory pool (which keeps up to 1 GiB between calls) and the call synchronises once, at the end.
+    // Large problems are cut into row panels of D (outputs are independent, Section 3.1 Step 1): B once, then per
+    // panel its rows of A and C in, the kernel, its rows of D out, on three streams chained by events, so that the
+    // copies of one panel run beside the arithmetic of another (two compute streams, so that a panel's last CTAs
+    // share the SMs with the next panel's first).
+    constexpr int MAX_PANELS = 16;
+    int panels = 1;
+    int64_t panel_rows = M;
+    if (M >= 1024 && a_bytes + b_bytes + c_bytes + d_bytes >= (size_t(32) << 20)) {
+        panel_rows = ((M + 7) / 8 + 127) / 128 * 128;              // about eight panels, whole CTA tiles each
+        if (panel_rows < 512) panel_rows = 512;
+        panels = int((M + panel_rows - 1) / panel_rows);
+        if (panels > MAX_PANELS) { panels = 1; panel_rows = M; }
+    }
+    cudaStream_t s_in = nullptr, s_k[2] = {nullptr, nullptr}, s_out = nullptr;
+    cudaEvent_t ev_in[MAX_PANELS] = {}, ev_k[MAX_PANELS] = {};
+    err = cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking);
+    if (err == cudaSuccess && panels > 1) {
+        err = cudaStreamCreateWithFlags(&s_k[0], cudaStreamNonBlocking);
+        if (err == cudaSuccess) err = cudaStreamCreateWithFlags(&s_k[1], cudaStreamNonBlocking);
+        if (err == cudaSuccess) err = cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking);
+        for (int p = 0; p < panels && err == cudaSuccess; ++p) {
+            err = cudaEventCreateWithFlags(&ev_in[p], cudaEventDisableTiming);
+            if (err == cudaSuccess) err = cudaEventCreateWithFlags(&ev_k[p], cudaEventDisableTiming);
+        }
+    }
     if (err == cudaSuccess) {
         int dev = 0;
         cudaMemPool_t pool = nullptr;
@@ -243,35 +265,78 @@ int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
         if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess)
             cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
     }
-    auto up = [&](void** dst, const void* src, size_t bytes) {
+    auto alloc = [&](void** dst, const void* src, size_t bytes) {
         if (err != cudaSuccess || !src || !bytes) return;
-        err = cudaMallocAsync(dst, bytes, stream);
-        if (err == cudaSuccess) err = cudaMemcpyAsync(*dst, src, bytes, cudaMemcpyHostToDevice, stream);
+        err = cudaMallocAsync(dst, bytes, s_in);
     };
-    up(&dA, A, a_bytes);
-    up(&dB, B, b_bytes);
-    up(&dC, C, c_bytes);
-    up(&dSA, g.sfa, sfa_bytes);
-    up(&dSB, g.sfb, sfb_bytes);
-    up(&dRS, g.row_scale, size_t(M) * 4);
-    up(&dCS, g.col_scale, size_t(N) * 4);
-    if (err == cudaSuccess) err = cudaMallocAsync(&dD, d_bytes, stream);
-    if (err == cudaSuccess) {
-        g.A = dA; g.B = dB; g.C = dC; g.D = dD;
-        g.sfa = static_cast<const uint8_t*>(dSA);
-        g.sfb = static_cast<const uint8_t*>(dSB);
-        g.row_scale = static_cast<const float*>(dRS);
-        g.col_scale = static_cast<const float*>(dCS);
-        st = run_gemm(model, g, opts ? opts->flags : 0, stream);
-        if (st == MMASIM_OK) err = cudaMemcpyAsync(D, dD, d_bytes, cudaMemcpyDeviceToHost, stream);
+    auto h2d = [&](void* dst, const void* src, size_t off, size_t bytes) {
+        if (err != cudaSuccess || !src || !bytes) return;
+        err = cudaMemcpyAsync(static_cast<unsigned char*>(dst) + off, static_cast<const unsigned char*>(src) + off, bytes,
+                              cudaMemcpyHostToDevice, s_in);
+    };
+    alloc(&dA, A, a_bytes);
+    alloc(&dB, B, b_bytes);
+    alloc(&dC, C, c_bytes);
+    alloc(&dSA, g.sfa, sfa_bytes);
+    alloc(&dSB, g.sfb, sfb_bytes);
+    alloc(&dRS, g.row_scale, size_t(M) * 4);
+    alloc(&dCS, g.col_scale, size_t(N) * 4);
+    alloc(&dD, D, d_bytes);
+    h2d(dB, B, 0, b_bytes);
+    h2d(dSB, g.sfb, 0, sfb_bytes);
+    h2d(dRS, g.row_scale, 0, size_t(M) * 4);
+    h2d(dCS, g.col_scale, 0, size_t(N) * 4);
+    const GemmArgs host = g;
+    for (int p = 0; p < panels && err == cudaSuccess && st == MMASIM_OK; ++p) {
+        const int64_t r0 = p * panel_rows, rows = (r0 + panel_rows <= M ? panel_rows : M - r0);
+        // byte ranges of the panel's rows (a row of packed 4-bit elements starts on a byte: leading dimensions are even)
+        const size_t a_off = size_t(r0 * host.lda) * info.a_bits / 8, a_len = size_t((rows - 1) * host.lda + K) * info.a_bits / 8;
+        const size_t c_off = size_t(r0 * host.ldc) * info.acc_bytes, c_len = size_t((rows - 1) * host.ldc + N) * info.acc_bytes;
+        const size_t d_off = size_t(r0 * host.ldd) * info.acc_bytes, d_len = size_t((rows - 1) * host.ldd + N) * info.acc_bytes;
+        h2d(dA, A, a_off, a_len);
+        h2d(dC, C, c_off, c_len);
+        h2d(dSA, host.sfa, size_t(r0 * host.ld_sfa), host.sfa ? size_t(rows * host.ld_sfa) : 0);
+        if (err != cudaSuccess) break;
+        cudaStream_t sk = panels > 1 ? s_k[p & 1] : s_in;
+        if (panels > 1) {
+            err = cudaEventRecord(ev_in[p], s_in);
+            if (err == cudaSuccess) err = cudaStreamWaitEvent(sk, ev_in[p], 0);
+            if (err != cudaSuccess) break;
+        }
+        GemmArgs q = host;
+        q.M = rows;
+        q.A = static_cast<const unsigned char*>(dA) + a_off;
+        q.B = dB;
+        q.C = dC ? static_cast<const unsigned char*>(dC) + c_off : nullptr;
+        q.D = static_cast<unsigned char*>(dD) + d_off;
+        q.sfa = dSA ? static_cast<const uint8_t*>(dSA) + r0 * host.ld_sfa : nullptr;
+        q.sfb = static_cast<const uint8_t*>(dSB);
+        q.row_scale = dRS ? static_cast<const float*>(dRS) + r0 : nullptr;
+        q.col_scale = static_cast<const float*>(dCS);
+        st = run_gemm(model, q, opts ? opts->flags : 0, sk);
+        if (st != MMASIM_OK) break;
+        cudaStream_t so = panels > 1 ? s_out : s_in;
+        if (panels > 1) {
+            err = cudaEventRecord(ev_k[p], sk);
+            if (err == cudaSuccess) err = cudaStreamWaitEvent(so, ev_k[p], 0);
+            if (err != cudaSuccess) break;
+        }
+        err = cudaMemcpyAsync(static_cast<unsigned char*>(D) + d_off, static_cast<unsigned char*>(dD) + d_off, d_len,
+                              cudaMemcpyDeviceToHost, so);
     }
-    if (stream) {
+    // everything drains, then the buffers go back to the pool in the order of the stream they came from
+    cudaStream_t all[] = {s_k[0], s_k[1], s_out};
+    for (cudaStream_t s : all)
+        if (s) { const cudaError_t e2 = cudaStreamSynchronize(s); if (err == cudaSuccess) err = e2; }
+    if (s_in) {
         void* bufs[] = {dA, dB, dC, dD, dSA, dSB, dRS, dCS};
-        for (void* b : bufs) if (b) cudaFreeAsync(b, stream);
-        const cudaError_t e2 = cudaStreamSynchronize(stream);
+        for (void* b : bufs) if (b) cudaFreeAsync(b, s_in);
+        const cudaError_t e2 = cudaStreamSynchronize(s_in);
         if (err == cudaSuccess) err = e2;
-        cudaStreamDestroy(stream);
     }
+    for (int p = 0; p < MAX_PANELS; ++p) { if (ev_in[p]) cudaEventDestroy(ev_in[p]); if (ev_k[p]) cudaEventDestroy(ev_k[p]); }
+    cudaStream_t streams[] = {s_in, s_k[0], s_k[1], s_out};
+    for (cudaStream_t s : streams) if (s) cudaStreamDestroy(s);
     if (err != cudaSuccess) {
         cudaGetLastError();
         set_error("mmasim_gemm_host: %s", cudaGetErrorString(err));

@@ -179,6 +179,25 @@ def test_host_entry_point_matches_device_entry_point():
     assert np.array_equal(got, want)
 
 
+@pytest.mark.parametrize("key, K", [(("hopper", "e4m3", "fp32"), 1024), (("blackwell", "mxe4m3", "fp32"), 512),
+                                    (("blackwell", "nvf4", "fp32"), 512), (("hopper", "fp16", "fp16"), 512)],
+                         ids=lambda k: "-".join(k) if isinstance(k, tuple) else str(k))
+def test_host_entry_point_in_row_panels(key, K):
+    # large enough for the panel pipeline of the host entry point (>= 1024 rows, >= 32 MiB), ragged last panel
+    from paper_2511_10909_b200 import mmasim
+    M, N = 4000 + 72, 3072
+    inp = wl.normal_inputs(key[1], key[2], M, N, K, seed=14)
+    model = mmasim.Model(*key)
+    kw = {}
+    if key[1] == "e4m3":
+        g = wl.rng(15)
+        kw = dict(k_chunk=128, row_scale=g.standard_normal(M).astype(np.float32), col_scale=g.standard_normal(N).astype(np.float32))
+    dkw = {k: (gu.dev(v) if isinstance(v, np.ndarray) else v) for k, v in kw.items()}
+    want = gu.run_gemm(key, inp, **dkw)
+    got = mmasim.gemm_host(model, inp["A"], inp["B"], inp["C"], sfa=inp.get("sfa"), sfb=inp.get("sfb"), **kw)
+    assert np.array_equal(got.view(want.dtype), want)
+
+
 def test_device_errors():
     from paper_2511_10909_b200 import mmasim
     model = mmasim.Model("hopper", "fp16", "fp32")
