@@ -58,7 +58,8 @@ bool fast_tfdpa_supported(const DevModel& m, const GemmArgs& g) {
     if (g.k_chunk % fast::KC) return false;
     if (kind == KIND_TR && g.k_chunk) return false;
     if (((g.lda * bytes) % 16) || ((g.ldb * bytes) % 16)) return false;      // 16-byte row starts for the vector loads
-    if (g.M > 65535ll * fast::BM) return false;
+    if (g.M > 65535ll * fast::BM) return false;                             // grid.y
+    if (g.N > 0x7FFFFFFFll - 128 || g.K > 0x7FFFFFFFll - 64) return false;   // 32-bit tile origins and k offsets in the kernels
     return true;
 }
 

@@ -41,7 +41,6 @@ namespace mmasim {
 namespace trop {
 
 using fast::BM;
-using fast::BN;
 using fast::KC;
 using fast::NT;
 using fast::CB;
@@ -60,7 +59,19 @@ constexpr int PE_CENTER = 1;            // pe(x) = 2^(6 (Exp(x) - PE_CENTER)); E
 __host__ __device__ constexpr int pe_shift(int base) { return base == 6 ? 5 : (base == 5 ? 3 : 1); }
 __host__ __device__ constexpr int pe_sub(int base) { return base == 6 ? 32 : (base == 5 ? 16 : 8); }
 __host__ __device__ constexpr uint32_t pe_mul(int base) { return base == 6 ? 0x2AAAAAABu : (base == 5 ? 0x33333334u : 0x40000000u); }  // ceil(2^32 / BASE)
-constexpr int TH = 4, TW = 8;           // micro-tile: 4 rows x 8 columns
+constexpr int TW = 8;                   // micro-tile: TH rows x 8 columns
+
+// Geometry by the height TH of the micro-tile.  TH = 4: warps 4 x 2, warp tile 32 x 32, CTA tile 128 x 64.
+// TH = 8: warps 2 x 4, warp tile 64 x 32, CTA tile 128 x 128 - sixteen operand words per 64 multiply-adds instead of
+// twelve per 32, at the price of 64 accumulator registers (used where nothing else has to live across the K loop).
+template <int TH>
+struct Geo {
+    static_assert(TH == 4 || TH == 8, "two or four accumulator fragments stacked");
+    static constexpr int WROWS = 8 * TH;                // rows of a warp tile
+    static constexpr int WARPS_R = BM / WROWS, WARPS_C = (NT / 32) / WARPS_R;
+    static constexpr int BN = 32 * WARPS_C;
+    static constexpr int NB = BN * KC / NT;             // elements of B staged per thread: 8 or 16
+};
 
 struct LutEntryT {      // 8 bytes: one shared load per staged element
     uint32_t op;        // staged FP32 operand
@@ -68,7 +79,9 @@ struct LutEntryT {      // 8 bytes: one shared load per staged element
                         // bit 16: sign; bit 24: finite and nonzero
 };
 
+template <int TH>
 struct PlanesT {
+    static constexpr int BN = Geo<TH>::BN;
     uint32_t a_op[KC][BM];              // [k][permuted row]
     uint32_t b_op[KC][BN];              // [k][permuted column]
     uint16_t a_pe[BM][PE_STRIDE];       // [row][k]
@@ -77,19 +90,24 @@ struct PlanesT {
     uint32_t b_sgn[BN], b_nz[BN];       // [permuted column]
 };
 
+template <int TH>
 struct SmemT {
-    PlanesT pl[2];
+    PlanesT<TH> pl[2];
     LutEntryT lut_a[256];
     LutEntryT lut_b[256];
     int special[3];
 };
 
-// Position of a row / column of the CTA tile inside the permuted planes.
-__device__ __forceinline__ int perm_row(int r) { return (r & ~31) | ((r & 7) << 2) | ((r >> 3) & 3); }
+// Position of a row / column of the CTA tile inside the permuted planes: the TH rows of a thread (g, g + 8, ...)
+// adjacent, its eight columns (8 j + 2 t, 8 j + 2 t + 1) contiguous.
+template <int TH>
+__device__ __forceinline__ int perm_row(int r) {
+    return TH == 4 ? ((r & ~31) | ((r & 7) << 2) | ((r >> 3) & 3)) : ((r & ~63) | ((r & 7) << 3) | ((r >> 3) & 7));
+}
 __device__ __forceinline__ int perm_col(int c) { return (c & ~31) | (((c >> 1) & 3) << 3) | (((c >> 3) & 3) << 1) | (c & 1); }
 
-template <int BASE>
-__device__ __forceinline__ void init_lut_t(SmemT& s, const FmtDesc& fa, const FmtDesc& fb, int pre, int guard, int tid) {
+template <int BASE, class SM>
+__device__ __forceinline__ void init_lut_t(SM& s, const FmtDesc& fa, const FmtDesc& fb, int pre, int guard, int tid) {
     const uint32_t da = decode_elem(fa, uint32_t(tid)), db = decode_elem(fb, uint32_t(tid));
     const bool fin_a = dec_cls(da) == CLS_FINITE, fin_b = dec_cls(db) == CLS_FINITE;
     const bool nz_a = fin_a && dec_sig(da) != 0u, nz_b = fin_b && dec_sig(db) != 0u;
@@ -108,31 +126,42 @@ __device__ __forceinline__ void init_lut_t(SmemT& s, const FmtDesc& fa, const Fm
 }
 
 // Staging of one chunk of KC = 32 elements of K.  Every thread takes sixteen consecutive elements of one row of A (row
-// tid % 128, half tid / 128) and eight of one column of B (column tid % 64, quarter tid / 64): the same work for all, so
-// that nobody waits at the barrier.  The raw bytes are fetched one chunk ahead into registers.
+// tid % 128, half tid / 128) and eight or sixteen of one column of B (column tid % BN): the same work for all, so that
+// nobody waits at the barrier.  The raw bytes are fetched one chunk ahead into registers.
+template <int TH>
 struct RawT {
-    uint4 a;
-    uint2 b;
+    uint32_t a[4];
+    uint32_t b[Geo<TH>::NB / 4];
 };
-static_assert(BM == 128 && BN == 64 && KC == 32 && NT == 256, "the task split of the staging");
+static_assert(BM == 128 && KC == 32 && NT == 256, "the task split of the staging");
 
-template <int EK>
-__device__ __forceinline__ void load_chunk_t(RawT& raw, const GemmArgs& g, int64_t row0, int64_t col0, int64_t k0, int tid) {
+template <int EK, int TH>
+__device__ __forceinline__ void load_chunk_t(RawT<TH>& raw, const GemmArgs& g, int64_t row0, int64_t col0, int64_t k0, int tid) {
     static_assert(Elem<EK>::BYTES == 1, "8-bit elements");
-    const int64_t i = row0 + (tid & 127), j = col0 + (tid & 63);
-    raw.a = make_uint4(0u, 0u, 0u, 0u);
-    raw.b = make_uint2(0u, 0u);
-    if (i < g.M) raw.a = *reinterpret_cast<const uint4*>(static_cast<const unsigned char*>(g.A) + i * g.lda + k0 + 16 * (tid >> 7));
-    if (j < g.N) raw.b = *reinterpret_cast<const uint2*>(static_cast<const unsigned char*>(g.B) + j * g.ldb + k0 + 8 * (tid >> 6));
+    constexpr int BN = Geo<TH>::BN, NB = Geo<TH>::NB;
+    const int64_t i = row0 + (tid & 127), j = col0 + (tid % BN);
+    uint4 va = make_uint4(0u, 0u, 0u, 0u);
+    if (i < g.M) va = *reinterpret_cast<const uint4*>(static_cast<const unsigned char*>(g.A) + i * g.lda + k0 + 16 * (tid >> 7));
+    raw.a[0] = va.x; raw.a[1] = va.y; raw.a[2] = va.z; raw.a[3] = va.w;
+    const unsigned char* pb = static_cast<const unsigned char*>(g.B) + j * g.ldb + k0 + NB * (tid / BN);
+    if (NB == 8) {
+        uint2 vb = make_uint2(0u, 0u);
+        if (j < g.N) vb = *reinterpret_cast<const uint2*>(pb);
+        raw.b[0] = vb.x; raw.b[1] = vb.y;
+    } else {
+        uint4 vb = make_uint4(0u, 0u, 0u, 0u);
+        if (j < g.N) vb = *reinterpret_cast<const uint4*>(pb);
+        raw.b[0] = vb.x; raw.b[1] = vb.y; raw.b[NB / 4 - 2] = vb.z; raw.b[NB / 4 - 1] = vb.w;
+    }
 }
 
-// Sixteen (A) or eight (B) elements of one row: operands k-major, pe words row-major, sign / nonzero bits into the masks.
-template <int N, bool IS_A>
-__device__ __forceinline__ uint32_t stage_row(SmemT& sm, PlanesT& s, const uint32_t (&w)[N / 4], int r, int part) {
+// N = 16 or 8 elements of one row: operands k-major, pe words row-major, sign / nonzero bits into the masks.
+template <int N, bool IS_A, int TH>
+__device__ __forceinline__ uint32_t stage_row(SmemT<TH>& sm, PlanesT<TH>& s, const uint32_t (&w)[N / 4], int r, int part) {
     const LutEntryT* lut = IS_A ? sm.lut_a : sm.lut_b;
-    const int pr = IS_A ? perm_row(r) : perm_col(r);
+    const int pr = IS_A ? perm_row<TH>(r) : perm_col(r);
     uint32_t* op = IS_A ? &s.a_op[part * N][pr] : &s.b_op[part * N][pr];
-    constexpr int STRIDE = IS_A ? BM : BN;
+    constexpr int STRIDE = IS_A ? BM : Geo<TH>::BN;
     uint32_t acc = 0u, spec = 0u, pw[N / 2];
 #pragma unroll
     for (int q = 0; q < N; q += 2) {
@@ -149,24 +178,27 @@ __device__ __forceinline__ uint32_t stage_row(SmemT& sm, PlanesT& s, const uint3
 #pragma unroll
     for (int q = 0; q < N / 8; ++q)
         reinterpret_cast<uint4*>(pe)[q] = make_uint4(pw[4 * q], pw[4 * q + 1], pw[4 * q + 2], pw[4 * q + 3]);
-    if (IS_A) {
-        reinterpret_cast<uint16_t*>(&s.a_sgn[pr])[part] = uint16_t(acc);
-        reinterpret_cast<uint16_t*>(&s.a_nz[pr])[part] = uint16_t(acc >> 16);
+    uint32_t* sgn = IS_A ? &s.a_sgn[pr] : &s.b_sgn[pr];
+    uint32_t* nz = IS_A ? &s.a_nz[pr] : &s.b_nz[pr];
+    if (N == 16) {
+        reinterpret_cast<uint16_t*>(sgn)[part] = uint16_t(acc);
+        reinterpret_cast<uint16_t*>(nz)[part] = uint16_t(acc >> 16);
     } else {
-        reinterpret_cast<uint8_t*>(&s.b_sgn[pr])[part] = uint8_t(acc);
-        reinterpret_cast<uint8_t*>(&s.b_nz[pr])[part] = uint8_t(acc >> 16);
+        reinterpret_cast<uint8_t*>(sgn)[part] = uint8_t(acc);
+        reinterpret_cast<uint8_t*>(nz)[part] = uint8_t(acc >> 16);
     }
     return spec;
 }
 
-__device__ __forceinline__ void store_chunk_t(SmemT& sm, PlanesT& s, const RawT& raw, int flag, int tid) {
-    const uint32_t wa[4] = {raw.a.x, raw.a.y, raw.a.z, raw.a.w};
-    const uint32_t wb[2] = {raw.b.x, raw.b.y};
-    const uint32_t spec = stage_row<16, true>(sm, s, wa, tid & 127, tid >> 7) | stage_row<8, false>(sm, s, wb, tid & 63, tid >> 6);
+template <int TH>
+__device__ __forceinline__ void store_chunk_t(SmemT<TH>& sm, PlanesT<TH>& s, const RawT<TH>& raw, int flag, int tid) {
+    constexpr int BN = Geo<TH>::BN, NB = Geo<TH>::NB;
+    const uint32_t spec = stage_row<16, true, TH>(sm, s, raw.a, tid & 127, tid >> 7) |
+                          stage_row<NB, false, TH>(sm, s, raw.b, tid % BN, tid / BN);
     if (spec & 0x8000u) atomicOr(&sm.special[flag], 1);
 }
 
-template <int EK, int L, int F, int RHO, bool PROMOTE, int BASE>
+template <int EK, int L, int F, int RHO, bool PROMOTE, int BASE, int TH>
 __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs g) {
     constexpr bool ACC16 = RHO == RHO_RNE_FP16;
     constexpr int NBLK = KC / L;
@@ -175,15 +207,18 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
     constexpr int KSUB = pe_sub(BASE) < L ? pe_sub(BASE) : L, NSUB = L / KSUB;        // terms per accumulation of P
     static_assert(!Elem<EK>::SIGNMAG && F <= 13, "8-bit inputs with F <= 13");
     static_assert(RHO == RHO_RZ_E8M13 || RHO == RHO_RNE_FP16, "rho of the F = 13 rows of Table 4");
+    using G = Geo<TH>;
+    constexpr int BN = G::BN;
+    using mask_t = std::conditional_t<(TH * TW > 32), unsigned long long, uint32_t>;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    SmemT& sm = *reinterpret_cast<SmemT*>(smem_raw);
+    SmemT<TH>& sm = *reinterpret_cast<SmemT<TH>*>(smem_raw);
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     const int gq = lane >> 2, tq = lane & 3;
-    const int64_t row0 = int64_t(blockIdx.y) * BM, col0 = int64_t(blockIdx.x) * BN;
-    const int wr = warp >> 1, wc = warp & 1;                                   // the warp's 32 x 32 part of the CTA tile
-    auto row_of = [&](int h) { return wr * 32 + gq + 8 * h; };                // inside the CTA tile
+    const int row0 = int(blockIdx.y) * BM, col0 = int(blockIdx.x) * BN;        // M, N < 2^31 (checked by the dispatcher)
+    const int wr = warp / G::WARPS_C, wc = warp % G::WARPS_C;                  // the warp's part of the CTA tile
+    auto row_of = [&](int h) { return wr * G::WROWS + 16 * (h >> 1) + 8 * (h & 1) + gq; };    // inside the CTA tile
     auto col_of = [&](int x) { return wc * 32 + 8 * (x >> 1) + 2 * tq + (x & 1); };
     const FmtDesc fa = fmt_desc(m.fmt_a), fb = fmt_desc(m.fmt_b);
     const int pre = F - (fa.mbits + fb.mbits);
@@ -209,9 +244,9 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
     if (tid == 0) sm.special[0] = sm.special[1] = sm.special[2] = 0;
 
     uint32_t cw[TH][TW];
-    uint32_t sp_nan = 0u, sp_pinf = 0u, sp_ninf = 0u;   // per output (bit h * TW + x)
+    mask_t sp_nan = 0, sp_pinf = 0, sp_ninf = 0;        // per output (bit h * TW + x)
     float promoted[PROMOTE ? TH : 1][PROMOTE ? TW : 1];
-#define MMASIM_SP_GET(h, x) ((((sp_nan >> ((h) * TW + (x))) & 1u)) | (((sp_pinf >> ((h) * TW + (x))) & 1u) << 1) | (((sp_ninf >> ((h) * TW + (x))) & 1u) << 2))
+#define MMASIM_SP_GET(h, x) (uint32_t((sp_nan >> ((h) * TW + (x))) & 1u) | (uint32_t((sp_pinf >> ((h) * TW + (x))) & 1u) << 1) | (uint32_t((sp_ninf >> ((h) * TW + (x))) & 1u) << 2))
 #define MMASIM_SP_WORD(h, x, w) (MMASIM_SP_GET(h, x) ? special_word(((MMASIM_SP_GET(h, x) & 1u) || (MMASIM_SP_GET(h, x) & 6u) == 6u) ? 1 : ((MMASIM_SP_GET(h, x) & 2u) ? 2 : 3), ACC16, true) : (w))
 #pragma unroll
     for (int h = 0; h < TH; ++h)
@@ -225,27 +260,28 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
             if (PROMOTE) { promoted[PROMOTE ? h : 0][PROMOTE ? x : 0] = __uint_as_float(w); w = 0u; }
             const AccDec d = decode_acc(w, ACC16);
             if (d.cls != CLS_FINITE) {
-                const uint32_t bit = 1u << (h * TW + x);
+                const mask_t bit = mask_t(1) << (h * TW + x);
                 if (d.cls == CLS_NAN) sp_nan |= bit; else if (d.sign) sp_ninf |= bit; else sp_pinf |= bit;
                 w = 0u;
             }
             cw[h][x] = w;
         }
 
-    RawT raw;
-    load_chunk_t<EK>(raw, g, row0, col0, 0, tid);
+    RawT<TH> raw;
+    load_chunk_t<EK, TH>(raw, g, row0, col0, 0, tid);
     __syncthreads();                                       // tables and flags are ready
-    store_chunk_t(sm, sm.pl[0], raw, 0, tid);
-    if (KC < g.K) load_chunk_t<EK>(raw, g, row0, col0, KC, tid);
+    store_chunk_t<TH>(sm, sm.pl[0], raw, 0, tid);
+    if (KC < g.K) load_chunk_t<EK, TH>(raw, g, row0, col0, KC, tid);
     __syncthreads();
     int chunk = 0;
-    for (int64_t k0 = 0; k0 < g.K; k0 += KC, ++chunk) {
+    const int K = int(g.K);
+    for (int k0 = 0; k0 < K; k0 += KC, ++chunk) {
         if (tid == 0) sm.special[(chunk + 2) % 3] = 0;
-        if (k0 + KC < g.K) {
-            store_chunk_t(sm, sm.pl[(chunk + 1) & 1], raw, (chunk + 1) % 3, tid);
-            if (k0 + 2 * KC < g.K) load_chunk_t<EK>(raw, g, row0, col0, k0 + 2 * KC, tid);
+        if (k0 + KC < K) {
+            store_chunk_t<TH>(sm, sm.pl[(chunk + 1) & 1], raw, (chunk + 1) % 3, tid);
+            if (k0 + 2 * KC < K) load_chunk_t<EK, TH>(raw, g, row0, col0, k0 + 2 * KC, tid);
         }
-        PlanesT& s = sm.pl[chunk & 1];
+        PlanesT<TH>& s = sm.pl[chunk & 1];
         const bool chunk_special = sm.special[chunk % 3] != 0;
 
 #pragma unroll 1
@@ -264,110 +300,115 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
                             const uint32_t yb = decode_elem(fb, raw_elem<EK>(g.B, j * g.ldb + k0 + kk));
                             ev.product(xa, yb);
                         }
-                        const uint32_t bit = 1u << (h * TW + x);
+                        const mask_t bit = mask_t(1) << (h * TW + x);
                         if (ev.nan) sp_nan |= bit;
                         if (ev.pinf) sp_pinf |= bit;
                         if (ev.ninf) sp_ninf |= bit;
                     }
             }
 
-            // ---- pass 1 on the tensor cores: P = sum_k pe(a_k) pe(b_k) for the warp's 32 x 32 outputs, one
-            // accumulation per sub-block of KSUB terms, the block's P the integer maximum of their words ----
-            uint32_t P[2][4][4];
+            // ---- pass 1 on the tensor cores: P = sum_k pe(a_k) pe(b_k), one accumulation per sub-block of KSUB terms,
+            // the block's P the integer maximum of their words; one accumulator fragment row (16 x 32 outputs of the
+            // warp, two rows of the micro-tile) at a time, followed at once by its sum registers ----
+            constexpr int NK = KSUB >= 16 ? KSUB / 16 : 1;                 // matrix instructions per accumulation
+            constexpr int AR = KSUB >= 16 ? 4 : 2, BR = KSUB >= 16 ? 2 : 1;
+            bool rare = false;
 #pragma unroll
-            for (int sub = 0; sub < NSUB; ++sub) {
-                constexpr int NK = KSUB >= 16 ? KSUB / 16 : 1;             // matrix instructions per accumulation
-                constexpr int AR = KSUB >= 16 ? 4 : 2, BR = KSUB >= 16 ? 2 : 1;
-                uint32_t af[2][NK][AR], bf[4][NK][BR];
+            for (int mt = 0; mt < TH / 2; ++mt) {
+                uint32_t P[4][4];
 #pragma unroll
-                for (int ks = 0; ks < NK; ++ks) {
-                    const int kq = kb + sub * KSUB + 16 * ks + 2 * tq;
+                for (int sub = 0; sub < NSUB; ++sub) {
+                    uint32_t af[NK][AR];
+                    const int ar = wr * G::WROWS + 16 * mt + gq;
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        bf[j][ks][0] = *reinterpret_cast<const uint32_t*>(&s.b_pe[wc * 32 + 8 * j + gq][kq]);
-                        if (BR == 2) bf[j][ks][BR - 1] = *reinterpret_cast<const uint32_t*>(&s.b_pe[wc * 32 + 8 * j + gq][kq + 8]);
-                    }
-#pragma unroll
-                    for (int mt = 0; mt < 2; ++mt) {
-                        const int ar = wr * 32 + 16 * mt + gq;
-                        af[mt][ks][0] = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar][kq]);
-                        af[mt][ks][1] = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar + 8][kq]);
+                    for (int ks = 0; ks < NK; ++ks) {
+                        const int kq = kb + sub * KSUB + 16 * ks + 2 * tq;
+                        af[ks][0] = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar][kq]);
+                        af[ks][1] = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar + 8][kq]);
                         if (AR == 4) {
-                            af[mt][ks][AR - 2] = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar][kq + 8]);
-                            af[mt][ks][AR - 1] = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar + 8][kq + 8]);
+                            af[ks][AR - 2] = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar][kq + 8]);
+                            af[ks][AR - 1] = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar + 8][kq + 8]);
                         }
                     }
-                }
-#pragma unroll
-                for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
+                        uint32_t bf[NK][BR];
+#pragma unroll
+                        for (int ks = 0; ks < NK; ++ks) {
+                            const int kq = kb + sub * KSUB + 16 * ks + 2 * tq;
+                            bf[ks][0] = *reinterpret_cast<const uint32_t*>(&s.b_pe[wc * 32 + 8 * j + gq][kq]);
+                            if (BR == 2) bf[ks][BR - 1] = *reinterpret_cast<const uint32_t*>(&s.b_pe[wc * 32 + 8 * j + gq][kq + 8]);
+                        }
                         float d[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                         for (int ks = 0; ks < NK; ++ks) {
                             if (KSUB >= 16)
                                 asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                                              : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                                             : "r"(af[mt][ks][0]), "r"(af[mt][ks][1]), "r"(af[mt][ks][AR - 2]), "r"(af[mt][ks][AR - 1]),
-                                               "r"(bf[j][ks][0]), "r"(bf[j][ks][BR - 1]));
+                                             : "r"(af[ks][0]), "r"(af[ks][1]), "r"(af[ks][AR - 2]), "r"(af[ks][AR - 1]),
+                                               "r"(bf[ks][0]), "r"(bf[ks][BR - 1]));
                             else
                                 asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
                                              : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                                             : "r"(af[mt][ks][0]), "r"(af[mt][ks][1]), "r"(bf[j][ks][0]));
+                                             : "r"(af[ks][0]), "r"(af[ks][1]), "r"(bf[ks][0]));
                         }
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
-                            P[mt][j][i] = sub == 0 ? __float_as_uint(d[i]) : max(P[mt][j][i], __float_as_uint(d[i]));
+                            P[j][i] = sub == 0 ? __float_as_uint(d[i]) : max(P[j][i], __float_as_uint(d[i]));
                     }
-            }
-            // e = max(exponent of the largest product, exponent of the accumulator), kept in the register of P
-            uint32_t out_of_range = 0u;
-#pragma unroll
-            for (int h = 0; h < TH; ++h)
-#pragma unroll
-                for (int x = 0; x < TW; ++x) {
-                    uint32_t& p = P[h >> 1][x >> 1][2 * (h & 1) + (x & 1)];
-                    const uint32_t t1 = __umulhi(p, MUL) + T1_ADD;
-                    uint32_t e;
-                    if (ACC16) {
-                        // a subnormal FP16 accumulator has the exponent -14, not that of its leading bit.  BASE 6: the
-                        // floor also covers c = 0, harmlessly (every nonzero E4M3 product has an exponent of at least
-                        // -12); with E5M2 operands products reach down to 2^-28 and a zero accumulator must not count
-                        uint32_t ca = __float_as_uint(__half2float(__ushort_as_half((unsigned short)(cw[h][x] & 0x7FFFu))));
-                        if (BASE == 6) e = uint32_t(__vimax3_s32(int(t1), int(ca), int(113u << 23)));
-                        else { if (ca) ca = max(ca, 113u << 23); e = max(t1, ca); }
-                    } else {
-                        e = max(t1, cw[h][x] & 0x7FFFFFFFu);
-                        out_of_range = __viaddmax_u32(e, 0u - E_LOW, out_of_range);
-                    }
-                    p = e;
                 }
-            const bool rare = !ACC16 && out_of_range > E_HIGH - E_LOW;
-            if (rare) {                                    // turn the outputs out of range into markers (see above)
+                // e = max(exponent of the largest product, exponent of the accumulator), kept in the register of P
+                uint32_t out_of_range = 0u;
 #pragma unroll
-                for (int h = 0; h < TH; ++h)
+                for (int hh = 0; hh < 2; ++hh)
 #pragma unroll
                     for (int x = 0; x < TW; ++x) {
-                        uint32_t& p = P[h >> 1][x >> 1][2 * (h & 1) + (x & 1)];
-                        if (p - E_LOW > E_HIGH - E_LOW) {
-                            const uint32_t c = cw[h][x];
-                            const uint32_t kept = (c & 0x7FFFFFFFu) ? (c >> 10) : 0u;      // rho(c); an exactly zero sum is +0
-                            p = E_KEEP;
-                            cw[h][x] = __float_as_uint(__uint2float_rn(kept) * __uint_as_float(uint32_t(E_KEEP >> 23) + uint32_t(23 - F) - 23u << 23));
+                        const int h = 2 * mt + hh;
+                        uint32_t& p = P[x >> 1][2 * hh + (x & 1)];
+                        const uint32_t t1 = __umulhi(p, MUL) + T1_ADD;
+                        uint32_t e;
+                        if (ACC16) {
+                            // a subnormal FP16 accumulator has the exponent -14, not that of its leading bit.  BASE 6: the
+                            // floor also covers c = 0, harmlessly (every nonzero E4M3 product has an exponent of at least
+                            // -12); with E5M2 operands products reach down to 2^-28 and a zero accumulator must not count
+                            uint32_t ca = __float_as_uint(__half2float(__ushort_as_half((unsigned short)(cw[h][x] & 0x7FFFu))));
+                            if (BASE == 6) e = uint32_t(__vimax3_s32(int(t1), int(ca), int(113u << 23)));
+                            else { if (ca) ca = max(ca, 113u << 23); e = max(t1, ca); }
+                        } else {
+                            e = max(t1, cw[h][x] & 0x7FFFFFFFu);
+                            out_of_range = __viaddmax_u32(e, 0u - E_LOW, out_of_range);
                         }
+                        p = e;
+                    }
+                if (!ACC16 && out_of_range > E_HIGH - E_LOW) {     // rare: turn the outputs out of range into markers (see above)
+                    rare = true;
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+                        for (int x = 0; x < TW; ++x) {
+                            const int h = 2 * mt + hh;
+                            uint32_t& p = P[x >> 1][2 * hh + (x & 1)];
+                            if (p - E_LOW > E_HIGH - E_LOW) {
+                                const uint32_t c = cw[h][x];
+                                const uint32_t kept = (c & 0x7FFFFFFFu) ? (c >> 10) : 0u;      // rho(c); an exactly zero sum is +0
+                                p = E_KEEP;
+                                cw[h][x] = __float_as_uint(__uint2float_rn(kept) * __uint_as_float(uint32_t(E_KEEP >> 23) + uint32_t(23 - F) - 23u << 23));
+                            }
+                        }
+                }
+                // the sum register with the accumulator term: floor((c + tiny) / unit); a negative c is one short
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+                    for (int x = 0; x < TW; ++x) {
+                        const int h = 2 * mt + hh;
+                        const uint32_t e = P[x >> 1][2 * hh + (x & 1)];
+                        const uint32_t c = cw[h][x];
+                        const uint32_t magic = (e & FIELD) + MAGIC_ADD + (c >> (ACC16 ? 15 : 31));
+                        const float cf = ACC16 ? __half2float(__ushort_as_half((unsigned short)c)) : __uint_as_float(c);
+                        cw[h][x] = __float_as_uint(__fadd_rd(__uint_as_float(__float_as_uint(cf) | 1u), __uint_as_float(magic)));
                     }
             }
-            // ---- the sum register with the accumulator term: floor((c + tiny) / unit); a negative c is one short ----
-#pragma unroll
-            for (int h = 0; h < TH; ++h)
-#pragma unroll
-                for (int x = 0; x < TW; ++x) {
-                    const uint32_t e = P[h >> 1][x >> 1][2 * (h & 1) + (x & 1)];
-                    const uint32_t c = cw[h][x];
-                    const uint32_t magic = (e & FIELD) + MAGIC_ADD + (c >> (ACC16 ? 15 : 31));
-                    const float cf = ACC16 ? __half2float(__ushort_as_half((unsigned short)c)) : __uint_as_float(c);
-                    cw[h][x] = __float_as_uint(__fadd_rd(__uint_as_float(__float_as_uint(cf) | 1u), __uint_as_float(magic)));
-                }
             // ---- pass 2: one fused multiply-add per term, rounding toward minus infinity onto the grid of S; two
             // columns of the micro-tile per instruction (fma.rm.f32x2: lanes (a_h, a_h) x (b_x, b_x+1) + (S_h,x, S_h,x+1)) ----
             {
@@ -379,10 +420,14 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
                         asm("mov.b64 %0, {%1, %2};" : "=l"(acc[h][xp]) : "r"(cw[h][2 * xp]), "r"(cw[h][2 * xp + 1]));
 #pragma unroll
                 for (int kk = kb; kk < kb + L; ++kk) {
-                    const float4 oa = *reinterpret_cast<const float4*>(&s.a_op[kk][wr * 32 + 4 * gq]);
+                    float oas[TH];
+#pragma unroll
+                    for (int q = 0; q < TH / 4; ++q) {
+                        const float4 oa = *reinterpret_cast<const float4*>(&s.a_op[kk][wr * G::WROWS + TH * gq + 4 * q]);
+                        oas[4 * q] = oa.x; oas[4 * q + 1] = oa.y; oas[4 * q + 2] = oa.z; oas[4 * q + 3] = oa.w;
+                    }
                     const ulonglong2 ob0 = *reinterpret_cast<const ulonglong2*>(&s.b_op[kk][wc * 32 + 8 * tq]);
                     const ulonglong2 ob1 = *reinterpret_cast<const ulonglong2*>(&s.b_op[kk][wc * 32 + 8 * tq + 4]);
-                    const float oas[TH] = {oa.x, oa.y, oa.z, oa.w};
                     const unsigned long long obv[TW / 2] = {ob0.x, ob0.y, ob1.x, ob1.y};
 #pragma unroll
                     for (int h = 0; h < TH; ++h) {
@@ -413,8 +458,8 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
             auto finish = [&](auto with_markers) {
 #pragma unroll
                 for (int h = 0; h < TH; ++h) {
-                    const uint32_t sa = s.a_sgn[wr * 32 + 4 * gq + h];
-                    const uint32_t nza = s.a_nz[wr * 32 + 4 * gq + h] & kmask;
+                    const uint32_t sa = s.a_sgn[wr * G::WROWS + TH * gq + h];
+                    const uint32_t nza = s.a_nz[wr * G::WROWS + TH * gq + h] & kmask;
 #pragma unroll
                     for (int x = 0; x < TW; ++x) {
                         // every negative nonzero term fell one unit short: bits + count is (1.5 * 2^23 + S) * unit
@@ -435,14 +480,14 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
 #pragma unroll
                     for (int x = 0; x < TW; ++x)
                         if ((cw[h][x] & 0x7FFFu) == 0x7C00u) {
-                            const uint32_t bit = 1u << (h * TW + x);
+                            const mask_t bit = mask_t(1) << (h * TW + x);
                             if (!((sp_nan | sp_pinf | sp_ninf) & bit)) { if (cw[h][x] >> 15) sp_ninf |= bit; else sp_pinf |= bit; }
                             cw[h][x] = 0u;
                         }
             }
         }
         __syncthreads();                                   // the other buffer is complete, this one is free
-        if (PROMOTE && ((k0 + KC) % g.k_chunk) == 0) {     // FP32 promotion of the partial sum every k_chunk elements
+        if (PROMOTE && ((k0 + KC) % int(g.k_chunk)) == 0) {     // FP32 promotion of the partial sum every k_chunk elements
 #pragma unroll
             for (int h = 0; h < TH; ++h)
 #pragma unroll
@@ -453,7 +498,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
                     promoted[PROMOTE ? h : 0][PROMOTE ? x : 0] = v;
                     cw[h][x] = 0u;
                 }
-            sp_nan = sp_pinf = sp_ninf = 0u;
+            sp_nan = sp_pinf = sp_ninf = 0;
         }
     }
 
@@ -478,23 +523,28 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
 #undef MMASIM_SP_WORD
 }
 
-template <int EK, int L, int F, int RHO, bool PROMOTE, int BASE>
+template <int EK, int L, int F, int RHO, bool PROMOTE, int BASE, int TH>
 cudaError_t launch_one_t(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
-    const size_t sh = sizeof(SmemT);
-    cudaError_t err = cudaFuncSetAttribute(tfdpa_trop_kernel<EK, L, F, RHO, PROMOTE, BASE>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
+    const size_t sh = sizeof(SmemT<TH>);
+    cudaError_t err = cudaFuncSetAttribute(tfdpa_trop_kernel<EK, L, F, RHO, PROMOTE, BASE, TH>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
     if (err != cudaSuccess) return err;
-    dim3 grid((unsigned)((g.N + BN - 1) / BN), (unsigned)((g.M + BM - 1) / BM), 1);
-    tfdpa_trop_kernel<EK, L, F, RHO, PROMOTE, BASE><<<grid, NT, sh, stream>>>(m, g);
+    dim3 grid((unsigned)((g.N + Geo<TH>::BN - 1) / Geo<TH>::BN), (unsigned)((g.M + BM - 1) / BM), 1);
+    tfdpa_trop_kernel<EK, L, F, RHO, PROMOTE, BASE, TH><<<grid, NT, sh, stream>>>(m, g);
     return cudaGetLastError();
 }
 
-// BASE by the exponent spread of the two element types (see pe_shift): both E4M3, one E5M2, both E5M2.
+// The tall micro-tile where the registers allow it: FP32 accumulators without promoted partial sums beside them.
 template <int EK, int L, int F, int RHO, int BASE>
 cudaError_t launch_variant_t(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
-    if (RHO != RHO_RNE_FP16 && g.k_chunk) return launch_one_t<EK, L, F, RHO, RHO != RHO_RNE_FP16, BASE>(m, g, stream);
-    return launch_one_t<EK, L, F, RHO, false, BASE>(m, g, stream);
+    if constexpr (RHO == RHO_RNE_FP16) {
+        return launch_one_t<EK, L, F, RHO, false, BASE, 4>(m, g, stream);
+    } else {
+        if (g.k_chunk) return launch_one_t<EK, L, F, RHO, true, BASE, 4>(m, g, stream);
+        return launch_one_t<EK, L, F, RHO, false, BASE, 8>(m, g, stream);
+    }
 }
 
+// BASE by the exponent spread of the two element types (see pe_shift): both E4M3, one E5M2, both E5M2.
 template <int EK, int L, int F, int RHO>
 cudaError_t launch_by_types_t(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
     const int wide = (m.fmt_a == EF_E5M2) + (m.fmt_b == EF_E5M2);
