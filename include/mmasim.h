@@ -137,7 +137,7 @@ int mmasim_dot_batch(const mmasim_model* model, int64_t n, int64_t K,
  * The device buffers are stream-ordered allocations (cudaMallocAsync) on a stream of the call's own; the device's
  * default memory pool is told to keep up to 1 GiB between calls, so repeated calls do not pay for allocation
  * (cudaMemPoolTrimTo on that pool returns the memory).  Pinned host buffers make the copies asynchronous.
- * Problems of 1024 rows and 32 MiB or more are cut into about eight row panels of D (outputs are independent,
+ * Problems of 1024 rows and 32 MiB or more are cut into up to eight row panels of D (outputs are independent,
  * Section 3.1 Step 1): B is copied once, then each panel's rows of A and C go in, its kernel runs and its rows of D
  * come back on separate streams, so that with pinned buffers the copies run beside the arithmetic. */
 int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,

@@ -233,7 +233,7 @@ int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
     cudaError_t err = cudaSuccess;
     // Stream-ordered allocations on a stream of this call's own: after the first call the buffers come out of the
     // device's default memory pool (which keeps up to 1 GiB between calls) and the call synchronises once, at the end.
-    // Large problems are cut into row panels of D (outputs are independent, Section 3.1 Step 1): B once, then per
+    // Large problems are cut into a few row panels of D (outputs are independent, Section 3.1 Step 1): B once, then per
     // panel its rows of A and C in, the kernel, its rows of D out, on three streams chained by events, so that the
     // copies of one panel run beside the arithmetic of another (two compute streams, so that a panel's last CTAs
     // share the SMs with the next panel's first).
@@ -241,7 +241,11 @@ int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
     int panels = 1;
     int64_t panel_rows = M;
     if (M >= 1024 && a_bytes + b_bytes + c_bytes + d_bytes >= (size_t(32) << 20)) {
-        panel_rows = ((M + 7) / 8 + 127) / 128 * 128;              // about eight panels, whole CTA tiles each
+        // whole CTA tiles, at most about eight panels, and at least 256 tiles of 128 x 128 per panel: with fewer a
+        // panel's kernel leaves most of the 296 CTA slots of the GPU empty
+        panel_rows = ((M + 7) / 8 + 127) / 128 * 128;
+        const int64_t fill_rows = 128 * ((256 + (N + 127) / 128 - 1) / ((N + 127) / 128));
+        if (panel_rows < fill_rows) panel_rows = fill_rows;
         if (panel_rows < 512) panel_rows = 512;
         panels = int((M + panel_rows - 1) / panel_rows);
         if (panels > MAX_PANELS) { panels = 1; panel_rows = M; }
