@@ -7,9 +7,11 @@
 //     register starts as the bare constant;
 //   * GTR-FDPA keeps two sums, of the even and of the odd elements, each with its own maximum exponent - the two
 //     16-bit lanes of the packed exponent pass are exactly these two maxima - and merges them with round-down.
-// What follows per block and output is integer work on T (read from the low word of the register): T and c are
-// aligned at E = max(e_max, Exp(c)) with round-down (arithmetic right shifts of two's-complement values) to F2 and
-// F fractional bits, with the "special truncation" of c in GTR-FDPA, and the sum is converted with RNE-FP32.
+// What follows per block and output works on T (read from the low word of the register): T and c are aligned at
+// E = max(e_max, Exp(c)) with round-down to F2 and F fractional bits - one fma.rd.f64 and one add.rd.f64 onto the
+// grids of 1.5 * 2^52 * 2^(E - F2) and 1.5 * 2^52 * 2^(E - F), every intermediate exact - with the "special
+// truncation" of c in GTR-FDPA, and the exact sum is converted with RNE-FP32 by one cvt.  The accumulator between
+// blocks is the output word itself.
 // A product of magnitude >= 2^128 is an infinity (Section 4.2): whenever a block's e_max could allow that, the thread
 // rescans the raw words of the block and records the event like any other infinity.  Zero products have no
 // exponent: a group without a nonzero product has T = 0 and an exponent lane that never wins a maximum.
@@ -25,66 +27,9 @@ using fast::EK_F16;
 using fast::EK_BF16;
 using fast::EK_TF32;
 
-struct TrAcc {
-    int cs;     // signed 24-bit significand (two's complement): value = cs * 2^(ce - CB - 23)
-    int ce;     // Exp(c) + CB; 0 for c = 0
-};
-
-__device__ __forceinline__ TrAcc tr_from_word(uint32_t w, uint32_t& sp) {
-    const AccDec d = decode_acc(w, false);
-    TrAcc a;
-    if (d.cls != CLS_FINITE) {
-        sp |= (d.cls == CLS_NAN) ? 1u : (d.sign ? 4u : 2u);
-        a.cs = 0;
-        a.ce = 0;
-        return a;
-    }
-    a.cs = d.sign ? -int(d.sig) : int(d.sig);
-    a.ce = d.sig ? d.exp + CB : 0;      // a zero accumulator has no exponent: 0 never decides E
-    return a;
-}
-
-__device__ __forceinline__ uint32_t tr_to_word(const TrAcc& a, uint32_t sp) {
-    if (sp) {
-        const int kind = ((sp & 1u) || (sp & 6u) == 6u) ? 1 : ((sp & 2u) ? 2 : 3);
-        return special_word(kind, false, false);
-    }
-    const uint32_t sign = a.cs < 0;
-    const uint32_t sig = uint32_t(abs(a.cs));
-    const uint32_t field = (sig >> 23) ? uint32_t(a.ce - CB + 127) : 0u;
-    return (sign << 31) | (field << 23) | (sig & 0x7FFFFFu);
-}
-
-__device__ __forceinline__ long long asr64_clamp(long long x, int d) { return x >> (d > 63 ? 63 : d); }
-
-// RNE-FP32 of S * 2^(eb - CB) for a 64-bit S when the result is a normal number or zero; otherwise (vmin / vmax leave
-// the normal range) the caller redoes the conversion with the generic routine.
-__device__ __forceinline__ void rne32_fast(long long S, int eb, TrAcc& a, int& vmin, int& vmax) {
-    const long long sg = S >> 63;
-    const unsigned long long mag = (unsigned long long)((S ^ sg) - sg);
-    const int msb = 63 - __clzll((long long)mag);                   // -1 for zero
-    const unsigned long long norm = msb >= 0 ? (mag << (63 - msb)) : 0ull;
-    const unsigned long long n2 = norm >> 1;                        // leading one at bit 62; 24 bits kept, 39 dropped
-    const unsigned long long r = (n2 + (((1ull << 38) - 1ull) + ((n2 >> 39) & 1ull))) >> 39;
-    const int carry = int(r >> 24);
-    const int sig = int(r >> carry);
-    int ve = eb + msb + carry;
-    ve = mag ? ve : -126 + CB;
-    vmin = min(vmin, ve);
-    vmax = max(vmax, ve);
-    a.ce = mag ? ve : 0;
-    a.cs = sg ? -sig : sig;
-}
-
-__device__ __noinline__ void rne32_slow(long long S, int e, TrAcc& a, uint32_t& sp) {
-    const uint32_t w = rho_apply(RHO_RNE_FP32, S, e);
-    a = tr_from_word(w, sp);
-}
-
 template <int EK, int L, bool GTR>
 __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g) {
     constexpr int NBLK = KC / L;
-    constexpr int EMINB = -126 + CB, EMAXB = 127 + CB;
     static_assert(KC % L == 0 && L % 2 == 0, "blocks tile the chunk; the exponent pass handles pairs of elements");
     using SM = Smem64<EK>;
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -103,8 +48,8 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
     init_lut64<EK>(sm, fa, fb, tid);
     if (tid == 0) sm.special[0] = sm.special[1] = sm.special[2] = 0;
 
-    TrAcc acc[TM][TN];
-    uint32_t sp_nan = 0u, sp_pinf = 0u, sp_ninf = 0u;
+    uint32_t cw[TM][TN];                                // the accumulator of each output: a finite FP32 word
+    uint32_t sp_nan = 0u, sp_pinf = 0u, sp_ninf = 0u;   // per output (bit r * TN + c): NaN / +inf / -inf seen so far
 #pragma unroll
     for (int r = 0; r < TM; ++r)
 #pragma unroll
@@ -112,11 +57,13 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
             const int64_t i = row0 + ty * TM + r, j = col0 + col_of(tx, c);
             uint32_t w = 0u;
             if (g.C && i < g.M && j < g.N) w = static_cast<const uint32_t*>(g.C)[i * g.ldc + j];
-            uint32_t ev = 0u;
-            acc[r][c] = tr_from_word(w, ev);
-            sp_nan |= (ev & 1u) << (r * TN + c);
-            sp_pinf |= ((ev >> 1) & 1u) << (r * TN + c);
-            sp_ninf |= ((ev >> 2) & 1u) << (r * TN + c);
+            const AccDec d = decode_acc(w, false);
+            if (d.cls != CLS_FINITE) {
+                const uint32_t bit = 1u << (r * TN + c);
+                if (d.cls == CLS_NAN) sp_nan |= bit; else if (d.sign) sp_ninf |= bit; else sp_pinf |= bit;
+                w = 0u;
+            }
+            cw[r][c] = w;
         }
 
     RawChunk<EK> raw;
@@ -227,8 +174,14 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
                         }
                 }
             }
-            // ---- merge, add the accumulator at E = max(e_max, Exp(c)) with round-down, RNE-FP32 ----
+            // ---- merge (Algorithm 10 Step 3 / Algorithm 11 Step 4) in FP64, where every quantity is exact:
+            //   E = max(e_max, Exp(c));  T2 = floor(T 2^(e_max - F) / q2) q2 with q2 = 2^(E - F2): one fma.rd onto the
+            //   grid of 1.5 * 2^52 * q2;  sc2 = floor(c / q1) q1 with q1 = 2^(E - F): one add.rd onto 1.5 * 2^52 * q1;
+            //   their sum has at most 40 significant bits; RNE-FP32 is one conversion.  An overflow is rare and sticky:
+            //   the loop tracks the largest result word, the flags are set in a second pass. ----
             const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
+            constexpr int E_FLOOR = CB - 400;          // below every real exponent; keeps the scales inside FP64 when nothing is live
+            uint32_t wmax = 0u;
 #pragma unroll
             for (int r = 0; r < TM; ++r) {
                 const uint32_t sa = s.a_sgn[ty * TM + r], nza = s.a_nz[ty * TM + r] & kmask;
@@ -248,25 +201,31 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
                         T = __double2loint(t0[r][c]) + __popc(negm);
                         emaxb = (__double2hiint(t0[r][c]) >> 20) - MAGIC_E;
                     }
-                    const TrAcc a = acc[r][c];
-                    const int E = max(emaxb, a.ce);
-                    const long long T2 = asr64_clamp((long long)T << (F2 - F), E - emaxb);       // RD_F2
-                    long long sc2 = asr64_clamp((long long)a.cs << (F - 23), E - a.ce);           // RD_F
-                    if (GTR && a.ce < E - F - 1) sc2 = 0;                                         // special truncation
-                    const long long S = T2 + (sc2 << (F2 - F));
-                    int vmin = EMINB, vmax = EMINB;
-                    rne32_fast(S, E - F2, acc[r][c], vmin, vmax);
-                    if (vmin < EMINB || vmax > EMAXB) {
-                        // the result is subnormal or overflows: by the book
-                        uint32_t ev = 0u;
-                        rne32_slow(S, E - CB - F2, acc[r][c], ev);
-                        const uint32_t bit = 1u << (r * TN + c);
-                        if (ev && !((sp_nan | sp_pinf | sp_ninf) & bit)) {         // overflow to infinity
-                            if (ev & 2u) sp_pinf |= bit;
-                            if (ev & 4u) sp_ninf |= bit;
-                        }
-                    }
+                    const uint32_t w0 = cw[r][c];
+                    const uint32_t ca = w0 & 0x7FFFFFFFu;
+                    const int ecb = ca ? int(max(ca >> 23, 1u)) + (CB - 127) : 0;       // Exp(c) + CB; a zero accumulator has no exponent
+                    const int E = max(max(emaxb, ecb), E_FLOOR);
+                    const double scale_t = __hiloint2double((max(emaxb, E_FLOOR) - CB - F + 1023) << 20, 0);     // 2^(e_max - F)
+                    const double m2 = __hiloint2double(((E - CB - F2 + 52 + 1023) << 20) | 0x00080000, 0);         // 1.5 * 2^52 * q2
+                    const double m1 = __hiloint2double(((E - CB - F + 52 + 1023) << 20) | 0x00080000, 0);          // 1.5 * 2^52 * q1
+                    const double t2 = __dsub_rn(__fma_rd(double(T), scale_t, m2), m2);                             // RD_F2
+                    double sc2 = __dsub_rn(__dadd_rd(double(__uint_as_float(w0)), m1), m1);                        // RD_F
+                    if (GTR && ecb < E - F - 1) sc2 = 0.0;                                                         // special truncation
+                    const uint32_t w = __float_as_uint(__double2float_rn(__dadd_rn(t2, sc2)));                     // exact sum, then rho
+                    wmax = max(wmax, w & 0x7FFFFFFFu);
+                    cw[r][c] = w;
                 }
+            }
+            if (wmax >= 0x7F800000u) {                     // rare: RNE-FP32 overflowed: +-infinity from now on
+#pragma unroll
+                for (int r = 0; r < TM; ++r)
+#pragma unroll
+                    for (int c = 0; c < TN; ++c)
+                        if ((cw[r][c] & 0x7FFFFFFFu) == 0x7F800000u) {
+                            const uint32_t bit = 1u << (r * TN + c);
+                            if (!((sp_nan | sp_pinf | sp_ninf) & bit)) { if (cw[r][c] >> 31) sp_ninf |= bit; else sp_pinf |= bit; }
+                            cw[r][c] = 0u;
+                        }
             }
         }
     }
@@ -279,7 +238,7 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
             if (i >= g.M || j >= g.N) continue;
             const uint32_t bit = r * TN + c;
             const uint32_t spv = ((sp_nan >> bit) & 1u) | (((sp_pinf >> bit) & 1u) << 1) | (((sp_ninf >> bit) & 1u) << 2);
-            uint32_t w = tr_to_word(acc[r][c], spv);
+            uint32_t w = spv ? special_word(((spv & 1u) || (spv & 6u) == 6u) ? 1 : ((spv & 2u) ? 2 : 3), false, false) : cw[r][c];
             if (g.row_scale) {
                 float sc = __fmul_rn(g.row_scale[i], g.col_scale[j]);
                 if (sc != sc) sc = __uint_as_float(0x7FFFFFFFu);
