@@ -1,4 +1,4 @@
-// Dispatch to the tuned T-FDPA kernels (see mmasim_tfdpa_fast.cuh for the kernel itself).
+// Dispatch to the tuned FDPA kernels (T-, ST-, TR-, GTR- and E-FDPA; see mmasim_tfdpa_fast.cuh for what they share).
 #include "mmasim_tfdpa_fast.cuh"
 
 namespace mmasim {
@@ -7,10 +7,15 @@ namespace {
 
 bool is8(int f) { return f == EF_E4M3 || f == EF_E5M2 || f == EF_E3M2 || f == EF_E2M3 || f == EF_E2M1; }
 
-constexpr int KIND_TR = 100;
+constexpr int KIND_TR = 100, KIND_E = 101;
 
-// 0: no tuned kernel; KIND_TR: the TR-/GTR-FDPA kernel; otherwise 1 + element kind of the T-FDPA kernel
+// 0: no tuned kernel; KIND_TR: the TR-/GTR-FDPA kernel; KIND_E: the E-FDPA kernel; otherwise 1 + element kind of the
+// T-FDPA kernel
 int kind_of(const DevModel& m) {
+    if (m.family == FAM_E) {
+        const bool ok = m.fmt_a == m.fmt_b && m.acc == ACC_F32 && ((m.fmt_a == EF_F16 && m.L == 4) || (m.fmt_a == EF_BF16 && m.L == 2));
+        return ok ? KIND_E : 0;
+    }
     if (m.family == FAM_TR || m.family == FAM_GTR) {
         if (m.F != 24 || m.F2 != 31 || m.rho != RHO_RNE_FP32 || m.inner_round || m.acc != ACC_F32) return 0;
         if (m.family == FAM_GTR) return (is8(m.fmt_a) && is8(m.fmt_b) && m.L == 16) ? KIND_TR : 0;
@@ -56,7 +61,7 @@ bool fast_tfdpa_supported(const DevModel& m, const GemmArgs& g) {
     const int bytes = fmt_desc(m.fmt_a).storage_bits / 8;
     if (g.K % fast::KC) return false;
     if (g.k_chunk % fast::KC) return false;
-    if (kind == KIND_TR && g.k_chunk) return false;
+    if ((kind == KIND_TR || kind == KIND_E) && g.k_chunk) return false;
     if (((g.lda * bytes) % 16) || ((g.ldb * bytes) % 16)) return false;      // 16-byte row starts for the vector loads
     if (g.M > 65535ll * fast::BM) return false;                             // grid.y
     if (g.N > 0x7FFFFFFFll - 128 || g.K > 0x7FFFFFFFll - 64) return false;   // 32-bit tile origins and k offsets in the kernels
@@ -68,6 +73,9 @@ int launch_fast_tfdpa(const DevModel& m, const GemmArgs& g, cudaStream_t stream)
     if (kind_of(m) == KIND_TR) {
         set_kernel_name(m.family == FAM_GTR ? "gtrfdpa" : "trfdpa");
         err = fast::launch_tr(m, g, stream);
+    } else if (kind_of(m) == KIND_E) {
+        set_kernel_name("efdpa");
+        err = fast::launch_e(m, g, stream);
     } else switch (kind_of(m) - 1) {
         case fast::EK_LUT8: set_kernel_name("tfdpa_lut8"); err = fast::launch_lut8(m, g, stream); break;
         case fast::EK_F16: set_kernel_name("tfdpa_f16"); err = fast::launch_f16(m, g, stream); break;

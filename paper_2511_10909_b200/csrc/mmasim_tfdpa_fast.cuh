@@ -19,6 +19,7 @@
 //   mmasim_tfdpa_trop.cuh   F = 13, 8-bit inputs: FP32 registers, e_max on the tensor cores
 //   mmasim_tfdpa_f64.cuh    F >= 23 and ST-FDPA: FP64 registers, e_max by fused add-max on 16-bit lanes
 //   mmasim_trfdpa_f64.cu    TR- / GTR-FDPA: two FP64 registers per output (even and odd terms)
+//   mmasim_efdpa_f64.cu     E-FDPA: the exact sum as a chain of FP64 multiply-adds where it fits a window
 //
 // Exponents, where staged as integers, carry a bias of 512 per element (1024 per product / accumulator) so that they
 // are positive 16-bit lane values; a zero element, like a zero accumulator, has no exponent and is staged as the
@@ -65,6 +66,7 @@ cudaError_t launch_f16(const DevModel& m, const GemmArgs& g, cudaStream_t stream
 cudaError_t launch_bf16(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
 cudaError_t launch_tf32(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
 cudaError_t launch_tr(const DevModel& m, const GemmArgs& g, cudaStream_t stream);    // TR-/GTR-FDPA (mmasim_trfdpa_f64.cu)
+cudaError_t launch_e(const DevModel& m, const GemmArgs& g, cudaStream_t stream);     // E-FDPA (mmasim_efdpa_f64.cu)
 
 }  // namespace fast
 }  // namespace mmasim

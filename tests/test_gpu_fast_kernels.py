@@ -343,3 +343,30 @@ def test_gst_fdpa_group_scaled(key):
     inp["sfb"][3, 0] = 0x7F if key[1] == "nvf4" else 0xFF
     inp["C"] = g.standard_normal((M, N)).astype(np.float32).view(np.uint32)
     _check(key, inp, expect_kernel="gstfdpa")
+
+
+@pytest.mark.parametrize("key", [("cdna1", "fp16", "fp32"), ("cdna1", "bf16", "fp32")], ids=lambda k: "-".join(k))
+def test_e_fdpa_exact_sum(key):
+    # the exact sum in FP64 where the block fits its window, by the book elsewhere: ordinary values (ragged shape),
+    # random bit streams (NaN, infinities, subnormals, any exponent spread), zeros and cancelling products, and
+    # accumulators from the subnormal range to the overflow boundary
+    g = wl.rng(41)
+    inp = wl.normal_inputs(key[1], key[2], 130, 70, 96, seed=42)
+    _check(key, inp, expect_kernel="efdpa")
+    M, N, K = 96, 64, 64
+    A = g.integers(0, 1 << 16, (M, K), dtype=np.uint16)
+    B = g.integers(0, 1 << 16, (N, K), dtype=np.uint16)
+    C = g.integers(0, 1 << 32, (M, N), dtype=np.uint32)
+    _check(key, {"A": A, "B": B, "C": C}, expect_kernel="efdpa")
+    inp = wl.normal_inputs(key[1], key[2], M, N, K, seed=43)
+    A = inp["A"].copy()
+    A[:, 1::2] = inp["A"][:, 0::2] ^ 0x8000                # exact cancellation of neighbouring products in half the rows
+    Bm = inp["B"].copy()
+    Bm[:, 1::2] = inp["B"][:, 0::2]
+    A[M // 2:], Bm[N // 2:] = inp["A"][M // 2:], inp["B"][N // 2:]
+    A[g.random((M, K)) < 0.05] = 0                         # zeros: +0 and -0
+    A[g.random((M, K)) < 0.02] = 0x8000
+    field = g.choice(np.r_[0:4, 100:150, 250:255], (M, N)).astype(np.uint32)
+    C = ((g.integers(0, 2, (M, N)).astype(np.uint32) << 31) | (field << 23) | g.integers(0, 1 << 23, (M, N)).astype(np.uint32)).astype(np.uint32)
+    C[g.random((M, N)) < 0.1] = 0x80000000
+    _check(key, {"A": A, "B": Bm, "C": C}, expect_kernel="efdpa")
