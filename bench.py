@@ -379,7 +379,7 @@ def run_ours(args):
 
 def run_sweep(args):
     """Every registry row at size^3 (config 5 / the per-model headline): MAC/s per model, optional oracle check of
-    seeded sampled outputs, one JSON line per model into gpurun_out/ and a summary line on stdout."""
+    seeded sampled outputs, one JSON line per model into the output folder (--out-dir) and a summary line on stdout."""
     import torch
     import oracle
     from paper_2511_10909_b200.build import build
@@ -391,8 +391,9 @@ def run_sweep(args):
     keys = sorted(oracle.REGISTRY)
     if args.models:
         keys = [k for k in keys if "-".join(k) in args.models.split(",")]
-    os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
-    out_path = os.path.join(ROOT, "gpurun_out", f"sweep_{size}.jsonl")
+    out_dir = args.out_dir if os.path.isabs(args.out_dir) else os.path.join(ROOT, args.out_dir)
+    os.makedirs(out_dir, exist_ok=True)
+    out_path = os.path.join(out_dir, f"sweep_{size}.jsonl")
     cache = {}
     rows = []
 
@@ -458,6 +459,7 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="time every registry row at --size^3 (not the bench line)")
     ap.add_argument("--size", type=int, default=4096)
     ap.add_argument("--check", type=int, default=0, help="with --sweep: compare this many seeded sampled outputs per model with the oracle")
+    ap.add_argument("--out-dir", default="gpurun_out", help="with --sweep: folder of the per-model JSON lines")
     ap.add_argument("--models", default="", help="with --sweep: comma-separated arch-infmt-acc names (default: all)")
     args = ap.parse_args()
     if args.sweep:
