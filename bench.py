@@ -63,6 +63,12 @@ def compute_dtype(kernel: str, model) -> str:
             "dot_tfdpa": "f64", "dot_ftz": "f32", "ftz_addmul": "f32", "fma_f32": "f32", "fma_f64": "f64", "gstfdpa": "int32"}.get(kernel, "int64")
 
 
+# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of the
+# workload; command and figures in profiles/tfdpa_trop_hopper_e4m3_2048.md).  The kernels are bound by arithmetic:
+# this is context, 0.4 % of what the memory could move in the kernel's time.
+NCU_DRAM_BYTES = {"cfg3": 101593856 + 34110464, "cfg3_2k": 25592832 + 38656}
+
+
 def algorithmic_ops_per_mac(model) -> float:
     """Integer operations per emulated MAC of the T-FDPA family: multiply, exponent add, maximum, distance,
     shift, accumulate (6 per term) plus about 25 per block for the accumulator term, normalisation and rho."""
@@ -388,7 +394,7 @@ def run_ours(args):
             # the fused-summation kernels spend exactly one fused multiply-add per emulated MAC: that pipe is the bound
             kind = fma_kind
             roofline = {"bound": "alu", "achieved": per_gpu_macs_s / 1e12, "peak": peaks[kind] / 1e12, "unit": "Tfma/s",
-                        "frac": per_gpu_macs_s / peaks[kind], "traffic": None, "kernel": kernel_name,
+                        "frac": per_gpu_macs_s / peaks[kind], "traffic": NCU_DRAM_BYTES.get(name), "kernel": kernel_name,
                         "algorithmic_fma_per_mac": 1.0,
                         "peak_source": f"measured live: independent fused multiply-adds rounded toward minus infinity on all SMs "
                                        f"(mmasim_int_peak kind {kind})" +
