@@ -50,6 +50,10 @@ WORKLOADS = {
                              "probe-style batch: 2^20 independent dot products of length 32, FP16, eight seeded input classes (subnormals, cancellation, outliers, inf/NaN, bit streams); Hopper FP16->FP32 model via mmasim_dot_batch"),
     "cfg4_dot_cdna2_fp16": (("cdna2", "fp16", "fp32"), (1 << 20, 1, 32),
                             "probe-style batch: 2^20 independent dot products of length 32, FP16, eight seeded input classes; CDNA2 FP16 model (FTZ-AddMul, P=4) via mmasim_dot_batch"),
+    "cdna3_bf16_2k": (("cdna3", "bf16", "fp32"), (2048, 2048, 2048),
+                      "BF16 2048^3 N(0,1) inputs (reduced case for profiler captures); CDNA3 BF16 model (TR-FDPA, L=8, F=24, F2=31)"),
+    "cdna1_fp16_2k": (("cdna1", "fp16", "fp32"), (2048, 2048, 2048),
+                      "FP16 2048^3 N(0,1) inputs (reduced case for profiler captures); CDNA1 FP16 model (E-FDPA, L=4)"),
     "blackwell_e4m3": (("blackwell", "e4m3", "fp32"), (4096, 4096, 4096),
                        "FP8 E4M3 4096^3 N(0,1) inputs; Blackwell FP8->FP32 model (L=32, F=25, RZ-FP32)"),
 }
@@ -60,7 +64,7 @@ def compute_dtype(kernel: str, model) -> str:
     if kernel == "tfdpa_lut8" and model.F <= 13:
         return "f32"
     return {"tfdpa_lut8": "f64", "tfdpa_f16": "f64", "tfdpa_bf16": "f64", "tfdpa_tf32": "f64", "trfdpa": "f64", "gtrfdpa": "f64",
-            "dot_tfdpa": "f64", "dot_ftz": "f32", "ftz_addmul": "f32", "fma_f32": "f32", "fma_f64": "f64", "gstfdpa": "int32"}.get(kernel, "int64")
+            "efdpa": "f64", "dot_tfdpa": "f64", "dot_ftz": "f32", "ftz_addmul": "f32", "fma_f32": "f32", "fma_f64": "f64", "gstfdpa": "int32"}.get(kernel, "int64")
 
 
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of the
@@ -390,7 +394,7 @@ def run_ours(args):
                     "algorithmic_int_ops_per_mac": ops_per_mac,
                     "peak_source": "measured live: independent 3-input integer adds on all SMs (mmasim_int_peak kind iadd3)",
                     "imad_peak": peaks["imad"] / 1e12}
-        if dtype in ("f32", "f64") and model.family in ("t", "st", "tr", "gtr"):
+        if dtype in ("f32", "f64") and model.family in ("t", "st", "tr", "gtr", "e"):
             # the fused-summation kernels spend exactly one fused multiply-add per emulated MAC: that pipe is the bound
             kind = fma_kind
             roofline = {"bound": "alu", "achieved": per_gpu_macs_s / 1e12, "peak": peaks[kind] / 1e12, "unit": "Tfma/s",

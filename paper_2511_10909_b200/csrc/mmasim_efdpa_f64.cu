@@ -131,8 +131,9 @@ __global__ void __launch_bounds__(NT, 1) efdpa64_kernel(DevModel m, GemmArgs g) 
 #pragma unroll
                     for (int c = 0; c < TN; ++c) sum[r][c] = __fma_rn(av[r], bv[c], sum[r][c]);
             }
-            // ---- the window test, the rounding, and the by-the-book route for what does not fit ----
+            // ---- the window test and the rounding; what does not fit keeps its accumulator and is marked ----
             const uint32_t kmask = (((L == 32) ? 0u : (1u << L)) - 1u) << kb;
+            uint32_t slow = 0u;                                    // bit r * TN + c: this output goes by the book
 #pragma unroll
             for (int r = 0; r < TM; ++r) {
                 const uint32_t nza = s.a_nz[ty * TM + r];
@@ -147,13 +148,21 @@ __global__ void __launch_bounds__(NT, 1) efdpa64_kernel(DevModel m, GemmArgs g) 
                     const int top = ca ? max(hi + 2, ec + 1) : hi + 2;
                     const int low = ca ? min(lo - FRAC, ec - 23) : lo - FRAC;
                     const bool all_nonzero = (nza & s.b_nz[col_of(tx, c)] & kmask) == kmask;
-                    uint32_t w = __float_as_uint(__double2float_rn(sum[r][c]));
-                    if (chunk_special || !all_nonzero || ca >= 0x7F800000u || top - low > WINDOW) {
-                        const int64_t i = row0 + ty * TM + r, j = col0 + col_of(tx, c);
-                        w = (i < g.M && j < g.N) ? efdpa_by_the_book<EK, L>(m, g.A, g.B, i * g.lda + k0 + kb, j * g.ldb + k0 + kb, w0) : 0u;
-                    }
-                    cw[r][c] = w;
+                    const bool fits = !chunk_special && all_nonzero && ca < 0x7F800000u && top - low <= WINDOW;
+                    slow |= uint32_t(!fits) << (r * TN + c);
+                    cw[r][c] = fits ? __float_as_uint(__double2float_rn(sum[r][c])) : w0;
                 }
+            }
+            if (slow) {                                        // rare
+#pragma unroll
+                for (int r = 0; r < TM; ++r)
+#pragma unroll
+                    for (int c = 0; c < TN; ++c)
+                        if ((slow >> (r * TN + c)) & 1u) {
+                            const int64_t i = row0 + ty * TM + r, j = col0 + col_of(tx, c);
+                            cw[r][c] = (i < g.M && j < g.N)
+                                           ? efdpa_by_the_book<EK, L>(m, g.A, g.B, i * g.lda + k0 + kb, j * g.ldb + k0 + kb, cw[r][c]) : 0u;
+                        }
             }
         }
     }
