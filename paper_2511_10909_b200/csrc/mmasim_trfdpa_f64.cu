@@ -44,6 +44,7 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
     // high word of 1.5 * 2^52 * 2^(e_max - F) is (e_max + CB) * 2^20 + MAGIC_K
     const int MAGIC_E = 1023 + 52 - F - CB;
     const int MAGIC_K = (MAGIC_E << 20) | 0x00080000;
+    constexpr int E_FLOOR = CB - 400;
 
     init_lut64<EK>(sm, fa, fb, tid);
     if (tid == 0) sm.special[0] = sm.special[1] = sm.special[2] = 0;
@@ -98,12 +99,14 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
             for (int r = 0; r < TM; ++r)
 #pragma unroll
                 for (int c = 0; c < TN; ++c) {
+                    // a group without a nonzero product (lane 0) gets E_FLOOR, below every real exponent: its sum stays 0
+                    // and the constants derived from its register's exponent stay inside FP64
                     const int lo = int(emp[r][c] & 0xFFFFu), hi = int(emp[r][c] >> 16);
                     if (GTR) {
-                        t0[r][c] = __hiloint2double(lo * (1 << 20) + MAGIC_K, 0);
-                        t1[GTR ? r : 0][GTR ? c : 0] = __hiloint2double(hi * (1 << 20) + MAGIC_K, 0);
+                        t0[r][c] = __hiloint2double(max(lo, E_FLOOR) * (1 << 20) + MAGIC_K, 0);
+                        t1[GTR ? r : 0][GTR ? c : 0] = __hiloint2double(max(hi, E_FLOOR) * (1 << 20) + MAGIC_K, 0);
                     } else {
-                        t0[r][c] = __hiloint2double(max(lo, hi) * (1 << 20) + MAGIC_K, 0);
+                        t0[r][c] = __hiloint2double(__vimax3_s32(lo, hi, E_FLOOR) * (1 << 20) + MAGIC_K, 0);
                     }
                     emax_all = max(emax_all, max(lo, hi));
                 }
@@ -180,7 +183,10 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
             //   their sum has at most 40 significant bits; RNE-FP32 is one conversion.  An overflow is rare and sticky:
             //   the loop tracks the largest result word, the flags are set in a second pass. ----
             const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
-            constexpr int E_FLOOR = CB - 400;          // below every real exponent; keeps the scales inside FP64 when nothing is live
+            // exponents as the exponent fields of doubles, in place (bits 20..30 of the high word): x20 = (x + 1023) << 20
+            constexpr int EXPF = 0x7FF00000;
+            const int k_reg = (52 - F) << 20;              // a sum register's field is that of 2^e_max plus 52 - F
+            const int k_m2 = ((52 - F2) << 20) | 0x00080000, k_m1 = (F2 - F) << 20, k_st = F << 20, k_gtr = (F + 1) << 20;
             uint32_t wmax = 0u;
 #pragma unroll
             for (int r = 0; r < TM; ++r) {
@@ -188,30 +194,31 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
 #pragma unroll
                 for (int c = 0; c < TN; ++c) {
                     const uint32_t negm = (sa ^ s.b_sgn[col_of(tx, c)]) & nza & s.b_nz[col_of(tx, c)];
-                    // the low word of a sum register is T (two's complement, |T| < 2^31); its exponent field gives e_max + CB
-                    int T, emaxb;
+                    // the low word of a sum register is T (two's complement, |T| < 2^31), its exponent field gives e_max
+                    int T, t20;
                     if (GTR) {
                         const int te = __double2loint(t0[r][c]) + __popc(negm & 0x55555555u);
                         const int to = __double2loint(t1[GTR ? r : 0][GTR ? c : 0]) + __popc(negm & 0xAAAAAAAAu);
-                        const int ee = (__double2hiint(t0[r][c]) >> 20) - MAGIC_E;
-                        const int eo = (__double2hiint(t1[GTR ? r : 0][GTR ? c : 0]) >> 20) - MAGIC_E;
-                        emaxb = max(ee, eo);
-                        T = fast::asr_clamp(te, emaxb - ee) + fast::asr_clamp(to, emaxb - eo);      // RD_F of both group sums
+                        const int e20 = __double2hiint(t0[r][c]) & EXPF, o20 = __double2hiint(t1[GTR ? r : 0][GTR ? c : 0]) & EXPF;
+                        t20 = max(e20, o20);
+                        T = fast::asr_clamp(te, (t20 - e20) >> 20) + fast::asr_clamp(to, (t20 - o20) >> 20);      // RD_F of both group sums
                     } else {
                         T = __double2loint(t0[r][c]) + __popc(negm);
-                        emaxb = (__double2hiint(t0[r][c]) >> 20) - MAGIC_E;
+                        t20 = __double2hiint(t0[r][c]) & EXPF;
                     }
                     const uint32_t w0 = cw[r][c];
-                    const uint32_t ca = w0 & 0x7FFFFFFFu;
-                    const int ecb = ca ? int(max(ca >> 23, 1u)) + (CB - 127) : 0;       // Exp(c) + CB; a zero accumulator has no exponent
-                    const int E = max(max(emaxb, ecb), E_FLOOR);
-                    const double scale_t = __hiloint2double((max(emaxb, E_FLOOR) - CB - F + 1023) << 20, 0);     // 2^(e_max - F)
-                    const double m2 = __hiloint2double(((E - CB - F2 + 52 + 1023) << 20) | 0x00080000, 0);         // 1.5 * 2^52 * q2
-                    const double m1 = __hiloint2double(((E - CB - F + 52 + 1023) << 20) | 0x00080000, 0);          // 1.5 * 2^52 * q1
-                    const double t2 = __dsub_rn(__fma_rd(double(T), scale_t, m2), m2);                             // RD_F2
-                    double sc2 = __dsub_rn(__dadd_rd(double(__uint_as_float(w0)), m1), m1);                        // RD_F
-                    if (GTR && ecb < E - F - 1) sc2 = 0.0;                                                         // special truncation
-                    const uint32_t w = __float_as_uint(__double2float_rn(__dadd_rn(t2, sc2)));                     // exact sum, then rho
+                    const double cd = double(__uint_as_float(w0));
+                    int ec20 = max(__double2hiint(cd) & EXPF, (1023 - 126) << 20);      // a subnormal accumulator has the exponent -126
+                    if ((w0 & 0x7FFFFFFFu) == 0u) ec20 = 0;                             // a zero accumulator has none
+                    const int em20 = t20 - k_reg;                                       // e_max
+                    const int E20 = max(em20, ec20);                                    // E = max(e_max, Exp(c))
+                    const double scale_t = __hiloint2double(em20 - k_st, 0);            // 2^(e_max - F)
+                    const double m2 = __hiloint2double(E20 + k_m2, 0);                  // 1.5 * 2^52 * 2^(E - F2)
+                    const double m1 = __hiloint2double(E20 + k_m2 + k_m1, 0);           // 1.5 * 2^52 * 2^(E - F)
+                    const double t2 = __dsub_rn(__fma_rd(double(T), scale_t, m2), m2);  // RD_F2
+                    double sc2 = __dsub_rn(__dadd_rd(cd, m1), m1);                      // RD_F
+                    if (GTR && ec20 < E20 - k_gtr) sc2 = 0.0;                           // special truncation
+                    const uint32_t w = __float_as_uint(__double2float_rn(__dadd_rn(t2, sc2)));      // exact sum, then rho
                     wmax = max(wmax, w & 0x7FFFFFFFu);
                     cw[r][c] = w;
                 }
