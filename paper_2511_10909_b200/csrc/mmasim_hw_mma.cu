@@ -22,6 +22,9 @@ enum HwKind : int {
     HW_F64 = 6,         // m8n8k4    f64 <- f64 x f64 + f64
     HW_F16_F32_K8 = 7,  // m16n8k8   f32 <- f16 x f16 + f32
     HW_TF32_F32_K4 = 8, // m16n8k4   f32 <- tf32 x tf32 + f32
+    HW_E4M3_F16 = 9,    // m16n8k32  f16 <- e4m3 x e4m3 + f16
+    HW_E5M2_F16 = 10,   // m16n8k32  f16 <- e5m2 x e5m2 + f16
+    HW_E4M3_E5M2_F32 = 11,  // m16n8k32  f32 <- e4m3 x e5m2 + f32
     HW_COUNT
 };
 
@@ -36,6 +39,9 @@ __host__ __device__ inline HwShape hw_shape(int kind) {
         case HW_E5M2_F32: return {16, 32, 1, 4};
         case HW_F64: return {8, 4, 8, 8};
         case HW_F16_F32_K8: return {16, 8, 2, 4};
+        case HW_E4M3_F16: return {16, 32, 1, 2};
+        case HW_E5M2_F16: return {16, 32, 1, 2};
+        case HW_E4M3_E5M2_F32: return {16, 32, 1, 4};
         default: return {16, 4, 4, 4};      // HW_TF32_F32_K4
     }
 }
@@ -135,6 +141,15 @@ __global__ void __launch_bounds__(128) hw_mma_kernel(int64_t tiles, int64_t K, c
         else if (KIND == HW_E5M2_F32)
             asm volatile("mma.sync.aligned.m16n8k32.row.col.f32.e5m2.e5m2.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                          : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+        else if (KIND == HW_E4M3_F16)
+            asm volatile("mma.sync.aligned.m16n8k32.row.col.f16.e4m3.e4m3.f16 {%0,%1}, {%2,%3,%4,%5}, {%6,%7}, {%0,%1};"
+                         : "+r"(c[0]), "+r"(c[1]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+        else if (KIND == HW_E5M2_F16)
+            asm volatile("mma.sync.aligned.m16n8k32.row.col.f16.e5m2.e5m2.f16 {%0,%1}, {%2,%3,%4,%5}, {%6,%7}, {%0,%1};"
+                         : "+r"(c[0]), "+r"(c[1]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+        else if (KIND == HW_E4M3_E5M2_F32)
+            asm volatile("mma.sync.aligned.m16n8k32.row.col.f32.e4m3.e5m2.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                         : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
         else if (KIND == HW_F16_F32_K8)
             asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
                          : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(b[0]));
@@ -180,6 +195,9 @@ int launch_hw_mma(int kind, int64_t M, int64_t K, const void* A, const void* B, 
         case HW_E5M2_F32: err = launch_hw<HW_E5M2_F32>(tiles, K, A, B, C, D, stream); break;
         case HW_F64: err = launch_hw<HW_F64>(tiles, K, A, B, C, D, stream); break;
         case HW_F16_F32_K8: err = launch_hw<HW_F16_F32_K8>(tiles, K, A, B, C, D, stream); break;
+        case HW_E4M3_F16: err = launch_hw<HW_E4M3_F16>(tiles, K, A, B, C, D, stream); break;
+        case HW_E5M2_F16: err = launch_hw<HW_E5M2_F16>(tiles, K, A, B, C, D, stream); break;
+        case HW_E4M3_E5M2_F32: err = launch_hw<HW_E4M3_E5M2_F32>(tiles, K, A, B, C, D, stream); break;
         default: err = launch_hw<HW_TF32_F32_K4>(tiles, K, A, B, C, D, stream); break;
     }
     if (err != cudaSuccess) { set_error("mmasim_hw_mma launch failed: %s", cudaGetErrorString(err)); return MMASIM_ERR_CUDA; }

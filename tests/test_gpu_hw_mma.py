@@ -136,3 +136,52 @@ def test_fp8_mma_sync_is_the_fp16_row_in_two_blocks_plus_an_fp32_addition(fmt, K
         pairs = wl.sample_pairs(M, 8, 400, seed=97)
         want = oracle.phi_gemm_sampled(oracle.lookup("blackwell", "fp16", "fp32"), wide(A), wide(B), C, pairs, k_chunk=32)
         gu.assert_samples_equal(hw, want, pairs, f"hardware {fmt} K={K} {mode} against the oracle's composition")
+
+
+def test_fp8_mma_sync_with_mixed_operand_types():
+    """A in E4M3, B in E5M2: the same composition."""
+    from paper_2511_10909_b200 import explore
+    _needs_b200()
+    g = wl.rng(98)
+    M, K = 1 << 12, 64
+    for mode in ("normal", "bits"):
+        A = wl.normal_inputs("e4m3", "fp32", M, 8, K, seed=99)["A"]
+        B = wl.normal_inputs("e5m2", "fp32", M, 8, K, seed=100)["B"]
+        C = wl.normal_inputs("e4m3", "fp32", M, 8, K, seed=101)["C"]
+        if mode == "bits":
+            A = g.integers(0, 256, A.shape, dtype=np.uint8)
+            B = g.integers(0, 256, B.shape, dtype=np.uint8)
+            C = g.integers(0, 1 << 32, C.shape, dtype=np.uint64).astype(np.uint32)
+        hw = _run("e4m3_e5m2_f32", A, B, C)
+        D = gu.host_words(explore.b200_fp8_mma_sync("e4m3", gu.dev(A), gu.dev(B), gu.dev(C), b_fmt="e5m2"))
+        assert np.array_equal(hw, D), (mode, int((hw != D).sum()))
+
+
+@pytest.mark.parametrize("fmt", ["e4m3", "e5m2"])
+def test_fp8_mma_sync_with_fp16_accumulator(fmt):
+    """FP8 inputs, FP16 accumulator: the two blocks of 16 run through the Blackwell FP16 -> FP16 row (RNE-FP16 after each
+    block) from a +0 accumulator, and C is added by an IEEE FP16 addition (NaN as 0x7FFF)."""
+    from paper_2511_10909_b200 import explore, mmasim
+    _needs_b200()
+    g = wl.rng(102)
+    M, K = 1 << 12, 32
+    i1 = [k for k in range(32) if k % 4 in (0, 1)]
+    i2 = [k for k in range(32) if k % 4 in (2, 3)]
+    model = mmasim.Model("blackwell", "fp16", "fp16")
+    for mode in ("normal", "bits"):
+        A = wl.normal_inputs(fmt, "fp32", M, 8, K, seed=103)["A"]
+        B = wl.normal_inputs(fmt, "fp32", M, 8, K, seed=104)["B"]
+        C = (g.standard_normal((M, 8)) * 2.0 ** g.integers(-6, 6, (M, 8))).astype(np.float16).view(np.uint16)
+        if mode == "bits":
+            A = g.integers(0, 256, A.shape, dtype=np.uint8)
+            B = g.integers(0, 256, B.shape, dtype=np.uint8)
+            C = g.integers(0, 1 << 16, C.shape).astype(np.uint16)
+        hw = _run(fmt + "_f16", A, B, C)
+        A16, B16 = explore.widen_fp8_to_fp16(fmt, gu.dev(A)), explore.widen_fp8_to_fp16(fmt, gu.dev(B))
+        zero = torch.zeros((M, 8), dtype=torch.int16, device="cuda")
+        t1 = mmasim.gemm(model, A16[:, i1].contiguous(), B16[:, i1].contiguous(), zero)
+        t2 = mmasim.gemm(model, A16[:, i2].contiguous(), B16[:, i2].contiguous(), t1)
+        d = t2.view(torch.float16) + gu.dev(C).view(torch.float16)
+        D = gu.host_words(d.view(torch.int16)).copy()
+        D[np.isnan(D.view(np.float16))] = 0x7FFF
+        assert np.array_equal(hw, D), (fmt, mode, int((hw != D).sum()))
