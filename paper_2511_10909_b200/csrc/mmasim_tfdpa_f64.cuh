@@ -28,6 +28,7 @@
 // sticky flags and rescan of the raw words (Section 4.2): their staged operands are the zero stand-ins.
 #pragma once
 #include <cuda_fp16.h>
+#include <type_traits>
 #include "mmasim_tfdpa_fast.cuh"
 
 namespace mmasim {
@@ -292,21 +293,22 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
     if (KC < g.K) load_chunk<EK>(raw, g, row0, col0, KC, tid);
     __syncthreads();
     uint32_t emp[TM][TN];                               // product exponents of the block that comes next
-    product_exponents<L>(&sm.pl[0].a_exp2[0][ty * TM], &sm.pl[0].b_exp2[0][tx * 2], emp);
 
     int chunk = 0;
     for (int64_t k0 = 0; k0 < g.K; k0 += KC, ++chunk) {
         auto& s = sm.pl[chunk & 1];
         auto& nx = sm.pl[(chunk + 1) & 1];
-        // decode chunk n + 1 into the other buffer (its raw words arrived during the previous iteration), fetch n + 2
-        if (tid == 0) sm.special[(chunk + 2) % 3] = 0;  // last read a chunk ago, next written after the coming barrier
-        __syncthreads();                                // every warp has left the other buffer
+        // decode chunk n + 1 into the other buffer (its raw words arrived during the previous iteration; every warp left
+        // that buffer before the barrier that ended the previous iteration), fetch n + 2.  One barrier per chunk: the
+        // warps drift apart, and some decode while others keep the FP64 pipe busy.
+        if (tid == 0) sm.special[(chunk + 2) % 3] = 0;  // last read two barriers ago, next written after the coming one
         if (k0 + KC < g.K) {
             store_chunk64<EK>(sm, nx, raw, (chunk + 1) % 3, tid);
             if (k0 + 2 * KC < g.K) load_chunk<EK>(raw, g, row0, col0, k0 + 2 * KC, tid);
         }
-        __syncthreads();                                // the other buffer is complete
         const bool chunk_special = sm.special[chunk % 3] != 0;
+        // the first block's product exponents (the other blocks' are taken beside the multiply-adds of their predecessor)
+        product_exponents<L>(&s.a_exp2[0][ty * TM], &s.b_exp2[0][tx * 2], emp);
 
         // ST-FDPA (Algorithm 8): Exp(alpha) of this thread's rows and Exp(beta) of its columns for this block of 32
         int sa_exp[ST ? TM : 1], sb_exp[ST ? TN : 1];
@@ -377,18 +379,20 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
                     const long long bitsum = __double_as_longlong(a0) + (long long)(cw[r][c] >> (ACC16 ? 15 : 31));
                     acc[r][c] = __longlong_as_double(bitsum);
                 }
-            // ---- one fused multiply-add per term, rounding toward minus infinity onto the grid of q; beside it the
-            // product exponents of the block that follows (the next chunk's first block after this chunk's last) ----
-            {
+            // ---- one fused multiply-add per term, rounding toward minus infinity onto the grid of q; beside it, while
+            // the chunk has another block, the product exponents of that block ----
+            auto multiply_adds = [&](auto with_exponents) {
+                constexpr bool FUSE = decltype(with_exponents)::value;
                 const double* a_p = &s.a_d[kb][ty * TM];
                 const double* b_p = &s.b_d[kb][tx * 2];
-                const bool same = blk + 1 < NBLK;
-                const uint32_t* ea_p = same ? &s.a_exp2[(kb + L) / 2 < KC / 2 ? (kb + L) / 2 : 0][ty * TM] : &nx.a_exp2[0][ty * TM];
-                const uint32_t* eb_p = same ? &s.b_exp2[(kb + L) / 2 < KC / 2 ? (kb + L) / 2 : 0][tx * 2] : &nx.b_exp2[0][tx * 2];
+                const uint32_t* ea_p = &s.a_exp2[FUSE ? (kb + L) / 2 : 0][ty * TM];
+                const uint32_t* eb_p = &s.b_exp2[FUSE ? (kb + L) / 2 : 0][tx * 2];
+                if (FUSE) {
 #pragma unroll
-                for (int r = 0; r < TM; ++r)
+                    for (int r = 0; r < TM; ++r)
 #pragma unroll
-                    for (int c = 0; c < TN; ++c) emp[r][c] = 0u;
+                        for (int c = 0; c < TN; ++c) emp[r][c] = 0u;
+                }
 #pragma unroll
                 for (int kq = 0; kq < L; ++kq) {
                     double av[TM], bv[TN];
@@ -403,7 +407,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
                         bv[0] = t0.x; bv[1] = t0.y; bv[2] = t1.x; bv[3] = t1.y;
                     }
                     uint32_t ea[TM], ebv[TN];
-                    if ((kq & 1) == 0) {
+                    if (FUSE && (kq & 1) == 0) {
                         const int kp = kq / 2;
                         const uint4 ea0 = *reinterpret_cast<const uint4*>(ea_p + kp * BM);
                         const uint2 eb0 = *reinterpret_cast<const uint2*>(eb_p + kp * BN);
@@ -416,10 +420,11 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
 #pragma unroll
                         for (int c = 0; c < TN; ++c) {
                             acc[r][c] = __fma_rd(av[r], bv[c], acc[r][c]);
-                            if ((kq & 1) == 0) emp[r][c] = __viaddmax_s16x2(ea[r], ebv[c], emp[r][c]);
+                            if (FUSE && (kq & 1) == 0) emp[r][c] = __viaddmax_s16x2(ea[r], ebv[c], emp[r][c]);
                         }
                 }
-            }
+            };
+            if (NBLK > 1 && blk + 1 < NBLK) multiply_adds(std::true_type{}); else multiply_adds(std::false_type{});
             // ---- sign corrections, rho.  An overflow (|v| >= 2^128, or an FP16 result that rounds to infinity) is rare
             // and sticky: the loop only tracks the largest result word, the flags are set in a second pass ----
             const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
@@ -462,6 +467,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
                 }
             }
         }
+        __syncthreads();                                // the other buffer is complete, this one is free
         // ---- FP32 promotion of the partial sum every k_chunk elements ----
         if (PROMOTE && ((k0 + KC) % g.k_chunk) == 0) {
 #pragma unroll
