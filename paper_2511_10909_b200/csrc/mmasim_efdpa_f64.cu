@@ -75,13 +75,13 @@ __global__ void __launch_bounds__(NT, 1) efdpa64_kernel(DevModel m, GemmArgs g) 
     for (int64_t k0 = 0; k0 < g.K; k0 += KC, ++chunk) {
         auto& s = sm.pl[chunk & 1];
         auto& nx = sm.pl[(chunk + 1) & 1];
+        // one barrier per chunk, at its end: every warp left the other buffer before the barrier that ended the previous
+        // iteration, so it can be filled while slower warps still compute on this one
         if (tid == 0) sm.special[(chunk + 2) % 3] = 0;
-        __syncthreads();                                // every warp has left the other buffer
         if (k0 + KC < g.K) {
             store_chunk64<EK>(sm, nx, raw, (chunk + 1) % 3, tid);
             if (k0 + 2 * KC < g.K) load_chunk<EK>(raw, g, row0, col0, k0 + 2 * KC, tid);
         }
-        __syncthreads();                                // the other buffer is complete
         const bool chunk_special = sm.special[chunk % 3] != 0;
 
 #pragma unroll 1
@@ -165,6 +165,7 @@ __global__ void __launch_bounds__(NT, 1) efdpa64_kernel(DevModel m, GemmArgs g) 
                         }
             }
         }
+        __syncthreads();                                // the other buffer is complete, this one is free
     }
 
 #pragma unroll

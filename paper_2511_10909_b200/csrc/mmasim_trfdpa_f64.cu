@@ -74,20 +74,21 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
     if (KC < g.K) load_chunk<EK>(raw, g, row0, col0, KC, tid);
     __syncthreads();
     uint32_t emp[TM][TN];                               // product exponents of the block that comes next (low lane: even elements)
-    product_exponents<L>(&sm.pl[0].a_exp2[0][ty * TM], &sm.pl[0].b_exp2[0][tx * 2], emp);
 
     int chunk = 0;
     for (int64_t k0 = 0; k0 < g.K; k0 += KC, ++chunk) {
         auto& s = sm.pl[chunk & 1];
         auto& nx = sm.pl[(chunk + 1) & 1];
+        // one barrier per chunk, at its end: every warp left the other buffer before the barrier that ended the previous
+        // iteration, so it can be filled while slower warps still compute on this one
         if (tid == 0) sm.special[(chunk + 2) % 3] = 0;
-        __syncthreads();                                // every warp has left the other buffer
         if (k0 + KC < g.K) {
             store_chunk64<EK>(sm, nx, raw, (chunk + 1) % 3, tid);
             if (k0 + 2 * KC < g.K) load_chunk<EK>(raw, g, row0, col0, k0 + 2 * KC, tid);
         }
-        __syncthreads();                                // the other buffer is complete
         const bool chunk_special = sm.special[chunk % 3] != 0;
+        // the first block's product exponents (the other blocks' are taken beside the multiply-adds of their predecessor)
+        product_exponents<L>(&s.a_exp2[0][ty * TM], &s.b_exp2[0][tx * 2], emp);
 
 #pragma unroll 1
         for (int blk = 0; blk < NBLK; ++blk) {
@@ -138,9 +139,10 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
             {
                 const double* a_p = &s.a_d[kb][ty * TM];
                 const double* b_p = &s.b_d[kb][tx * 2];
-                const bool same = blk + 1 < NBLK;
-                const uint32_t* ea_p = same ? &s.a_exp2[(kb + L) / 2 < KC / 2 ? (kb + L) / 2 : 0][ty * TM] : &nx.a_exp2[0][ty * TM];
-                const uint32_t* eb_p = same ? &s.b_exp2[(kb + L) / 2 < KC / 2 ? (kb + L) / 2 : 0][tx * 2] : &nx.b_exp2[0][tx * 2];
+                // the next block of this chunk (after the chunk's last block the pass reads its first block again; that
+                // result is replaced at the start of the next chunk)
+                const uint32_t* ea_p = &s.a_exp2[(kb + L) / 2 < KC / 2 ? (kb + L) / 2 : 0][ty * TM];
+                const uint32_t* eb_p = &s.b_exp2[(kb + L) / 2 < KC / 2 ? (kb + L) / 2 : 0][tx * 2];
 #pragma unroll
                 for (int r = 0; r < TM; ++r)
 #pragma unroll
@@ -235,6 +237,7 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
                         }
             }
         }
+        __syncthreads();                                // the other buffer is complete, this one is free
     }
 
 #pragma unroll
