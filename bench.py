@@ -151,13 +151,16 @@ class ClockSampler:
     def _poll(self):
         n = self.nvml
         reasons_of = getattr(n, "nvmlDeviceGetCurrentClocksEventReasons", None) or n.nvmlDeviceGetCurrentClocksThrottleReasons
+        try:
+            mx = n.nvmlDeviceGetMaxClockInfo(self.handle, n.NVML_CLOCK_SM)
+        except Exception:
+            mx = 0
         while not self.stop_flag:
             try:
-                self.samples.append((n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM),
-                                     n.nvmlDeviceGetMaxClockInfo(self.handle, n.NVML_CLOCK_SM), int(reasons_of(self.handle))))
+                self.samples.append((n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM), mx, int(reasons_of(self.handle))))
             except Exception:
                 pass
-            time.sleep(0.004)
+            time.sleep(0.001)
 
     def _read(self):
         for line in self.proc.stdout:
