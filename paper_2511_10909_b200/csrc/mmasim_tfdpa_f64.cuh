@@ -371,13 +371,12 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
                     if (ST) rel -= sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0];
                     if ((cw[r][c] & (ACC16 ? 0x7FFFu : 0x7FFFFFFFu)) == 0u) rel = 0;       // c = 0 has no exponent
                     const int emax = __vimax3_s32(int(emp[r][c] & 0xFFFFu), int(emp[r][c] >> 16), rel);     // e_max + CB
-                    const double magic = __hiloint2double(emax * (1 << 20) + MAGIC_K, 0);
+                    // the +1 of a negative c sits in the constant's low word: one unit of the grid either way
+                    const double magic = __hiloint2double(emax * (1 << 20) + MAGIC_K, int(cw[r][c] >> (ACC16 ? 15 : 31)));
                     double cd = ACC16 ? double(__half2float(__ushort_as_half((unsigned short)cw[r][c]))) : double(__uint_as_float(cw[r][c]));
                     if (ST) cd = __dmul_rn(cd, pow2d(-(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0])));
                     cd = __hiloint2double(__double2hiint(cd), __double2loint(cd) | 1);
-                    const double a0 = __dadd_rd(cd, magic);
-                    const long long bitsum = __double_as_longlong(a0) + (long long)(cw[r][c] >> (ACC16 ? 15 : 31));
-                    acc[r][c] = __longlong_as_double(bitsum);
+                    acc[r][c] = __dadd_rd(cd, magic);
                 }
             // ---- one fused multiply-add per term, rounding toward minus infinity onto the grid of q; beside it, while
             // the chunk has another block, the product exponents of that block ----
