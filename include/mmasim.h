@@ -163,7 +163,8 @@ typedef enum {
     MMASIM_HW_TF32_F32_K4 = 8,  /* m16n8k4 */
     MMASIM_HW_E4M3_F16 = 9,     /* m16n8k32, FP8 inputs, FP16 accumulator */
     MMASIM_HW_E5M2_F16 = 10,    /* m16n8k32 */
-    MMASIM_HW_E4M3_E5M2_F32 = 11 /* m16n8k32, A in E4M3, B in E5M2 */
+    MMASIM_HW_E4M3_E5M2_F32 = 11, /* m16n8k32, A in E4M3, B in E5M2 */
+    MMASIM_HW_E4M3_F32_K16 = 12  /* m16n8k16 */
 } mmasim_hw_kind;
 int mmasim_hw_mma(int kind, int64_t M, int64_t K, const void* A, const void* B, const void* C, void* D, void* stream);
 

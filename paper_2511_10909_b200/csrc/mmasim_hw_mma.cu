@@ -25,6 +25,7 @@ enum HwKind : int {
     HW_E4M3_F16 = 9,    // m16n8k32  f16 <- e4m3 x e4m3 + f16
     HW_E5M2_F16 = 10,   // m16n8k32  f16 <- e5m2 x e5m2 + f16
     HW_E4M3_E5M2_F32 = 11,  // m16n8k32  f32 <- e4m3 x e5m2 + f32
+    HW_E4M3_F32_K16 = 12,   // m16n8k16  f32 <- e4m3 x e4m3 + f32
     HW_COUNT
 };
 
@@ -42,6 +43,7 @@ __host__ __device__ inline HwShape hw_shape(int kind) {
         case HW_E4M3_F16: return {16, 32, 1, 2};
         case HW_E5M2_F16: return {16, 32, 1, 2};
         case HW_E4M3_E5M2_F32: return {16, 32, 1, 4};
+        case HW_E4M3_F32_K16: return {16, 16, 1, 4};
         default: return {16, 4, 4, 4};      // HW_TF32_F32_K4
     }
 }
@@ -118,10 +120,12 @@ __global__ void __launch_bounds__(128) hw_mma_kernel(int64_t tiles, int64_t K, c
             auto quad = [](const unsigned char* p) { return uint32_t(p[0]) | (uint32_t(p[1]) << 8) | (uint32_t(p[2]) << 16) | (uint32_t(p[3]) << 24); };
             a[0] = quad(ap + (row0 + gid) * K + k0 + tg * 4);
             a[1] = quad(ap + (row0 + gid + 8) * K + k0 + tg * 4);
-            a[2] = quad(ap + (row0 + gid) * K + k0 + tg * 4 + 16);
-            a[3] = quad(ap + (row0 + gid + 8) * K + k0 + tg * 4 + 16);
             b[0] = quad(bp + int64_t(gid) * K + k0 + tg * 4);
-            b[1] = quad(bp + int64_t(gid) * K + k0 + tg * 4 + 16);
+            if (sh.k == 32) {                   // k16: a0, a1 and b0 only
+                a[2] = quad(ap + (row0 + gid) * K + k0 + tg * 4 + 16);
+                a[3] = quad(ap + (row0 + gid + 8) * K + k0 + tg * 4 + 16);
+                b[1] = quad(bp + int64_t(gid) * K + k0 + tg * 4 + 16);
+            }
         }
         if (KIND == HW_F16_F32)
             asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -150,6 +154,9 @@ __global__ void __launch_bounds__(128) hw_mma_kernel(int64_t tiles, int64_t K, c
         else if (KIND == HW_E4M3_E5M2_F32)
             asm volatile("mma.sync.aligned.m16n8k32.row.col.f32.e4m3.e5m2.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                          : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+        else if (KIND == HW_E4M3_F32_K16)
+            asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.e4m3.e4m3.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+                         : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(b[0]));
         else if (KIND == HW_F16_F32_K8)
             asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
                          : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(b[0]));
@@ -198,6 +205,7 @@ int launch_hw_mma(int kind, int64_t M, int64_t K, const void* A, const void* B, 
         case HW_E4M3_F16: err = launch_hw<HW_E4M3_F16>(tiles, K, A, B, C, D, stream); break;
         case HW_E5M2_F16: err = launch_hw<HW_E5M2_F16>(tiles, K, A, B, C, D, stream); break;
         case HW_E4M3_E5M2_F32: err = launch_hw<HW_E4M3_E5M2_F32>(tiles, K, A, B, C, D, stream); break;
+        case HW_E4M3_F32_K16: err = launch_hw<HW_E4M3_F32_K16>(tiles, K, A, B, C, D, stream); break;
         default: err = launch_hw<HW_TF32_F32_K4>(tiles, K, A, B, C, D, stream); break;
     }
     if (err != cudaSuccess) { set_error("mmasim_hw_mma launch failed: %s", cudaGetErrorString(err)); return MMASIM_ERR_CUDA; }

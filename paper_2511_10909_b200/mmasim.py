@@ -250,7 +250,7 @@ def error_stats(acc: str, D, ref, stats=None, *, stream=None):
 
 
 HW_KINDS = ["f16_f32", "f16_f16", "bf16_f32", "tf32_f32", "e4m3_f32", "e5m2_f32", "f64", "f16_f32_k8", "tf32_f32_k4",
-            "e4m3_f16", "e5m2_f16", "e4m3_e5m2_f32"]
+            "e4m3_f16", "e5m2_f16", "e4m3_e5m2_f32", "e4m3_f32_k16"]
 _HW_ACC_BYTES = {"f16_f16": 2, "f64": 8, "e4m3_f16": 2, "e5m2_f16": 2}
 
 

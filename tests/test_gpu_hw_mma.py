@@ -185,3 +185,28 @@ def test_fp8_mma_sync_with_fp16_accumulator(fmt):
         D = gu.host_words(d.view(torch.int16)).copy()
         D[np.isnan(D.view(np.float16))] = 0x7FFF
         assert np.array_equal(hw, D), (fmt, mode, int((hw != D).sum()))
+
+
+@pytest.mark.parametrize("K", [16, 48])
+def test_fp8_k16_mma_sync_is_two_blocks_of_eight(K):
+    """m16n8k16 on E4M3: the same scheme with the halves of one operand register per row - two fused blocks of 8 (the
+    Blackwell FP16 row with L = 8: the FP16 instruction of that length) chained from +0, then the FP32 addition of C."""
+    from paper_2511_10909_b200 import explore, mmasim
+    _needs_b200()
+    g = wl.rng(105 + K)
+    M = 1 << 12
+    order = [16 * q + k for q in range(K // 16) for half in ((0, 1), (2, 3)) for k in range(16) if k % 4 in half]
+    p = torch.tensor(order, device="cuda")
+    model = mmasim.Model("blackwell", "fp16", "fp32", l_max=8)
+    for mode in ("normal", "bits"):
+        inp = wl.normal_inputs("e4m3", "fp32", M, 8, K, seed=106)
+        A, B, C = inp["A"], inp["B"], inp["C"]
+        if mode == "bits":
+            A = g.integers(0, 256, A.shape, dtype=np.uint8)
+            B = g.integers(0, 256, B.shape, dtype=np.uint8)
+            C = g.integers(0, 1 << 32, C.shape, dtype=np.uint64).astype(np.uint32)
+        hw = _run("e4m3_f32_k16", A, B, C)
+        A16 = explore.widen_fp8_to_fp16("e4m3", gu.dev(A))[:, p].contiguous()
+        B16 = explore.widen_fp8_to_fp16("e4m3", gu.dev(B))[:, p].contiguous()
+        D = gu.host_words(mmasim.gemm(model, A16, B16, gu.dev(C), k_chunk=16))
+        assert np.array_equal(hw, D), (K, mode, int((hw != D).sum()))
