@@ -36,13 +36,15 @@ def test_fragment_layouts_with_exact_integers():
     g = wl.rng(90)
     M = 64
     for kind, (fmt, acc, k) in list(KINDS.items()) + [("e4m3_f32", ("e4m3", "fp32", 32)), ("e5m2_f32", ("e5m2", "fp32", 32)),
+                                                       ("e4m3_f16", ("e4m3", "fp16", 32)), ("e5m2_f16", ("e5m2", "fp16", 32)),
+                                                       ("e4m3_e5m2_f32", ("e4m3", "fp32", 32)), ("e4m3_f32_k16", ("e4m3", "fp32", 16)),
                                                        ("f64", ("fp64", "fp64", 4))]:
         for K in (k, 3 * k):
             a = g.integers(-2, 3, (M, K)); b = g.integers(-2, 3, (8, K)); c = g.integers(-8, 9, (M, 8))
             if fmt == "fp64":
                 A, B, C = (x.astype(np.float64).view(np.uint64) for x in (a, b, c))
             else:
-                A, B = wl.cast(a.astype(np.float32), fmt), wl.cast(b.astype(np.float32), fmt)
+                A, B = wl.cast(a.astype(np.float32), fmt), wl.cast(b.astype(np.float32), "e5m2" if kind == "e4m3_e5m2_f32" else fmt)
                 C = c.astype(np.float32).view(np.uint32) if acc == "fp32" else c.astype(np.float16).view(np.uint16)
             D = _run(kind, A, B, C)
             want = a @ b.T + c
