@@ -67,10 +67,78 @@ def compute_dtype(kernel: str, model) -> str:
             "efdpa": "f64", "dot_tfdpa": "f64", "dot_ftz": "f32", "ftz_addmul": "f32", "fma_f32": "f32", "fma_f64": "f64", "gstfdpa": "int32"}.get(kernel, "int64")
 
 
-# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of the
-# workload; command and figures in profiles/tfdpa_trop_hopper_e4m3_2048.md).  The kernels are bound by arithmetic:
-# this is context, 0.4 % of what the memory could move in the kernel's time.
+# DRAM bytes per launch of the dominant kernel: dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of
+# the workload, a STORED CONSTANT, not a figure of this run.  The kernels are bound by arithmetic: this is context,
+# 0.4 % of what the memory could move in the kernel's time.
 NCU_DRAM_BYTES = {"cfg3": 101593856 + 34110464, "cfg3_2k": 25592832 + 38656}
+
+SMS = 148
+# The pipe that bounds each kernel: (name, instruction kinds of the issue-rate micro-benchmark that witness its rate,
+# nominal results per SM and clock, pipe instructions per emulated MAC).
+#   f32 fused summation (F = 13): one FP32 fused multiply-add per term; f64 fused summation (F >= 23, TR, GTR, E): one
+#   FP64 fused multiply-add per term; Phi_FMA: the multiply-add itself; Phi_FTZ-AddMul: one multiply and one add per
+#   term (two FP32-pipe instructions); GST-FDPA: one 4-way byte dot product per four terms.
+FP32_KINDS = ("ffma.rm", "ffma2.rm", "ffma.rn.x16", "ffma.rn.x32", "ffma.rm.x16", "ffma2.rm.x16")
+FP64_KINDS = ("dfma", "dfma.rn.x16", "dfma.rn.x32", "dfma.rm.x16")
+PIPES = {
+    "fp32_fma": ("FP32 fused multiply-add issue", FP32_KINDS, 128.0),
+    "fp64_fma": ("FP64 fused multiply-add issue", FP64_KINDS, 64.0),
+    "int_dp4a": ("4-way byte dot-product issue", ("dp4a",), 64.0),
+    "int_alu": ("3-input integer add issue", ("iadd3",), 64.0),
+}
+
+
+def pipe_of(kernel: str, model):
+    """(pipe key, pipe instructions per emulated MAC) of the kernel a model dispatches to."""
+    if kernel == "tfdpa_lut8" and model.F <= 13:
+        return "fp32_fma", 1.0
+    if kernel in ("tfdpa_lut8", "tfdpa_f16", "tfdpa_bf16", "tfdpa_tf32", "trfdpa", "gtrfdpa", "efdpa", "fma_f64"):
+        return "fp64_fma", 1.0
+    if kernel == "fma_f32":
+        return "fp32_fma", 1.0
+    if kernel == "ftz_addmul":
+        return "fp32_fma", 2.0
+    if kernel == "gstfdpa":
+        return "int_dp4a", 0.25
+    return "int_alu", algorithmic_ops_per_mac(model)
+
+
+def measure_pipe_peaks(mmasim, torch, dev, pipes):
+    """Issue rates of the given pipes, measured live: every witness kind at 2, 4 and 8 CTAs of 256 threads per SM, best
+    of three launches each; returns {pipe: {"peak": ops/s, "witness": kind, "ctas_per_sm": n, "all": {kind: ops/s}}}."""
+    sink = torch.zeros(4, dtype=torch.int32, device=dev)
+    out = {}
+    for pipe in pipes:
+        _, kinds, _ = PIPES[pipe]
+        best, who, occ, every = 0.0, None, 0, {}
+        for kind in kinds:
+            kbest = 0.0
+            for ctas in (2, 4, 8):
+                mmasim.int_peak(kind, SMS * ctas, 256, sink)
+                for _ in range(3):
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    ops = mmasim.int_peak(kind, SMS * ctas, 8192 // ctas, sink)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    rate = ops / (e0.elapsed_time(e1) * 1e-3)
+                    kbest = max(kbest, rate)
+                    if rate > best:
+                        best, who, occ = rate, kind, ctas
+            every[kind] = kbest
+        out[pipe] = {"peak": best, "witness": who, "ctas_per_sm": occ, "all": every}
+    return out
+
+
+# One model per kernel template (and per block length where the per-block work matters): the per-model leg of the line.
+PER_MODEL = [("hopper", "e4m3", "fp32"), ("hopper", "e4m3", "fp16"), ("ada", "e5m2", "fp32"),
+             ("volta", "fp16", "fp32"), ("ampere", "fp16", "fp32"), ("hopper", "fp16", "fp32"), ("hopper", "fp16", "fp16"),
+             ("ampere", "bf16", "fp32"), ("hopper", "bf16", "fp32"), ("ampere", "tf32", "fp32"), ("hopper", "tf32", "fp32"),
+             ("blackwell", "e4m3", "fp32"), ("blackwell", "e2m1", "fp32"), ("blackwell", "mxe4m3", "fp32"),
+             ("blackwell", "mxf4", "fp32"), ("blackwell", "nvf4", "fp32"),
+             ("cdna3", "bf16", "fp32"), ("cdna3", "tf32", "fp32"), ("cdna3", "e4m3", "fp32"),
+             ("cdna1", "fp16", "fp32"), ("cdna1", "bf16", "fp32"), ("cdna2", "fp16", "fp32"), ("cdna2", "bf16", "fp32"),
+             ("cdna1", "fp32", "fp32"), ("hopper", "fp64", "fp64")]
 
 
 def algorithmic_ops_per_mac(model) -> float:
@@ -306,23 +374,11 @@ def run_ours(args):
     torch.cuda.synchronize()
     kernel_name = mmasim.last_kernel()
 
-    # issue-rate peaks, measured live (independent chains of one instruction kind on every SM); best of five after a
-    # warm run: the 3-input integer add (the unit of the paper-level operation count), the integer multiply-add, and
-    # the multiply-add the timed kernel sums with (FP32 or FP64, rounded toward minus infinity)
-    sink = torch.zeros(4, dtype=torch.int32, device=dev)
-    peaks = {}
-    fma_kind = {"f32": "ffma.rm", "f64": "dfma"}.get(compute_dtype(kernel_name, model))
-    for kind in ("iadd3", "imad") + ((fma_kind,) if fma_kind else ()):
-        best = 0.0
-        mmasim.int_peak(kind, 148 * 8, 4096, sink)
-        for _ in range(5):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            ops = mmasim.int_peak(kind, 148 * 8, 16384, sink)       # about 2 ms per launch
-            e1.record()
-            torch.cuda.synchronize()
-            best = max(best, ops / (e0.elapsed_time(e1) * 1e-3))
-        peaks[kind] = best
+    # issue-rate peaks, measured live (independent chains of one instruction kind on every SM, several witnesses and
+    # occupancies per pipe, the best counts): the pipe the timed kernel is bound by, and the 3-input integer add that is
+    # the unit of the paper-level operation count
+    pipe_key, pipe_ops_per_mac = pipe_of(kernel_name, model)
+    peaks = measure_pipe_peaks(mmasim, torch, dev, sorted({pipe_key, "int_alu"})) if not is_dot else {}
 
     # ---- timed region: K steps, device timers, L2 flushed between steps ----
     sampler = ClockSampler(local_rank)
@@ -375,40 +431,109 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    ops_per_mac = algorithmic_ops_per_mac(model)
     per_gpu_macs_s = value / world
-    achieved = per_gpu_macs_s * ops_per_mac
-    peak = peaks["iadd3"]
+    sm_mhz = clocks.get("sm_mhz") or 1965.0
+    hbm_peak, hbm_src = 6650.0, "fallback 6.65 TB/s (MEASURED_PEAKS.json absent)"
+    try:
+        hbm_peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["hbm_gbs"])
+        hbm_src = "MEASURED_PEAKS.json hbm_gbs (STREAM-style copy)"
+    except (OSError, KeyError, ValueError):
+        pass
+
+    def pipe_view(pipe, ops_per_mac, macs_s):
+        """Fractions of one pipe: against the best live witness and against the nominal rate at the sampled clock."""
+        label, _, per_clk = PIPES[pipe]
+        nominal = SMS * per_clk * sm_mhz * 1e6
+        measured = peaks[pipe]["peak"]
+        achieved = macs_s * ops_per_mac
+        return {"pipe": label, "pipe_ops_per_mac": ops_per_mac, "achieved": achieved / 1e12, "peak": measured / 1e12,
+                "unit": "Tops/s", "frac": achieved / measured, "peak_nominal": nominal / 1e12, "frac_nominal": achieved / nominal,
+                "peak_source": f"measured live, best witness {peaks[pipe]['witness']} at {peaks[pipe]['ctas_per_sm']} CTAs/SM "
+                               f"(= {measured / (SMS * sm_mhz * 1e6):.1f} per SM and clock at the sampled {sm_mhz:.0f} MHz); "
+                               f"nominal {per_clk:.0f} per SM and clock",
+                "witnesses": {k: v / 1e12 for k, v in peaks[pipe]["all"].items()}}
+
     if is_dot:
         esz = inp["A"].dtype.itemsize
         bytes_per_dot = 2 * K * esz + 8
-        hbm_peak, src = 6650.0, "fallback 6.65 TB/s (MEASURED_PEAKS.json absent)"
-        try:
-            hbm_peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["hbm_gbs"])
-            src = "MEASURED_PEAKS.json hbm_gbs (STREAM-style copy)"
-        except (OSError, KeyError, ValueError):
-            pass
         gbs = per_gpu_macs_s / K * bytes_per_dot / 1e9
         roofline = {"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gbs / hbm_peak, "traffic": None,
-                    "kernel": kernel_name, "algorithmic_bytes_per_dot": bytes_per_dot, "peak_source": src}
+                    "kernel": kernel_name, "algorithmic_bytes_per_dot": bytes_per_dot, "peak_source": hbm_src}
     else:
-        dtype = compute_dtype(kernel_name, model)
-        int_view = {"achieved": achieved / 1e12, "peak": peak / 1e12, "unit": "Tint-op/s", "frac": achieved / peak,
-                    "algorithmic_int_ops_per_mac": ops_per_mac,
-                    "peak_source": "measured live: independent 3-input integer adds on all SMs (mmasim_int_peak kind iadd3)",
-                    "imad_peak": peaks["imad"] / 1e12}
-        if dtype in ("f32", "f64") and model.family in ("t", "st", "tr", "gtr", "e"):
-            # the fused-summation kernels spend exactly one fused multiply-add per emulated MAC: that pipe is the bound
-            kind = fma_kind
-            roofline = {"bound": "alu", "achieved": per_gpu_macs_s / 1e12, "peak": peaks[kind] / 1e12, "unit": "Tfma/s",
-                        "frac": per_gpu_macs_s / peaks[kind], "traffic": NCU_DRAM_BYTES.get(name), "kernel": kernel_name,
-                        "algorithmic_fma_per_mac": 1.0,
-                        "peak_source": f"measured live: independent fused multiply-adds rounded toward minus infinity on all SMs "
-                                       f"(mmasim_int_peak kind {kind})" +
-                                       ("; nominal FP32 rate 148 SMs x 128 lanes x 1.965 GHz = 37.2 Tfma/s" if dtype == "f32" else ""),
-                        "paper_level_integer_count": int_view}
-        else:
-            roofline = {"bound": "alu", "traffic": None, "kernel": kernel_name, **int_view}
+        ops_per_mac = algorithmic_ops_per_mac(model)
+        int_view = pipe_view("int_alu", ops_per_mac, per_gpu_macs_s)
+        int_view["note"] = ("the count of 6 integer operations per term + 25 per block is not a floor for this formulation: the "
+                            "kernel replaces multiply / distance / shift / add by one fused multiply-add and the maximum by a "
+                            "tensor-core product of powers, so this fraction may exceed 1 and bounds nothing")
+        roofline = {"bound": "alu", **pipe_view(pipe_key, pipe_ops_per_mac, per_gpu_macs_s), "kernel": kernel_name,
+                    "traffic": NCU_DRAM_BYTES.get(name),
+                    "traffic_source": "stored constant from one ncu capture of this workload (not measured in this run)" if name in NCU_DRAM_BYTES else None,
+                    "paper_level_integer_count": int_view}
+
+    # ---- per-model leg: one model per kernel template at 4096^3, three launches each after one warm-up, L2 flushed ----
+    per_model, dot_line = None, None
+    if not args.skip_extras and not is_dot and world == 1 and not args.no_per_model:
+        from paper_2511_10909_b200 import workloads as wl
+        size = args.per_model_size
+        pm_peaks_needed = set()
+        rows, cache = [], {}
+        for pk in PER_MODEL:
+            ck = (pk[1], pk[2])
+            if ck not in cache:
+                cache.clear()
+                cache[ck] = {k: to_dev(v) for k, v in wl.normal_inputs(pk[1], pk[2], size, size, size, seed=5).items()}
+            t = cache[ck]
+            mdl = mmasim.Model(*pk)
+            pkw = dict(sfa=t["sfa"], sfb=t["sfb"]) if "sfa" in t else {}
+            out = mmasim.gemm(mdl, t["A"], t["B"], t["C"], K=size, **pkw)
+            torch.cuda.synchronize()
+            kern = mmasim.last_kernel()
+            best, tot = None, 0.0
+            for _ in range(3):
+                flush.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                mmasim.gemm(mdl, t["A"], t["B"], t["C"], out=out, K=size, **pkw)
+                e1.record()
+                torch.cuda.synchronize()
+                ms = e0.elapsed_time(e1)
+                tot += ms
+                best = ms if best is None else min(best, ms)
+            pp, opm = pipe_of(kern, mdl)
+            pm_peaks_needed.add(pp)
+            rows.append({"model": "-".join(pk), "kernel": kern, "ms": tot / 3, "ms_best": best,
+                         "macs_per_s": float(size) ** 3 / (tot / 3 * 1e-3), "_pipe": pp, "_opm": opm})
+            del out
+        cache.clear()
+        peaks.update(measure_pipe_peaks(mmasim, torch, dev, sorted(pm_peaks_needed - set(peaks))))
+        per_model = []
+        for r in rows:
+            v = pipe_view(r.pop("_pipe"), r.pop("_opm"), r["macs_per_s"])
+            r.update(pipe=v["pipe"], pipe_ops_per_mac=v["pipe_ops_per_mac"], frac=v["frac"], frac_nominal=v["frac_nominal"])
+            per_model.append(r)
+        # the HBM-bound probe-style batch (config 4): 2^20 dots of length 32, FP16, both kernel kinds
+        dot_line = []
+        for dk in (("hopper", "fp16", "fp32"), ("cdna2", "fp16", "fp32")):
+            A4, B4, C4 = wl.cfg4("fp16", 32)
+            tA, tB, tC = to_dev(A4), to_dev(B4), to_dev(C4)
+            mdl = mmasim.Model(*dk)
+            o4 = mmasim.dot_batch(mdl, tA, tB, tC)
+            torch.cuda.synchronize()
+            tot = 0.0
+            for _ in range(5):
+                flush.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                mmasim.dot_batch(mdl, tA, tB, tC, out=o4)
+                e1.record()
+                torch.cuda.synchronize()
+                tot += e0.elapsed_time(e1)
+            nbytes = (1 << 20) * (2 * 32 * 2 + 8)
+            gbs = nbytes / (tot / 5 * 1e-3) / 1e9
+            dot_line.append({"model": "-".join(dk), "kernel": mmasim.last_kernel(), "dots": 1 << 20, "K": 32, "us": tot / 5 * 1e3,
+                             "macs_per_s": (1 << 25) / (tot / 5 * 1e-3), "bound": "hbm", "achieved_gbs": gbs, "peak_gbs": hbm_peak,
+                             "frac": gbs / hbm_peak, "peak_source": hbm_src})
+            del tA, tB, tC, o4
     if args.skip_extras or is_dot:
         cpu_value, cpu_info = None, {"cores": 0, "sample": "skipped"}
     else:
@@ -422,6 +547,7 @@ def run_ours(args):
         "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps,
         "roofline": roofline,
         "cpu_baseline": {"value": cpu_value, "unit": UNIT, "kind": "oracle", **cpu_info},
+        "per_model": per_model, "per_model_size": args.per_model_size if per_model else None, "dot_batch": dot_line,
     }
     print(json.dumps(line))
     if dist is not None:
@@ -507,10 +633,12 @@ def main():
     ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS))
     ap.add_argument("--skip-extras", action="store_true",
                     help="skip the end-to-end and CPU-oracle legs (profiler captures only; not a valid bench line)")
+    ap.add_argument("--no-per-model", action="store_true", help="skip the per-model and dot_batch legs of the line")
+    ap.add_argument("--per-model-size", type=int, default=4096, help="M = N = K of the per-model leg")
     ap.add_argument("--sweep", action="store_true", help="time every registry row at --size^3 (not the bench line)")
     ap.add_argument("--size", type=int, default=4096)
     ap.add_argument("--check", type=int, default=0, help="with --sweep: compare this many seeded sampled outputs per model with the oracle")
-    ap.add_argument("--out-dir", default="gpurun_out", help="with --sweep: folder of the per-model JSON lines")
+    ap.add_argument("--out-dir", default="sweep_out", help="with --sweep: folder of the per-model JSON lines")
     ap.add_argument("--models", default="", help="with --sweep: comma-separated arch-infmt-acc names (default: all)")
     args = ap.parse_args()
     if args.sweep:

@@ -134,14 +134,19 @@ int mmasim_dot_batch(const mmasim_model* model, int64_t n, int64_t K,
 
 /* mmasim_gemm_ex on HOST buffers: allocates device memory, copies A, B, C (and scales) to the device, runs,
  * copies D back and frees; synchronous.  Fields of opts that are pointers are host pointers here.
- * The device buffers are stream-ordered allocations (cudaMallocAsync) on a stream of the call's own; the device's
- * default memory pool is told to keep up to 1 GiB between calls, so repeated calls do not pay for allocation
- * (cudaMemPoolTrimTo on that pool returns the memory).  Pinned host buffers make the copies asynchronous.
+ * The device buffers are stream-ordered allocations on a stream of the call's own, out of a memory pool that the
+ * library creates per device on first use and that keeps up to 1 GiB between calls, so repeated calls do not pay
+ * for allocation; mmasim_host_release() destroys the pools and returns the memory.  The device's default memory
+ * pool and its attributes are not touched.  Pinned host buffers make the copies asynchronous.
  * Problems of 1024 rows and 32 MiB or more are cut into up to eight row panels of D (outputs are independent,
  * Section 3.1 Step 1): B is copied once, then each panel's rows of A and C go in, its kernel runs and its rows of D
  * come back on separate streams, so that with pinned buffers the copies run beside the arithmetic. */
 int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
                      const void* A, const void* B, const void* C, void* D, const mmasim_gemm_opts* opts);
+
+/* Destroys the memory pools mmasim_gemm_host created (every device); no mmasim_gemm_host call may be in flight.
+ * The next mmasim_gemm_host call creates a new pool.  No counterpart in the paper. */
+int mmasim_host_release(void);
 
 /* The hardware's own matrix multiply-accumulate, for differential runs of the models against the machine they
  * describe (Section 3.1, Step 4; Section 3.2: an MMA interface is D = MMA(A, B, C) on one instruction).  Runs the
@@ -178,12 +183,24 @@ int mmasim_hw_mma(int kind, int64_t M, int64_t K, const void* A, const void* B, 
  * All pointers are device pointers. */
 int mmasim_error_stats(int acc_fmt, int64_t n, const void* D, const double* ref, double* stats, void* stream);
 
-/* Integer-issue micro-benchmark used as the roofline denominator (no counterpart in the paper): launches
- * `blocks` CTAs of 256 threads, each thread running `iters` rounds of 8 independent dependent-chain integer
- * operations of the given kind (0: 3-input add, 1: logic, 2: funnel shift, 3: 32-bit multiply-add, 4: the
- * add/max/shift/add mix of one emulated MAC).  `sink` (device, >= 4 bytes) receives a value that keeps the
- * work alive.  The caller times the launch; operations per launch = blocks * 256 * iters * 8 * ops_per_round,
- * where ops_per_round is returned through *ops_per_round. */
+/* Issue-rate micro-benchmarks, the roofline denominators (no counterpart in the paper).  Launches `blocks` CTAs of
+ * 256 threads; every thread runs `iters` (rounded up to a multiple of 8) times 8 rounds of independent operations of
+ * the given kind.  `sink` (device, >= 4 bytes) receives a value that keeps the work alive.  The caller times the
+ * launch; counted operations per launch = blocks * 256 * iters * 8 * (*ops_per_round).  Kinds:
+ *    0 iadd3          3-input integer add              1 lop3           3-input logic
+ *    2 shf            funnel shift                     3 imad           32-bit integer multiply-add
+ *    4 macmix         add / max / sub / shift / add of one emulated term (5 operations per round)
+ *    5 viaddmax       fused add-max, 32-bit            6 viaddmax16x2   fused add-max on two 16-bit lanes
+ *    7 f2i            float -> int conversion          8 fmul           FP32 multiply
+ *    9 popc           population count + add          10 imad+alu       one multiply-add and one add per round
+ *   11 fmul+alu       FP32 multiply and integer add   12 imad.wide      32 x 32 -> 64-bit multiply
+ *   13 mac_d1, 14 mac_d2   two integer forms of one emulated term
+ *   15 dp4a           4-way byte dot product          16 dfma           FP64 multiply-add, 8 dependent chains
+ *   17 dfma+alu       FP64 multiply-add and add-max   18 ffma.rm        FP32 multiply-add toward -inf, 8 chains
+ *   19 ffma2.rm       packed two-lane fma.rm.f32x2, 8 chains
+ *   20 ffma.rn.x16, 21 ffma.rn.x32, 22 ffma.rm.x16, 23 ffma2.rm.x16 (lanes counted), 24 dfma.rn.x16, 25 dfma.rn.x32,
+ *   26 dfma.rm.x16    the same instructions with 16 / 32 independent accumulators per thread and loop-invariant
+ *                     multiplicands (no operand-fetch conflicts): the second witness of the pipe rates. */
 int mmasim_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t* ops_per_round, void* stream);
 
 /* Name of the kernel variant the last mmasim_gemm* call on this thread dispatched to ("generic", ...). */

@@ -3,6 +3,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include "mmasim_internal.h"
 
@@ -109,6 +110,37 @@ int build_args(const mmasim_model* model, int64_t M, int64_t N, int64_t K, const
     return MMASIM_OK;
 }
 
+// Staging memory of mmasim_gemm_host: one memory pool per device, the library's own (the device's default pool and
+// its attributes are the caller's and stay untouched), created on first use, keeping up to 1 GiB between calls.
+constexpr int MAX_DEVICES = 64;
+std::mutex g_pool_mutex;
+cudaMemPool_t g_pools[MAX_DEVICES] = {};
+
+cudaError_t host_pool(cudaMemPool_t* out) {
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_pool_mutex);
+    if (!g_pools[dev]) {
+        cudaMemPoolProps props;
+        std::memset(&props, 0, sizeof(props));
+        props.allocType = cudaMemAllocationTypePinned;
+        props.handleTypes = cudaMemHandleTypeNone;
+        props.location.type = cudaMemLocationTypeDevice;
+        props.location.id = dev;
+        cudaMemPool_t pool = nullptr;
+        err = cudaMemPoolCreate(&pool, &props);
+        if (err != cudaSuccess) return err;
+        unsigned long long keep = 1ull << 30;
+        err = cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+        if (err != cudaSuccess) { cudaMemPoolDestroy(pool); return err; }
+        g_pools[dev] = pool;
+    }
+    *out = g_pools[dev];
+    return cudaSuccess;
+}
+
 }  // namespace
 }  // namespace mmasim
 
@@ -181,6 +213,10 @@ int mmasim_gemm_ex(const mmasim_model* model, int64_t M, int64_t N, int64_t K, c
     if ((st = check_device_ptr(B, "B")) != MMASIM_OK) return st;
     if ((st = check_device_ptr(D, "D")) != MMASIM_OK) return st;
     if (C && (st = check_device_ptr(C, "C")) != MMASIM_OK) return st;
+    if (g.sfa && (st = check_device_ptr(g.sfa, "opts->sfa")) != MMASIM_OK) return st;
+    if (g.sfb && (st = check_device_ptr(g.sfb, "opts->sfb")) != MMASIM_OK) return st;
+    if (g.row_scale && (st = check_device_ptr(g.row_scale, "opts->row_scale")) != MMASIM_OK) return st;
+    if (g.col_scale && (st = check_device_ptr(g.col_scale, "opts->col_scale")) != MMASIM_OK) return st;
     return run_gemm(model, g, opts ? opts->flags : 0, static_cast<cudaStream_t>(stream));
 }
 
@@ -232,7 +268,7 @@ int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
     void *dA = nullptr, *dB = nullptr, *dC = nullptr, *dD = nullptr, *dSA = nullptr, *dSB = nullptr, *dRS = nullptr, *dCS = nullptr;
     cudaError_t err = cudaSuccess;
     // Stream-ordered allocations on a stream of this call's own: after the first call the buffers come out of the
-    // device's default memory pool (which keeps up to 1 GiB between calls) and the call synchronises once, at the end.
+    // library's own memory pool (which keeps up to 1 GiB between calls) and the call synchronises once, at the end.
     // Large problems are cut into a few row panels of D (outputs are independent, Section 3.1 Step 1): B once, then per
     // panel its rows of A and C in, the kernel, its rows of D out, on three streams chained by events, so that the
     // copies of one panel run beside the arithmetic of another (two compute streams, so that a panel's last CTAs
@@ -262,16 +298,11 @@ int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
             if (err == cudaSuccess) err = cudaEventCreateWithFlags(&ev_k[p], cudaEventDisableTiming);
         }
     }
-    if (err == cudaSuccess) {
-        int dev = 0;
-        cudaMemPool_t pool = nullptr;
-        unsigned long long keep = 1ull << 30;
-        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess)
-            cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
-    }
+    cudaMemPool_t pool = nullptr;
+    if (err == cudaSuccess) err = host_pool(&pool);
     auto alloc = [&](void** dst, const void* src, size_t bytes) {
         if (err != cudaSuccess || !src || !bytes) return;
-        err = cudaMallocAsync(dst, bytes, s_in);
+        err = cudaMallocFromPoolAsync(dst, bytes, pool, s_in);
     };
     auto h2d = [&](void* dst, const void* src, size_t off, size_t bytes) {
         if (err != cudaSuccess || !src || !bytes) return;
@@ -351,18 +382,46 @@ int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
 
 int mmasim_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t* ops_per_round, void* stream) {
     if (!sink || !ops_per_round || blocks < 1 || iters < 1 || kind < 0) { set_error("mmasim_int_peak: bad argument"); return MMASIM_ERR_INVALID_ARG; }
+    const int st = check_device_ptr(sink, "sink");
+    if (st != MMASIM_OK) return st;
     return launch_int_peak(kind, blocks, iters, sink, ops_per_round, static_cast<cudaStream_t>(stream));
 }
 
 int mmasim_hw_mma(int kind, int64_t M, int64_t K, const void* A, const void* B, const void* C, void* D, void* stream) {
     if (!A || !B || !D) { set_error("mmasim_hw_mma: A, B and D must not be NULL"); return MMASIM_ERR_INVALID_ARG; }
+    int st;
+    if ((st = check_device_ptr(A, "A")) != MMASIM_OK) return st;
+    if ((st = check_device_ptr(B, "B")) != MMASIM_OK) return st;
+    if ((st = check_device_ptr(D, "D")) != MMASIM_OK) return st;
+    if (C && (st = check_device_ptr(C, "C")) != MMASIM_OK) return st;
     return launch_hw_mma(kind, M, K, A, B, C, D, static_cast<cudaStream_t>(stream));
 }
 
 int mmasim_error_stats(int acc_fmt, int64_t n, const void* D, const double* ref, double* stats, void* stream) {
     if (!D || !ref || !stats || n < 1) { set_error("mmasim_error_stats: bad argument"); return MMASIM_ERR_INVALID_ARG; }
+    int st;
+    if ((st = check_device_ptr(D, "D")) != MMASIM_OK) return st;
+    if ((st = check_device_ptr(ref, "ref")) != MMASIM_OK) return st;
+    if ((st = check_device_ptr(stats, "stats")) != MMASIM_OK) return st;
     return launch_error_stats(acc_fmt == MMASIM_ACC_F16 ? ACC_F16 : (acc_fmt == MMASIM_ACC_F32 ? ACC_F32 : -1), n, D, ref, stats,
                               static_cast<cudaStream_t>(stream));
+}
+
+int mmasim_host_release(void) {
+    std::lock_guard<std::mutex> lock(g_pool_mutex);
+    cudaError_t err = cudaSuccess;
+    for (int d = 0; d < MAX_DEVICES; ++d)
+        if (g_pools[d]) {
+            const cudaError_t e = cudaMemPoolDestroy(g_pools[d]);
+            if (err == cudaSuccess) err = e;
+            g_pools[d] = nullptr;
+        }
+    if (err != cudaSuccess) {
+        cudaGetLastError();
+        set_error("mmasim_host_release: %s", cudaGetErrorString(err));
+        return MMASIM_ERR_CUDA;
+    }
+    return MMASIM_OK;
 }
 
 const char* mmasim_last_kernel(void) { return g_kernel; }

@@ -129,14 +129,20 @@ __device__ __forceinline__ uint32_t rho_apply(int rho, int64_t S, int e) {
 // ---------------------------------------------------------------------------------------------------------
 // Fixed-point alignment helpers.  rz: truncate the magnitude (sign-magnitude), rd: floor.
 // ---------------------------------------------------------------------------------------------------------
+// A zero operand stays zero whatever the shift (zero terms reach here with meaningless distances); nonzero operands
+// never meet a left shift of 64 or more (every aligned term fits 64 bits by construction).  Left shifts are done on
+// the unsigned magnitude / two's-complement bits.
 __device__ __forceinline__ int64_t rz_scale(int64_t n, int sh) {
+    if (n == 0) return 0;
     const bool neg = n < 0;
-    uint64_t m = neg ? uint64_t(-n) : uint64_t(n);
-    if (sh >= 0) m <<= sh; else m = (sh <= -64) ? 0ull : (m >> (-sh));
+    uint64_t m = neg ? 0ull - uint64_t(n) : uint64_t(n);
+    if (sh >= 0) m = (sh >= 64) ? 0ull : (m << sh);
+    else m = (sh <= -64) ? 0ull : (m >> (-sh));
     return neg ? -int64_t(m) : int64_t(m);
 }
 __device__ __forceinline__ int64_t rd_scale(int64_t n, int sh) {
-    if (sh >= 0) return n << sh;
+    if (n == 0) return 0;
+    if (sh >= 0) return (sh >= 64) ? 0ll : int64_t(uint64_t(n) << sh);
     return (sh <= -64) ? (n < 0 ? -1ll : 0ll) : (n >> (-sh));
 }
 
@@ -225,7 +231,7 @@ __device__ __forceinline__ uint32_t gst_block(const uint32_t* a, const uint32_t*
     for (int g = 0; g < ng; ++g) {                                  // Step 1
         int p = 0;                                                  // units of 2^-2 (E2M1: Exp >= 0, 1 mantissa bit)
         for (int k = g * m.G; k < (g + 1) * m.G; ++k)
-            p += (dec_ssig(a[k]) * dec_ssig(b[k])) << (dec_exp(a[k]) + dec_exp(b[k]));
+            p += (dec_ssig(a[k]) * dec_ssig(b[k])) * (1 << (dec_exp(a[k]) + dec_exp(b[k])));
         const int j = (g * m.G) / m.k_block;
         s[g] = int64_t(p) * int64_t(dec_sig(sfa[j])) * int64_t(dec_sig(sfb[j]));
         e[g] = dec_exp(sfa[j]) + dec_exp(sfb[j]);
@@ -297,7 +303,7 @@ __device__ __forceinline__ uint32_t tr_block(const uint32_t* a, const uint32_t* 
         sc2 = rd_scale(sc, (dc.exp - E) + F - 23);
     }
     if (grouped && dc.exp < E - F - 1) sc2 = 0;                     // special truncation
-    const int64_t S = T2 + (sc2 << (F2 - F));
+    const int64_t S = T2 + sc2 * (int64_t(1) << (F2 - F));
     return rho_apply(m.rho, S, E - F2);
 }
 

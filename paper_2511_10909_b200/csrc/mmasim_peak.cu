@@ -8,7 +8,8 @@ namespace {
 
 enum PeakKind : int {
     PK_IADD3 = 0, PK_LOP3, PK_SHF, PK_IMAD, PK_MACMIX, PK_VIADDMAX, PK_VIADDMAX16X2, PK_F2I, PK_FMUL, PK_POPC,
-    PK_IMAD_PLUS_ALU, PK_FMUL_PLUS_ALU, PK_IMAD_WIDE, PK_MAC_D1, PK_MAC_D2, PK_DP4A, PK_DFMA, PK_DFMA_PLUS_ALU, PK_FFMA_RM, PK_FFMA2_RM, PK_COUNT
+    PK_IMAD_PLUS_ALU, PK_FMUL_PLUS_ALU, PK_IMAD_WIDE, PK_MAC_D1, PK_MAC_D2, PK_DP4A, PK_DFMA, PK_DFMA_PLUS_ALU, PK_FFMA_RM, PK_FFMA2_RM,
+    PK_FFMA_RN_X16, PK_FFMA_RN_X32, PK_FFMA_RM_X16, PK_FFMA2_RM_X16, PK_DFMA_RN_X16, PK_DFMA_RN_X32, PK_DFMA_RM_X16, PK_COUNT
 };
 
 template <int KIND>
@@ -129,6 +130,60 @@ __global__ void __launch_bounds__(256) peak_kernel_f32(int64_t iters, int* sink)
     if (r == 0.12345f) *sink = 1;
 }
 
+// Second witness of the floating-point multiply-add rates: NACC independent accumulators per thread, the two
+// multiplicands loop-invariant registers (c_i = x * y + c_i: two source registers besides the accumulator, so that no
+// operand-fetch conflict hides the pipe's own rate), round-to-nearest or toward minus infinity, FP32 (scalar or the
+// packed two-lane instruction) or FP64.  One round = NACC multiply-adds (2 NACC lanes for the packed form).
+template <typename T, int NACC, bool RM, bool PACKED>
+__global__ void __launch_bounds__(256) peak_kernel_fma(int64_t iters, int* sink) {
+    T x[2], c[NACC];
+    unsigned long long x2[2], c2[NACC];
+    x[0] = T(1) + T(1e-7) * T(threadIdx.x);
+    x[1] = T(1) - T(1e-7) * T(threadIdx.x + 3);
+#pragma unroll
+    for (int i = 0; i < NACC; ++i) c[i] = T(i);
+    if (PACKED) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) asm("mov.b64 %0, {%1, %1};" : "=l"(x2[i]) : "f"(float(x[i])));
+#pragma unroll
+        for (int i = 0; i < NACC; ++i) asm("mov.b64 %0, {%1, %2};" : "=l"(c2[i]) : "f"(float(i)), "f"(float(i) + 0.5f));
+    }
+    for (int64_t it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int i = 0; i < NACC; ++i) {
+            if (PACKED) asm volatile("fma.rm.f32x2 %0, %1, %2, %0;" : "+l"(c2[i]) : "l"(x2[0]), "l"(x2[1]));
+            else if (sizeof(T) == 4) {
+                if (RM) asm volatile("fma.rm.f32 %0, %1, %2, %0;" : "+f"(*reinterpret_cast<float*>(&c[i])) : "f"(float(x[0])), "f"(float(x[1])));
+                else asm volatile("fma.rn.f32 %0, %1, %2, %0;" : "+f"(*reinterpret_cast<float*>(&c[i])) : "f"(float(x[0])), "f"(float(x[1])));
+            } else {
+                if (RM) asm volatile("fma.rm.f64 %0, %1, %2, %0;" : "+d"(*reinterpret_cast<double*>(&c[i])) : "d"(double(x[0])), "d"(double(x[1])));
+                else asm volatile("fma.rn.f64 %0, %1, %2, %0;" : "+d"(*reinterpret_cast<double*>(&c[i])) : "d"(double(x[0])), "d"(double(x[1])));
+            }
+        }
+    }
+    T r = T(0);
+#pragma unroll
+    for (int i = 0; i < NACC; ++i) {
+        if (PACKED) {
+            float lo, hi;
+            asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(c2[i]));
+            r += T(lo + hi);
+        } else r += c[i];
+    }
+    if (r == T(0.12345)) *sink = 1;
+}
+
+template <typename T, int NACC, bool RM, bool PACKED>
+int launch_fma(int64_t blocks, int64_t iters, void* sink, int32_t* ops_per_round, cudaStream_t stream) {
+    // the host counts blocks * 256 * iters8 * 8 * ops_per_round operations, iters8 = iters rounded up to a multiple of 8:
+    // run iters8 * 8 rounds of NACC multiply-adds and report NACC (lanes: twice that for the packed form) per round
+    *ops_per_round = NACC * (PACKED ? 2 : 1);
+    peak_kernel_fma<T, NACC, RM, PACKED><<<(unsigned)blocks, 256, 0, stream>>>(iters * 8, static_cast<int*>(sink));
+    const cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) { set_error("int_peak launch failed: %s", cudaGetErrorString(err)); return MMASIM_ERR_CUDA; }
+    return MMASIM_OK;
+}
+
 template <int KIND>
 int launch(int64_t blocks, int64_t iters, void* sink, cudaStream_t stream) {
     peak_kernel<KIND><<<(unsigned)blocks, 256, 0, stream>>>(iters, static_cast<int*>(sink));
@@ -176,6 +231,13 @@ int launch_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t
             if (err != cudaSuccess) { set_error("int_peak launch failed: %s", cudaGetErrorString(err)); return MMASIM_ERR_CUDA; }
             return MMASIM_OK;
         }
+        case PK_FFMA_RN_X16: return launch_fma<float, 16, false, false>(blocks, iters, sink, ops_per_round, stream);
+        case PK_FFMA_RN_X32: return launch_fma<float, 32, false, false>(blocks, iters, sink, ops_per_round, stream);
+        case PK_FFMA_RM_X16: return launch_fma<float, 16, true, false>(blocks, iters, sink, ops_per_round, stream);
+        case PK_FFMA2_RM_X16: return launch_fma<float, 16, true, true>(blocks, iters, sink, ops_per_round, stream);
+        case PK_DFMA_RN_X16: return launch_fma<double, 16, false, false>(blocks, iters, sink, ops_per_round, stream);
+        case PK_DFMA_RN_X32: return launch_fma<double, 32, false, false>(blocks, iters, sink, ops_per_round, stream);
+        case PK_DFMA_RM_X16: return launch_fma<double, 16, true, false>(blocks, iters, sink, ops_per_round, stream);
         default: set_error("mmasim_int_peak: unknown kind %d", kind); return MMASIM_ERR_INVALID_ARG;
     }
 }

@@ -73,6 +73,8 @@ def _load():
     lib.mmasim_hw_mma.argtypes = [c_int, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.mmasim_error_stats.restype = c_int
     lib.mmasim_error_stats.argtypes = [c_int, c_int64, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.mmasim_host_release.restype = c_int
+    lib.mmasim_host_release.argtypes = []
     lib.mmasim_last_kernel.restype = c_char_p
     lib.mmasim_last_error.restype = c_char_p
     return lib
@@ -172,66 +174,130 @@ def _make_opts(sfa=None, sfb=None, k_chunk=0, row_scale=None, col_scale=None, fo
     return o
 
 
+def _matrix(t, name, rows, cols, bits, device):
+    """Checks one matrix argument (CUDA tensor, element width, shape, unit inner stride) and returns its leading
+    dimension in storage words; `cols` is the number of storage words per row that the call reads or writes."""
+    if t is None:
+        return 0
+    if not t.is_cuda or t.device != device:
+        raise MmasimError(1, f"{name} must be a CUDA tensor on {device} (no CPU fallback)")
+    if t.element_size() * 8 != bits:
+        raise MmasimError(1, f"{name} has {t.element_size() * 8}-bit elements, the model needs {bits}-bit words")
+    if t.dim() != 2 or t.shape[0] < rows or t.shape[1] < cols:
+        raise MmasimError(3, f"{name} has shape {tuple(t.shape)}, the call needs at least {rows} x {cols}")
+    if t.shape[1] > 1 and t.stride(1) != 1:
+        raise MmasimError(3, f"{name} must be contiguous along its rows (stride {t.stride(1)})")
+    ld = t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1])
+    if ld < cols:
+        raise MmasimError(3, f"{name}: row stride {ld} is smaller than the row length {cols}")
+    return ld
+
+
+def _vector(t, name, n, bytes_per, device):
+    if t is None:
+        return
+    if not t.is_cuda or t.device != device:
+        raise MmasimError(1, f"{name} must be a CUDA tensor on {device}")
+    if not t.is_contiguous() or t.element_size() != bytes_per or t.numel() < n:
+        raise MmasimError(3, f"{name} must be a contiguous tensor of at least {n} {bytes_per}-byte elements")
+
+
 def gemm(model: Model, A, B, C=None, out=None, *, M=None, N=None, K=None, sfa=None, sfb=None, k_chunk=0,
          row_scale=None, col_scale=None, force_generic=False, stream=None):
     """D = Phi(A, B, C) on CUDA tensors of raw words.
 
     A: M x K, B: N x K (each row is one column of the paper's K x N matrix), C/D: M x N words of the accumulator
-    type (integer tensors of the element width; FP4 of the GST models packed two per byte, so A is M x K/2 uint8
-    and K must be passed).  Returns D (allocated with torch if ``out`` is None).
+    type (integer tensors of the element width; FP4 of the GST models packed two per byte, so A is M x K/2 uint8).
+    Row-strided views are accepted (the row stride becomes the leading dimension lda / ldb / ldc / ldd of
+    mmasim_gemm_ex); the inner dimension must be contiguous.  Returns D (allocated with torch if ``out`` is None).
     """
     import torch
     if not A.is_cuda:
         raise MmasimError(1, "mmasim.gemm needs CUDA tensors (no CPU fallback); use gemm_host for host buffers")
+    per_word = 2 if model.a_bits == 4 else 1                 # elements per storage word
     M = A.shape[0] if M is None else M
     N = B.shape[0] if N is None else N
     if K is None:
-        K = A.shape[1] * (2 if model.a_bits == 4 else 1)
+        K = A.shape[1] * per_word
     if out is None:
         out = torch.empty((M, N), dtype=_acc_dtype(model), device=A.device)
-    plain = sfa is None and not k_chunk and row_scale is None and not force_generic
+    dev = A.device
+    kw = -(-K // per_word)
+    lda = _matrix(A, "A", M, kw, max(model.a_bits, 8), dev) * per_word
+    ldb = _matrix(B, "B", N, kw, max(model.b_bits, 8), dev) * per_word
+    ldc = _matrix(C, "C", M, N, model.acc_bytes * 8, dev)
+    ldd = _matrix(out, "out", M, N, model.acc_bytes * 8, dev)
+    if model.k_block:
+        nsf = -(-K // model.k_block)
+        for t, name, rows in ((sfa, "sfa", M), (sfb, "sfb", N)):
+            if t is not None and (_matrix(t, name, rows, nsf, 8, dev) != nsf):
+                raise MmasimError(3, f"{name} must be a packed {rows} x {nsf} byte matrix")
+    _vector(row_scale, "row_scale", M, 4, dev)
+    _vector(col_scale, "col_scale", N, 4, dev)
+    strided = (lda, ldb) != (K, K) or (C is not None and ldc != N) or ldd != N
+    plain = sfa is None and not k_chunk and row_scale is None and not force_generic and not strided
     if plain:
         _check(_lib.mmasim_gemm(model._h, M, N, K, _ptr(A), _ptr(B), _ptr(C), _ptr(out), _stream(stream)))
     else:
-        o = _make_opts(_ptr(sfa), _ptr(sfb), k_chunk, _ptr(row_scale), _ptr(col_scale), force_generic)
+        o = _make_opts(_ptr(sfa), _ptr(sfb), k_chunk, _ptr(row_scale), _ptr(col_scale), force_generic,
+                       lda, ldb, ldc, ldd)
         _check(_lib.mmasim_gemm_ex(model._h, M, N, K, _ptr(A), _ptr(B), _ptr(C), _ptr(out), byref(o), _stream(stream)))
     return out
 
 
 def dot_batch(model: Model, A, B, C=None, out=None, *, stream=None):
-    """d_t = Phi(a_t, b_t, c_t) for the n rows of A and B (n x K CUDA tensors of raw words)."""
+    """d_t = Phi(a_t, b_t, c_t) for the n rows of A and B (contiguous n x K CUDA tensors of raw words)."""
     import torch
     if not A.is_cuda:
         raise MmasimError(1, "mmasim.dot_batch needs CUDA tensors (no CPU fallback)")
     n, K = A.shape
     if out is None:
         out = torch.empty((n,), dtype=_acc_dtype(model), device=A.device)
+    dev = A.device
+    for t, name, bits in ((A, "A", model.a_bits), (B, "B", model.b_bits)):
+        if _matrix(t, name, n, K, max(bits, 8), dev) != K and n > 1:
+            raise MmasimError(3, f"{name} must be a packed n x K matrix")
+    _vector(C, "C", n, model.acc_bytes, dev)
+    _vector(out, "out", n, model.acc_bytes, dev)
     _check(_lib.mmasim_dot_batch(model._h, n, K, _ptr(A), _ptr(B), _ptr(C), _ptr(out), _stream(stream)))
     return out
 
 
 def gemm_host(model: Model, A, B, C=None, *, K=None, sfa=None, sfb=None, k_chunk=0, row_scale=None, col_scale=None,
               out=None):
-    """As gemm, on host buffers (numpy arrays or CPU tensors): the library copies to the device and back."""
+    """As gemm, on host buffers (numpy arrays or CPU tensors): the library copies to the device and back.
+    Row-strided numpy views of A, B, C and ``out`` are passed with their strides as leading dimensions."""
     import numpy as np
 
-    def as_np(x):
+    def as_np(x, keep_rows=False):
         if x is None:
             return None
         if hasattr(x, "numpy"):
             x = x.numpy()
+        if keep_rows and x.ndim == 2 and (x.shape[1] == 1 or x.strides[1] == x.itemsize) and x.strides[0] >= x.shape[1] * x.itemsize \
+                and x.strides[0] % x.itemsize == 0:
+            return x
         return np.ascontiguousarray(x)
 
-    A, B, C, sfa, sfb, row_scale, col_scale = map(as_np, (A, B, C, sfa, sfb, row_scale, col_scale))
+    A, B, C, out = (as_np(x, True) for x in (A, B, C, out))
+    sfa, sfb, row_scale, col_scale = map(as_np, (sfa, sfb, row_scale, col_scale))
+    per_word = 2 if model.a_bits == 4 else 1
     M, N = A.shape[0], B.shape[0]
     if K is None:
-        K = A.shape[1] * (2 if model.a_bits == 4 else 1)
+        K = A.shape[1] * per_word
     if out is None:
         out = np.empty((M, N), dtype={8: np.uint64, 4: np.uint32, 2: np.uint16}[model.acc_bytes])
+    ld = lambda x: 0 if x is None else x.strides[0] // x.itemsize
     p = lambda x: None if x is None else c_void_p(x.ctypes.data)
-    o = _make_opts(p(sfa), p(sfb), k_chunk, p(row_scale), p(col_scale))
+    o = _make_opts(p(sfa), p(sfb), k_chunk, p(row_scale), p(col_scale), False,
+                   ld(A) * per_word, ld(B) * per_word, ld(C), ld(out))
     _check(_lib.mmasim_gemm_host(model._h, M, N, K, p(A), p(B), p(C), p(out), byref(o)))
     return out
+
+
+def host_release():
+    """Destroys the device memory pools that gemm_host keeps between calls."""
+    _check(_lib.mmasim_host_release())
 
 
 STAT_NAMES = ["count", "sum", "sum_abs", "sum_sq", "negative", "positive", "max_abs", "sum_rel"]
@@ -269,7 +335,8 @@ def hw_mma(kind: str, A, B, C=None, out=None, *, stream=None):
 
 
 PEAK_KINDS = ["iadd3", "lop3", "shf", "imad", "macmix", "viaddmax", "viaddmax16x2", "f2i", "fmul", "popc",
-              "imad+alu", "fmul+alu", "imad.wide", "mac_d1", "mac_d2", "dp4a", "dfma", "dfma+alu", "ffma.rm", "ffma2.rm"]
+              "imad+alu", "fmul+alu", "imad.wide", "mac_d1", "mac_d2", "dp4a", "dfma", "dfma+alu", "ffma.rm", "ffma2.rm",
+              "ffma.rn.x16", "ffma.rn.x32", "ffma.rm.x16", "ffma2.rm.x16", "dfma.rn.x16", "dfma.rn.x32", "dfma.rm.x16"]
 
 
 def int_peak(kind: str, blocks: int, iters: int, sink, stream=None) -> int:

@@ -95,26 +95,34 @@ def test_dot_batch_ragged(key, K, n):
     assert bad.size == 0, (key, K, n, bad[:5], [hex(int(D[i])) for i in bad[:5]], [hex(int(want[i])) for i in bad[:5]])
 
 
-# ---- config 4 at full size: 2^20 dots, sampled dots checked (all classes), CDNA2 FP16 and an NVIDIA model ----
-@pytest.mark.parametrize("key,K", [(("cdna2", "fp16", "fp32"), 32), (("hopper", "fp16", "fp32"), 32),
-                                   (("hopper", "bf16", "fp32"), 16), (("cdna2", "bf16", "fp32"), 4),
-                                   (("hopper", "tf32", "fp32"), 8)], ids=str)
-def test_cfg4_full_size_sampled(key, K):
+# ---- config 4 at full size: 2^20 dots, EVERY dot checked (all eight classes), the CDNA2 models and an NVIDIA model in
+# each of the three formats, K = 4, 8, 16, 32 ----
+CFG4_FULL = [("cdna2", "fp16", "fp32"), ("cdna2", "bf16", "fp32"), ("cdna2", "bf16_1k", "fp32"),
+             ("hopper", "fp16", "fp32"), ("hopper", "bf16", "fp32"), ("hopper", "tf32", "fp32")]
+
+
+@pytest.mark.parametrize("K", [4, 8, 16, 32])
+@pytest.mark.parametrize("key", CFG4_FULL, ids=lambda k: "-".join(k))
+def test_cfg4_full_size_every_dot(key, K):
+    from paper_2511_10909_b200 import mmasim
     n = 1 << 20
     m, A, B, C, D = _dot_case(key, K, n)
-    idx = wl.rng(44).integers(0, n, 16384)
-    want = oracle.phi_dot_batch(m, A[idx], B[idx], C[idx])
-    assert np.array_equal(D[idx].astype(np.uint64), want)
+    assert mmasim.last_kernel() in ("dot_tfdpa", "dot_ftz")
+    want = oracle.phi_dot_batch(m, A, B, C)
+    bad = np.flatnonzero(D.astype(np.uint64) != want)
+    assert bad.size == 0, (key, K, bad.size, bad[:5], [hex(int(D[i])) for i in bad[:5]], [hex(int(want[i])) for i in bad[:5]])
 
 
-# ---- config 2: BF16 2048^3 under the Ampere model; sampled outputs and two full rows -----------------------
+# ---- config 2: BF16 2048^3 under the Ampere model; 65 536 sampled outputs and four full lines (two rows, two columns) -----------------------
 def test_cfg2_sampled():
     A, B, C = wl.cfg2()
     inp = {"A": A, "B": B, "C": C}
     key = ("ampere", "bf16", "fp32")
     D = gu.run_gemm(key, inp)
-    pairs = np.concatenate([wl.sample_pairs(2048, 2048, 12288, seed=2),
+    pairs = np.concatenate([wl.sample_pairs(2048, 2048, 65536, seed=2),
                             np.stack([np.full(2048, 5), np.arange(2048)], 1),
+                            np.stack([np.full(2048, 2047), np.arange(2048)], 1),
+                            np.stack([np.arange(2048), np.full(2048, 0)], 1),
                             np.stack([np.arange(2048), np.full(2048, 2047)], 1)])
     gu.assert_samples_equal(D, gu.oracle_samples(key, inp, pairs), pairs, "cfg2")
 
@@ -130,7 +138,7 @@ def test_cfg3_plain_sampled(cfg3_inputs):
     key = ("hopper", "e4m3", "fp32")
     inp = cfg3_inputs
     D = gu.run_gemm(key, inp)
-    pairs = wl.sample_pairs(4096, 4096, 6144, seed=3)
+    pairs = wl.sample_pairs(4096, 4096, 16384, seed=3)
     gu.assert_samples_equal(D, gu.oracle_samples(key, inp, pairs), pairs, "cfg3")
 
 
@@ -138,7 +146,7 @@ def test_cfg3_chunk128_promotion_and_dequant(cfg3_inputs):
     key = ("hopper", "e4m3", "fp32")
     inp = cfg3_inputs
     D = gu.run_gemm(key, inp, k_chunk=128, row_scale=gu.dev(inp["sa"]), col_scale=gu.dev(inp["sb"]))
-    pairs = wl.sample_pairs(4096, 4096, 6144, seed=33)
+    pairs = wl.sample_pairs(4096, 4096, 16384, seed=33)
     want = gu.oracle_samples(key, inp, pairs, k_chunk=128, row_scale=inp["sa"].view(np.uint32),
                              col_scale=inp["sb"].view(np.uint32))
     gu.assert_samples_equal(D, want, pairs, "cfg3 chunk 128")
@@ -159,7 +167,7 @@ def test_independence_of_outputs():
         assert (D == D[0, 0]).all()
 
 
-def test_c_aliases_d_and_leading_dimensions():
+def test_c_aliases_d():
     from paper_2511_10909_b200 import mmasim
     inp = wl.normal_inputs("bf16", "fp32", 40, 24, 64, seed=12)
     key = ("hopper", "bf16", "fp32")

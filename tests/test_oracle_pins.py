@@ -884,3 +884,216 @@ def test_chunk_promotion_composition():
     p1 = phi_dot(m, a[128:], b[128:], 0)
     want = np.float32(np.float32(np.float32(0.3) + np.uint32(p0).view(np.float32)) + np.uint32(p1).view(np.float32))
     assert chunk_promote_dot(m, a, b, c, 128) == int(want.view(np.uint32))
+
+
+# --------------------------------------------------------------------------
+# GTR-FDPA Step 4 (Algorithm 11), worked by hand from the printed steps: F = 24, F2 = 31
+# --------------------------------------------------------------------------
+def test_gtr_step4_T_is_aligned_with_F2_when_c_has_the_larger_exponent():
+    fmt = FORMATS["e5m2"]
+    w = lambda x: exact_word("e5m2", x)
+    # products 2^-14 (slot 0, even group) and 2^-16 (slot 1, odd group); c = 2^10, so E = Exp(c) = 10 > e_max = -14.
+    # T = 2^-14 + 2^-16 exactly (Step 3 keeps 24 fractional bits below 2^-14).
+    # Step 4: T' = RD_31(T * 2^(e_max - E)) has units of 2^(10-31) = 2^-21: both bits of T survive.
+    #         S = 2^10 + 2^-14 + 2^-16, just above the midpoint 2^10 + 2^-14 of the FP32 grid (ulp 2^-13): RNE goes up.
+    # Had T been cut at F = 24 fractional bits (units 2^-14), S would be the exact tie and RNE would return 2^10.
+    a = [w(2.0 ** -7), w(2.0 ** -8)] + [0] * 14
+    b = [w(2.0 ** -7), w(2.0 ** -8)] + [0] * 14
+    d = ops.gtr_fdpa(a, b, f32_word(2.0 ** 10), fmt, fmt, 24, 31)
+    assert d == f32_word(2.0 ** 10 + 2.0 ** -13)
+    # the same with a negative T = -2^-16: RD_31 keeps it exactly, S = 2^10 - 2^-16 rounds (RNE) back to 2^10;
+    # with 24 fractional bits RD would give -2^-14 and S = 2^10 - 2^-14, a representable number
+    a = [w(-(2.0 ** -8))] + [0] * 15
+    b = [w(2.0 ** -8)] + [0] * 15
+    d = ops.gtr_fdpa(a, b, f32_word(2.0 ** 10), fmt, fmt, 24, 31)
+    assert d == f32_word(2.0 ** 10)
+    # a negative T whose only bit lies below 2^-14 but on the F2 grid: -2^-20 is kept, S = 2^10 - 2^-20 -> RNE -> 2^10
+    a = [w(-(2.0 ** -10))] + [0] * 15
+    b = [w(2.0 ** -10)] + [0] * 15
+    assert ops.gtr_fdpa(a, b, f32_word(2.0 ** 10), fmt, fmt, 24, 31) == f32_word(2.0 ** 10)
+
+
+def test_gtr_step4_special_truncation_threshold_and_round_down_of_c():
+    fmt = FORMATS["e5m2"]
+    w = lambda x: exact_word("e5m2", x)
+    a = [w(2.0 ** 10)] + [0] * 15
+    b = [w(2.0 ** 10)] + [0] * 15                          # T = 2^20, e_max = E = 20, units of s_c' are 2^(20-24) = 2^-4
+    g = lambda c: word_f32(ops.gtr_fdpa(a, b, f32_word(c), fmt, fmt, 24, 31))
+    # Exp(c) = -5 = E - F - 1: not below the threshold; RD_24(-2^-5) = -1 unit = -2^-4 (round down, not toward zero)
+    assert g(-(2.0 ** -5)) == 2.0 ** 20 - 2.0 ** -4
+    assert g(-(1.75 * 2.0 ** -5)) == 2.0 ** 20 - 2.0 ** -4
+    # Exp(c) = -6 = E - F - 2 < E - F - 1: special truncation, s_c' = 0 although RD alone would give -1 unit
+    assert g(-(2.0 ** -6)) == 2.0 ** 20
+    assert g(-(1.9999999 * 2.0 ** -6)) == 2.0 ** 20
+    # positive c of the same sizes rounds down to 0 either way
+    assert g(2.0 ** -5) == 2.0 ** 20
+    assert g(2.0 ** -6) == 2.0 ** 20
+    # Exp(c) = -4 = E - F: one full unit, and one unit plus lower bits (negative: floor takes two units)
+    assert g(-(2.0 ** -4)) == 2.0 ** 20 - 2.0 ** -4
+    assert g(-(1.5 * 2.0 ** -4)) == 2.0 ** 20 - 2.0 ** -3
+
+
+def test_gtr_step4_tie_above_power_of_two_goes_to_even():
+    fmt = FORMATS["e5m2"]
+    w = lambda x: exact_word("e5m2", x)
+    a = [w(2.0 ** 10)] + [0] * 15
+    b = [w(2.0 ** 10)] + [0] * 15
+    d = ops.gtr_fdpa(a, b, f32_word(1.5 * 2.0 ** -4), fmt, fmt, 24, 31)   # s_c' = RD(1.5 units) = 1 unit = 2^-4
+    assert word_f32(d) == 2.0 ** 20                                        # 2^20 + 2^-4: tie, even neighbour
+
+
+# --------------------------------------------------------------------------
+# GST-FDPA Step 2 (Algorithm 9): the accumulator term is truncated toward zero like every other term
+# --------------------------------------------------------------------------
+def test_gst_accumulator_term_is_truncated_toward_zero():
+    m = lookup("blackwell", "mxf4", "fp32")
+    a = [0x2] + [0] * 63                                    # 1.0 * 1.0 in group 0, block scale 2^20 * 2^0
+    b = [0x2] + [0] * 63
+    sfa, sfb = [127 + 20, 127], [127, 127]
+    # e_max = 20 (the group's scale exponents), unit of the fused sum 2^(20-35) = 2^-15.
+    # c = -(1 + 2^-23): RZ_35 drops the 2^-23 bit and leaves -1 (floor would leave -(1 + 2^-15)).
+    # S = 2^20 - 1, an FP32 number (ulp 2^-4 below 2^20).  With floor: 2^20 - 1 - 2^-15 -> RZ-FP32 -> 2^20 - 1 - 2^-4.
+    c = f32_word(-(1.0 + 2.0 ** -23))
+    assert phi_dot(m, a, b, c, sfa, sfb) == f32_word(2.0 ** 20 - 1.0)
+    # the mirrored case: RZ of +(1 + 2^-23) is +1 as well
+    c = f32_word(1.0 + 2.0 ** -23)
+    assert phi_dot(m, a, b, c, sfa, sfb) == f32_word(2.0 ** 20 + 1.0)
+    # a negative accumulator entirely below one unit vanishes (floor would subtract a whole unit)
+    c = f32_word(-(2.0 ** -16))
+    assert phi_dot(m, a, b, c, sfa, sfb) == f32_word(2.0 ** 20)
+
+
+# --------------------------------------------------------------------------
+# dequantisation epilogue: D = fl32(fl32(sa * sb) * d), in that order, NaN as the CUDA cores encode it
+# --------------------------------------------------------------------------
+def test_dequant_against_numpy_float32():
+    from oracle.models import dequant
+    rng = np.random.Generator(np.random.Philox(23))
+    n = 4000
+    sa = rng.standard_normal(n).astype(np.float32) * np.float32(3.0)
+    sb = np.exp(rng.standard_normal(n) * 3).astype(np.float32)
+    d = (rng.standard_normal(n) * np.exp(rng.standard_normal(n) * 5)).astype(np.float32)
+    with np.errstate(all="ignore"):
+        want = ((sa * sb) * d).view(np.uint32)
+        other = (sa * (sb * d)).view(np.uint32)
+    assert int((want != other).sum()) > 200            # the order of the two multiplications matters on these inputs
+    for i in range(n):
+        got = dequant(int(d[i:i + 1].view(np.uint32)[0]), int(sa[i:i + 1].view(np.uint32)[0]),
+                      int(sb[i:i + 1].view(np.uint32)[0]))
+        assert got == int(want[i]), i
+    # special values: NaN in any position -> 0x7FFFFFFF; inf * 0 -> NaN; inf * finite -> inf with the product's sign;
+    # overflow of the first product is not undone by a small d
+    inf, nan = f32_word(float("inf")), 0x7FC00001
+    one, zero, big, tiny = f32_word(1.0), 0, f32_word(2.0 ** 100), f32_word(2.0 ** -120)
+    assert dequant(nan, one, one) == 0x7FFFFFFF
+    assert dequant(one, nan, one) == 0x7FFFFFFF
+    assert dequant(one, one, 0xFFC00000) == 0x7FFFFFFF
+    assert dequant(zero, inf, one) == 0x7FFFFFFF
+    assert dequant(f32_word(-2.0), inf, one) == f32_word(float("-inf"))
+    assert dequant(tiny, big, big) == inf              # fl32(2^200) = inf first, then inf * 2^-120
+    assert dequant(big, big, tiny) == f32_word(2.0 ** 80)
+    # subnormal results round to nearest even on the 2^-149 grid
+    assert dequant(f32_word(1.5), f32_word(2.0 ** -75), f32_word(2.0 ** -74)) == 2      # 1.5 * 2^-149 -> 2 * 2^-149
+    assert dequant(f32_word(2.5), f32_word(2.0 ** -75), f32_word(2.0 ** -74)) == 2      # 2.5 units: tie -> even
+
+
+# --------------------------------------------------------------------------
+# TR-/GTR-FDPA: the second-stage alignment of T rounds DOWN (Algorithm 10 Step 3, Algorithm 11 Step 4)
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("family", ["tr", "gtr"])
+def test_tr_gtr_T_is_rounded_down_at_F2(family):
+    # products -2^-15 and -2^-24, c = 2^10: E = 10, one unit of T' is 2^(10-31) = 2^-21.
+    # T = -(64 + 1/8) units: RD gives -65 units (RZ would give -64).  S = 2^10 - 65 * 2^-21 lies beyond the midpoint
+    # 2^10 - 2^-15 of the FP32 grid below 2^10 (spacing 2^-14), so RNE-FP32 gives 2^10 - 2^-14; with -64 units S would
+    # be that midpoint exactly and round to the even neighbour 2^10.
+    name = "fp16" if family == "tr" else "e5m2"
+    fmt = FORMATS[name]
+    w = lambda x: exact_word(name, x)
+    L = 8 if family == "tr" else 16
+    a = [w(-(2.0 ** -8)), w(-(2.0 ** -12))] + [0] * (L - 2)
+    b = [w(2.0 ** -7), w(2.0 ** -12)] + [0] * (L - 2)
+    op = ops.tr_fdpa if family == "tr" else ops.gtr_fdpa
+    assert op(a, b, f32_word(2.0 ** 10), fmt, fmt, 24, 31) == f32_word(2.0 ** 10 - 2.0 ** -14)
+    # the positive mirror image: RD drops the 1/8 unit, S = 2^10 + 2^-15 is a quarter of the FP32 spacing above 2^10
+    # (2^-13) and rounds to 2^10
+    a[0], a[1] = w(2.0 ** -8), w(2.0 ** -12)
+    assert op(a, b, f32_word(2.0 ** 10), fmt, fmt, 24, 31) == f32_word(2.0 ** 10)
+
+
+def test_tr_product_overflow_is_an_infinity_before_the_sum():
+    # Section 4.2: a TR-FDPA product of magnitude >= 2^128 is an infinity, whatever the other terms would cancel
+    fmt = FORMATS["bf16"]
+    w = lambda x: exact_word("bf16", x)
+    z = [0] * 6
+    inf, ninf, nan = f32_word(float("inf")), f32_word(float("-inf")), 0x7FC00000
+    # 2^64 * 2^64 = 2^128 exactly: +inf although the second product takes half of it away again
+    assert ops.tr_fdpa([w(2.0 ** 64), w(-(2.0 ** 63))] + z, [w(2.0 ** 64), w(2.0 ** 64)] + z, 0, fmt, fmt, 24, 31) == inf
+    # +2^128 and -2^128: inf - inf = NaN (the exact sum would be 0)
+    assert ops.tr_fdpa([w(2.0 ** 64), w(-(2.0 ** 64))] + z, [w(2.0 ** 64), w(2.0 ** 64)] + z, 0, fmt, fmt, 24, 31) == nan
+    assert ops.tr_fdpa([w(-(2.0 ** 64))] + [0] * 7, [w(2.0 ** 64)] + [0] * 7, 0, fmt, fmt, 24, 31) == ninf
+    # just below the threshold the product is an ordinary number: (2 - 2^-7) * 2^127 - 2^127 = (1 - 2^-7) * 2^127
+    big = w((2.0 - 2.0 ** -7) * 2.0 ** 63)
+    d = ops.tr_fdpa([big, w(-(2.0 ** 63))] + z, [w(2.0 ** 64), w(2.0 ** 64)] + z, 0, fmt, fmt, 24, 31)
+    assert d == f32_word((1.0 - 2.0 ** -7) * 2.0 ** 127)
+    # and a sum of finite products that reaches 2^128 overflows only in the final conversion
+    d = ops.tr_fdpa([big, big] + z, [w(2.0 ** 64), w(2.0 ** 64)] + z, 0, fmt, fmt, 24, 31)
+    assert d == inf
+
+
+# --------------------------------------------------------------------------
+# zero accumulators have no exponent (the reading the B200 confirms for its FP16 / BF16 rows)
+# --------------------------------------------------------------------------
+def test_zero_accumulator_takes_no_part_in_e_max():
+    # FP16 accumulator +0 (its exponent would be -14): products 2^-25 and 2^-40.  e_max = -25, nothing is cut,
+    # S = 2^-25 + 2^-40 is above the midpoint between 0 and the smallest FP16 number 2^-24: RNE-FP16 gives 2^-24.
+    # Were the zero counted, units of 2^(-14-25) would drop the 2^-40 and the exact tie would go to the even side, 0.
+    m = lookup("blackwell", "fp16", "fp16")
+    w = lambda x: f16_word(x)
+    a = [w(2.0 ** -12), w(2.0 ** -20)] + [0] * 14
+    b = [w(2.0 ** -13), w(2.0 ** -20)] + [0] * 14
+    assert phi_dot(m, a, b, 0) == 0x0001
+    # FP32 accumulator +0 (its exponent would be -126): +2^-149 and -2^-160 under RZ-FP32.  The exact sum is below
+    # 2^-149 and truncates to 0; units of 2^(-126-25) would cut the negative term away first and leave 2^-149.
+    m = lookup("blackwell", "bf16", "fp32")
+    w = lambda x: exact_word("bf16", x)
+    a = [w(2.0 ** -75), w(-(2.0 ** -80))] + [0] * 14
+    b = [w(2.0 ** -74), w(2.0 ** -80)] + [0] * 14
+    assert phi_dot(m, a, b, 0) == 0
+    assert phi_dot(m, a, b, f32_word(-0.0)) == 0
+    # TR-FDPA with c = 0: E = e_max; 2^-150 + 2^-160 is above the midpoint of (0, 2^-149) and rounds up
+    fmt = FORMATS["bf16"]
+    a = [w(2.0 ** -75), w(2.0 ** -80)] + [0] * 6
+    b = [w(2.0 ** -75), w(2.0 ** -80)] + [0] * 6
+    assert ops.tr_fdpa(a, b, 0, fmt, fmt, 24, 31) == 0x00000001
+
+
+# --------------------------------------------------------------------------
+# GST-FDPA Step 2: group terms are truncated toward zero; zero groups and a zero accumulator have no exponent
+# --------------------------------------------------------------------------
+def test_gst_negative_group_term_is_truncated_toward_zero():
+    m = lookup("blackwell", "mxf4", "fp32")
+    a = [0x2] + [0] * 63           # +1.0 in group 0, scaled by 2^36: e_max = 36, one unit of the fused sum is 2
+    b = [0x2] + [0] * 63
+    a[32], b[32] = 0x1, 0x9        # 0.5 * -0.5 = -0.25 in group 2 (second scale block, scale 1)
+    # RZ_35(-0.25 / 2) = 0: S = 2^36.  Rounding down would give -1 unit, 2^36 - 2, and RZ-FP32 then 2^36 - 2^12.
+    assert phi_dot(m, a, b, 0, [127 + 36, 127], [127, 127]) == f32_word(2.0 ** 36)
+
+
+def test_gst_zero_group_and_zero_accumulator_have_no_exponent():
+    m = lookup("blackwell", "mxf4", "fp32")
+    # group 0 and 1 (scale 2^40) hold only zeros, group 2 (scale 1) holds 1.0: the large scale of the empty groups must
+    # not raise e_max, or 1.0 would fall below the unit 2^(40-35)
+    a = [0] * 64
+    b = [0] * 64
+    a[32], b[32] = 0x2, 0x2
+    assert phi_dot(m, a, b, 0, [127 + 40, 127], [127, 127]) == f32_word(1.0)
+    # c = +0: group 0 gives +0.25 * 2^-147 = 2^-149, group 2 gives -0.25 * 2^-163 = -2^-165.  e_max = -147, both terms are
+    # exact, S = 2^-149 - 2^-165 > 0 truncates (RZ-FP32) to +0.  Were the zero accumulator counted with the exponent -126,
+    # units of 2^-161 would cut the negative term to 0 first and leave 2^-149.
+    a = [0x1] + [0] * 63
+    b = [0x1] + [0] * 63
+    a[32], b[32] = 0x1, 0x9
+    assert phi_dot(m, a, b, 0, [27, 27], [80, 64]) == 0
+    # control: with the first group alone the smallest subnormal comes out
+    a[32] = 0
+    assert phi_dot(m, a, b, 0, [27, 27], [80, 64]) == 1
