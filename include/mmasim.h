@@ -140,7 +140,8 @@ int mmasim_dot_batch(const mmasim_model* model, int64_t n, int64_t K,
  * pool and its attributes are not touched.  Pinned host buffers make the copies asynchronous.
  * Problems of 1024 rows and 32 MiB or more are cut into up to eight row panels of D (outputs are independent,
  * Section 3.1 Step 1): B is copied once, then each panel's rows of A and C go in, its kernel runs and its rows of D
- * come back on separate streams, so that with pinned buffers the copies run beside the arithmetic. */
+ * come back on separate streams, so that with pinned buffers the copies run beside the arithmetic.
+ * With opts->ldd > N only the N words of every row of D are written; the words between rows stay the caller's. */
 int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
                      const void* A, const void* B, const void* C, void* D, const mmasim_gemm_opts* opts);
 
@@ -200,7 +201,9 @@ int mmasim_error_stats(int acc_fmt, int64_t n, const void* D, const double* ref,
  *   19 ffma2.rm       packed two-lane fma.rm.f32x2, 8 chains
  *   20 ffma.rn.x16, 21 ffma.rn.x32, 22 ffma.rm.x16, 23 ffma2.rm.x16 (lanes counted), 24 dfma.rn.x16, 25 dfma.rn.x32,
  *   26 dfma.rm.x16    the same instructions with 16 / 32 independent accumulators per thread and loop-invariant
- *                     multiplicands (no operand-fetch conflicts): the second witness of the pipe rates. */
+ *                     multiplicands (no operand-fetch conflicts): the second witness of the pipe rates.
+ *   27 dmma.rm.k4, 28 dmma.rm.k16   the FP64 matrix instruction rounding toward -inf (mma.sync m8n8k4 / m16n8k16),
+ *                     multiply-adds counted. */
 int mmasim_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t* ops_per_round, void* stream);
 
 /* Name of the kernel variant the last mmasim_gemm* call on this thread dispatched to ("generic", ...). */

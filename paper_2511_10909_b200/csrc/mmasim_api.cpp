@@ -110,13 +110,19 @@ int build_args(const mmasim_model* model, int64_t M, int64_t N, int64_t K, const
     return MMASIM_OK;
 }
 
-// Staging memory of mmasim_gemm_host: one memory pool per device, the library's own (the device's default pool and
-// its attributes are the caller's and stay untouched), created on first use, keeping up to 1 GiB between calls.
+}  // namespace
+
+namespace {
+// Device memory the library takes for itself (the staging buffers of mmasim_gemm_host, the decoded operand blocks of
+// the tuned kernels): one memory pool per device, the library's own (the device's default pool and its attributes are
+// the caller's and stay untouched), created on first use, keeping up to 1 GiB between calls.
 constexpr int MAX_DEVICES = 64;
 std::mutex g_pool_mutex;
 cudaMemPool_t g_pools[MAX_DEVICES] = {};
 
-cudaError_t host_pool(cudaMemPool_t* out) {
+}  // namespace
+
+cudaError_t scratch_pool(cudaMemPool_t* out) {
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
@@ -141,7 +147,7 @@ cudaError_t host_pool(cudaMemPool_t* out) {
     return cudaSuccess;
 }
 
-}  // namespace
+
 }  // namespace mmasim
 
 using namespace mmasim;
@@ -299,7 +305,7 @@ int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
         }
     }
     cudaMemPool_t pool = nullptr;
-    if (err == cudaSuccess) err = host_pool(&pool);
+    if (err == cudaSuccess) err = scratch_pool(&pool);
     auto alloc = [&](void** dst, const void* src, size_t bytes) {
         if (err != cudaSuccess || !src || !bytes) return;
         err = cudaMallocFromPoolAsync(dst, bytes, pool, s_in);
@@ -356,8 +362,14 @@ int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
             if (err == cudaSuccess) err = cudaStreamWaitEvent(so, ev_k[p], 0);
             if (err != cudaSuccess) break;
         }
-        err = cudaMemcpyAsync(static_cast<unsigned char*>(D) + d_off, static_cast<unsigned char*>(dD) + d_off, d_len,
-                              cudaMemcpyDeviceToHost, so);
+        // only the N words of every row go back: with ldd > N the words between the rows of the caller's D are not the library's
+        if (host.ldd == N)
+            err = cudaMemcpyAsync(static_cast<unsigned char*>(D) + d_off, static_cast<unsigned char*>(dD) + d_off, d_len,
+                                  cudaMemcpyDeviceToHost, so);
+        else
+            err = cudaMemcpy2DAsync(static_cast<unsigned char*>(D) + d_off, size_t(host.ldd) * info.acc_bytes,
+                                    static_cast<unsigned char*>(dD) + d_off, size_t(host.ldd) * info.acc_bytes,
+                                    size_t(N) * info.acc_bytes, size_t(rows), cudaMemcpyDeviceToHost, so);
     }
     // everything drains, then the buffers go back to the pool in the order of the stream they came from
     cudaStream_t all[] = {s_k[0], s_k[1], s_out};

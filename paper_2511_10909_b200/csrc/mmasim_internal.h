@@ -101,6 +101,7 @@ int launch_error_stats(int acc, int64_t n, const void* D, const double* ref, dou
 // mmasim_peak.cu
 int launch_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t* ops_per_round, cudaStream_t stream);
 // mmasim_api.cpp
+cudaError_t scratch_pool(cudaMemPool_t* out);   // the library's own memory pool of the current device (created on first use)
 void set_error(const char* fmt, ...);
 void set_kernel_name(const char* name);
 }  // namespace mmasim

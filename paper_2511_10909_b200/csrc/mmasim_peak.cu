@@ -9,7 +9,7 @@ namespace {
 enum PeakKind : int {
     PK_IADD3 = 0, PK_LOP3, PK_SHF, PK_IMAD, PK_MACMIX, PK_VIADDMAX, PK_VIADDMAX16X2, PK_F2I, PK_FMUL, PK_POPC,
     PK_IMAD_PLUS_ALU, PK_FMUL_PLUS_ALU, PK_IMAD_WIDE, PK_MAC_D1, PK_MAC_D2, PK_DP4A, PK_DFMA, PK_DFMA_PLUS_ALU, PK_FFMA_RM, PK_FFMA2_RM,
-    PK_FFMA_RN_X16, PK_FFMA_RN_X32, PK_FFMA_RM_X16, PK_FFMA2_RM_X16, PK_DFMA_RN_X16, PK_DFMA_RN_X32, PK_DFMA_RM_X16, PK_COUNT
+    PK_FFMA_RN_X16, PK_FFMA_RN_X32, PK_FFMA_RM_X16, PK_FFMA2_RM_X16, PK_DFMA_RN_X16, PK_DFMA_RN_X32, PK_DFMA_RM_X16, PK_DMMA_RM_K4, PK_DMMA_RM_K16, PK_COUNT
 };
 
 template <int KIND>
@@ -173,6 +173,45 @@ __global__ void __launch_bounds__(256) peak_kernel_fma(int64_t iters, int* sink)
     if (r == T(0.12345)) *sink = 1;
 }
 
+// The FP64 matrix instruction rounding toward minus infinity (mma.sync m8n8k4 with eight independent accumulator tiles per
+// warp, m16n8k16 with four): per thread and round 8 x 8 = 64 and 4 x 64 = 256 multiply-adds.
+template <bool K16>
+__global__ void __launch_bounds__(256) peak_kernel_dmma(int64_t iters, int* sink) {
+    double a[8], b[4], c[8][2];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { a[i] = 1.0 + 1e-9 * double(threadIdx.x + i); c[i][0] = double(i); c[i][1] = double(i) + 0.5; }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) b[i] = 1.0 - 1e-9 * double(threadIdx.x + 2 * i);
+    for (int64_t it = 0; it < iters; ++it) {
+        if (K16) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                asm volatile("mma.sync.aligned.m16n8k16.row.col.rm.f64.f64.f64.f64 {%0,%1,%2,%3}, {%4,%5,%6,%7,%8,%9,%10,%11}, {%12,%13,%14,%15}, {%0,%1,%2,%3};"
+                             : "+d"(c[2 * i][0]), "+d"(c[2 * i][1]), "+d"(c[2 * i + 1][0]), "+d"(c[2 * i + 1][1])
+                             : "d"(a[0]), "d"(a[1]), "d"(a[2]), "d"(a[3]), "d"(a[4]), "d"(a[5]), "d"(a[6]), "d"(a[7]),
+                               "d"(b[0]), "d"(b[1]), "d"(b[2]), "d"(b[3]));
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                asm volatile("mma.sync.aligned.m8n8k4.row.col.rm.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                             : "+d"(c[i][0]), "+d"(c[i][1]) : "d"(a[i & 1]), "d"(b[i & 3]));
+        }
+    }
+    double r = 0.0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) r += c[i][0] + c[i][1];
+    if (r == 0.12345) *sink = 1;
+}
+
+template <bool K16>
+int launch_dmma(int64_t blocks, int64_t iters, void* sink, int32_t* ops_per_round, cudaStream_t stream) {
+    *ops_per_round = K16 ? 256 : 64;
+    peak_kernel_dmma<K16><<<(unsigned)blocks, 256, 0, stream>>>(iters * 8, static_cast<int*>(sink));
+    const cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) { set_error("int_peak launch failed: %s", cudaGetErrorString(err)); return MMASIM_ERR_CUDA; }
+    return MMASIM_OK;
+}
+
 template <typename T, int NACC, bool RM, bool PACKED>
 int launch_fma(int64_t blocks, int64_t iters, void* sink, int32_t* ops_per_round, cudaStream_t stream) {
     // the host counts blocks * 256 * iters8 * 8 * ops_per_round operations, iters8 = iters rounded up to a multiple of 8:
@@ -238,6 +277,8 @@ int launch_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t
         case PK_DFMA_RN_X16: return launch_fma<double, 16, false, false>(blocks, iters, sink, ops_per_round, stream);
         case PK_DFMA_RN_X32: return launch_fma<double, 32, false, false>(blocks, iters, sink, ops_per_round, stream);
         case PK_DFMA_RM_X16: return launch_fma<double, 16, true, false>(blocks, iters, sink, ops_per_round, stream);
+        case PK_DMMA_RM_K4: return launch_dmma<false>(blocks, iters, sink, ops_per_round, stream);
+        case PK_DMMA_RM_K16: return launch_dmma<true>(blocks, iters, sink, ops_per_round, stream);
         default: set_error("mmasim_int_peak: unknown kind %d", kind); return MMASIM_ERR_INVALID_ARG;
     }
 }

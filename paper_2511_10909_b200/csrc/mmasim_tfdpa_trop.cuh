@@ -79,23 +79,24 @@ struct LutEntryT {      // 8 bytes: one shared load per staged element
                         // bit 16: sign; bit 24: finite and nonzero
 };
 
-template <int TH>
-struct PlanesT {
-    static constexpr int BN = Geo<TH>::BN;
-    uint32_t a_op[KC][BM];              // [k][permuted row]
-    uint32_t b_op[KC][BN];              // [k][permuted column]
-    uint16_t a_pe[BM][PE_STRIDE];       // [row][k]
-    uint16_t b_pe[BN][PE_STRIDE];       // [column][k]
-    uint32_t a_sgn[BM], a_nz[BM];       // [permuted row]: bit k = sign / nonzero of element k of the chunk
-    uint32_t b_sgn[BN], b_nz[BN];       // [permuted column]
+// One operand's share of a chunk of KC = 32 elements of K, decoded: R rows of A (or columns of B).  A decode kernel
+// writes these blocks to scratch memory once per GEMM; the main kernel brings them in with one bulk copy each.
+template <int R>
+struct BlkT {
+    uint32_t op[KC][R];                 // [k][permuted row]: FP32 operands
+    uint16_t pe[R][PE_STRIDE];          // [row][k]: BF16 exponent powers for the tensor cores
+    uint32_t sgn[R], nz[R];             // [permuted row]: bit k = sign / nonzero of element k of the chunk
+    uint32_t special;                   // nonzero: the block holds an infinity or a NaN
+    uint32_t pad[3];
 };
+static_assert(sizeof(BlkT<128>) % 16 == 0 && sizeof(BlkT<64>) % 16 == 0, "bulk copies move multiples of 16 bytes");
 
 template <int TH>
 struct SmemT {
-    PlanesT<TH> pl[2];
-    LutEntryT lut_a[256];
-    LutEntryT lut_b[256];
-    int special[3];
+    BlkT<BM> a[2];
+    BlkT<Geo<TH>::BN> b[2];
+    unsigned long long full[2];         // mbarriers: the bulk copies of a buffer have landed
+    int error;                          // a bounded wait ran out
 };
 
 // Position of a row / column of the CTA tile inside the permuted planes: the TH rows of a thread (g, g + 8, ...)
@@ -106,8 +107,8 @@ __device__ __forceinline__ int perm_row(int r) {
 }
 __device__ __forceinline__ int perm_col(int c) { return (c & ~31) | (((c >> 1) & 3) << 3) | (((c >> 3) & 3) << 1) | (c & 1); }
 
-template <int BASE, class SM>
-__device__ __forceinline__ void init_lut_t(SM& s, const FmtDesc& fa, const FmtDesc& fb, int pre, int guard, int tid) {
+template <int BASE>
+__device__ __forceinline__ void init_lut_t(LutEntryT* lut_a, LutEntryT* lut_b, const FmtDesc& fa, const FmtDesc& fb, int pre, int guard, int tid) {
     const uint32_t da = decode_elem(fa, uint32_t(tid)), db = decode_elem(fb, uint32_t(tid));
     const bool fin_a = dec_cls(da) == CLS_FINITE, fin_b = dec_cls(db) == CLS_FINITE;
     const bool nz_a = fin_a && dec_sig(da) != 0u, nz_b = fin_b && dec_sig(db) != 0u;
@@ -121,85 +122,107 @@ __device__ __forceinline__ void init_lut_t(SM& s, const FmtDesc& fa, const FmtDe
     eb.op = nz_b ? __float_as_uint(ldexpf(float(sb * (1 << (pre + guard)) + ub), dec_exp(db) - (fa.mbits + fb.mbits + pre + guard))) : 0u;
     eb.y = (nz_b ? uint32_t((127 + pe_shift(BASE) + BASE * (dec_exp(db) - PE_CENTER)) << 7) : 0u) | (fin_b ? 0u : 0x8000u) |
            (fin_b ? (dec_sign(db) << 16) | (uint32_t(nz_b) << 24) : 0u);
-    s.lut_a[tid] = ea;
-    s.lut_b[tid] = eb;
-}
-
-// Staging of one chunk of KC = 32 elements of K.  Every thread takes sixteen consecutive elements of one row of A (row
-// tid % 128, half tid / 128) and eight or sixteen of one column of B (column tid % BN): the same work for all, so that
-// nobody waits at the barrier.  The raw bytes are fetched one chunk ahead into registers.
-template <int TH>
-struct RawT {
-    uint32_t a[4];
-    uint32_t b[Geo<TH>::NB / 4];
-};
-static_assert(BM == 128 && KC == 32 && NT == 256, "the task split of the staging");
-
-template <int EK, int TH>
-__device__ __forceinline__ void load_chunk_t(RawT<TH>& raw, const GemmArgs& g, int64_t row0, int64_t col0, int64_t k0, int tid) {
-    static_assert(Elem<EK>::BYTES == 1, "8-bit elements");
-    constexpr int BN = Geo<TH>::BN, NB = Geo<TH>::NB;
-    const int64_t i = row0 + (tid & 127), j = col0 + (tid % BN);
-    uint4 va = make_uint4(0u, 0u, 0u, 0u);
-    if (i < g.M) va = *reinterpret_cast<const uint4*>(static_cast<const unsigned char*>(g.A) + i * g.lda + k0 + 16 * (tid >> 7));
-    raw.a[0] = va.x; raw.a[1] = va.y; raw.a[2] = va.z; raw.a[3] = va.w;
-    const unsigned char* pb = static_cast<const unsigned char*>(g.B) + j * g.ldb + k0 + NB * (tid / BN);
-    if (NB == 8) {
-        uint2 vb = make_uint2(0u, 0u);
-        if (j < g.N) vb = *reinterpret_cast<const uint2*>(pb);
-        raw.b[0] = vb.x; raw.b[1] = vb.y;
-    } else {
-        uint4 vb = make_uint4(0u, 0u, 0u, 0u);
-        if (j < g.N) vb = *reinterpret_cast<const uint4*>(pb);
-        raw.b[0] = vb.x; raw.b[1] = vb.y; raw.b[NB / 4 - 2] = vb.z; raw.b[NB / 4 - 1] = vb.w;
-    }
+    lut_a[tid] = ea;
+    lut_b[tid] = eb;
 }
 
 // N = 16 or 8 elements of one row: operands k-major, pe words row-major, sign / nonzero bits into the masks.
-template <int N, bool IS_A, int TH>
-__device__ __forceinline__ uint32_t stage_row(SmemT<TH>& sm, PlanesT<TH>& s, const uint32_t (&w)[N / 4], int r, int part) {
-    const LutEntryT* lut = IS_A ? sm.lut_a : sm.lut_b;
-    const int pr = IS_A ? perm_row<TH>(r) : perm_col(r);
-    uint32_t* op = IS_A ? &s.a_op[part * N][pr] : &s.b_op[part * N][pr];
-    constexpr int STRIDE = IS_A ? BM : Geo<TH>::BN;
+template <int N, int R>
+__device__ __forceinline__ uint32_t stage_row(const LutEntryT* lut, BlkT<R>& s, const uint32_t (&w)[N / 4], int r, int pr, int part) {
+    uint32_t* op = &s.op[part * N][pr];
     uint32_t acc = 0u, spec = 0u, pw[N / 2];
 #pragma unroll
     for (int q = 0; q < N; q += 2) {
         const uint2 e0 = *reinterpret_cast<const uint2*>(&lut[(w[q / 4] >> (8 * (q % 4))) & 0xFFu]);
         const uint2 e1 = *reinterpret_cast<const uint2*>(&lut[(w[q / 4] >> (8 * (q % 4) + 8)) & 0xFFu]);
-        op[q * STRIDE] = e0.x;
-        op[(q + 1) * STRIDE] = e1.x;
+        op[q * R] = e0.x;
+        op[(q + 1) * R] = e1.x;
         // sign byte -> bits 0.., nonzero byte -> bits 16..
         acc += (__byte_perm(e0.y, 0u, 0x4342) << q) + (__byte_perm(e1.y, 0u, 0x4342) << (q + 1));
         spec |= e0.y | e1.y;
         pw[q / 2] = __byte_perm(e0.y, e1.y, 0x5410);
     }
-    uint16_t* pe = IS_A ? &s.a_pe[r][part * N] : &s.b_pe[r][part * N];
+    uint16_t* pe = &s.pe[r][part * N];
 #pragma unroll
     for (int q = 0; q < N / 8; ++q)
         reinterpret_cast<uint4*>(pe)[q] = make_uint4(pw[4 * q], pw[4 * q + 1], pw[4 * q + 2], pw[4 * q + 3]);
-    uint32_t* sgn = IS_A ? &s.a_sgn[pr] : &s.b_sgn[pr];
-    uint32_t* nz = IS_A ? &s.a_nz[pr] : &s.b_nz[pr];
     if (N == 16) {
-        reinterpret_cast<uint16_t*>(sgn)[part] = uint16_t(acc);
-        reinterpret_cast<uint16_t*>(nz)[part] = uint16_t(acc >> 16);
+        reinterpret_cast<uint16_t*>(&s.sgn[pr])[part] = uint16_t(acc);
+        reinterpret_cast<uint16_t*>(&s.nz[pr])[part] = uint16_t(acc >> 16);
     } else {
-        reinterpret_cast<uint8_t*>(sgn)[part] = uint8_t(acc);
-        reinterpret_cast<uint8_t*>(nz)[part] = uint8_t(acc >> 16);
+        reinterpret_cast<uint8_t*>(&s.sgn[pr])[part] = uint8_t(acc);
+        reinterpret_cast<uint8_t*>(&s.nz[pr])[part] = uint8_t(acc >> 16);
     }
     return spec;
 }
 
-template <int TH>
-__device__ __forceinline__ void store_chunk_t(SmemT<TH>& sm, PlanesT<TH>& s, const RawT<TH>& raw, int flag, int tid) {
-    constexpr int BN = Geo<TH>::BN, NB = Geo<TH>::NB;
-    const uint32_t spec = stage_row<16, true, TH>(sm, s, raw.a, tid & 127, tid >> 7) |
-                          stage_row<NB, false, TH>(sm, s, raw.b, tid % BN, tid / BN);
-    if (spec & 0x8000u) atomicOr(&sm.special[flag], 1);
+// Decode pass: one CTA decodes one block (R rows of A or columns of B x 32 elements of K) through a 256-entry table of
+// 8-byte entries into shared memory and copies it to its place in the scratch array dst[tile][chunk].  Every thread
+// takes 16 (R = 128) or 8 (R = 64) consecutive elements of one row.  Rows beyond the matrix decode as zeros.
+static_assert(BM == 128 && KC == 32 && NT == 256, "the task split of the decode pass");
+template <int BASE, int R, bool IS_A, int TH>
+__global__ void __launch_bounds__(NT) trop_decode_kernel(DevModel m, const unsigned char* src, int64_t rows, int64_t ld, int F,
+                                                         BlkT<R>* dst) {
+    __shared__ __align__(16) LutEntryT lut_a[256];
+    __shared__ __align__(16) LutEntryT lut_b[256];
+    __shared__ __align__(16) BlkT<R> blk;
+    const int tid = threadIdx.x;
+    const FmtDesc fa = fmt_desc(m.fmt_a), fb = fmt_desc(m.fmt_b);
+    init_lut_t<BASE>(lut_a, lut_b, fa, fb, F - (fa.mbits + fb.mbits), fa.mbits + 1, tid);
+    if (tid == 0) { blk.special = 0u; blk.pad[0] = blk.pad[1] = blk.pad[2] = 0u; }
+    constexpr int N = R * KC / NT;                      // elements per thread: 16 or 8
+    const int r = tid % R, part = tid / R;
+    const int64_t i = int64_t(blockIdx.y) * R + r, k0 = int64_t(blockIdx.x) * KC;
+    uint32_t w[N / 4];
+    if (N == 16) {
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (i < rows) v = *reinterpret_cast<const uint4*>(src + i * ld + k0 + N * part);
+        w[0] = v.x; w[1] = v.y; w[N / 4 - 2] = v.z; w[N / 4 - 1] = v.w;
+    } else {
+        uint2 v = make_uint2(0u, 0u);
+        if (i < rows) v = *reinterpret_cast<const uint2*>(src + i * ld + k0 + N * part);
+        w[0] = v.x; w[1] = v.y;
+    }
+    __syncthreads();
+    const uint32_t spec = stage_row<N, R>(IS_A ? lut_a : lut_b, blk, w, r, IS_A ? perm_row<TH>(r) : perm_col(r), part);
+    if (spec & 0x8000u) atomicOr(&blk.special, 1u);
+    __syncthreads();
+    uint4* out = reinterpret_cast<uint4*>(dst + (int64_t(blockIdx.y) * gridDim.x + blockIdx.x));
+    const uint4* in = reinterpret_cast<const uint4*>(&blk);
+    for (int q = tid; q < int(sizeof(BlkT<R>) / 16); q += NT) out[q] = in[q];
 }
 
+// ---- bulk copies and their barrier: inline PTX ----
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return uint32_t(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+// Waits for the given phase of the barrier; gives up after a bounded number of polls (each poll itself blocks for a
+// bounded, implementation-defined time) and returns false.
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity) {
+    const uint32_t addr = smem_addr(bar);
+    for (int spin = 0; spin < (1 << 22); ++spin) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+// Set when a bounded wait on a bulk copy ran out (never in a healthy run); read by mmasim_device_status.
+__device__ unsigned int g_trop_timeouts = 0u;
+
 template <int EK, int L, int F, int RHO, bool PROMOTE, int BASE, int TH>
-__global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs g) {
+__global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs g, const BlkT<BM>* __restrict__ wa,
+                                                           const BlkT<Geo<TH>::BN>* __restrict__ wb) {
     constexpr bool ACC16 = RHO == RHO_RNE_FP16;
     constexpr int NBLK = KC / L;
     static_assert(KC % L == 0 && L % 16 == 0, "a block is one or two k16 matrix instructions");
@@ -240,8 +263,24 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
     constexpr uint32_t E_HIGH = (241u << 23) - 1u;
     constexpr uint32_t E_KEEP = 243u << 23, KEEP = E_KEEP + MAGIC_ADD;
     static_assert(F == 13 || ACC16, "the kept word is carried as its upper 22 bits");
-    if (tid < 256) init_lut_t<BASE>(sm, fa, fb, pre, guard, tid);
-    if (tid == 0) sm.special[0] = sm.special[1] = sm.special[2] = 0;
+    // the decoded blocks of this tile row of A and tile column of B, chunk after chunk, land in two buffers by bulk copies
+    const int K = int(g.K), NCH = K / KC;
+    const BlkT<BM>* src_a = wa + int64_t(blockIdx.y) * NCH;
+    const BlkT<BN>* src_b = wb + int64_t(blockIdx.x) * NCH;
+    auto issue = [&](int n) {                              // one thread: both copies of chunk n into buffer n & 1
+        unsigned long long* bar = &sm.full[n & 1];
+        mbar_expect_tx(bar, uint32_t(sizeof(BlkT<BM>) + sizeof(BlkT<BN>)));
+        bulk_load(&sm.a[n & 1], src_a + n, uint32_t(sizeof(BlkT<BM>)), bar);
+        bulk_load(&sm.b[n & 1], src_b + n, uint32_t(sizeof(BlkT<BN>)), bar);
+    };
+    if (tid == 0) {
+        sm.error = 0;
+        mbar_init(&sm.full[0], 1u);
+        mbar_init(&sm.full[1], 1u);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        issue(0);
+        if (NCH > 1) issue(1);
+    }
 
     uint32_t cw[TH][TW];
     mask_t sp_nan = 0, sp_pinf = 0, sp_ninf = 0;        // per output (bit h * TW + x)
@@ -267,22 +306,15 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
             cw[h][x] = w;
         }
 
-    RawT<TH> raw;
-    load_chunk_t<EK, TH>(raw, g, row0, col0, 0, tid);
-    __syncthreads();                                       // tables and flags are ready
-    store_chunk_t<TH>(sm, sm.pl[0], raw, 0, tid);
-    if (KC < g.K) load_chunk_t<EK, TH>(raw, g, row0, col0, KC, tid);
-    __syncthreads();
-    int chunk = 0;
-    const int K = int(g.K);
-    for (int k0 = 0; k0 < K; k0 += KC, ++chunk) {
-        if (tid == 0) sm.special[(chunk + 2) % 3] = 0;
-        if (k0 + KC < K) {
-            store_chunk_t<TH>(sm, sm.pl[(chunk + 1) & 1], raw, (chunk + 1) % 3, tid);
-            if (k0 + 2 * KC < K) load_chunk_t<EK, TH>(raw, g, row0, col0, k0 + 2 * KC, tid);
-        }
-        PlanesT<TH>& s = sm.pl[chunk & 1];
-        const bool chunk_special = sm.special[chunk % 3] != 0;
+    __syncthreads();                                       // the barriers are initialised
+    for (int chunk = 0; chunk < NCH; ++chunk) {
+        const int k0 = chunk * KC;
+        // a wait that runs out is recorded and the chunk computed on whatever is there; every thread sees the flag after
+        // the barrier at the end of the chunk, and the CTA leaves together without storing anything
+        if (!mbar_wait(&sm.full[chunk & 1], uint32_t(chunk >> 1) & 1u)) *reinterpret_cast<volatile int*>(&sm.error) = 1;
+        const BlkT<BM>& sa_blk = sm.a[chunk & 1];
+        const BlkT<BN>& sb_blk = sm.b[chunk & 1];
+        const bool chunk_special = (sa_blk.special | sb_blk.special) != 0u;
 
 #pragma unroll 1
         for (int blk = 0; blk < NBLK; ++blk) {
@@ -323,11 +355,11 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
 #pragma unroll
                     for (int ks = 0; ks < NK; ++ks) {
                         const int kq = kb + sub * KSUB + 16 * ks + 2 * tq;
-                        af[ks][0] = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar][kq]);
-                        af[ks][1] = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar + 8][kq]);
+                        af[ks][0] = *reinterpret_cast<const uint32_t*>(&sa_blk.pe[ar][kq]);
+                        af[ks][1] = *reinterpret_cast<const uint32_t*>(&sa_blk.pe[ar + 8][kq]);
                         if (AR == 4) {
-                            af[ks][AR - 2] = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar][kq + 8]);
-                            af[ks][AR - 1] = *reinterpret_cast<const uint32_t*>(&s.a_pe[ar + 8][kq + 8]);
+                            af[ks][AR - 2] = *reinterpret_cast<const uint32_t*>(&sa_blk.pe[ar][kq + 8]);
+                            af[ks][AR - 1] = *reinterpret_cast<const uint32_t*>(&sa_blk.pe[ar + 8][kq + 8]);
                         }
                     }
 #pragma unroll
@@ -336,8 +368,8 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
 #pragma unroll
                         for (int ks = 0; ks < NK; ++ks) {
                             const int kq = kb + sub * KSUB + 16 * ks + 2 * tq;
-                            bf[ks][0] = *reinterpret_cast<const uint32_t*>(&s.b_pe[wc * 32 + 8 * j + gq][kq]);
-                            if (BR == 2) bf[ks][BR - 1] = *reinterpret_cast<const uint32_t*>(&s.b_pe[wc * 32 + 8 * j + gq][kq + 8]);
+                            bf[ks][0] = *reinterpret_cast<const uint32_t*>(&sb_blk.pe[wc * 32 + 8 * j + gq][kq]);
+                            if (BR == 2) bf[ks][BR - 1] = *reinterpret_cast<const uint32_t*>(&sb_blk.pe[wc * 32 + 8 * j + gq][kq + 8]);
                         }
                         float d[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -423,11 +455,11 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
                     float oas[TH];
 #pragma unroll
                     for (int q = 0; q < TH / 4; ++q) {
-                        const float4 oa = *reinterpret_cast<const float4*>(&s.a_op[kk][wr * G::WROWS + TH * gq + 4 * q]);
+                        const float4 oa = *reinterpret_cast<const float4*>(&sa_blk.op[kk][wr * G::WROWS + TH * gq + 4 * q]);
                         oas[4 * q] = oa.x; oas[4 * q + 1] = oa.y; oas[4 * q + 2] = oa.z; oas[4 * q + 3] = oa.w;
                     }
-                    const ulonglong2 ob0 = *reinterpret_cast<const ulonglong2*>(&s.b_op[kk][wc * 32 + 8 * tq]);
-                    const ulonglong2 ob1 = *reinterpret_cast<const ulonglong2*>(&s.b_op[kk][wc * 32 + 8 * tq + 4]);
+                    const ulonglong2 ob0 = *reinterpret_cast<const ulonglong2*>(&sb_blk.op[kk][wc * 32 + 8 * tq]);
+                    const ulonglong2 ob1 = *reinterpret_cast<const ulonglong2*>(&sb_blk.op[kk][wc * 32 + 8 * tq + 4]);
                     const unsigned long long obv[TW / 2] = {ob0.x, ob0.y, ob1.x, ob1.y};
 #pragma unroll
                     for (int h = 0; h < TH; ++h) {
@@ -450,16 +482,16 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
             uint32_t sbv[TW], nzb[TW];
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
-                const uint4 u = *reinterpret_cast<const uint4*>(&s.b_sgn[wc * 32 + 8 * tq + 4 * q]);
-                const uint4 v = *reinterpret_cast<const uint4*>(&s.b_nz[wc * 32 + 8 * tq + 4 * q]);
+                const uint4 u = *reinterpret_cast<const uint4*>(&sb_blk.sgn[wc * 32 + 8 * tq + 4 * q]);
+                const uint4 v = *reinterpret_cast<const uint4*>(&sb_blk.nz[wc * 32 + 8 * tq + 4 * q]);
                 sbv[4 * q] = u.x; sbv[4 * q + 1] = u.y; sbv[4 * q + 2] = u.z; sbv[4 * q + 3] = u.w;
                 nzb[4 * q] = v.x; nzb[4 * q + 1] = v.y; nzb[4 * q + 2] = v.z; nzb[4 * q + 3] = v.w;
             }
             auto finish = [&](auto with_markers) {
 #pragma unroll
                 for (int h = 0; h < TH; ++h) {
-                    const uint32_t sa = s.a_sgn[wr * G::WROWS + TH * gq + h];
-                    const uint32_t nza = s.a_nz[wr * G::WROWS + TH * gq + h] & kmask;
+                    const uint32_t sa = sa_blk.sgn[wr * G::WROWS + TH * gq + h];
+                    const uint32_t nza = sa_blk.nz[wr * G::WROWS + TH * gq + h] & kmask;
 #pragma unroll
                     for (int x = 0; x < TW; ++x) {
                         // every negative nonzero term fell one unit short: bits + count is (1.5 * 2^23 + S) * unit
@@ -486,7 +518,9 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
                         }
             }
         }
-        __syncthreads();                                   // the other buffer is complete, this one is free
+        __syncthreads();                                   // everybody has finished with this buffer
+        if (*reinterpret_cast<volatile int*>(&sm.error)) break;
+        if (tid == 0 && chunk + 2 < NCH) issue(chunk + 2);
         if (PROMOTE && ((k0 + KC) % int(g.k_chunk)) == 0) {     // FP32 promotion of the partial sum every k_chunk elements
 #pragma unroll
             for (int h = 0; h < TH; ++h)
@@ -502,6 +536,14 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
         }
     }
 
+    if (*reinterpret_cast<volatile int*>(&sm.error)) {     // a copy never arrived: count it, give the copies in flight one more
+        if (tid == 0) {                                    // bounded wait each, and store nothing
+            atomicAdd(&g_trop_timeouts, 1u);
+            mbar_wait(&sm.full[0], 0u);
+            mbar_wait(&sm.full[1], 0u);
+        }
+        return;
+    }
 #pragma unroll
     for (int h = 0; h < TH; ++h)
 #pragma unroll
@@ -525,12 +567,28 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
 
 template <int EK, int L, int F, int RHO, bool PROMOTE, int BASE, int TH>
 cudaError_t launch_one_t(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
+    constexpr int BN = Geo<TH>::BN;
     const size_t sh = sizeof(SmemT<TH>);
     cudaError_t err = cudaFuncSetAttribute(tfdpa_trop_kernel<EK, L, F, RHO, PROMOTE, BASE, TH>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
     if (err != cudaSuccess) return err;
-    dim3 grid((unsigned)((g.N + Geo<TH>::BN - 1) / Geo<TH>::BN), (unsigned)((g.M + BM - 1) / BM), 1);
-    tfdpa_trop_kernel<EK, L, F, RHO, PROMOTE, BASE, TH><<<grid, NT, sh, stream>>>(m, g);
-    return cudaGetLastError();
+    const int64_t tiles_m = (g.M + BM - 1) / BM, tiles_n = (g.N + BN - 1) / BN, nch = g.K / KC;
+    // scratch: the decoded blocks of A and B, stream-ordered out of the library's pool and returned to it behind the kernel
+    const size_t bytes_a = size_t(tiles_m * nch) * sizeof(BlkT<BM>), bytes_b = size_t(tiles_n * nch) * sizeof(BlkT<BN>);
+    cudaMemPool_t pool = nullptr;
+    if ((err = scratch_pool(&pool)) != cudaSuccess) return err;
+    void* ws = nullptr;
+    if ((err = cudaMallocFromPoolAsync(&ws, bytes_a + bytes_b, pool, stream)) != cudaSuccess) return err;
+    BlkT<BM>* wa = static_cast<BlkT<BM>*>(ws);
+    BlkT<BN>* wb = reinterpret_cast<BlkT<BN>*>(static_cast<unsigned char*>(ws) + bytes_a);
+    trop_decode_kernel<BASE, BM, true, TH><<<dim3((unsigned)nch, (unsigned)tiles_m), NT, 0, stream>>>(
+        m, static_cast<const unsigned char*>(g.A), g.M, g.lda, F, wa);
+    trop_decode_kernel<BASE, BN, false, TH><<<dim3((unsigned)nch, (unsigned)tiles_n), NT, 0, stream>>>(
+        m, static_cast<const unsigned char*>(g.B), g.N, g.ldb, F, wb);
+    dim3 grid((unsigned)tiles_n, (unsigned)tiles_m, 1);
+    tfdpa_trop_kernel<EK, L, F, RHO, PROMOTE, BASE, TH><<<grid, NT, sh, stream>>>(m, g, wa, wb);
+    err = cudaGetLastError();
+    const cudaError_t err2 = cudaFreeAsync(ws, stream);
+    return err != cudaSuccess ? err : err2;
 }
 
 // The tall micro-tile where the registers allow it: FP32 accumulators without promoted partial sums beside them.
