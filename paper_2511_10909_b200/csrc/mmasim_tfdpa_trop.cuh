@@ -52,13 +52,14 @@ constexpr int PE_CENTER = 1;            // pe(x) = 2^(6 (Exp(x) - PE_CENTER)); E
 // pe(x) = 2^(BASE (Exp(x) - PE_CENTER)), the B plane times 2^pe_shift so that 127 + pe_shift is a multiple of BASE and
 // the exponent field of P is BASE * (e_max + constant) + 0..BASE-1.  A sum of at most 2^(BASE-1) terms stays within a
 // factor 2^(BASE-1) of its largest term; the spread of the exponents decides which BASE fits the FP32 range:
-//   BASE 6: blocks of up to 32 terms in one accumulation; E4M3 x E4M3 (product exponents -12..16: 6 * 28 = 168 binades)
+//   BASE 8: blocks of up to 32 terms in one accumulation; E4M3 x E4M3 (product exponents -12..16: 8 * 28 = 224 binades,
+//           plus the 5 binades a sum of 32 terms can grow; the division by 8 is a shift)
 //   BASE 5: sub-blocks of 16 terms; E4M3 x E5M2 (-20..23: 5 * 43 = 215 binades)
 //   BASE 4: sub-blocks of 8 terms;  E5M2 x E5M2 (-28..30: 4 * 58 = 232 binades)
 // The block maximum is then the integer maximum of the sub-blocks' P words.
-__host__ __device__ constexpr int pe_shift(int base) { return base == 6 ? 5 : (base == 5 ? 3 : 1); }
-__host__ __device__ constexpr int pe_sub(int base) { return base == 6 ? 32 : (base == 5 ? 16 : 8); }
-__host__ __device__ constexpr uint32_t pe_mul(int base) { return base == 6 ? 0x2AAAAAABu : (base == 5 ? 0x33333334u : 0x40000000u); }  // ceil(2^32 / BASE)
+__host__ __device__ constexpr int pe_shift(int base) { return base == 8 ? 1 : (base == 5 ? 3 : 1); }
+__host__ __device__ constexpr int pe_sub(int base) { return base == 8 ? 32 : (base == 5 ? 16 : 8); }
+__host__ __device__ constexpr uint32_t pe_mul(int base) { return base == 5 ? 0x33333334u : 0u; }  // ceil(2^32 / BASE); powers of two shift
 constexpr int TW = 8;                   // micro-tile: TH rows x 8 columns
 
 // Geometry by the height TH of the micro-tile.  TH = 4: warps 4 x 2, warp tile 32 x 32, CTA tile 128 x 64.
@@ -226,7 +227,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
     constexpr bool ACC16 = RHO == RHO_RNE_FP16;
     constexpr int NBLK = KC / L;
     static_assert(KC % L == 0 && L % 16 == 0, "a block is one or two k16 matrix instructions");
-    static_assert(BASE == 4 || BASE == 5 || BASE == 6, "see pe_shift");
+    static_assert(BASE == 4 || BASE == 5 || BASE == 8, "see pe_shift");
     constexpr int KSUB = pe_sub(BASE) < L ? pe_sub(BASE) : L, NSUB = L / KSUB;        // terms per accumulation of P
     static_assert(!Elem<EK>::SIGNMAG && F <= 13, "8-bit inputs with F <= 13");
     static_assert(RHO == RHO_RZ_E8M13 || RHO == RHO_RNE_FP16, "rho of the F = 13 rows of Table 4");
@@ -254,6 +255,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
     // Sum register: (1.5 * 2^23 + S) * 2^(e_max - F), exponent field e + (23 - F).
     constexpr uint32_t MUL = pe_mul(BASE), T1_ADD = uint32_t(127 - (127 + pe_shift(BASE)) / BASE + 2 * PE_CENTER) << 23;
     constexpr uint32_t FIELD = 0x7F800000u, HALF = 0x00400000u;
+    constexpr uint32_t RHO_MASK = ACC16 ? 0xFFFFFFFFu : 0xFFFFFC00u;   // RZ-E8M13 of an FP32 word whose exponent stays
     constexpr uint32_t MAGIC_ADD = (uint32_t(23 - F) << 23) | HALF;
     // Below E_LOW no product is nonzero, above E_HIGH the register would overflow (and every product is far below one
     // unit of the accumulator): the result is rho of the accumulator alone.  Such an output rides through pass 2 as a
@@ -397,17 +399,19 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
                     for (int x = 0; x < TW; ++x) {
                         const int h = 2 * mt + hh;
                         uint32_t& p = P[x >> 1][2 * hh + (x & 1)];
-                        const uint32_t t1 = __umulhi(p, MUL) + T1_ADD;
+                        const uint32_t t1 = (BASE == 5 ? __umulhi(p, MUL) : (p >> (BASE == 8 ? 3 : 2))) + T1_ADD;
                         uint32_t e;
                         if (ACC16) {
                             // a subnormal FP16 accumulator has the exponent -14, not that of its leading bit.  BASE 6: the
                             // floor also covers c = 0, harmlessly (every nonzero E4M3 product has an exponent of at least
                             // -12); with E5M2 operands products reach down to 2^-28 and a zero accumulator must not count
                             uint32_t ca = __float_as_uint(__half2float(__ushort_as_half((unsigned short)(cw[h][x] & 0x7FFFu))));
-                            if (BASE == 6) e = uint32_t(__vimax3_s32(int(t1), int(ca), int(113u << 23)));
+                            if (BASE == 8) e = uint32_t(__vimax3_s32(int(t1), int(ca), int(113u << 23)));
                             else { if (ca) ca = max(ca, 113u << 23); e = max(t1, ca); }
                         } else {
-                            e = max(t1, cw[h][x] & 0x7FFFFFFFu);
+                            // |c| and t1 are positive FP32 patterns: their order as numbers is their order as words, and
+                            // the absolute value rides on the instruction
+                            e = __float_as_uint(fmaxf(__uint_as_float(t1), fabsf(__uint_as_float(cw[h][x]))));
                             out_of_range = __viaddmax_u32(e, 0u - E_LOW, out_of_range);
                         }
                         p = e;
@@ -432,13 +436,19 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh)
 #pragma unroll
-                    for (int x = 0; x < TW; ++x) {
+                    for (int xp = 0; xp < TW / 2; ++xp) {          // two adjacent columns per packed addition
                         const int h = 2 * mt + hh;
-                        const uint32_t e = P[x >> 1][2 * hh + (x & 1)];
-                        const uint32_t c = cw[h][x];
-                        const uint32_t magic = (e & FIELD) + MAGIC_ADD + (c >> (ACC16 ? 15 : 31));
-                        const float cf = ACC16 ? __half2float(__ushort_as_half((unsigned short)c)) : __uint_as_float(c);
-                        cw[h][x] = __float_as_uint(__fadd_rd(__uint_as_float(__float_as_uint(cf) | 1u), __uint_as_float(magic)));
+                        uint32_t magic[2], cb[2];
+#pragma unroll
+                        for (int q = 0; q < 2; ++q) {
+                            const uint32_t e = P[xp][2 * hh + q];
+                            const uint32_t c = cw[h][2 * xp + q];
+                            magic[q] = (e & FIELD) + MAGIC_ADD + (c >> (ACC16 ? 15 : 31));
+                            const float cf = ACC16 ? __half2float(__ushort_as_half((unsigned short)c)) : __uint_as_float(c);
+                            cb[q] = __float_as_uint(cf) | 1u;
+                        }
+                        asm("{\n\t.reg .b64 a, b, r;\n\tmov.b64 a, {%2, %3};\n\tmov.b64 b, {%4, %5};\n\tadd.rm.f32x2 r, a, b;\n\tmov.b64 {%0, %1}, r;\n\t}"
+                            : "=r"(cw[h][2 * xp]), "=r"(cw[h][2 * xp + 1]) : "r"(cb[0]), "r"(cb[1]), "r"(magic[0]), "r"(magic[1]));
                     }
             }
             // ---- pass 2: one fused multiply-add per term, rounding toward minus infinity onto the grid of S; two
@@ -492,14 +502,23 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
                 for (int h = 0; h < TH; ++h) {
                     const uint32_t sa = sa_blk.sgn[wr * G::WROWS + TH * gq + h];
                     const uint32_t nza = sa_blk.nz[wr * G::WROWS + TH * gq + h] & kmask;
+                    uint32_t bitsv[TW], vv[TW];
+#pragma unroll
+                    for (int x = 0; x < TW; ++x)                   // every negative nonzero term fell one unit short:
+                        bitsv[x] = cw[h][x] + uint32_t(__popc((sa ^ sbv[x]) & nza & nzb[x]));   // (1.5 * 2^23 + S) * unit
+#pragma unroll
+                    for (int xp = 0; xp < TW / 2; ++xp)            // S * unit, exact; two columns per packed subtraction
+                        asm("{\n\t.reg .b64 a, b, r;\n\tmov.b64 a, {%2, %3};\n\tmov.b64 b, {%4, %5};\n\tsub.rn.f32x2 r, a, b;\n\tmov.b64 {%0, %1}, r;\n\t}"
+                            : "=r"(vv[2 * xp]), "=r"(vv[2 * xp + 1])
+                            : "r"(bitsv[2 * xp]), "r"(bitsv[2 * xp + 1]), "r"((bitsv[2 * xp] & FIELD) | HALF), "r"((bitsv[2 * xp + 1] & FIELD) | HALF));
 #pragma unroll
                     for (int x = 0; x < TW; ++x) {
-                        // every negative nonzero term fell one unit short: bits + count is (1.5 * 2^23 + S) * unit
-                        const uint32_t bits = cw[h][x] + uint32_t(__popc((sa ^ sbv[x]) & nza & nzb[x]));
-                        const float v = __fsub_rn(__uint_as_float(bits), __uint_as_float((bits & FIELD) | HALF));   // S * unit, exact
+                        const uint32_t bits = bitsv[x];
+                        const float v = __uint_as_float(vv[x]);
                         uint32_t w;
                         if (ACC16) { w = uint32_t(__half_as_ushort(__float2half_rn(v))); wmax = max(wmax, w & 0x7FFFu); }
-                        else w = __float_as_uint(v) & 0xFFFFFC00u;
+                        else w = __float_as_uint(v);     // RZ-E8M13 is applied where the word leaves the chain (below): the next
+                                                         // block's alignment truncates on a grid at least as coarse
                         if (decltype(with_markers)::value && bits >= KEEP) w = (bits - KEEP) << 10;
                         cw[h][x] = w;
                     }
@@ -526,7 +545,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
             for (int h = 0; h < TH; ++h)
 #pragma unroll
                 for (int x = 0; x < TW; ++x) {
-                    const float part = __uint_as_float(MMASIM_SP_WORD(h, x, cw[h][x]));
+                    const float part = __uint_as_float(MMASIM_SP_WORD(h, x, cw[h][x] & RHO_MASK));
                     float v = __fadd_rn(promoted[PROMOTE ? h : 0][PROMOTE ? x : 0], part);
                     if (v != v) v = __uint_as_float(0x7FFFFFFFu);
                     promoted[PROMOTE ? h : 0][PROMOTE ? x : 0] = v;
@@ -550,7 +569,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
         for (int x = 0; x < TW; ++x) {
             const int64_t i = row0 + row_of(h), j = col0 + col_of(x);
             if (i >= g.M || j >= g.N) continue;
-            uint32_t w = PROMOTE ? __float_as_uint(promoted[PROMOTE ? h : 0][PROMOTE ? x : 0]) : MMASIM_SP_WORD(h, x, cw[h][x]);
+            uint32_t w = PROMOTE ? __float_as_uint(promoted[PROMOTE ? h : 0][PROMOTE ? x : 0]) : MMASIM_SP_WORD(h, x, cw[h][x] & RHO_MASK);
             if (g.row_scale) {
                 float sc = __fmul_rn(g.row_scale[i], g.col_scale[j]);
                 if (sc != sc) sc = __uint_as_float(0x7FFFFFFFu);
@@ -607,7 +626,7 @@ template <int EK, int L, int F, int RHO>
 cudaError_t launch_by_types_t(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
     const int wide = (m.fmt_a == EF_E5M2) + (m.fmt_b == EF_E5M2);
     if ((m.fmt_a != EF_E4M3 && m.fmt_a != EF_E5M2) || (m.fmt_b != EF_E4M3 && m.fmt_b != EF_E5M2)) return cudaErrorInvalidValue;
-    if (wide == 0) return launch_variant_t<EK, L, F, RHO, 6>(m, g, stream);
+    if (wide == 0) return launch_variant_t<EK, L, F, RHO, 8>(m, g, stream);
     if (wide == 1) return launch_variant_t<EK, L, F, RHO, 5>(m, g, stream);
     return launch_variant_t<EK, L, F, RHO, 4>(m, g, stream);
 }
