@@ -126,6 +126,27 @@ int mmasim_gemm_ex(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
                    const void* A, const void* B, const void* C, void* D,
                    const mmasim_gemm_opts* opts, void* stream);
 
+/* mmasim_gemm_ex without any device-memory allocation, for callers that cannot allocate when they call: code inside a
+ * region where the allocator must not be touched (a latency-critical loop, a thread that may not take the allocator's
+ * locks, a process whose memory budget is fixed at start-up), where mmasim_gemm_ex would take stream-ordered scratch
+ * out of the library's pool.  The paper has no counterpart; this is a property of the library, not of a model.
+ *   - Serves the FP8 models with F = 13 (the Ada and Hopper FP8 rows of Table 4, A and B in E4M3 or E5M2), K a multiple
+ *     of 32, row strides of A and B multiples of 16 bytes; anything else returns MMASIM_ERR_UNSUPPORTED.  Inputs,
+ *     outputs and opts (k_chunk, row_scale / col_scale, leading dimensions) as for mmasim_gemm_ex; results are the same
+ *     words.
+ *   - The scratch (the decoded operands: about (ceil(M/128) + ceil(N/128)) * K/32 * 27 KiB, with 64-column tiles of B
+ *     for FP16 accumulators and k_chunk) lives in a fixed 32 MiB device array that every GPU loading the library holds
+ *     until the process ends.  A problem that needs more returns MMASIM_ERR_SHAPE and the message states both sizes
+ *     (1024 x 1024 x 1024 needs 14 MiB; 2048 x 2048 x 512 fits, 2048^3 does not).
+ *   - The first call on each device looks the array's address up (with that device current); make that first call
+ *     outside any stream capture.  No call allocates or frees device memory.
+ *   - All calls share the one array, which keeps the previous call's contents; every call rewrites the part it reads,
+ *     so nothing has to be cleared.  Two calls whose work overlaps on the GPU (different streams, or one stream of each
+ *     of two host threads) race on it: order them on one stream or with events. */
+int mmasim_gemm_noalloc(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
+                        const void* A, const void* B, const void* C, void* D,
+                        const mmasim_gemm_opts* opts, void* stream);
+
 /* n independent dot-product-accumulates d_t = Phi(a_t, b_t, c_t) (Equation 4), the shape of the paper's probe
  * vectors (Section 3.1): A, B are n x K row-major, C (may be NULL) and D hold n accumulator words.
  * Unscaled models only. */

@@ -226,6 +226,24 @@ int mmasim_gemm_ex(const mmasim_model* model, int64_t M, int64_t N, int64_t K, c
     return run_gemm(model, g, opts ? opts->flags : 0, static_cast<cudaStream_t>(stream));
 }
 
+int mmasim_gemm_noalloc(const mmasim_model* model, int64_t M, int64_t N, int64_t K, const void* A, const void* B,
+                        const void* C, void* D, const mmasim_gemm_opts* opts, void* stream) {
+    GemmArgs g;
+    int st = build_args(model, M, N, K, A, B, C, D, opts, &g);
+    if (st != MMASIM_OK) return st;
+    if (!aligned16(A) || !aligned16(B) || !aligned16(D) || (C && !aligned16(C))) {
+        set_error("A, B, C and D must be 16-byte aligned");
+        return MMASIM_ERR_ALIGN;
+    }
+    if ((st = check_device_ptr(A, "A")) != MMASIM_OK) return st;
+    if ((st = check_device_ptr(B, "B")) != MMASIM_OK) return st;
+    if ((st = check_device_ptr(D, "D")) != MMASIM_OK) return st;
+    if (C && (st = check_device_ptr(C, "C")) != MMASIM_OK) return st;
+    if (g.row_scale && (st = check_device_ptr(g.row_scale, "opts->row_scale")) != MMASIM_OK) return st;
+    if (g.col_scale && (st = check_device_ptr(g.col_scale, "opts->col_scale")) != MMASIM_OK) return st;
+    return launch_gemm_noalloc(model->dev, g, static_cast<cudaStream_t>(stream));
+}
+
 int mmasim_gemm(const mmasim_model* model, int64_t M, int64_t N, int64_t K, const void* A, const void* B,
                 const void* C, void* D, void* stream) {
     return mmasim_gemm_ex(model, M, N, K, A, B, C, D, nullptr, stream);

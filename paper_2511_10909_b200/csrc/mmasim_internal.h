@@ -85,6 +85,7 @@ int launch_generic(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
 // mmasim_tfdpa_fast.cu
 bool fast_tfdpa_supported(const DevModel& m, const GemmArgs& g);
 int launch_fast_tfdpa(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
+int launch_gemm_noalloc(const DevModel& m, const GemmArgs& g, cudaStream_t stream);   // status code; sets the error message
 // mmasim_fp_fast.cu
 bool fast_fp_supported(const DevModel& m, const GemmArgs& g);
 int launch_fast_fp(const DevModel& m, const GemmArgs& g, cudaStream_t stream);

@@ -68,6 +68,27 @@ bool fast_tfdpa_supported(const DevModel& m, const GemmArgs& g) {
     return true;
 }
 
+int launch_gemm_noalloc(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
+    if (!fast::noalloc_supported(m) || !fast_tfdpa_supported(m, g)) {
+        set_error("mmasim_gemm_noalloc serves the FP8 models with F = 13 (Ada and Hopper FP8 rows), K a multiple of 32 and "
+                  "16-byte row strides; this call needs another kernel");
+        return MMASIM_ERR_UNSUPPORTED;
+    }
+    const size_t need = fast::noalloc_need(m, g), cap = fast::noalloc_capacity();
+    if (need > cap) {
+        set_error("mmasim_gemm_noalloc: this problem needs %zu bytes of scratch, the fixed array holds %zu "
+                  "(about (ceil(M/128) + ceil(N/128)) * K/32 * 27 KiB); use mmasim_gemm_ex", need, cap);
+        return MMASIM_ERR_SHAPE;
+    }
+    set_kernel_name("tfdpa_lut8_noalloc");
+    const cudaError_t err = fast::launch_noalloc(m, g, stream);
+    if (err != cudaSuccess) {
+        set_error("mmasim_gemm_noalloc: %s", cudaGetErrorString(err));
+        return MMASIM_ERR_CUDA;
+    }
+    return MMASIM_OK;
+}
+
 int launch_fast_tfdpa(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
     cudaError_t err = cudaErrorInvalidValue;
     if (kind_of(m) == KIND_TR) {

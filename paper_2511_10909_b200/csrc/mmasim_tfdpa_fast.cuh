@@ -65,6 +65,11 @@ cudaError_t launch_lut8(const DevModel& m, const GemmArgs& g, cudaStream_t strea
 cudaError_t launch_f16(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
 cudaError_t launch_bf16(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
 cudaError_t launch_tf32(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
+// the allocation-free variant of the F = 13 kernel (mmasim_tfdpa_fast_lut8.cu): scratch in a fixed device array
+bool noalloc_supported(const DevModel& m);
+size_t noalloc_capacity();
+size_t noalloc_need(const DevModel& m, const GemmArgs& g);
+cudaError_t launch_noalloc(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
 cudaError_t launch_tr(const DevModel& m, const GemmArgs& g, cudaStream_t stream);    // TR-/GTR-FDPA (mmasim_trfdpa_f64.cu)
 cudaError_t launch_e(const DevModel& m, const GemmArgs& g, cudaStream_t stream);     // E-FDPA (mmasim_efdpa_f64.cu)
 

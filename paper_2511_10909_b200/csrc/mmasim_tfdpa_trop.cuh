@@ -584,19 +584,36 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
 #undef MMASIM_SP_WORD
 }
 
+// Where the decoded blocks go: memory of the caller's (given != nullptr, capacity bytes) or, by default, a stream-ordered
+// allocation out of the library's pool, returned to it behind the kernel.
+struct Scratch {
+    void* given = nullptr;
+    size_t capacity = 0;
+};
+
+template <int TH>
+size_t scratch_bytes_one(const GemmArgs& g) {
+    constexpr int BN = Geo<TH>::BN;
+    const int64_t tiles_m = (g.M + BM - 1) / BM, tiles_n = (g.N + BN - 1) / BN, nch = g.K / KC;
+    return size_t(tiles_m * nch) * sizeof(BlkT<BM>) + size_t(tiles_n * nch) * sizeof(BlkT<BN>);
+}
+
 template <int EK, int L, int F, int RHO, bool PROMOTE, int BASE, int TH>
-cudaError_t launch_one_t(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
+cudaError_t launch_one_t(const DevModel& m, const GemmArgs& g, cudaStream_t stream, const Scratch& sc) {
     constexpr int BN = Geo<TH>::BN;
     const size_t sh = sizeof(SmemT<TH>);
     cudaError_t err = cudaFuncSetAttribute(tfdpa_trop_kernel<EK, L, F, RHO, PROMOTE, BASE, TH>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
     if (err != cudaSuccess) return err;
     const int64_t tiles_m = (g.M + BM - 1) / BM, tiles_n = (g.N + BN - 1) / BN, nch = g.K / KC;
-    // scratch: the decoded blocks of A and B, stream-ordered out of the library's pool and returned to it behind the kernel
     const size_t bytes_a = size_t(tiles_m * nch) * sizeof(BlkT<BM>), bytes_b = size_t(tiles_n * nch) * sizeof(BlkT<BN>);
-    cudaMemPool_t pool = nullptr;
-    if ((err = scratch_pool(&pool)) != cudaSuccess) return err;
-    void* ws = nullptr;
-    if ((err = cudaMallocFromPoolAsync(&ws, bytes_a + bytes_b, pool, stream)) != cudaSuccess) return err;
+    void* ws = sc.given;
+    if (ws) {
+        if (bytes_a + bytes_b > sc.capacity) return cudaErrorInvalidValue;      // the caller checked: never reached
+    } else {
+        cudaMemPool_t pool = nullptr;
+        if ((err = scratch_pool(&pool)) != cudaSuccess) return err;
+        if ((err = cudaMallocFromPoolAsync(&ws, bytes_a + bytes_b, pool, stream)) != cudaSuccess) return err;
+    }
     BlkT<BM>* wa = static_cast<BlkT<BM>*>(ws);
     BlkT<BN>* wb = reinterpret_cast<BlkT<BN>*>(static_cast<unsigned char*>(ws) + bytes_a);
     trop_decode_kernel<BASE, BM, true, TH><<<dim3((unsigned)nch, (unsigned)tiles_m), NT, 0, stream>>>(
@@ -606,29 +623,35 @@ cudaError_t launch_one_t(const DevModel& m, const GemmArgs& g, cudaStream_t stre
     dim3 grid((unsigned)tiles_n, (unsigned)tiles_m, 1);
     tfdpa_trop_kernel<EK, L, F, RHO, PROMOTE, BASE, TH><<<grid, NT, sh, stream>>>(m, g, wa, wb);
     err = cudaGetLastError();
+    if (sc.given) return err;
     const cudaError_t err2 = cudaFreeAsync(ws, stream);
     return err != cudaSuccess ? err : err2;
 }
 
 // The tall micro-tile where the registers allow it: FP32 accumulators without promoted partial sums beside them.
+inline bool tall_tile(const DevModel& m, const GemmArgs& g) { return m.rho != RHO_RNE_FP16 && !g.k_chunk; }
+inline size_t scratch_bytes(const DevModel& m, const GemmArgs& g) {
+    return tall_tile(m, g) ? scratch_bytes_one<8>(g) : scratch_bytes_one<4>(g);
+}
+
 template <int EK, int L, int F, int RHO, int BASE>
-cudaError_t launch_variant_t(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
+cudaError_t launch_variant_t(const DevModel& m, const GemmArgs& g, cudaStream_t stream, const Scratch& sc) {
     if constexpr (RHO == RHO_RNE_FP16) {
-        return launch_one_t<EK, L, F, RHO, false, BASE, 4>(m, g, stream);
+        return launch_one_t<EK, L, F, RHO, false, BASE, 4>(m, g, stream, sc);
     } else {
-        if (g.k_chunk) return launch_one_t<EK, L, F, RHO, true, BASE, 4>(m, g, stream);
-        return launch_one_t<EK, L, F, RHO, false, BASE, 8>(m, g, stream);
+        if (g.k_chunk) return launch_one_t<EK, L, F, RHO, true, BASE, 4>(m, g, stream, sc);
+        return launch_one_t<EK, L, F, RHO, false, BASE, 8>(m, g, stream, sc);
     }
 }
 
 // BASE by the exponent spread of the two element types (see pe_shift): both E4M3, one E5M2, both E5M2.
 template <int EK, int L, int F, int RHO>
-cudaError_t launch_by_types_t(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
+cudaError_t launch_by_types_t(const DevModel& m, const GemmArgs& g, cudaStream_t stream, const Scratch& sc = Scratch()) {
     const int wide = (m.fmt_a == EF_E5M2) + (m.fmt_b == EF_E5M2);
     if ((m.fmt_a != EF_E4M3 && m.fmt_a != EF_E5M2) || (m.fmt_b != EF_E4M3 && m.fmt_b != EF_E5M2)) return cudaErrorInvalidValue;
-    if (wide == 0) return launch_variant_t<EK, L, F, RHO, 8>(m, g, stream);
-    if (wide == 1) return launch_variant_t<EK, L, F, RHO, 5>(m, g, stream);
-    return launch_variant_t<EK, L, F, RHO, 4>(m, g, stream);
+    if (wide == 0) return launch_variant_t<EK, L, F, RHO, 8>(m, g, stream, sc);
+    if (wide == 1) return launch_variant_t<EK, L, F, RHO, 5>(m, g, stream, sc);
+    return launch_variant_t<EK, L, F, RHO, 4>(m, g, stream, sc);
 }
 
 }  // namespace trop

@@ -62,6 +62,9 @@ def _load():
     lib.mmasim_gemm_ex.restype = c_int
     lib.mmasim_gemm_ex.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
                                    POINTER(_GemmOpts), c_void_p]
+    lib.mmasim_gemm_noalloc.restype = c_int
+    lib.mmasim_gemm_noalloc.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
+                                        POINTER(_GemmOpts), c_void_p]
     lib.mmasim_dot_batch.restype = c_int
     lib.mmasim_dot_batch.argtypes = [c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.mmasim_gemm_host.restype = c_int
@@ -242,6 +245,26 @@ def gemm(model: Model, A, B, C=None, out=None, *, M=None, N=None, K=None, sfa=No
         o = _make_opts(_ptr(sfa), _ptr(sfb), k_chunk, _ptr(row_scale), _ptr(col_scale), force_generic,
                        lda, ldb, ldc, ldd)
         _check(_lib.mmasim_gemm_ex(model._h, M, N, K, _ptr(A), _ptr(B), _ptr(C), _ptr(out), byref(o), _stream(stream)))
+    return out
+
+
+def gemm_noalloc(model: Model, A, B, C, out, *, k_chunk=0, row_scale=None, col_scale=None, stream=None):
+    """D = Phi(A, B, C) into the caller's ``out`` through mmasim_gemm_noalloc: no device memory is allocated or freed
+    by the call (the scratch of the kernel is a fixed array inside the library), for callers that must not touch the
+    allocator when they call.  FP8 models with F = 13 only; contiguous CUDA tensors; ``out`` is required, since
+    creating it here would allocate.  Calls share the scratch: keep them ordered on one stream."""
+    if not A.is_cuda:
+        raise MmasimError(1, "mmasim.gemm_noalloc needs CUDA tensors (no CPU fallback)")
+    dev = A.device
+    M, N, K = A.shape[0], B.shape[0], A.shape[1]
+    lda = _matrix(A, "A", M, K, 8, dev)
+    ldb = _matrix(B, "B", N, K, 8, dev)
+    ldc = _matrix(C, "C", M, N, model.acc_bytes * 8, dev)
+    ldd = _matrix(out, "out", M, N, model.acc_bytes * 8, dev)
+    _vector(row_scale, "row_scale", M, 4, dev)
+    _vector(col_scale, "col_scale", N, 4, dev)
+    o = _make_opts(None, None, k_chunk, _ptr(row_scale), _ptr(col_scale), False, lda, ldb, ldc, ldd)
+    _check(_lib.mmasim_gemm_noalloc(model._h, M, N, K, _ptr(A), _ptr(B), _ptr(C), _ptr(out), byref(o), _stream(stream)))
     return out
 
 
