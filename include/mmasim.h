@@ -38,7 +38,7 @@ typedef enum {
     MMASIM_ERR_SHAPE = 3,       /* M, N, K < 1, K not a multiple of the model's block, bad k_chunk or ld */
     MMASIM_ERR_ALIGN = 4,       /* pointer or leading dimension not aligned as documented */
     MMASIM_ERR_CUDA = 5,        /* a CUDA runtime call failed (message holds the CUDA error string) */
-    MMASIM_ERR_TIMEOUT = 6      /* reserved: a bounded device-side wait gave up */
+    MMASIM_ERR_TIMEOUT = 6      /* a bounded device-side wait gave up (reported through a status word, see mmasim_hw_umma) */
 } mmasim_status;
 
 /* The ten architectures of Section 3.2. */
@@ -194,6 +194,24 @@ typedef enum {
     MMASIM_HW_E4M3_F32_K16 = 12  /* m16n8k16 */
 } mmasim_hw_kind;
 int mmasim_hw_mma(int kind, int64_t M, int64_t K, const void* A, const void* B, const void* C, void* D, void* stream);
+
+/* The same for the B200's fifth-generation matrix instruction, tcgen05.mma (the instruction class of the paper's Blackwell
+ * FP8 / FP6 / FP4 rows, Table 3's UTC*MMA entries; Section 3.2, Section 3.1 Step 4).  One instruction tile of 128 rows:
+ *   D (M x 16) = A (M x K, row-major) * B^T (B is 16 x K, row-major, shared by all tiles) + C (M x 16, may be NULL = +0),
+ * FP32 accumulator words, M a multiple of 128, K a multiple of the instruction's K (16 for FP16 / BF16, 8 for TF32, 32
+ * for the 8-bit kinds); a longer K chains instructions through the accumulator in tensor memory, ascending k.  Element
+ * layouts as for mmasim_gemm (TF32 in 32-bit words; FP8, FP6 and FP4 one element per byte in the low bits); all
+ * pointers are device pointers.  `status` (device, 4 bytes, zeroed by the caller) receives MMASIM_ERR_TIMEOUT if the
+ * kernel's bounded wait for the instruction ran out; the kernel then stores nothing, releases what it holds and
+ * returns.  MMASIM_UMMA_SELFTEST_TIMEOUT issues nothing, so that this wait runs out after about a millisecond: the
+ * test of the give-up path (A, B, D are still needed as valid buffers). */
+typedef enum {
+    MMASIM_UMMA_F16_F32 = 0, MMASIM_UMMA_BF16_F32 = 1, MMASIM_UMMA_TF32_F32 = 2, MMASIM_UMMA_E4M3_F32 = 3,
+    MMASIM_UMMA_E5M2_F32 = 4, MMASIM_UMMA_E4M3_E5M2_F32 = 5, MMASIM_UMMA_E2M3_F32 = 6, MMASIM_UMMA_E3M2_F32 = 7,
+    MMASIM_UMMA_E2M1_F32 = 8, MMASIM_UMMA_SELFTEST_TIMEOUT = 9
+} mmasim_umma_kind;
+int mmasim_hw_umma(int kind, int64_t M, int64_t K, const void* A, const void* B, const void* C, void* D, int32_t* status,
+                   void* stream);
 
 /* Error statistics of n model outputs D (accumulator words, acc_fmt MMASIM_ACC_F32 or MMASIM_ACC_F16) against an
  * FP64 reference `ref` (n doubles): the reduction behind the accuracy analysis of Section 6 - the deviation

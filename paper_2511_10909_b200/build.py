@@ -10,7 +10,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmmasim.so")
 SOURCES = ["mmasim_api.cpp", "mmasim_registry.cpp", "mmasim_generic.cu", "mmasim_tfdpa_fast.cu",
            "mmasim_tfdpa_fast_lut8.cu", "mmasim_tfdpa_fast_f16.cu", "mmasim_tfdpa_fast_bf16.cu", "mmasim_trfdpa_f64.cu", "mmasim_efdpa_f64.cu", "mmasim_fp_fast.cu", "mmasim_gst_fast.cu",
-           "mmasim_dot_stream.cu", "mmasim_peak.cu", "mmasim_hw_mma.cu", "mmasim_stats.cu"]
+           "mmasim_dot_stream.cu", "mmasim_peak.cu", "mmasim_hw_mma.cu", "mmasim_hw_umma.cu", "mmasim_stats.cu"]
 HEADERS = ["mmasim_internal.h", "mmasim_device.cuh", "mmasim_tfdpa_fast.cuh", "mmasim_tfdpa_f64.cuh", "mmasim_tfdpa_trop.cuh", os.path.join("..", "..", "include", "mmasim.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--fmad=false"]

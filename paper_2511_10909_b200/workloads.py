@@ -271,8 +271,58 @@ def sample_pairs(M: int, N: int, count: int, seed: int):
     return np.stack([g.integers(0, M, count), g.integers(0, N, count)], axis=1)
 
 
-def hw_tiles(fmt: str, acc: str, K: int, M: int, seed: int = 9):
-    """Inputs for one hardware MMA shape: A (M x K), B (8 x K), C (M x 8) raw words.
+def hw_tiles8(fmt: str, K: int, M: int, nb: int = 16, seed: int = 19, b_fmt: str | None = None):
+    """Inputs for a hardware MMA on 8-bit-container types (FP8, FP6, FP4): A (M x K), B (nb x K) codes, C (M x nb) FP32.
+
+    Row classes of A by index mod 4: N(0,1) values cast to the format; uniformly random codes (NaN and infinity codes
+    included where the format has them); random codes with about half of the elements +-0; cancelling pairs (x, -x) of
+    random finite codes, shuffled along K.  The rows of B take the classes in turn; C mixes N(0,1), zeros, values far
+    above and far below the products, and random FP32 bit patterns.
+    """
+    g = rng(seed, stream=K + (hash(fmt) & 0xFF))
+    b_fmt = b_fmt or fmt
+
+    def mat(rows, f):
+        ebits, mbits, _, special = _SMALL[f]
+        width = 1 + ebits + mbits
+        sign = 1 << (width - 1)
+        x = cast_small(g.standard_normal((rows, K)).astype(np.float32) * np.float32(2.0), f)
+        codes = g.integers(0, 1 << width, (rows, K)).astype(np.uint8)
+        cls = (np.arange(rows) % 4)[:, None]
+        x = np.where(cls == 1, codes, x)
+        zeros = (g.random((rows, K)) < 0.5)
+        x = np.where((cls == 2) & zeros, codes & sign, np.where(cls == 2, codes, x))
+        half = K // 2
+        fin = codes.copy()
+        if special == "ieee":
+            top = ((1 << ebits) - 1) << mbits
+            fin = np.where((fin & top) == top, fin & ~np.uint8(1 << mbits), fin)          # exponent field below the top one
+        elif special == "fn":
+            fin = np.where((fin & (sign - 1)) == sign - 1, fin & ~np.uint8(1), fin)      # not the NaN code
+        pair = np.concatenate([fin[:, :half], fin[:, :half] ^ np.uint8(sign)], axis=1)
+        perm = np.argsort(g.random((rows, K)), axis=1)
+        other = np.take_along_axis(np.concatenate([fin[:, half:], fin[:, half:]], axis=1), perm, 1)
+        pair = np.take_along_axis(pair, perm, 1)
+        x = np.where(cls == 3, pair, x)
+        return np.ascontiguousarray(x.astype(np.uint8)), np.ascontiguousarray(other.astype(np.uint8))
+
+    A, _ = mat(M, fmt)
+    B, B_other = mat(nb, b_fmt)
+    # class 3 of B: the partner of A's pairs is the same column value twice, so that a_k b_k + a_k' b_k' cancels exactly
+    B[np.arange(nb) % 4 == 3] = B_other[np.arange(nb) % 4 == 3]
+    c = g.standard_normal((M, nb)).astype(np.float32)
+    kind = g.integers(0, 8, (M, nb))
+    c = np.where(kind == 1, np.float32(0), c)
+    c = np.where(kind == 2, c * np.float32(2.0 ** 40), c)
+    c = np.where(kind == 3, c * np.float32(2.0 ** -40), c)
+    C = c.view(np.uint32).copy()
+    bits = g.integers(0, 1 << 32, (M, nb), dtype=np.uint64).astype(np.uint32)
+    C = np.where(kind == 4, bits, C)
+    return A, B, np.ascontiguousarray(C)
+
+
+def hw_tiles(fmt: str, acc: str, K: int, M: int, seed: int = 9, nb: int = 8):
+    """Inputs for one hardware MMA shape: A (M x K), B (nb x K), C (M x nb) raw words.
 
     FP16 / BF16 / TF32: the eight input classes of config 4 (row class = row index mod 8; the eight rows of B take
     one class each), plus zero-heavy rows (every 16th row of A has about a third of its elements replaced by +-0).
@@ -285,15 +335,15 @@ def hw_tiles(fmt: str, acc: str, K: int, M: int, seed: int = 9):
             wide = (np.arange(shape[0]) % 4 == 3)[:, None]
             x = np.where(wide, x * np.exp2(g.integers(-40, 40, shape)), x)
             return np.ascontiguousarray(x.view(np.uint64))
-        return mat((M, K)), mat((8, K)), mat((M, 8))
+        return mat((M, K)), mat((nb, K)), mat((M, nb))
     A, _, C1 = cfg4(fmt, K, n=M)
-    _, B, _ = cfg4(fmt, K, n=8)
+    _, B, _ = cfg4(fmt, K, n=nb)
     zero_rows = np.flatnonzero(np.arange(M) % 16 == 9)
     z = g.random((zero_rows.size, K)) < 0.33
     sign = A.dtype.type(1 << (A.dtype.itemsize * 8 - 1))
     A[zero_rows] = np.where(z, A[zero_rows] & sign, A[zero_rows])
-    _, _, C2 = cfg4(fmt, K, n=M * 8)
-    C = C2.reshape(M, 8).copy()
+    _, _, C2 = cfg4(fmt, K, n=M * nb)
+    C = C2.reshape(M, nb).copy()
     C[np.arange(M) % 16 == 1] = 0                      # a few all-zero accumulator rows
     if acc == "fp16":
         C = (C >> 16).astype(np.uint16)                # the top half of an FP32 word: an arbitrary FP16 word
