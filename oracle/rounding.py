@@ -8,6 +8,8 @@ Readings where the paper is silent:
 * on overflow every conversion gives +-inf, the round-to-zero ones too (they
   do not saturate at the largest finite value: the B200's mma.sync, which the
   Blackwell rows describe, returns +-inf);
+* a result of magnitude zero under the NVIDIA conversions (RZ-FP32, RZ-E8M13, RNE-FP16) is +0, also when a negative
+  sum underflows (the B200 does so through both of its matrix instructions); RNE-FP32 keeps the sign;
 * RZ-E8M13 is an FP32 word whose low 10 mantissa bits are zero: 8 exponent
   bits, 13 mantissa bits, subnormals on a 2**-139 grid.
 """
@@ -63,7 +65,19 @@ def round_dyadic(m: int, e: int, ebits: int, mbits: int, bias: int, mode: str,
     return (sign << sign_shift) | n             # subnormal or zero (field 0)
 
 
+# conversions of the NVIDIA models (T-, ST-, GST-FDPA): a result of magnitude zero is +0 whatever the sign of the sum
+ZERO_IS_POSITIVE = {"RZ-FP32", "RZ-E8M13", "RNE-FP16"}
+
+
 def rho(name: str, m: int, e: int) -> int:
-    """Apply the conversion function ``name`` of Table 2 to ``m * 2**e``; exact zero -> +0."""
+    """Apply the conversion function ``name`` of Table 2 to ``m * 2**e``; exact zero -> +0.
+
+    Under RZ-FP32, RZ-E8M13 and RNE-FP16 a nonzero sum that converts to zero gives +0 as well (the B200 returns +0 for
+    a negative sum below the smallest subnormal, through mma.sync and through tcgen05.mma, for FP32 and FP16 outputs);
+    RNE-FP32, the conversion of the AMD models, keeps the sign as IEEE-754 rounding does (no hardware pin).
+    """
     ebits, mbits, bias, mode, lsh = RHO[name]
-    return round_dyadic(m, e, ebits, mbits, bias, mode) << lsh
+    w = round_dyadic(m, e, ebits, mbits, bias, mode)
+    if name in ZERO_IS_POSITIVE and (w & ((1 << (ebits + mbits)) - 1)) == 0:
+        w = 0
+    return w << lsh

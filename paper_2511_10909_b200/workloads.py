@@ -279,7 +279,7 @@ def hw_tiles8(fmt: str, K: int, M: int, nb: int = 16, seed: int = 19, b_fmt: str
     random finite codes, shuffled along K.  The rows of B take the classes in turn; C mixes N(0,1), zeros, values far
     above and far below the products, and random FP32 bit patterns.
     """
-    g = rng(seed, stream=K + (hash(fmt) & 0xFF))
+    g = rng(seed, stream=K + 1000 * sum(fmt.encode()))
     b_fmt = b_fmt or fmt
 
     def mat(rows, f):
