@@ -208,10 +208,14 @@ int mmasim_hw_mma(int kind, int64_t M, int64_t K, const void* A, const void* B, 
 typedef enum {
     MMASIM_UMMA_F16_F32 = 0, MMASIM_UMMA_BF16_F32 = 1, MMASIM_UMMA_TF32_F32 = 2, MMASIM_UMMA_E4M3_F32 = 3,
     MMASIM_UMMA_E5M2_F32 = 4, MMASIM_UMMA_E4M3_E5M2_F32 = 5, MMASIM_UMMA_E2M3_F32 = 6, MMASIM_UMMA_E3M2_F32 = 7,
-    MMASIM_UMMA_E2M1_F32 = 8, MMASIM_UMMA_SELFTEST_TIMEOUT = 9
+    MMASIM_UMMA_E2M1_F32 = 8, MMASIM_UMMA_SELFTEST_TIMEOUT = 9,
+    /* block-scaled kinds: sfa (M x K/k_block bytes) and sfb (16 x K/k_block bytes), device, row-major, as for mmasim_gemm_ex */
+    MMASIM_UMMA_MXE4M3 = 10, MMASIM_UMMA_MXE5M2 = 11, MMASIM_UMMA_MXE2M3 = 12, MMASIM_UMMA_MXE3M2 = 13, MMASIM_UMMA_MXE2M1 = 14,
+    MMASIM_UMMA_MXF4 = 15,      /* packed FP4, E8M0 scale per 32 elements, K a multiple of 64 */
+    MMASIM_UMMA_NVF4 = 16       /* packed FP4, UE4M3 scale per 16 elements, K a multiple of 64 */
 } mmasim_umma_kind;
-int mmasim_hw_umma(int kind, int64_t M, int64_t K, const void* A, const void* B, const void* C, void* D, int32_t* status,
-                   void* stream);
+int mmasim_hw_umma(int kind, int64_t M, int64_t K, const void* A, const void* B, const void* C, void* D,
+                   const void* sfa, const void* sfb, int32_t* status, void* stream);
 
 /* Error statistics of n model outputs D (accumulator words, acc_fmt MMASIM_ACC_F32 or MMASIM_ACC_F16) against an
  * FP64 reference `ref` (n doubles): the reduction behind the accuracy analysis of Section 6 - the deviation

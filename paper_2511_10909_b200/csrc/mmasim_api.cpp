@@ -427,8 +427,8 @@ int mmasim_hw_mma(int kind, int64_t M, int64_t K, const void* A, const void* B, 
     return launch_hw_mma(kind, M, K, A, B, C, D, static_cast<cudaStream_t>(stream));
 }
 
-int mmasim_hw_umma(int kind, int64_t M, int64_t K, const void* A, const void* B, const void* C, void* D, int32_t* status,
-                   void* stream) {
+int mmasim_hw_umma(int kind, int64_t M, int64_t K, const void* A, const void* B, const void* C, void* D, const void* sfa,
+                   const void* sfb, int32_t* status, void* stream) {
     if (!A || !B || !D || !status) { set_error("mmasim_hw_umma: A, B, D and status must not be NULL"); return MMASIM_ERR_INVALID_ARG; }
     int st;
     if ((st = check_device_ptr(A, "A")) != MMASIM_OK) return st;
@@ -436,8 +436,10 @@ int mmasim_hw_umma(int kind, int64_t M, int64_t K, const void* A, const void* B,
     if ((st = check_device_ptr(D, "D")) != MMASIM_OK) return st;
     if ((st = check_device_ptr(status, "status")) != MMASIM_OK) return st;
     if (C && (st = check_device_ptr(C, "C")) != MMASIM_OK) return st;
+    if (sfa && (st = check_device_ptr(sfa, "sfa")) != MMASIM_OK) return st;
+    if (sfb && (st = check_device_ptr(sfb, "sfb")) != MMASIM_OK) return st;
     if (!aligned16(A) || !aligned16(B)) { set_error("mmasim_hw_umma: A and B must be 16-byte aligned"); return MMASIM_ERR_ALIGN; }
-    return launch_hw_umma(kind, M, K, A, B, C, D, status, static_cast<cudaStream_t>(stream));
+    return launch_hw_umma(kind, M, K, A, B, C, D, sfa, sfb, status, static_cast<cudaStream_t>(stream));
 }
 
 int mmasim_error_stats(int acc_fmt, int64_t n, const void* D, const double* ref, double* stats, void* stream) {

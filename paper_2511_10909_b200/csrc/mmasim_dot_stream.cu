@@ -212,7 +212,9 @@ __device__ __forceinline__ uint32_t tfdpa_dot(const Rows& rows, int K, int F, ui
         else if (fabs(v) >= 3.402823669209385e38) cw = (__double2hiint(v) < 0 ? 0xFF800000u : 0x7F800000u);   // |v| >= 2^128: overflow
         else cw = (v != v) ? 0x7FFFFFFFu : __float_as_uint(__double2float_rz(v));
     }
-    return cw;
+    // a chain's last word of magnitude zero is +0, also when a negative sum underflowed (in between the sign of a zero
+    // does not matter: a zero accumulator has no exponent and adds nothing)
+    return positive_zero(cw, ACC16 ? 0x7FFFu : 0x7FFFFFFFu);
 }
 
 template <int EK, int L, int RHO, bool STAGED>

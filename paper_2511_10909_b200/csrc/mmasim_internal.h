@@ -98,8 +98,8 @@ int launch_dot_stream(const DevModel& m, const GemmArgs& g, cudaStream_t stream)
 // mmasim_hw_mma.cu
 int launch_hw_mma(int kind, int64_t M, int64_t K, const void* A, const void* B, const void* C, void* D, cudaStream_t stream);
 // mmasim_hw_umma.cu
-int launch_hw_umma(int kind, int64_t M, int64_t K, const void* A, const void* B, const void* C, void* D, int32_t* status,
-                   cudaStream_t stream);
+int launch_hw_umma(int kind, int64_t M, int64_t K, const void* A, const void* B, const void* C, void* D, const void* sfa,
+                   const void* sfb, int32_t* status, cudaStream_t stream);
 // mmasim_stats.cu
 int launch_error_stats(int acc, int64_t n, const void* D, const double* ref, double* stats, cudaStream_t stream);
 // mmasim_peak.cu

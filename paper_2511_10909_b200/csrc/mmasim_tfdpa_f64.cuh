@@ -42,8 +42,9 @@ using fast::CB;
 using fast::Elem;
 using fast::raw_elem;
 
-// 512 threads own the 128 x 64 tile of D, 4 x 4 outputs each: sixteen warps per SM keep the FP64 pipe fed while the
-// per-thread state (accumulators, product exponents of the next block, operands) stays within 128 registers.
+// 512 threads own the 128 x 64 tile of D, 4 x 4 outputs each (a warp: 32 x 16, the accumulator tiles of eight FP64 matrix
+// instructions): sixteen warps per SM keep the FP64 pipe fed while the per-thread state (accumulators, product exponents
+// of the next block, operand fragments) stays within 128 registers.
 constexpr int TM = 4, TN = 4, NT = 512;
 
 // The raw words of one chunk, E::TASK consecutive elements of one row of A or B per task (as in the integer kernels).
@@ -88,19 +89,45 @@ struct LutEntry64 {
     uint32_t bits;      // bit 0: sign; bit 1: infinity or NaN; bit 2: nonzero finite
 };
 
+// Operand planes are row-major (k contiguous) with a pitch of KP doubles = 288 bytes: the fragment loads of the FP64
+// matrix instruction (lane (g, t) reads element (row 8 i + g, k 4 s + t)) then hit sixteen different bank pairs per
+// half-warp.  Exponent planes and masks are indexed by the permuted row / column (see perm_row64 / perm_col64), so that
+// the four rows and the four columns of a thread are adjacent.
+constexpr int KP = KC + 4;
+template <int EK, bool ROWMAJOR = false>
+struct Planes64;
 template <int EK>
-struct Planes64 {
+struct Planes64<EK, true> {
+    static constexpr bool ROW_MAJOR = true;
+    double a_d[BM][KP];
+    double b_d[BN][KP];
+    uint32_t a_exp2[KC / 2][BM];    // [pair p][permuted row]: exponents of elements 2p (low half) and 2p + 1 (high half)
+    uint32_t b_exp2[KC / 2][BN];
+    uint32_t a_sgn[BM], b_sgn[BN];  // [permuted row]: bit k = sign of element k of the chunk
+    uint32_t a_nz[BM], b_nz[BN];    // [permuted row]: bit k = element k is finite and nonzero
+};
+// The k-major layout of the kernels that still issue one scalar FP64 multiply-add per term (TR-, GTR- and E-FDPA): a
+// thread owns rows 4 ty .. 4 ty + 3 and the columns col_of(tx, c); nothing is permuted.
+template <int EK>
+struct Planes64<EK, false> {
+    static constexpr bool ROW_MAJOR = false;
     double a_d[KC][BM];
     double b_d[KC][BN];
-    uint32_t a_exp2[KC / 2][BM];    // exponents of elements 2p (low half) and 2p + 1 (high half)
+    uint32_t a_exp2[KC / 2][BM];
     uint32_t b_exp2[KC / 2][BN];
-    uint32_t a_sgn[BM], b_sgn[BN];  // bit k of row r: sign of element k of the chunk
-    uint32_t a_nz[BM], b_nz[BN];    // bit k of row r: element k is finite and nonzero
+    uint32_t a_sgn[BM], b_sgn[BN];
+    uint32_t a_nz[BM], b_nz[BN];
 };
 
-template <int EK>
+// A warp owns 32 rows x 16 columns of the CTA tile, as four by two accumulator tiles of the 8 x 8 x 4 FP64 matrix
+// instruction; a thread's outputs are its share of those tiles: rows g + 8 r (g = lane / 4, r = 0..3) and columns
+// 8 (c / 2) + 2 t + c % 2 (t = lane % 4, c = 0..3).  Permuted positions put a thread's rows / columns side by side.
+__device__ __forceinline__ int perm_row64(int r) { return (r & ~31) | ((r & 7) << 2) | ((r >> 3) & 3); }
+__device__ __forceinline__ int perm_col64(int c) { return (c & ~15) | (((c >> 1) & 3) << 2) | (((c >> 3) & 1) << 1) | (c & 1); }
+
+template <int EK, bool ROWMAJOR = false>
 struct Smem64 {
-    Planes64<EK> pl[2];             // the chunk being computed and the one being decoded
+    Planes64<EK, ROWMAJOR> pl[2];   // the chunk being computed and the one being decoded
     LutEntry64 lut_a[Elem<EK>::SIGNMAG ? 1 : 256];
     LutEntry64 lut_b[Elem<EK>::SIGNMAG ? 1 : 256];
     int special[3];                 // chunk (by index mod 3) holds an infinity or a NaN
@@ -150,6 +177,7 @@ __device__ __forceinline__ void store_chunk64(SM& sm, PL& s, const RawChunk<EK>&
         const int u = is_a ? task : task - BM * R::TPR;
         const int rows = is_a ? BM : BN;
         const int r = u % rows, h = u / rows;
+        const int pr = !PL::ROW_MAJOR ? r : (is_a ? perm_row64(r) : perm_col64(r));
         uint32_t bits = 0u, prev_exp = 0u;
 #pragma unroll
         for (int q = 0; q < E::TASK; ++q) {
@@ -191,31 +219,32 @@ __device__ __forceinline__ void store_chunk64(SM& sm, PL& s, const RawChunk<EK>&
                 op = __hiloint2double(int(hi | (sign << 31)), int(lo));
                 bits += (sign | (nzbit << 16)) << q;
             }
-            if (is_a) s.a_d[kk][r] = op; else s.b_d[kk][r] = op;
+            if (PL::ROW_MAJOR) { if (is_a) s.a_d[r][kk] = op; else s.b_d[r][kk] = op; }
+            else { if (is_a) s.a_d[kk][r] = op; else s.b_d[kk][r] = op; }
             if (q & 1) {
                 const uint32_t pair = prev_exp | (expb << 16);
-                if (is_a) s.a_exp2[kk / 2][r] = pair; else s.b_exp2[kk / 2][r] = pair;
+                if (is_a) s.a_exp2[kk / 2][pr] = pair; else s.b_exp2[kk / 2][pr] = pair;
             }
             prev_exp = expb;
         }
         // sign and nonzero bits of the task's elements go to bits [h * TASK, h * TASK + TASK) of the row's masks
         if (E::TASK == 16) {
-            if (is_a) { reinterpret_cast<uint16_t*>(&s.a_sgn[r])[h] = uint16_t(bits); reinterpret_cast<uint16_t*>(&s.a_nz[r])[h] = uint16_t(bits >> 16); }
-            else { reinterpret_cast<uint16_t*>(&s.b_sgn[r])[h] = uint16_t(bits); reinterpret_cast<uint16_t*>(&s.b_nz[r])[h] = uint16_t(bits >> 16); }
+            if (is_a) { reinterpret_cast<uint16_t*>(&s.a_sgn[pr])[h] = uint16_t(bits); reinterpret_cast<uint16_t*>(&s.a_nz[pr])[h] = uint16_t(bits >> 16); }
+            else { reinterpret_cast<uint16_t*>(&s.b_sgn[pr])[h] = uint16_t(bits); reinterpret_cast<uint16_t*>(&s.b_nz[pr])[h] = uint16_t(bits >> 16); }
         } else {
-            if (is_a) { reinterpret_cast<uint8_t*>(&s.a_sgn[r])[h] = uint8_t(bits); reinterpret_cast<uint8_t*>(&s.a_nz[r])[h] = uint8_t(bits >> 16); }
-            else { reinterpret_cast<uint8_t*>(&s.b_sgn[r])[h] = uint8_t(bits); reinterpret_cast<uint8_t*>(&s.b_nz[r])[h] = uint8_t(bits >> 16); }
+            if (is_a) { reinterpret_cast<uint8_t*>(&s.a_sgn[pr])[h] = uint8_t(bits); reinterpret_cast<uint8_t*>(&s.a_nz[pr])[h] = uint8_t(bits >> 16); }
+            else { reinterpret_cast<uint8_t*>(&s.b_sgn[pr])[h] = uint8_t(bits); reinterpret_cast<uint8_t*>(&s.b_nz[pr])[h] = uint8_t(bits >> 16); }
         }
     }
     if (spec) atomicOr(&sm.special[flag], 1);
 }
 
-// Columns of a thread's micro-tile: two adjacent pairs, 32 columns apart, so that the sixteen threads of a row of the
-// thread grid read 256 contiguous bytes of B operands per 16-byte load.
+// Columns of a thread's micro-tile in the k-major layout: two adjacent pairs, 32 columns apart, so that the sixteen
+// threads of a row of the thread grid read 256 contiguous bytes of B operands per 16-byte load.
 __device__ __forceinline__ int col_of(int tx, int c) { return (c >> 1) * (BN / 2) + tx * 2 + (c & 1); }
 
 // Largest exponent sum of the products of one block (pass 1 of Algorithm 7 without the accumulator), two elements
-// per instruction: lane 0 holds the even elements' maximum, lane 1 the odd ones'.
+// per instruction: lane 0 holds the even elements' maximum, lane 1 the odd ones'.  k-major layout.
 template <int L>
 __device__ __forceinline__ void product_exponents(const uint32_t* ea_p, const uint32_t* eb_p, uint32_t (&emp)[TM][TN]) {
 #pragma unroll
@@ -236,6 +265,27 @@ __device__ __forceinline__ void product_exponents(const uint32_t* ea_p, const ui
     }
 }
 
+// The same for the permuted layout: ea_p / eb_p point at the thread's four adjacent (permuted) rows / columns of the
+// first pair of the block.
+template <int L>
+__device__ __forceinline__ void product_exponents_adj(const uint32_t* ea_p, const uint32_t* eb_p, uint32_t (&emp)[TM][TN]) {
+#pragma unroll
+    for (int r = 0; r < TM; ++r)
+#pragma unroll
+        for (int c = 0; c < TN; ++c) emp[r][c] = 0u;
+#pragma unroll
+    for (int kp = 0; kp < L / 2; ++kp) {
+        const uint4 ea0 = *reinterpret_cast<const uint4*>(ea_p + kp * BM);
+        const uint4 eb0 = *reinterpret_cast<const uint4*>(eb_p + kp * BN);
+        const uint32_t ea[TM] = {ea0.x, ea0.y, ea0.z, ea0.w};
+        const uint32_t ebv[TN] = {eb0.x, eb0.y, eb0.z, eb0.w};
+#pragma unroll
+        for (int r = 0; r < TM; ++r)
+#pragma unroll
+            for (int c = 0; c < TN; ++c) emp[r][c] = __viaddmax_s16x2(ea[r], ebv[c], emp[r][c]);
+    }
+}
+
 // One CTA per SM, 512 threads, a 4 x 4 micro-tile per thread.  The FP64 pipe is the bound (one fma.rm.f64 per term),
 // so everything else is arranged to run beside it: the staged planes are double-buffered (the next chunk is decoded
 // between two barriers while its raw words were fetched a chunk earlier), and the product-exponent pass of block
@@ -247,14 +297,18 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
     constexpr bool ACC16 = RHO == RHO_RNE_FP16;
     constexpr int NBLK = KC / L;
     static_assert(RHO == RHO_RZ_FP32 || RHO == RHO_RNE_FP16, "rho is a single conversion from FP64");
-    static_assert(KC % L == 0 && L % 2 == 0, "blocks tile the chunk; pass 1 handles pairs of elements");
+    static_assert(KC % L == 0 && L % 4 == 0, "blocks tile the chunk; pass 1 handles pairs of elements");
     static_assert(!ST || L == KC, "ST-FDPA: one scale factor pair per block of 32 (Algorithm 8)");
-    using SM = Smem64<EK>;
+    using SM = Smem64<EK, true>;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     SM& sm = *reinterpret_cast<SM*>(smem_raw);
 
     const int tid = threadIdx.x;
-    const int tx = tid % 16, ty = tid / 16;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int wr = warp >> 2, wc = warp & 3, gq = lane >> 2, tq = lane & 3;      // warp grid 4 x 4, warp tile 32 x 16
+    const int prow = wr * 32 + gq * 4, pcol = wc * 16 + tq * 4;                  // the thread's first permuted row / column
+    auto row_at = [&](int r) { return wr * 32 + gq + 8 * r; };                   // inside the CTA tile
+    auto col_at = [&](int c) { return wc * 16 + 8 * (c >> 1) + 2 * tq + (c & 1); };
     const int64_t row0 = int64_t(blockIdx.y) * BM, col0 = int64_t(blockIdx.x) * BN;
     const FmtDesc fa = fmt_desc(m.fmt_a), fb = fmt_desc(m.fmt_b);
     // high word of 1.5 * 2^52 * 2^(e_max - F) is (e_max + CB) * 2^20 + MAGIC_K
@@ -271,7 +325,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
     for (int r = 0; r < TM; ++r)
 #pragma unroll
         for (int c = 0; c < TN; ++c) {
-            const int64_t i = row0 + ty * TM + r, j = col0 + col_of(tx, c);
+            const int64_t i = row0 + row_at(r), j = col0 + col_at(c);
             uint32_t w = 0u;
             if (g.C && i < g.M && j < g.N)
                 w = ACC16 ? uint32_t(static_cast<const uint16_t*>(g.C)[i * g.ldc + j])
@@ -308,7 +362,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
         }
         const bool chunk_special = sm.special[chunk % 3] != 0;
         // the first block's product exponents (the other blocks' are taken beside the multiply-adds of their predecessor)
-        product_exponents<L>(&s.a_exp2[0][ty * TM], &s.b_exp2[0][tx * 2], emp);
+        product_exponents_adj<L>(&s.a_exp2[0][prow], &s.b_exp2[0][pcol], emp);
 
         // ST-FDPA (Algorithm 8): Exp(alpha) of this thread's rows and Exp(beta) of its columns for this block of 32
         int sa_exp[ST ? TM : 1], sb_exp[ST ? TN : 1];
@@ -317,14 +371,14 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
             uint32_t scale_nan = 0u;                    // bit r * TN + c: alpha or beta of that output is NaN
 #pragma unroll
             for (int r = 0; r < TM; ++r) {
-                const int64_t i = row0 + ty * TM + r;
+                const int64_t i = row0 + row_at(r);
                 const uint32_t w = i < g.M ? uint32_t(g.sfa[i * g.ld_sfa + sblk]) : 127u;
                 sa_exp[ST ? r : 0] = int(w) - 127;
                 if (w == 0xFFu) scale_nan |= ((1u << TN) - 1u) << (r * TN);
             }
 #pragma unroll
             for (int c = 0; c < TN; ++c) {
-                const int64_t j = col0 + col_of(tx, c);
+                const int64_t j = col0 + col_at(c);
                 const uint32_t w = j < g.N ? uint32_t(g.sfb[j * g.ld_sfb + sblk]) : 127u;
                 sb_exp[ST ? c : 0] = int(w) - 127;
                 if (w == 0xFFu) scale_nan |= 0x11111111u << c;
@@ -342,7 +396,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
                 for (int r = 0; r < TM; ++r)
 #pragma unroll 1
                     for (int c = 0; c < TN; ++c) {
-                        const int64_t i = row0 + ty * TM + r, j = col0 + col_of(tx, c);
+                        const int64_t i = row0 + row_at(r), j = col0 + col_at(c);
                         if (i >= g.M || j >= g.N) continue;
                         Special ev;
                         for (int kk = kb; kk < kb + L; ++kk) {
@@ -382,45 +436,43 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
             // the chunk has another block, the product exponents of that block ----
             auto multiply_adds = [&](auto with_exponents) {
                 constexpr bool FUSE = decltype(with_exponents)::value;
-                const double* a_p = &s.a_d[kb][ty * TM];
-                const double* b_p = &s.b_d[kb][tx * 2];
-                const uint32_t* ea_p = &s.a_exp2[FUSE ? (kb + L) / 2 : 0][ty * TM];
-                const uint32_t* eb_p = &s.b_exp2[FUSE ? (kb + L) / 2 : 0][tx * 2];
+                const uint32_t* ea_p = &s.a_exp2[FUSE ? (kb + L) / 2 : 0][prow];
+                const uint32_t* eb_p = &s.b_exp2[FUSE ? (kb + L) / 2 : 0][pcol];
                 if (FUSE) {
 #pragma unroll
                     for (int r = 0; r < TM; ++r)
 #pragma unroll
                         for (int c = 0; c < TN; ++c) emp[r][c] = 0u;
                 }
+                // four terms per matrix instruction (mma.sync m8n8k4, FP64, rounding toward minus infinity: a chain of four
+                // fused multiply-adds per output, each rounded onto the grid of q); operand fragments: lane (g, t) holds
+                // A[8 r + g][k + t] and B[8 j + g][k + t]
 #pragma unroll
-                for (int kq = 0; kq < L; ++kq) {
-                    double av[TM], bv[TN];
+                for (int ks = 0; ks < L; ks += 4) {
+                    double af[TM], bf[TN / 2];
 #pragma unroll
-                    for (int r = 0; r < TM; r += 2) {
-                        const double2 t = *reinterpret_cast<const double2*>(a_p + kq * BM + r);
-                        av[r] = t.x; av[r + 1] = t.y;
-                    }
-                    {
-                        const double2 t0 = *reinterpret_cast<const double2*>(b_p + kq * BN);
-                        const double2 t1 = *reinterpret_cast<const double2*>(b_p + kq * BN + BN / 2);
-                        bv[0] = t0.x; bv[1] = t0.y; bv[2] = t1.x; bv[3] = t1.y;
-                    }
-                    uint32_t ea[TM], ebv[TN];
-                    if (FUSE && (kq & 1) == 0) {
-                        const int kp = kq / 2;
-                        const uint4 ea0 = *reinterpret_cast<const uint4*>(ea_p + kp * BM);
-                        const uint2 eb0 = *reinterpret_cast<const uint2*>(eb_p + kp * BN);
-                        const uint2 eb1 = *reinterpret_cast<const uint2*>(eb_p + kp * BN + BN / 2);
-                        ea[0] = ea0.x; ea[1] = ea0.y; ea[2] = ea0.z; ea[3] = ea0.w;
-                        ebv[0] = eb0.x; ebv[1] = eb0.y; ebv[2] = eb1.x; ebv[3] = eb1.y;
-                    }
+                    for (int r = 0; r < TM; ++r) af[r] = s.a_d[wr * 32 + 8 * r + gq][kb + ks + tq];
+#pragma unroll
+                    for (int j = 0; j < TN / 2; ++j) bf[j] = s.b_d[wc * 16 + 8 * j + gq][kb + ks + tq];
 #pragma unroll
                     for (int r = 0; r < TM; ++r)
 #pragma unroll
-                        for (int c = 0; c < TN; ++c) {
-                            acc[r][c] = __fma_rd(av[r], bv[c], acc[r][c]);
-                            if (FUSE && (kq & 1) == 0) emp[r][c] = __viaddmax_s16x2(ea[r], ebv[c], emp[r][c]);
+                        for (int j = 0; j < TN / 2; ++j)
+                            asm volatile("mma.sync.aligned.m8n8k4.row.col.rm.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                                         : "+d"(acc[r][2 * j]), "+d"(acc[r][2 * j + 1]) : "d"(af[r]), "d"(bf[j]));
+                    if (FUSE) {
+#pragma unroll
+                        for (int kp = ks / 2; kp < ks / 2 + 2; ++kp) {
+                            const uint4 ea0 = *reinterpret_cast<const uint4*>(ea_p + kp * BM);
+                            const uint4 eb0 = *reinterpret_cast<const uint4*>(eb_p + kp * BN);
+                            const uint32_t ea[TM] = {ea0.x, ea0.y, ea0.z, ea0.w};
+                            const uint32_t ebv[TN] = {eb0.x, eb0.y, eb0.z, eb0.w};
+#pragma unroll
+                            for (int r = 0; r < TM; ++r)
+#pragma unroll
+                                for (int c = 0; c < TN; ++c) emp[r][c] = __viaddmax_s16x2(ea[r], ebv[c], emp[r][c]);
                         }
+                    }
                 }
             };
             if (NBLK > 1 && blk + 1 < NBLK) multiply_adds(std::true_type{}); else multiply_adds(std::false_type{});
@@ -431,7 +483,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
             constexpr uint32_t SUSPECT = ACC16 ? 0x7C00u : 0x7F7FFFFFu;   // FP16: infinity; FP32: cvt.rz saturates at the largest finite word
             uint32_t wmax = 0u;
             auto block_value = [&](int r, int c, uint32_t sa, uint32_t nza) -> double {
-                const int nneg = __popc((sa ^ s.b_sgn[col_of(tx, c)]) & nza & s.b_nz[col_of(tx, c)]);
+                const int nneg = __popc((sa ^ s.b_sgn[pcol + c]) & nza & s.b_nz[pcol + c]);
                 const long long bits = __double_as_longlong(acc[r][c]) + (long long)nneg;
                 const int hi = int(bits >> 32);
                 const double magic = __hiloint2double((hi & 0x7FF00000) | 0x00080000, 0);
@@ -441,7 +493,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
             };
 #pragma unroll
             for (int r = 0; r < TM; ++r) {
-                const uint32_t sa = s.a_sgn[ty * TM + r], nza = s.a_nz[ty * TM + r] & kmask;
+                const uint32_t sa = s.a_sgn[prow + r], nza = s.a_nz[prow + r] & kmask;
 #pragma unroll
                 for (int c = 0; c < TN; ++c) {
                     const double v = block_value(r, c, sa, nza);
@@ -453,7 +505,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
             if (wmax >= SUSPECT) {
 #pragma unroll
                 for (int r = 0; r < TM; ++r) {
-                    const uint32_t sa = s.a_sgn[ty * TM + r], nza = s.a_nz[ty * TM + r] & kmask;
+                    const uint32_t sa = s.a_sgn[prow + r], nza = s.a_nz[prow + r] & kmask;
 #pragma unroll
                     for (int c = 0; c < TN; ++c) {
                         if ((cw[r][c] & ABS) != SUSPECT) continue;
@@ -474,7 +526,8 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
 #pragma unroll
                 for (int c = 0; c < TN; ++c) {
                     const uint32_t sp = MMASIM_SP_GET(r, c);
-                    const uint32_t pw = sp ? special_word(((sp & 1u) || (sp & 6u) == 6u) ? 1 : ((sp & 2u) ? 2 : 3), ACC16, true) : cw[r][c];
+                    const uint32_t pw = sp ? special_word(((sp & 1u) || (sp & 6u) == 6u) ? 1 : ((sp & 2u) ? 2 : 3), ACC16, true)
+                                           : positive_zero(cw[r][c], 0x7FFFFFFFu);
                     float v = __fadd_rn(promoted[PROMOTE ? r : 0][PROMOTE ? c : 0], __uint_as_float(pw));
                     if (v != v) v = __uint_as_float(0x7FFFFFFFu);
                     promoted[PROMOTE ? r : 0][PROMOTE ? c : 0] = v;
@@ -489,11 +542,12 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
     for (int r = 0; r < TM; ++r)
 #pragma unroll
         for (int c = 0; c < TN; ++c) {
-            const int64_t i = row0 + ty * TM + r, j = col0 + col_of(tx, c);
+            const int64_t i = row0 + row_at(r), j = col0 + col_at(c);
             if (i >= g.M || j >= g.N) continue;
             const uint32_t sp = MMASIM_SP_GET(r, c);
             uint32_t w = PROMOTE ? __float_as_uint(promoted[PROMOTE ? r : 0][PROMOTE ? c : 0])
-                                 : (sp ? special_word(((sp & 1u) || (sp & 6u) == 6u) ? 1 : ((sp & 2u) ? 2 : 3), ACC16, true) : cw[r][c]);
+                                 : (sp ? special_word(((sp & 1u) || (sp & 6u) == 6u) ? 1 : ((sp & 2u) ? 2 : 3), ACC16, true)
+                                       : positive_zero(cw[r][c], ACC16 ? 0x7FFFu : 0x7FFFFFFFu));   // a zero result is +0
             if (g.row_scale) {
                 float sc = __fmul_rn(g.row_scale[i], g.col_scale[j]);
                 if (sc != sc) sc = __uint_as_float(0x7FFFFFFFu);
@@ -509,7 +563,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
 
 template <int EK, int L, int RHO, bool PROMOTE, bool ST = false>
 cudaError_t launch_one64(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
-    const size_t sh = sizeof(Smem64<EK>);
+    const size_t sh = sizeof(Smem64<EK, true>);
     cudaError_t err = cudaFuncSetAttribute(tfdpa64_kernel<EK, L, RHO, PROMOTE, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
     if (err != cudaSuccess) return err;
     dim3 grid((unsigned)((g.N + BN - 1) / BN), (unsigned)((g.M + BM - 1) / BM), 1);

@@ -545,7 +545,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
             for (int h = 0; h < TH; ++h)
 #pragma unroll
                 for (int x = 0; x < TW; ++x) {
-                    const float part = __uint_as_float(MMASIM_SP_WORD(h, x, cw[h][x] & RHO_MASK));
+                    const float part = __uint_as_float(MMASIM_SP_WORD(h, x, positive_zero(cw[h][x] & RHO_MASK, 0x7FFFFFFFu)));
                     float v = __fadd_rn(promoted[PROMOTE ? h : 0][PROMOTE ? x : 0], part);
                     if (v != v) v = __uint_as_float(0x7FFFFFFFu);
                     promoted[PROMOTE ? h : 0][PROMOTE ? x : 0] = v;
@@ -569,7 +569,9 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
         for (int x = 0; x < TW; ++x) {
             const int64_t i = row0 + row_of(h), j = col0 + col_of(x);
             if (i >= g.M || j >= g.N) continue;
-            uint32_t w = PROMOTE ? __float_as_uint(promoted[PROMOTE ? h : 0][PROMOTE ? x : 0]) : MMASIM_SP_WORD(h, x, cw[h][x] & RHO_MASK);
+            // a chain's last word of magnitude zero is +0 (in between the sign of a zero does not matter: it has no exponent)
+            uint32_t w = PROMOTE ? __float_as_uint(promoted[PROMOTE ? h : 0][PROMOTE ? x : 0])
+                                 : MMASIM_SP_WORD(h, x, positive_zero(cw[h][x] & RHO_MASK, ACC16 ? 0x7FFFu : 0x7FFFFFFFu));
             if (g.row_scale) {
                 float sc = __fmul_rn(g.row_scale[i], g.col_scale[j]);
                 if (sc != sc) sc = __uint_as_float(0x7FFFFFFFu);

@@ -105,3 +105,48 @@ def test_hw_umma_rejects_bad_arguments():
     A = torch.zeros((128, 48), dtype=torch.uint8, device="cuda")
     with pytest.raises(mmasim.MmasimError):
         mmasim.hw_umma("e4m3_f32", A, torch.zeros((16, 48), dtype=torch.uint8, device="cuda"))   # K = 48: not a multiple of 32
+
+
+# ---- block-scaled kinds: ST-FDPA (Algorithm 8) and GST-FDPA (Algorithm 9) against the instruction ----------------------
+SCALED = {"mxe4m3": ("e4m3", 32, 32), "mxe5m2": ("e5m2", 32, 32), "mxe2m3": ("e2m3", 32, 32), "mxe3m2": ("e3m2", 32, 32),
+          "mxe2m1": ("e2m1", 32, 32), "mxf4": ("e2m1", 64, 32), "nvf4": ("e2m1", 64, 16)}      # element, K of one instruction, k_block
+
+
+def _scaled_inputs(kind, K, M, wide):
+    elem, k, kb = SCALED[kind]
+    A, B, C = wl.hw_tiles8(elem, K, M, nb=16, seed=29)
+    g = wl.rng(95, stream=K + len(kind))
+    nsf = K // kb
+    if kind == "nvf4":                                   # UE4M3 codes: any 7-bit code (0x7F is the NaN), some zeros
+        sfa = g.integers(0, 127, (M, nsf)).astype(np.uint8)
+        sfb = g.integers(0, 127, (16, nsf)).astype(np.uint8)
+        if wide:
+            sfa[g.random((M, nsf)) < 0.02] = 0x7F
+            sfa[g.random((M, nsf)) < 0.05] = 0
+    else:                                                # E8M0: a band around 1 or, wide, the whole range with NaN codes
+        lo, hi = (0, 255) if wide else (127 - 12, 127 + 12)
+        sfa = g.integers(lo, hi + 1, (M, nsf)).astype(np.uint8)
+        sfb = g.integers(lo, hi + 1, (16, nsf)).astype(np.uint8)
+        if wide:
+            sfb[g.random((16, nsf)) < 0.9] = 127          # keep most products inside the FP32 range
+    if kind in ("mxf4", "nvf4"):
+        A, B = wl.pack_fp4(A), wl.pack_fp4(B)
+    return A, B, C, sfa, sfb
+
+
+@pytest.mark.parametrize("kind", list(SCALED))
+@pytest.mark.parametrize("chain,wide", [(1, False), (2, False), (2, True)])
+def test_block_scaled_models_match_tcgen05(kind, chain, wide):
+    from paper_2511_10909_b200 import mmasim
+    _needs_b200()
+    elem, k, kb = SCALED[kind]
+    K, M = k * chain, 1 << 12
+    A, B, C, sfa, sfb = _scaled_inputs(kind, K, M, wide)
+    hw = gu.host_words(mmasim.hw_umma(kind, gu.dev(A), gu.dev(B), gu.dev(C), sfa=gu.dev(sfa), sfb=gu.dev(sfb), K=K))
+    key = ("blackwell", kind, "fp32")
+    inp = {"A": A, "B": B, "C": C, "sfa": sfa, "sfb": sfb}
+    D = gu.run_gemm(key, inp, K=K)
+    bad = np.argwhere(hw != D)
+    assert bad.size == 0, (kind, K, wide, len(bad), [(tuple(x), hex(int(hw[tuple(x)])), hex(int(D[tuple(x)]))) for x in bad[:6]])
+    pairs = wl.sample_pairs(M, 16, 512, seed=96)
+    gu.assert_samples_equal(hw, gu.oracle_samples(key, inp, pairs), pairs, f"hardware tcgen05 {kind} K={K} against the oracle")
