@@ -317,7 +317,18 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
     init_lut64<EK>(sm, fa, fb, tid);
     if (tid == 0) sm.special[0] = sm.special[1] = sm.special[2] = 0;
 
-    uint32_t cw[TM][TN];                                // the accumulator of each output: a finite FP32 / FP16 word
+    // FP32 accumulators live between blocks as doubles ("state"): the value RZ-FP32 produced, exactly, with bit 0 of the
+    // low word set so that the next block's addition (rounded toward minus infinity) never finds it on its grid; the
+    // conversion function is then a mask on the double's low word and the exponent of c is the double's own field.
+    // Results outside the range of normal FP32 numbers (zero, subnormal, overflow) leave the fast path.
+    constexpr bool DS = !ACC16;
+    // (a zero of either sign becomes the positive state: under ST scaling the set bit of -0 could underflow away and leave
+    // the +1 of a negative accumulator uncompensated)
+    auto state_of = [](uint32_t w) { const double d = (w & 0x7FFFFFFFu) ? double(__uint_as_float(w)) : 0.0; return __hiloint2double(__double2hiint(d), __double2loint(d) | 1); };
+    auto word_of = [](double st) { return __float_as_uint(__double2float_rz(__hiloint2double(__double2hiint(st), __double2loint(st) & ~1))); };
+    double cs[DS ? TM : 1][DS ? TN : 1];
+    uint32_t sub_mask = 0u;                             // outputs whose accumulator is a nonzero FP32 subnormal: Exp(c) = -126
+    uint32_t cw[TM][TN];                                // the accumulator of each output: a finite FP32 / FP16 word (FP16 path)
     uint32_t sp_nan = 0u, sp_pinf = 0u, sp_ninf = 0u;   // per output (bit r * TN + c): NaN / +inf / -inf seen so far
     float promoted[PROMOTE ? TM : 1][PROMOTE ? TN : 1];
 #define MMASIM_SP_GET(r, c) ((((sp_nan >> ((r) * TN + (c))) & 1u)) | (((sp_pinf >> ((r) * TN + (c))) & 1u) << 1) | (((sp_ninf >> ((r) * TN + (c))) & 1u) << 2))
@@ -338,6 +349,10 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
                 w = 0u;
             }
             cw[r][c] = w;
+            if (DS) {
+                cs[DS ? r : 0][DS ? c : 0] = state_of(w);
+                if ((w & 0x7F800000u) == 0u && (w & 0x007FFFFFu) != 0u) sub_mask |= 1u << (r * TN + c);
+            }
         }
 
     RawChunk<EK> raw;
@@ -416,6 +431,37 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
             // the grid: a negative c floors to the one's complement), then + 1 if c < 0.
             // ST: the products are compared against Exp(c) minus the block's scale exponents, c is scaled likewise.
             double acc[TM][TN];
+            if (DS) {
+                // keys are exponent fields of doubles in place: (Exp + 1023) << 20.  Products: the larger 16-bit lane of emp
+                // (Exp + CB, CB = 1024); c: the state's own field (0 for c = 0: below every real key), minus the scale
+                // exponents for ST; an FP32 subnormal c counts with Exp = -126 (rare: patched below).
+                constexpr int KM = ((52 - 0) << 20) | 0x00080000;    // + (e_max - F) gives the high word of 1.5 * 2^52 * q
+                const int km = KM - (m.F << 20);
+                auto start = [&](int r, int c, bool subnormal_c) {
+                    const double st = cs[DS ? r : 0][DS ? c : 0];
+                    const int hi = __double2hiint(st);
+                    int keyc = subnormal_c ? (1023 - 126) << 20 : hi & 0x7FF00000;
+                    if (ST) keyc -= (sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]) << 20;
+                    const uint32_t e2 = emp[r][c];
+                    const int keyp = int(__vmaxu2(e2, __byte_perm(e2, 0u, 0x1032)) & 0xFFFFu) * (1 << 20) - (1 << 20);
+                    const int e20 = ST ? __vimax3_s32(keyp, keyc, 0) : max(keyp, keyc);
+                    // the +1 of a negative c sits in the constant's low word: one unit of the grid either way
+                    const double magic = __hiloint2double(e20 + km, int(uint32_t(hi) >> 31));
+                    const double x = ST ? __dmul_rn(st, pow2d(-(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]))) : st;
+                    acc[r][c] = __dadd_rd(x, magic);
+                };
+#pragma unroll
+                for (int r = 0; r < TM; ++r)
+#pragma unroll
+                    for (int c = 0; c < TN; ++c) start(r, c, false);
+                if (sub_mask) {                         // rare: redo the outputs whose accumulator is an FP32 subnormal
+#pragma unroll
+                    for (int r = 0; r < TM; ++r)
+#pragma unroll
+                        for (int c = 0; c < TN; ++c)
+                            if ((sub_mask >> (r * TN + c)) & 1u) start(r, c, true);
+                }
+            } else
 #pragma unroll
             for (int r = 0; r < TM; ++r)
 #pragma unroll
@@ -491,6 +537,39 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
                 if (ST) v = __dmul_rn(v, pow2d(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]));
                 return v;
             };
+            if (DS) {
+                bool odd = false;                       // some result is not a normal FP32 number
+#pragma unroll
+                for (int r = 0; r < TM; ++r) {
+                    const uint32_t sa = s.a_sgn[prow + r], nza = s.a_nz[prow + r] & kmask;
+#pragma unroll
+                    for (int c = 0; c < TN; ++c) {
+                        const double v = block_value(r, c, sa, nza);
+                        odd = odd || !(fabs(v) >= 1.1754943508222875e-38) || !(fabs(v) < 3.402823669209385e38);
+                        // RZ-FP32 of a number in the normal range: the low 29 bits of the double's significand go
+                        cs[DS ? r : 0][DS ? c : 0] = __hiloint2double(__double2hiint(v), (__double2loint(v) & int(0xE0000000u)) | 1);
+                    }
+                }
+                if (odd || sub_mask) {                  // rare: zero, FP32 subnormal or overflow somewhere in the micro-tile
+                    sub_mask = 0u;
+#pragma unroll
+                    for (int r = 0; r < TM; ++r)
+#pragma unroll
+                        for (int c = 0; c < TN; ++c) {
+                            const double st = cs[DS ? r : 0][DS ? c : 0];
+                            const double v = __hiloint2double(__double2hiint(st), __double2loint(st) & ~1);
+                            const uint32_t bit = 1u << (r * TN + c);
+                            if (fabs(v) >= 3.402823669209385e38) {                        // |v| >= 2^128: +-infinity from now on
+                                if (!((sp_nan | sp_pinf | sp_ninf) & bit)) { if (v < 0.0) sp_ninf |= bit; else sp_pinf |= bit; }
+                                cs[DS ? r : 0][DS ? c : 0] = state_of(0u);
+                            } else if (fabs(v) < 1.1754943508222875e-38) {                // zero or below 2^-126: the word decides
+                                const uint32_t w = __float_as_uint(__double2float_rz(v));
+                                cs[DS ? r : 0][DS ? c : 0] = state_of(w);
+                                if (w & 0x7FFFFFFFu) sub_mask |= bit;
+                            }
+                        }
+                }
+            } else {
 #pragma unroll
             for (int r = 0; r < TM; ++r) {
                 const uint32_t sa = s.a_sgn[prow + r], nza = s.a_nz[prow + r] & kmask;
@@ -502,7 +581,8 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
                     cw[r][c] = w;
                 }
             }
-            if (wmax >= SUSPECT) {
+            }
+            if (!DS && wmax >= SUSPECT) {
 #pragma unroll
                 for (int r = 0; r < TM; ++r) {
                     const uint32_t sa = s.a_sgn[prow + r], nza = s.a_nz[prow + r] & kmask;
@@ -527,13 +607,15 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
                 for (int c = 0; c < TN; ++c) {
                     const uint32_t sp = MMASIM_SP_GET(r, c);
                     const uint32_t pw = sp ? special_word(((sp & 1u) || (sp & 6u) == 6u) ? 1 : ((sp & 2u) ? 2 : 3), ACC16, true)
-                                           : positive_zero(cw[r][c], 0x7FFFFFFFu);
+                                           : positive_zero(DS ? word_of(cs[DS ? r : 0][DS ? c : 0]) : cw[r][c], 0x7FFFFFFFu);
                     float v = __fadd_rn(promoted[PROMOTE ? r : 0][PROMOTE ? c : 0], __uint_as_float(pw));
                     if (v != v) v = __uint_as_float(0x7FFFFFFFu);
                     promoted[PROMOTE ? r : 0][PROMOTE ? c : 0] = v;
                     cw[r][c] = 0u;
+                    if (DS) cs[DS ? r : 0][DS ? c : 0] = state_of(0u);
                 }
             sp_nan = sp_pinf = sp_ninf = 0u;
+            sub_mask = 0u;
         }
     }
 
@@ -547,7 +629,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
             const uint32_t sp = MMASIM_SP_GET(r, c);
             uint32_t w = PROMOTE ? __float_as_uint(promoted[PROMOTE ? r : 0][PROMOTE ? c : 0])
                                  : (sp ? special_word(((sp & 1u) || (sp & 6u) == 6u) ? 1 : ((sp & 2u) ? 2 : 3), ACC16, true)
-                                       : positive_zero(cw[r][c], ACC16 ? 0x7FFFu : 0x7FFFFFFFu));   // a zero result is +0
+                                       : positive_zero(DS ? word_of(cs[DS ? r : 0][DS ? c : 0]) : cw[r][c], ACC16 ? 0x7FFFu : 0x7FFFFFFFu));   // a zero result is +0
             if (g.row_scale) {
                 float sc = __fmul_rn(g.row_scale[i], g.col_scale[j]);
                 if (sc != sc) sc = __uint_as_float(0x7FFFFFFFu);
