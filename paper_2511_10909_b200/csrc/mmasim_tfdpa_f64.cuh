@@ -239,6 +239,135 @@ __device__ __forceinline__ void store_chunk64(SM& sm, PL& s, const RawChunk<EK>&
     if (spec) atomicOr(&sm.special[flag], 1);
 }
 
+// One operand's share of a chunk of KC = 32 elements of K, decoded for the matrix-instruction kernel: R rows of A (or
+// columns of B).  A decode kernel writes these blocks to scratch memory once per GEMM; the main kernel brings them in with
+// one bulk copy each.  Layouts as in Planes64<EK, true>; `pe` holds BF16 powers 2^(BASE (Exp - 1)) for the tensor-core
+// exponent maximum of the element kinds whose exponent sums fit (FP16 and the 8-bit kinds).
+constexpr int PE_STRIDE64 = KC + 8;     // 80 bytes per row: fragment loads hit 32 different banks
+template <int R>
+struct Blk64 {
+    double d[R][KP];
+    uint32_t exp2[KC / 2][R];
+    uint16_t pe[R][PE_STRIDE64];
+    uint32_t sgn[R], nz[R];
+    uint32_t special, pad[3];
+};
+static_assert(sizeof(Blk64<BM>) % 16 == 0 && sizeof(Blk64<BN>) % 16 == 0, "bulk copies move multiples of 16 bytes");
+
+struct SmemMM {
+    Blk64<BM> a[2];
+    Blk64<BN> b[2];
+    unsigned long long full[2];         // mbarriers: the bulk copies of a buffer have landed
+    int error;                          // a bounded wait ran out
+};
+
+// Base of the exponent powers by element kinds (see the F = 13 kernel for the argument): a sum of at most 2^(BASE-1)
+// terms stays within 2^(BASE-1) of its largest term, and BASE times the spread of the exponent sums has to fit FP32.
+//   FP16 x FP16 (sums -28..30): BASE 4, sub-blocks of 8 terms; 8-bit kinds: 8 (E4M3 / FP6 / FP4 only: one accumulation of
+//   32), 5 (one E5M2 operand: sub-blocks of 16), 4 (two: sub-blocks of 8); BF16 and TF32 do not fit: BASE 0, add-max pass.
+__host__ __device__ constexpr int pe64_shift(int base) { return base == 5 ? 3 : 1; }       // (127 + shift) % base == 0
+__host__ __device__ constexpr int pe64_sub(int base) { return base == 8 ? 32 : (base == 5 ? 16 : 8); }
+
+// Decode pass: one CTA of 256 threads decodes one block (R rows x 32 elements) into shared memory and copies it to its
+// place dst[tile][chunk].  Rows beyond the matrix decode as zeros.
+template <int EK, int R, bool IS_A, int BASE>
+__global__ void __launch_bounds__(256) decode64_kernel(DevModel m, const unsigned char* src, int64_t rows, int64_t ld, Blk64<R>* dst) {
+    using E = Elem<EK>;
+    constexpr int TPR = KC / E::TASK, TASKS = R * TPR, WORDS = E::TASK * E::BYTES / 4;
+    extern __shared__ __align__(16) unsigned char dec_smem[];
+    LutEntry64* lut = reinterpret_cast<LutEntry64*>(dec_smem);
+    Blk64<R>& blk = *reinterpret_cast<Blk64<R>*>(dec_smem + 256 * sizeof(LutEntry64));
+    const int tid = threadIdx.x;
+    if (!E::SIGNMAG) {
+        const FmtDesc f = fmt_desc(IS_A ? m.fmt_a : m.fmt_b);
+        const uint32_t dd = decode_elem(f, uint32_t(tid));
+        const bool fin = dec_cls(dd) == CLS_FINITE;
+        const uint32_t sg = fin ? dec_sig(dd) : 0u;
+        LutEntry64 e;
+        e.op = IS_A ? operand_a(fin ? dec_sign(dd) : 0u, sg, fin ? dec_exp(dd) : 0, f.mbits)
+                    : operand_b(fin ? dec_sign(dd) : 0u, sg, fin ? dec_exp(dd) : 0, f.mbits);
+        e.exp = sg ? uint32_t(dec_exp(dd) + EB) : 0u;
+        e.bits = (fin ? dec_sign(dd) : 0u) | (fin ? 0u : 2u) | (sg ? 4u : 0u);
+        lut[tid] = e;
+    }
+    if (tid == 0) { blk.special = 0u; blk.pad[0] = blk.pad[1] = blk.pad[2] = 0u; }
+    __syncthreads();
+    const int64_t k0 = int64_t(blockIdx.x) * KC;
+    uint32_t spec = 0u;
+    for (int task = tid; task < TASKS; task += 256) {
+        const int r = task % R, h = task / R;
+        const int pr = IS_A ? perm_row64(r) : perm_col64(r);
+        const int64_t grow = int64_t(blockIdx.y) * R + r;
+        uint32_t w[WORDS];
+#pragma unroll
+        for (int q = 0; q < WORDS / 4; ++q) {
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (grow < rows) v = reinterpret_cast<const uint4*>(src + (grow * ld + k0 + h * E::TASK) * E::BYTES)[q];
+            w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
+        }
+        uint32_t bits = 0u, prev_exp = 0u, pw[E::TASK / 2];
+#pragma unroll
+        for (int q = 0; q < E::TASK; ++q) {
+            const int kk = h * E::TASK + q;
+            double op;
+            uint32_t expb;
+            if (!E::SIGNMAG) {
+                const uint32_t byte = (w[q / 4] >> (8 * (q % 4))) & 0xFFu;
+                const LutEntry64 e = lut[byte];
+                op = e.op;
+                expb = e.exp;
+                bits += ((e.bits & 1u) | ((e.bits & 4u) << 14)) << q;
+                spec |= e.bits & 2u;
+            } else {
+                const uint32_t x = E::BYTES == 2 ? ((w[q / 2] >> (16 * (q % 2))) & 0xFFFFu) : w[q];
+                constexpr uint32_t TOP = (1u << E::EBITS) - 1u;
+                const uint32_t xx = x >> E::LOW;
+                const uint32_t mag = xx & ((1u << (E::EBITS + E::MBITS)) - 1u);
+                const uint32_t field = mag >> E::MBITS;
+                const uint32_t sign = (xx >> (E::EBITS + E::MBITS)) & 1u;
+                uint32_t hi = 0u, lo = 0u, nzbit = 1u;
+                expb = 0u;
+                if (field - 1u < TOP - 1u) {
+                    hi = (mag << (20 - E::MBITS)) + (uint32_t(1023 - E::BIAS) << 20);
+                    lo = IS_A ? 0u : (1u << (22 - E::MBITS));
+                    expb = field + uint32_t(EB - E::BIAS);
+                } else if (field == 0u && mag != 0u) {
+                    const double v = IS_A ? operand_a(0u, mag, 1 - E::BIAS, E::MBITS) : operand_b(0u, mag, 1 - E::BIAS, E::MBITS);
+                    hi = uint32_t(__double2hiint(v));
+                    lo = uint32_t(__double2loint(v));
+                    expb = uint32_t(1 - E::BIAS + EB);
+                } else {
+                    nzbit = 0u;
+                    spec |= uint32_t(field == TOP);
+                }
+                op = __hiloint2double(int(hi | (sign << 31)), int(lo));
+                bits += (sign | (nzbit << 16)) << q;
+            }
+            blk.d[r][kk] = op;
+            // BF16 word of 2^(BASE (Exp - 1)) (the B plane times 2^shift); 0 for an element without exponent
+            const uint32_t pe = (BASE && expb) ? uint32_t((127 + (IS_A ? 0 : pe64_shift(BASE)) + BASE * (int(expb) - EB - 1)) << 7) : 0u;
+            if (q & 1) {
+                blk.exp2[kk / 2][pr] = prev_exp | (expb << 16);
+                pw[q / 2] |= pe << 16;
+            } else pw[q / 2] = pe;
+            prev_exp = expb;
+        }
+#pragma unroll
+        for (int q = 0; q < E::TASK / 8; ++q)
+            reinterpret_cast<uint4*>(&blk.pe[r][h * E::TASK])[q] = make_uint4(pw[4 * q], pw[4 * q + 1], pw[4 * q + 2], pw[4 * q + 3]);
+        if (E::TASK == 16) {
+            reinterpret_cast<uint16_t*>(&blk.sgn[pr])[h] = uint16_t(bits); reinterpret_cast<uint16_t*>(&blk.nz[pr])[h] = uint16_t(bits >> 16);
+        } else {
+            reinterpret_cast<uint8_t*>(&blk.sgn[pr])[h] = uint8_t(bits); reinterpret_cast<uint8_t*>(&blk.nz[pr])[h] = uint8_t(bits >> 16);
+        }
+    }
+    if (spec) atomicOr(&blk.special, 1u);
+    __syncthreads();
+    uint4* out = reinterpret_cast<uint4*>(dst + (int64_t(blockIdx.y) * gridDim.x + blockIdx.x));
+    const uint4* in = reinterpret_cast<const uint4*>(&blk);
+    for (int q = tid; q < int(sizeof(Blk64<R>) / 16); q += 256) out[q] = in[q];
+}
+
 // Columns of a thread's micro-tile in the k-major layout: two adjacent pairs, 32 columns apart, so that the sixteen
 // threads of a row of the thread grid read 256 contiguous bytes of B operands per 16-byte load.
 __device__ __forceinline__ int col_of(int tx, int c) { return (c >> 1) * (BN / 2) + tx * 2 + (c & 1); }
@@ -292,16 +421,16 @@ __device__ __forceinline__ void product_exponents_adj(const uint32_t* ea_p, cons
 // n + 1 is fused, instruction by instruction, into the multiply-add pass of block n - the integer pipe works in
 // the issue slots that the FP64 pipe leaves free.
 template <int EK, int L, int RHO, bool PROMOTE, bool ST>
-__global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) {
+__global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, const Blk64<BM>* __restrict__ wa,
+                                                        const Blk64<BN>* __restrict__ wb) {
     using E = Elem<EK>;
     constexpr bool ACC16 = RHO == RHO_RNE_FP16;
     constexpr int NBLK = KC / L;
     static_assert(RHO == RHO_RZ_FP32 || RHO == RHO_RNE_FP16, "rho is a single conversion from FP64");
     static_assert(KC % L == 0 && L % 4 == 0, "blocks tile the chunk; pass 1 handles pairs of elements");
     static_assert(!ST || L == KC, "ST-FDPA: one scale factor pair per block of 32 (Algorithm 8)");
-    using SM = Smem64<EK, true>;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    SM& sm = *reinterpret_cast<SM*>(smem_raw);
+    SmemMM& sm = *reinterpret_cast<SmemMM*>(smem_raw);
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
@@ -314,8 +443,24 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
     // high word of 1.5 * 2^52 * 2^(e_max - F) is (e_max + CB) * 2^20 + MAGIC_K
     const int MAGIC_K = ((1023 + 52 - m.F - CB) << 20) | 0x00080000;
 
-    init_lut64<EK>(sm, fa, fb, tid);
-    if (tid == 0) sm.special[0] = sm.special[1] = sm.special[2] = 0;
+    // the decoded blocks of this tile row of A and tile column of B, chunk after chunk, land in two buffers by bulk copies
+    const int NCH = int(g.K / KC);
+    const Blk64<BM>* src_a = wa + int64_t(blockIdx.y) * NCH;
+    const Blk64<BN>* src_b = wb + int64_t(blockIdx.x) * NCH;
+    auto issue = [&](int n) {                              // one thread: both copies of chunk n into buffer n & 1
+        unsigned long long* bar = &sm.full[n & 1];
+        fast::mbar_expect_tx(bar, uint32_t(sizeof(Blk64<BM>) + sizeof(Blk64<BN>)));
+        fast::bulk_load(&sm.a[n & 1], src_a + n, uint32_t(sizeof(Blk64<BM>)), bar);
+        fast::bulk_load(&sm.b[n & 1], src_b + n, uint32_t(sizeof(Blk64<BN>)), bar);
+    };
+    if (tid == 0) {
+        sm.error = 0;
+        fast::mbar_init(&sm.full[0], 1u);
+        fast::mbar_init(&sm.full[1], 1u);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        issue(0);
+        if (NCH > 1) issue(1);
+    }
 
     // FP32 accumulators live between blocks as doubles ("state"): the value RZ-FP32 produced, exactly, with bit 0 of the
     // low word set so that the next block's addition (rounded toward minus infinity) never finds it on its grid; the
@@ -355,29 +500,19 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
             }
         }
 
-    RawChunk<EK> raw;
-    load_chunk<EK>(raw, g, row0, col0, 0, tid);
-    __syncthreads();                                    // tables and flags are ready
-    store_chunk64<EK>(sm, sm.pl[0], raw, 0, tid);
-    if (KC < g.K) load_chunk<EK>(raw, g, row0, col0, KC, tid);
-    __syncthreads();
+    __syncthreads();                                    // the barriers are initialised
     uint32_t emp[TM][TN];                               // product exponents of the block that comes next
 
-    int chunk = 0;
-    for (int64_t k0 = 0; k0 < g.K; k0 += KC, ++chunk) {
-        auto& s = sm.pl[chunk & 1];
-        auto& nx = sm.pl[(chunk + 1) & 1];
-        // decode chunk n + 1 into the other buffer (its raw words arrived during the previous iteration; every warp left
-        // that buffer before the barrier that ended the previous iteration), fetch n + 2.  One barrier per chunk: the
-        // warps drift apart, and some decode while others keep the FP64 pipe busy.
-        if (tid == 0) sm.special[(chunk + 2) % 3] = 0;  // last read two barriers ago, next written after the coming one
-        if (k0 + KC < g.K) {
-            store_chunk64<EK>(sm, nx, raw, (chunk + 1) % 3, tid);
-            if (k0 + 2 * KC < g.K) load_chunk<EK>(raw, g, row0, col0, k0 + 2 * KC, tid);
-        }
-        const bool chunk_special = sm.special[chunk % 3] != 0;
+    for (int chunk = 0; chunk < NCH; ++chunk) {
+        const int64_t k0 = int64_t(chunk) * KC;
+        // a wait that runs out is recorded and the chunk computed on whatever is there; every thread sees the flag after
+        // the barrier at the end of the chunk, and the CTA leaves together without storing anything
+        if (!fast::mbar_wait(&sm.full[chunk & 1], uint32_t(chunk >> 1) & 1u)) *reinterpret_cast<volatile int*>(&sm.error) = 1;
+        const Blk64<BM>& sa_blk = sm.a[chunk & 1];
+        const Blk64<BN>& sb_blk = sm.b[chunk & 1];
+        const bool chunk_special = (sa_blk.special | sb_blk.special) != 0u;
         // the first block's product exponents (the other blocks' are taken beside the multiply-adds of their predecessor)
-        product_exponents_adj<L>(&s.a_exp2[0][prow], &s.b_exp2[0][pcol], emp);
+        product_exponents_adj<L>(&sa_blk.exp2[0][prow], &sb_blk.exp2[0][pcol], emp);
 
         // ST-FDPA (Algorithm 8): Exp(alpha) of this thread's rows and Exp(beta) of its columns for this block of 32
         int sa_exp[ST ? TM : 1], sb_exp[ST ? TN : 1];
@@ -482,8 +617,8 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
             // the chunk has another block, the product exponents of that block ----
             auto multiply_adds = [&](auto with_exponents) {
                 constexpr bool FUSE = decltype(with_exponents)::value;
-                const uint32_t* ea_p = &s.a_exp2[FUSE ? (kb + L) / 2 : 0][prow];
-                const uint32_t* eb_p = &s.b_exp2[FUSE ? (kb + L) / 2 : 0][pcol];
+                const uint32_t* ea_p = &sa_blk.exp2[FUSE ? (kb + L) / 2 : 0][prow];
+                const uint32_t* eb_p = &sb_blk.exp2[FUSE ? (kb + L) / 2 : 0][pcol];
                 if (FUSE) {
 #pragma unroll
                     for (int r = 0; r < TM; ++r)
@@ -497,9 +632,9 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
                 for (int ks = 0; ks < L; ks += 4) {
                     double af[TM], bf[TN / 2];
 #pragma unroll
-                    for (int r = 0; r < TM; ++r) af[r] = s.a_d[wr * 32 + 8 * r + gq][kb + ks + tq];
+                    for (int r = 0; r < TM; ++r) af[r] = sa_blk.d[wr * 32 + 8 * r + gq][kb + ks + tq];
 #pragma unroll
-                    for (int j = 0; j < TN / 2; ++j) bf[j] = s.b_d[wc * 16 + 8 * j + gq][kb + ks + tq];
+                    for (int j = 0; j < TN / 2; ++j) bf[j] = sb_blk.d[wc * 16 + 8 * j + gq][kb + ks + tq];
 #pragma unroll
                     for (int r = 0; r < TM; ++r)
 #pragma unroll
@@ -529,7 +664,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
             constexpr uint32_t SUSPECT = ACC16 ? 0x7C00u : 0x7F7FFFFFu;   // FP16: infinity; FP32: cvt.rz saturates at the largest finite word
             uint32_t wmax = 0u;
             auto block_value = [&](int r, int c, uint32_t sa, uint32_t nza) -> double {
-                const int nneg = __popc((sa ^ s.b_sgn[pcol + c]) & nza & s.b_nz[pcol + c]);
+                const int nneg = __popc((sa ^ sb_blk.sgn[pcol + c]) & nza & sb_blk.nz[pcol + c]);
                 const long long bits = __double_as_longlong(acc[r][c]) + (long long)nneg;
                 const int hi = int(bits >> 32);
                 const double magic = __hiloint2double((hi & 0x7FF00000) | 0x00080000, 0);
@@ -541,7 +676,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
                 bool odd = false;                       // some result is not a normal FP32 number
 #pragma unroll
                 for (int r = 0; r < TM; ++r) {
-                    const uint32_t sa = s.a_sgn[prow + r], nza = s.a_nz[prow + r] & kmask;
+                    const uint32_t sa = sa_blk.sgn[prow + r], nza = sa_blk.nz[prow + r] & kmask;
 #pragma unroll
                     for (int c = 0; c < TN; ++c) {
                         const double v = block_value(r, c, sa, nza);
@@ -572,7 +707,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
             } else {
 #pragma unroll
             for (int r = 0; r < TM; ++r) {
-                const uint32_t sa = s.a_sgn[prow + r], nza = s.a_nz[prow + r] & kmask;
+                const uint32_t sa = sa_blk.sgn[prow + r], nza = sa_blk.nz[prow + r] & kmask;
 #pragma unroll
                 for (int c = 0; c < TN; ++c) {
                     const double v = block_value(r, c, sa, nza);
@@ -585,7 +720,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
             if (!DS && wmax >= SUSPECT) {
 #pragma unroll
                 for (int r = 0; r < TM; ++r) {
-                    const uint32_t sa = s.a_sgn[prow + r], nza = s.a_nz[prow + r] & kmask;
+                    const uint32_t sa = sa_blk.sgn[prow + r], nza = sa_blk.nz[prow + r] & kmask;
 #pragma unroll
                     for (int c = 0; c < TN; ++c) {
                         if ((cw[r][c] & ABS) != SUSPECT) continue;
@@ -598,7 +733,9 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
                 }
             }
         }
-        __syncthreads();                                // the other buffer is complete, this one is free
+        __syncthreads();                                // everybody has finished with this buffer
+        if (*reinterpret_cast<volatile int*>(&sm.error)) break;
+        if (tid == 0 && chunk + 2 < NCH) issue(chunk + 2);
         // ---- FP32 promotion of the partial sum every k_chunk elements ----
         if (PROMOTE && ((k0 + KC) % g.k_chunk) == 0) {
 #pragma unroll
@@ -619,6 +756,14 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
         }
     }
 
+    if (*reinterpret_cast<volatile int*>(&sm.error)) {  // a copy never arrived: count it, give the copies in flight one more
+        if (tid == 0) {                                 // bounded wait each, and store nothing
+            atomicAdd(&fast::g_copy_timeouts, 1u);
+            fast::mbar_wait(&sm.full[0], 0u);
+            fast::mbar_wait(&sm.full[1], 0u);
+        }
+        return;
+    }
     // ---- store ----
 #pragma unroll
     for (int r = 0; r < TM; ++r)
@@ -645,12 +790,31 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g) 
 
 template <int EK, int L, int RHO, bool PROMOTE, bool ST = false>
 cudaError_t launch_one64(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
-    const size_t sh = sizeof(Smem64<EK, true>);
+    constexpr int BASE = 0;
+    const size_t sh = sizeof(SmemMM);
     cudaError_t err = cudaFuncSetAttribute(tfdpa64_kernel<EK, L, RHO, PROMOTE, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
     if (err != cudaSuccess) return err;
-    dim3 grid((unsigned)((g.N + BN - 1) / BN), (unsigned)((g.M + BM - 1) / BM), 1);
-    tfdpa64_kernel<EK, L, RHO, PROMOTE, ST><<<grid, NT, sh, stream>>>(m, g);
-    return cudaGetLastError();
+    const size_t dsh_a = 256 * sizeof(LutEntry64) + sizeof(Blk64<BM>), dsh_b = 256 * sizeof(LutEntry64) + sizeof(Blk64<BN>);
+    if ((err = cudaFuncSetAttribute(decode64_kernel<EK, BM, true, BASE>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(dsh_a))) != cudaSuccess) return err;
+    if ((err = cudaFuncSetAttribute(decode64_kernel<EK, BN, false, BASE>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(dsh_b))) != cudaSuccess) return err;
+    const int64_t tiles_m = (g.M + BM - 1) / BM, tiles_n = (g.N + BN - 1) / BN, nch = g.K / KC;
+    // scratch: the decoded blocks of A and B, stream-ordered out of the library's pool and returned to it behind the kernel
+    const size_t bytes_a = size_t(tiles_m * nch) * sizeof(Blk64<BM>), bytes_b = size_t(tiles_n * nch) * sizeof(Blk64<BN>);
+    cudaMemPool_t pool = nullptr;
+    if ((err = scratch_pool(&pool)) != cudaSuccess) return err;
+    void* ws = nullptr;
+    if ((err = cudaMallocFromPoolAsync(&ws, bytes_a + bytes_b, pool, stream)) != cudaSuccess) return err;
+    Blk64<BM>* wa = static_cast<Blk64<BM>*>(ws);
+    Blk64<BN>* wb = reinterpret_cast<Blk64<BN>*>(static_cast<unsigned char*>(ws) + bytes_a);
+    decode64_kernel<EK, BM, true, BASE><<<dim3((unsigned)nch, (unsigned)tiles_m), 256, dsh_a, stream>>>(
+        m, static_cast<const unsigned char*>(g.A), g.M, g.lda, wa);
+    decode64_kernel<EK, BN, false, BASE><<<dim3((unsigned)nch, (unsigned)tiles_n), 256, dsh_b, stream>>>(
+        m, static_cast<const unsigned char*>(g.B), g.N, g.ldb, wb);
+    dim3 grid((unsigned)tiles_n, (unsigned)tiles_m, 1);
+    tfdpa64_kernel<EK, L, RHO, PROMOTE, ST><<<grid, NT, sh, stream>>>(m, g, wa, wb);
+    err = cudaGetLastError();
+    const cudaError_t err2 = cudaFreeAsync(ws, stream);
+    return err != cudaSuccess ? err : err2;
 }
 
 // With or without FP32 promotion (FP32 accumulators only).

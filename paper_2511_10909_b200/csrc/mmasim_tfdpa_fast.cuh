@@ -60,6 +60,34 @@ __device__ __forceinline__ uint32_t raw_elem(const void* p, int64_t idx) {
     return static_cast<const uint32_t*>(p)[idx];
 }
 
+// ---- bulk copies and their barrier: inline PTX ----
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return uint32_t(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+// Waits for the given phase of the barrier; gives up after a bounded number of polls (each poll itself blocks for a
+// bounded, implementation-defined time) and returns false.
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity) {
+    const uint32_t addr = smem_addr(bar);
+    for (int spin = 0; spin < (1 << 22); ++spin) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+// Counts the CTAs whose bounded wait on a bulk copy ran out (never in a healthy run; such a CTA stores nothing).
+static __device__ unsigned int g_copy_timeouts = 0u;
+
 // Per element kind: returns cudaErrorInvalidValue when (L, F, rho) has no instantiation.
 cudaError_t launch_lut8(const DevModel& m, const GemmArgs& g, cudaStream_t stream);
 cudaError_t launch_f16(const DevModel& m, const GemmArgs& g, cudaStream_t stream);

@@ -46,6 +46,11 @@ using fast::NT;
 using fast::CB;
 using fast::Elem;
 using fast::raw_elem;
+using fast::mbar_init;
+using fast::mbar_expect_tx;
+using fast::bulk_load;
+using fast::mbar_wait;
+using fast::smem_addr;
 
 constexpr int PE_STRIDE = KC + 8;       // BF16 elements per row of a pe plane: 80 bytes, fragment loads hit 32 different banks
 constexpr int PE_CENTER = 1;            // pe(x) = 2^(6 (Exp(x) - PE_CENTER)); E4M3: Exp in [-6, 8]
@@ -193,33 +198,6 @@ __global__ void __launch_bounds__(NT) trop_decode_kernel(DevModel m, const unsig
     for (int q = tid; q < int(sizeof(BlkT<R>) / 16); q += NT) out[q] = in[q];
 }
 
-// ---- bulk copies and their barrier: inline PTX ----
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return uint32_t(__cvta_generic_to_shared(p)); }
-__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_addr(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_addr(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 :: "r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
-}
-// Waits for the given phase of the barrier; gives up after a bounded number of polls (each poll itself blocks for a
-// bounded, implementation-defined time) and returns false.
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity) {
-    const uint32_t addr = smem_addr(bar);
-    for (int spin = 0; spin < (1 << 22); ++spin) {
-        uint32_t done;
-        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(done) : "r"(addr), "r"(parity) : "memory");
-        if (done) return true;
-    }
-    return false;
-}
-
-// Set when a bounded wait on a bulk copy ran out (never in a healthy run); read by mmasim_device_status.
-__device__ unsigned int g_trop_timeouts = 0u;
 
 template <int EK, int L, int F, int RHO, bool PROMOTE, int BASE, int TH>
 __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs g, const BlkT<BM>* __restrict__ wa,
@@ -557,7 +535,7 @@ __global__ void __launch_bounds__(NT, 2) tfdpa_trop_kernel(DevModel m, GemmArgs 
 
     if (*reinterpret_cast<volatile int*>(&sm.error)) {     // a copy never arrived: count it, give the copies in flight one more
         if (tid == 0) {                                    // bounded wait each, and store nothing
-            atomicAdd(&g_trop_timeouts, 1u);
+            atomicAdd(&fast::g_copy_timeouts, 1u);
             mbar_wait(&sm.full[0], 0u);
             mbar_wait(&sm.full[1], 0u);
         }
