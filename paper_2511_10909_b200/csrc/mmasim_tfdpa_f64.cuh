@@ -420,9 +420,14 @@ __device__ __forceinline__ void product_exponents_adj(const uint32_t* ea_p, cons
 // between two barriers while its raw words were fetched a chunk earlier), and the product-exponent pass of block
 // n + 1 is fused, instruction by instruction, into the multiply-add pass of block n - the integer pipe works in
 // the issue slots that the FP64 pipe leaves free.
-template <int EK, int L, int RHO, bool PROMOTE, bool ST>
+template <int EK, int L, int RHO, bool PROMOTE, bool ST, int BASE>
 __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, const Blk64<BM>* __restrict__ wa,
                                                         const Blk64<BN>* __restrict__ wb) {
+    // BASE > 0: the block maximum of the product exponents comes from the tensor cores (a product of powers BASE^Exp on
+    // BF16 planes, as in the F = 13 kernel); BASE = 0: from fused add-max instructions on packed exponent pairs.
+    static_assert(BASE == 0 || ((BASE == 4 || BASE == 8) && L >= 8), "see pe64_shift / pe64_sub");
+    constexpr int LB = BASE == 8 ? 3 : 2;                       // log2(BASE)
+    constexpr int KP2 = (1023 + 2 - (127 + 1) / (BASE ? BASE : 1)) << 20;   // P-domain key + KP2 = (e_max + 1023) << 20
     using E = Elem<EK>;
     constexpr bool ACC16 = RHO == RHO_RNE_FP16;
     constexpr int NBLK = KC / L;
@@ -512,7 +517,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
         const Blk64<BN>& sb_blk = sm.b[chunk & 1];
         const bool chunk_special = (sa_blk.special | sb_blk.special) != 0u;
         // the first block's product exponents (the other blocks' are taken beside the multiply-adds of their predecessor)
-        product_exponents_adj<L>(&sa_blk.exp2[0][prow], &sb_blk.exp2[0][pcol], emp);
+        if (BASE == 0) product_exponents_adj<L>(&sa_blk.exp2[0][prow], &sb_blk.exp2[0][pcol], emp);
 
         // ST-FDPA (Algorithm 8): Exp(alpha) of this thread's rows and Exp(beta) of its columns for this block of 32
         int sa_exp[ST ? TM : 1], sb_exp[ST ? TN : 1];
@@ -561,6 +566,63 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                     }
             }
 
+            if (BASE) {
+                // ---- pass 1 on the tensor cores: P = sum_k pe(a_k) pe(b_k) per sub-block of KSUB terms, the block's P the
+                // integer maximum of their words; emp receives the raw words (0: no nonzero product) ----
+                constexpr int KSUB = pe64_sub(BASE) < L ? pe64_sub(BASE) : L, NSUB = L / KSUB;
+                constexpr int NK = KSUB >= 16 ? KSUB / 16 : 1, AR = KSUB >= 16 ? 4 : 2, BR = KSUB >= 16 ? 2 : 1;
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt) {
+                    uint32_t P[2][4];
+#pragma unroll
+                    for (int sub = 0; sub < NSUB; ++sub) {
+                        uint32_t af[NK][AR];
+                        const int ar = wr * 32 + 16 * mt + gq;
+#pragma unroll
+                        for (int ks = 0; ks < NK; ++ks) {
+                            const int kq = kb + sub * KSUB + 16 * ks + 2 * tq;
+                            af[ks][0] = *reinterpret_cast<const uint32_t*>(&sa_blk.pe[ar][kq]);
+                            af[ks][1] = *reinterpret_cast<const uint32_t*>(&sa_blk.pe[ar + 8][kq]);
+                            if (AR == 4) {
+                                af[ks][AR - 2] = *reinterpret_cast<const uint32_t*>(&sa_blk.pe[ar][kq + 8]);
+                                af[ks][AR - 1] = *reinterpret_cast<const uint32_t*>(&sa_blk.pe[ar + 8][kq + 8]);
+                            }
+                        }
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {
+                            uint32_t bf[NK][BR];
+#pragma unroll
+                            for (int ks = 0; ks < NK; ++ks) {
+                                const int kq = kb + sub * KSUB + 16 * ks + 2 * tq;
+                                bf[ks][0] = *reinterpret_cast<const uint32_t*>(&sb_blk.pe[wc * 16 + 8 * j + gq][kq]);
+                                if (BR == 2) bf[ks][BR - 1] = *reinterpret_cast<const uint32_t*>(&sb_blk.pe[wc * 16 + 8 * j + gq][kq + 8]);
+                            }
+                            float d[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                            for (int ks = 0; ks < NK; ++ks) {
+                                if (KSUB >= 16)
+                                    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                                                 : "r"(af[ks][0]), "r"(af[ks][1]), "r"(af[ks][AR - 2]), "r"(af[ks][AR - 1]),
+                                                   "r"(bf[ks][0]), "r"(bf[ks][BR - 1]));
+                                else
+                                    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+                                                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                                                 : "r"(af[ks][0]), "r"(af[ks][1]), "r"(bf[ks][0]));
+                            }
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                P[j][i] = sub == 0 ? __float_as_uint(d[i]) : max(P[j][i], __float_as_uint(d[i]));
+                        }
+                    }
+                    // accumulator fragment (rows g, g + 8 of the 16-row tile; columns 2 t, 2 t + 1 of the 8-column tile) ->
+                    // the thread's outputs r = 2 mt + (i >> 1), c = 2 j + (i & 1)
+#pragma unroll
+                    for (int j = 0; j < 2; ++j)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) emp[2 * mt + (i >> 1)][2 * j + (i & 1)] = P[j][i];
+                }
+            }
             // ---- e_max = max(Exp(c), product exponents) and the accumulator term:
             // acc = 1.5 * 2^52 * q + floor(c' / q) * q, c' = c with the lowest mantissa bit of its double set (never on
             // the grid: a negative c floors to the one's complement), then + 1 if c < 0.
@@ -578,7 +640,10 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                     int keyc = subnormal_c ? (1023 - 126) << 20 : hi & 0x7FF00000;
                     if (ST) keyc -= (sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]) << 20;
                     const uint32_t e2 = emp[r][c];
-                    const int keyp = int(__vmaxu2(e2, __byte_perm(e2, 0u, 0x1032)) & 0xFFFFu) * (1 << 20) - (1 << 20);
+                    // BASE > 0: the exponent field of P over BASE, in place; P = 0 gives a key two binades below the
+                    // smallest real one, which is wrong only for an even smaller c: the epilogue repairs that case
+                    const int keyp = BASE ? int((e2 >> (3 + LB)) & 0xFFF00000u) + KP2
+                                          : int(__vmaxu2(e2, __byte_perm(e2, 0u, 0x1032)) & 0xFFFFu) * (1 << 20) - (1 << 20);
                     const int e20 = ST ? __vimax3_s32(keyp, keyc, 0) : max(keyp, keyc);
                     // the +1 of a negative c sits in the constant's low word: one unit of the grid either way
                     const double magic = __hiloint2double(e20 + km, int(uint32_t(hi) >> 31));
@@ -605,7 +670,8 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                     int rel = int(max(field, 1u)) + (CB - (ACC16 ? 15 : 127));
                     if (ST) rel -= sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0];
                     if ((cw[r][c] & (ACC16 ? 0x7FFFu : 0x7FFFFFFFu)) == 0u) rel = 0;       // c = 0 has no exponent
-                    const int emax = __vimax3_s32(int(emp[r][c] & 0xFFFFu), int(emp[r][c] >> 16), rel);     // e_max + CB
+                    const int emax = BASE ? max(int(emp[r][c] >> (23 + LB)) + (CB + 2 - (127 + 1) / (BASE ? BASE : 1)), rel)
+                                          : __vimax3_s32(int(emp[r][c] & 0xFFFFu), int(emp[r][c] >> 16), rel);     // e_max + CB
                     // the +1 of a negative c sits in the constant's low word: one unit of the grid either way
                     const double magic = __hiloint2double(emax * (1 << 20) + MAGIC_K, int(cw[r][c] >> (ACC16 ? 15 : 31)));
                     double cd = ACC16 ? double(__half2float(__ushort_as_half((unsigned short)cw[r][c]))) : double(__uint_as_float(cw[r][c]));
@@ -656,15 +722,18 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                     }
                 }
             };
-            if (NBLK > 1 && blk + 1 < NBLK) multiply_adds(std::true_type{}); else multiply_adds(std::false_type{});
+            if (BASE == 0 && NBLK > 1 && blk + 1 < NBLK) multiply_adds(std::true_type{}); else multiply_adds(std::false_type{});
             // ---- sign corrections, rho.  An overflow (|v| >= 2^128, or an FP16 result that rounds to infinity) is rare
             // and sticky: the loop only tracks the largest result word, the flags are set in a second pass ----
             const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
             constexpr uint32_t ABS = ACC16 ? 0x7FFFu : 0x7FFFFFFFu;
             constexpr uint32_t SUSPECT = ACC16 ? 0x7C00u : 0x7F7FFFFFu;   // FP16: infinity; FP32: cvt.rz saturates at the largest finite word
             uint32_t wmax = 0u;
+            bool no_product = false;                    // BASE > 0: some output of the micro-tile has no nonzero product
             auto block_value = [&](int r, int c, uint32_t sa, uint32_t nza) -> double {
-                const int nneg = __popc((sa ^ sb_blk.sgn[pcol + c]) & nza & sb_blk.nz[pcol + c]);
+                const uint32_t live = nza & sb_blk.nz[pcol + c];
+                if (BASE) no_product = no_product || live == 0u;
+                const int nneg = __popc((sa ^ sb_blk.sgn[pcol + c]) & live);
                 const long long bits = __double_as_longlong(acc[r][c]) + (long long)nneg;
                 const int hi = int(bits >> 32);
                 const double magic = __hiloint2double((hi & 0x7FF00000) | 0x00080000, 0);
@@ -674,6 +743,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
             };
             if (DS) {
                 bool odd = false;                       // some result is not a normal FP32 number
+                double nv[DS ? TM : 1][DS ? TN : 1];
 #pragma unroll
                 for (int r = 0; r < TM; ++r) {
                     const uint32_t sa = sa_blk.sgn[prow + r], nza = sa_blk.nz[prow + r] & kmask;
@@ -682,9 +752,21 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                         const double v = block_value(r, c, sa, nza);
                         odd = odd || !(fabs(v) >= 1.1754943508222875e-38) || !(fabs(v) < 3.402823669209385e38);
                         // RZ-FP32 of a number in the normal range: the low 29 bits of the double's significand go
-                        cs[DS ? r : 0][DS ? c : 0] = __hiloint2double(__double2hiint(v), (__double2loint(v) & int(0xE0000000u)) | 1);
+                        nv[DS ? r : 0][DS ? c : 0] = __hiloint2double(__double2hiint(v), (__double2loint(v) & int(0xE0000000u)) | 1);
                     }
                 }
+                if (BASE && no_product) {               // rare: no nonzero product: the block returns its accumulator
+                    odd = true;
+#pragma unroll
+                    for (int r = 0; r < TM; ++r)
+#pragma unroll
+                        for (int c = 0; c < TN; ++c)
+                            if ((sa_blk.nz[prow + r] & kmask & sb_blk.nz[pcol + c]) == 0u) nv[DS ? r : 0][DS ? c : 0] = cs[DS ? r : 0][DS ? c : 0];
+                }
+#pragma unroll
+                for (int r = 0; r < TM; ++r)
+#pragma unroll
+                    for (int c = 0; c < TN; ++c) cs[DS ? r : 0][DS ? c : 0] = nv[DS ? r : 0][DS ? c : 0];
                 if (odd || sub_mask) {                  // rare: zero, FP32 subnormal or overflow somewhere in the micro-tile
                     sub_mask = 0u;
 #pragma unroll
@@ -705,6 +787,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                         }
                 }
             } else {
+            uint32_t nw[TM][TN];
 #pragma unroll
             for (int r = 0; r < TM; ++r) {
                 const uint32_t sa = sa_blk.sgn[prow + r], nza = sa_blk.nz[prow + r] & kmask;
@@ -713,9 +796,20 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                     const double v = block_value(r, c, sa, nza);
                     const uint32_t w = ACC16 ? uint32_t(__half_as_ushort(__double2half(v))) : __float_as_uint(__double2float_rz(v));
                     wmax = max(wmax, w & ABS);
-                    cw[r][c] = w;
+                    nw[r][c] = w;
                 }
             }
+            if (BASE && no_product) {                   // rare: no nonzero product: the block returns its accumulator
+#pragma unroll
+                for (int r = 0; r < TM; ++r)
+#pragma unroll
+                    for (int c = 0; c < TN; ++c)
+                        if ((sa_blk.nz[prow + r] & kmask & sb_blk.nz[pcol + c]) == 0u) nw[r][c] = cw[r][c];
+            }
+#pragma unroll
+            for (int r = 0; r < TM; ++r)
+#pragma unroll
+                for (int c = 0; c < TN; ++c) cw[r][c] = nw[r][c];
             }
             if (!DS && wmax >= SUSPECT) {
 #pragma unroll
@@ -788,11 +882,10 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
 #undef MMASIM_SP_GET
 }
 
-template <int EK, int L, int RHO, bool PROMOTE, bool ST = false>
-cudaError_t launch_one64(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
-    constexpr int BASE = 0;
+template <int EK, int L, int RHO, bool PROMOTE, bool ST, int BASE>
+cudaError_t launch_one64b(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
     const size_t sh = sizeof(SmemMM);
-    cudaError_t err = cudaFuncSetAttribute(tfdpa64_kernel<EK, L, RHO, PROMOTE, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
+    cudaError_t err = cudaFuncSetAttribute(tfdpa64_kernel<EK, L, RHO, PROMOTE, ST, BASE>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
     if (err != cudaSuccess) return err;
     const size_t dsh_a = 256 * sizeof(LutEntry64) + sizeof(Blk64<BM>), dsh_b = 256 * sizeof(LutEntry64) + sizeof(Blk64<BN>);
     if ((err = cudaFuncSetAttribute(decode64_kernel<EK, BM, true, BASE>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(dsh_a))) != cudaSuccess) return err;
@@ -811,10 +904,21 @@ cudaError_t launch_one64(const DevModel& m, const GemmArgs& g, cudaStream_t stre
     decode64_kernel<EK, BN, false, BASE><<<dim3((unsigned)nch, (unsigned)tiles_n), 256, dsh_b, stream>>>(
         m, static_cast<const unsigned char*>(g.B), g.N, g.ldb, wb);
     dim3 grid((unsigned)tiles_n, (unsigned)tiles_m, 1);
-    tfdpa64_kernel<EK, L, RHO, PROMOTE, ST><<<grid, NT, sh, stream>>>(m, g, wa, wb);
+    tfdpa64_kernel<EK, L, RHO, PROMOTE, ST, BASE><<<grid, NT, sh, stream>>>(m, g, wa, wb);
     err = cudaGetLastError();
     const cudaError_t err2 = cudaFreeAsync(ws, stream);
     return err != cudaSuccess ? err : err2;
+}
+
+// The base of the tensor-core exponent maximum by element kinds: FP16 (blocks of 8 or 16) 4; 8-bit kinds 4 with an E5M2
+// operand, else 8; BF16, TF32 and blocks of 4: the add-max pass.
+template <int EK, int L, int RHO, bool PROMOTE, bool ST = false>
+cudaError_t launch_one64(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
+    if constexpr (EK == fast::EK_F16 && L >= 8) return launch_one64b<EK, L, RHO, PROMOTE, ST, 4>(m, g, stream);
+    else if constexpr (EK == fast::EK_LUT8 && L >= 8) {
+        if (m.fmt_a == EF_E5M2 || m.fmt_b == EF_E5M2) return launch_one64b<EK, L, RHO, PROMOTE, ST, 4>(m, g, stream);
+        return launch_one64b<EK, L, RHO, PROMOTE, ST, 8>(m, g, stream);
+    } else return launch_one64b<EK, L, RHO, PROMOTE, ST, 0>(m, g, stream);
 }
 
 // With or without FP32 promotion (FP32 accumulators only).
