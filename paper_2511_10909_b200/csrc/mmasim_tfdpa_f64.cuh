@@ -628,20 +628,21 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
             // the grid: a negative c floors to the one's complement), then + 1 if c < 0.
             // ST: the products are compared against Exp(c) minus the block's scale exponents, c is scaled likewise.
             double acc[TM][TN];
-            if (DS) {
-                // keys are exponent fields of doubles in place: (Exp + 1023) << 20.  Products: the larger 16-bit lane of emp
-                // (Exp + CB, CB = 1024); c: the state's own field (0 for c = 0: below every real key), minus the scale
-                // exponents for ST; an FP32 subnormal c counts with Exp = -126 (rare: patched below).
-                constexpr int KM = ((52 - 0) << 20) | 0x00080000;    // + (e_max - F) gives the high word of 1.5 * 2^52 * q
-                const int km = KM - (m.F << 20);
-                auto start = [&](int r, int c, bool subnormal_c) {
+            // keys (FP32 accumulators) are exponent fields of doubles in place: (Exp + 1023) << 20.  Products: the larger
+            // 16-bit lane of emp (Exp + CB, CB = 1024) or, BASE > 0, the exponent field of P over BASE; c: the state's own
+            // field (0 for c = 0: below every real key), minus the scale exponents for ST; an FP32 subnormal c counts with
+            // Exp = -126 (rare: patched after the pass over the outputs).
+            constexpr int KM = (52 << 20) | 0x00080000;              // + (e_max - F) gives the high word of 1.5 * 2^52 * q
+            const int km = KM - (m.F << 20);
+            auto start = [&](int r, int c, bool subnormal_c) {
+                if (DS) {
                     const double st = cs[DS ? r : 0][DS ? c : 0];
                     const int hi = __double2hiint(st);
                     int keyc = subnormal_c ? (1023 - 126) << 20 : hi & 0x7FF00000;
                     if (ST) keyc -= (sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]) << 20;
                     const uint32_t e2 = emp[r][c];
-                    // BASE > 0: the exponent field of P over BASE, in place; P = 0 gives a key two binades below the
-                    // smallest real one, which is wrong only for an even smaller c: the epilogue repairs that case
+                    // BASE > 0: P = 0 gives a key two binades below the smallest real one, which is wrong only for an even
+                    // smaller c: the epilogue repairs that case
                     const int keyp = BASE ? int((e2 >> (3 + LB)) & 0xFFF00000u) + KP2
                                           : int(__vmaxu2(e2, __byte_perm(e2, 0u, 0x1032)) & 0xFFFFu) * (1 << 20) - (1 << 20);
                     const int e20 = ST ? __vimax3_s32(keyp, keyc, 0) : max(keyp, keyc);
@@ -649,88 +650,55 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                     const double magic = __hiloint2double(e20 + km, int(uint32_t(hi) >> 31));
                     const double x = ST ? __dmul_rn(st, pow2d(-(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]))) : st;
                     acc[r][c] = __dadd_rd(x, magic);
-                };
-#pragma unroll
-                for (int r = 0; r < TM; ++r)
-#pragma unroll
-                    for (int c = 0; c < TN; ++c) start(r, c, false);
-                if (sub_mask) {                         // rare: redo the outputs whose accumulator is an FP32 subnormal
-#pragma unroll
-                    for (int r = 0; r < TM; ++r)
-#pragma unroll
-                        for (int c = 0; c < TN; ++c)
-                            if ((sub_mask >> (r * TN + c)) & 1u) start(r, c, true);
-                }
-            } else
-#pragma unroll
-            for (int r = 0; r < TM; ++r)
-#pragma unroll
-                for (int c = 0; c < TN; ++c) {
+                } else {
                     const uint32_t field = ACC16 ? (cw[r][c] >> 10) & 0x1Fu : (cw[r][c] >> 23) & 0xFFu;
                     int rel = int(max(field, 1u)) + (CB - (ACC16 ? 15 : 127));
                     if (ST) rel -= sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0];
                     if ((cw[r][c] & (ACC16 ? 0x7FFFu : 0x7FFFFFFFu)) == 0u) rel = 0;       // c = 0 has no exponent
                     const int emax = BASE ? max(int(emp[r][c] >> (23 + LB)) + (CB + 2 - (127 + 1) / (BASE ? BASE : 1)), rel)
                                           : __vimax3_s32(int(emp[r][c] & 0xFFFFu), int(emp[r][c] >> 16), rel);     // e_max + CB
-                    // the +1 of a negative c sits in the constant's low word: one unit of the grid either way
                     const double magic = __hiloint2double(emax * (1 << 20) + MAGIC_K, int(cw[r][c] >> (ACC16 ? 15 : 31)));
                     double cd = ACC16 ? double(__half2float(__ushort_as_half((unsigned short)cw[r][c]))) : double(__uint_as_float(cw[r][c]));
                     if (ST) cd = __dmul_rn(cd, pow2d(-(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0])));
                     cd = __hiloint2double(__double2hiint(cd), __double2loint(cd) | 1);
                     acc[r][c] = __dadd_rd(cd, magic);
                 }
-            // ---- one fused multiply-add per term, rounding toward minus infinity onto the grid of q; beside it, while
-            // the chunk has another block, the product exponents of that block ----
-            auto multiply_adds = [&](auto with_exponents) {
-                constexpr bool FUSE = decltype(with_exponents)::value;
-                const uint32_t* ea_p = &sa_blk.exp2[FUSE ? (kb + L) / 2 : 0][prow];
-                const uint32_t* eb_p = &sb_blk.exp2[FUSE ? (kb + L) / 2 : 0][pcol];
-                if (FUSE) {
+            };
+            auto restart_subnormals = [&](int r0) {     // rare: redo the outputs whose accumulator is an FP32 subnormal
+                if (DS && sub_mask) {
 #pragma unroll
-                    for (int r = 0; r < TM; ++r)
+                    for (int r = r0; r < r0 + 2; ++r)
 #pragma unroll
-                        for (int c = 0; c < TN; ++c) emp[r][c] = 0u;
-                }
-                // four terms per matrix instruction (mma.sync m8n8k4, FP64, rounding toward minus infinity: a chain of four
-                // fused multiply-adds per output, each rounded onto the grid of q); operand fragments: lane (g, t) holds
-                // A[8 r + g][k + t] and B[8 j + g][k + t]
-#pragma unroll
-                for (int ks = 0; ks < L; ks += 4) {
-                    double af[TM], bf[TN / 2];
-#pragma unroll
-                    for (int r = 0; r < TM; ++r) af[r] = sa_blk.d[wr * 32 + 8 * r + gq][kb + ks + tq];
-#pragma unroll
-                    for (int j = 0; j < TN / 2; ++j) bf[j] = sb_blk.d[wc * 16 + 8 * j + gq][kb + ks + tq];
-#pragma unroll
-                    for (int r = 0; r < TM; ++r)
-#pragma unroll
-                        for (int j = 0; j < TN / 2; ++j)
-                            asm volatile("mma.sync.aligned.m8n8k4.row.col.rm.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
-                                         : "+d"(acc[r][2 * j]), "+d"(acc[r][2 * j + 1]) : "d"(af[r]), "d"(bf[j]));
-                    if (FUSE) {
-#pragma unroll
-                        for (int kp = ks / 2; kp < ks / 2 + 2; ++kp) {
-                            const uint4 ea0 = *reinterpret_cast<const uint4*>(ea_p + kp * BM);
-                            const uint4 eb0 = *reinterpret_cast<const uint4*>(eb_p + kp * BN);
-                            const uint32_t ea[TM] = {ea0.x, ea0.y, ea0.z, ea0.w};
-                            const uint32_t ebv[TN] = {eb0.x, eb0.y, eb0.z, eb0.w};
-#pragma unroll
-                            for (int r = 0; r < TM; ++r)
-#pragma unroll
-                                for (int c = 0; c < TN; ++c) emp[r][c] = __viaddmax_s16x2(ea[r], ebv[c], emp[r][c]);
-                        }
-                    }
+                        for (int c = 0; c < TN; ++c)
+                            if ((sub_mask >> (r * TN + c)) & 1u) start(r, c, true);
                 }
             };
-            if (BASE == 0 && NBLK > 1 && blk + 1 < NBLK) multiply_adds(std::true_type{}); else multiply_adds(std::false_type{});
+            // four terms per matrix instruction (mma.sync m8n8k4, FP64, rounding toward minus infinity: a chain of four fused
+            // multiply-adds per output, each rounded onto the grid of q) for the rows 2 half, 2 half + 1 of the micro-tile;
+            // operand fragments: lane (g, t) holds A[8 r + g][k + t] and B[8 j + g][k + t]
+            auto mma_half = [&](int half, int ks) {
+                double af[2], bf[TN / 2];
+#pragma unroll
+                for (int r = 0; r < 2; ++r) af[r] = sa_blk.d[wr * 32 + 8 * (2 * half + r) + gq][kb + ks + tq];
+#pragma unroll
+                for (int j = 0; j < TN / 2; ++j) bf[j] = sb_blk.d[wc * 16 + 8 * j + gq][kb + ks + tq];
+#pragma unroll
+                for (int r = 0; r < 2; ++r)
+#pragma unroll
+                    for (int j = 0; j < TN / 2; ++j)
+                        asm volatile("mma.sync.aligned.m8n8k4.row.col.rm.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                                     : "+d"(acc[2 * half + r][2 * j]), "+d"(acc[2 * half + r][2 * j + 1]) : "d"(af[r]), "d"(bf[j]));
+            };
             // ---- sign corrections, rho.  An overflow (|v| >= 2^128, or an FP16 result that rounds to infinity) is rare
-            // and sticky: the loop only tracks the largest result word, the flags are set in a second pass ----
+            // and sticky: the loop only tracks it, the flags are set in a second pass ----
             const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
             constexpr uint32_t ABS = ACC16 ? 0x7FFFu : 0x7FFFFFFFu;
             constexpr uint32_t SUSPECT = ACC16 ? 0x7C00u : 0x7F7FFFFFu;   // FP16: infinity; FP32: cvt.rz saturates at the largest finite word
             uint32_t wmax = 0u;
             bool no_product = false;                    // BASE > 0: some output of the micro-tile has no nonzero product
-            auto block_value = [&](int r, int c, uint32_t sa, uint32_t nza) -> double {
+            bool odd = false;                           // FP32 state: some result is not a normal FP32 number
+            auto block_value = [&](int r, int c) -> double {
+                const uint32_t sa = sa_blk.sgn[prow + r], nza = sa_blk.nz[prow + r] & kmask;
                 const uint32_t live = nza & sb_blk.nz[pcol + c];
                 if (BASE) no_product = no_product || live == 0u;
                 const int nneg = __popc((sa ^ sb_blk.sgn[pcol + c]) & live);
@@ -741,20 +709,69 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                 if (ST) v = __dmul_rn(v, pow2d(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]));
                 return v;
             };
-            if (DS) {
-                bool odd = false;                       // some result is not a normal FP32 number
-                double nv[DS ? TM : 1][DS ? TN : 1];
+            double nv[DS ? TM : 1][DS ? TN : 1];
+            uint32_t nw[DS ? 1 : TM][DS ? 1 : TN];
+            auto finish = [&](int r, int c) {
+                const double v = block_value(r, c);
+                if (DS) {
+                    odd = odd || !(fabs(v) >= 1.1754943508222875e-38) || !(fabs(v) < 3.402823669209385e38);
+                    // RZ-FP32 of a number in the normal range: the low 29 bits of the double's significand go
+                    nv[DS ? r : 0][DS ? c : 0] = __hiloint2double(__double2hiint(v), (__double2loint(v) & int(0xE0000000u)) | 1);
+                } else {
+                    const uint32_t w = ACC16 ? uint32_t(__half_as_ushort(__double2half(v))) : __float_as_uint(__double2float_rz(v));
+                    wmax = max(wmax, w & ABS);
+                    nw[DS ? 0 : r][DS ? 0 : c] = w;
+                }
+            };
+
+            // ---- the block in two halves of the micro-tile (rows 0, 1 and rows 2, 3), so that the multiply-adds of one half
+            // (FP64 pipe) are issued between the integer work of the other: start(A); [multiply-adds(A) | start(B)];
+            // [multiply-adds(B) | finish(A), and the product exponents of the next block]; finish(B) ----
+            constexpr int NKS = L / 4, PER = 8 / (NKS < 8 ? NKS : 8);
+            const bool fuse = BASE == 0 && NBLK > 1 && blk + 1 < NBLK;
 #pragma unroll
-                for (int r = 0; r < TM; ++r) {
-                    const uint32_t sa = sa_blk.sgn[prow + r], nza = sa_blk.nz[prow + r] & kmask;
+            for (int o = 0; o < 8; ++o) start(o / TN, o % TN, false);
+            restart_subnormals(0);
 #pragma unroll
-                    for (int c = 0; c < TN; ++c) {
-                        const double v = block_value(r, c, sa, nza);
-                        odd = odd || !(fabs(v) >= 1.1754943508222875e-38) || !(fabs(v) < 3.402823669209385e38);
-                        // RZ-FP32 of a number in the normal range: the low 29 bits of the double's significand go
-                        nv[DS ? r : 0][DS ? c : 0] = __hiloint2double(__double2hiint(v), (__double2loint(v) & int(0xE0000000u)) | 1);
+            for (int ksi = 0; ksi < NKS; ++ksi) {
+                mma_half(0, 4 * ksi);
+#pragma unroll
+                for (int q = 0; q < PER; ++q)
+                    if (ksi * PER + q < 8) start(2 + (ksi * PER + q) / TN, (ksi * PER + q) % TN, false);
+            }
+            restart_subnormals(2);
+#pragma unroll
+            for (int ksi = 0; ksi < NKS; ++ksi) {
+                mma_half(1, 4 * ksi);
+#pragma unroll
+                for (int q = 0; q < PER; ++q)
+                    if (ksi * PER + q < 8) finish((ksi * PER + q) / TN, (ksi * PER + q) % TN);
+                if (fuse) {                             // the product exponents of the next block (add-max kinds)
+                    const uint32_t* ea_p = &sa_blk.exp2[(kb + L) / 2 < KC / 2 ? (kb + L) / 2 : 0][prow];
+                    const uint32_t* eb_p = &sb_blk.exp2[(kb + L) / 2 < KC / 2 ? (kb + L) / 2 : 0][pcol];
+                    if (ksi == 0) {
+#pragma unroll
+                        for (int r = 0; r < TM; ++r)
+#pragma unroll
+                            for (int c = 0; c < TN; ++c) emp[r][c] = 0u;
+                    }
+#pragma unroll
+                    for (int kp = 2 * ksi; kp < 2 * ksi + 2; ++kp) {
+                        const uint4 ea0 = *reinterpret_cast<const uint4*>(ea_p + kp * BM);
+                        const uint4 eb0 = *reinterpret_cast<const uint4*>(eb_p + kp * BN);
+                        const uint32_t ea[TM] = {ea0.x, ea0.y, ea0.z, ea0.w};
+                        const uint32_t ebv[TN] = {eb0.x, eb0.y, eb0.z, eb0.w};
+#pragma unroll
+                        for (int r = 0; r < TM; ++r)
+#pragma unroll
+                            for (int c = 0; c < TN; ++c) emp[r][c] = __viaddmax_s16x2(ea[r], ebv[c], emp[r][c]);
                     }
                 }
+            }
+#pragma unroll
+            for (int o = 8; o < 16; ++o) finish(o / TN, o % TN);
+
+            if (DS) {
                 if (BASE && no_product) {               // rare: no nonzero product: the block returns its accumulator
                     odd = true;
 #pragma unroll
@@ -787,44 +804,31 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                         }
                 }
             } else {
-            uint32_t nw[TM][TN];
+                if (BASE && no_product) {               // rare: no nonzero product: the block returns its accumulator
 #pragma unroll
-            for (int r = 0; r < TM; ++r) {
-                const uint32_t sa = sa_blk.sgn[prow + r], nza = sa_blk.nz[prow + r] & kmask;
+                    for (int r = 0; r < TM; ++r)
 #pragma unroll
-                for (int c = 0; c < TN; ++c) {
-                    const double v = block_value(r, c, sa, nza);
-                    const uint32_t w = ACC16 ? uint32_t(__half_as_ushort(__double2half(v))) : __float_as_uint(__double2float_rz(v));
-                    wmax = max(wmax, w & ABS);
-                    nw[r][c] = w;
+                        for (int c = 0; c < TN; ++c)
+                            if ((sa_blk.nz[prow + r] & kmask & sb_blk.nz[pcol + c]) == 0u) nw[DS ? 0 : r][DS ? 0 : c] = cw[r][c];
                 }
-            }
-            if (BASE && no_product) {                   // rare: no nonzero product: the block returns its accumulator
+                if (wmax >= SUSPECT) {                  // rare: overflow of the conversion: sticky infinities
+#pragma unroll
+                    for (int r = 0; r < TM; ++r)
+#pragma unroll
+                        for (int c = 0; c < TN; ++c) {
+                            if ((nw[DS ? 0 : r][DS ? 0 : c] & ABS) != SUSPECT) continue;
+                            if (BASE && (sa_blk.nz[prow + r] & kmask & sb_blk.nz[pcol + c]) == 0u) continue;   // the kept accumulator
+                            const double v = block_value(r, c);
+                            if (!ACC16 && fabs(v) < 3.402823669209385e38) continue;       // below 2^128: the largest finite number, legitimately
+                            const uint32_t bit = 1u << (r * TN + c);
+                            if (!((sp_nan | sp_pinf | sp_ninf) & bit)) { if (v < 0.0) sp_ninf |= bit; else sp_pinf |= bit; }
+                            nw[DS ? 0 : r][DS ? 0 : c] = 0u;                              // +-infinity from now on
+                        }
+                }
 #pragma unroll
                 for (int r = 0; r < TM; ++r)
 #pragma unroll
-                    for (int c = 0; c < TN; ++c)
-                        if ((sa_blk.nz[prow + r] & kmask & sb_blk.nz[pcol + c]) == 0u) nw[r][c] = cw[r][c];
-            }
-#pragma unroll
-            for (int r = 0; r < TM; ++r)
-#pragma unroll
-                for (int c = 0; c < TN; ++c) cw[r][c] = nw[r][c];
-            }
-            if (!DS && wmax >= SUSPECT) {
-#pragma unroll
-                for (int r = 0; r < TM; ++r) {
-                    const uint32_t sa = sa_blk.sgn[prow + r], nza = sa_blk.nz[prow + r] & kmask;
-#pragma unroll
-                    for (int c = 0; c < TN; ++c) {
-                        if ((cw[r][c] & ABS) != SUSPECT) continue;
-                        const double v = block_value(r, c, sa, nza);
-                        if (!ACC16 && fabs(v) < 3.402823669209385e38) continue;       // below 2^128: the largest finite number, legitimately
-                        const uint32_t bit = 1u << (r * TN + c);
-                        if (!((sp_nan | sp_pinf | sp_ninf) & bit)) { if (v < 0.0) sp_ninf |= bit; else sp_pinf |= bit; }
-                        cw[r][c] = 0u;                                                // +-infinity from now on
-                    }
-                }
+                    for (int c = 0; c < TN; ++c) cw[r][c] = nw[DS ? 0 : r][DS ? 0 : c];
             }
         }
         __syncthreads();                                // everybody has finished with this buffer
