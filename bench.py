@@ -72,6 +72,9 @@ def compute_dtype(kernel: str, model) -> str:
 # 0.4 % of what the memory could move in the kernel's time.
 NCU_DRAM_BYTES = {"cfg3": 101593856 + 34110464, "cfg3_2k": 25592832 + 38656}
 
+# kernels one library call launches: the tuned fused-summation kernels decode A and B into scratch blocks first
+KERNELS_PER_CALL = {"tfdpa_lut8": 3, "tfdpa_f16": 3, "tfdpa_bf16": 3, "tfdpa_tf32": 3}
+
 SMS = 148
 # The pipe that bounds each kernel: (name, instruction kinds of the issue-rate micro-benchmark that witness its rate,
 # nominal results per SM and clock, pipe instructions per emulated MAC).
@@ -544,7 +547,7 @@ def run_ours(args):
         "dtype": compute_dtype(kernel_name, model), "data": "synthetic",
         "config": {"workload": f"{name}: {desc}", "model": "-".join(key), "M": M, "N": N, "K": K,
                    "l2": "flushed between timed steps (256 MiB write)", "parallelism": f"replicas x{world} (independent batches, no exchange)"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * KERNELS_PER_CALL.get(kernel_name, 1),
         "roofline": roofline,
         "cpu_baseline": {"value": cpu_value, "unit": UNIT, "kind": "oracle", **cpu_info},
         "per_model": per_model, "per_model_size": args.per_model_size if per_model else None, "dot_batch": dot_line,
@@ -552,6 +555,44 @@ def run_ours(args):
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def native_difference(torch, key, model, dA, dB, dC, D):
+    """Context column of config 5: on how many outputs does the B200's own tensor-core GEMM (cuBLAS through torch.mm /
+    torch._scaled_mm, FP32 or FP64 result, C added afterwards in the accumulator type) differ from the model's words?
+    The library GEMM is only the other side of this comparison; its summation order is its own business."""
+    in_fmt, acc = key[1], key[2]
+    try:
+        if in_fmt in ("fp16", "bf16", "bf16_1k") and acc == "fp32":
+            dt = torch.float16 if in_fmt == "fp16" else torch.bfloat16
+            nat = torch.mm(dA.view(dt), dB.view(dt).t(), out_dtype=torch.float32) + dC.view(torch.float32)
+            op = "torch.mm(out_dtype=float32) + C"
+        elif in_fmt == "tf32":
+            old = torch.backends.cuda.matmul.allow_tf32
+            torch.backends.cuda.matmul.allow_tf32 = True
+            nat = torch.mm(dA.view(torch.float32), dB.view(torch.float32).t()) + dC.view(torch.float32)
+            torch.backends.cuda.matmul.allow_tf32 = old
+            op = "torch.mm (TF32 allowed) + C"
+        elif in_fmt == "fp32":
+            old = torch.backends.cuda.matmul.allow_tf32
+            torch.backends.cuda.matmul.allow_tf32 = False
+            nat = torch.mm(dA.view(torch.float32), dB.view(torch.float32).t()) + dC.view(torch.float32)
+            torch.backends.cuda.matmul.allow_tf32 = old
+            op = "torch.mm (FP32) + C"
+        elif in_fmt == "fp64":
+            nat = torch.mm(dA.view(torch.float64), dB.view(torch.float64).t()) + dC.view(torch.float64)
+            op = "torch.mm (FP64) + C"
+        elif in_fmt in ("e4m3", "e5m2") and acc == "fp32":
+            dt = torch.float8_e4m3fn if in_fmt == "e4m3" else torch.float8_e5m2
+            one = torch.ones((), dtype=torch.float32, device=dA.device)
+            nat = torch._scaled_mm(dA.view(dt), dB.view(dt).t(), scale_a=one, scale_b=one, out_dtype=torch.float32) + dC.view(torch.float32)
+            op = "torch._scaled_mm(out_dtype=float32) + C"
+        else:
+            return {"native_op": None, "native_differs": None}
+    except Exception as exc:                                   # an operand combination this torch / cuBLAS does not offer
+        return {"native_op": f"unavailable: {type(exc).__name__}", "native_differs": None}
+    words = nat.view(torch.int32 if nat.dtype == torch.float32 else torch.int64)
+    return {"native_op": op, "native_differs": int((words != D.view(words.dtype)).sum().item()), "outputs": int(D.numel())}
 
 
 def run_sweep(args):
@@ -601,6 +642,8 @@ def run_sweep(args):
             ms = e0.elapsed_time(e1) / args.steps
             row = {"model": "-".join(key), "family": model.family, "kernel": mmasim.last_kernel(), "size": size,
                    "ms": ms, "macs_per_s": float(M) * N * K / (ms * 1e-3)}
+            if args.native:
+                row.update(native_difference(torch, key, model, dA, dB, dC, D))
             if args.check:
                 pairs = wl.sample_pairs(M, N, args.check, seed=55)
                 A, B = inp["A"], inp["B"]
@@ -639,6 +682,9 @@ def main():
     ap.add_argument("--size", type=int, default=4096)
     ap.add_argument("--check", type=int, default=0, help="with --sweep: compare this many seeded sampled outputs per model with the oracle")
     ap.add_argument("--out-dir", default="sweep_out", help="with --sweep: folder of the per-model JSON lines")
+    ap.add_argument("--native", action="store_true",
+                    help="with --sweep: also count the outputs on which the B200's native tensor-core GEMM (torch.mm / torch._scaled_mm) "
+                         "differs from each model (context only)")
     ap.add_argument("--models", default="", help="with --sweep: comma-separated arch-infmt-acc names (default: all)")
     args = ap.parse_args()
     if args.sweep:
