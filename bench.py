@@ -54,6 +54,16 @@ WORKLOADS = {
                       "BF16 2048^3 N(0,1) inputs (reduced case for profiler captures); CDNA3 BF16 model (TR-FDPA, L=8, F=24, F2=31)"),
     "cdna1_fp16_2k": (("cdna1", "fp16", "fp32"), (2048, 2048, 2048),
                       "FP16 2048^3 N(0,1) inputs (reduced case for profiler captures); CDNA1 FP16 model (E-FDPA, L=4)"),
+    "cdna3_tf32_2k": (("cdna3", "tf32", "fp32"), (2048, 2048, 2048),
+                      "TF32 2048^3 N(0,1) inputs (reduced case for profiler captures); CDNA3 TF32 model (TR-FDPA, L=4)"),
+    "cdna3_e4m3_2k": (("cdna3", "e4m3", "fp32"), (2048, 2048, 2048),
+                      "FP8 E4M3 2048^3 N(0,1) inputs (reduced case for profiler captures); CDNA3 FP8 model (GTR-FDPA, L=16)"),
+    "volta_fp16_2k": (("volta", "fp16", "fp32"), (2048, 2048, 2048),
+                      "FP16 2048^3 N(0,1) inputs (reduced case for profiler captures); Volta FP16->FP32 model (L=4, F=23)"),
+    "blackwell_mxf4_2k": (("blackwell", "mxf4", "fp32"), (2048, 2048, 2048),
+                          "MXFP4 2048^3 N(0,1) inputs with E8M0 block scales (reduced case for profiler captures); Blackwell MXFP4 model (GST-FDPA, L=64, G=16, F=35)"),
+    "cdna1_fp32_2k": (("cdna1", "fp32", "fp32"), (2048, 2048, 2048),
+                      "FP32 2048^3 N(0,1) inputs (reduced case for profiler captures); CDNA1 FP32 model (FMA chain)"),
     "blackwell_e4m3": (("blackwell", "e4m3", "fp32"), (4096, 4096, 4096),
                        "FP8 E4M3 4096^3 N(0,1) inputs; Blackwell FP8->FP32 model (L=32, F=25, RZ-FP32)"),
 }
@@ -167,7 +177,7 @@ def make_inputs(name):
         A, B, C = wl.cfg4(key[1], K, n=M)
         return {"A": A, "B": B, "C": C, "dot": True}
     d = wl.normal_inputs(key[1], key[2], M, N, K, seed=5)
-    return {"A": d["A"], "B": d["B"], "C": d["C"]}
+    return {k: d[k] for k in ("A", "B", "C", "sfa", "sfb") if k in d}
 
 
 def max_over_ranks(value: float, dist=None, device=None) -> float:
@@ -281,6 +291,8 @@ def oracle_sample_rate(name, inp, seconds_target=15.0, processes=None):
     kw = {}
     if "k_chunk" in inp:
         kw.update(k_chunk=inp["k_chunk"], row_scale=inp["row_scale"].view(np.uint32), col_scale=inp["col_scale"].view(np.uint32))
+    if "sfa" in inp:
+        kw.update(SFA=inp["sfa"], SFB=inp["sfb"])
     probe = wl.sample_pairs(M, N, 64 * cores, seed=77)
     t0 = time.perf_counter()
     oracle.phi_gemm_sampled(m, inp["A"], inp["B"], inp["C"], probe, processes=cores, **kw)
@@ -308,6 +320,8 @@ def run_reference(args):
     kw = {}
     if "k_chunk" in inp:
         kw.update(k_chunk=inp["k_chunk"], row_scale=inp["row_scale"].view(np.uint32), col_scale=inp["col_scale"].view(np.uint32))
+    if "sfa" in inp:
+        kw.update(SFA=inp["sfa"], SFB=inp["sfb"])
     n = 512 * cores
     times = []
     for step in range(args.warmup + args.steps):
@@ -359,7 +373,9 @@ def run_ours(args):
     kw = {}
     if "k_chunk" in inp:
         kw = dict(k_chunk=inp["k_chunk"], row_scale=to_dev(inp["row_scale"]), col_scale=to_dev(inp["col_scale"]))
-    dD = torch.empty((M, N), dtype=torch.int32 if model.acc_bytes == 4 else torch.int16, device=dev)
+    if "sfa" in inp:
+        kw.update(sfa=to_dev(inp["sfa"]), sfb=to_dev(inp["sfb"]))
+    dD = torch.empty((M, N), dtype={2: torch.int16, 4: torch.int32, 8: torch.int64}[model.acc_bytes], device=dev)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # larger than the 126 MB L2
 
     is_dot = bool(inp.get("dot"))
@@ -415,6 +431,8 @@ def run_ours(args):
         hkw = {}
         if "k_chunk" in inp:
             hkw = dict(k_chunk=inp["k_chunk"], row_scale=pinned(inp["row_scale"]), col_scale=pinned(inp["col_scale"]))
+        if "sfa" in inp:
+            hkw.update(sfa=pinned(inp["sfa"]), sfb=pinned(inp["sfb"]))
         n_e2e = max(1, min(args.steps, 3))
         mmasim.gemm_host(model, hA, hB, hC, out=hD.numpy(), **hkw)
         torch.cuda.synchronize()

@@ -246,7 +246,9 @@ int mmasim_error_stats(int acc_fmt, int64_t n, const void* D, const double* ref,
  *   26 dfma.rm.x16    the same instructions with 16 / 32 independent accumulators per thread and loop-invariant
  *                     multiplicands (no operand-fetch conflicts): the second witness of the pipe rates.
  *   27 dmma.rm.k4, 28 dmma.rm.k16   the FP64 matrix instruction rounding toward -inf (mma.sync m8n8k4 / m16n8k16),
- *                     multiply-adds counted. */
+ *                     multiply-adds counted.
+ *   29 cvt.f32.f64 (FP32 -> FP64 -> FP32), 30 cvt.s32.f64 (s32 -> FP64 -> s32): conversion pairs, both counted;
+ *   31 dadd.rm.x16    add.rm.f64 with 16 independent accumulators. */
 int mmasim_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t* ops_per_round, void* stream);
 
 /* Name of the kernel variant the last mmasim_gemm* call on this thread dispatched to ("generic", ...). */

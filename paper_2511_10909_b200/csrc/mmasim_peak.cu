@@ -9,7 +9,7 @@ namespace {
 enum PeakKind : int {
     PK_IADD3 = 0, PK_LOP3, PK_SHF, PK_IMAD, PK_MACMIX, PK_VIADDMAX, PK_VIADDMAX16X2, PK_F2I, PK_FMUL, PK_POPC,
     PK_IMAD_PLUS_ALU, PK_FMUL_PLUS_ALU, PK_IMAD_WIDE, PK_MAC_D1, PK_MAC_D2, PK_DP4A, PK_DFMA, PK_DFMA_PLUS_ALU, PK_FFMA_RM, PK_FFMA2_RM,
-    PK_FFMA_RN_X16, PK_FFMA_RN_X32, PK_FFMA_RM_X16, PK_FFMA2_RM_X16, PK_DFMA_RN_X16, PK_DFMA_RN_X32, PK_DFMA_RM_X16, PK_DMMA_RM_K4, PK_DMMA_RM_K16, PK_COUNT
+    PK_FFMA_RN_X16, PK_FFMA_RN_X32, PK_FFMA_RM_X16, PK_FFMA2_RM_X16, PK_DFMA_RN_X16, PK_DFMA_RN_X32, PK_DFMA_RM_X16, PK_DMMA_RM_K4, PK_DMMA_RM_K16, PK_CVT_F32_F64, PK_CVT_S32_F64, PK_DADD_RM_X16, PK_COUNT
 };
 
 template <int KIND>
@@ -203,6 +203,38 @@ __global__ void __launch_bounds__(256) peak_kernel_dmma(int64_t iters, int* sink
     if (r == 0.12345) *sink = 1;
 }
 
+// Conversions and additions around the FP64 pipe, sixteen independent chains per thread: MODE 0: FP32 -> FP64 -> FP32
+// (cvt.f64.f32, cvt.rn.f32.f64), MODE 1: s32 -> FP64 -> s32 (cvt.rn.f64.s32, cvt.rzi.s32.f64), MODE 2: add.rm.f64.
+// One round = 16 chains x (2 conversions | 1 addition).
+template <int MODE>
+__global__ void __launch_bounds__(256) peak_kernel_cvt(int64_t iters, int* sink) {
+    float f[16]; int x[16]; double d[16];
+    const double inc = 1.0 + 1e-9 * double(threadIdx.x);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { f[i] = 1.0f + float(i + threadIdx.x); x[i] = i + int(threadIdx.x); d[i] = double(i); }
+    for (int64_t it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            if (MODE == 0) { double t; asm volatile("cvt.f64.f32 %0, %1;" : "=d"(t) : "f"(f[i])); asm volatile("cvt.rn.f32.f64 %0, %1;" : "=f"(f[i]) : "d"(t)); }
+            else if (MODE == 1) { double t; asm volatile("cvt.rn.f64.s32 %0, %1;" : "=d"(t) : "r"(x[i])); asm volatile("cvt.rzi.s32.f64 %0, %1;" : "=r"(x[i]) : "d"(t)); }
+            else asm volatile("add.rm.f64 %0, %0, %1;" : "+d"(d[i]) : "d"(inc));
+        }
+    }
+    double r = 0.0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) r += double(f[i]) + double(x[i]) + d[i];
+    if (r == 0.12345) *sink = 1;
+}
+
+template <int MODE>
+int launch_cvt(int64_t blocks, int64_t iters, void* sink, int32_t* ops_per_round, cudaStream_t stream) {
+    *ops_per_round = MODE == 2 ? 16 : 32;
+    peak_kernel_cvt<MODE><<<(unsigned)blocks, 256, 0, stream>>>(iters * 8, static_cast<int*>(sink));
+    const cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) { set_error("int_peak launch failed: %s", cudaGetErrorString(err)); return MMASIM_ERR_CUDA; }
+    return MMASIM_OK;
+}
+
 template <bool K16>
 int launch_dmma(int64_t blocks, int64_t iters, void* sink, int32_t* ops_per_round, cudaStream_t stream) {
     *ops_per_round = K16 ? 256 : 64;
@@ -279,6 +311,9 @@ int launch_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t
         case PK_DFMA_RM_X16: return launch_fma<double, 16, true, false>(blocks, iters, sink, ops_per_round, stream);
         case PK_DMMA_RM_K4: return launch_dmma<false>(blocks, iters, sink, ops_per_round, stream);
         case PK_DMMA_RM_K16: return launch_dmma<true>(blocks, iters, sink, ops_per_round, stream);
+        case PK_CVT_F32_F64: return launch_cvt<0>(blocks, iters, sink, ops_per_round, stream);
+        case PK_CVT_S32_F64: return launch_cvt<1>(blocks, iters, sink, ops_per_round, stream);
+        case PK_DADD_RM_X16: return launch_cvt<2>(blocks, iters, sink, ops_per_round, stream);
         default: set_error("mmasim_int_peak: unknown kind %d", kind); return MMASIM_ERR_INVALID_ARG;
     }
 }

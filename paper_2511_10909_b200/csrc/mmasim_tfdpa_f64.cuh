@@ -270,7 +270,9 @@ __host__ __device__ constexpr int pe64_sub(int base) { return base == 8 ? 32 : (
 
 // Decode pass: one CTA of 256 threads decodes one block (R rows x 32 elements) into shared memory and copies it to its
 // place dst[tile][chunk].  Rows beyond the matrix decode as zeros.
-template <int EK, int R, bool IS_A, int BASE>
+// EOSPLIT (GTR-FDPA, blocks of 16): inside each block of 16 the operand plane holds the even elements first, then the odd
+// ones, so that a matrix instruction sums four elements of one group; exponent pairs and masks keep the order of K.
+template <int EK, int R, bool IS_A, int BASE, bool EOSPLIT = false>
 __global__ void __launch_bounds__(256) decode64_kernel(DevModel m, const unsigned char* src, int64_t rows, int64_t ld, Blk64<R>* dst) {
     using E = Elem<EK>;
     constexpr int TPR = KC / E::TASK, TASKS = R * TPR, WORDS = E::TASK * E::BYTES / 4;
@@ -343,7 +345,7 @@ __global__ void __launch_bounds__(256) decode64_kernel(DevModel m, const unsigne
                 op = __hiloint2double(int(hi | (sign << 31)), int(lo));
                 bits += (sign | (nzbit << 16)) << q;
             }
-            blk.d[r][kk] = op;
+            blk.d[r][EOSPLIT ? ((kk & ~15) | ((kk & 1) << 3) | ((kk & 15) >> 1)) : kk] = op;
             // BF16 word of 2^(BASE (Exp - 1)) (the B plane times 2^shift); 0 for an element without exponent
             const uint32_t pe = (BASE && expb) ? uint32_t((127 + (IS_A ? 0 : pe64_shift(BASE)) + BASE * (int(expb) - EB - 1)) << 7) : 0u;
             if (q & 1) {

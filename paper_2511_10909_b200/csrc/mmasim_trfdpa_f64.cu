@@ -28,15 +28,19 @@ using fast::EK_BF16;
 using fast::EK_TF32;
 
 template <int EK, int L, bool GTR>
-__global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g) {
+__global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g, const Blk64<BM>* __restrict__ wa,
+                                                         const Blk64<BN>* __restrict__ wb) {
     constexpr int NBLK = KC / L;
-    static_assert(KC % L == 0 && L % 2 == 0, "blocks tile the chunk; the exponent pass handles pairs of elements");
-    using SM = Smem64<EK>;
+    static_assert(KC % L == 0 && L % 4 == 0 && (!GTR || L == 16), "blocks tile the chunk; a matrix instruction takes four terms");
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    SM& sm = *reinterpret_cast<SM*>(smem_raw);
+    SmemMM& sm = *reinterpret_cast<SmemMM*>(smem_raw);
 
     const int tid = threadIdx.x;
-    const int tx = tid % 16, ty = tid / 16;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int wr = warp >> 2, wc = warp & 3, gq = lane >> 2, tq = lane & 3;      // warp grid 4 x 4, warp tile 32 x 16
+    const int prow = wr * 32 + gq * 4, pcol = wc * 16 + tq * 4;                  // the thread's first permuted row / column
+    auto row_at = [&](int r) { return wr * 32 + gq + 8 * r; };                   // inside the CTA tile
+    auto col_at = [&](int c) { return wc * 16 + 8 * (c >> 1) + 2 * tq + (c & 1); };
     const int64_t row0 = int64_t(blockIdx.y) * BM, col0 = int64_t(blockIdx.x) * BN;
     const FmtDesc fa = fmt_desc(m.fmt_a), fb = fmt_desc(m.fmt_b);
     const int F = m.F, F2 = m.F2;
@@ -46,8 +50,24 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
     const int MAGIC_K = (MAGIC_E << 20) | 0x00080000;
     constexpr int E_FLOOR = CB - 400;
 
-    init_lut64<EK>(sm, fa, fb, tid);
-    if (tid == 0) sm.special[0] = sm.special[1] = sm.special[2] = 0;
+    // the decoded blocks of this tile row of A and tile column of B, chunk after chunk, land in two buffers by bulk copies
+    const int NCH = int(g.K / KC);
+    const Blk64<BM>* src_a = wa + int64_t(blockIdx.y) * NCH;
+    const Blk64<BN>* src_b = wb + int64_t(blockIdx.x) * NCH;
+    auto issue = [&](int n) {                              // one thread: both copies of chunk n into buffer n & 1
+        unsigned long long* bar = &sm.full[n & 1];
+        fast::mbar_expect_tx(bar, uint32_t(sizeof(Blk64<BM>) + sizeof(Blk64<BN>)));
+        fast::bulk_load(&sm.a[n & 1], src_a + n, uint32_t(sizeof(Blk64<BM>)), bar);
+        fast::bulk_load(&sm.b[n & 1], src_b + n, uint32_t(sizeof(Blk64<BN>)), bar);
+    };
+    if (tid == 0) {
+        sm.error = 0;
+        fast::mbar_init(&sm.full[0], 1u);
+        fast::mbar_init(&sm.full[1], 1u);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        issue(0);
+        if (NCH > 1) issue(1);
+    }
 
     uint32_t cw[TM][TN];                                // the accumulator of each output: a finite FP32 word
     uint32_t sp_nan = 0u, sp_pinf = 0u, sp_ninf = 0u;   // per output (bit r * TN + c): NaN / +inf / -inf seen so far
@@ -55,7 +75,7 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
     for (int r = 0; r < TM; ++r)
 #pragma unroll
         for (int c = 0; c < TN; ++c) {
-            const int64_t i = row0 + ty * TM + r, j = col0 + col_of(tx, c);
+            const int64_t i = row0 + row_at(r), j = col0 + col_at(c);
             uint32_t w = 0u;
             if (g.C && i < g.M && j < g.N) w = static_cast<const uint32_t*>(g.C)[i * g.ldc + j];
             const AccDec d = decode_acc(w, false);
@@ -67,57 +87,36 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
             cw[r][c] = w;
         }
 
-    RawChunk<EK> raw;
-    load_chunk<EK>(raw, g, row0, col0, 0, tid);
-    __syncthreads();                                    // tables and flags are ready
-    store_chunk64<EK>(sm, sm.pl[0], raw, 0, tid);
-    if (KC < g.K) load_chunk<EK>(raw, g, row0, col0, KC, tid);
-    __syncthreads();
+    __syncthreads();                                    // the barriers are initialised
     uint32_t emp[TM][TN];                               // product exponents of the block that comes next (low lane: even elements)
 
-    int chunk = 0;
-    for (int64_t k0 = 0; k0 < g.K; k0 += KC, ++chunk) {
-        auto& s = sm.pl[chunk & 1];
-        auto& nx = sm.pl[(chunk + 1) & 1];
-        // one barrier per chunk, at its end: every warp left the other buffer before the barrier that ended the previous
-        // iteration, so it can be filled while slower warps still compute on this one
-        if (tid == 0) sm.special[(chunk + 2) % 3] = 0;
-        if (k0 + KC < g.K) {
-            store_chunk64<EK>(sm, nx, raw, (chunk + 1) % 3, tid);
-            if (k0 + 2 * KC < g.K) load_chunk<EK>(raw, g, row0, col0, k0 + 2 * KC, tid);
-        }
-        const bool chunk_special = sm.special[chunk % 3] != 0;
+    for (int chunk = 0; chunk < NCH; ++chunk) {
+        const int64_t k0 = int64_t(chunk) * KC;
+        // a wait that runs out is recorded and the chunk computed on whatever is there; every thread sees the flag after
+        // the barrier at the end of the chunk, and the CTA leaves together without storing anything
+        if (!fast::mbar_wait(&sm.full[chunk & 1], uint32_t(chunk >> 1) & 1u)) *reinterpret_cast<volatile int*>(&sm.error) = 1;
+        const Blk64<BM>& sa_blk = sm.a[chunk & 1];
+        const Blk64<BN>& sb_blk = sm.b[chunk & 1];
+        const bool chunk_special = (sa_blk.special | sb_blk.special) != 0u;
         // the first block's product exponents (the other blocks' are taken beside the multiply-adds of their predecessor)
-        product_exponents<L>(&s.a_exp2[0][ty * TM], &s.b_exp2[0][tx * 2], emp);
+        product_exponents_adj<L>(&sa_blk.exp2[0][prow], &sb_blk.exp2[0][pcol], emp);
 
 #pragma unroll 1
         for (int blk = 0; blk < NBLK; ++blk) {
             const int kb = blk * L;
-            // ---- sum registers: the bare constants at the maximum exponents of this block's products ----
-            double t0[TM][TN], t1[GTR ? TM : 1][GTR ? TN : 1];
-            int emax_all = 0;
+            // ---- rare: infinities / NaNs in the chunk, or products that may reach 2^128: events of this block ----
+            uint32_t emax2 = 0u;
 #pragma unroll
             for (int r = 0; r < TM; ++r)
 #pragma unroll
-                for (int c = 0; c < TN; ++c) {
-                    // a group without a nonzero product (lane 0) gets E_FLOOR, below every real exponent: its sum stays 0
-                    // and the constants derived from its register's exponent stay inside FP64
-                    const int lo = int(emp[r][c] & 0xFFFFu), hi = int(emp[r][c] >> 16);
-                    if (GTR) {
-                        t0[r][c] = __hiloint2double(max(lo, E_FLOOR) * (1 << 20) + MAGIC_K, 0);
-                        t1[GTR ? r : 0][GTR ? c : 0] = __hiloint2double(max(hi, E_FLOOR) * (1 << 20) + MAGIC_K, 0);
-                    } else {
-                        t0[r][c] = __hiloint2double(__vimax3_s32(lo, hi, E_FLOOR) * (1 << 20) + MAGIC_K, 0);
-                    }
-                    emax_all = max(emax_all, max(lo, hi));
-                }
-            // ---- rare: infinities / NaNs in the chunk, or products that may reach 2^128: events of this block ----
+                for (int c = 0; c < TN; ++c) emax2 = __vmaxu2(emax2, emp[r][c]);
+            const int emax_all = int(max(emax2 & 0xFFFFu, emax2 >> 16));
             if (chunk_special || emax_all - CB >= 126) {
 #pragma unroll 1
                 for (int r = 0; r < TM; ++r)
 #pragma unroll 1
                     for (int c = 0; c < TN; ++c) {
-                        const int64_t i = row0 + ty * TM + r, j = col0 + col_of(tx, c);
+                        const int64_t i = row0 + row_at(r), j = col0 + col_at(c);
                         if (i >= g.M || j >= g.N) continue;
                         Special ev;
                         for (int kk = kb; kk < kb + L; ++kk) {
@@ -135,50 +134,41 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
                         if (ev.ninf) sp_ninf |= bit;
                     }
             }
-            // ---- one fused multiply-add per term; beside it the product exponents of the block that follows ----
-            {
-                const double* a_p = &s.a_d[kb][ty * TM];
-                const double* b_p = &s.b_d[kb][tx * 2];
-                // the next block of this chunk (after the chunk's last block the pass reads its first block again; that
-                // result is replaced at the start of the next chunk)
-                const uint32_t* ea_p = &s.a_exp2[(kb + L) / 2 < KC / 2 ? (kb + L) / 2 : 0][ty * TM];
-                const uint32_t* eb_p = &s.b_exp2[(kb + L) / 2 < KC / 2 ? (kb + L) / 2 : 0][tx * 2];
-#pragma unroll
-                for (int r = 0; r < TM; ++r)
-#pragma unroll
-                    for (int c = 0; c < TN; ++c) emp[r][c] = 0u;
-#pragma unroll
-                for (int kq = 0; kq < L; ++kq) {
-                    double av[TM], bv[TN];
-#pragma unroll
-                    for (int r = 0; r < TM; r += 2) {
-                        const double2 t = *reinterpret_cast<const double2*>(a_p + kq * BM + r);
-                        av[r] = t.x; av[r + 1] = t.y;
-                    }
-                    {
-                        const double2 u0 = *reinterpret_cast<const double2*>(b_p + kq * BN);
-                        const double2 u1 = *reinterpret_cast<const double2*>(b_p + kq * BN + BN / 2);
-                        bv[0] = u0.x; bv[1] = u0.y; bv[2] = u1.x; bv[3] = u1.y;
-                    }
-                    uint32_t ea[TM], ebv[TN];
-                    if ((kq & 1) == 0) {
-                        const int kp = kq / 2;
-                        const uint4 ea0 = *reinterpret_cast<const uint4*>(ea_p + kp * BM);
-                        const uint2 eb0 = *reinterpret_cast<const uint2*>(eb_p + kp * BN);
-                        const uint2 eb1 = *reinterpret_cast<const uint2*>(eb_p + kp * BN + BN / 2);
-                        ea[0] = ea0.x; ea[1] = ea0.y; ea[2] = ea0.z; ea[3] = ea0.w;
-                        ebv[0] = eb0.x; ebv[1] = eb0.y; ebv[2] = eb1.x; ebv[3] = eb1.y;
-                    }
-#pragma unroll
-                    for (int r = 0; r < TM; ++r)
-#pragma unroll
-                        for (int c = 0; c < TN; ++c) {
-                            if (GTR && (kq & 1)) t1[GTR ? r : 0][GTR ? c : 0] = __fma_rd(av[r], bv[c], t1[GTR ? r : 0][GTR ? c : 0]);
-                            else t0[r][c] = __fma_rd(av[r], bv[c], t0[r][c]);
-                            if ((kq & 1) == 0) emp[r][c] = __viaddmax_s16x2(ea[r], ebv[c], emp[r][c]);
-                        }
+            // ---- sum registers: the bare constants at the maximum exponents of this block's products; a group without a
+            // nonzero product (lane 0) gets E_FLOOR, below every real exponent: its sum stays 0 and the constants derived from
+            // its register's exponent stay inside FP64 ----
+            double t0[TM][TN], t1[GTR ? TM : 1][GTR ? TN : 1];
+            auto start = [&](int r, int c) {
+                const int lo = int(emp[r][c] & 0xFFFFu), hi = int(emp[r][c] >> 16);
+                if (GTR) {
+                    t0[r][c] = __hiloint2double(max(lo, E_FLOOR) * (1 << 20) + MAGIC_K, 0);
+                    t1[GTR ? r : 0][GTR ? c : 0] = __hiloint2double(max(hi, E_FLOOR) * (1 << 20) + MAGIC_K, 0);
+                } else {
+                    t0[r][c] = __hiloint2double(__vimax3_s32(lo, hi, E_FLOOR) * (1 << 20) + MAGIC_K, 0);
                 }
-            }
+            };
+            // four terms per matrix instruction (mma.sync m8n8k4, FP64, rounding toward minus infinity) for the rows
+            // 2 half, 2 half + 1 of the micro-tile; lane (g, t) holds A[8 r + g][k + t] and B[8 j + g][k + t].  GTR: the plane
+            // holds the eight even elements of the block first, then the eight odd ones.
+            auto mma_half = [&](int half, int ks) {
+                double af[2], bf[TN / 2];
+#pragma unroll
+                for (int r = 0; r < 2; ++r) af[r] = sa_blk.d[wr * 32 + 8 * (2 * half + r) + gq][kb + ks + tq];
+#pragma unroll
+                for (int j = 0; j < TN / 2; ++j) bf[j] = sb_blk.d[wc * 16 + 8 * j + gq][kb + ks + tq];
+#pragma unroll
+                for (int r = 0; r < 2; ++r)
+#pragma unroll
+                    for (int j = 0; j < TN / 2; ++j) {
+                        if (GTR && ks >= 8)
+                            asm volatile("mma.sync.aligned.m8n8k4.row.col.rm.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                                         : "+d"(t1[GTR ? 2 * half + r : 0][GTR ? 2 * j : 0]), "+d"(t1[GTR ? 2 * half + r : 0][GTR ? 2 * j + 1 : 0])
+                                         : "d"(af[r]), "d"(bf[j]));
+                        else
+                            asm volatile("mma.sync.aligned.m8n8k4.row.col.rm.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                                         : "+d"(t0[2 * half + r][2 * j]), "+d"(t0[2 * half + r][2 * j + 1]) : "d"(af[r]), "d"(bf[j]));
+                    }
+            };
             // ---- merge (Algorithm 10 Step 3 / Algorithm 11 Step 4) in FP64, where every quantity is exact:
             //   E = max(e_max, Exp(c));  T2 = floor(T 2^(e_max - F) / q2) q2 with q2 = 2^(E - F2): one fma.rd onto the
             //   grid of 1.5 * 2^52 * q2;  sc2 = floor(c / q1) q1 with q1 = 2^(E - F): one add.rd onto 1.5 * 2^52 * q1;
@@ -190,41 +180,78 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
             const int k_reg = (52 - F) << 20;              // a sum register's field is that of 2^e_max plus 52 - F
             const int k_m2 = ((52 - F2) << 20) | 0x00080000, k_m1 = (F2 - F) << 20, k_st = F << 20, k_gtr = (F + 1) << 20;
             uint32_t wmax = 0u;
+            auto merge = [&](int r, int c) {
+                const uint32_t sa = sa_blk.sgn[prow + r], nza = sa_blk.nz[prow + r] & kmask;
+                const uint32_t negm = (sa ^ sb_blk.sgn[pcol + c]) & nza & sb_blk.nz[pcol + c];
+                // the low word of a sum register is T (two's complement, |T| < 2^31), its exponent field gives e_max
+                int T, t20;
+                if (GTR) {
+                    const double u0 = t0[r][c], u1 = t1[GTR ? r : 0][GTR ? c : 0];
+                    const int te = __double2loint(u0) + __popc(negm & 0x55555555u);
+                    const int to = __double2loint(u1) + __popc(negm & 0xAAAAAAAAu);
+                    const int e20 = __double2hiint(u0) & EXPF, o20 = __double2hiint(u1) & EXPF;
+                    t20 = max(e20, o20);
+                    T = fast::asr_clamp(te, (t20 - e20) >> 20) + fast::asr_clamp(to, (t20 - o20) >> 20);      // RD_F of both group sums
+                } else {
+                    T = __double2loint(t0[r][c]) + __popc(negm);
+                    t20 = __double2hiint(t0[r][c]) & EXPF;
+                }
+                const uint32_t w0 = cw[r][c];
+                const double cd = double(__uint_as_float(w0));
+                int ec20 = max(__double2hiint(cd) & EXPF, (1023 - 126) << 20);      // a subnormal accumulator has the exponent -126
+                if ((w0 & 0x7FFFFFFFu) == 0u) ec20 = 0;                             // a zero accumulator has none
+                const int em20 = t20 - k_reg;                                       // e_max
+                const int E20 = max(em20, ec20);                                    // E = max(e_max, Exp(c))
+                const double scale_t = __hiloint2double(em20 - k_st, 0);            // 2^(e_max - F)
+                const double m2 = __hiloint2double(E20 + k_m2, 0);                  // 1.5 * 2^52 * 2^(E - F2)
+                const double m1 = __hiloint2double(E20 + k_m2 + k_m1, 0);           // 1.5 * 2^52 * 2^(E - F)
+                const double t2 = __dsub_rn(__fma_rd(double(T), scale_t, m2), m2);  // RD_F2
+                double sc2 = __dsub_rn(__dadd_rd(cd, m1), m1);                      // RD_F
+                if (GTR && ec20 < E20 - k_gtr) sc2 = 0.0;                           // special truncation
+                const uint32_t w = __float_as_uint(__double2float_rn(__dadd_rn(t2, sc2)));      // exact sum, then rho
+                wmax = max(wmax, w & 0x7FFFFFFFu);
+                cw[r][c] = w;
+            };
+
+            // ---- the block in two halves of the micro-tile (rows 0, 1 and rows 2, 3): the matrix instructions of one half
+            // are issued between the merge of the other and the product exponents of the next block ----
+            constexpr int NKS = L / 4, PER = 8 / (NKS < 8 ? NKS : 8);
+            const bool fuse = NBLK > 1 && blk + 1 < NBLK;
 #pragma unroll
-            for (int r = 0; r < TM; ++r) {
-                const uint32_t sa = s.a_sgn[ty * TM + r], nza = s.a_nz[ty * TM + r] & kmask;
+            for (int o = 0; o < 16; ++o) start(o / TN, o % TN);
 #pragma unroll
-                for (int c = 0; c < TN; ++c) {
-                    const uint32_t negm = (sa ^ s.b_sgn[col_of(tx, c)]) & nza & s.b_nz[col_of(tx, c)];
-                    // the low word of a sum register is T (two's complement, |T| < 2^31), its exponent field gives e_max
-                    int T, t20;
-                    if (GTR) {
-                        const int te = __double2loint(t0[r][c]) + __popc(negm & 0x55555555u);
-                        const int to = __double2loint(t1[GTR ? r : 0][GTR ? c : 0]) + __popc(negm & 0xAAAAAAAAu);
-                        const int e20 = __double2hiint(t0[r][c]) & EXPF, o20 = __double2hiint(t1[GTR ? r : 0][GTR ? c : 0]) & EXPF;
-                        t20 = max(e20, o20);
-                        T = fast::asr_clamp(te, (t20 - e20) >> 20) + fast::asr_clamp(to, (t20 - o20) >> 20);      // RD_F of both group sums
-                    } else {
-                        T = __double2loint(t0[r][c]) + __popc(negm);
-                        t20 = __double2hiint(t0[r][c]) & EXPF;
+            for (int ksi = 0; ksi < NKS; ++ksi) mma_half(0, 4 * ksi);
+#pragma unroll
+            for (int ksi = 0; ksi < NKS; ++ksi) {
+                mma_half(1, 4 * ksi);
+#pragma unroll
+                for (int q = 0; q < PER; ++q)
+                    if (ksi * PER + q < 8) merge((ksi * PER + q) / TN, (ksi * PER + q) % TN);
+                if (fuse) {                             // the product exponents of the next block
+                    const uint32_t* ea_p = &sa_blk.exp2[(kb + L) / 2][prow];
+                    const uint32_t* eb_p = &sb_blk.exp2[(kb + L) / 2][pcol];
+                    if (ksi == 0) {
+#pragma unroll
+                        for (int r = 0; r < TM; ++r)
+#pragma unroll
+                            for (int c = 0; c < TN; ++c) emp[r][c] = 0u;
                     }
-                    const uint32_t w0 = cw[r][c];
-                    const double cd = double(__uint_as_float(w0));
-                    int ec20 = max(__double2hiint(cd) & EXPF, (1023 - 126) << 20);      // a subnormal accumulator has the exponent -126
-                    if ((w0 & 0x7FFFFFFFu) == 0u) ec20 = 0;                             // a zero accumulator has none
-                    const int em20 = t20 - k_reg;                                       // e_max
-                    const int E20 = max(em20, ec20);                                    // E = max(e_max, Exp(c))
-                    const double scale_t = __hiloint2double(em20 - k_st, 0);            // 2^(e_max - F)
-                    const double m2 = __hiloint2double(E20 + k_m2, 0);                  // 1.5 * 2^52 * 2^(E - F2)
-                    const double m1 = __hiloint2double(E20 + k_m2 + k_m1, 0);           // 1.5 * 2^52 * 2^(E - F)
-                    const double t2 = __dsub_rn(__fma_rd(double(T), scale_t, m2), m2);  // RD_F2
-                    double sc2 = __dsub_rn(__dadd_rd(cd, m1), m1);                      // RD_F
-                    if (GTR && ec20 < E20 - k_gtr) sc2 = 0.0;                           // special truncation
-                    const uint32_t w = __float_as_uint(__double2float_rn(__dadd_rn(t2, sc2)));      // exact sum, then rho
-                    wmax = max(wmax, w & 0x7FFFFFFFu);
-                    cw[r][c] = w;
+#pragma unroll
+                    for (int kp = 2 * ksi; kp < 2 * ksi + 2; ++kp) {
+                        const uint4 ea0 = *reinterpret_cast<const uint4*>(ea_p + kp * BM);
+                        const uint4 eb0 = *reinterpret_cast<const uint4*>(eb_p + kp * BN);
+                        const uint32_t ea[TM] = {ea0.x, ea0.y, ea0.z, ea0.w};
+                        const uint32_t ebv[TN] = {eb0.x, eb0.y, eb0.z, eb0.w};
+#pragma unroll
+                        for (int r = 0; r < TM; ++r)
+#pragma unroll
+                            for (int c = 0; c < TN; ++c) emp[r][c] = __viaddmax_s16x2(ea[r], ebv[c], emp[r][c]);
+                    }
                 }
             }
+#pragma unroll
+            for (int o = 8; o < 16; ++o) merge(o / TN, o % TN);
+
             if (wmax >= 0x7F800000u) {                     // rare: RNE-FP32 overflowed: +-infinity from now on
 #pragma unroll
                 for (int r = 0; r < TM; ++r)
@@ -237,14 +264,24 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
                         }
             }
         }
-        __syncthreads();                                // the other buffer is complete, this one is free
+        __syncthreads();                                // everybody has finished with this buffer
+        if (*reinterpret_cast<volatile int*>(&sm.error)) break;
+        if (tid == 0 && chunk + 2 < NCH) issue(chunk + 2);
     }
 
+    if (*reinterpret_cast<volatile int*>(&sm.error)) {  // a copy never arrived: count it, give the copies in flight one more
+        if (tid == 0) {                                 // bounded wait each, and store nothing
+            atomicAdd(&fast::g_copy_timeouts, 1u);
+            fast::mbar_wait(&sm.full[0], 0u);
+            fast::mbar_wait(&sm.full[1], 0u);
+        }
+        return;
+    }
 #pragma unroll
     for (int r = 0; r < TM; ++r)
 #pragma unroll
         for (int c = 0; c < TN; ++c) {
-            const int64_t i = row0 + ty * TM + r, j = col0 + col_of(tx, c);
+            const int64_t i = row0 + row_at(r), j = col0 + col_at(c);
             if (i >= g.M || j >= g.N) continue;
             const uint32_t bit = r * TN + c;
             const uint32_t spv = ((sp_nan >> bit) & 1u) | (((sp_pinf >> bit) & 1u) << 1) | (((sp_ninf >> bit) & 1u) << 2);
@@ -262,12 +299,30 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g)
 
 template <int EK, int L, bool GTR>
 cudaError_t launch_tr_one(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
-    const size_t sh = sizeof(Smem64<EK>);
+    const size_t sh = sizeof(SmemMM);
     cudaError_t err = cudaFuncSetAttribute(trfdpa64_kernel<EK, L, GTR>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sh));
     if (err != cudaSuccess) return err;
-    dim3 grid((unsigned)((g.N + BN - 1) / BN), (unsigned)((g.M + BM - 1) / BM), 1);
-    trfdpa64_kernel<EK, L, GTR><<<grid, NT, sh, stream>>>(m, g);
-    return cudaGetLastError();
+    const size_t dsh_a = 256 * sizeof(LutEntry64) + sizeof(Blk64<BM>), dsh_b = 256 * sizeof(LutEntry64) + sizeof(Blk64<BN>);
+    if ((err = cudaFuncSetAttribute(decode64_kernel<EK, BM, true, 0, GTR>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(dsh_a))) != cudaSuccess) return err;
+    if ((err = cudaFuncSetAttribute(decode64_kernel<EK, BN, false, 0, GTR>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(dsh_b))) != cudaSuccess) return err;
+    const int64_t tiles_m = (g.M + BM - 1) / BM, tiles_n = (g.N + BN - 1) / BN, nch = g.K / KC;
+    // scratch: the decoded blocks of A and B, stream-ordered out of the library's pool and returned to it behind the kernel
+    const size_t bytes_a = size_t(tiles_m * nch) * sizeof(Blk64<BM>), bytes_b = size_t(tiles_n * nch) * sizeof(Blk64<BN>);
+    cudaMemPool_t pool = nullptr;
+    if ((err = scratch_pool(&pool)) != cudaSuccess) return err;
+    void* ws = nullptr;
+    if ((err = cudaMallocFromPoolAsync(&ws, bytes_a + bytes_b, pool, stream)) != cudaSuccess) return err;
+    Blk64<BM>* wa = static_cast<Blk64<BM>*>(ws);
+    Blk64<BN>* wb = reinterpret_cast<Blk64<BN>*>(static_cast<unsigned char*>(ws) + bytes_a);
+    decode64_kernel<EK, BM, true, 0, GTR><<<dim3((unsigned)nch, (unsigned)tiles_m), 256, dsh_a, stream>>>(
+        m, static_cast<const unsigned char*>(g.A), g.M, g.lda, wa);
+    decode64_kernel<EK, BN, false, 0, GTR><<<dim3((unsigned)nch, (unsigned)tiles_n), 256, dsh_b, stream>>>(
+        m, static_cast<const unsigned char*>(g.B), g.N, g.ldb, wb);
+    dim3 grid((unsigned)tiles_n, (unsigned)tiles_m, 1);
+    trfdpa64_kernel<EK, L, GTR><<<grid, NT, sh, stream>>>(m, g, wa, wb);
+    err = cudaGetLastError();
+    const cudaError_t err2 = cudaFreeAsync(ws, stream);
+    return err != cudaSuccess ? err : err2;
 }
 
 }  // namespace

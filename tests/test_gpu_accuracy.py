@@ -63,3 +63,20 @@ def test_hopper_fp8_summation_precision_is_the_bottleneck():
     blackwell = accuracy.deviation_stats(mmasim.Model("blackwell", "e4m3", "fp32"), dA, dB, dC, ref)
     assert hopper["mean_abs"] > 100 * blackwell["mean_abs"]
     assert hopper["mean"] != 0.0
+
+
+def test_risky_designs_at_gemm_scale():
+    """Table 10, row by row: each design named there shows as a larger (or one-sided) deviation from the real result than
+    the nearest row without it, on the same inputs."""
+    from paper_2511_10909_b200 import accuracy
+    r = accuracy.risky_designs()
+    ftz = r["input_ftz"]
+    assert ftz["cdna2"]["mean_abs"] > 100 * ftz["cdna1"]["mean_abs"]           # flushed FP16 subnormals
+    assert r["small_F"]["F13"]["mean_abs"] > 100 * r["small_F"]["F25"]["mean_abs"]
+    assert r["rz_e8m13"]["RZ-E8M13"]["mean_abs"] > 100 * r["rz_e8m13"]["RZ-FP32"]["mean_abs"]
+    assert r["rne_fp16"]["fp16_out"]["mean_abs"] > 100 * r["rne_fp16"]["fp32_out"]["mean_abs"]
+    asym = r["asymmetry"]
+    assert asym["hopper-fp16"]["asymmetric"] == 0
+    for k in ("cdna3-fp16", "cdna3-bf16", "cdna3-e4m3"):
+        assert asym[k]["asymmetric"] > 0.05 * asym[k]["count"], (k, asym[k])
+        assert asym[k]["mean_sum"] < 0                                          # round-down: both signs lean the same way
