@@ -396,14 +396,19 @@ __device__ __forceinline__ void product_exponents(const uint32_t* ea_p, const ui
     }
 }
 
+// Multipliers read from the constant bank, so that the compiler keeps integer multiply-adds (which issue beside the
+// integer pipe) instead of rewriting them as shifts and additions on it.
+static __constant__ int c_mul64[4] = {1 << 20, 16, 1, 0};
+__device__ __forceinline__ int imad(int a, int b, int c) {
+    int d;
+    asm("mad.lo.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
 // The same for the permuted layout: ea_p / eb_p point at the thread's four adjacent (permuted) rows / columns of the
 // first pair of the block.
 template <int L>
 __device__ __forceinline__ void product_exponents_adj(const uint32_t* ea_p, const uint32_t* eb_p, uint32_t (&emp)[TM][TN]) {
-#pragma unroll
-    for (int r = 0; r < TM; ++r)
-#pragma unroll
-        for (int c = 0; c < TN; ++c) emp[r][c] = 0u;
 #pragma unroll
     for (int kp = 0; kp < L / 2; ++kp) {
         const uint4 ea0 = *reinterpret_cast<const uint4*>(ea_p + kp * BM);
@@ -413,7 +418,7 @@ __device__ __forceinline__ void product_exponents_adj(const uint32_t* ea_p, cons
 #pragma unroll
         for (int r = 0; r < TM; ++r)
 #pragma unroll
-            for (int c = 0; c < TN; ++c) emp[r][c] = __viaddmax_s16x2(ea[r], ebv[c], emp[r][c]);
+            for (int c = 0; c < TN; ++c) emp[r][c] = __viaddmax_s16x2(ea[r], ebv[c], kp == 0 ? 0u : emp[r][c]);
     }
 }
 
@@ -474,6 +479,10 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
     // conversion function is then a mask on the double's low word and the exponent of c is the double's own field.
     // Results outside the range of normal FP32 numbers (zero, subnormal, overflow) leave the fast path.
     constexpr bool DS = !ACC16;
+    // blocks of at most 8 terms: |S| < 2^(F+1) + L * 2^(F+2) < 2^31, so the sum register's low word, started at 2^31, never
+    // carries into the high word
+    constexpr bool NARROW = DS && L <= 8;
+    constexpr int UNROLL_BLK = (L <= 4 || (L <= 8 && BASE == 0)) ? 2 : 1;   // short blocks: two per trip of the block loop
     // (a zero of either sign becomes the positive state: under ST scaling the set bit of -0 could underflow away and leave
     // the +1 of a negative accumulator uncompensated)
     auto state_of = [](uint32_t w) { const double d = (w & 0x7FFFFFFFu) ? double(__uint_as_float(w)) : 0.0; return __hiloint2double(__double2hiint(d), __double2loint(d) | 1); };
@@ -543,7 +552,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
             sp_nan |= scale_nan;                        // a NaN scale factor makes the block result NaN
         }
 
-#pragma unroll 1
+#pragma unroll UNROLL_BLK
         for (int blk = 0; blk < NBLK; ++blk) {
             const int kb = blk * L;
             // ---- rare: the chunk holds an infinity or a NaN: special-value events of this block (Section 4.2).
@@ -640,16 +649,27 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                 if (DS) {
                     const double st = cs[DS ? r : 0][DS ? c : 0];
                     const int hi = __double2hiint(st);
-                    int keyc = subnormal_c ? (1023 - 126) << 20 : hi & 0x7FF00000;
+                    // the keys keep whatever sits below their exponent fields (mantissa bits of c, the other 16-bit lane): it
+                    // decides nothing but ties between equal exponents, and one mask after the maximum removes it
+                    int keyc = subnormal_c ? (1023 - 126) << 20 : hi & 0x7FFFFFFF;
                     if (ST) keyc -= (sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]) << 20;
                     const uint32_t e2 = emp[r][c];
-                    // BASE > 0: P = 0 gives a key two binades below the smallest real one, which is wrong only for an even
-                    // smaller c: the epilogue repairs that case
-                    const int keyp = BASE ? int((e2 >> (3 + LB)) & 0xFFF00000u) + KP2
-                                          : int(__vmaxu2(e2, __byte_perm(e2, 0u, 0x1032)) & 0xFFFFu) * (1 << 20) - (1 << 20);
-                    const int e20 = ST ? __vimax3_s32(keyp, keyc, 0) : max(keyp, keyc);
-                    // the +1 of a negative c sits in the constant's low word: one unit of the grid either way
-                    const double magic = __hiloint2double(e20 + km, int(uint32_t(hi) >> 31));
+                    int m;
+                    if (BASE) {
+                        // P = 0 gives a key two binades below the smallest real one, which is wrong only for an even smaller c:
+                        // the epilogue repairs that case
+                        m = ST ? __vimax3_s32(int(e2 >> (3 + LB)) + KP2, keyc, 0) : __viaddmax_s32(int(e2 >> (3 + LB)), KP2, keyc);
+                    } else {
+                        // the two 16-bit lanes (Exp + CB of the even and the odd elements) moved to the exponent field by
+                        // multiplications, which run beside the integer pipe
+                        const int klo = imad(int(e2), c_mul64[0], -(1 << 20)), khi = imad(int(e2), c_mul64[1], -(1 << 20));
+                        m = __vimax3_s32(klo, khi, ST ? max(keyc, 0) : keyc);
+                    }
+                    const int e20 = m & 0x7FF00000;
+                    // the +1 of a negative c sits in the constant's low word: one unit of the grid either way.  Short blocks:
+                    // the low word starts at 2^31, so that the sign correction of the epilogue is a 32-bit addition
+                    const int mlo = NARROW ? int(__funnelshift_l(uint32_t(hi), 0x40000000u, 1)) : int(uint32_t(hi) >> 31);
+                    const double magic = __hiloint2double(imad(e20, c_mul64[2], km), mlo);
                     const double x = ST ? __dmul_rn(st, pow2d(-(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]))) : st;
                     acc[r][c] = __dadd_rd(x, magic);
                 } else {
@@ -698,27 +718,38 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
             constexpr uint32_t SUSPECT = ACC16 ? 0x7C00u : 0x7F7FFFFFu;   // FP16: infinity; FP32: cvt.rz saturates at the largest finite word
             uint32_t wmax = 0u;
             bool no_product = false;                    // BASE > 0: some output of the micro-tile has no nonzero product
-            bool odd = false;                           // FP32 state: some result is not a normal FP32 number
+            // FP32 state: the largest (high word of |v|) - (that of 2^-126), unsigned: a v outside the normal FP32 range -
+            // zero and the subnormal range wrap to the top - shows as a value of (that of 2^128) - (that of 2^-126) or more
+            constexpr uint32_t LOWHI = uint32_t(1023 - 126) << 20, SPANHI = uint32_t(128 + 126) << 20;
+            uint32_t urange = 0u;
             auto block_value = [&](int r, int c) -> double {
                 const uint32_t sa = sa_blk.sgn[prow + r], nza = sa_blk.nz[prow + r] & kmask;
                 const uint32_t live = nza & sb_blk.nz[pcol + c];
                 if (BASE) no_product = no_product || live == 0u;
                 const int nneg = __popc((sa ^ sb_blk.sgn[pcol + c]) & live);
-                const long long bits = __double_as_longlong(acc[r][c]) + (long long)nneg;
-                const int hi = int(bits >> 32);
-                const double magic = __hiloint2double((hi & 0x7FF00000) | 0x00080000, 0);
-                double v = __dsub_rn(__longlong_as_double(bits), magic);              // S * q, exact; +0 when S = 0
+                double v;
+                if (NARROW) {
+                    const int hi = __double2hiint(acc[r][c]);
+                    const double magic = __hiloint2double((hi & 0x7FF00000) | 0x00080000, int(0x80000000u));
+                    v = __dsub_rn(__hiloint2double(hi, __double2loint(acc[r][c]) + nneg), magic);
+                } else {
+                    const long long bits = __double_as_longlong(acc[r][c]) + (long long)nneg;
+                    const int hi = int(bits >> 32);
+                    const double magic = __hiloint2double((hi & 0x7FF00000) | 0x00080000, 0);
+                    v = __dsub_rn(__longlong_as_double(bits), magic);                 // S * q, exact; +0 when S = 0
+                }
                 if (ST) v = __dmul_rn(v, pow2d(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]));
                 return v;
             };
-            double nv[DS ? TM : 1][DS ? TN : 1];
+            double nv[DS && BASE ? TM : 1][DS && BASE ? TN : 1];      // BASE > 0: the old accumulators survive until the repair below
             uint32_t nw[DS ? 1 : TM][DS ? 1 : TN];
             auto finish = [&](int r, int c) {
                 const double v = block_value(r, c);
                 if (DS) {
-                    odd = odd || !(fabs(v) >= 1.1754943508222875e-38) || !(fabs(v) < 3.402823669209385e38);
+                    urange = __viaddmax_u32(uint32_t(__double2hiint(v)) & 0x7FFFFFFFu, 0u - LOWHI, urange);
                     // RZ-FP32 of a number in the normal range: the low 29 bits of the double's significand go
-                    nv[DS ? r : 0][DS ? c : 0] = __hiloint2double(__double2hiint(v), (__double2loint(v) & int(0xE0000000u)) | 1);
+                    const double st = __hiloint2double(__double2hiint(v), (__double2loint(v) & int(0xE0000000u)) | 1);
+                    if (BASE) nv[BASE ? r : 0][BASE ? c : 0] = st; else cs[DS ? r : 0][DS ? c : 0] = st;
                 } else {
                     const uint32_t w = ACC16 ? uint32_t(__half_as_ushort(__double2half(v))) : __float_as_uint(__double2float_rz(v));
                     wmax = max(wmax, w & ABS);
@@ -751,12 +782,6 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                 if (fuse) {                             // the product exponents of the next block (add-max kinds)
                     const uint32_t* ea_p = &sa_blk.exp2[(kb + L) / 2 < KC / 2 ? (kb + L) / 2 : 0][prow];
                     const uint32_t* eb_p = &sb_blk.exp2[(kb + L) / 2 < KC / 2 ? (kb + L) / 2 : 0][pcol];
-                    if (ksi == 0) {
-#pragma unroll
-                        for (int r = 0; r < TM; ++r)
-#pragma unroll
-                            for (int c = 0; c < TN; ++c) emp[r][c] = 0u;
-                    }
 #pragma unroll
                     for (int kp = 2 * ksi; kp < 2 * ksi + 2; ++kp) {
                         const uint4 ea0 = *reinterpret_cast<const uint4*>(ea_p + kp * BM);
@@ -766,7 +791,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
 #pragma unroll
                         for (int r = 0; r < TM; ++r)
 #pragma unroll
-                            for (int c = 0; c < TN; ++c) emp[r][c] = __viaddmax_s16x2(ea[r], ebv[c], emp[r][c]);
+                            for (int c = 0; c < TN; ++c) emp[r][c] = __viaddmax_s16x2(ea[r], ebv[c], kp == 0 ? 0u : emp[r][c]);
                     }
                 }
             }
@@ -774,18 +799,19 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
             for (int o = 8; o < 16; ++o) finish(o / TN, o % TN);
 
             if (DS) {
+                bool odd = urange >= SPANHI;            // some result is not a normal FP32 number
                 if (BASE && no_product) {               // rare: no nonzero product: the block returns its accumulator
                     odd = true;
 #pragma unroll
                     for (int r = 0; r < TM; ++r)
 #pragma unroll
                         for (int c = 0; c < TN; ++c)
-                            if ((sa_blk.nz[prow + r] & kmask & sb_blk.nz[pcol + c]) == 0u) nv[DS ? r : 0][DS ? c : 0] = cs[DS ? r : 0][DS ? c : 0];
+                            if ((sa_blk.nz[prow + r] & kmask & sb_blk.nz[pcol + c]) == 0u) nv[BASE ? r : 0][BASE ? c : 0] = cs[DS ? r : 0][DS ? c : 0];
                 }
 #pragma unroll
                 for (int r = 0; r < TM; ++r)
 #pragma unroll
-                    for (int c = 0; c < TN; ++c) cs[DS ? r : 0][DS ? c : 0] = nv[DS ? r : 0][DS ? c : 0];
+                    for (int c = 0; c < TN; ++c) if (BASE) cs[DS ? r : 0][DS ? c : 0] = nv[BASE ? r : 0][BASE ? c : 0];
                 if (odd || sub_mask) {                  // rare: zero, FP32 subnormal or overflow somewhere in the micro-tile
                     sub_mask = 0u;
 #pragma unroll

@@ -47,8 +47,6 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g,
     const int frac = fa.mbits + fb.mbits;
     // high word of 1.5 * 2^52 * 2^(e_max - F) is (e_max + CB) * 2^20 + MAGIC_K
     const int MAGIC_E = 1023 + 52 - F - CB;
-    const int MAGIC_K = (MAGIC_E << 20) | 0x00080000;
-    constexpr int E_FLOOR = CB - 400;
 
     // the decoded blocks of this tile row of A and tile column of B, chunk after chunk, land in two buffers by bulk copies
     const int NCH = int(g.K / KC);
@@ -69,7 +67,9 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g,
         if (NCH > 1) issue(1);
     }
 
-    uint32_t cw[TM][TN];                                // the accumulator of each output: a finite FP32 word
+    // The accumulator of each output lives between blocks as a double holding the FP32 value (exact); its exponent field is
+    // Exp(c) in place: zero has the field 0 (no exponent), an FP32 subnormal a field below that of 2^-126 (it counts as -126).
+    double cs[TM][TN];
     uint32_t sp_nan = 0u, sp_pinf = 0u, sp_ninf = 0u;   // per output (bit r * TN + c): NaN / +inf / -inf seen so far
 #pragma unroll
     for (int r = 0; r < TM; ++r)
@@ -84,7 +84,7 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g,
                 if (d.cls == CLS_NAN) sp_nan |= bit; else if (d.sign) sp_ninf |= bit; else sp_pinf |= bit;
                 w = 0u;
             }
-            cw[r][c] = w;
+            cs[r][c] = double(__uint_as_float(w));
         }
 
     __syncthreads();                                    // the barriers are initialised
@@ -135,16 +135,19 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g,
                     }
             }
             // ---- sum registers: the bare constants at the maximum exponents of this block's products; a group without a
-            // nonzero product (lane 0) gets E_FLOOR, below every real exponent: its sum stays 0 and the constants derived from
-            // its register's exponent stay inside FP64 ----
+            // nonzero product (lane 0) gets an exponent far below every real one: its sum stays 0 ----
+            constexpr int EXPF = 0x7FF00000, HALF = 0x00080000, LOW0 = int(0x80000000u);
             double t0[TM][TN], t1[GTR ? TM : 1][GTR ? TN : 1];
+            // (the two 16-bit lanes reach the exponent field by multiplications, which issue beside the integer pipe; what is
+            // left below the field is masked away; the low word starts at 2^31: |T| < 2^30, so the sign correction of the
+            // merge is a 32-bit addition that never carries)
             auto start = [&](int r, int c) {
-                const int lo = int(emp[r][c] & 0xFFFFu), hi = int(emp[r][c] >> 16);
+                const int klo = imad(int(emp[r][c]), c_mul64[0], MAGIC_E << 20), khi = imad(int(emp[r][c]), c_mul64[1], MAGIC_E << 20);
                 if (GTR) {
-                    t0[r][c] = __hiloint2double(max(lo, E_FLOOR) * (1 << 20) + MAGIC_K, 0);
-                    t1[GTR ? r : 0][GTR ? c : 0] = __hiloint2double(max(hi, E_FLOOR) * (1 << 20) + MAGIC_K, 0);
+                    t0[r][c] = __hiloint2double((klo & EXPF) | HALF, LOW0);
+                    t1[GTR ? r : 0][GTR ? c : 0] = __hiloint2double((khi & EXPF) | HALF, LOW0);
                 } else {
-                    t0[r][c] = __hiloint2double(__vimax3_s32(lo, hi, E_FLOOR) * (1 << 20) + MAGIC_K, 0);
+                    t0[r][c] = __hiloint2double((max(klo, khi) & EXPF) | HALF, LOW0);
                 }
             };
             // four terms per matrix instruction (mma.sync m8n8k4, FP64, rounding toward minus infinity) for the rows
@@ -169,48 +172,56 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g,
                                          : "+d"(t0[2 * half + r][2 * j]), "+d"(t0[2 * half + r][2 * j + 1]) : "d"(af[r]), "d"(bf[j]));
                     }
             };
-            // ---- merge (Algorithm 10 Step 3 / Algorithm 11 Step 4) in FP64, where every quantity is exact:
-            //   E = max(e_max, Exp(c));  T2 = floor(T 2^(e_max - F) / q2) q2 with q2 = 2^(E - F2): one fma.rd onto the
-            //   grid of 1.5 * 2^52 * q2;  sc2 = floor(c / q1) q1 with q1 = 2^(E - F): one add.rd onto 1.5 * 2^52 * q1;
-            //   their sum has at most 40 significant bits; RNE-FP32 is one conversion.  An overflow is rare and sticky:
-            //   the loop tracks the largest result word, the flags are set in a second pass. ----
+            // ---- merge (Algorithm 10 Step 3 / Algorithm 11 Step 4) in FP64, where every quantity is exact.
+            //   E = max(e_max, Exp(c)); T is rounded down onto 2^(E - F2), c onto 2^(E - F).  Whichever of the two exponents
+            //   is larger, both roundings can be taken on the one grid qv = 2^max(e_max - F, Exp(c) - F2): the operand that
+            //   needs no rounding (T when E = e_max, c when E = Exp(c)) is a multiple of qv anyway.  With Mv = 1.5 * 2^52 * qv:
+            //       Z1 = RD(c + Mv);   Z = RD(T q + Z1) = Mv + RD_qv(c) + RD_qv(T q);   v = Z - Mv     (at most 40 bits)
+            //   T q is the sum register minus its constant (after the sign correction, added to the register's bit pattern).
+            //   RNE-FP32 of v is one more addition and subtraction of a constant, 1.5 * 2^52 * 2^(Exp(v) - 23), the exponent
+            //   clamped at -126 for the subnormal range; the sign of v is copied onto the result (a negative sum that rounds
+            //   to zero is -0 under RNE-FP32).  A result of 2^128 or more is rare and sticky: the loop tracks the largest
+            //   exponent, the flags are set in a second pass. ----
             const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
             // exponents as the exponent fields of doubles, in place (bits 20..30 of the high word): x20 = (x + 1023) << 20
-            constexpr int EXPF = 0x7FF00000;
-            const int k_reg = (52 - F) << 20;              // a sum register's field is that of 2^e_max plus 52 - F
-            const int k_m2 = ((52 - F2) << 20) | 0x00080000, k_m1 = (F2 - F) << 20, k_st = F << 20, k_gtr = (F + 1) << 20;
-            uint32_t wmax = 0u;
+            constexpr uint32_t LOWF = (1023 - 126) << 20, HIGHF = (1023 + 126) << 20;
+            const uint32_t k_c = uint32_t(((52 - F2) << 20) | HALF) + 1u;   // (field of Exp(c)) - 1 + k_c: high word of 1.5 * 2^52 * 2^(Exp(c) - F2)
+            constexpr uint32_t k_gtr = (53u << 20) + 1u;   // a sum register's field minus Exp(c)'s beyond which c is dropped (GTR)
+            int fmax = 0;
             auto merge = [&](int r, int c) {
                 const uint32_t sa = sa_blk.sgn[prow + r], nza = sa_blk.nz[prow + r] & kmask;
                 const uint32_t negm = (sa ^ sb_blk.sgn[pcol + c]) & nza & sb_blk.nz[pcol + c];
-                // the low word of a sum register is T (two's complement, |T| < 2^31), its exponent field gives e_max
-                int T, t20;
+                double Y;                                   // T * 2^(e_max - F)
+                int m0hi;                                   // high word of the sum register's constant (e_max in place)
                 if (GTR) {
+                    // both group sums rounded down onto the coarser of their two grids, then added (Algorithm 11 Step 3)
                     const double u0 = t0[r][c], u1 = t1[GTR ? r : 0][GTR ? c : 0];
-                    const int te = __double2loint(u0) + __popc(negm & 0x55555555u);
-                    const int to = __double2loint(u1) + __popc(negm & 0xAAAAAAAAu);
-                    const int e20 = __double2hiint(u0) & EXPF, o20 = __double2hiint(u1) & EXPF;
-                    t20 = max(e20, o20);
-                    T = fast::asr_clamp(te, (t20 - e20) >> 20) + fast::asr_clamp(to, (t20 - o20) >> 20);      // RD_F of both group sums
+                    const int e_hi = (__double2hiint(u0) & EXPF) | HALF, o_hi = (__double2hiint(u1) & EXPF) | HALF;
+                    m0hi = max(e_hi, o_hi);
+                    const double ye = __dsub_rn(__hiloint2double(__double2hiint(u0), __double2loint(u0) + __popc(negm & 0x55555555u)),
+                                                __hiloint2double(e_hi, LOW0));
+                    const double yo = __dsub_rn(__hiloint2double(__double2hiint(u1), __double2loint(u1) + __popc(negm & 0xAAAAAAAAu)),
+                                                __hiloint2double(o_hi, LOW0));
+                    const double mm = __hiloint2double(m0hi, 0);
+                    Y = __dsub_rn(__dadd_rd(yo, __dadd_rd(ye, mm)), mm);
                 } else {
-                    T = __double2loint(t0[r][c]) + __popc(negm);
-                    t20 = __double2hiint(t0[r][c]) & EXPF;
+                    const double u0 = t0[r][c];
+                    m0hi = (__double2hiint(u0) & EXPF) | HALF;
+                    Y = __dsub_rn(__hiloint2double(__double2hiint(u0), __double2loint(u0) + __popc(negm)), __hiloint2double(m0hi, LOW0));
                 }
-                const uint32_t w0 = cw[r][c];
-                const double cd = double(__uint_as_float(w0));
-                int ec20 = max(__double2hiint(cd) & EXPF, (1023 - 126) << 20);      // a subnormal accumulator has the exponent -126
-                if ((w0 & 0x7FFFFFFFu) == 0u) ec20 = 0;                             // a zero accumulator has none
-                const int em20 = t20 - k_reg;                                       // e_max
-                const int E20 = max(em20, ec20);                                    // E = max(e_max, Exp(c))
-                const double scale_t = __hiloint2double(em20 - k_st, 0);            // 2^(e_max - F)
-                const double m2 = __hiloint2double(E20 + k_m2, 0);                  // 1.5 * 2^52 * 2^(E - F2)
-                const double m1 = __hiloint2double(E20 + k_m2 + k_m1, 0);           // 1.5 * 2^52 * 2^(E - F)
-                const double t2 = __dsub_rn(__fma_rd(double(T), scale_t, m2), m2);  // RD_F2
-                double sc2 = __dsub_rn(__dadd_rd(cd, m1), m1);                      // RD_F
-                if (GTR && ec20 < E20 - k_gtr) sc2 = 0.0;                           // special truncation
-                const uint32_t w = __float_as_uint(__double2float_rn(__dadd_rn(t2, sc2)));      // exact sum, then rho
-                wmax = max(wmax, w & 0x7FFFFFFFu);
-                cw[r][c] = w;
+                double st = cs[r][c];
+                // the field of Exp(c), minus one: zero wraps to the top and comes back as 0 when the one is added again (inside
+                // k_c, k_gtr); a subnormal accumulator counts as -126
+                const uint32_t ecm = __viaddmax_u32(uint32_t(__double2hiint(st) & EXPF), 0xFFFFFFFFu, LOWF - 1u);
+                if (GTR && int(ecm + k_gtr) < m0hi - HALF) st = 0.0;                // special truncation (Algorithm 11 Step 4)
+                const double Mv = __hiloint2double(__viaddmax_s32(int(ecm), int(k_c), m0hi), 0);   // 1.5 * 2^52 * qv
+                const double v = __dsub_rn(__dadd_rd(Y, __dadd_rd(st, Mv)), Mv);
+                const int vhi = __double2hiint(v);
+                const int fv = vhi & EXPF;
+                fmax = max(fmax, fv);
+                const double Mr = __hiloint2double(__viaddmax_s32(fv, (29 << 20) | HALF, int(LOWF) + ((29 << 20) | HALF)), 0);
+                const double rr = __dsub_rn(__dadd_rn(v, Mr), Mr);                  // RNE-FP32 as a double
+                cs[r][c] = __hiloint2double(__double2hiint(rr) | (vhi & int(0x80000000u)), __double2loint(rr));
             };
 
             // ---- the block in two halves of the micro-tile (rows 0, 1 and rows 2, 3): the matrix instructions of one half
@@ -251,16 +262,15 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g,
             }
 #pragma unroll
             for (int o = 8; o < 16; ++o) merge(o / TN, o % TN);
-
-            if (wmax >= 0x7F800000u) {                     // rare: RNE-FP32 overflowed: +-infinity from now on
+            if (fmax > int(HIGHF)) {                       // rare: RNE-FP32 overflowed somewhere: +-infinity from now on
 #pragma unroll
                 for (int r = 0; r < TM; ++r)
 #pragma unroll
                     for (int c = 0; c < TN; ++c)
-                        if ((cw[r][c] & 0x7FFFFFFFu) == 0x7F800000u) {
+                        if (fabs(cs[r][c]) >= 3.402823669209385e38) {
                             const uint32_t bit = 1u << (r * TN + c);
-                            if (!((sp_nan | sp_pinf | sp_ninf) & bit)) { if (cw[r][c] >> 31) sp_ninf |= bit; else sp_pinf |= bit; }
-                            cw[r][c] = 0u;
+                            if (!((sp_nan | sp_pinf | sp_ninf) & bit)) { if (cs[r][c] < 0.0) sp_ninf |= bit; else sp_pinf |= bit; }
+                            cs[r][c] = 0.0;
                         }
             }
         }
@@ -285,7 +295,8 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g,
             if (i >= g.M || j >= g.N) continue;
             const uint32_t bit = r * TN + c;
             const uint32_t spv = ((sp_nan >> bit) & 1u) | (((sp_pinf >> bit) & 1u) << 1) | (((sp_ninf >> bit) & 1u) << 2);
-            uint32_t w = spv ? special_word(((spv & 1u) || (spv & 6u) == 6u) ? 1 : ((spv & 2u) ? 2 : 3), false, false) : cw[r][c];
+            uint32_t w = spv ? special_word(((spv & 1u) || (spv & 6u) == 6u) ? 1 : ((spv & 2u) ? 2 : 3), false, false)
+                             : __float_as_uint(__double2float_rn(cs[r][c]));
             if (g.row_scale) {
                 float sc = __fmul_rn(g.row_scale[i], g.col_scale[j]);
                 if (sc != sc) sc = __uint_as_float(0x7FFFFFFFu);
