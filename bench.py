@@ -77,10 +77,14 @@ def compute_dtype(kernel: str, model) -> str:
             "efdpa": "f64", "dot_tfdpa": "f64", "dot_ftz": "f32", "ftz_addmul": "f32", "fma_f32": "f32", "fma_f64": "f64", "gstfdpa": "int32"}.get(kernel, "int64")
 
 
-# DRAM bytes per launch of the dominant kernel: dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of
-# the workload, a STORED CONSTANT, not a figure of this run.  The kernels are bound by arithmetic: this is context,
-# 0.4 % of what the memory could move in the kernel's time.
-NCU_DRAM_BYTES = {"cfg3": 101593856 + 34110464, "cfg3_2k": 25592832 + 38656}
+# DRAM bytes per step (the main kernel and the two decode launches before it): dram__bytes_read.sum +
+# dram__bytes_write.sum of a one-pass ncu capture of the same workload at its full size, a STORED CONSTANT, not a figure
+# of this run.  Algorithmic bytes are 168 MB at 4096^3 (operands once, C and D); the rest is the decoded operand blocks
+# (226 MB, larger than the L2) written once and re-read by the tiles of later waves.  The kernels are bound by arithmetic:
+# 1.18 GB in 4.2 ms is 4 % of what the memory could move in that time.
+NCU_DRAM_BYTES = {"cfg3": (980664832 + 65643264) + (16788480 + 52632832) + (16789248 + 49752576),
+                  "cfg3_2k": (74762496 + 1387776) + 4204288 + 4204800}
+NCU_ALGORITHMIC_BYTES = {"cfg3": 2 * 4096 * 4096 + 2 * 4 * 4096 * 4096, "cfg3_2k": 2 * 2048 * 2048 + 2 * 4 * 2048 * 2048}
 
 # kernels one library call launches: the tuned fused-summation kernels decode A and B into scratch blocks first
 KERNELS_PER_CALL = {"tfdpa_lut8": 3, "tfdpa_f16": 3, "tfdpa_bf16": 3, "tfdpa_tf32": 3, "trfdpa": 3, "gtrfdpa": 3, "efdpa": 3}
@@ -488,7 +492,8 @@ def run_ours(args):
                             "tensor-core product of powers, so this fraction may exceed 1 and bounds nothing")
         roofline = {"bound": "alu", **pipe_view(pipe_key, pipe_ops_per_mac, per_gpu_macs_s), "kernel": kernel_name,
                     "traffic": NCU_DRAM_BYTES.get(name),
-                    "traffic_source": "stored constant from one ncu capture of this workload (not measured in this run)" if name in NCU_DRAM_BYTES else None,
+                    "traffic_source": "stored constant from a one-pass ncu capture of this workload at full size, main kernel + both decode launches (not measured in this run)" if name in NCU_DRAM_BYTES else None,
+                    "algorithmic_bytes": NCU_ALGORITHMIC_BYTES.get(name),
                     "paper_level_integer_count": int_view}
 
     # ---- per-model leg: one model per kernel template at 4096^3, three launches each after one warm-up, L2 flushed ----
