@@ -101,7 +101,7 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g,
         // the first block's product exponents (the other blocks' are taken beside the multiply-adds of their predecessor)
         product_exponents_adj<L>(&sa_blk.exp2[0][prow], &sb_blk.exp2[0][pcol], emp);
 
-#pragma unroll 1
+#pragma unroll (L <= 8 ? 2 : 1)
         for (int blk = 0; blk < NBLK; ++blk) {
             const int kb = blk * L;
             // ---- rare: infinities / NaNs in the chunk, or products that may reach 2^128: events of this block ----
