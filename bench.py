@@ -96,7 +96,7 @@ SMS = 148
 #   FP64 fused multiply-add per term; Phi_FMA: the multiply-add itself; Phi_FTZ-AddMul: one multiply and one add per
 #   term (two FP32-pipe instructions); GST-FDPA: one 4-way byte dot product per four terms.
 FP32_KINDS = ("ffma.rm", "ffma2.rm", "ffma.rn.x16", "ffma.rn.x32", "ffma.rm.x16", "ffma2.rm.x16")
-FP64_KINDS = ("dfma", "dfma.rn.x16", "dfma.rn.x32", "dfma.rm.x16")
+FP64_KINDS = ("dfma", "dfma.rn.x16", "dfma.rn.x32", "dfma.rm.x16", "dmma.rm.k4")
 PIPES = {
     "fp32_fma": ("FP32 fused multiply-add issue", FP32_KINDS, 128.0),
     "fp64_fma": ("FP64 fused multiply-add issue", FP64_KINDS, 64.0),
