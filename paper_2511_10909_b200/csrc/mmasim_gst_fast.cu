@@ -213,10 +213,6 @@ __global__ void __launch_bounds__(NT, 2) gst_kernel(DevModel m, GemmArgs g) {
             for (int grp = 0; grp < 4; ++grp) {
                 int p[RH][TN];
 #pragma unroll
-                for (int r = 0; r < RH; ++r)
-#pragma unroll
-                    for (int c = 0; c < TN; ++c) p[r][c] = 0;
-#pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int4 a4 = *reinterpret_cast<const int4*>(&s.a[grp * 4 + j][ty * TM + rh]);
                     const int4 b4 = *reinterpret_cast<const int4*>(&s.b[grp * 4 + j][tx * TN]);
@@ -224,7 +220,7 @@ __global__ void __launch_bounds__(NT, 2) gst_kernel(DevModel m, GemmArgs g) {
 #pragma unroll
                     for (int r = 0; r < RH; ++r)
 #pragma unroll
-                        for (int c = 0; c < TN; ++c) p[r][c] = __dp4a(av[r], bv[c], p[r][c]);
+                        for (int c = 0; c < TN; ++c) p[r][c] = __dp4a(av[r], bv[c], j == 0 ? 0 : p[r][c]);
                 }
                 const uint4 sa4 = *reinterpret_cast<const uint4*>(&s.sa[grp][ty * TM + rh]);
                 const uint4 sb4 = *reinterpret_cast<const uint4*>(&s.sb[grp][tx * TN]);
