@@ -198,7 +198,7 @@ int mmasim_hw_mma(int kind, int64_t M, int64_t K, const void* A, const void* B, 
 /* The same for the B200's fifth-generation matrix instruction, tcgen05.mma (the instruction class of the paper's Blackwell
  * FP8 / FP6 / FP4 rows, Table 3's UTC*MMA entries; Section 3.2, Section 3.1 Step 4).  One instruction tile of 128 rows:
  *   D (M x 16) = A (M x K, row-major) * B^T (B is 16 x K, row-major, shared by all tiles) + C (M x 16, may be NULL = +0),
- * FP32 accumulator words, M a multiple of 128, K a multiple of the instruction's K (16 for FP16 / BF16, 8 for TF32, 32
+ * accumulator words (FP32; 16-bit FP16 words for the kinds 17-20), M a multiple of 128, K a multiple of the instruction's K (16 for FP16 / BF16, 8 for TF32, 32
  * for the 8-bit kinds); a longer K chains instructions through the accumulator in tensor memory, ascending k.  Element
  * layouts as for mmasim_gemm (TF32 in 32-bit words; FP8, FP6 and FP4 one element per byte in the low bits); all
  * pointers are device pointers.  `status` (device, 4 bytes, zeroed by the caller) receives MMASIM_ERR_TIMEOUT if the
@@ -212,7 +212,10 @@ typedef enum {
     /* block-scaled kinds: sfa (M x K/k_block bytes) and sfb (16 x K/k_block bytes), device, row-major, as for mmasim_gemm_ex */
     MMASIM_UMMA_MXE4M3 = 10, MMASIM_UMMA_MXE5M2 = 11, MMASIM_UMMA_MXE2M3 = 12, MMASIM_UMMA_MXE3M2 = 13, MMASIM_UMMA_MXE2M1 = 14,
     MMASIM_UMMA_MXF4 = 15,      /* packed FP4, E8M0 scale per 32 elements, K a multiple of 64 */
-    MMASIM_UMMA_NVF4 = 16       /* packed FP4, UE4M3 scale per 16 elements, K a multiple of 64 */
+    MMASIM_UMMA_NVF4 = 16,      /* packed FP4, UE4M3 scale per 16 elements, K a multiple of 64 */
+    /* FP16 accumulator (C and D are M x 16 16-bit words): kind::f16 with FP16 inputs, kind::f8f6f4 with E4M3 / E5M2 /
+     * E2M1 inputs - the Blackwell FP16-accumulator rows of Tables 3 and 4 (T-FDPA with rho = RNE-FP16) */
+    MMASIM_UMMA_F16_F16 = 17, MMASIM_UMMA_E4M3_F16 = 18, MMASIM_UMMA_E5M2_F16 = 19, MMASIM_UMMA_E2M1_F16 = 20
 } mmasim_umma_kind;
 int mmasim_hw_umma(int kind, int64_t M, int64_t K, const void* A, const void* B, const void* C, void* D,
                    const void* sfa, const void* sfb, int32_t* status, void* stream);

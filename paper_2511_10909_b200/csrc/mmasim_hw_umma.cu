@@ -9,6 +9,7 @@
 // mbarrier.try_wait until a clock budget runs out, then records MMASIM_ERR_TIMEOUT in the caller's status word, frees
 // the tensor memory it holds and returns.  MMASIM_UMMA_SELFTEST_TIMEOUT exercises exactly that path: nothing is issued,
 // so nobody ever arrives at the barrier.
+#include <cstdlib>
 #include "mmasim_internal.h"
 
 namespace mmasim {
@@ -20,7 +21,8 @@ constexpr int SFA_COL = 16, SFB_COL = 32, SF_GROUPS = 4;    // tensor-memory col
 enum UmmaKind : int {
     UK_F16_F32 = 0, UK_BF16_F32, UK_TF32_F32, UK_E4M3_F32, UK_E5M2_F32, UK_E4M3_E5M2_F32, UK_E2M3_F32, UK_E3M2_F32, UK_E2M1_F32,
     UK_SELFTEST_TIMEOUT,
-    UK_MXE4M3, UK_MXE5M2, UK_MXE2M3, UK_MXE3M2, UK_MXE2M1, UK_MXF4, UK_NVF4, UK_COUNT
+    UK_MXE4M3, UK_MXE5M2, UK_MXE2M3, UK_MXE3M2, UK_MXE2M1, UK_MXF4, UK_NVF4,
+    UK_F16_F16, UK_E4M3_F16, UK_E5M2_F16, UK_E2M1_F16, UK_COUNT
 };
 
 struct UmmaShape {
@@ -30,6 +32,7 @@ struct UmmaShape {
                         // 4: kind::mxf4 (packed FP4, E8M0 per 32), 5: kind::mxf4nvf4 (packed FP4, UE4M3 per 16)
     int a_fmt, b_fmt;   // format codes of the instruction descriptor
     int sf_per_step;    // scale factors per row and instruction (0: unscaled)
+    int acc16;          // 1: FP16 accumulator (C and D are 16-bit words)
 };
 
 __host__ __device__ inline UmmaShape umma_shape(int kind) {
@@ -50,14 +53,18 @@ __host__ __device__ inline UmmaShape umma_shape(int kind) {
         case UK_MXE2M1: return {1, 32, 3, 5, 5, 1};
         case UK_MXF4: return {0, 64, 4, 1, 1, 2};           // elem_bytes 0: two elements per byte
         case UK_NVF4: return {0, 64, 5, 1, 1, 4};
+        case UK_F16_F16: return {2, 16, 0, 0, 0, 0, 1};
+        case UK_E4M3_F16: return {1, 32, 2, 0, 0, 0, 1};
+        case UK_E5M2_F16: return {1, 32, 2, 1, 1, 0, 1};
+        case UK_E2M1_F16: return {1, 32, 2, 5, 5, 0, 1};
         default: return {1, 32, 2, 0, 0, 0};
     }
 }
 
-// Instruction descriptor: D format FP32 (bits 4-5 = 1), A / B formats (bits 7-9, 10-12), both operands K-major (bits 15,
+// Instruction descriptor: D format (bits 4-5: 1 FP32, 0 FP16), A / B formats (bits 7-9, 10-12), both operands K-major (bits 15,
 // 16 = 0), N / 8 in bits 17-22, M / 16 in bits 24-28.
 __host__ __device__ inline uint32_t instr_desc(const UmmaShape& s) {
-    return (1u << 4) | (uint32_t(s.a_fmt) << 7) | (uint32_t(s.b_fmt) << 10) | (uint32_t(TILE_N >> 3) << 17) | (uint32_t(TILE_M >> 4) << 24);
+    return (s.acc16 ? 0u : (1u << 4)) | (uint32_t(s.a_fmt) << 7) | (uint32_t(s.b_fmt) << 10) | (uint32_t(TILE_N >> 3) << 17) | (uint32_t(TILE_M >> 4) << 24);
 }
 // Block-scaled kinds: no D format field (the accumulator is FP32); which of the four scale bytes of a tensor-memory word
 // the instruction uses in bits 4-5 (B) and 29-30 (A); scale type in bit 23 (1: E8M0, 0: UE4M3).
@@ -129,7 +136,7 @@ __device__ __forceinline__ void issue_mma_scaled(uint32_t d_tmem, uint64_t adesc
 }
 
 __global__ void __launch_bounds__(NTHREADS) hw_umma_kernel(int kind, int64_t K, const unsigned char* A, const unsigned char* B,
-                                                          const uint32_t* C, uint32_t* D, const unsigned char* SFA,
+                                                          const void* Cv, void* Dv, const unsigned char* SFA,
                                                           const unsigned char* SFB, int32_t* status, long long wait_clocks) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) unsigned long long mbar;
@@ -162,9 +169,18 @@ __global__ void __launch_bounds__(NTHREADS) hw_umma_kernel(int kind, int64_t K, 
     const uint32_t taddr = tmem_base + (uint32_t(32 * warp) << 16);       // this warp's 32 lanes = rows 32 w .. 32 w + 31
 
     // C into tensor memory: thread (warp, lane) holds row 32 warp + lane, TILE_N columns
+    // (FP16 accumulators: 16-bit words; in tensor memory one per 32-bit column, in its low half - found with exact integers)
+    const uint32_t* C = static_cast<const uint32_t*>(Cv);
+    const uint16_t* C16 = static_cast<const uint16_t*>(Cv);
+    uint32_t* D = static_cast<uint32_t*>(Dv);
+    uint16_t* D16 = static_cast<uint16_t*>(Dv);
     uint32_t c[TILE_N];
 #pragma unroll
-    for (int j = 0; j < TILE_N; ++j) c[j] = C ? C[(row0 + 32 * warp + lane) * TILE_N + j] : 0u;
+    for (int j = 0; j < TILE_N; ++j) {
+        const int64_t idx = (row0 + 32 * warp + lane) * TILE_N + j;
+        c[j] = !Cv ? 0u : (sh.acc16 ? uint32_t(C16[idx]) : C[idx]);
+    }
+
     asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
                  :: "r"(taddr), "r"(c[0]), "r"(c[1]), "r"(c[2]), "r"(c[3]), "r"(c[4]), "r"(c[5]), "r"(c[6]), "r"(c[7]),
                     "r"(c[8]), "r"(c[9]), "r"(c[10]), "r"(c[11]), "r"(c[12]), "r"(c[13]), "r"(c[14]), "r"(c[15]) : "memory");
@@ -245,7 +261,11 @@ __global__ void __launch_bounds__(NTHREADS) hw_umma_kernel(int kind, int64_t K, 
                      : "r"(taddr) : "memory");
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-        for (int j = 0; j < TILE_N; ++j) D[(row0 + 32 * warp + lane) * TILE_N + j] = d[j];
+        for (int j = 0; j < TILE_N; ++j) {
+            const int64_t idx = (row0 + 32 * warp + lane) * TILE_N + j;
+            if (!sh.acc16) D[idx] = d[j];
+            else D16[idx] = uint16_t(d[j]);
+        }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -276,8 +296,8 @@ int launch_hw_umma(int kind, int64_t M, int64_t K, const void* A, const void* B,
         // about one second at the SM's top clock; the self-test gives up after about a millisecond
         const long long wait_clocks = kind == UK_SELFTEST_TIMEOUT ? 2000000ll : 2000000000ll;
         hw_umma_kernel<<<unsigned(M / TILE_M), NTHREADS, smem, stream>>>(kind, K, static_cast<const unsigned char*>(A),
-                                                                        static_cast<const unsigned char*>(B), static_cast<const uint32_t*>(C),
-                                                                        static_cast<uint32_t*>(D), static_cast<const unsigned char*>(sfa),
+                                                                        static_cast<const unsigned char*>(B), C, D,
+                                                                        static_cast<const unsigned char*>(sfa),
                                                                         static_cast<const unsigned char*>(sfb), status, wait_clocks);
         err = cudaGetLastError();
     }

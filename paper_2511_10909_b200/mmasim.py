@@ -360,12 +360,13 @@ def hw_mma(kind: str, A, B, C=None, out=None, *, stream=None):
 
 
 UMMA_KINDS = ["f16_f32", "bf16_f32", "tf32_f32", "e4m3_f32", "e5m2_f32", "e4m3_e5m2_f32", "e2m3_f32", "e3m2_f32", "e2m1_f32",
-              "selftest_timeout", "mxe4m3", "mxe5m2", "mxe2m3", "mxe3m2", "mxe2m1", "mxf4", "nvf4"]
+              "selftest_timeout", "mxe4m3", "mxe5m2", "mxe2m3", "mxe3m2", "mxe2m1", "mxf4", "nvf4",
+              "f16_f16", "e4m3_f16", "e5m2_f16", "e2m1_f16"]
 
 
 def hw_umma(kind: str, A, B, C=None, out=None, *, sfa=None, sfb=None, K=None, stream=None):
     """The B200's `tcgen05.mma` of the given kind on every 128-row tile of A against the 16 rows of B:
-    D (M x 16) = A (M x K) * B^T + C, CUDA tensors of raw words, FP32 accumulator.  Raises MmasimError(6) if the
+    D (M x 16) = A (M x K) * B^T + C, CUDA tensors of raw words; FP32 accumulator words, 16-bit FP16 words for the `*_f16` kinds.  Raises MmasimError(6) if the
     kernel's bounded wait for the instruction ran out (the call synchronises to read the status word)."""
     import torch
     if not A.is_cuda:
@@ -374,7 +375,7 @@ def hw_umma(kind: str, A, B, C=None, out=None, *, sfa=None, sfb=None, K=None, st
     if K is None:
         K = A.shape[1] * (2 if kind in ("mxf4", "nvf4") else 1)      # packed FP4: two elements per byte
     if out is None:
-        out = torch.empty((M, 16), dtype=torch.int32, device=A.device)
+        out = torch.empty((M, 16), dtype=torch.int16 if kind.endswith("_f16") else torch.int32, device=A.device)
     status = torch.zeros(1, dtype=torch.int32, device=A.device)
     _check(_lib.mmasim_hw_umma(UMMA_KINDS.index(kind), M, K, _ptr(A), _ptr(B), _ptr(C), _ptr(out), _ptr(sfa), _ptr(sfb),
                                _ptr(status), _stream(stream)))

@@ -150,3 +150,49 @@ def test_block_scaled_models_match_tcgen05(kind, chain, wide):
     assert bad.size == 0, (kind, K, wide, len(bad), [(tuple(x), hex(int(hw[tuple(x)])), hex(int(D[tuple(x)]))) for x in bad[:6]])
     pairs = wl.sample_pairs(M, 16, 512, seed=96)
     gu.assert_samples_equal(hw, gu.oracle_samples(key, inp, pairs), pairs, f"hardware tcgen05 {kind} K={K} against the oracle")
+
+
+# FP16 accumulators: kind -> (element format, K of one instruction)
+KINDS16 = {"f16_f16": ("fp16", 16), "e4m3_f16": ("e4m3", 32), "e5m2_f16": ("e5m2", 32), "e2m1_f16": ("e2m1", 32)}
+
+
+def _tiles16(fa, K, M):
+    if fa == "fp16":
+        return wl.hw_tiles(fa, "fp16", K, M, nb=16)
+    A, B, C32 = wl.hw_tiles8(fa, K, M, nb=16)
+    # FP16 accumulator words: the FP32 values that fit, cast; everything else an arbitrary 16-bit pattern
+    c = C32.view(np.float32)
+    with np.errstate(over="ignore", invalid="ignore"):
+        fits = np.isfinite(c) & (np.abs(c) < 6.0e4)
+        C = np.where(fits, c.astype(np.float16).view(np.uint16), (C32 >> 16).astype(np.uint16))
+    return A, B, np.ascontiguousarray(C.astype(np.uint16))
+
+
+def test_fp16_accumulator_layout_with_exact_integers():
+    _needs_b200()
+    g = wl.rng(97)
+    for kind, (fa, k) in KINDS16.items():
+        for K, M in ((k, 128), (4 * k, 256)):
+            lim = 2 if fa == "e2m1" else 3
+            a = g.integers(-lim, lim + 1, (M, K)); b = g.integers(-lim, lim + 1, (16, K)); c = g.integers(-50, 51, (M, 16))
+            D = _run(kind, wl.cast(a.astype(np.float32), fa), wl.cast(b.astype(np.float32), fa), c.astype(np.float16).view(np.uint16))
+            assert np.array_equal(D.view(np.float16).astype(np.int64), a @ b.T + c), (kind, K)
+
+
+@pytest.mark.parametrize("kind", list(KINDS16))
+@pytest.mark.parametrize("chain", [1, 3])
+def test_blackwell_fp16_accumulator_rows_match_tcgen05(kind, chain):
+    """The FP16-accumulator rows of the Blackwell column (T-FDPA with rho = RNE-FP16 after every instruction)."""
+    from paper_2511_10909_b200 import mmasim
+    _needs_b200()
+    fa, k = KINDS16[kind]
+    K, M = k * chain, 1 << 13
+    A, B, C = _tiles16(fa, K, M)
+    hw = _run(kind, A, B, C)
+    key = ("blackwell", fa, "fp16")
+    D = gu.host_words(mmasim.gemm(mmasim.Model(*key), gu.dev(A), gu.dev(B), gu.dev(C)))
+    bad = np.argwhere(hw != D)
+    assert bad.size == 0, (kind, K, len(bad), [(tuple(x), hex(int(hw[tuple(x)])), hex(int(D[tuple(x)]))) for x in bad[:6]])
+    pairs = wl.sample_pairs(M, 16, 768, seed=98)
+    want = gu.oracle_samples(key, {"A": A, "B": B, "C": C}, pairs)
+    gu.assert_samples_equal(hw, want, pairs, f"hardware tcgen05 {kind} K={K} against the oracle")
