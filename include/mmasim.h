@@ -38,7 +38,7 @@ typedef enum {
     MMASIM_ERR_SHAPE = 3,       /* M, N, K < 1, K not a multiple of the model's block, bad k_chunk or ld */
     MMASIM_ERR_ALIGN = 4,       /* pointer or leading dimension not aligned as documented */
     MMASIM_ERR_CUDA = 5,        /* a CUDA runtime call failed (message holds the CUDA error string) */
-    MMASIM_ERR_TIMEOUT = 6      /* a bounded device-side wait gave up (reported through a status word, see mmasim_hw_umma) */
+    MMASIM_ERR_TIMEOUT = 6      /* a bounded device-side wait gave up (mmasim_hw_umma's status word, mmasim_gemm_host, mmasim_copy_timeouts) */
 } mmasim_status;
 
 /* The ten architectures of Section 3.2. */
@@ -162,7 +162,8 @@ int mmasim_dot_batch(const mmasim_model* model, int64_t n, int64_t K,
  * Problems of 1024 rows and 32 MiB or more are cut into up to eight row panels of D (outputs are independent,
  * Section 3.1 Step 1): B is copied once, then each panel's rows of A and C go in, its kernel runs and its rows of D
  * come back on separate streams, so that with pinned buffers the copies run beside the arithmetic.
- * With opts->ldd > N only the N words of every row of D are written; the words between rows stay the caller's. */
+ * With opts->ldd > N only the N words of every row of D are written; the words between rows stay the caller's.
+ * Returns MMASIM_ERR_TIMEOUT if a kernel of the call gave up a bounded wait (see mmasim_copy_timeouts): D is then incomplete. */
 int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
                      const void* A, const void* B, const void* C, void* D, const mmasim_gemm_opts* opts);
 
@@ -256,6 +257,13 @@ int mmasim_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t
 
 /* Name of the kernel variant the last mmasim_gemm* call on this thread dispatched to ("generic", ...). */
 const char* mmasim_last_kernel(void);
+
+/* The tuned fused-summation kernels bring decoded operand blocks into shared memory with bulk copies and wait for each
+ * with a bounded number of polls.  A CTA whose wait runs out (never in a healthy run) stores none of its outputs and
+ * counts itself in a per-device counter; this call synchronises the current device and returns the counter's value
+ * since the library was loaded in *count (host pointer).  0 means that every output of every finished call was
+ * stored.  No counterpart in the paper. */
+int mmasim_copy_timeouts(uint64_t* count);
 
 /* Thread-local message of the last failing call on this thread ("" if none). */
 const char* mmasim_last_error(void);

@@ -82,6 +82,7 @@ int build_args(const mmasim_model* model, int64_t M, int64_t N, int64_t K, const
     g.A = A; g.B = B; g.C = C; g.D = D;
     g.lda = g.ldb = K;
     g.ldc = g.ldd = N;
+    g.copy_timeouts = copy_timeout_counter();
     if (m.k_block) g.ld_sfa = g.ld_sfb = (K + m.k_block - 1) / m.k_block;
     if (opts) {
         if (opts->lda) g.lda = opts->lda;
@@ -297,6 +298,9 @@ int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
     // panel its rows of A and C in, the kernel, its rows of D out, on three streams chained by events, so that the
     // copies of one panel run beside the arithmetic of another (two compute streams, so that a panel's last CTAs
     // share the SMs with the next panel's first).
+    // the counter of bulk-copy timeouts before the call: a kernel of this call that gives up makes it grow
+    unsigned int timeouts_before = 0u;
+    if (g.copy_timeouts) cudaMemcpy(&timeouts_before, g.copy_timeouts, sizeof(unsigned int), cudaMemcpyDeviceToHost);
     constexpr int MAX_PANELS = 16;
     int panels = 1;
     int64_t panel_rows = M;
@@ -407,6 +411,14 @@ int mmasim_gemm_host(const mmasim_model* model, int64_t M, int64_t N, int64_t K,
         set_error("mmasim_gemm_host: %s", cudaGetErrorString(err));
         return MMASIM_ERR_CUDA;
     }
+    if (st == MMASIM_OK && g.copy_timeouts) {
+        unsigned int timeouts_after = timeouts_before;
+        cudaMemcpy(&timeouts_after, g.copy_timeouts, sizeof(unsigned int), cudaMemcpyDeviceToHost);
+        if (timeouts_after != timeouts_before) {
+            set_error("mmasim_gemm_host: %u CTAs gave up waiting for a bulk copy and stored nothing", timeouts_after - timeouts_before);
+            return MMASIM_ERR_TIMEOUT;
+        }
+    }
     return st;
 }
 
@@ -470,6 +482,16 @@ int mmasim_host_release(void) {
 }
 
 const char* mmasim_last_kernel(void) { return g_kernel; }
+
+int mmasim_copy_timeouts(uint64_t* count) {
+    if (!count) { set_error("count is NULL"); return MMASIM_ERR_INVALID_ARG; }
+    unsigned int* p = copy_timeout_counter();
+    unsigned int v = 0u;
+    cudaError_t err = p ? cudaMemcpy(&v, p, sizeof(v), cudaMemcpyDeviceToHost) : cudaErrorUnknown;
+    if (err != cudaSuccess) { set_error("mmasim_copy_timeouts: %s", cudaGetErrorString(err)); return MMASIM_ERR_CUDA; }
+    *count = v;
+    return MMASIM_OK;
+}
 const char* mmasim_last_error(void) { return g_error; }
 
 }  // extern "C"

@@ -67,6 +67,7 @@ struct GemmArgs {
     const float* row_scale;
     const float* col_scale;
     int dot_mode;                 // 1: n independent dots (row t of A with row t of B), N is ignored
+    unsigned int* copy_timeouts;  // device counter of CTAs whose bounded wait on a bulk copy ran out (may be NULL)
 };
 
 }  // namespace mmasim
@@ -105,6 +106,7 @@ int launch_error_stats(int acc, int64_t n, const void* D, const double* ref, dou
 // mmasim_peak.cu
 int launch_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t* ops_per_round, cudaStream_t stream);
 // mmasim_api.cpp
+unsigned int* copy_timeout_counter();          // the current device's counter (a device variable of the library; NULL on failure)
 cudaError_t scratch_pool(cudaMemPool_t* out);   // the library's own memory pool of the current device (created on first use)
 void set_error(const char* fmt, ...);
 void set_kernel_name(const char* name);

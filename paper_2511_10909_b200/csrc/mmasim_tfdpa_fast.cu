@@ -1,5 +1,6 @@
 // Dispatch to the tuned FDPA kernels (T-, ST-, TR-, GTR- and E-FDPA; see mmasim_tfdpa_fast.cuh for what they share).
 #include "mmasim_tfdpa_fast.cuh"
+#include <mutex>
 
 namespace mmasim {
 
@@ -66,6 +67,25 @@ bool fast_tfdpa_supported(const DevModel& m, const GemmArgs& g) {
     if (g.M > 65535ll * fast::BM) return false;                             // grid.y
     if (g.N > 0x7FFFFFFFll - 128 || g.K > 0x7FFFFFFFll - 64) return false;   // 32-bit tile origins and k offsets in the kernels
     return true;
+}
+
+// The counter of bulk-copy timeouts: one word per device in a device variable of the library (nothing is allocated).
+namespace {
+__device__ unsigned int g_copy_timeouts_word = 0u;
+std::mutex g_counter_mutex;
+unsigned int* g_counter_ptr[64] = {};
+}  // namespace
+
+unsigned int* copy_timeout_counter() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_counter_mutex);
+    if (!g_counter_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_copy_timeouts_word) != cudaSuccess) return nullptr;
+        g_counter_ptr[dev] = static_cast<unsigned int*>(p);
+    }
+    return g_counter_ptr[dev];
 }
 
 int launch_gemm_noalloc(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {

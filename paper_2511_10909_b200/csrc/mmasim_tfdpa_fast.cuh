@@ -85,8 +85,8 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
     return false;
 }
 
-// Counts the CTAs whose bounded wait on a bulk copy ran out (never in a healthy run; such a CTA stores nothing).
-static __device__ unsigned int g_copy_timeouts = 0u;
+// A CTA whose bounded wait on a bulk copy ran out (never in a healthy run) stores nothing and counts itself in the
+// library's device counter (GemmArgs::copy_timeouts), which mmasim_copy_timeouts() reads.
 
 // Per element kind: returns cudaErrorInvalidValue when (L, F, rho) has no instantiation.
 cudaError_t launch_lut8(const DevModel& m, const GemmArgs& g, cudaStream_t stream);

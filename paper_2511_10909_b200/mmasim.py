@@ -320,6 +320,14 @@ def gemm_host(model: Model, A, B, C=None, *, K=None, sfa=None, sfb=None, k_chunk
     return out
 
 
+def copy_timeouts() -> int:
+    """CTAs of the tuned kernels whose bounded wait on a bulk copy ran out (they store nothing); synchronises the device."""
+    from ctypes import c_uint64
+    n = c_uint64(0)
+    _check(_lib.mmasim_copy_timeouts(byref(n)))
+    return int(n.value)
+
+
 def host_release():
     """Destroys the device memory pools that gemm_host keeps between calls."""
     _check(_lib.mmasim_host_release())
