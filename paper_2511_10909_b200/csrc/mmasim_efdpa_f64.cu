@@ -40,6 +40,7 @@ template <int EK, int L>
 __global__ void __launch_bounds__(NT, 1) efdpa64_kernel(DevModel m, GemmArgs g, const Blk64<BM>* __restrict__ wa,
                                                         const Blk64<BN>* __restrict__ wb) {
     constexpr int NBLK = KC / L;
+    constexpr bool SCALAR = L == 2;                     // (with blocks of 4 the matrix instruction wins: 12.3 against 15.4 ms at 4096^3)
     static_assert(L == 2 || L == 4, "one matrix instruction (four terms) per block");
     extern __shared__ __align__(16) unsigned char smem_raw[];
     SmemMM& sm = *reinterpret_cast<SmemMM*>(smem_raw);
@@ -90,38 +91,72 @@ __global__ void __launch_bounds__(NT, 1) efdpa64_kernel(DevModel m, GemmArgs g, 
         for (int blk = 0; blk < NBLK; ++blk) {
             const int kb = blk * L;
             uint32_t slow = chunk_special ? 0xFFFFu : 0u;   // bit r * TN + c: this output goes by the book
-            // operand fragments of the block's matrix instruction: lane (g, t) holds A[8 r + g][kb + t], B[8 j + g][kb + t];
-            // blocks of two elements leave the lanes t = 2, 3 empty
-            double af[TM], bf[TN / 2];
-            const bool lane_used = L == 4 || tq < 2;
+            if (SCALAR) {
+                // blocks of two elements would leave half of a matrix instruction empty: scalar multiply-adds, L per chain
+                double av[TM][L], bv[TN][L];
 #pragma unroll
-            for (int r = 0; r < TM; ++r) af[r] = lane_used ? sa_blk.d[wr * 32 + 8 * r + gq][kb + (L == 4 ? tq : (tq & 1))] : 0.0;
+                for (int r = 0; r < TM; ++r) {
 #pragma unroll
-            for (int j = 0; j < TN / 2; ++j) {
-                const double x = sb_blk.d[wc * 16 + 8 * j + gq][kb + (L == 4 ? tq : (tq & 1))];
-                bf[j] = lane_used ? __hiloint2double(__double2hiint(x), 0) : 0.0;
-            }
-#pragma unroll
-            for (int r = 0; r < TM; ++r)
-#pragma unroll
-                for (int j = 0; j < TN / 2; ++j) {
-                    // the accumulator as a double; adding +0 turns a -0 (which Algorithm 6 treats like +0) into +0
-                    double lo0 = __dadd_rn(double(__uint_as_float(cw[r][2 * j])), 0.0);
-                    double lo1 = __dadd_rn(double(__uint_as_float(cw[r][2 * j + 1])), 0.0);
-                    double hi0 = lo0, hi1 = lo1;
-                    asm volatile("mma.sync.aligned.m8n8k4.row.col.rm.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
-                                 : "+d"(lo0), "+d"(lo1) : "d"(af[r]), "d"(bf[j]));
-                    asm volatile("mma.sync.aligned.m8n8k4.row.col.rp.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
-                                 : "+d"(hi0), "+d"(hi1) : "d"(af[r]), "d"(bf[j]));
-                    // the same double (bit for bit: not -0 against +0, not a NaN): the exact sum
-                    // (the stand-ins of infinities and NaNs are zeros: in such a chunk the accumulator waits for the by-the-book pass)
-                    const bool fits0 = !chunk_special && lo0 == hi0 && __double2hiint(lo0) == __double2hiint(hi0);
-                    const bool fits1 = !chunk_special && lo1 == hi1 && __double2hiint(lo1) == __double2hiint(hi1);
-                    if (!fits0) slow |= 1u << (r * TN + 2 * j);
-                    if (!fits1) slow |= 1u << (r * TN + 2 * j + 1);
-                    if (fits0) cw[r][2 * j] = __float_as_uint(__double2float_rn(lo0));
-                    if (fits1) cw[r][2 * j + 1] = __float_as_uint(__double2float_rn(lo1));
+                    for (int q = 0; q < L / 2; ++q) {
+                        const double2 t = *reinterpret_cast<const double2*>(&sa_blk.d[row_at(r)][kb + 2 * q]);
+                        av[r][2 * q] = t.x; av[r][2 * q + 1] = t.y;
+                    }
                 }
+#pragma unroll
+                for (int c = 0; c < TN; ++c) {
+#pragma unroll
+                    for (int q = 0; q < L / 2; ++q) {
+                        const double2 t = *reinterpret_cast<const double2*>(&sb_blk.d[col_at(c)][kb + 2 * q]);
+                        bv[c][2 * q] = __hiloint2double(__double2hiint(t.x), 0); bv[c][2 * q + 1] = __hiloint2double(__double2hiint(t.y), 0);
+                    }
+                }
+#pragma unroll
+                for (int r = 0; r < TM; ++r)
+#pragma unroll
+                    for (int c = 0; c < TN; ++c) {
+                        // the accumulator as a double; adding +0 turns a -0 (which Algorithm 6 treats like +0) into +0
+                        const double c0 = __dadd_rn(double(__uint_as_float(cw[r][c])), 0.0);
+                        double lo = c0, hi = c0;
+#pragma unroll
+                        for (int k = 0; k < L; ++k) { lo = __fma_rd(av[r][k], bv[c][k], lo); hi = __fma_ru(av[r][k], bv[c][k], hi); }
+                        const bool fits = !chunk_special && lo == hi && __double2hiint(lo) == __double2hiint(hi);
+                        if (!fits) slow |= 1u << (r * TN + c);
+                        if (fits) cw[r][c] = __float_as_uint(__double2float_rn(lo));
+                    }
+            } else {
+                // operand fragments of the block's matrix instruction: lane (g, t) holds A[8 r + g][kb + t], B[8 j + g][kb + t];
+                // blocks of two elements leave the lanes t = 2, 3 empty
+                double af[TM], bf[TN / 2];
+                const bool lane_used = L == 4 || tq < 2;
+    #pragma unroll
+                for (int r = 0; r < TM; ++r) af[r] = lane_used ? sa_blk.d[wr * 32 + 8 * r + gq][kb + (L == 4 ? tq : (tq & 1))] : 0.0;
+    #pragma unroll
+                for (int j = 0; j < TN / 2; ++j) {
+                    const double x = sb_blk.d[wc * 16 + 8 * j + gq][kb + (L == 4 ? tq : (tq & 1))];
+                    bf[j] = lane_used ? __hiloint2double(__double2hiint(x), 0) : 0.0;
+                }
+    #pragma unroll
+                for (int r = 0; r < TM; ++r)
+    #pragma unroll
+                    for (int j = 0; j < TN / 2; ++j) {
+                        // the accumulator as a double; adding +0 turns a -0 (which Algorithm 6 treats like +0) into +0
+                        double lo0 = __dadd_rn(double(__uint_as_float(cw[r][2 * j])), 0.0);
+                        double lo1 = __dadd_rn(double(__uint_as_float(cw[r][2 * j + 1])), 0.0);
+                        double hi0 = lo0, hi1 = lo1;
+                        asm volatile("mma.sync.aligned.m8n8k4.row.col.rm.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                                     : "+d"(lo0), "+d"(lo1) : "d"(af[r]), "d"(bf[j]));
+                        asm volatile("mma.sync.aligned.m8n8k4.row.col.rp.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                                     : "+d"(hi0), "+d"(hi1) : "d"(af[r]), "d"(bf[j]));
+                        // the same double (bit for bit: not -0 against +0, not a NaN): the exact sum
+                        // (the stand-ins of infinities and NaNs are zeros: in such a chunk the accumulator waits for the by-the-book pass)
+                        const bool fits0 = !chunk_special && lo0 == hi0 && __double2hiint(lo0) == __double2hiint(hi0);
+                        const bool fits1 = !chunk_special && lo1 == hi1 && __double2hiint(lo1) == __double2hiint(hi1);
+                        if (!fits0) slow |= 1u << (r * TN + 2 * j);
+                        if (!fits1) slow |= 1u << (r * TN + 2 * j + 1);
+                        if (fits0) cw[r][2 * j] = __float_as_uint(__double2float_rn(lo0));
+                        if (fits1) cw[r][2 * j + 1] = __float_as_uint(__double2float_rn(lo1));
+                    }
+            }
             if (slow) {                                        // rare
 #pragma unroll
                 for (int r = 0; r < TM; ++r)
