@@ -252,7 +252,9 @@ int mmasim_error_stats(int acc_fmt, int64_t n, const void* D, const double* ref,
  *   27 dmma.rm.k4, 28 dmma.rm.k16   the FP64 matrix instruction rounding toward -inf (mma.sync m8n8k4 / m16n8k16),
  *                     multiply-adds counted.
  *   29 cvt.f32.f64 (FP32 -> FP64 -> FP32), 30 cvt.s32.f64 (s32 -> FP64 -> s32): conversion pairs, both counted;
- *   31 dadd.rm.x16    add.rm.f64 with 16 independent accumulators. */
+ *   31 dadd.rm.x16    add.rm.f64 with 16 independent accumulators.
+ *   32 ffma2.rm.x16+alu   kind 23 with one independent integer addition beside every packed multiply-add (the
+ *                     multiply-add lanes are counted): whether the FP32 and the integer pipe issue side by side. */
 int mmasim_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t* ops_per_round, void* stream);
 
 /* Name of the kernel variant the last mmasim_gemm* call on this thread dispatched to ("generic", ...). */

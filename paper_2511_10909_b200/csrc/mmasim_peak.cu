@@ -9,7 +9,7 @@ namespace {
 enum PeakKind : int {
     PK_IADD3 = 0, PK_LOP3, PK_SHF, PK_IMAD, PK_MACMIX, PK_VIADDMAX, PK_VIADDMAX16X2, PK_F2I, PK_FMUL, PK_POPC,
     PK_IMAD_PLUS_ALU, PK_FMUL_PLUS_ALU, PK_IMAD_WIDE, PK_MAC_D1, PK_MAC_D2, PK_DP4A, PK_DFMA, PK_DFMA_PLUS_ALU, PK_FFMA_RM, PK_FFMA2_RM,
-    PK_FFMA_RN_X16, PK_FFMA_RN_X32, PK_FFMA_RM_X16, PK_FFMA2_RM_X16, PK_DFMA_RN_X16, PK_DFMA_RN_X32, PK_DFMA_RM_X16, PK_DMMA_RM_K4, PK_DMMA_RM_K16, PK_CVT_F32_F64, PK_CVT_S32_F64, PK_DADD_RM_X16, PK_COUNT
+    PK_FFMA_RN_X16, PK_FFMA_RN_X32, PK_FFMA_RM_X16, PK_FFMA2_RM_X16, PK_DFMA_RN_X16, PK_DFMA_RN_X32, PK_DFMA_RM_X16, PK_DMMA_RM_K4, PK_DMMA_RM_K16, PK_CVT_F32_F64, PK_CVT_S32_F64, PK_DADD_RM_X16, PK_FFMA2_PLUS_ALU, PK_COUNT
 };
 
 template <int KIND>
@@ -226,6 +226,34 @@ __global__ void __launch_bounds__(256) peak_kernel_cvt(int64_t iters, int* sink)
     if (r == 0.12345) *sink = 1;
 }
 
+// Sixteen packed FP32 multiply-adds (fma.rm.f32x2, loop-invariant multiplicands) and sixteen independent 3-input integer
+// additions per round, interleaved: do the two pipes issue side by side?  Counted: the 32 multiply-add lanes per round.
+__global__ void __launch_bounds__(256) peak_kernel_ffma2_alu(int64_t iters, int* sink) {
+    unsigned long long x2[2], c2[16];
+    int y[16];
+    const float xa = 1.0f + 1e-7f * float(threadIdx.x), xb = 1.0f - 1e-7f * float(threadIdx.x + 3);
+    asm("mov.b64 %0, {%1, %1};" : "=l"(x2[0]) : "f"(xa));
+    asm("mov.b64 %0, {%1, %1};" : "=l"(x2[1]) : "f"(xb));
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { asm("mov.b64 %0, {%1, %2};" : "=l"(c2[i]) : "f"(float(i)), "f"(float(i) + 0.5f)); y[i] = int(threadIdx.x) + i; }
+    for (int64_t it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            asm volatile("fma.rm.f32x2 %0, %1, %2, %0;" : "+l"(c2[i]) : "l"(x2[0]), "l"(x2[1]));
+            asm volatile("add.s32 %0, %0, %1;" : "+r"(y[i]) : "r"(y[(i + 5) & 15]));
+        }
+    }
+    float r = 0.f;
+    int z = 0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        float lo, hi;
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(c2[i]));
+        r += lo + hi; z += y[i];
+    }
+    if (r == 0.12345f || z == 0x12345678) *sink = 1;
+}
+
 template <int MODE>
 int launch_cvt(int64_t blocks, int64_t iters, void* sink, int32_t* ops_per_round, cudaStream_t stream) {
     *ops_per_round = MODE == 2 ? 16 : 32;
@@ -314,6 +342,13 @@ int launch_int_peak(int kind, int64_t blocks, int64_t iters, void* sink, int32_t
         case PK_CVT_F32_F64: return launch_cvt<0>(blocks, iters, sink, ops_per_round, stream);
         case PK_CVT_S32_F64: return launch_cvt<1>(blocks, iters, sink, ops_per_round, stream);
         case PK_DADD_RM_X16: return launch_cvt<2>(blocks, iters, sink, ops_per_round, stream);
+        case PK_FFMA2_PLUS_ALU: {
+            *ops_per_round = 32;
+            peak_kernel_ffma2_alu<<<(unsigned)blocks, 256, 0, stream>>>(iters * 8, static_cast<int*>(sink));
+            const cudaError_t err = cudaGetLastError();
+            if (err != cudaSuccess) { set_error("int_peak launch failed: %s", cudaGetErrorString(err)); return MMASIM_ERR_CUDA; }
+            return MMASIM_OK;
+        }
         default: set_error("mmasim_int_peak: unknown kind %d", kind); return MMASIM_ERR_INVALID_ARG;
     }
 }

@@ -396,7 +396,7 @@ def hw_umma(kind: str, A, B, C=None, out=None, *, sfa=None, sfb=None, K=None, st
 PEAK_KINDS = ["iadd3", "lop3", "shf", "imad", "macmix", "viaddmax", "viaddmax16x2", "f2i", "fmul", "popc",
               "imad+alu", "fmul+alu", "imad.wide", "mac_d1", "mac_d2", "dp4a", "dfma", "dfma+alu", "ffma.rm", "ffma2.rm",
               "ffma.rn.x16", "ffma.rn.x32", "ffma.rm.x16", "ffma2.rm.x16", "dfma.rn.x16", "dfma.rn.x32", "dfma.rm.x16", "dmma.rm.k4", "dmma.rm.k16",
-              "cvt.f32.f64", "cvt.s32.f64", "dadd.rm.x16"]
+              "cvt.f32.f64", "cvt.s32.f64", "dadd.rm.x16", "ffma2.rm.x16+alu"]
 
 
 def int_peak(kind: str, blocks: int, iters: int, sink, stream=None) -> int:
