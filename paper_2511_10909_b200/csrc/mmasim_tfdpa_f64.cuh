@@ -942,11 +942,12 @@ cudaError_t launch_one64b(const DevModel& m, const GemmArgs& g, cudaStream_t str
     return err != cudaSuccess ? err : err2;
 }
 
-// The base of the tensor-core exponent maximum by element kinds: FP16 (blocks of 8 or 16) 4; 8-bit kinds 4 with an E5M2
-// operand, else 8; BF16, TF32 and blocks of 4: the add-max pass.
+// The base of the tensor-core exponent maximum by element kinds: FP16 (blocks of 16) 4; 8-bit kinds 4 with an E5M2
+// operand, else 8; BF16, TF32 and blocks of 4 and 8: the add-max pass (for blocks of 8 it is as fast, and two of them
+// are unrolled per loop trip).
 template <int EK, int L, int RHO, bool PROMOTE, bool ST = false>
 cudaError_t launch_one64(const DevModel& m, const GemmArgs& g, cudaStream_t stream) {
-    if constexpr (EK == fast::EK_F16 && L >= 8) return launch_one64b<EK, L, RHO, PROMOTE, ST, 4>(m, g, stream);
+    if constexpr (EK == fast::EK_F16 && L >= 16) return launch_one64b<EK, L, RHO, PROMOTE, ST, 4>(m, g, stream);
     else if constexpr (EK == fast::EK_LUT8 && L >= 8) {
         if (m.fmt_a == EF_E5M2 || m.fmt_b == EF_E5M2) return launch_one64b<EK, L, RHO, PROMOTE, ST, 4>(m, g, stream);
         return launch_one64b<EK, L, RHO, PROMOTE, ST, 8>(m, g, stream);
