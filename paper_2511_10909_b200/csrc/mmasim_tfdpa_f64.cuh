@@ -482,7 +482,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
     // blocks of at most 8 terms: |S| < 2^(F+1) + L * 2^(F+2) < 2^31, so the sum register's low word, started at 2^31, never
     // carries into the high word
     constexpr bool NARROW = DS && L <= 8;
-    constexpr int UNROLL_BLK = (L <= 4 || (L <= 8 && BASE == 0)) ? 2 : 1;   // short blocks: two per trip of the block loop
+    constexpr int UNROLL_BLK = (L <= 4 || (L <= 16 && BASE == 0)) ? 2 : 1;  // two blocks per trip of the block loop
     // (a zero of either sign becomes the positive state: under ST scaling the set bit of -0 could underflow away and leave
     // the +1 of a negative accumulator uncompensated)
     auto state_of = [](uint32_t w) { const double d = (w & 0x7FFFFFFFu) ? double(__uint_as_float(w)) : 0.0; return __hiloint2double(__double2hiint(d), __double2loint(d) | 1); };
