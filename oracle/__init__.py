@@ -23,6 +23,6 @@ from .ops import (  # noqa: F401
     tr_fdpa, gtr_fdpa, ieee_add_f32, ieee_mul_f32,
 )
 from .models import (  # noqa: F401
-    Model, REGISTRY, lookup, phi_dot, phi_gemm, phi_gemm_sampled, phi_dot_batch,
+    Model, REGISTRY, lookup, printed, phi_dot, phi_gemm, phi_gemm_sampled, phi_dot_batch,
     ARCHS, chunk_promote_dot,
 )

@@ -39,6 +39,7 @@ class Model:
     G: int = 0             # GST group size
     k_block: int = 0       # elements per scale factor (ST: 32; GST: 32 or 16)
     scale: str = ""        # scale-factor format
+    literal_emax: bool = False   # the maximum exponent over every term, as Algorithms 7-11 print it (not reading R2)
 
 
 def _build_registry():
@@ -108,6 +109,12 @@ def _build_registry():
 REGISTRY = _build_registry()
 
 
+def printed(m: Model) -> Model:
+    """The same registry row with the maximum exponent taken over every term, as Algorithms 7-11 print it."""
+    from dataclasses import replace
+    return replace(m, literal_emax=True)
+
+
 def lookup(arch: str, in_fmt: str, acc: str) -> Model:
     return REGISTRY[(arch, in_fmt, acc)]
 
@@ -144,17 +151,18 @@ def _fdpa_block(m: Model, a, b, d, sfa, sfb, k0, L):
     fa = fb = FORMATS[m.elem]
     fc = FORMATS[m.acc]
     if m.family == "t":
-        return ops.t_fdpa(a, b, d, fa, fb, fc, m.F, m.rho)
+        return ops.t_fdpa(a, b, d, fa, fb, fc, m.F, m.rho, literal_emax=m.literal_emax)
     if m.family == "st":
         j = k0 // m.k_block
-        return ops.st_fdpa(a, b, d, sfa[j], sfb[j], fa, fb, m.F, m.rho)
+        return ops.st_fdpa(a, b, d, sfa[j], sfb[j], fa, fb, m.F, m.rho, literal_emax=m.literal_emax)
     if m.family == "gst":
         j0, n = k0 // m.k_block, max(L // m.k_block, 1)
-        return ops.gst_fdpa(a, b, d, sfa[j0:j0 + n], sfb[j0:j0 + n], FORMATS[m.scale], m.k_block, m.G, m.F, m.rho)
+        return ops.gst_fdpa(a, b, d, sfa[j0:j0 + n], sfb[j0:j0 + n], FORMATS[m.scale], m.k_block, m.G, m.F, m.rho,
+                            literal_emax=m.literal_emax)
     if m.family == "tr":
-        return ops.tr_fdpa(a, b, d, fa, fb, m.F, m.F2, m.rho)
+        return ops.tr_fdpa(a, b, d, fa, fb, m.F, m.F2, m.rho, literal_emax=m.literal_emax)
     if m.family == "gtr":
-        return ops.gtr_fdpa(a, b, d, fa, fb, m.F, m.F2, m.rho)
+        return ops.gtr_fdpa(a, b, d, fa, fb, m.F, m.F2, m.rho, literal_emax=m.literal_emax)
     if m.family == "e":
         return ops.e_fdpa(a, b, d, fa, fb)
     raise ValueError(m.family)

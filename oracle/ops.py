@@ -132,12 +132,15 @@ _RHO_OUT = {"RZ-FP32": "fp32", "RZ-E8M13": "fp32", "RNE-FP32": "fp32", "RNE-FP16
 # Algorithm 7 (T-FDPA), Algorithm 8 (ST-FDPA)
 # ----------------------------------------------------------------------------
 def t_fdpa(a, b, c, fmt_a: Format, fmt_b: Format, fmt_c: Format, F, rho_name: str,
-           scale_exp: int = 0, scale_nan: bool = False) -> int:
+           scale_exp: int = 0, scale_nan: bool = False, literal_emax: bool = False) -> int:
     """One T-FDPA block: words a[0..L), b[0..L), accumulator word c -> output word.
 
     ``F`` is the number of fractional bits of the fused sum; ``F=None`` means
     unlimited precision (no truncation), used only by tests.  ``scale_exp`` is
-    the ST-FDPA addend Exp(alpha)+Exp(beta) (0 for plain T-FDPA).
+    the ST-FDPA addend Exp(alpha)+Exp(beta) (0 for plain T-FDPA).  ``literal_emax``
+    takes the maximum of Step 2 over every term as Algorithm 7 prints it (a zero
+    term counts with the exponent of its operands, Exp = 1 - bias for a zero)
+    instead of reading R2.
     """
     da = list(map(decoder(fmt_a), a))
     db = list(map(decoder(fmt_b), b))
@@ -151,7 +154,10 @@ def t_fdpa(a, b, c, fmt_a: Format, fmt_b: Format, fmt_c: Format, F, rho_name: st
     e = [x.exp + y.exp + scale_exp for x, y in zip(da, db)]
     # Step 2: truncated fused sum of L+1 terms
     s_c, e_c = _signed_sig(dc), dc.exp
-    live = [ek for sk, ek in zip(s, e) if sk] + ([e_c] if s_c else [])   # R2: zero terms have no exponent
+    if literal_emax:
+        live = list(e) + [e_c]
+    else:
+        live = [ek for sk, ek in zip(s, e) if sk] + ([e_c] if s_c else [])   # R2: zero terms have no exponent
     if not live:
         return rho(rho_name, 0, 0)
     e_max = max(live)
@@ -168,20 +174,20 @@ def t_fdpa(a, b, c, fmt_a: Format, fmt_b: Format, fmt_c: Format, F, rho_name: st
 
 
 def st_fdpa(a, b, c, alpha: int, beta: int, fmt_a: Format, fmt_b: Format, F: int,
-            rho_name: str) -> int:
+            rho_name: str, literal_emax: bool = False) -> int:
     """One ST-FDPA block: T-FDPA with Exp(alpha)+Exp(beta) added to every e_k (E8M0 scales)."""
     e8 = FORMATS["e8m0"]
     dal, dbe = decode(e8, alpha), decode(e8, beta)
     nan = dal.cls == NAN or dbe.cls == NAN
     return t_fdpa(a, b, c, fmt_a, fmt_b, FP32, F, rho_name,
-                  scale_exp=dal.exp + dbe.exp, scale_nan=nan)
+                  scale_exp=dal.exp + dbe.exp, scale_nan=nan, literal_emax=literal_emax)
 
 
 # ----------------------------------------------------------------------------
 # Algorithm 9 (GST-FDPA)
 # ----------------------------------------------------------------------------
 def gst_fdpa(a, b, c, alphas, betas, scale_fmt: Format, k_block: int, G: int, F: int,
-             rho_name: str) -> int:
+             rho_name: str, literal_emax: bool = False) -> int:
     """One GST-FDPA block over L = len(a) FP4 (E2M1) elements.
 
     ``alphas`` / ``betas`` hold L/k_block scale words each (reading R10).
@@ -220,6 +226,8 @@ def gst_fdpa(a, b, c, alphas, betas, scale_fmt: Format, k_block: int, G: int, F:
     scaled = [eg for g, eg in enumerate(e)
               if has_product[g] and dal[(g * G) // k_block].sig and dbe[(g * G) // k_block].sig]
     live = scaled + ([e_c] if s_c else [])
+    if literal_emax:                             # Algorithm 9 as printed: every group and the accumulator
+        live = list(e) + [e_c]
     if not live:
         return rho(rho_name, 0, 0)
     e_max = max(live)
@@ -253,7 +261,7 @@ def _products_with_overflow(da, db, frac):
 
 
 def tr_fdpa(a, b, c, fmt_a: Format, fmt_b: Format, F: int, F2: int, rho_name: str = "RNE-FP32",
-            inner_round: str = "RD") -> int:
+            inner_round: str = "RD", literal_emax: bool = False) -> int:
     """One TR-FDPA block.  ``inner_round='RZ'`` gives the paper's hypothetical symmetric variant."""
     da = list(map(decoder(fmt_a), a))
     db = list(map(decoder(fmt_b), b))
@@ -266,13 +274,13 @@ def tr_fdpa(a, b, c, fmt_a: Format, fmt_b: Format, F: int, F2: int, rho_name: st
     rnd = rd_scale if inner_round == "RD" else rz_scale
     # Step 2: truncated fused sum of the L products (c excluded)
     s_c, e_c = _signed_sig(dc), dc.exp
-    live = [ek for sk, ek in zip(s, e) if sk]                # R2: zero products have no exponent
+    live = [ek for sk, ek in zip(s, e) if sk or literal_emax]    # R2: zero products have no exponent
     if not live:                                             # T = 0: the block returns RNE(c) = c, or +0
         return rho(rho_name, s_c, e_c - FP32.mbits)
     e_max = max(live)
     T = sum(rz_scale(sk, (ek - e_max) + F - frac) for sk, ek in zip(s, e))     # units 2**(e_max - F)
     # Step 3: rounded sum of T and c at E = max(e_max, e_c)
-    E = max(e_max, e_c) if s_c else e_max
+    E = max(e_max, e_c) if (s_c or literal_emax) else e_max
     T2 = rnd(T, (e_max - E) + F2 - F)                      # RD_F2(T * 2**(e_max - E)), units 2**(E - F2)
     sc2 = rnd(s_c, (e_c - E) + F - FP32.mbits)             # RD_F(s_c * 2**(e_c - E)), units 2**(E - F)
     S = T2 + (sc2 << (F2 - F))                             # units 2**(E - F2)
@@ -280,7 +288,7 @@ def tr_fdpa(a, b, c, fmt_a: Format, fmt_b: Format, F: int, F2: int, rho_name: st
 
 
 def gtr_fdpa(a, b, c, fmt_a: Format, fmt_b: Format, F: int, F2: int,
-             rho_name: str = "RNE-FP32") -> int:
+             rho_name: str = "RNE-FP32", literal_emax: bool = False) -> int:
     """One GTR-FDPA block (even / odd index groups, rounded-down merges, special truncation of c)."""
     da = list(map(decoder(fmt_a), a))
     db = list(map(decoder(fmt_b), b))
@@ -294,7 +302,7 @@ def gtr_fdpa(a, b, c, fmt_a: Format, fmt_b: Format, F: int, F2: int,
     s_c, e_c = _signed_sig(dc), dc.exp
 
     def group(ss, ee):
-        live = [ek for sk, ek in zip(ss, ee) if sk]         # R2: zero products have no exponent
+        live = [ek for sk, ek in zip(ss, ee) if sk or literal_emax]     # R2: zero products have no exponent
         if not live:
             return 0, None
         g_max = max(live)
@@ -309,7 +317,7 @@ def gtr_fdpa(a, b, c, fmt_a: Format, fmt_b: Format, F: int, F2: int,
     T = (rd_scale(T_even, e_even - e_max) if e_even is not None else 0) + \
         (rd_scale(T_odd, e_odd - e_max) if e_odd is not None else 0)          # units 2**(e_max - F)
     # Step 4: final rounded sum with c
-    E = max(e_max, e_c) if s_c else e_max
+    E = max(e_max, e_c) if (s_c or literal_emax) else e_max
     T2 = rd_scale(T, (e_max - E) + F2 - F)
     sc2 = rd_scale(s_c, (e_c - E) + F - FP32.mbits)
     if e_c < E - F - 1:

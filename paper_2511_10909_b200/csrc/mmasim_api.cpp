@@ -59,7 +59,7 @@ int check_k(const DevModel& m, int64_t K) {
 
 int run_gemm(const mmasim_model* model, const GemmArgs& g, int flags, cudaStream_t stream) {
     const DevModel& m = model->dev;
-    if (!(flags & MMASIM_GEMM_FORCE_GENERIC)) {
+    if (!(flags & MMASIM_GEMM_FORCE_GENERIC) && !m.literal_emax) {
         if (fast_tfdpa_supported(m, g)) return launch_fast_tfdpa(m, g, stream);
         if (fast_fp_supported(m, g)) return launch_fast_fp(m, g, stream);
         if (fast_gst_supported(m, g)) return launch_fast_gst(m, g, stream);
@@ -188,6 +188,10 @@ mmasim_model* mmasim_create_model_ex(int arch, int a_fmt, int b_fmt, int acc_fmt
             if (ov->inner_round > 1 || d.family != FAM_TR) { set_error("inner_round applies to TR-FDPA models only"); return nullptr; }
             d.inner_round = ov->inner_round;
         }
+        if (ov->literal_emax > 0) {
+            if (!fdpa && d.family != FAM_GST) { set_error("literal_emax applies to T-, ST-, GST-, TR- and GTR-FDPA models only"); return nullptr; }
+            d.literal_emax = 1;
+        }
         tmp.info.l_max = d.L; tmp.info.F = d.F; tmp.info.F2 = d.F2; tmp.info.rho = d.rho; tmp.info.inner_round = d.inner_round;
     }
     mmasim_model* m = new (std::nothrow) mmasim_model(tmp);
@@ -274,7 +278,7 @@ int mmasim_dot_batch(const mmasim_model* model, int64_t n, int64_t K, const void
     g.lda = g.ldb = K;
     g.ldc = g.ldd = 1;
     g.dot_mode = 1;
-    if (dot_stream_supported(m, g)) return launch_dot_stream(m, g, static_cast<cudaStream_t>(stream));
+    if (!m.literal_emax && dot_stream_supported(m, g)) return launch_dot_stream(m, g, static_cast<cudaStream_t>(stream));
     set_kernel_name("generic_dot");
     return launch_generic(m, g, static_cast<cudaStream_t>(stream));
 }

@@ -192,10 +192,11 @@ __device__ __forceinline__ uint32_t tfdpa_block(const uint32_t* a, const uint32_
     sp.acc(dc);
     // a term whose value is zero has no exponent: it takes no part in the maximum
     constexpr int NO_EXP = -100000;
-    int e_max = dc.sig ? dc.exp : NO_EXP;
+    // (m.literal_emax: every term takes part, as Algorithm 7 prints it)
+    int e_max = (dc.sig || m.literal_emax) ? dc.exp : NO_EXP;
     for (int k = 0; k < L; ++k) {                                   // Step 1 exponents, Step 2 maximum
         sp.product(a[k], b[k]);
-        const int ek = (dec_sig(a[k]) && dec_sig(b[k])) ? dec_exp(a[k]) + dec_exp(b[k]) + scale_exp : NO_EXP;
+        const int ek = ((dec_sig(a[k]) && dec_sig(b[k])) || m.literal_emax) ? dec_exp(a[k]) + dec_exp(b[k]) + scale_exp : NO_EXP;
         e_max = ek > e_max ? ek : e_max;
     }
     const int kind = sp.result();
@@ -231,7 +232,7 @@ __device__ __forceinline__ uint32_t gst_block(const uint32_t* a, const uint32_t*
     int64_t s[4];
     int e[4];
     constexpr int NO_EXP = -100000;                                 // a zero accumulator takes no part in the maximum
-    int e_max = dc.sig ? dc.exp : NO_EXP;
+    int e_max = (dc.sig || m.literal_emax) ? dc.exp : NO_EXP;
     for (int g = 0; g < ng; ++g) {                                  // Step 1
         int p = 0;                                                  // units of 2^-2 (E2M1: Exp >= 0, 1 mantissa bit)
         bool has_product = false;                                   // some a_k * b_k of the group is nonzero
@@ -243,7 +244,7 @@ __device__ __forceinline__ uint32_t gst_block(const uint32_t* a, const uint32_t*
         s[g] = int64_t(p) * int64_t(dec_sig(sfa[j])) * int64_t(dec_sig(sfb[j]));
         e[g] = dec_exp(sfa[j]) + dec_exp(sfb[j]);
         // a group of zero products, or under a zero scale factor, has no exponent; one whose products cancel has
-        if (has_product && dec_sig(sfa[j]) && dec_sig(sfb[j])) e_max = e[g] > e_max ? e[g] : e_max;
+        if ((has_product && dec_sig(sfa[j]) && dec_sig(sfb[j])) || m.literal_emax) e_max = e[g] > e_max ? e[g] : e_max;
     }
     if (e_max == NO_EXP) return 0u;
     int64_t S = 0;
@@ -277,7 +278,7 @@ __device__ __forceinline__ uint32_t tr_block(const uint32_t* a, const uint32_t* 
             const int ek = dec_exp(a[k]) + dec_exp(b[k]);
             if (product_overflows(sk, ek, m.frac)) sp.add_inf(sk < 0);
             const int g = grouped ? (k & 1) : 0;
-            if (sk != 0) e_grp[g] = ek > e_grp[g] ? ek : e_grp[g];  // zero products take no part in the maximum
+            if (sk != 0 || m.literal_emax) e_grp[g] = ek > e_grp[g] ? ek : e_grp[g];  // zero products take no part in the maximum (unless as printed)
         }
     }
     const int kind = sp.result();
@@ -301,7 +302,7 @@ __device__ __forceinline__ uint32_t tr_block(const uint32_t* a, const uint32_t* 
     }
     const int64_t sc = dc.sign ? -int64_t(dc.sig) : int64_t(dc.sig);
     if (e_max == -100000) return rho_apply(m.rho, sc, dc.exp - 23);  // every product is zero: the block returns c (or +0)
-    const int E = (dc.sig && dc.exp > e_max) ? dc.exp : e_max;
+    const int E = ((dc.sig || m.literal_emax) && dc.exp > e_max) ? dc.exp : e_max;
     int64_t T2, sc2;
     if (m.inner_round == 1) {                                       // hypothetical RZ variant (Section 6.2.4)
         T2 = rz_scale(T, (e_max - E) + F2 - F);

@@ -280,7 +280,7 @@ __global__ void __launch_bounds__(NT, 2) gst_kernel(DevModel m, GemmArgs g) {
 }  // namespace
 
 bool fast_gst_supported(const DevModel& m, const GemmArgs& g) {
-    if (m.family != FAM_GST || g.dot_mode || g.k_chunk || g.row_scale) return false;
+    if (m.family != FAM_GST || g.dot_mode || g.k_chunk || g.row_scale || m.literal_emax) return false;
     if (m.L != 64 || m.G != 16 || m.F != 35 || m.rho != RHO_RZ_FP32 || !m.packed4) return false;
     if (g.K % KC) return false;
     if ((g.lda % 32) || (g.ldb % 32)) return false;                 // 16-byte row starts (two elements per byte)

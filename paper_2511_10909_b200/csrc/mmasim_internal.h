@@ -50,6 +50,7 @@ struct DevModel {
     int frac;             // fractional bits of a product term (mbits_a + mbits_b; GST: 2 + 2 * scale mbits)
     int inner_round;      // 0: paper; 1: TR second stage in RZ
     int packed4;          // A and B hold two FP4 codes per byte
+    int literal_emax;     // 1: the maximum exponent over every term, as Algorithms 7-11 print it (generic kernels only)
 };
 
 // Per-call arguments common to the GEMM-shaped kernels.

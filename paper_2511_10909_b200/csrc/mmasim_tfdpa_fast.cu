@@ -58,7 +58,7 @@ int kind_of(const DevModel& m) {
 
 bool fast_tfdpa_supported(const DevModel& m, const GemmArgs& g) {
     const int kind = kind_of(m);
-    if (!kind || g.dot_mode) return false;
+    if (!kind || g.dot_mode || m.literal_emax) return false;
     const int bytes = fmt_desc(m.fmt_a).storage_bits / 8;
     if (g.K % fast::KC) return false;
     if (g.k_chunk % fast::KC) return false;

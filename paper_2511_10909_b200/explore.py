@@ -110,3 +110,12 @@ def _stats(acc: str, D, ref) -> dict:
     n = max(s[0], 1.0)
     return {"count": int(s[0]), "mean": s[1] / n, "mean_abs": s[2] / n, "rms": (s[3] / n) ** 0.5, "negative": s[4] / n,
             "positive": s[5] / n, "max_abs": s[6], "mean_rel": s[7] / n}
+
+
+def printed_form_difference(arch: str, in_fmt: str, acc: str, A, B, C=None, **kw) -> dict:
+    """On how many outputs does the registry row change when the maximum exponent of the fused sum runs over every term,
+    as Algorithms 7-11 print it, instead of over the nonzero terms (what the B200's own rows do)?  Runs the row and its
+    `literal_emax` override on the same inputs; returns the count, the number of outputs and both results."""
+    row = mmasim.gemm(mmasim.Model(arch, in_fmt, acc), A, B, C, **kw)
+    lit = mmasim.gemm(mmasim.Model(arch, in_fmt, acc, literal_emax=1), A, B, C, **kw)
+    return {"differing": int((row != lit).sum()), "outputs": row.numel(), "row": row, "printed": lit}

@@ -35,7 +35,7 @@ class _Info(Structure):
 
 
 class _Overrides(Structure):
-    _fields_ = [(n, c_int32) for n in ("l_max", "F", "F2", "rho", "inner_round")]
+    _fields_ = [(n, c_int32) for n in ("l_max", "F", "F2", "rho", "inner_round", "literal_emax")]
 
 
 class _GemmOpts(Structure):
@@ -108,7 +108,7 @@ class Model:
         self.arch, self.in_fmt, self.acc, self.b_fmt = arch, in_fmt, acc, b_fmt or in_fmt
         ov = None
         if overrides:
-            vals = {k: -1 for k in ("l_max", "F", "F2", "rho", "inner_round")}
+            vals = {k: -1 for k in ("l_max", "F", "F2", "rho", "inner_round", "literal_emax")}
             for k, v in overrides.items():
                 if k not in vals:
                     raise TypeError(f"unknown override {k}")

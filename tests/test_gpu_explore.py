@@ -75,3 +75,43 @@ def test_fp8_through_the_fp16_instruction():
     assert r["native"]["mean_abs"] > 100 * r["via_fp16"]["mean_abs"]
     w = explore.widen_fp8_to_fp16("e4m3", gu.dev(A)).cpu().numpy().view(np.float16).astype(np.float64)
     np.testing.assert_array_equal(w, torch.from_numpy(A).view(torch.float8_e4m3fn).double().numpy())
+
+
+@pytest.mark.parametrize("key", [("ampere", "fp16", "fp32"), ("blackwell", "mxe4m3", "fp32"), ("blackwell", "nvf4", "fp32"),
+                                 ("cdna3", "bf16", "fp32"), ("cdna3", "e4m3", "fp32")], ids=lambda k: "-".join(k))
+def test_printed_form_override_matches_the_oracle_and_differs_on_zero_heavy_inputs(key):
+    """The `literal_emax` override (maximum exponent over every term, as Algorithms 7-11 print it) against the oracle's
+    printed form on inputs with many zero elements and zero or tiny accumulators; the row itself (reading R2, decided by
+    the B200) differs from it on some of these outputs, and not at all on inputs without zeros."""
+    import oracle
+    from paper_2511_10909_b200 import explore, mmasim
+    g = wl.rng(77)
+    M, N, K = 96, 64, 128
+    inp = wl.normal_inputs(key[1], key[2], M, N, K, seed=78)
+    A, B = inp["A"].copy(), inp["B"].copy()
+    packed = key[1] in ("mxf4", "nvf4")
+    zero = g.random(A.shape) < (0.35 if packed else 0.6)
+    A[zero] = 0
+    A[::3] = 0                                               # whole rows of zeros: blocks without any nonzero product
+    # small values beside the zeros, so that a zero term's exponent can exceed every nonzero product's
+    if not packed and A.dtype.itemsize == 2:
+        A[~zero] = wl.cast((g.standard_normal(A.shape) * 2.0 ** -12).astype(np.float32), key[1])[~zero]
+    C = (g.standard_normal((M, N)) * 2.0 ** g.integers(-60, -20, (M, N))).astype(np.float32).view(np.uint32)
+    C[g.random((M, N)) < 0.5] = 0
+    kw = {k: gu.dev(inp[k]) for k in ("sfa", "sfb") if k in inp}
+    r = explore.printed_form_difference(*key, gu.dev(A), gu.dev(B), gu.dev(C), **kw)
+    assert mmasim.last_kernel() == "generic"
+    lit = gu.host_words(r["printed"])
+    pairs = wl.sample_pairs(M, N, 500, seed=79)
+    Au, Bu = (gu.unpack_fp4(A), gu.unpack_fp4(B)) if packed else (A, B)
+    want = oracle.phi_gemm_sampled(oracle.printed(oracle.lookup(*key)), Au, Bu, C, pairs, SFA=inp.get("sfa"), SFB=inp.get("sfb"))
+    gu.assert_samples_equal(lit, want, pairs, f"printed form of {key}")
+    if oracle.lookup(*key).family in ("t", "st", "gst"):     # (a block of zero products keeps a tiny accumulator under R2 and
+        assert r["differing"] > 0, key                       # truncates it away when the zero products count)
+    dense = wl.normal_inputs(key[1], key[2], M, N, K, seed=80)
+    if not packed:                                           # no zero elements, nonzero accumulators: nothing changes
+        kw = {k: gu.dev(dense[k]) for k in ("sfa", "sfb") if k in dense}
+        r2 = explore.printed_form_difference(*key, gu.dev(dense["A"]), gu.dev(dense["B"]), gu.dev(dense["C"]), **kw)
+        zeros_in = int((dense["A"].astype(np.int64) << 1 == 0).sum() + (dense["B"].astype(np.int64) << 1 == 0).sum())
+        if zeros_in == 0:
+            assert r2["differing"] == 0, key

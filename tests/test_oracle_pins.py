@@ -1173,3 +1173,43 @@ def test_gst_group_with_a_zero_scale_factor_has_no_exponent():
     # the same call with a nonzero (tiny) scale in place of the zero one: the group counts, e_max = 7 - 6 = 1 at least
     sfb2 = [0x01, one, one, one]         # 2^-9: the group's value 36 * 2^7 * 2^-9 = 9, e_g = 7 + (-6) = 1
     assert phi_dot(m, a, b, f32_word(-1.5 * 2.0 ** -35), sfa, sfb2) == f32_word(10.0)
+
+
+def test_printed_form_of_the_maximum_exponent_is_reachable_and_differs_only_on_zero_terms():
+    """Algorithms 7-11 print the maximum over every term; reading R2 (decided by the B200) leaves zero terms out.  The
+    printed form is an option of the oracle (and an override of the library): on the inputs that separate the two it gives
+    the value the printed algorithm gives by hand, and without zero terms both forms agree."""
+    from oracle import printed
+    m = lookup("hopper", "fp16", "fp32")
+    h = lambda x: exact_word("fp16", x)
+    a = [h(0.0), h(2.0 ** -14)] + [0] * 14
+    b = [h(2.0 ** 15), h(1.5 * 2.0 ** -14)] + [0] * 14
+    # printed: the zero product counts with Exp(0) + Exp(2^15) = -14 + 15 = 1, the grid is 2^(1 - 25), and 1.5 * 2^-28 is
+    # truncated away; R2: it survives
+    assert word_f32(phi_dot(printed(m), a, b, 0)) == 0.0
+    assert word_f32(phi_dot(m, a, b, 0)) == 1.5 * 2.0 ** -28
+    # a zero accumulator counts with Exp = -126 in the printed form: no effect here (every product exponent is larger) ...
+    assert phi_dot(printed(m), [h(3.0)] * 16, [h(0.5)] * 16, 0) == phi_dot(m, [h(3.0)] * 16, [h(0.5)] * 16, 0)
+    # TR-FDPA (Algorithm 10): a zero accumulator counted with Exp = -126 makes E = -126, and T is rounded down onto
+    # 2^(-126 - 31) before the final rounding.  One product 145/128 * 2^-100 times 226/128 * 2^-51 = 2^-150 (1 + 2^-14):
+    # exactly (R2: E = e_max) it lies above the tie between 0 and 2^-149 and rounds to 2^-149; rounded down onto 2^-157
+    # first it is the tie itself, which RNE sends to the even neighbour 0
+    hb = lambda x: exact_word("bf16", x)
+    mt = lookup("cdna3", "bf16", "fp32")
+    at = [hb(145 / 128 * 2.0 ** -100)] + [0] * 7
+    bt = [hb(226 / 128 * 2.0 ** -51)] + [0] * 7
+    assert phi_dot(mt, at, bt, 0) == 0x00000001
+    assert phi_dot(printed(mt), at, bt, 0) == 0x00000000
+    # random inputs without zeros: both forms agree (the option changes nothing but the treatment of zero terms)
+    rng = random.Random(31)
+    for key in (("ampere", "fp16", "fp32"), ("blackwell", "e4m3", "fp32"), ("cdna3", "fp16", "fp32"), ("cdna3", "e5m2", "fp32")):
+        mm = lookup(*key)
+        fmt = FORMATS[mm.elem]
+        for _ in range(100):
+            av, bv = [], []
+            while len(av) < mm.L:
+                x, y = _rand_finite(rng, fmt), _rand_finite(rng, fmt)
+                if (x & ((1 << (fmt.ebits + fmt.mbits)) - 1)) and (y & ((1 << (fmt.ebits + fmt.mbits)) - 1)):
+                    av.append(x); bv.append(y)
+            c = f32_word(rng.gauss(0.0, 1.0))
+            assert phi_dot(mm, av, bv, c) == phi_dot(printed(mm), av, bv, c), key
