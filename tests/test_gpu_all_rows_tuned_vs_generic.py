@@ -1,0 +1,74 @@
+"""Every registry row on seeded random shapes: the kernel the dispatcher picks against the generic kernels on every output
+word, and against the oracle on sampled outputs.  Two inputs per row: N(0,1) values in the row's format (with zero
+elements and zero accumulators mixed in), and raw random bit patterns for A, B, C and the scale factors (NaN, infinity,
+subnormals, any exponent spread).  Shapes are ragged against every tile size; K is a multiple of the row's block."""
+import zlib
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2511_10909_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+gu = pytest.importorskip("gpu_util") if torch.cuda.is_available() else None
+
+
+def _keys():
+    if not torch.cuda.is_available():
+        return []
+    from paper_2511_10909_b200 import mmasim
+    return list(mmasim.model_keys())
+
+
+def _word_dtype(nbytes):
+    return {1: np.uint8, 2: np.uint16, 4: np.uint32, 8: np.uint64}[nbytes]
+
+
+@pytest.mark.parametrize("key", _keys(), ids=lambda k: "-".join(k))
+def test_row_on_random_shapes(key):
+    from paper_2511_10909_b200 import mmasim
+    g = wl.rng(zlib.crc32("-".join(key).encode()))
+    model = mmasim.Model(*key)
+    kmul = 64 if key[1] in ("mxf4", "nvf4") else 32
+    M, N, K = int(g.integers(1, 300)), int(g.integers(1, 200)), kmul * int(g.integers(1, 6))
+    # ---- ordinary values with zeros mixed in ----
+    inp = wl.normal_inputs(key[1], key[2], M, N, K, seed=int(g.integers(1, 1 << 30)))
+    A, B, C = inp["A"].copy(), inp["B"].copy(), inp["C"].copy()
+    A[g.random(A.shape) < 0.1] = 0
+    B[g.random(B.shape) < 0.05] = 0
+    C[g.random(C.shape) < 0.2] = 0
+    inp.update(A=A, B=B, C=C)
+    D = gu.run_gemm(key, inp)
+    kernel = mmasim.last_kernel()
+    G = gu.run_gemm(key, inp, force_generic=True)
+    assert mmasim.last_kernel() == "generic"
+    bad = np.argwhere(D != G)
+    assert bad.size == 0, (key, kernel, (M, N, K), len(bad), bad[:4])
+    pairs = wl.sample_pairs(M, N, 64, seed=M * 1000 + N)
+    gu.assert_samples_equal(D, gu.oracle_samples(key, inp, pairs), pairs, f"{key} {kernel} {(M, N, K)}")
+    # ---- raw bit patterns ----
+    wild = {"A": g.integers(0, 256, A.shape, dtype=np.uint8) if A.dtype.itemsize == 1
+            else g.integers(0, 1 << (8 * A.dtype.itemsize - 1), A.shape, dtype=np.uint64).astype(_word_dtype(A.dtype.itemsize)) * 2
+            + g.integers(0, 2, A.shape).astype(_word_dtype(A.dtype.itemsize))}
+    wild["B"] = (g.integers(0, 256, B.shape, dtype=np.uint8) if B.dtype.itemsize == 1
+                 else g.integers(0, 1 << (8 * B.dtype.itemsize - 1), B.shape, dtype=np.uint64).astype(_word_dtype(B.dtype.itemsize)) * 2
+                 + g.integers(0, 2, B.shape).astype(_word_dtype(B.dtype.itemsize)))
+    wild["C"] = (g.integers(0, 1 << (8 * C.dtype.itemsize - 1), C.shape, dtype=np.uint64).astype(_word_dtype(C.dtype.itemsize)) * 2
+                 + g.integers(0, 2, C.shape).astype(_word_dtype(C.dtype.itemsize)))
+    if key[1] not in ("mxf4", "nvf4") and A.dtype.itemsize == 1:
+        # one element per byte in the low bits: keep the codes inside the format's width
+        bits = model.a_bits if model.a_bits < 8 else 8
+        width = {"e4m3": 8, "e5m2": 8, "e3m2": 6, "e2m3": 6, "e2m1": 4}.get(key[1].replace("mx", ""), bits)
+        wild["A"] &= np.uint8((1 << width) - 1)
+        wild["B"] &= np.uint8((1 << width) - 1)
+    if "sfa" in inp:
+        wild["sfa"] = g.integers(0, 256, inp["sfa"].shape, dtype=np.uint8)
+        wild["sfb"] = g.integers(0, 256, inp["sfb"].shape, dtype=np.uint8)
+    D = gu.run_gemm(key, wild)
+    kernel = mmasim.last_kernel()
+    G = gu.run_gemm(key, wild, force_generic=True)
+    bad = np.argwhere(D != G)
+    assert bad.size == 0, (key, kernel, (M, N, K), "bit patterns", len(bad), bad[:4])
+    gu.assert_samples_equal(D, gu.oracle_samples(key, wild, pairs), pairs, f"{key} {kernel} {(M, N, K)} bit patterns")
