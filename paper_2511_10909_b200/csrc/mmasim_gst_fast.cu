@@ -178,7 +178,7 @@ __global__ void __launch_bounds__(NT, 2) gst_kernel(DevModel m, GemmArgs g) {
 #pragma unroll
                     for (int r = 0; r < RH; ++r)
 #pragma unroll
-                        for (int c = 0; c < TN; ++c) key[r][c] = max(key[r][c], int(sav[r] + sbv[c]));
+                        for (int c = 0; c < TN; ++c) key[r][c] = __viaddmax_s32(int(sav[r]), int(sbv[c]), key[r][c]);
                 } else {
                     const uint4 fa4 = *reinterpret_cast<const uint4*>(&s.fa[grp >> 1][ty * TM + rh]);
                     const uint4 fb4 = *reinterpret_cast<const uint4*>(&s.fb[grp >> 1][tx * TN]);
@@ -220,19 +220,26 @@ __global__ void __launch_bounds__(NT, 2) gst_kernel(DevModel m, GemmArgs g) {
 #pragma unroll
                     for (int r = 0; r < RH; ++r)
 #pragma unroll
-                        for (int c = 0; c < TN; ++c) p[r][c] = __dp4a(av[r], bv[c], j == 0 ? 0 : p[r][c]);
+                        for (int c = 0; c < TN; ++c) p[r][c] = __dp4a(av[r], bv[c], j == 0 ? (NVF4 ? 0 : int(0x80000000u)) : p[r][c]);
                 }
                 const uint4 sa4 = *reinterpret_cast<const uint4*>(&s.sa[grp][ty * TM + rh]);
                 const uint4 sb4 = *reinterpret_cast<const uint4*>(&s.sb[grp][tx * TN]);
                 const uint32_t sag[RH] = {sa4.x, sa4.y, sa4.z, sa4.w}, sbg[TN] = {sb4.x, sb4.y, sb4.z, sb4.w};
+                int ea20[RH], eb20[TN];             // exponent fields: their sum is the high word of 2^(e_g - frac)
+#pragma unroll
+                for (int r = 0; r < RH; ++r) ea20[r] = int(sag[r] & uint32_t(EXPF)) - (FRAC << 20);
+#pragma unroll
+                for (int c = 0; c < TN; ++c) eb20[c] = int(sbg[c] & uint32_t(EXPF));
 #pragma unroll
                 for (int r = 0; r < RH; ++r)
 #pragma unroll
                     for (int c = 0; c < TN; ++c) {
-                        int sg = p[r][c];
-                        if (NVF4) sg = sg * int(sag[r] & 0xFFu) * int(sbg[c] & 0xFFu);
-                        const double gd = __dsub_rn(__hiloint2double(0x43300000, sg ^ int(0x80000000u)), two52_31);
-                        const double sc = __hiloint2double(int((sag[r] + sbg[c]) & uint32_t(EXPF)) - (FRAC << 20), 0);   // 2^(e_g - frac)
+                        // (MXFP4: the dot product was started at 2^31, which is the form the conversion below wants)
+                        int sgx = p[r][c];                                          // s_g ^ 2^31
+                        if (NVF4) sgx = (sgx * int(sag[r] & 0xFFu) * int(sbg[c] & 0xFFu)) ^ int(0x80000000u);
+                        const int sg = ~sgx;                                        // its sign bit is that of s_g
+                        const double gd = __dsub_rn(__hiloint2double(0x43300000, sgx), two52_31);
+                        const double sc = __hiloint2double(ea20[r] + eb20[c], 0);                       // 2^(e_g - frac)
                         const double Ms = __hiloint2double(mhi[r][c] | (sg & int(0x80000000u)), 0);
                         S[r][c] = __dsub_rn(__dadd_rn(S[r][c], __fma_rz(gd, sc, Ms)), Ms);
                     }
