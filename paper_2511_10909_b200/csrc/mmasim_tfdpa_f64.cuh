@@ -398,10 +398,24 @@ __device__ __forceinline__ void product_exponents(const uint32_t* ea_p, const ui
 
 // Multipliers read from the constant bank, so that the compiler keeps integer multiply-adds (which issue beside the
 // integer pipe) instead of rewriting them as shifts and additions on it.
-static __constant__ int c_mul64[4] = {1 << 20, 16, 1, 0};
+static __constant__ int c_mul64[8] = {1 << 20, 16, 1, 0, 1 << 21, 32, 2, int(0x80000000u)};
 __device__ __forceinline__ int imad(int a, int b, int c) {
     int d;
     asm("mad.lo.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+// max(|a|, b, c) of three words read as FP32 numbers, in one instruction (the absolute value is an operand modifier).
+// For nonnegative words the order of FP32 numbers is the order of the integers; a negative b or c reads as a negative
+// number or a NaN and loses either way (the maximum of a NaN and a number is the number).
+__device__ __forceinline__ int fmax3_abs(int a, int b, int c) {
+    float d;
+    asm("{ .reg .f32 t; abs.f32 t, %1; max.f32 %0, t, %2, %3; }" : "=f"(d) : "f"(__int_as_float(a)), "f"(__int_as_float(b)), "f"(__int_as_float(c)));
+    return __float_as_int(d);
+}
+// high word of a * b, plus c: with b = 2^31 a logical shift right by one, with b = 2 the top bit of a
+__device__ __forceinline__ uint32_t imad_hi(uint32_t a, int b, uint32_t c) {
+    uint32_t d;
+    asm("mad.hi.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
     return d;
 }
 
@@ -483,6 +497,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
     // carries into the high word
     constexpr bool NARROW = DS && L <= 8;
     constexpr int UNROLL_BLK = (L <= 4 || (L <= 16 && BASE == 0)) ? 2 : 1;  // two blocks per trip of the block loop
+    constexpr bool K2 = DS && BASE == 0 && !ST;          // keys and range check on doubled high words (see start)
     // (a zero of either sign becomes the positive state: under ST scaling the set bit of -0 could underflow away and leave
     // the +1 of a negative accumulator uncompensated)
     auto state_of = [](uint32_t w) { const double d = (w & 0x7FFFFFFFu) ? double(__uint_as_float(w)) : 0.0; return __hiloint2double(__double2hiint(d), __double2loint(d) | 1); };
@@ -663,7 +678,8 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                         // the two 16-bit lanes (Exp + CB of the even and the odd elements) moved to the exponent field by
                         // multiplications, which run beside the integer pipe
                         const int klo = imad(int(e2), c_mul64[0], -(1 << 20)), khi = imad(int(e2), c_mul64[1], -(1 << 20));
-                        m = __vimax3_s32(klo, khi, ST ? max(keyc, 0) : keyc);
+                        if (ST) m = __vimax3_s32(klo, khi, max(keyc, 0));
+                        else m = fmax3_abs(subnormal_c ? keyc : hi, klo, khi);
                     }
                     const int e20 = m & 0x7FF00000;
                     // the +1 of a negative c sits in the constant's low word: one unit of the grid either way.  Short blocks:
@@ -746,7 +762,8 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
             auto finish = [&](int r, int c) {
                 const double v = block_value(r, c);
                 if (DS) {
-                    urange = __viaddmax_u32(uint32_t(__double2hiint(v)) & 0x7FFFFFFFu, 0u - LOWHI, urange);
+                    if (K2) urange = max(uint32_t(imad(__double2hiint(v), c_mul64[6], int(0u - 2u * LOWHI))), urange);
+                    else urange = __viaddmax_u32(uint32_t(__double2hiint(v)) & 0x7FFFFFFFu, 0u - LOWHI, urange);
                     // RZ-FP32 of a number in the normal range: the low 29 bits of the double's significand go
                     const double st = __hiloint2double(__double2hiint(v), (__double2loint(v) & int(0xE0000000u)) | 1);
                     if (BASE) nv[BASE ? r : 0][BASE ? c : 0] = st; else cs[DS ? r : 0][DS ? c : 0] = st;
@@ -799,7 +816,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
             for (int o = 8; o < 16; ++o) finish(o / TN, o % TN);
 
             if (DS) {
-                bool odd = urange >= SPANHI;            // some result is not a normal FP32 number
+                bool odd = urange >= (K2 ? 2u * SPANHI : SPANHI);   // some result is not a normal FP32 number
                 if (BASE && no_product) {               // rare: no nonzero product: the block returns its accumulator
                     odd = true;
 #pragma unroll
