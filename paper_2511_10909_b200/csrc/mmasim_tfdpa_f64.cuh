@@ -250,7 +250,9 @@ struct Blk64 {
     uint32_t exp2[KC / 2][R];
     uint16_t pe[R][PE_STRIDE64];
     uint32_t sgn[R], nz[R];
-    uint32_t special, pad[3];
+    uint32_t special;               // the block holds an infinity or a NaN
+    uint32_t max_exp;               // the largest Exp(x) + EB of the block's elements (0: all zero)
+    uint32_t pad[2];
 };
 static_assert(sizeof(Blk64<BM>) % 16 == 0 && sizeof(Blk64<BN>) % 16 == 0, "bulk copies move multiples of 16 bytes");
 
@@ -292,10 +294,10 @@ __global__ void __launch_bounds__(256) decode64_kernel(DevModel m, const unsigne
         e.bits = (fin ? dec_sign(dd) : 0u) | (fin ? 0u : 2u) | (sg ? 4u : 0u);
         lut[tid] = e;
     }
-    if (tid == 0) { blk.special = 0u; blk.pad[0] = blk.pad[1] = blk.pad[2] = 0u; }
+    if (tid == 0) { blk.special = 0u; blk.max_exp = 0u; blk.pad[0] = blk.pad[1] = 0u; }
     __syncthreads();
     const int64_t k0 = int64_t(blockIdx.x) * KC;
-    uint32_t spec = 0u;
+    uint32_t spec = 0u, top_exp = 0u;
     for (int task = tid; task < TASKS; task += 256) {
         const int r = task % R, h = task / R;
         const int pr = IS_A ? perm_row64(r) : perm_col64(r);
@@ -353,6 +355,7 @@ __global__ void __launch_bounds__(256) decode64_kernel(DevModel m, const unsigne
                 pw[q / 2] |= pe << 16;
             } else pw[q / 2] = pe;
             prev_exp = expb;
+            top_exp = max(top_exp, expb);
         }
 #pragma unroll
         for (int q = 0; q < E::TASK / 8; ++q)
@@ -364,6 +367,8 @@ __global__ void __launch_bounds__(256) decode64_kernel(DevModel m, const unsigne
         }
     }
     if (spec) atomicOr(&blk.special, 1u);
+    top_exp = __reduce_max_sync(0xFFFFFFFFu, top_exp);
+    if ((tid & 31) == 0 && top_exp) atomicMax(&blk.max_exp, top_exp);
     __syncthreads();
     uint4* out = reinterpret_cast<uint4*>(dst + (int64_t(blockIdx.y) * gridDim.x + blockIdx.x));
     const uint4* in = reinterpret_cast<const uint4*>(&blk);
@@ -497,6 +502,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
     // carries into the high word
     constexpr bool NARROW = DS && L <= 8;
     constexpr int UNROLL_BLK = (L <= 4 || (L <= 16 && BASE == 0)) ? 2 : 1;  // two blocks per trip of the block loop
+    constexpr bool KEEP_MH = NARROW && L <= 4;
     constexpr bool K2 = DS && BASE == 0 && !ST;          // keys and range check on doubled high words (see start)
     // (a zero of either sign becomes the positive state: under ST scaling the set bit of -0 could underflow away and leave
     // the +1 of a negative accumulator uncompensated)
@@ -654,6 +660,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
             // the grid: a negative c floors to the one's complement), then + 1 if c < 0.
             // ST: the products are compared against Exp(c) minus the block's scale exponents, c is scaled likewise.
             double acc[TM][TN];
+            int mhi[KEEP_MH ? TM : 1][KEEP_MH ? TN : 1];   // high word of each output's 1.5 * 2^52 * q
             // keys (FP32 accumulators) are exponent fields of doubles in place: (Exp + 1023) << 20.  Products: the larger
             // 16-bit lane of emp (Exp + CB, CB = 1024) or, BASE > 0, the exponent field of P over BASE; c: the state's own
             // field (0 for c = 0: below every real key), minus the scale exponents for ST; an FP32 subnormal c counts with
@@ -685,7 +692,9 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                     // the +1 of a negative c sits in the constant's low word: one unit of the grid either way.  Short blocks:
                     // the low word starts at 2^31, so that the sign correction of the epilogue is a 32-bit addition
                     const int mlo = NARROW ? int(__funnelshift_l(uint32_t(hi), 0x40000000u, 1)) : int(uint32_t(hi) >> 31);
-                    const double magic = __hiloint2double(imad(e20, c_mul64[2], km), mlo);
+                    const int mh = imad(e20, c_mul64[2], km);
+                    if (KEEP_MH) mhi[KEEP_MH ? r : 0][KEEP_MH ? c : 0] = mh;
+                    const double magic = __hiloint2double(mh, mlo);
                     const double x = ST ? __dmul_rn(st, pow2d(-(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]))) : st;
                     acc[r][c] = __dadd_rd(x, magic);
                 } else {
@@ -745,8 +754,10 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                 const int nneg = __popc((sa ^ sb_blk.sgn[pcol + c]) & live);
                 double v;
                 if (NARROW) {
+                    // the register never leaves its binade: its exponent field is the constant's (blocks of 4 keep the
+                    // high word of the start's constant instead of masking it out again)
                     const int hi = __double2hiint(acc[r][c]);
-                    const double magic = __hiloint2double((hi & 0x7FF00000) | 0x00080000, int(0x80000000u));
+                    const double magic = __hiloint2double(KEEP_MH ? mhi[KEEP_MH ? r : 0][KEEP_MH ? c : 0] : (hi & 0x7FF00000) | 0x00080000, int(0x80000000u));
                     v = __dsub_rn(__hiloint2double(hi, __double2loint(acc[r][c]) + nneg), magic);
                 } else {
                     const long long bits = __double_as_longlong(acc[r][c]) + (long long)nneg;
