@@ -175,16 +175,15 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g,
             //   needs no rounding (T when E = e_max, c when E = Exp(c)) is a multiple of qv anyway.  With Mv = 1.5 * 2^52 * qv:
             //       Z1 = RD(c + Mv);   Z = RD(T q + Z1) = Mv + RD_qv(c) + RD_qv(T q);   v = Z - Mv     (at most 40 bits)
             //   T q is the sum register minus its constant (after the sign correction, added to the register's bit pattern).
-            //   RNE-FP32 of v is one more addition and subtraction of a constant, 1.5 * 2^52 * 2^(Exp(v) - 23), the exponent
-            //   clamped at -126 for the subnormal range; the sign of v is copied onto the result (a negative sum that rounds
-            //   to zero is -0 under RNE-FP32).  A result of 2^128 or more is rare and sticky: the loop tracks the largest
-            //   exponent, the flags are set in a second pass. ----
+            //   RNE-FP32 of v is the conversion instruction (a negative sum that rounds to zero is -0, a magnitude that rounds
+            //   to 2^128 becomes infinity), and the conversion back gives the accumulator of the next block.  An infinity is
+            //   rare and sticky: the loop tracks the largest magnitude, the flags are set in a second pass. ----
             const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
             // exponents as the exponent fields of doubles, in place (bits 20..30 of the high word): x20 = (x + 1023) << 20
-            constexpr uint32_t LOWF = (1023 - 126) << 20, HIGHF = (1023 + 126) << 20;
+            constexpr uint32_t LOWF = (1023 - 126) << 20;
             const uint32_t k_c = uint32_t(((52 - F2) << 20) | HALF) + 1u;   // (field of Exp(c)) - 1 + k_c: high word of 1.5 * 2^52 * 2^(Exp(c) - F2)
             constexpr uint32_t k_gtr = (53u << 20) + 1u;   // a sum register's field minus Exp(c)'s beyond which c is dropped (GTR)
-            int fmax = 0, fpend = 0;
+            float wmax = 0.f;
             auto merge = [&](int r, int c) {
                 const uint32_t sa = sa_blk.sgn[prow + r], nza = sa_blk.nz[prow + r] & kmask;
                 const uint32_t negm = (sa ^ sb_blk.sgn[pcol + c]) & nza & sb_blk.nz[pcol + c];
@@ -213,12 +212,11 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g,
                 if (GTR && int(ecm + k_gtr) < m0hi - HALF) st = 0.0;                // special truncation (Algorithm 11 Step 4)
                 const double Mv = __hiloint2double(__viaddmax_s32(int(ecm), int(k_c), m0hi), 0);   // 1.5 * 2^52 * qv
                 const double v = __dsub_rn(__dadd_rd(Y, __dadd_rd(st, Mv)), Mv);
-                const int vhi = __double2hiint(v);
-                const int fv = vhi & EXPF;
-                if (c & 1) fmax = __vimax3_s32(fmax, fpend, fv); else fpend = fv;   // two outputs per three-input maximum
-                const double Mr = __hiloint2double(__viaddmax_s32(fv, (29 << 20) | HALF, int(LOWF) + ((29 << 20) | HALF)), 0);
-                const double rr = __dsub_rn(__dadd_rn(v, Mr), Mr);                  // RNE-FP32 as a double
-                cs[r][c] = __hiloint2double(__double2hiint(rr) | (vhi & int(0x80000000u)), __double2loint(rr));
+                // RNE-FP32 (subnormal range, the sign of a zero and the overflow to infinity included) is the conversion
+                // instruction itself; back as a double the result is the next block's accumulator
+                const float w = __double2float_rn(v);
+                wmax = fmaxf(fabsf(w), wmax);
+                cs[r][c] = double(w);
             };
 
             // ---- the block in two halves of the micro-tile (rows 0, 1 and rows 2, 3): the matrix instructions of one half
@@ -259,7 +257,7 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g,
             }
 #pragma unroll
             for (int o = 8; o < 16; ++o) merge(o / TN, o % TN);
-            if (fmax > int(HIGHF)) {                       // rare: RNE-FP32 overflowed somewhere: +-infinity from now on
+            if (wmax > 3.4028234663852886e38f) {            // rare: RNE-FP32 overflowed somewhere: +-infinity from now on
 #pragma unroll
                 for (int r = 0; r < TM; ++r)
 #pragma unroll
