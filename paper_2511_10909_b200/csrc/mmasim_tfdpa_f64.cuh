@@ -503,7 +503,6 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
     constexpr bool NARROW = DS && L <= 8;
     constexpr int UNROLL_BLK = (L <= 4 || (L <= 16 && BASE == 0)) ? 2 : 1;  // two blocks per trip of the block loop
     constexpr bool KEEP_MH = NARROW && L <= 4;
-    constexpr bool K2 = DS && BASE == 0 && !ST;          // keys and range check on doubled high words (see start)
     // (a zero of either sign becomes the positive state: under ST scaling the set bit of -0 could underflow away and leave
     // the +1 of a negative accumulator uncompensated)
     auto state_of = [](uint32_t w) { const double d = (w & 0x7FFFFFFFu) ? double(__uint_as_float(w)) : 0.0; return __hiloint2double(__double2hiint(d), __double2loint(d) | 1); };
@@ -680,7 +679,8 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                     if (BASE) {
                         // P = 0 gives a key two binades below the smallest real one, which is wrong only for an even smaller c:
                         // the epilogue repairs that case
-                        m = ST ? __vimax3_s32(int(e2 >> (3 + LB)) + KP2, keyc, 0) : __viaddmax_s32(int(e2 >> (3 + LB)), KP2, keyc);
+                        if (ST) m = __vimax3_s32(int(e2 >> (3 + LB)) + KP2, keyc, 0);
+                        else { const int kp = imad(int(e2 >> (3 + LB)), c_mul64[2], KP2); m = fmax3_abs(subnormal_c ? keyc : hi, kp, kp); }
                     } else {
                         // the two 16-bit lanes (Exp + CB of the even and the odd elements) moved to the exponent field by
                         // multiplications, which run beside the integer pipe
@@ -773,8 +773,8 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
             auto finish = [&](int r, int c) {
                 const double v = block_value(r, c);
                 if (DS) {
-                    if (K2) urange = max(uint32_t(imad(__double2hiint(v), c_mul64[6], int(0u - 2u * LOWHI))), urange);
-                    else urange = __viaddmax_u32(uint32_t(__double2hiint(v)) & 0x7FFFFFFFu, 0u - LOWHI, urange);
+                    // (twice the high word: the sign leaves at the top, and a multiply-add is not on the integer pipe)
+                    urange = max(uint32_t(imad(__double2hiint(v), c_mul64[6], int(0u - 2u * LOWHI))), urange);
                     // RZ-FP32 of a number in the normal range: the low 29 bits of the double's significand go
                     const double st = __hiloint2double(__double2hiint(v), (__double2loint(v) & int(0xE0000000u)) | 1);
                     if (BASE) nv[BASE ? r : 0][BASE ? c : 0] = st; else cs[DS ? r : 0][DS ? c : 0] = st;
@@ -827,7 +827,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
             for (int o = 8; o < 16; ++o) finish(o / TN, o % TN);
 
             if (DS) {
-                bool odd = urange >= (K2 ? 2u * SPANHI : SPANHI);   // some result is not a normal FP32 number
+                bool odd = urange >= 2u * SPANHI;       // some result is not a normal FP32 number
                 if (BASE && no_product) {               // rare: no nonzero product: the block returns its accumulator
                     odd = true;
 #pragma unroll
