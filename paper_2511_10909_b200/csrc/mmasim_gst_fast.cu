@@ -12,8 +12,7 @@
 // fractional bits and added.  Alignment, truncation and addition run on the FP64 pipe, where all of it is exact: with
 // q = 2^(e_max - F) and M = 1.5 * 2^52 * q carrying the sign of the term,  fma.rz(s_g, 2^(e_g - frac), M)  is
 // M + RZ_q(term) - the sum has the term's sign, so rounding toward zero truncates its magnitude - and two exact additions
-// move that into the block's sum; s_g becomes a double without a conversion instruction (the integer as the low word
-// of 2^52 + 2^31, minus that constant).  Exponents are handled as exponent fields of doubles in place: the staged scale
+// move that into the block's sum; s_g becomes a double by one conversion instruction (exact).  Exponents are handled as exponent fields of doubles in place: the staged scale
 // words hold (Exp + bias) << 20 with the significand below, the sum of an A word and a B word is the field of
 // 2^(Exp(alpha) + Exp(beta)) (with the two significands added below it, masked away after the maximum).  RZ-FP32 is one
 // conversion instruction.  Liveness of a group needs its per-element nonzero masks (16 bits per row and group); a row
@@ -99,8 +98,6 @@ __global__ void __launch_bounds__(NT, 2) gst_kernel(DevModel m, GemmArgs g) {
             }
             cw[r][c] = w;
         }
-    // 2^52 + 2^31: an integer n becomes the double n by taking n ^ 2^31 as the low word of this constant and subtracting it
-    const double two52_31 = __hiloint2double(0x43300000, int(0x80000000u));
 
     for (int64_t k0 = 0; k0 < g.K; k0 += KC) {
         __syncthreads();
@@ -220,7 +217,7 @@ __global__ void __launch_bounds__(NT, 2) gst_kernel(DevModel m, GemmArgs g) {
 #pragma unroll
                     for (int r = 0; r < RH; ++r)
 #pragma unroll
-                        for (int c = 0; c < TN; ++c) p[r][c] = __dp4a(av[r], bv[c], j == 0 ? (NVF4 ? 0 : int(0x80000000u)) : p[r][c]);
+                        for (int c = 0; c < TN; ++c) p[r][c] = __dp4a(av[r], bv[c], j == 0 ? 0 : p[r][c]);
                 }
                 const uint4 sa4 = *reinterpret_cast<const uint4*>(&s.sa[grp][ty * TM + rh]);
                 const uint4 sb4 = *reinterpret_cast<const uint4*>(&s.sb[grp][tx * TN]);
@@ -234,11 +231,9 @@ __global__ void __launch_bounds__(NT, 2) gst_kernel(DevModel m, GemmArgs g) {
                 for (int r = 0; r < RH; ++r)
 #pragma unroll
                     for (int c = 0; c < TN; ++c) {
-                        // (MXFP4: the dot product was started at 2^31, which is the form the conversion below wants)
-                        int sgx = p[r][c];                                          // s_g ^ 2^31
-                        if (NVF4) sgx = (sgx * int(sag[r] & 0xFFu) * int(sbg[c] & 0xFFu)) ^ int(0x80000000u);
-                        const int sg = ~sgx;                                        // its sign bit is that of s_g
-                        const double gd = __dsub_rn(__hiloint2double(0x43300000, sgx), two52_31);
+                        int sg = p[r][c];
+                        if (NVF4) sg = sg * int(sag[r] & 0xFFu) * int(sbg[c] & 0xFFu);
+                        const double gd = __int2double_rn(sg);                      // exact
                         const double sc = __hiloint2double(ea20[r] + eb20[c], 0);                       // 2^(e_g - frac)
                         const double Ms = __hiloint2double(mhi[r][c] | (sg & int(0x80000000u)), 0);
                         S[r][c] = __dsub_rn(__dadd_rn(S[r][c], __fma_rz(gd, sc, Ms)), Ms);
