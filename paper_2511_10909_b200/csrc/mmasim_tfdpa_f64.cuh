@@ -21,9 +21,10 @@
 // A term whose value is zero has no exponent and takes no part in e_max: zero elements are staged with the exponent
 // word 0, far below every real exponent sum, and a zero c enters the maximum as 0 as well.
 //
-// rho (Table 2) is one conversion instruction per block and output: cvt.rz.f32.f64 (keeps subnormals; a result of
-// magnitude >= 2^128 is an overflow and becomes infinity) or cvt.rn.f16.f64; an infinity is recorded as a sticky
-// special value.
+// rho (Table 2): the accumulator lives between blocks as a double.  RZ-FP32 of a result in the normal range is a mask on
+// the double's low word; RNE-FP16 is cvt.rn.f16.f64 and the half converted back.  Zero, subnormal and overflowing results
+// are found by one range check on the exponent field and take a rare path (cvt.rz.f32.f64 keeps subnormals; a magnitude of
+// 2^128 or more, or a half that rounded to infinity, becomes a sticky infinity).
 // e_max is computed as in the integer kernels (fused add-max on two 16-bit lanes); NaN / infinity inputs use the same
 // sticky flags and rescan of the raw words (Section 4.2): their staged operands are the zero stand-ins.
 #pragma once
@@ -471,8 +472,6 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
     auto col_at = [&](int c) { return wc * 16 + 8 * (c >> 1) + 2 * tq + (c & 1); };
     const int64_t row0 = int64_t(blockIdx.y) * BM, col0 = int64_t(blockIdx.x) * BN;
     const FmtDesc fa = fmt_desc(m.fmt_a), fb = fmt_desc(m.fmt_b);
-    // high word of 1.5 * 2^52 * 2^(e_max - F) is (e_max + CB) * 2^20 + MAGIC_K
-    const int MAGIC_K = ((1023 + 52 - m.F - CB) << 20) | 0x00080000;
 
     // the decoded blocks of this tile row of A and tile column of B, chunk after chunk, land in two buffers by bulk copies
     const int NCH = int(g.K / KC);
@@ -496,8 +495,9 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
     // FP32 accumulators live between blocks as doubles ("state"): the value RZ-FP32 produced, exactly, with bit 0 of the
     // low word set so that the next block's addition (rounded toward minus infinity) never finds it on its grid; the
     // conversion function is then a mask on the double's low word and the exponent of c is the double's own field.
-    // Results outside the range of normal FP32 numbers (zero, subnormal, overflow) leave the fast path.
-    constexpr bool DS = !ACC16;
+    // Results outside the range of normal FP32 numbers (zero, subnormal, overflow) leave the fast path.  FP16
+    // accumulators live the same way, as the exact doubles of the rounded halves (normal range 2^-14 .. 2^16).
+    constexpr bool DS = true;
     // blocks of at most 8 terms: |S| < 2^(F+1) + L * 2^(F+2) < 2^31, so the sum register's low word, started at 2^31, never
     // carries into the high word
     constexpr bool NARROW = DS && L <= 8;
@@ -505,11 +505,21 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
     constexpr bool KEEP_MH = NARROW && L <= 4;
     // (a zero of either sign becomes the positive state: under ST scaling the set bit of -0 could underflow away and leave
     // the +1 of a negative accumulator uncompensated)
-    auto state_of = [](uint32_t w) { const double d = (w & 0x7FFFFFFFu) ? double(__uint_as_float(w)) : 0.0; return __hiloint2double(__double2hiint(d), __double2loint(d) | 1); };
-    auto word_of = [](double st) { return __float_as_uint(__double2float_rz(__hiloint2double(__double2hiint(st), __double2loint(st) & ~1))); };
+    auto state_of = [](uint32_t w) {
+        double d = 0.0;
+        if (ACC16) { if (w & 0x7FFFu) d = double(__half2float(__ushort_as_half((unsigned short)w))); }
+        else if (w & 0x7FFFFFFFu) d = double(__uint_as_float(w));
+        return __hiloint2double(__double2hiint(d), __double2loint(d) | 1);
+    };
+    auto word_of = [](double st) {
+        const double d = __hiloint2double(__double2hiint(st), __double2loint(st) & ~1);
+        return ACC16 ? uint32_t(__half_as_ushort(__double2half(d))) : __float_as_uint(__double2float_rz(d));
+    };
+    // the range of normal numbers of the accumulator's format, as exponent fields of doubles
+    constexpr int EXP_LOW = ACC16 ? -14 : -126, EXP_TOP = ACC16 ? 16 : 128;
     double cs[DS ? TM : 1][DS ? TN : 1];
     uint32_t sub_mask = 0u;                             // outputs whose accumulator is a nonzero FP32 subnormal: Exp(c) = -126
-    uint32_t cw[TM][TN];                                // the accumulator of each output: a finite FP32 / FP16 word (FP16 path)
+    uint32_t cw[TM][TN];                                // the words of C as read (finite ones; the rest become flags)
     uint32_t sp_nan = 0u, sp_pinf = 0u, sp_ninf = 0u;   // per output (bit r * TN + c): NaN / +inf / -inf seen so far
     float promoted[PROMOTE ? TM : 1][PROMOTE ? TN : 1];
 #define MMASIM_SP_GET(r, c) ((((sp_nan >> ((r) * TN + (c))) & 1u)) | (((sp_pinf >> ((r) * TN + (c))) & 1u) << 1) | (((sp_ninf >> ((r) * TN + (c))) & 1u) << 2))
@@ -532,7 +542,8 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
             cw[r][c] = w;
             if (DS) {
                 cs[DS ? r : 0][DS ? c : 0] = state_of(w);
-                if ((w & 0x7F800000u) == 0u && (w & 0x007FFFFFu) != 0u) sub_mask |= 1u << (r * TN + c);
+                if (ACC16 ? ((w & 0x7C00u) == 0u && (w & 0x03FFu) != 0u) : ((w & 0x7F800000u) == 0u && (w & 0x007FFFFFu) != 0u))
+                    sub_mask |= 1u << (r * TN + c);
             }
         }
 
@@ -672,7 +683,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                     const int hi = __double2hiint(st);
                     // the keys keep whatever sits below their exponent fields (mantissa bits of c, the other 16-bit lane): it
                     // decides nothing but ties between equal exponents, and one mask after the maximum removes it
-                    int keyc = subnormal_c ? (1023 - 126) << 20 : hi & 0x7FFFFFFF;
+                    int keyc = subnormal_c ? (1023 + EXP_LOW) << 20 : hi & 0x7FFFFFFF;
                     if (ST) keyc -= (sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]) << 20;
                     const uint32_t e2 = emp[r][c];
                     int m;
@@ -697,18 +708,6 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                     const double magic = __hiloint2double(mh, mlo);
                     const double x = ST ? __dmul_rn(st, pow2d(-(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]))) : st;
                     acc[r][c] = __dadd_rd(x, magic);
-                } else {
-                    const uint32_t field = ACC16 ? (cw[r][c] >> 10) & 0x1Fu : (cw[r][c] >> 23) & 0xFFu;
-                    int rel = int(max(field, 1u)) + (CB - (ACC16 ? 15 : 127));
-                    if (ST) rel -= sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0];
-                    if ((cw[r][c] & (ACC16 ? 0x7FFFu : 0x7FFFFFFFu)) == 0u) rel = 0;       // c = 0 has no exponent
-                    const int emax = BASE ? max(int(emp[r][c] >> (23 + LB)) + (CB + 2 - (127 + 1) / (BASE ? BASE : 1)), rel)
-                                          : __vimax3_s32(int(emp[r][c] & 0xFFFFu), int(emp[r][c] >> 16), rel);     // e_max + CB
-                    const double magic = __hiloint2double(emax * (1 << 20) + MAGIC_K, int(cw[r][c] >> (ACC16 ? 15 : 31)));
-                    double cd = ACC16 ? double(__half2float(__ushort_as_half((unsigned short)cw[r][c]))) : double(__uint_as_float(cw[r][c]));
-                    if (ST) cd = __dmul_rn(cd, pow2d(-(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0])));
-                    cd = __hiloint2double(__double2hiint(cd), __double2loint(cd) | 1);
-                    acc[r][c] = __dadd_rd(cd, magic);
                 }
             };
             auto restart_subnormals = [&](int r0) {     // rare: redo the outputs whose accumulator is an FP32 subnormal
@@ -739,13 +738,10 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
             // ---- sign corrections, rho.  An overflow (|v| >= 2^128, or an FP16 result that rounds to infinity) is rare
             // and sticky: the loop only tracks it, the flags are set in a second pass ----
             const uint32_t kmask = (L == 32) ? 0xFFFFFFFFu : (((1u << L) - 1u) << kb);
-            constexpr uint32_t ABS = ACC16 ? 0x7FFFu : 0x7FFFFFFFu;
-            constexpr uint32_t SUSPECT = ACC16 ? 0x7C00u : 0x7F7FFFFFu;   // FP16: infinity; FP32: cvt.rz saturates at the largest finite word
-            uint32_t wmax = 0u;
             bool no_product = false;                    // BASE > 0: some output of the micro-tile has no nonzero product
             // FP32 state: the largest (high word of |v|) - (that of 2^-126), unsigned: a v outside the normal FP32 range -
             // zero and the subnormal range wrap to the top - shows as a value of (that of 2^128) - (that of 2^-126) or more
-            constexpr uint32_t LOWHI = uint32_t(1023 - 126) << 20, SPANHI = uint32_t(128 + 126) << 20;
+            constexpr uint32_t LOWHI = uint32_t(1023 + EXP_LOW) << 20, SPANHI = uint32_t(EXP_TOP - EXP_LOW) << 20;
             uint32_t urange = 0u;
             auto block_value = [&](int r, int c) -> double {
                 const uint32_t sa = sa_blk.sgn[prow + r], nza = sa_blk.nz[prow + r] & kmask;
@@ -769,19 +765,22 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                 return v;
             };
             double nv[DS && BASE ? TM : 1][DS && BASE ? TN : 1];      // BASE > 0: the old accumulators survive until the repair below
-            uint32_t nw[DS ? 1 : TM][DS ? 1 : TN];
             auto finish = [&](int r, int c) {
                 const double v = block_value(r, c);
-                if (DS) {
+                if (ACC16) {
+                    // RNE-FP16 is the conversion instruction (subnormal range and the overflow to infinity included); the
+                    // half as a double again is the next accumulator, and its exponent field says whether it is a normal number
+                    double x;
+                    asm("cvt.f64.f16 %0, %1;" : "=d"(x) : "h"(__half_as_ushort(__double2half(v))));
+                    urange = max(uint32_t(imad(__double2hiint(x), c_mul64[6], int(0u - 2u * LOWHI))), urange);
+                    const double st = __hiloint2double(__double2hiint(x), __double2loint(x) | 1);
+                    if (BASE) nv[BASE ? r : 0][BASE ? c : 0] = st; else cs[DS ? r : 0][DS ? c : 0] = st;
+                } else if (DS) {
                     // (twice the high word: the sign leaves at the top, and a multiply-add is not on the integer pipe)
                     urange = max(uint32_t(imad(__double2hiint(v), c_mul64[6], int(0u - 2u * LOWHI))), urange);
                     // RZ-FP32 of a number in the normal range: the low 29 bits of the double's significand go
                     const double st = __hiloint2double(__double2hiint(v), (__double2loint(v) & int(0xE0000000u)) | 1);
                     if (BASE) nv[BASE ? r : 0][BASE ? c : 0] = st; else cs[DS ? r : 0][DS ? c : 0] = st;
-                } else {
-                    const uint32_t w = ACC16 ? uint32_t(__half_as_ushort(__double2half(v))) : __float_as_uint(__double2float_rz(v));
-                    wmax = max(wmax, w & ABS);
-                    nw[DS ? 0 : r][DS ? 0 : c] = w;
                 }
             };
 
@@ -849,42 +848,16 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                             const double st = cs[DS ? r : 0][DS ? c : 0];
                             const double v = __hiloint2double(__double2hiint(st), __double2loint(st) & ~1);
                             const uint32_t bit = 1u << (r * TN + c);
-                            if (fabs(v) >= 3.402823669209385e38) {                        // |v| >= 2^128: +-infinity from now on
+                            if (fabs(v) >= (ACC16 ? 65536.0 : 3.402823669209385e38)) {    // |v| >= 2^128 (FP16: the half is infinity): +-infinity from now on
                                 if (!((sp_nan | sp_pinf | sp_ninf) & bit)) { if (v < 0.0) sp_ninf |= bit; else sp_pinf |= bit; }
                                 cs[DS ? r : 0][DS ? c : 0] = state_of(0u);
-                            } else if (fabs(v) < 1.1754943508222875e-38) {                // zero or below 2^-126: the word decides
-                                const uint32_t w = __float_as_uint(__double2float_rz(v));
+                            } else if (fabs(v) < (ACC16 ? 6.103515625e-05 : 1.1754943508222875e-38)) {   // zero or below the normal range: the word decides
+                                const uint32_t w = ACC16 ? uint32_t(__half_as_ushort(__double2half(v))) : __float_as_uint(__double2float_rz(v));
                                 cs[DS ? r : 0][DS ? c : 0] = state_of(w);
-                                if (w & 0x7FFFFFFFu) sub_mask |= bit;
+                                if (w & (ACC16 ? 0x7FFFu : 0x7FFFFFFFu)) sub_mask |= bit;
                             }
                         }
                 }
-            } else {
-                if (BASE && no_product) {               // rare: no nonzero product: the block returns its accumulator
-#pragma unroll
-                    for (int r = 0; r < TM; ++r)
-#pragma unroll
-                        for (int c = 0; c < TN; ++c)
-                            if ((sa_blk.nz[prow + r] & kmask & sb_blk.nz[pcol + c]) == 0u) nw[DS ? 0 : r][DS ? 0 : c] = cw[r][c];
-                }
-                if (wmax >= SUSPECT) {                  // rare: overflow of the conversion: sticky infinities
-#pragma unroll
-                    for (int r = 0; r < TM; ++r)
-#pragma unroll
-                        for (int c = 0; c < TN; ++c) {
-                            if ((nw[DS ? 0 : r][DS ? 0 : c] & ABS) != SUSPECT) continue;
-                            if (BASE && (sa_blk.nz[prow + r] & kmask & sb_blk.nz[pcol + c]) == 0u) continue;   // the kept accumulator
-                            const double v = block_value(r, c);
-                            if (!ACC16 && fabs(v) < 3.402823669209385e38) continue;       // below 2^128: the largest finite number, legitimately
-                            const uint32_t bit = 1u << (r * TN + c);
-                            if (!((sp_nan | sp_pinf | sp_ninf) & bit)) { if (v < 0.0) sp_ninf |= bit; else sp_pinf |= bit; }
-                            nw[DS ? 0 : r][DS ? 0 : c] = 0u;                              // +-infinity from now on
-                        }
-                }
-#pragma unroll
-                for (int r = 0; r < TM; ++r)
-#pragma unroll
-                    for (int c = 0; c < TN; ++c) cw[r][c] = nw[DS ? 0 : r][DS ? 0 : c];
             }
         }
         __syncthreads();                                // everybody has finished with this buffer
