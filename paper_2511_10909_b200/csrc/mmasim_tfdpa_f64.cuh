@@ -251,6 +251,7 @@ struct Blk64 {
     uint32_t exp2[KC / 2][R];
     uint16_t pe[R][PE_STRIDE64];
     uint32_t sgn[R], nz[R];
+    uint8_t sf[R];                  // [permuted row]: the E8M0 scale factor of the row for this block of 32 (ST-FDPA), else 127
     uint32_t special;               // the block holds an infinity or a NaN
     uint32_t max_exp;               // the largest Exp(x) + EB of the block's elements (0: all zero)
     uint32_t pad[2];
@@ -276,7 +277,8 @@ __host__ __device__ constexpr int pe64_sub(int base) { return base == 8 ? 32 : (
 // EOSPLIT (GTR-FDPA, blocks of 16): inside each block of 16 the operand plane holds the even elements first, then the odd
 // ones, so that a matrix instruction sums four elements of one group; exponent pairs and masks keep the order of K.
 template <int EK, int R, bool IS_A, int BASE, bool EOSPLIT = false>
-__global__ void __launch_bounds__(256) decode64_kernel(DevModel m, const unsigned char* src, int64_t rows, int64_t ld, Blk64<R>* dst) {
+__global__ void __launch_bounds__(256) decode64_kernel(DevModel m, const unsigned char* src, int64_t rows, int64_t ld, Blk64<R>* dst,
+                                                       const uint8_t* sf = nullptr, int64_t ld_sf = 0) {
     using E = Elem<EK>;
     constexpr int TPR = KC / E::TASK, TASKS = R * TPR, WORDS = E::TASK * E::BYTES / 4;
     extern __shared__ __align__(16) unsigned char dec_smem[];
@@ -310,6 +312,16 @@ __global__ void __launch_bounds__(256) decode64_kernel(DevModel m, const unsigne
             if (grow < rows) v = reinterpret_cast<const uint4*>(src + (grow * ld + k0 + h * E::TASK) * E::BYTES)[q];
             w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
         }
+        // ST-FDPA (Algorithm 8): the row's scale factor for this block of 32 multiplies its operands here, exactly (an
+        // addition to the exponent field of a nonzero double); exponent planes stay unscaled, the main kernel adds
+        // Exp(alpha) + Exp(beta) to the block maximum.  A NaN scale factor stages zeros (the output is NaN by its flag).
+        int sc20 = 0;
+        bool sc_nan = false;
+        if (sf) {
+            const uint32_t sbyte = grow < rows ? uint32_t(sf[grow * ld_sf + blockIdx.x]) : 127u;
+            sc20 = (int(sbyte) - 127) << 20;
+            sc_nan = sbyte == 0xFFu;
+        }
         uint32_t bits = 0u, prev_exp = 0u, pw[E::TASK / 2];
 #pragma unroll
         for (int q = 0; q < E::TASK; ++q) {
@@ -320,6 +332,10 @@ __global__ void __launch_bounds__(256) decode64_kernel(DevModel m, const unsigne
                 const uint32_t byte = (w[q / 4] >> (8 * (q % 4))) & 0xFFu;
                 const LutEntry64 e = lut[byte];
                 op = e.op;
+                if (sf) {
+                    const int ohi = __double2hiint(op);
+                    op = ((ohi & 0x7FFFFFFF) == 0 || sc_nan) ? 0.0 : __hiloint2double(ohi + sc20, __double2loint(op));
+                }
                 expb = e.exp;
                 bits += ((e.bits & 1u) | ((e.bits & 4u) << 14)) << q;
                 spec |= e.bits & 2u;
@@ -368,6 +384,10 @@ __global__ void __launch_bounds__(256) decode64_kernel(DevModel m, const unsigne
         }
     }
     if (spec) atomicOr(&blk.special, 1u);
+    if (tid < R) {                                      // the scale factors travel with the block (rows beyond the matrix: 2^0)
+        const int64_t grow = int64_t(blockIdx.y) * R + tid;
+        blk.sf[IS_A ? perm_row64(tid) : perm_col64(tid)] = (sf && grow < rows) ? sf[grow * ld_sf + blockIdx.x] : uint8_t(127);
+    }
     top_exp = __reduce_max_sync(0xFFFFFFFFu, top_exp);
     if ((tid & 31) == 0 && top_exp) atomicMax(&blk.max_exp, top_exp);
     __syncthreads();
@@ -503,8 +523,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
     constexpr bool NARROW = DS && L <= 8;
     constexpr int UNROLL_BLK = (L <= 4 || (L <= 16 && BASE == 0)) ? 2 : 1;  // two blocks per trip of the block loop
     constexpr bool KEEP_MH = NARROW && L <= 4;
-    // (a zero of either sign becomes the positive state: under ST scaling the set bit of -0 could underflow away and leave
-    // the +1 of a negative accumulator uncompensated)
+    // (a zero of either sign becomes the positive state)
     auto state_of = [](uint32_t w) {
         double d = 0.0;
         if (ACC16) { if (w & 0x7FFFu) d = double(__half2float(__ushort_as_half((unsigned short)w))); }
@@ -561,23 +580,27 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
         // the first block's product exponents (the other blocks' are taken beside the multiply-adds of their predecessor)
         if (BASE == 0) product_exponents_adj<L>(&sa_blk.exp2[0][prow], &sb_blk.exp2[0][pcol], emp);
 
-        // ST-FDPA (Algorithm 8): Exp(alpha) of this thread's rows and Exp(beta) of its columns for this block of 32
+        // ST-FDPA (Algorithm 8): Exp(alpha) of this thread's rows and Exp(beta) of its columns for this block of 32, as
+        // exponent-field increments.  The staged operands already carry the scale factors (decode pass), so the products,
+        // their sum and the accumulator all live in the one scaled domain and only the block maximum needs the sum added.
+        static_assert(!ST || BASE > 0, "the scaled rows all take their maximum from the tensor cores");
         int sa_exp[ST ? TM : 1], sb_exp[ST ? TN : 1];
         if (ST) {
-            const int64_t sblk = k0 / KC;
+            // (the scale bytes came in with the decoded blocks: one 32-bit shared load for the thread's four rows / columns)
+            static_assert(TM == 4 && TN == 4, "four scale bytes per load");
+            const uint32_t wa4 = *reinterpret_cast<const uint32_t*>(&sa_blk.sf[prow]);
+            const uint32_t wb4 = *reinterpret_cast<const uint32_t*>(&sb_blk.sf[pcol]);
             uint32_t scale_nan = 0u;                    // bit r * TN + c: alpha or beta of that output is NaN
 #pragma unroll
             for (int r = 0; r < TM; ++r) {
-                const int64_t i = row0 + row_at(r);
-                const uint32_t w = i < g.M ? uint32_t(g.sfa[i * g.ld_sfa + sblk]) : 127u;
-                sa_exp[ST ? r : 0] = int(w) - 127;
+                const uint32_t w = (wa4 >> (8 * r)) & 0xFFu;
+                sa_exp[ST ? r : 0] = ((int(w) - 127) << 20) + KP2;   // in place of a double's exponent field, with the key's constant
                 if (w == 0xFFu) scale_nan |= ((1u << TN) - 1u) << (r * TN);
             }
 #pragma unroll
             for (int c = 0; c < TN; ++c) {
-                const int64_t j = col0 + col_at(c);
-                const uint32_t w = j < g.N ? uint32_t(g.sfb[j * g.ld_sfb + sblk]) : 127u;
-                sb_exp[ST ? c : 0] = int(w) - 127;
+                const uint32_t w = (wb4 >> (8 * c)) & 0xFFu;
+                sb_exp[ST ? c : 0] = (int(w) - 127) << 20;
                 if (w == 0xFFu) scale_nan |= 0x11111111u << c;
             }
             sp_nan |= scale_nan;                        // a NaN scale factor makes the block result NaN
@@ -668,13 +691,13 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
             // ---- e_max = max(Exp(c), product exponents) and the accumulator term:
             // acc = 1.5 * 2^52 * q + floor(c' / q) * q, c' = c with the lowest mantissa bit of its double set (never on
             // the grid: a negative c floors to the one's complement), then + 1 if c < 0.
-            // ST: the products are compared against Exp(c) minus the block's scale exponents, c is scaled likewise.
+            // ST: the staged operands carry the scale factors, the key of the products gets Exp(alpha) + Exp(beta) added.
             double acc[TM][TN];
             int mhi[KEEP_MH ? TM : 1][KEEP_MH ? TN : 1];   // high word of each output's 1.5 * 2^52 * q
             // keys (FP32 accumulators) are exponent fields of doubles in place: (Exp + 1023) << 20.  Products: the larger
             // 16-bit lane of emp (Exp + CB, CB = 1024) or, BASE > 0, the exponent field of P over BASE; c: the state's own
-            // field (0 for c = 0: below every real key), minus the scale exponents for ST; an FP32 subnormal c counts with
-            // Exp = -126 (rare: patched after the pass over the outputs).
+            // field (0 for c = 0: below every real key); a subnormal c counts with Exp = -126 (FP16: -14; rare: patched
+            // after the pass over the outputs).
             constexpr int KM = (52 << 20) | 0x00080000;              // + (e_max - F) gives the high word of 1.5 * 2^52 * q
             const int km = KM - (m.F << 20);
             auto start = [&](int r, int c, bool subnormal_c) {
@@ -684,20 +707,19 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                     // the keys keep whatever sits below their exponent fields (mantissa bits of c, the other 16-bit lane): it
                     // decides nothing but ties between equal exponents, and one mask after the maximum removes it
                     int keyc = subnormal_c ? (1023 + EXP_LOW) << 20 : hi & 0x7FFFFFFF;
-                    if (ST) keyc -= (sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]) << 20;
                     const uint32_t e2 = emp[r][c];
                     int m;
                     if (BASE) {
                         // P = 0 gives a key two binades below the smallest real one, which is wrong only for an even smaller c:
                         // the epilogue repairs that case
-                        if (ST) m = __vimax3_s32(int(e2 >> (3 + LB)) + KP2, keyc, 0);
-                        else { const int kp = imad(int(e2 >> (3 + LB)), c_mul64[2], KP2); m = fmax3_abs(subnormal_c ? keyc : hi, kp, kp); }
+                        const int kp = ST ? int(e2 >> (3 + LB)) + sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]
+                                          : imad(int(e2 >> (3 + LB)), c_mul64[2], KP2);
+                        m = fmax3_abs(subnormal_c ? keyc : hi, kp, kp);
                     } else {
                         // the two 16-bit lanes (Exp + CB of the even and the odd elements) moved to the exponent field by
                         // multiplications, which run beside the integer pipe
                         const int klo = imad(int(e2), c_mul64[0], -(1 << 20)), khi = imad(int(e2), c_mul64[1], -(1 << 20));
-                        if (ST) m = __vimax3_s32(klo, khi, max(keyc, 0));
-                        else m = fmax3_abs(subnormal_c ? keyc : hi, klo, khi);
+                        m = fmax3_abs(subnormal_c ? keyc : hi, klo, khi);
                     }
                     const int e20 = m & 0x7FF00000;
                     // the +1 of a negative c sits in the constant's low word: one unit of the grid either way.  Short blocks:
@@ -706,8 +728,7 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                     const int mh = imad(e20, c_mul64[2], km);
                     if (KEEP_MH) mhi[KEEP_MH ? r : 0][KEEP_MH ? c : 0] = mh;
                     const double magic = __hiloint2double(mh, mlo);
-                    const double x = ST ? __dmul_rn(st, pow2d(-(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]))) : st;
-                    acc[r][c] = __dadd_rd(x, magic);
+                    acc[r][c] = __dadd_rd(st, magic);
                 }
             };
             auto restart_subnormals = [&](int r0) {     // rare: redo the outputs whose accumulator is an FP32 subnormal
@@ -761,7 +782,6 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                     const double magic = __hiloint2double((hi & 0x7FF00000) | 0x00080000, 0);
                     v = __dsub_rn(__longlong_as_double(bits), magic);                 // S * q, exact; +0 when S = 0
                 }
-                if (ST) v = __dmul_rn(v, pow2d(sa_exp[ST ? r : 0] + sb_exp[ST ? c : 0]));
                 return v;
             };
             double nv[DS && BASE ? TM : 1][DS && BASE ? TN : 1];      // BASE > 0: the old accumulators survive until the repair below
@@ -933,9 +953,9 @@ cudaError_t launch_one64b(const DevModel& m, const GemmArgs& g, cudaStream_t str
     Blk64<BM>* wa = static_cast<Blk64<BM>*>(ws);
     Blk64<BN>* wb = reinterpret_cast<Blk64<BN>*>(static_cast<unsigned char*>(ws) + bytes_a);
     decode64_kernel<EK, BM, true, BASE><<<dim3((unsigned)nch, (unsigned)tiles_m), 256, dsh_a, stream>>>(
-        m, static_cast<const unsigned char*>(g.A), g.M, g.lda, wa);
+        m, static_cast<const unsigned char*>(g.A), g.M, g.lda, wa, ST ? g.sfa : nullptr, g.ld_sfa);
     decode64_kernel<EK, BN, false, BASE><<<dim3((unsigned)nch, (unsigned)tiles_n), 256, dsh_b, stream>>>(
-        m, static_cast<const unsigned char*>(g.B), g.N, g.ldb, wb);
+        m, static_cast<const unsigned char*>(g.B), g.N, g.ldb, wb, ST ? g.sfb : nullptr, g.ld_sfb);
     dim3 grid((unsigned)tiles_n, (unsigned)tiles_m, 1);
     tfdpa64_kernel<EK, L, RHO, PROMOTE, ST, BASE><<<grid, NT, sh, stream>>>(m, g, wa, wb);
     err = cudaGetLastError();
