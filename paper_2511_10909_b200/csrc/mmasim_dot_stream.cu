@@ -4,7 +4,7 @@
 //   T-FDPA (Algorithm 7) for FP16 / BF16 / TF32 inputs, L in {4, 8, 16}, F in 23..25, rho in {RZ-FP32, RNE-FP16}
 //   Phi_FTZ-AddMul (Algorithm 2) for FP16 / BF16 inputs, P in {2, 4}
 // Two ways to bring the rows in:
-//   staged - rows of 8, 16, 32, 64 or 128 bytes: the CTA's 256 rows of A and of B are one contiguous range each, copied
+//   staged - rows of 8, 16, 32, 64 or 128 bytes: the CTA's 128 rows of A and of B are one contiguous range each, copied
 //            to shared memory with 16-byte asynchronous copies (consecutive threads, consecutive chunks: every
 //            sector of a request is used), chunks XOR-swizzled so that each thread then reads its own row without bank
 //            conflicts; several CTAs per SM keep the copies of one tile under the arithmetic of another
@@ -21,7 +21,7 @@ using fast::EK_F16;
 using fast::EK_BF16;
 using fast::EK_TF32;
 
-constexpr int DOT_THREADS = 256;
+constexpr int DOT_THREADS = 128;
 
 // ---- where a thread finds its two rows ----
 struct GlobalRows {                      // row pointers into global memory
@@ -314,7 +314,7 @@ dot_ftz_kernel(int64_t n, int64_t K, const void* A, const void* B, const void* C
     }
 }
 
-// Rows of 8 to 128 bytes (a power of two) are staged through shared memory: 2 * 256 rows per CTA.
+// Rows of 8 to 128 bytes (a power of two) are staged through shared memory: 2 * 128 rows per CTA.
 bool staged_rows(int64_t row_bytes) {
     return row_bytes == 8 || row_bytes == 16 || row_bytes == 32 || row_bytes == 64 || row_bytes == 128;
 }
