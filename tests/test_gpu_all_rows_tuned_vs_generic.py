@@ -72,3 +72,58 @@ def test_row_on_random_shapes(key):
     bad = np.argwhere(D != G)
     assert bad.size == 0, (key, kernel, (M, N, K), "bit patterns", len(bad), bad[:4])
     gu.assert_samples_equal(D, gu.oracle_samples(key, wild, pairs), pairs, f"{key} {kernel} {(M, N, K)} bit patterns")
+
+
+def _raw_words(g, shape, itemsize):
+    if itemsize == 1:
+        return g.integers(0, 256, shape, dtype=np.uint8)
+    return (g.integers(0, 1 << (8 * itemsize - 1), shape, dtype=np.uint64).astype(_word_dtype(itemsize)) * 2
+            + g.integers(0, 2, shape).astype(_word_dtype(itemsize)))
+
+
+_SMALL_WIDTH = {"e4m3": 8, "e5m2": 8, "e3m2": 6, "e2m3": 6, "e2m1": 4}
+
+
+@pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("MMASIM_PARITY_SEEDS", "3"))))
+def test_rows_on_more_seeds_and_magnitudes(seed):
+    """Every registry row again on further seeded shapes, the dispatcher's kernel against the generic kernels on every
+    output word, with four inputs each: ordinary values with zeros, raw bit patterns, and the bit patterns with the top
+    exponent bit of every word cleared (tiny products: zero and subnormal results) or set (huge ones: overflow, infinities
+    and NaNs).  MMASIM_PARITY_SEEDS sets the number of seeds (default 3; 240 ran clean)."""
+    from paper_2511_10909_b200 import mmasim
+    for key in mmasim.model_keys():
+        g = wl.rng(zlib.crc32(("-".join(key) + f"#{seed}").encode()))
+        packed4 = key[1] in ("mxf4", "nvf4")
+        kmul = 64 if packed4 else 32
+        M, N, K = int(g.integers(1, 400)), int(g.integers(1, 300)), kmul * int(g.integers(1, 9))
+        inp = wl.normal_inputs(key[1], key[2], M, N, K, seed=int(g.integers(1, 1 << 30)))
+        A, B, C = inp["A"].copy(), inp["B"].copy(), inp["C"].copy()
+        A[g.random(A.shape) < 0.1] = 0
+        B[g.random(B.shape) < 0.05] = 0
+        C[g.random(C.shape) < 0.2] = 0
+        inp.update(A=A, B=B, C=C)
+        cases = [("values", inp)]
+        wild = {k: _raw_words(g, inp[k].shape, inp[k].dtype.itemsize) for k in ("A", "B", "C")}
+        width = 8 * A.dtype.itemsize
+        if not packed4 and A.dtype.itemsize == 1:
+            width = _SMALL_WIDTH.get(key[1].replace("mx", ""), 8)
+            wild["A"] &= np.uint8((1 << width) - 1)
+            wild["B"] &= np.uint8((1 << width) - 1)
+        if "sfa" in inp:
+            wild["sfa"] = g.integers(0, 256, inp["sfa"].shape, dtype=np.uint8)
+            wild["sfb"] = g.integers(0, 256, inp["sfb"].shape, dtype=np.uint8)
+        cases.append(("bit patterns", wild))
+        for name, setbit in (("small magnitudes", False), ("large magnitudes", True)):
+            v = {k: x.copy() for k, x in wild.items()}
+            for k in ("A", "B", "C"):
+                if packed4 and k != "C":
+                    continue
+                top = v[k].dtype.type(1 << ((8 * C.dtype.itemsize if k == "C" else width) - 2))
+                v[k] = (v[k] | top) if setbit else (v[k] & ~top)
+            cases.append((name, v))
+        for name, x in cases:
+            D = gu.run_gemm(key, x)
+            kernel = mmasim.last_kernel()
+            G = gu.run_gemm(key, x, force_generic=True)
+            bad = np.argwhere(D != G)
+            assert bad.size == 0, (key, kernel, (M, N, K), name, len(bad), bad[:4])
