@@ -87,7 +87,7 @@ _SMALL_WIDTH = {"e4m3": 8, "e5m2": 8, "e3m2": 6, "e2m3": 6, "e2m1": 4}
 @pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("MMASIM_PARITY_SEEDS", "3"))))
 def test_rows_on_more_seeds_and_magnitudes(seed):
     """Every registry row again on further seeded shapes, the dispatcher's kernel against the generic kernels on every
-    output word, with four inputs each: ordinary values with zeros, raw bit patterns, and the bit patterns with the top
+    output word and against the oracle on 16 sampled outputs, with four inputs each: ordinary values with zeros, raw bit patterns, and the bit patterns with the top
     exponent bit of every word cleared (tiny products: zero and subnormal results) or set (huge ones: overflow, infinities
     and NaNs).  MMASIM_PARITY_SEEDS sets the number of seeds (default 3; 240 ran clean)."""
     from paper_2511_10909_b200 import mmasim
@@ -127,3 +127,5 @@ def test_rows_on_more_seeds_and_magnitudes(seed):
             G = gu.run_gemm(key, x, force_generic=True)
             bad = np.argwhere(D != G)
             assert bad.size == 0, (key, kernel, (M, N, K), name, len(bad), bad[:4])
+            pairs = wl.sample_pairs(M, N, 16, seed=M * 1000 + N + seed)
+            gu.assert_samples_equal(D, gu.oracle_samples(key, x, pairs), pairs, f"{key} {kernel} {(M, N, K)} {name}")
