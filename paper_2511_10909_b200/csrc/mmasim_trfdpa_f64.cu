@@ -135,6 +135,8 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g,
             // nonzero product (lane 0) gets an exponent far below every real one: its sum stays 0 ----
             constexpr int EXPF = 0x7FF00000, HALF = 0x00080000, LOW0 = int(0x80000000u);
             double t0[TM][TN], t1[GTR ? TM : 1][GTR ? TN : 1];
+            constexpr bool KEEP_M0 = !GTR && L <= 8;       // short blocks keep the high word of the constant from the start of the block to the merge
+            int m0k[KEEP_M0 ? TM : 1][KEEP_M0 ? TN : 1];
             // (the two 16-bit lanes reach the exponent field by multiplications, which issue beside the integer pipe; what is
             // left below the field is masked away; the low word starts at 2^31: |T| < 2^30, so the sign correction of the
             // merge is a 32-bit addition that never carries)
@@ -144,7 +146,9 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g,
                     t0[r][c] = __hiloint2double((klo & EXPF) | HALF, LOW0);
                     t1[GTR ? r : 0][GTR ? c : 0] = __hiloint2double((khi & EXPF) | HALF, LOW0);
                 } else {
-                    t0[r][c] = __hiloint2double((max(klo, khi) & EXPF) | HALF, LOW0);
+                    const int mh = (max(klo, khi) & EXPF) | HALF;
+                    if (KEEP_M0) m0k[KEEP_M0 ? r : 0][KEEP_M0 ? c : 0] = mh;
+                    t0[r][c] = __hiloint2double(mh, LOW0);
                 }
             };
             // four terms per matrix instruction (mma.sync m8n8k4, FP64, rounding toward minus infinity) for the rows
@@ -202,7 +206,7 @@ __global__ void __launch_bounds__(NT, 1) trfdpa64_kernel(DevModel m, GemmArgs g,
                     Y = __dsub_rn(__dadd_rd(yo, __dadd_rd(ye, mm)), mm);
                 } else {
                     const double u0 = t0[r][c];
-                    m0hi = (__double2hiint(u0) & EXPF) | HALF;
+                    m0hi = KEEP_M0 ? m0k[KEEP_M0 ? r : 0][KEEP_M0 ? c : 0] : (__double2hiint(u0) & EXPF) | HALF;
                     Y = __dsub_rn(__hiloint2double(__double2hiint(u0), __double2loint(u0) + __popc(negm)), __hiloint2double(m0hi, LOW0));
                 }
                 double st = cs[r][c];
