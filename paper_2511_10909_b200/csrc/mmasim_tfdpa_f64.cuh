@@ -522,7 +522,8 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
     // carries into the high word
     constexpr bool NARROW = DS && L <= 8;
     constexpr int UNROLL_BLK = (L <= 4 || (L <= 16 && BASE == 0)) ? 2 : 1;  // two blocks per trip of the block loop
-    constexpr bool KEEP_MH = NARROW && L <= 4;
+    // where it measured faster: blocks of 4, and the long blocks of the add-max kinds (BF16, L = 16)
+    constexpr bool KEEP_MH = (NARROW && L <= 4) || (!NARROW && BASE == 0);
     // (a zero of either sign becomes the positive state)
     auto state_of = [](uint32_t w) {
         double d = 0.0;
@@ -771,15 +772,15 @@ __global__ void __launch_bounds__(NT, 1) tfdpa64_kernel(DevModel m, GemmArgs g, 
                 const int nneg = __popc((sa ^ sb_blk.sgn[pcol + c]) & live);
                 double v;
                 if (NARROW) {
-                    // the register never leaves its binade: its exponent field is the constant's (blocks of 4 keep the
-                    // high word of the start's constant instead of masking it out again)
+                    // the register never leaves its binade: its exponent field is the constant's (KEEP_MH: the high word of
+                    // the start's constant is kept instead of masked out of the register again)
                     const int hi = __double2hiint(acc[r][c]);
                     const double magic = __hiloint2double(KEEP_MH ? mhi[KEEP_MH ? r : 0][KEEP_MH ? c : 0] : (hi & 0x7FF00000) | 0x00080000, int(0x80000000u));
                     v = __dsub_rn(__hiloint2double(hi, __double2loint(acc[r][c]) + nneg), magic);
                 } else {
                     const long long bits = __double_as_longlong(acc[r][c]) + (long long)nneg;
                     const int hi = int(bits >> 32);
-                    const double magic = __hiloint2double((hi & 0x7FF00000) | 0x00080000, 0);
+                    const double magic = __hiloint2double(KEEP_MH ? mhi[KEEP_MH ? r : 0][KEEP_MH ? c : 0] : (hi & 0x7FF00000) | 0x00080000, 0);
                     v = __dsub_rn(__longlong_as_double(bits), magic);                 // S * q, exact; +0 when S = 0
                 }
                 return v;
